@@ -1,0 +1,494 @@
+/*
+ * HiFloat8 (HiF8) reference oracle -- TEST INFRASTRUCTURE, NOT PRODUCT CODE.
+ *
+ * A plain, slow, value-level CPU implementation of the HiF8 format and of the
+ * conversions defined in "Ascend HiFloat8 Format for Deep Learning"
+ * (arXiv 2409.16626).  Only the test-suite, the smoke check and the benchmark's
+ * CPU-baseline leg may call it.  It shares no code, table or constant with the
+ * CUDA library; the CUDA library never calls it.
+ *
+ * Everything is computed on real values held in `double` (all three source
+ * formats and every HiF8 value embed exactly in a double, and scaling by a
+ * power of two is exact), following the paper's definitions step by step:
+ *
+ *   byte -> value            Section 2.1: Table 1 (fields), Table 2 (dot prefix
+ *                            code), Table 3 (exponent ranges / mantissa width),
+ *                            Eq. 1 (normal), Eq. 2 (denormal), specials.
+ *   value -> byte, TA / TE   Section 3.1 "Rounding Half": nearest representable
+ *                            value, found by a linear scan of all 256 codes;
+ *                            ties away from zero (TA) or to the even kept
+ *                            significand (TE).
+ *   value -> byte, SR family Section 3.2 "Hybrid Rounding": threshold T versus
+ *                            discarded fraction F; SR14 / SR2 simplified forms;
+ *                            Eq. 3 hybrid switch on |E| < 4.
+ *   options                  Section 3: saturation on overflow, NaN to zero.
+ *   scaling                  Section 4.2 / 5.1: power-of-two per-tensor scale,
+ *                            amax, descale (Algorithm 1, "Scale & Cast" and
+ *                            "MatMul & Restore" steps).
+ *
+ * Readings taken where the paper is silent are marked "READING" below.
+ * Pin status: every function here is pinned by tests/test_oracle_pins.py
+ * against values the paper prints (Table 4 patterns, the abstract's counts,
+ * the TE/TA worked example, the 0.5 / 0.75 / 1 ulp error bounds, the 2^-20 tie
+ * probability, the SR expectation identity) and by closed forms.  The bit-level
+ * placement of F14 inside the discarded field (Fig. 2 of the paper is not
+ * available) is pinned only through the 1-ulp bound and unbiasedness.
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { O_F32 = 0, O_BF16 = 1, O_F16 = 2 };
+enum { O_TA = 0, O_HR = 1, O_SSR = 2, O_TE = 3, O_SR = 4 };
+enum { O_SATURATE = 1u, O_NAN_TO_ZERO = 2u };
+
+/* kind of a decoded byte */
+enum { K_ZERO = 0, K_FINITE = 1, K_INF = 2, K_NAN = 3 };
+
+typedef struct {
+    int kind;      /* K_* */
+    int sign;      /* 1 = negative */
+    int is_dml;    /* denormal equation used */
+    int D;         /* dot value 0..4 (NML only) */
+    int E;         /* exponent */
+    int w;         /* mantissa width */
+    int M;         /* mantissa field */
+    double value;  /* signed real value; for K_INF the Eq. 1 value +-1.5*2^15 */
+} hif8_fields;
+
+/* ------------------------------------------------------------------------- *
+ * Section 2.1: parse one byte into its four fields and its value.
+ * Bit order (READING, matches every pattern of Table 4): bit 7 = sign, the dot
+ * field starts at bit 6, the mantissa ends at bit 0.
+ * ------------------------------------------------------------------------- */
+static hif8_fields parse_code(unsigned b)
+{
+    hif8_fields f;
+    memset(&f, 0, sizeof f);
+    f.sign = (b >> 7) & 1;
+    int pos = 6; /* next unread bit */
+    int b6 = (b >> 6) & 1, b5 = (b >> 5) & 1, b4 = (b >> 4) & 1, b3 = (b >> 3) & 1;
+    int dml = 0, D = 0;
+    /* Table 2: 11 -> 4, 10 -> 3, 01 -> 2, 001 -> 1, 0001 -> 0, 0000 -> DML */
+    if (b6 == 1 && b5 == 1)      { D = 4; pos = 4; }
+    else if (b6 == 1 && b5 == 0) { D = 3; pos = 4; }
+    else if (b6 == 0 && b5 == 1) { D = 2; pos = 4; }
+    else if (b4 == 1)            { D = 1; pos = 3; }
+    else if (b3 == 1)            { D = 0; pos = 2; }
+    else                         { dml = 1; pos = 2; }
+
+    if (dml) {
+        /* Eq. 2: X = (-1)^S * 2^(M-23), M in [1,7]; M = 0 is zero (S=0) or NaN (S=1) */
+        int M = b & 7;
+        f.is_dml = 1; f.w = 3; f.M = M;
+        if (M == 0) {
+            f.kind = f.sign ? K_NAN : K_ZERO;
+            f.value = f.sign ? NAN : 0.0;
+            return f;
+        }
+        f.kind = K_FINITE;
+        f.E = M - 23;
+        f.value = ldexp(1.0, f.E) * (f.sign ? -1.0 : 1.0);
+        return f;
+    }
+    /* exponent field: D bits, Em = {Se, Mag[2:end]}, magnitude MSB implicit 1 */
+    int E = 0;
+    if (D > 0) {
+        int Se = (b >> pos) & 1; pos--;
+        int mag = 1; /* implicit leading magnitude bit */
+        for (int i = 1; i < D; i++) { mag = (mag << 1) | ((b >> pos) & 1); pos--; }
+        E = Se ? -mag : mag;
+    }
+    int w = pos + 1; /* remaining low bits are the mantissa */
+    int M = b & ((1 << w) - 1);
+    f.D = D; f.E = E; f.w = w; f.M = M;
+    /* Eq. 1: X = (-1)^S * 2^E * 1.M */
+    double mag = ldexp(1.0 + (double)M / (double)(1 << w), E);
+    f.value = f.sign ? -mag : mag;
+    /* the two patterns of largest magnitude 2^15 * 1.5 are the infinities */
+    f.kind = (E == 15 && M == 1) ? K_INF : K_FINITE;
+    return f;
+}
+
+void hif8o_parse(unsigned code, int* kind, int* sign, int* is_dml, int* D, int* E, int* w, int* M,
+                 double* value)
+{
+    hif8_fields f = parse_code(code & 0xFF);
+    *kind = f.kind; *sign = f.sign; *is_dml = f.is_dml; *D = f.D; *E = f.E; *w = f.w; *M = f.M;
+    *value = f.value;
+}
+
+/* value of a byte as an IEEE double: NaN, +-Inf, +0 or the finite value */
+double hif8o_value(unsigned code)
+{
+    hif8_fields f = parse_code(code & 0xFF);
+    if (f.kind == K_NAN) return NAN;
+    if (f.kind == K_INF) return f.sign ? -INFINITY : INFINITY;
+    return f.value;
+}
+
+/* ------------------------------------------------------------------------- *
+ * Source / destination formats (IEEE binary32, binary16, bfloat16) by formula.
+ * ------------------------------------------------------------------------- */
+static double src_to_double(const void* p, size_t i, int dtype, uint32_t* raw)
+{
+    if (dtype == O_F32) {
+        uint32_t u; memcpy(&u, (const char*)p + 4 * i, 4);
+        float f; memcpy(&f, &u, 4);
+        *raw = u;
+        return (double)f;
+    }
+    uint16_t h; memcpy(&h, (const char*)p + 2 * i, 2);
+    *raw = h;
+    if (dtype == O_BF16) {
+        uint32_t u = (uint32_t)h << 16; /* bfloat16 is the upper half of a binary32 */
+        float f; memcpy(&f, &u, 4);
+        return (double)f;
+    }
+    /* binary16: 1 sign, 5 exponent (bias 15), 10 fraction bits */
+    int s = (h >> 15) & 1, e = (h >> 10) & 31, m = h & 1023;
+    double v;
+    if (e == 31) v = m ? NAN : INFINITY;
+    else if (e == 0) v = ldexp((double)m, -24);
+    else v = ldexp(1.0 + (double)m / 1024.0, e - 15);
+    return s ? -v : v;
+}
+
+/* round a double to a binary interchange format with `ebits` exponent bits and
+ * `mbits` fraction bits, IEEE round-to-nearest-even, returning the encoding.
+ * NaN -> canonical positive quiet NaN (READING: the paper says nothing about
+ * payloads). */
+static uint32_t round_to_format(double v, int ebits, int mbits)
+{
+    uint32_t expmask = (1u << ebits) - 1u;
+    if (isnan(v)) return (expmask << mbits) | (1u << (mbits - 1));
+    uint32_t sign = signbit(v) ? 1u : 0u;
+    uint32_t sbit = sign << (ebits + mbits);
+    double a = fabs(v);
+    if (isinf(a)) return sbit | (expmask << mbits);
+    if (a == 0.0) return sbit;
+    int bias = (1 << (ebits - 1)) - 1;
+    int emin = 1 - bias, emax = bias;
+    int ex; (void)frexp(a, &ex);
+    int e = ex - 1;                 /* a in [2^e, 2^(e+1)) */
+    if (e < emin) e = emin;         /* subnormal spacing */
+    double q = ldexp(a, mbits - e); /* exact */
+    double r = nearbyint(q);        /* default rounding mode: ties to even */
+    double two_m = ldexp(1.0, mbits);
+    if (r >= 2.0 * two_m) { e += 1; r = two_m; }
+    if (e > emax) return sbit | (expmask << mbits);
+    if (r < two_m) return sbit | (uint32_t)r;                      /* subnormal or zero */
+    return sbit | ((uint32_t)(e + bias) << mbits) | (uint32_t)(r - two_m);
+}
+
+static void store_as(void* p, size_t i, int dtype, double v)
+{
+    if (dtype == O_F32) { uint32_t u = round_to_format(v, 8, 23); memcpy((char*)p + 4 * i, &u, 4); }
+    else if (dtype == O_BF16) { uint16_t h = (uint16_t)round_to_format(v, 8, 7); memcpy((char*)p + 2 * i, &h, 2); }
+    else { uint16_t h = (uint16_t)round_to_format(v, 5, 10); memcpy((char*)p + 2 * i, &h, 2); }
+}
+
+uint32_t hif8o_round_to_format(double v, int ebits, int mbits) { return round_to_format(v, ebits, mbits); }
+
+/* ------------------------------------------------------------------------- *
+ * Counter-based generator for standard SR: Philox4x32-10 (Salmon, Moraes, Dror,
+ * Shaw, "Parallel random numbers: as easy as 1, 2, 3", SC'11), written from the
+ * published round function and constants.  READING: element i uses counter
+ * (i/4 low, i/4 high, 0, 0), key (seed low, seed high), output word i mod 4.
+ * ------------------------------------------------------------------------- */
+static void philox4x32_10(uint32_t ctr[4], uint32_t k0, uint32_t k1)
+{
+    const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+    for (int r = 0; r < 10; r++) {
+        uint64_t p0 = (uint64_t)M0 * ctr[0], p1 = (uint64_t)M1 * ctr[2];
+        uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0;
+        uint32_t hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
+        uint32_t n0 = hi1 ^ ctr[1] ^ k0, n1 = lo1, n2 = hi0 ^ ctr[3] ^ k1, n3 = lo0;
+        ctr[0] = n0; ctr[1] = n1; ctr[2] = n2; ctr[3] = n3;
+        k0 += W0; k1 += W1;
+    }
+}
+
+uint32_t hif8o_sr_word(uint64_t seed, uint64_t idx)
+{
+    uint64_t blk = idx >> 2;
+    uint32_t c[4] = { (uint32_t)blk, (uint32_t)(blk >> 32), 0u, 0u };
+    philox4x32_10(c, (uint32_t)seed, (uint32_t)(seed >> 32));
+    return c[idx & 3];
+}
+
+void hif8o_philox4x32_10(const uint32_t ctr_in[4], const uint32_t key[2], uint32_t out[4])
+{
+    uint32_t c[4] = { ctr_in[0], ctr_in[1], ctr_in[2], ctr_in[3] };
+    philox4x32_10(c, key[0], key[1]);
+    memcpy(out, c, sizeof c);
+}
+
+/* ------------------------------------------------------------------------- *
+ * Encoding of one real value.
+ * ------------------------------------------------------------------------- */
+#define INF_CAND 49152.0 /* 1.5 * 2^15: the Eq. 1 value that the Inf patterns replace */
+
+/* Nearest-of-256 by a literal scan (Section 3.1).  The Inf patterns take part
+ * with their Eq. 1 value +-1.5*2^15, i.e. rounding happens first and a result
+ * of that magnitude is infinity (READING).  Exact tie: TA -> larger magnitude;
+ * TE -> the neighbour whose integer significand K = value/ulp is even, where
+ * ulp is the spacing of the two neighbours (READING for 0-bit binades and below
+ * 2^-22: K counts the implicit one, K = 0 for the value zero). */
+static unsigned nearest_scan(double y, int te)
+{
+    /* at or beyond the largest candidate nothing else can be nearer (this also keeps every
+     * difference below exactly representable) */
+    if (fabs(y) >= INF_CAND) return signbit(y) ? 0xEFu : 0x6Fu;
+    unsigned best = 0; double bestd = INFINITY, bestv = 0.0;
+    for (unsigned c = 0; c < 256; c++) {
+        hif8_fields f = parse_code(c);
+        if (f.kind == K_NAN) continue;
+        double v = f.value;            /* K_INF carries +-1.5*2^15 */
+        double d = fabs(y - v);
+        if (d < bestd) { best = c; bestd = d; bestv = v; }
+        else if (d == bestd) {
+            /* two candidates at the same distance: they bracket y */
+            double lo = fabs(v) < fabs(bestv) ? v : bestv, hi = fabs(v) < fabs(bestv) ? bestv : v;
+            int take_hi;
+            if (!te) take_hi = 1;
+            else {
+                double ulp = fabs(hi) - fabs(lo);
+                double Klo = fabs(lo) / ulp;
+                take_hi = (fmod(Klo, 2.0) != 0.0); /* lo odd -> hi is even */
+            }
+            double pick = take_hi ? hi : lo;
+            if (pick == v) { best = c; bestv = v; }
+        }
+    }
+    return best;
+}
+
+/* positive magnitudes in increasing order: 0, the finite positive values, then
+ * the Inf candidate; returns their count and the code of each */
+static int build_sorted_magnitudes(double* mags, unsigned* codes)
+{
+    int n = 0;
+    for (unsigned c = 0; c < 128; c++) {
+        hif8_fields f = parse_code(c);
+        if (f.kind == K_NAN) continue;
+        mags[n] = f.value; codes[n] = c; n++;
+    }
+    for (int i = 1; i < n; i++) { /* insertion sort */
+        double m = mags[i]; unsigned c = codes[i]; int j = i - 1;
+        while (j >= 0 && mags[j] > m) { mags[j + 1] = mags[j]; codes[j + 1] = codes[j]; j--; }
+        mags[j + 1] = m; codes[j + 1] = c;
+    }
+    return n;
+}
+
+/* the table above, built once when the library is loaded */
+static double g_mags[130];
+static unsigned g_codes[130];
+static int g_nmags;
+__attribute__((constructor)) static void init_tables(void) { g_nmags = build_sorted_magnitudes(g_mags, g_codes); }
+
+/* The threshold family (Section 3.2).  a = |y| finite.  L <= a < U are table
+ * neighbours (L may be 0, U may be the Inf candidate), ulp = U - L,
+ * F = (a - L)/ulp in [0,1).  With an N-bit threshold T_N and F_N = floor(F*2^N),
+ * one is added to the kept bits iff F_N != 0 and F_N >= T_N.  (READING: the
+ * F_N != 0 guard keeps representable inputs fixed when T_N = 0.) */
+static unsigned threshold_round(double a, int N, uint32_t T)
+{
+    const double* mags = g_mags; const unsigned* codes = g_codes;
+    int n = g_nmags;
+    if (a >= mags[n - 1]) return codes[n - 1];
+    int i = 0;
+    while (i + 1 < n && mags[i + 1] <= a) i++;
+    double L = mags[i], U = mags[i + 1];
+    double F = (a - L) / (U - L);
+    double FN = floor(ldexp(F, N));
+    int up = (FN != 0.0) && (FN >= (double)T);
+    return up ? codes[i + 1] : codes[i];
+}
+
+/* same nearest rule as nearest_scan but through the neighbour pair; used only
+ * as the quick variant for very large sweeps and cross-checked by the tests */
+static unsigned nearest_pair(double y, int te)
+{
+    const double* mags = g_mags; const unsigned* codes = g_codes;
+    int n = g_nmags;
+    double a = fabs(y);
+    unsigned sgn = signbit(y) ? 0x80u : 0u, c;
+    if (a >= mags[n - 1]) c = codes[n - 1];
+    else {
+        int lo = 0, hi = n - 1; /* mags[lo] <= a < mags[hi] */
+        while (hi - lo > 1) { int mid = (lo + hi) / 2; if (mags[mid] <= a) lo = mid; else hi = mid; }
+        double L = mags[lo], U = mags[hi], dl = a - L, du = U - a;
+        if (dl < du) c = codes[lo];
+        else if (du < dl) c = codes[hi];
+        else if (!te) c = codes[hi];
+        else c = (fmod(L / (U - L), 2.0) != 0.0) ? codes[hi] : codes[lo];
+    }
+    return c == 0 ? 0u : (c | sgn);
+}
+
+static unsigned encode_value(double x, uint32_t raw, int dtype, int scale_exp, int rnd,
+                             unsigned flags, uint64_t seed, uint64_t idx, int quick)
+{
+    if (isnan(x)) return (flags & O_NAN_TO_ZERO) ? 0x00u : 0x80u;
+    double y = ldexp(x, scale_exp); /* exact: "Scale" step, power of two */
+    unsigned sgn = signbit(y) ? 0x80u : 0u;
+    double a = fabs(y);
+    unsigned code;
+    int mode = rnd;
+    if (isinf(a)) code = 0x6Fu | sgn;
+    else {
+        if (mode == O_HR) {
+            /* Eq. 3: TA if |E| < 4, simplified SR otherwise; E = exponent of the
+             * value presented to the converter (READING: after scaling) */
+            if (a == 0.0) mode = O_TA;
+            else { int ex; (void)frexp(a, &ex); int E = ex - 1; mode = (abs(E) < 4) ? O_TA : O_SSR; }
+        }
+        if (mode == O_TA || mode == O_TE) {
+            code = quick ? nearest_pair(y, mode == O_TE) : nearest_scan(y, mode == O_TE);
+        } else {
+            int N; uint32_t T;
+            if (mode == O_SSR) {
+                if (dtype == O_F32) { N = 14; T = raw & 0x3FFFu; }       /* SR14: 14 LSBs of the source */
+                else { N = 2; T = 2u * (raw & 1u) + 1u; }                /* SR2: {source LSB, fixed 1} */
+            } else {
+                N = (dtype == O_F32) ? 24 : 16;                         /* READING: threshold width */
+                T = hif8o_sr_word(seed, idx) >> (32 - N);
+            }
+            code = threshold_round(a, N, T);
+            if (code != 0) code |= sgn;
+        }
+    }
+    if ((code & 0x7F) == 0x6F && (flags & O_SATURATE)) code = (code & 0x80u) | 0x6Eu;
+    if ((code & 0x7F) == 0) code = 0; /* a zero result has one pattern; 0x80 is NaN */
+    return code;
+}
+
+/* ------------------------------------------------------------------------- *
+ * Array entry points
+ * ------------------------------------------------------------------------- */
+int hif8o_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+void hif8o_encode(const void* src, int dtype, uint8_t* dst, size_t n, int scale_exp, int rnd,
+                  unsigned flags, uint64_t seed, int quick)
+{
+#pragma omp parallel for schedule(static)
+    for (long long i = 0; i < (long long)n; i++) {
+        uint32_t raw; double x = src_to_double(src, (size_t)i, dtype, &raw);
+        dst[i] = (uint8_t)encode_value(x, raw, dtype, scale_exp, rnd, flags, seed, (uint64_t)i, quick);
+    }
+}
+
+/* encode the FP32 values whose encodings are first, first+1, ... (exhaustive sweeps) */
+void hif8o_encode_f32_range(uint32_t first, size_t n, uint8_t* dst, int scale_exp, int rnd,
+                            unsigned flags, uint64_t seed, int quick)
+{
+#pragma omp parallel for schedule(static)
+    for (long long i = 0; i < (long long)n; i++) {
+        uint32_t u = first + (uint32_t)i; float f; memcpy(&f, &u, 4);
+        dst[i] = (uint8_t)encode_value((double)f, u, O_F32, scale_exp, rnd, flags, seed, (uint64_t)i, quick);
+    }
+}
+
+/* dst = value(src) * 2^-scale_exp rounded (RNE) to the destination format */
+void hif8o_decode(const uint8_t* src, void* dst, int dtype, size_t n, int scale_exp)
+{
+#pragma omp parallel for schedule(static)
+    for (long long i = 0; i < (long long)n; i++) {
+        double v = hif8o_value(src[i]);
+        store_as(dst, (size_t)i, dtype, ldexp(v, -scale_exp));
+    }
+}
+
+/* amax over the finite elements and the power-of-two scale that brings it into
+ * [2^target_exp, 2^(target_exp+1)).  READING of "update the scale factor by a
+ * certain algorithm": scale_exp = target_exp - floor(log2 amax), clamped to
+ * [-126,126]; no finite non-zero element -> 0.  NaN / Inf do not take part. */
+void hif8o_amax_scale(const void* src, int dtype, size_t n, int target_exp, float* amax_out,
+                      int* scale_exp_out)
+{
+    double amax = 0.0;
+#pragma omp parallel for reduction(max : amax) schedule(static)
+    for (long long i = 0; i < (long long)n; i++) {
+        uint32_t raw; double x = fabs(src_to_double(src, (size_t)i, dtype, &raw));
+        if (isfinite(x) && x > amax) amax = x;
+    }
+    int se = 0;
+    if (amax > 0.0) {
+        int ex; (void)frexp(amax, &ex);
+        se = target_exp - (ex - 1);
+        if (se > 126) se = 126;
+        if (se < -126) se = -126;
+    }
+    *amax_out = (float)amax; /* exact: amax is a source value */
+    *scale_exp_out = se;
+}
+
+/* quantize-dequantize in the source format ("simulated HiF8", Section 4) */
+void hif8o_fake_quant(const void* src, void* dst, int dtype, size_t n, int scale_exp, int rnd,
+                      unsigned flags, uint64_t seed, int quick)
+{
+#pragma omp parallel for schedule(static)
+    for (long long i = 0; i < (long long)n; i++) {
+        uint32_t raw; double x = src_to_double(src, (size_t)i, dtype, &raw);
+        unsigned c = encode_value(x, raw, dtype, scale_exp, rnd, flags, seed, (uint64_t)i, quick);
+        store_as(dst, (size_t)i, dtype, ldexp(hif8o_value(c), -scale_exp));
+    }
+}
+
+/* Algorithm 1, "MatMul & Restore": C*[m,n] = 2^-(sa+sw) * sum_k dec(A[m,k]) dec(W[k,n]) in
+ * double, and S[m,n] = 2^-(sa+sw) * sum_k |dec(A) dec(W)|, for `count` listed entries.
+ * A is [M,K] row-major with leading dimension lda; W is [K,N] (ldw) or, when w_is_nk, [N,K]. */
+void hif8o_gemm_entries(const uint8_t* Aq, long long lda, const uint8_t* Wq, long long ldw, int w_is_nk,
+                        int K, int sa, int sw, const long long* rows, const long long* cols,
+                        size_t count, double* Cstar, double* S)
+{
+    double tab[256];
+    for (unsigned c = 0; c < 256; c++) tab[c] = hif8o_value(c);
+#pragma omp parallel for schedule(dynamic, 64)
+    for (long long t = 0; t < (long long)count; t++) {
+        long long m = rows[t], n = cols[t];
+        double acc = 0.0, sab = 0.0;
+        for (int k = 0; k < K; k++) {
+            double a = tab[Aq[m * lda + k]];
+            double w = w_is_nk ? tab[Wq[n * ldw + k]] : tab[Wq[(long long)k * ldw + n]];
+            double p = a * w;
+            acc += p; sab += fabs(p);
+        }
+        Cstar[t] = ldexp(acc, -(sa + sw));
+        S[t] = ldexp(sab, -(sa + sw));
+    }
+}
+
+void hif8o_gemm_full(const uint8_t* Aq, long long lda, const uint8_t* Wq, long long ldw, int w_is_nk,
+                     int M, int N, int K, int sa, int sw, double* Cstar, double* S)
+{
+    double tab[256];
+    for (unsigned c = 0; c < 256; c++) tab[c] = hif8o_value(c);
+#pragma omp parallel for schedule(static)
+    for (long long m = 0; m < M; m++)
+        for (long long n = 0; n < N; n++) {
+            double acc = 0.0, sab = 0.0;
+            for (int k = 0; k < K; k++) {
+                double a = tab[Aq[m * lda + k]];
+                double w = w_is_nk ? tab[Wq[n * ldw + k]] : tab[Wq[(long long)k * ldw + n]];
+                double p = a * w;
+                acc += p; sab += fabs(p);
+            }
+            Cstar[m * N + n] = ldexp(acc, -(sa + sw));
+            S[m * N + n] = ldexp(sab, -(sa + sw));
+        }
+}
