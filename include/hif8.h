@@ -1,0 +1,151 @@
+/*
+ * hif8.h -- C ABI of the B200 (sm_100a) HiFloat8 conversion library.
+ *
+ * HiFloat8 (HiF8) is the 8-bit tapered floating-point format of "Ascend HiFloat8 Format for Deep
+ * Learning" (arXiv 2409.16626), Section 2.1: one byte = sign | dot field (prefix code, Table 2) |
+ * sign-magnitude exponent with implicit leading 1 (Table 3) | 3/2/1-bit mantissa; normal values follow
+ * Eq. 1, the denormal extension follows Eq. 2; 0x00 is the single zero, 0x80 is NaN, 0x6F / 0xEF are
+ * +-Inf (Table 4).
+ *
+ * Conventions for every entry point
+ *   - All data pointers are DEVICE pointers owned by the caller (any CUDA allocation); the library
+ *     never allocates, frees or copies to the host, and never synchronises.  All work is enqueued on
+ *     `stream` (a cudaStream_t; NULL = the legacy default stream) of the current device.
+ *   - Tensors are contiguous, element count `n`.  Any byte alignment is accepted; 16-byte aligned
+ *     pointers take the vectorised path, others a slower scalar kernel with identical results.
+ *   - Return value: HIF8_OK or an error code (see hif8_status_string).  Argument errors are detected
+ *     before anything is launched and leave all outputs untouched.  NaN / Inf inputs are data.
+ *   - `scale_exp` is the exponent E of a power-of-two scale 2^E (Section 4.2: scale factors are
+ *     integer powers of two, so scaling only adds to the exponent), limited to [-126, 126].
+ *   - The library needs a CUDA device of compute capability 10.0 and fails with HIF8_ERR_CUDA elsewhere.
+ */
+#ifndef HIF8_H
+#define HIF8_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st* hif8_stream_t; /* same type as cudaStream_t */
+
+/* element formats of the high-precision side (Section 3: FP32, FP16 and BF16 sources) */
+typedef enum { HIF8_F32 = 0, HIF8_BF16 = 1, HIF8_F16 = 2 } hif8_dtype_t;
+
+/* rounding methods of Section 3 */
+typedef enum {
+    HIF8_RND_TA = 0,  /* Section 3.1: round half away from zero (the default everywhere)               */
+    HIF8_RND_HR = 1,  /* Eq. 3: hybrid -- TA if |E| < 4, simplified stochastic rounding if |E| >= 4    */
+    HIF8_RND_SSR = 2, /* Section 3.2 simplified SR for every E: SR14 (FP32 source), SR2 (FP16 / BF16)  */
+    HIF8_RND_TE = 3,  /* Section 3.1: round half to even                                               */
+    HIF8_RND_SR = 4   /* Section 3.2 standard SR; thresholds from Philox4x32-10 keyed by `seed`         */
+} hif8_round_t;
+
+/* the two options of Section 3 */
+enum {
+    HIF8_FLAG_SATURATE = 1u,   /* overflow (and a source +-Inf) gives +-2^15 instead of +-Inf */
+    HIF8_FLAG_NAN_TO_ZERO = 2u /* a source NaN gives 0x00 instead of 0x80                     */
+};
+
+enum {
+    HIF8_OK = 0,
+    HIF8_ERR_NULL = 1,        /* a required pointer is NULL                         */
+    HIF8_ERR_DTYPE = 2,       /* unknown element format                             */
+    HIF8_ERR_ROUND = 3,       /* unknown rounding method                            */
+    HIF8_ERR_FLAGS = 4,       /* unknown option bits                                */
+    HIF8_ERR_SCALE_RANGE = 5, /* scale or target exponent outside [-126, 126]       */
+    HIF8_ERR_SHAPE = 6,       /* negative or unsupported extent / leading dimension */
+    HIF8_ERR_ALIGN = 7,       /* GEMM operand not 16-byte aligned                   */
+    HIF8_ERR_WORKSPACE = 8,   /* workspace missing or too small                     */
+    HIF8_ERR_CUDA = 9,        /* a CUDA call failed (launch error, wrong device)    */
+    HIF8_ERR_DEVICE_TIMEOUT = 10 /* a bounded device-side wait gave up             */
+};
+
+/* which call a workspace size is asked for */
+enum { HIF8_WS_AMAX_SCALE_ENCODE = 0, HIF8_WS_FAKE_QUANT = 1, HIF8_WS_GEMM = 2 };
+
+/*
+ * High-precision tensor -> HiF8 bytes (Section 3, "conversion from high-precision formats to HiF8").
+ *   dst[i] = To_HiF8_<rnd>( src[i] * 2^scale_exp )
+ * The scaled value is rounded as if 1.5*2^15 were representable; a result of that magnitude or more is
+ * +-Inf (or +-2^15 with HIF8_FLAG_SATURATE).  Magnitudes that round to zero give 0x00 for either sign.
+ * src: n elements of `src_dtype`; dst: n bytes; they must not overlap.  `seed` is used by HIF8_RND_SR only:
+ * element i takes word (i mod 4) of Philox4x32-10 with counter (i/4, 0, 0) and key `seed`; its top 24 bits
+ * (FP32 source) or 16 bits (16-bit sources) are the threshold T of Section 3.2.
+ */
+int hif8_encode(const void* src, int src_dtype, uint8_t* dst, size_t n, int scale_exp, int rnd,
+                unsigned flags, uint64_t seed, hif8_stream_t stream);
+
+/*
+ * HiF8 bytes -> high-precision tensor (Eq. 1, Eq. 2, Table 4 specials), with the descale of
+ * Algorithm 1 ("Restore"):   dst[i] = value(src[i]) * 2^(-scale_exp)
+ * rounded to nearest-even into `dst_dtype` when not representable (only possible at the far ends of the
+ * scale range, or for FP16 destinations).  0x80 gives the canonical quiet NaN, 0x6F / 0xEF give +-Inf.
+ * src: n bytes; dst: n elements; no overlap.
+ */
+int hif8_decode(const uint8_t* src, void* dst, int dst_dtype, size_t n, int scale_exp,
+                hif8_stream_t stream);
+
+/*
+ * Per-tensor scaled conversion (Section 5.1 "Per-Tensor Scaling"; Algorithm 1 "Scale & Cast").
+ *   d_scale_exp_in == NULL  (just-in-time):  amax = max |src[i]| over finite elements;
+ *        scale_exp = clamp(target_exp - floor(log2 amax), -126, 126)  (0 if amax is 0), so that
+ *        amax * 2^scale_exp lies in [2^target_exp, 2^(target_exp+1)); then dst = To_HiF8(src * 2^scale_exp).
+ *        Two kernels, the scale never leaves the device.
+ *   d_scale_exp_in != NULL  (delayed scaling, the paper's "Amax every 10 iterations"): the scale exponent
+ *        is read from that device int; amax of this tensor is still produced for the next update.  One pass.
+ * Outputs (device scalars, each may be NULL): d_amax_out (float, exact), d_scale_exp_out (int, the exponent
+ * used), d_scale_out (float 2^scale_exp).  workspace: hif8_workspace_bytes(HIF8_WS_AMAX_SCALE_ENCODE, n)
+ * bytes of device memory, 256-byte aligned, contents irrelevant on entry and undefined on return.
+ * target_exp in [-22, 15]; 14 keeps amax just below the largest finite value 2^15.
+ */
+int hif8_amax_scale_encode(const void* src, int src_dtype, uint8_t* dst, size_t n, int target_exp, int rnd,
+                           unsigned flags, uint64_t seed, const int* d_scale_exp_in, float* d_amax_out,
+                           int* d_scale_exp_out, float* d_scale_out, void* workspace,
+                           size_t workspace_bytes, hif8_stream_t stream);
+
+/*
+ * Quantize-dequantize in the source format ("simulated HiF8", Section 4: values are converted to only those
+ * representable in HiF8):   dst[i] = value( To_HiF8_<rnd>(src[i] * 2^e) ) * 2^(-e)   in `dtype`.
+ *   use_amax == 0: e = scale_or_target_exp.  No workspace needed (may be NULL).
+ *   use_amax == 1: e derived from the tensor's amax with target exponent scale_or_target_exp, as in
+ *                  hif8_amax_scale_encode (two kernels); workspace as for HIF8_WS_FAKE_QUANT.
+ * dst may be the same pointer as src (in place); partial overlap is not allowed.
+ * d_amax_out / d_scale_exp_out: optional device scalars as above.
+ */
+int hif8_fake_quant(const void* src, void* dst, int dtype, size_t n, int use_amax, int scale_or_target_exp,
+                    int rnd, unsigned flags, uint64_t seed, float* d_amax_out, int* d_scale_exp_out,
+                    void* workspace, size_t workspace_bytes, hif8_stream_t stream);
+
+/*
+ * GEMM with HiF8 operands decoded in-kernel (Algorithm 1, "MatMul & Restore"; Section 4.1: only the GEMM
+ * inputs are HiF8):   C[m,n] = 2^-(sa+sw) * sum_k value(Aq[m,k]) * value(Wq[k,n])
+ * Decoded values are exact in BF16; products are accumulated in FP32 on the tensor cores.
+ *   Aq: [M,K] row-major bytes, leading dimension lda.  Wq: [K,N] (w_is_nk = 0) or [N,K] (w_is_nk = 1)
+ *   row-major bytes, leading dimension ldw.  C: [M,N] row-major, `c_dtype` HIF8_BF16 or HIF8_F32, ldc.
+ *   d_scale_exp_a / d_scale_exp_w: device ints sa, sw (NULL = 0).
+ * Pointers and leading dimensions must be multiples of 16 bytes (HIF8_ERR_ALIGN); K must be a multiple of
+ * 16.  workspace: hif8_workspace_bytes(HIF8_WS_GEMM, 0) bytes (may be 0 -> NULL allowed).
+ */
+int hif8_gemm(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int64_t ldw, int w_is_nk, void* C,
+              int64_t ldc, int c_dtype, int M, int N, int K, const int* d_scale_exp_a,
+              const int* d_scale_exp_w, void* workspace, size_t workspace_bytes, hif8_stream_t stream);
+
+/* bytes of device workspace a call needs (which = HIF8_WS_*; n = element count, ignored for GEMM) */
+size_t hif8_workspace_bytes(int which, size_t n);
+
+/* static, NUL-terminated description of a status code */
+const char* hif8_status_string(int status);
+
+/*
+ * Number of kernels the library has launched from this process since it was loaded (all entry points,
+ * all streams).  Host-side counter for tests and benchmarks.
+ */
+uint64_t hif8_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HIF8_H */

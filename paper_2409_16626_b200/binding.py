@@ -1,0 +1,109 @@
+"""ctypes binding of libhif8.so.  Argument marshalling only: every step runs in the CUDA kernels.
+
+Functions carry the C names and argument order of include/hif8.h.  Tensors are torch CUDA tensors (used for
+device memory and streams only); pointers may also be given as plain ints.  A missing or unloadable library
+is an error: there is no fallback path.
+"""
+import ctypes as C
+import os
+
+import torch
+
+F32, BF16, F16 = 0, 1, 2
+RND_TA, RND_HR, RND_SSR, RND_TE, RND_SR = 0, 1, 2, 3, 4
+FLAG_SATURATE, FLAG_NAN_TO_ZERO = 1, 2
+WS_AMAX_SCALE_ENCODE, WS_FAKE_QUANT, WS_GEMM = 0, 1, 2
+OK = 0
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libhif8.so")
+EXPORTS = ["hif8_encode", "hif8_decode", "hif8_amax_scale_encode", "hif8_fake_quant", "hif8_gemm",
+           "hif8_workspace_bytes", "hif8_status_string", "hif8_launch_count"]
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2409_16626_b200.build` (needs nvcc)")
+lib = C.CDLL(LIB_PATH)
+
+_vp, _sz, _i, _u, _u64, _i64 = C.c_void_p, C.c_size_t, C.c_int, C.c_uint, C.c_uint64, C.c_int64
+lib.hif8_encode.argtypes = [_vp, _i, _vp, _sz, _i, _i, _u, _u64, _vp]
+lib.hif8_decode.argtypes = [_vp, _vp, _i, _sz, _i, _vp]
+lib.hif8_amax_scale_encode.argtypes = [_vp, _i, _vp, _sz, _i, _i, _u, _u64, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+lib.hif8_fake_quant.argtypes = [_vp, _vp, _i, _sz, _i, _i, _i, _u, _u64, _vp, _vp, _vp, _sz, _vp]
+lib.hif8_gemm.argtypes = [_vp, _i64, _vp, _i64, _i, _vp, _i64, _i, _i, _i, _i, _vp, _vp, _vp, _sz, _vp]
+lib.hif8_workspace_bytes.argtypes = [_i, _sz]
+lib.hif8_workspace_bytes.restype = _sz
+lib.hif8_status_string.argtypes = [_i]
+lib.hif8_status_string.restype = C.c_char_p
+lib.hif8_launch_count.restype = _u64
+for _n in ("hif8_encode", "hif8_decode", "hif8_amax_scale_encode", "hif8_fake_quant", "hif8_gemm"):
+    getattr(lib, _n).restype = _i
+
+
+class Hif8Error(RuntimeError):
+    def __init__(self, status):
+        self.status = status
+        super().__init__(f"hif8 status {status}: {hif8_status_string(status)}")
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    return t.data_ptr()
+
+
+def _stream(stream):
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def _check(rc, check):
+    if check and rc != OK:
+        raise Hif8Error(rc)
+    return rc
+
+
+def hif8_status_string(status):
+    return lib.hif8_status_string(int(status)).decode()
+
+
+def hif8_workspace_bytes(which, n=0):
+    return int(lib.hif8_workspace_bytes(which, n))
+
+
+def hif8_launch_count():
+    return int(lib.hif8_launch_count())
+
+
+def hif8_encode(src, src_dtype, dst, n, scale_exp=0, rnd=RND_TA, flags=0, seed=0, stream=None, check=True):
+    return _check(lib.hif8_encode(_ptr(src), src_dtype, _ptr(dst), n, scale_exp, rnd, flags, seed, _stream(stream)), check)
+
+
+def hif8_decode(src, dst, dst_dtype, n, scale_exp=0, stream=None, check=True):
+    return _check(lib.hif8_decode(_ptr(src), _ptr(dst), dst_dtype, n, scale_exp, _stream(stream)), check)
+
+
+def hif8_amax_scale_encode(src, src_dtype, dst, n, target_exp=14, rnd=RND_TA, flags=0, seed=0, d_scale_exp_in=None,
+                           d_amax_out=None, d_scale_exp_out=None, d_scale_out=None, workspace=None,
+                           workspace_bytes=0, stream=None, check=True):
+    return _check(lib.hif8_amax_scale_encode(_ptr(src), src_dtype, _ptr(dst), n, target_exp, rnd, flags, seed,
+                                             _ptr(d_scale_exp_in), _ptr(d_amax_out), _ptr(d_scale_exp_out),
+                                             _ptr(d_scale_out), _ptr(workspace), workspace_bytes, _stream(stream)), check)
+
+
+def hif8_fake_quant(src, dst, dtype, n, use_amax=0, scale_or_target_exp=0, rnd=RND_TA, flags=0, seed=0,
+                    d_amax_out=None, d_scale_exp_out=None, workspace=None, workspace_bytes=0, stream=None, check=True):
+    return _check(lib.hif8_fake_quant(_ptr(src), _ptr(dst), dtype, n, use_amax, scale_or_target_exp, rnd, flags, seed,
+                                      _ptr(d_amax_out), _ptr(d_scale_exp_out), _ptr(workspace), workspace_bytes,
+                                      _stream(stream)), check)
+
+
+def hif8_gemm(Aq, lda, Wq, ldw, w_is_nk, Cmat, ldc, c_dtype, M, N, K, d_scale_exp_a=None, d_scale_exp_w=None,
+              workspace=None, workspace_bytes=0, stream=None, check=True):
+    return _check(lib.hif8_gemm(_ptr(Aq), lda, _ptr(Wq), ldw, w_is_nk, _ptr(Cmat), ldc, c_dtype, M, N, K,
+                                _ptr(d_scale_exp_a), _ptr(d_scale_exp_w), _ptr(workspace), workspace_bytes,
+                                _stream(stream)), check)

@@ -1,0 +1,747 @@
+// HiF8 streaming conversion kernels for sm_100a: encode, decode, amax, fake-quant.
+//
+// Format: "Ascend HiFloat8 Format for Deep Learning" (arXiv 2409.16626), Section 2.1 (Tables 1-3, Eq. 1-2);
+// rounding: Section 3 (TA / TE, standard and simplified stochastic rounding, Eq. 3 hybrid); scaling:
+// Section 4.2 / 5.1 (power-of-two per-tensor scale, amax).
+//
+// Design notes
+//  * Every element is first scaled with one FP32 multiply by 2^scale_exp.  The product is exact whenever it
+//    matters (a normal result keeps all 24 significand bits; results below 2^-126 are far below the
+//    smallest HiF8 value 2^-22), FP32 subnormal sources are normalised by the hardware, +-Inf stays +-Inf and
+//    every NaN becomes one canonical pattern.
+//  * Round-half-away (TA) of the scaled binary32 pattern depends only on its sign, exponent and top four
+//    mantissa bits (the widest HiF8 mantissa is 3 bits plus the rounding bit), so the whole conversion is one
+//    lookup in an 8 KiB table indexed by the top 13 bits; the table is built at compile time from the field
+//    definitions and staged in shared memory.
+//  * The other rounding methods add a method-specific increment below the kept bits (so that the carry does
+//    the rounding, including across binade and mantissa-width boundaries), clear the discarded bits and use the
+//    same table to pack the fields.
+//  * Memory access: one 16-byte load per thread and instruction, consecutive lanes on consecutive 16-byte
+//    groups, four independent groups in flight per thread; grids are a multiple of the SM count.
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdint>
+
+#include "hif8.h"
+
+namespace hif8 {
+
+std::atomic<uint64_t> g_launches{0};
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kUnroll = 4;
+constexpr int kBlocksPerSM = 8;
+constexpr uint32_t kShSlow = 255;  // marks binades below 2^-22 in the shift table
+
+// ------------------------------------------------------------------------------------------------
+// Field packing (Table 1: sign | dot | exponent | mantissa; Table 2 prefix code; Table 3 exponent ranges)
+// ------------------------------------------------------------------------------------------------
+__host__ __device__ constexpr int mant_width(int E)
+{
+    int a = E < 0 ? -E : E;
+    return (E <= -16) ? 0 : (a <= 3 ? 3 : (a <= 7 ? 2 : 1));
+}
+
+// magnitude byte (bit 7 clear) of 2^E * 1.M, E in [-22, 15], M already `mant_width(E)` bits wide
+__host__ __device__ constexpr uint32_t pack_magnitude(int E, uint32_t M)
+{
+    if (E <= -16) return (uint32_t)(E + 23);  // Eq. 2: denormal, mantissa field = E + 23
+    uint32_t a = (uint32_t)(E < 0 ? -E : E), se = E < 0 ? 1u : 0u;
+    if (a == 0) return 0x08u | M;                                     // dot 0001
+    if (a == 1) return 0x10u | (se << 3) | M;                         // dot 001, Em = {Se}
+    if (a <= 3) return 0x20u | (se << 4) | ((a & 1u) << 3) | M;       // dot 01,  Em = {Se, Mag[2]}
+    if (a <= 7) return 0x40u | (se << 4) | ((a & 3u) << 2) | M;       // dot 10,  Em = {Se, Mag[2:3]}
+    return 0x60u | (se << 4) | ((a & 7u) << 1) | M;                   // dot 11,  Em = {Se, Mag[2:4]}
+}
+
+// Round-half-away result for the binary32 patterns whose top 13 bits are `idx`
+// (1 sign, 8 exponent, 4 mantissa bits).
+__host__ __device__ constexpr uint8_t ta_entry(uint32_t idx)
+{
+    uint32_t sign = (idx >> 12) << 7;
+    int e = (int)((idx >> 4) & 0xFF);
+    uint32_t m4 = idx & 0xF;
+    if (e == 255) return m4 ? (uint8_t)0x80 : (uint8_t)(sign | 0x6F);   // NaN (canonical has m4 = 15) / Inf
+    int E = e - 127;
+    if (E >= 16) return (uint8_t)(sign | 0x6F);
+    if (E <= -24) return 0;                       // below half of 2^-22: the single zero pattern
+    if (E == -23) return (uint8_t)(sign | 0x01);  // [2^-23, 2^-22) rounds up to 2^-22 (tie away)
+    int w = mant_width(E);
+    uint32_t M = m4 >> (4 - w);
+    uint32_t rbit = (m4 >> (3 - w)) & 1u;         // MSB of the discarded bits
+    M += rbit;
+    if (M == (1u << w)) { M = 0; E += 1; }        // carry into the exponent; the mantissa is then zero
+    if (E >= 16) return (uint8_t)(sign | 0x6F);
+    return (uint8_t)(sign | pack_magnitude(E, M));  // E = 15, M = 1 is the Inf pattern by construction
+}
+
+struct TaTable { uint8_t v[8192]; };
+constexpr TaTable make_ta_table()
+{
+    TaTable t{};
+    for (uint32_t i = 0; i < 8192; i++) t.v[i] = ta_entry(i);
+    return t;
+}
+__device__ const TaTable g_ta_table = make_ta_table();
+
+// value of one byte as binary32 bits (Eq. 1 / Eq. 2 / specials)
+__device__ __forceinline__ uint32_t decode_bits_f32(uint32_t c)
+{
+    uint32_t sign = (c & 0x80u) << 24, m = c & 0x7Fu;
+    if (m == 0) return sign ? 0x7FC00000u : 0u;
+    if (m == 0x6F) return sign | 0x7F800000u;
+    if (m < 8) return sign | ((m + 104u) << 23);  // 2^(m-23)
+    int E; uint32_t M, w;
+    if (m < 0x10)      { E = 0; M = m & 7; w = 3; }
+    else if (m < 0x20) { E = 1; M = m & 7; w = 3; if (m & 0x08) E = -E; }
+    else if (m < 0x40) { E = 2 | ((m >> 3) & 1); M = m & 7; w = 3; if (m & 0x10) E = -E; }
+    else if (m < 0x60) { E = 4 | ((m >> 2) & 3); M = m & 3; w = 2; if (m & 0x10) E = -E; }
+    else               { E = 8 | ((m >> 1) & 7); M = m & 1; w = 1; if (m & 0x10) E = -E; }
+    return sign | ((uint32_t)(E + 127) << 23) | (M << (23 - w));
+}
+
+// ------------------------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11): counter (c0, c1, 0, 0), key (k0, k1)
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t k0, uint32_t k1)
+{
+    uint32_t x0 = c0, x1 = c1, x2 = 0, x3 = 0;
+#pragma unroll
+    for (int r = 0; r < 10; r++) {
+        uint32_t hi0 = __umulhi(0xD2511F53u, x0), lo0 = 0xD2511F53u * x0;
+        uint32_t hi1 = __umulhi(0xCD9E8D57u, x2), lo1 = 0xCD9E8D57u * x2;
+        uint32_t n0 = hi1 ^ x1 ^ k0, n2 = hi0 ^ x3 ^ k1;
+        x0 = n0; x1 = lo1; x2 = n2; x3 = lo0;
+        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
+    }
+    return make_uint4(x0, x1, x2, x3);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Scale handling
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ int clamp_exp(int e) { return e < -126 ? -126 : (e > 126 ? 126 : e); }
+__device__ __forceinline__ float pow2f(int e) { return __uint_as_float((uint32_t)(e + 127) << 23); }  // |e| <= 126
+
+// scale exponent from the bits of amax (a non-negative finite binary32)
+__device__ __forceinline__ int scale_exp_from_amax(uint32_t ab, int target_exp)
+{
+    if (ab == 0) return 0;
+    int e = (ab >> 23) ? (int)(ab >> 23) - 127 : (31 - __clz(ab)) - 149;  // floor(log2 amax)
+    return clamp_exp(target_exp - e);
+}
+
+struct ConvParams {
+    const void* src;
+    void* dst;
+    unsigned long long n;
+    int scale_exp;                // used when neither pointer below is set
+    const int* d_scale_exp;       // delayed scaling: exponent read from the device
+    const uint32_t* d_amax_bits;  // just-in-time scaling: exponent derived from this amax
+    int target_exp;
+    unsigned flags;
+    unsigned long long seed;
+    uint32_t* amax_accum;         // when the kernel also reduces amax: accumulator and ticket (2 words)
+    float* d_amax_out;
+    int* d_scale_exp_out;
+    float* d_scale_out;
+};
+
+template <int SRC> struct SrcTraits;
+template <> struct SrcTraits<HIF8_F32>  { static constexpr int kPerVec = 4; };
+template <> struct SrcTraits<HIF8_BF16> { static constexpr int kPerVec = 8; };
+template <> struct SrcTraits<HIF8_F16>  { static constexpr int kPerVec = 8; };
+
+// element k of a 16-byte source vector: its value as binary32 and its raw encoding
+template <int SRC>
+__device__ __forceinline__ void unpack(const uint4& v, int k, float& x, uint32_t& raw)
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    if (SRC == HIF8_F32) { raw = w[k]; x = __uint_as_float(raw); }
+    else {
+        uint32_t word = w[k >> 1];
+        raw = (k & 1) ? (word >> 16) : (word & 0xFFFFu);
+        if (SRC == HIF8_BF16) x = __uint_as_float(raw << 16);
+        else x = __half2float(__ushort_as_half((unsigned short)raw));
+    }
+}
+
+template <int SRC>
+__device__ __forceinline__ void load_scalar(const void* p, unsigned long long i, float& x, uint32_t& raw)
+{
+    if (SRC == HIF8_F32) { raw = reinterpret_cast<const uint32_t*>(p)[i]; x = __uint_as_float(raw); }
+    else {
+        raw = reinterpret_cast<const unsigned short*>(p)[i];
+        if (SRC == HIF8_BF16) x = __uint_as_float(raw << 16);
+        else x = __half2float(__ushort_as_half((unsigned short)raw));
+    }
+}
+
+// binary32 value -> encoding of the destination format, round to nearest even
+template <int DT> __device__ __forceinline__ uint32_t to_bits(float v)
+{
+    if (DT == HIF8_F32) return (v != v) ? 0x7FC00000u : __float_as_uint(v);
+    if (DT == HIF8_BF16) {
+        if (v != v) return 0x7FC0u;
+        return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v));
+    }
+    if (v != v) return 0x7E00u;
+    return (uint32_t)__half_as_ushort(__float2half_rn(v));
+}
+
+// ------------------------------------------------------------------------------------------------
+// One element: scaled value -> HiF8 byte
+// ------------------------------------------------------------------------------------------------
+template <int MODE, int SRC>
+__device__ __forceinline__ uint32_t encode_one(float x, uint32_t raw, float scale, const uint8_t* s_ta,
+                                               const uint8_t* s_sh, uint32_t word)
+{
+    const float y = x * scale;
+    const uint32_t t = __float_as_uint(y);
+    if (MODE == HIF8_RND_TA) return s_ta[t >> 19];
+
+    const uint32_t a = t & 0x7FFFFFFFu;
+    const uint32_t sh = s_sh[a >> 23];  // number of discarded mantissa bits (23 - width); 0: nothing to round
+    // threshold T of Section 3.2 (with the guard that a zero fraction never rounds up: compare with max(T,1))
+    constexpr int kSrBits = (SRC == HIF8_F32) ? 24 : 16;
+    if (sh == kShSlow) {
+        // |y| < 2^-22: kept bits are zero, the fraction is F = |y| / 2^-22 and the result is 0 or 2^-22
+        const float ya = fabsf(y);
+        bool up;
+        if (MODE == HIF8_RND_TE) up = ya > 1.1920928955078125e-07f;  // above 2^-23; the tie goes to the even 0
+        else {
+            float fn; uint32_t T;
+            if (MODE == HIF8_RND_SR) { fn = floorf(ya * exp2f(22.f + kSrBits)); T = word >> (32 - kSrBits); }
+            else if (SRC == HIF8_F32) { fn = floorf(ya * 68719476736.f); T = raw & 0x3FFFu; }  // F14 = floor(F 2^14)
+            else { fn = floorf(ya * 16777216.f); T = 2u * (raw & 1u) + 1u; }                // F2 = floor(F 2^2)
+            up = fn >= (float)max(T, 1u);
+        }
+        return up ? (((t >> 24) & 0x80u) | 0x01u) : 0u;
+    }
+    const uint32_t s = sh ? sh : 23u;
+    uint32_t inc;
+    if (MODE == HIF8_RND_TE) {
+        // add half-1, plus one when the kept significand is odd (implicit one when no mantissa bit is kept)
+        uint32_t lsb = (s == 23u) ? 1u : ((t >> s) & 1u);
+        inc = (1u << (s - 1)) - 1u + lsb;
+    } else {
+        uint32_t inc_ssr;
+        if (SRC == HIF8_F32) inc_ssr = (0x4000u - max(raw & 0x3FFFu, 1u)) << (s - 14);  // SR14
+        else inc_ssr = (3u - 2u * (raw & 1u)) << (s - 2);                                // SR2: 4 - T2
+        if (MODE == HIF8_RND_SSR) inc = inc_ssr;
+        else if (MODE == HIF8_RND_HR) {
+            int E = (int)(a >> 23) - 127;                                                // Eq. 3
+            inc = (E > -4 && E < 4) ? (1u << (s - 1)) : inc_ssr;
+        } else {  // standard SR
+            uint32_t T = max(word >> (32 - kSrBits), 1u);
+            if (SRC == HIF8_F32) {
+                uint32_t k = 24u - s;  // F24 = discarded << k; up iff discarded >= ceil(T / 2^k)
+                inc = (1u << s) - ((T + (1u << k) - 1u) >> k);
+            } else inc = (0x10000u - T) << (s - 16);
+        }
+    }
+    if (sh == 0) inc = 0;
+    const uint32_t tr = (t + inc) & ~((1u << sh) - 1u);
+    return s_ta[tr >> 19];
+}
+
+// ------------------------------------------------------------------------------------------------
+// Block set-up: tables into shared memory, scale
+// ------------------------------------------------------------------------------------------------
+struct __align__(16) SmemTables {
+    uint8_t ta[8192];
+    uint8_t sh[256];
+    float dec[256];
+};
+
+template <bool NEED_TA, bool NEED_SH, bool NEED_DEC>
+__device__ __forceinline__ void setup_tables(SmemTables& s, unsigned flags)
+{
+    if (NEED_TA) {
+        const uint4* g = reinterpret_cast<const uint4*>(g_ta_table.v);
+        uint4* d = reinterpret_cast<uint4*>(s.ta);
+        for (int i = threadIdx.x; i < 512; i += kThreads) {
+            uint4 v = g[i];
+            if (flags) {  // Section 3 options: patch the Inf / NaN entries
+                uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                for (int j = 0; j < 4; j++) {
+                    uint32_t o = 0;
+#pragma unroll
+                    for (int b = 0; b < 4; b++) {
+                        uint32_t c = (w[j] >> (8 * b)) & 0xFFu;
+                        if ((flags & HIF8_FLAG_SATURATE) && (c & 0x7Fu) == 0x6Fu) c &= 0xFEu;
+                        if ((flags & HIF8_FLAG_NAN_TO_ZERO) && c == 0x80u) c = 0;
+                        o |= c << (8 * b);
+                    }
+                    w[j] = o;
+                }
+                v = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+            d[i] = v;
+        }
+    }
+    if (NEED_SH) {
+        int e = threadIdx.x;  // kThreads == 256 biased exponents
+        int E = e - 127;
+        s.sh[e] = (E >= 16 || e == 255) ? 0 : (E <= -23 ? kShSlow : (uint8_t)(23 - mant_width(E)));
+    }
+    if (NEED_DEC) s.dec[threadIdx.x] = __uint_as_float(decode_bits_f32(threadIdx.x));
+    __syncthreads();
+}
+
+__device__ __forceinline__ int resolve_scale_exp(const ConvParams& p)
+{
+    if (p.d_amax_bits) return scale_exp_from_amax(*p.d_amax_bits, p.target_exp);
+    if (p.d_scale_exp) return clamp_exp(*p.d_scale_exp);
+    return p.scale_exp;
+}
+
+// amax contribution of a value: |x| for finite x, ignored (NaN) otherwise; fmaxf drops NaN operands
+__device__ __forceinline__ float amax_step(float acc, float x) { return fmaxf(acc, fmaf(x, 0.0f, fabsf(x))); }
+
+__device__ __forceinline__ void block_amax_commit(float acc, uint32_t* accum)
+{
+    __shared__ uint32_t s_part[kThreads / 32];
+    uint32_t v = __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(acc));  // non-negative floats order as integers
+    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = v;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        v = threadIdx.x < kThreads / 32 ? s_part[threadIdx.x] : 0u;
+        v = __reduce_max_sync(0xFFFFFFFFu, v);
+        if (threadIdx.x == 0 && v) atomicMax(accum, v);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Encode / fake-quant kernel.  FQ = false: bytes out.  FQ = true: dequantized values in the source format.
+// AMAX = true: also reduce amax of the source into p.amax_accum[0]; the last block publishes it.
+// ------------------------------------------------------------------------------------------------
+template <int SRC, int MODE, bool FQ, bool AMAX>
+__global__ void __launch_bounds__(kThreads) convert_kernel(const ConvParams p, unsigned long long n_vec)
+{
+    __shared__ SmemTables sm;
+    setup_tables<true, MODE != HIF8_RND_TA, FQ>(sm, p.flags);
+    const int se = resolve_scale_exp(p);
+    const float scale = pow2f(se);
+    const int da = (-se) / 2, db = -se - da;  // descale in two exact steps (the first cannot leave the normal range)
+    const float d1 = pow2f(da), d2 = pow2f(db);
+    constexpr int PV = SrcTraits<SRC>::kPerVec;
+    const uint32_t k0 = (uint32_t)p.seed, k1 = (uint32_t)(p.seed >> 32);
+    float amax = 0.f;
+
+    const uint4* src = reinterpret_cast<const uint4*>(p.src);
+    const unsigned long long stride = (unsigned long long)gridDim.x * kThreads * kUnroll;
+    for (unsigned long long base = (unsigned long long)blockIdx.x * kThreads * kUnroll; base < n_vec; base += stride) {
+        uint4 v[kUnroll];
+#pragma unroll
+        for (int j = 0; j < kUnroll; j++) {
+            unsigned long long u = base + (unsigned long long)j * kThreads + threadIdx.x;
+            if (u < n_vec) v[j] = __ldcs(src + u); else v[j] = make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int j = 0; j < kUnroll; j++) {
+            unsigned long long u = base + (unsigned long long)j * kThreads + threadIdx.x;
+            if (u >= n_vec) continue;
+            uint32_t codes[PV];
+            uint4 r0 = make_uint4(0, 0, 0, 0), r1 = r0;
+            if (MODE == HIF8_RND_SR) {
+                r0 = philox4x32_10((uint32_t)(u * (PV / 4)), (uint32_t)((u * (PV / 4)) >> 32), k0, k1);
+                if (PV == 8) r1 = philox4x32_10((uint32_t)(u * 2 + 1), (uint32_t)((u * 2 + 1) >> 32), k0, k1);
+            }
+            const uint32_t rw[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+#pragma unroll
+            for (int k = 0; k < PV; k++) {
+                float x; uint32_t raw;
+                unpack<SRC>(v[j], k, x, raw);
+                if (AMAX) amax = amax_step(amax, x);
+                codes[k] = encode_one<MODE, SRC>(x, raw, scale, sm.ta, sm.sh, rw[k]);
+            }
+            if (!FQ) {
+                uint32_t w0 = codes[0] | (codes[1] << 8) | (codes[2] << 16) | (codes[3] << 24);
+                if (PV == 4) __stcs(reinterpret_cast<uint32_t*>(p.dst) + u, w0);
+                else {
+                    uint32_t w1 = codes[4] | (codes[5] << 8) | (codes[6] << 16) | (codes[7] << 24);
+                    __stcs(reinterpret_cast<uint2*>(p.dst) + u, make_uint2(w0, w1));
+                }
+            } else {
+                uint32_t o[PV];
+#pragma unroll
+                for (int k = 0; k < PV; k++) o[k] = to_bits<SRC>(sm.dec[codes[k]] * d1 * d2);
+                uint4 out;
+                if (PV == 4) out = make_uint4(o[0], o[1], o[2], o[3]);
+                else out = make_uint4(o[0] | (o[1] << 16), o[2] | (o[3] << 16), o[4] | (o[5] << 16), o[6] | (o[7] << 16));
+                __stcs(reinterpret_cast<uint4*>(p.dst) + u, out);
+            }
+        }
+    }
+    // elements not covered by whole vectors (tail, or everything when the pointers are not 16-byte aligned)
+    {
+        const unsigned long long first = n_vec * PV;
+        const unsigned long long tid = (unsigned long long)blockIdx.x * kThreads + threadIdx.x;
+        for (unsigned long long i = first + tid; i < p.n; i += (unsigned long long)gridDim.x * kThreads) {
+            float x; uint32_t raw;
+            load_scalar<SRC>(p.src, i, x, raw);
+            if (AMAX) amax = amax_step(amax, x);
+            uint32_t word = 0;
+            if (MODE == HIF8_RND_SR) {
+                uint4 r = philox4x32_10((uint32_t)(i >> 2), (uint32_t)(i >> 34), k0, k1);
+                const uint32_t rr[4] = {r.x, r.y, r.z, r.w};
+                word = rr[i & 3];
+            }
+            uint32_t c = encode_one<MODE, SRC>(x, raw, scale, sm.ta, sm.sh, word);
+            if (!FQ) reinterpret_cast<uint8_t*>(p.dst)[i] = (uint8_t)c;
+            else {
+                uint32_t o = to_bits<SRC>(sm.dec[c] * d1 * d2);
+                if (SRC == HIF8_F32) reinterpret_cast<uint32_t*>(p.dst)[i] = o;
+                else reinterpret_cast<unsigned short*>(p.dst)[i] = (unsigned short)o;
+            }
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        if (p.d_scale_exp_out) *p.d_scale_exp_out = se;
+        if (p.d_scale_out) *p.d_scale_out = scale;
+        if (!AMAX && p.d_amax_out && p.d_amax_bits) *p.d_amax_out = __uint_as_float(*p.d_amax_bits);
+    }
+    if (AMAX) {
+        block_amax_commit(amax, p.amax_accum);
+        if (threadIdx.x == 0) {
+            __threadfence();
+            uint32_t ticket = atomicAdd(p.amax_accum + 1, 1u);
+            if (ticket == gridDim.x - 1) {  // last block: every partial maximum is visible
+                __threadfence();
+                uint32_t ab = atomicMax(p.amax_accum, 0u);
+                if (p.d_amax_out) *p.d_amax_out = __uint_as_float(ab);
+            }
+        }
+    }
+}
+
+// amax only (first pass of just-in-time scaling)
+template <int SRC>
+__global__ void __launch_bounds__(kThreads) amax_kernel(const void* __restrict__ srcv, unsigned long long n,
+                                                        unsigned long long n_vec, uint32_t* accum)
+{
+    constexpr int PV = SrcTraits<SRC>::kPerVec;
+    const uint4* src = reinterpret_cast<const uint4*>(srcv);
+    float amax = 0.f;
+    const unsigned long long stride = (unsigned long long)gridDim.x * kThreads * kUnroll;
+    for (unsigned long long base = (unsigned long long)blockIdx.x * kThreads * kUnroll; base < n_vec; base += stride) {
+        uint4 v[kUnroll];
+#pragma unroll
+        for (int j = 0; j < kUnroll; j++) {
+            unsigned long long u = base + (unsigned long long)j * kThreads + threadIdx.x;
+            v[j] = (u < n_vec) ? __ldg(src + u) : make_uint4(0, 0, 0, 0);  // default policy: keep lines for the second pass
+        }
+#pragma unroll
+        for (int j = 0; j < kUnroll; j++) {
+#pragma unroll
+            for (int k = 0; k < PV; k++) {
+                float x; uint32_t raw;
+                unpack<SRC>(v[j], k, x, raw);
+                amax = amax_step(amax, x);
+            }
+        }
+    }
+    const unsigned long long tid = (unsigned long long)blockIdx.x * kThreads + threadIdx.x;
+    for (unsigned long long i = n_vec * PV + tid; i < n; i += (unsigned long long)gridDim.x * kThreads) {
+        float x; uint32_t raw;
+        load_scalar<SRC>(srcv, i, x, raw);
+        amax = amax_step(amax, x);
+    }
+    block_amax_commit(amax, accum);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Decode kernel: bytes -> DT, times 2^-scale_exp
+// ------------------------------------------------------------------------------------------------
+template <int DT>
+__global__ void __launch_bounds__(kThreads) decode_kernel(const uint8_t* __restrict__ src, void* __restrict__ dst,
+                                                          unsigned long long n, unsigned long long n_vec, int se)
+{
+    __shared__ SmemTables sm;
+    setup_tables<false, false, true>(sm, 0);
+    const int da = (-se) / 2, db = -se - da;
+    const float d1 = pow2f(da), d2 = pow2f(db);
+    constexpr int PV = SrcTraits<DT>::kPerVec;  // codes per 16-byte store
+    const unsigned long long stride = (unsigned long long)gridDim.x * kThreads * kUnroll;
+    for (unsigned long long base = (unsigned long long)blockIdx.x * kThreads * kUnroll; base < n_vec; base += stride) {
+        uint2 v[kUnroll];
+#pragma unroll
+        for (int j = 0; j < kUnroll; j++) {
+            unsigned long long u = base + (unsigned long long)j * kThreads + threadIdx.x;
+            v[j] = make_uint2(0, 0);
+            if (u < n_vec) {
+                if (PV == 4) v[j].x = __ldcs(reinterpret_cast<const uint32_t*>(src) + u);
+                else v[j] = __ldcs(reinterpret_cast<const uint2*>(src) + u);
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < kUnroll; j++) {
+            unsigned long long u = base + (unsigned long long)j * kThreads + threadIdx.x;
+            if (u >= n_vec) continue;
+            uint32_t o[PV];
+#pragma unroll
+            for (int k = 0; k < PV; k++) {
+                uint32_t c = ((k < 4 ? v[j].x : v[j].y) >> (8 * (k & 3))) & 0xFFu;
+                o[k] = to_bits<DT>(sm.dec[c] * d1 * d2);
+            }
+            uint4 out;
+            if (PV == 4) out = make_uint4(o[0], o[1], o[2], o[3]);
+            else out = make_uint4(o[0] | (o[1] << 16), o[2] | (o[3] << 16), o[4] | (o[5] << 16), o[6] | (o[7] << 16));
+            __stcs(reinterpret_cast<uint4*>(dst) + u, out);
+        }
+    }
+    const unsigned long long tid = (unsigned long long)blockIdx.x * kThreads + threadIdx.x;
+    for (unsigned long long i = n_vec * PV + tid; i < n; i += (unsigned long long)gridDim.x * kThreads) {
+        uint32_t o = to_bits<DT>(sm.dec[src[i]] * d1 * d2);
+        if (DT == HIF8_F32) reinterpret_cast<uint32_t*>(dst)[i] = o;
+        else reinterpret_cast<unsigned short*>(dst)[i] = (unsigned short)o;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Host side
+// ------------------------------------------------------------------------------------------------
+int g_sm_count[64];
+int g_cc[64];
+
+int device_info(int* sms)
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return HIF8_ERR_CUDA;
+    if (g_sm_count[dev] == 0) {
+        int n = 0, major = 0, minor = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return HIF8_ERR_CUDA;
+        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+        cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, dev);
+        g_cc[dev] = major * 10 + minor;
+        g_sm_count[dev] = n;
+    }
+    if (g_cc[dev] != 100) return HIF8_ERR_CUDA;
+    *sms = g_sm_count[dev];
+    return HIF8_OK;
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+unsigned grid_for(unsigned long long n_vec, unsigned long long n, int sms)
+{
+    unsigned long long per_block = (unsigned long long)kThreads * kUnroll;
+    unsigned long long need = n_vec ? (n_vec + per_block - 1) / per_block : (n + kThreads - 1) / kThreads;
+    unsigned long long cap = (unsigned long long)sms * kBlocksPerSM;
+    if (need >= cap) return (unsigned)cap;
+    if (need == 0) need = 1;
+    return (unsigned)need;
+}
+
+template <int SRC, int MODE, bool FQ, bool AMAX>
+int launch_convert(const ConvParams& p, bool vec_ok, int sms, cudaStream_t st)
+{
+    constexpr int PV = SrcTraits<SRC>::kPerVec;
+    unsigned long long n_vec = vec_ok ? p.n / PV : 0;
+    unsigned grid = grid_for(n_vec, p.n, sms);
+    convert_kernel<SRC, MODE, FQ, AMAX><<<grid, kThreads, 0, st>>>(p, n_vec);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
+}
+
+template <int SRC, bool FQ, bool AMAX>
+int dispatch_mode(int rnd, const ConvParams& p, bool vec_ok, int sms, cudaStream_t st)
+{
+    switch (rnd) {
+        case HIF8_RND_TA: return launch_convert<SRC, HIF8_RND_TA, FQ, AMAX>(p, vec_ok, sms, st);
+        case HIF8_RND_HR: return launch_convert<SRC, HIF8_RND_HR, FQ, AMAX>(p, vec_ok, sms, st);
+        case HIF8_RND_SSR: return launch_convert<SRC, HIF8_RND_SSR, FQ, AMAX>(p, vec_ok, sms, st);
+        case HIF8_RND_TE: return launch_convert<SRC, HIF8_RND_TE, FQ, AMAX>(p, vec_ok, sms, st);
+        default: return launch_convert<SRC, HIF8_RND_SR, FQ, AMAX>(p, vec_ok, sms, st);
+    }
+}
+
+template <bool FQ, bool AMAX>
+int dispatch_convert(int dtype, int rnd, const ConvParams& p, bool vec_ok, int sms, cudaStream_t st)
+{
+    switch (dtype) {
+        case HIF8_F32: return dispatch_mode<HIF8_F32, FQ, AMAX>(rnd, p, vec_ok, sms, st);
+        case HIF8_BF16: return dispatch_mode<HIF8_BF16, FQ, AMAX>(rnd, p, vec_ok, sms, st);
+        default: return dispatch_mode<HIF8_F16, FQ, AMAX>(rnd, p, vec_ok, sms, st);
+    }
+}
+
+int launch_amax(const void* src, int dtype, unsigned long long n, uint32_t* accum, int sms, cudaStream_t st)
+{
+    bool vec_ok = aligned16(src);
+    unsigned long long pv = dtype == HIF8_F32 ? 4 : 8;
+    unsigned long long n_vec = vec_ok ? n / pv : 0;
+    unsigned grid = grid_for(n_vec, n, sms);
+    switch (dtype) {
+        case HIF8_F32: amax_kernel<HIF8_F32><<<grid, kThreads, 0, st>>>(src, n, n_vec, accum); break;
+        case HIF8_BF16: amax_kernel<HIF8_BF16><<<grid, kThreads, 0, st>>>(src, n, n_vec, accum); break;
+        default: amax_kernel<HIF8_F16><<<grid, kThreads, 0, st>>>(src, n, n_vec, accum); break;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
+}
+
+int check_common(int dtype, int rnd, unsigned flags)
+{
+    if (dtype != HIF8_F32 && dtype != HIF8_BF16 && dtype != HIF8_F16) return HIF8_ERR_DTYPE;
+    if (rnd < HIF8_RND_TA || rnd > HIF8_RND_SR) return HIF8_ERR_ROUND;
+    if (flags & ~(HIF8_FLAG_SATURATE | HIF8_FLAG_NAN_TO_ZERO)) return HIF8_ERR_FLAGS;
+    return HIF8_OK;
+}
+
+constexpr size_t kConvWorkspaceBytes = 256;
+
+}  // namespace
+}  // namespace hif8
+
+using namespace hif8;
+
+extern "C" {
+
+int hif8_encode(const void* src, int src_dtype, uint8_t* dst, size_t n, int scale_exp, int rnd, unsigned flags,
+                uint64_t seed, hif8_stream_t stream)
+{
+    int rc = check_common(src_dtype, rnd, flags);
+    if (rc) return rc;
+    if (scale_exp < -126 || scale_exp > 126) return HIF8_ERR_SCALE_RANGE;
+    if (n == 0) return HIF8_OK;
+    if (!src || !dst) return HIF8_ERR_NULL;
+    int sms; rc = device_info(&sms);
+    if (rc) return rc;
+    ConvParams p{};
+    p.src = src; p.dst = dst; p.n = n; p.scale_exp = scale_exp; p.flags = flags; p.seed = seed;
+    size_t out_align = src_dtype == HIF8_F32 ? 4 : 8;
+    bool vec_ok = aligned16(src) && (reinterpret_cast<uintptr_t>(dst) % out_align) == 0;
+    return dispatch_convert<false, false>(src_dtype, rnd, p, vec_ok, sms, (cudaStream_t)stream);
+}
+
+int hif8_decode(const uint8_t* src, void* dst, int dst_dtype, size_t n, int scale_exp, hif8_stream_t stream)
+{
+    if (dst_dtype != HIF8_F32 && dst_dtype != HIF8_BF16 && dst_dtype != HIF8_F16) return HIF8_ERR_DTYPE;
+    if (scale_exp < -126 || scale_exp > 126) return HIF8_ERR_SCALE_RANGE;
+    if (n == 0) return HIF8_OK;
+    if (!src || !dst) return HIF8_ERR_NULL;
+    int sms; int rc = device_info(&sms);
+    if (rc) return rc;
+    unsigned long long pv = dst_dtype == HIF8_F32 ? 4 : 8;
+    bool vec_ok = aligned16(dst) && (reinterpret_cast<uintptr_t>(src) % pv) == 0;
+    unsigned long long n_vec = vec_ok ? n / pv : 0;
+    unsigned grid = grid_for(n_vec, n, sms);
+    cudaStream_t st = (cudaStream_t)stream;
+    switch (dst_dtype) {
+        case HIF8_F32: decode_kernel<HIF8_F32><<<grid, kThreads, 0, st>>>(src, dst, n, n_vec, scale_exp); break;
+        case HIF8_BF16: decode_kernel<HIF8_BF16><<<grid, kThreads, 0, st>>>(src, dst, n, n_vec, scale_exp); break;
+        default: decode_kernel<HIF8_F16><<<grid, kThreads, 0, st>>>(src, dst, n, n_vec, scale_exp); break;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
+}
+
+// shared by hif8_amax_scale_encode and hif8_fake_quant
+static int scaled_convert(bool fq, const void* src, void* dst, int dtype, size_t n, bool jit, int target_exp,
+                          const int* d_scale_exp_in, int scale_exp, int rnd, unsigned flags, uint64_t seed,
+                          float* d_amax_out, int* d_scale_exp_out, float* d_scale_out, void* workspace,
+                          size_t workspace_bytes, bool want_amax, cudaStream_t st)
+{
+    int sms; int rc = device_info(&sms);
+    if (rc) return rc;
+    uint32_t* ws = reinterpret_cast<uint32_t*>(workspace);
+    ConvParams p{};
+    p.src = src; p.dst = dst; p.n = n; p.flags = flags; p.seed = seed; p.target_exp = target_exp;
+    p.scale_exp = scale_exp; p.d_scale_exp = d_scale_exp_in;
+    p.d_amax_out = d_amax_out; p.d_scale_exp_out = d_scale_exp_out; p.d_scale_out = d_scale_out;
+    size_t out_align = fq ? 16 : (dtype == HIF8_F32 ? 4 : 8);
+    bool vec_ok = aligned16(src) && (reinterpret_cast<uintptr_t>(dst) % out_align) == 0;
+    if (jit || want_amax) {
+        if (!ws || workspace_bytes < kConvWorkspaceBytes || (reinterpret_cast<uintptr_t>(ws) & 255u)) return HIF8_ERR_WORKSPACE;
+        if (cudaMemsetAsync(ws, 0, 8, st) != cudaSuccess) return HIF8_ERR_CUDA;
+    }
+    if (jit) {
+        rc = launch_amax(src, dtype, n, ws, sms, st);
+        if (rc) return rc;
+        p.d_amax_bits = ws;
+        return fq ? dispatch_convert<true, false>(dtype, rnd, p, vec_ok, sms, st)
+                  : dispatch_convert<false, false>(dtype, rnd, p, vec_ok, sms, st);
+    }
+    if (want_amax) {
+        p.amax_accum = ws;
+        return fq ? dispatch_convert<true, true>(dtype, rnd, p, vec_ok, sms, st)
+                  : dispatch_convert<false, true>(dtype, rnd, p, vec_ok, sms, st);
+    }
+    return fq ? dispatch_convert<true, false>(dtype, rnd, p, vec_ok, sms, st)
+              : dispatch_convert<false, false>(dtype, rnd, p, vec_ok, sms, st);
+}
+
+int hif8_amax_scale_encode(const void* src, int src_dtype, uint8_t* dst, size_t n, int target_exp, int rnd,
+                           unsigned flags, uint64_t seed, const int* d_scale_exp_in, float* d_amax_out,
+                           int* d_scale_exp_out, float* d_scale_out, void* workspace, size_t workspace_bytes,
+                           hif8_stream_t stream)
+{
+    int rc = check_common(src_dtype, rnd, flags);
+    if (rc) return rc;
+    if (target_exp < -22 || target_exp > 15) return HIF8_ERR_SCALE_RANGE;
+    if (!workspace || workspace_bytes < kConvWorkspaceBytes || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+        return HIF8_ERR_WORKSPACE;
+    if (n && (!src || !dst)) return HIF8_ERR_NULL;
+    bool jit = d_scale_exp_in == nullptr;
+    return scaled_convert(false, src, dst, src_dtype, n, jit, target_exp, d_scale_exp_in, 0, rnd, flags, seed,
+                          d_amax_out, d_scale_exp_out, d_scale_out, workspace, workspace_bytes, !jit,
+                          (cudaStream_t)stream);
+}
+
+int hif8_fake_quant(const void* src, void* dst, int dtype, size_t n, int use_amax, int scale_or_target_exp, int rnd,
+                    unsigned flags, uint64_t seed, float* d_amax_out, int* d_scale_exp_out, void* workspace,
+                    size_t workspace_bytes, hif8_stream_t stream)
+{
+    int rc = check_common(dtype, rnd, flags);
+    if (rc) return rc;
+    if (use_amax) {
+        if (scale_or_target_exp < -22 || scale_or_target_exp > 15) return HIF8_ERR_SCALE_RANGE;
+        if (!workspace || workspace_bytes < kConvWorkspaceBytes || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+            return HIF8_ERR_WORKSPACE;
+    } else if (scale_or_target_exp < -126 || scale_or_target_exp > 126) return HIF8_ERR_SCALE_RANGE;
+    if (n && (!src || !dst)) return HIF8_ERR_NULL;
+    if (n == 0 && !use_amax) return HIF8_OK;
+    return scaled_convert(true, src, dst, dtype, n, use_amax != 0, scale_or_target_exp, nullptr,
+                          use_amax ? 0 : scale_or_target_exp, rnd, flags, seed, d_amax_out, d_scale_exp_out, nullptr,
+                          workspace, workspace_bytes, false, (cudaStream_t)stream);
+}
+
+size_t hif8_workspace_bytes(int which, size_t n)
+{
+    (void)n;
+    switch (which) {
+        case HIF8_WS_AMAX_SCALE_ENCODE:
+        case HIF8_WS_FAKE_QUANT: return kConvWorkspaceBytes;
+        default: return 0;
+    }
+}
+
+const char* hif8_status_string(int status)
+{
+    switch (status) {
+        case HIF8_OK: return "ok";
+        case HIF8_ERR_NULL: return "required pointer is NULL";
+        case HIF8_ERR_DTYPE: return "unknown element format";
+        case HIF8_ERR_ROUND: return "unknown rounding method";
+        case HIF8_ERR_FLAGS: return "unknown option bits";
+        case HIF8_ERR_SCALE_RANGE: return "scale or target exponent out of range";
+        case HIF8_ERR_SHAPE: return "unsupported extent or leading dimension";
+        case HIF8_ERR_ALIGN: return "operand not 16-byte aligned";
+        case HIF8_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case HIF8_ERR_CUDA: return "CUDA call failed or device is not compute capability 10.0";
+        case HIF8_ERR_DEVICE_TIMEOUT: return "bounded device-side wait gave up";
+        default: return "unknown status";
+    }
+}
+
+uint64_t hif8_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

@@ -1,0 +1,48 @@
+"""Host-side checks that need no GPU: the library loads, exports every declared symbol, and rejects bad
+arguments before touching a device."""
+import ctypes
+import os
+import re
+
+import paper_2409_16626_b200 as H
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "hif8.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(hif8_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    lib = ctypes.CDLL(H.LIB_PATH)
+    names = declared_symbols()
+    assert {"hif8_encode", "hif8_decode", "hif8_amax_scale_encode", "hif8_fake_quant", "hif8_gemm"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_status_strings_and_workspace():
+    for s in range(0, 11):
+        assert H.hif8_status_string(s) not in ("", "unknown status")
+    assert H.hif8_status_string(99) == "unknown status"
+    assert H.hif8_workspace_bytes(H.WS_AMAX_SCALE_ENCODE, 1 << 20) >= 8
+    assert H.hif8_workspace_bytes(H.WS_FAKE_QUANT, 1 << 20) >= 8
+
+
+def test_argument_errors_before_any_launch():
+    before = H.hif8_launch_count()
+    assert H.hif8_encode(0, 7, 0, 16, stream=0, check=False) == 2            # dtype
+    assert H.hif8_encode(0, H.F32, 0, 16, rnd=9, stream=0, check=False) == 3  # rounding
+    assert H.hif8_encode(0, H.F32, 0, 16, flags=8, stream=0, check=False) == 4
+    assert H.hif8_encode(0, H.F32, 0, 16, scale_exp=127, stream=0, check=False) == 5
+    assert H.hif8_encode(0, H.F32, 0, 0, stream=0, check=False) == 0         # empty tensor is fine
+    assert H.hif8_decode(0, 0, 5, 16, stream=0, check=False) == 2
+    assert H.hif8_decode(0, 0, H.F16, 16, scale_exp=-127, stream=0, check=False) == 5
+    assert H.hif8_decode(0, 0, H.F16, 0, stream=0, check=False) == 0
+    assert H.hif8_amax_scale_encode(0, H.F32, 0, 16, target_exp=16, stream=0, check=False) == 5
+    assert H.hif8_amax_scale_encode(0, H.F32, 0, 16, target_exp=14, stream=0, check=False) == 8   # no workspace
+    assert H.hif8_fake_quant(0, 0, H.BF16, 16, use_amax=1, scale_or_target_exp=14, stream=0, check=False) == 8
+    assert H.hif8_fake_quant(0, 0, H.BF16, 16, use_amax=0, scale_or_target_exp=200, stream=0, check=False) == 5
+    assert H.hif8_launch_count() == before
