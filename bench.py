@@ -1,0 +1,291 @@
+#!/usr/bin/env python
+"""Benchmark of the HiF8 conversion hot path on B200.
+
+One step = per-tensor scaled encode (amax -> power-of-two scale -> HiF8 bytes, just-in-time form) followed
+by decode back to FP32 of one FP32 4096x4096 N(0,1) tensor (synthetic, seeded).  The metric is algorithmic
+bytes moved per second: 9 B/element for the encode call (4 read for amax, 4 read + 1 written for the
+conversion) plus 5 B/element for the decode call (1 read, 4 written).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+N > 1 is launched under torch.distributed.run, one rank per GPU; ranks convert independent tensors (no
+data-path collective, weak scaling) and rank 0 prints the single JSON line.
+`--impl reference` times the CPU oracle (oracle/) on a bounded sample of the same workload.
+"""
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads as W  # noqa: E402
+
+ROWS, COLS = 4096, 4096
+N_EL = ROWS * COLS
+BYTES_ENCODE = 9 * N_EL   # amax read + conversion read + byte write
+BYTES_DECODE = 5 * N_EL
+BYTES_STEP = BYTES_ENCODE + BYTES_DECODE
+POOL = 6                  # rotating buffer sets: 6 x 64 MiB of input alone exceeds the 126 MB L2
+WORKLOAD = "fp32_4096x4096_normal_amax_scale_encode_then_decode"
+METRIC = "hif8_encode_decode_throughput"
+UNIT = "GB/s"
+
+
+def env_int(name, default):
+    try:
+        return int(os.environ.get(name, default))
+    except ValueError:
+        return default
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def __enter__(self):
+        if self.nv is not None:
+            self._thread = threading.Thread(target=self._run, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join()
+
+    def summary(self):
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def cpu_baseline(sample_elems):
+    """The oracle as it stands (brute-force nearest-of-256 encode), on a leading slice of the same tensor."""
+    from oracle import hif8_oracle as O
+    x = W.normal_f32((ROWS, COLS), seed=1234).reshape(-1)[:sample_elems]
+    t0 = time.perf_counter()
+    _, se = O.amax_scale(x, O.F32, 14)
+    codes = O.encode(x, O.F32, se, O.TA, 0, quick=False)
+    O.decode(codes, O.F32, se)
+    dt = time.perf_counter() - t0
+    return {"value": 14 * sample_elems / dt / 1e9, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
+            "sample": f"first {sample_elems} of {N_EL} elements: amax + brute-force TA encode + decode, {dt:.2f} s",
+            "elements_per_s": sample_elems / dt}
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    from oracle import hif8_oracle as O
+    sample = 1 << 20
+    x = W.normal_f32((ROWS, COLS), seed=1234).reshape(-1)[:sample]
+
+    def step():
+        _, se = O.amax_scale(x, O.F32, 14)
+        codes = O.encode(x, O.F32, se, O.TA, 0, quick=False)
+        O.decode(codes, O.F32, se)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    value = 14 * sample / dt / 1e9
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "sample": f"first {sample} of {N_EL} elements per step"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
+                             "sample": f"first {sample} of {N_EL} elements per step"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    rank, world, local = env_int("RANK", 0), env_int("WORLD_SIZE", 1), env_int("LOCAL_RANK", 0)
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    import paper_2409_16626_b200 as H
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    # ---- synthetic inputs: POOL independent N(0,1) tensors per rank, resident in HBM
+    srcs = [torch.from_numpy(W.normal_f32((ROWS, COLS), seed=1234 + 100 * rank + i)).cuda() for i in range(POOL)]
+    codes = [torch.empty(N_EL, dtype=torch.uint8, device="cuda") for _ in range(POOL)]
+    backs = [torch.empty(N_EL, dtype=torch.float32, device="cuda") for _ in range(POOL)]
+    wsb = H.hif8_workspace_bytes(H.WS_AMAX_SCALE_ENCODE, N_EL)
+    ws = torch.empty(max(wsb, 256), dtype=torch.uint8, device="cuda")
+    scal = torch.zeros(4, dtype=torch.int32, device="cuda")   # amax, scale_exp, scale
+    stream = torch.cuda.current_stream()
+    sp = stream.cuda_stream
+
+    def encode_call(i):
+        H.hif8_amax_scale_encode(srcs[i], H.F32, codes[i], N_EL, 14, H.RND_TA, 0, 0, None, scal[0:1], scal[1:2], scal[2:3],
+                                 ws, wsb, stream=sp)
+
+    def decode_call(i, se):
+        H.hif8_decode(codes[i], backs[i], H.F32, N_EL, se, stream=sp)
+
+    encode_call(0)
+    torch.cuda.synchronize()
+    se = int(scal[1].item())   # same distribution for every tensor of the pool: the descale exponent is fixed up front
+
+    for w in range(args.warmup):
+        encode_call(w % POOL)
+        decode_call(w % POOL, se)
+    torch.cuda.synchronize()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- timed region: device-resident inputs, CUDA events on the launching stream
+    K = args.steps
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * K + 1)]
+    launches0 = H.hif8_launch_count()
+    barrier()
+    with ClockSampler(local) as clk:
+        ev[0].record(stream)
+        for k in range(K):
+            i = k % POOL
+            encode_call(i)
+            ev[2 * k + 1].record(stream)
+            decode_call(i, se)
+            ev[2 * k + 2].record(stream)
+        torch.cuda.synchronize()
+    barrier()
+    launches = H.hif8_launch_count() - launches0
+    total_ms = ev[0].elapsed_time(ev[2 * K])
+    enc_ms = sum(ev[2 * k].elapsed_time(ev[2 * k + 1]) for k in range(K)) / K
+    dec_ms = sum(ev[2 * k + 1].elapsed_time(ev[2 * k + 2]) for k in range(K)) / K
+
+    # ---- end to end: pinned host input -> device, both calls, results back to pinned host memory
+    E = max(3, min(args.e2e_steps, K))
+    h_src = torch.from_numpy(W.normal_f32((ROWS, COLS), seed=999 + rank)).pin_memory()
+    h_codes = torch.empty(N_EL, dtype=torch.uint8).pin_memory()
+    h_back = torch.empty(N_EL, dtype=torch.float32).pin_memory()
+
+    def e2e_step(i):
+        srcs[i].copy_(h_src, non_blocking=True)
+        encode_call(i)
+        decode_call(i, se)
+        h_codes.copy_(codes[i], non_blocking=True)
+        h_back.copy_(backs[i].view(-1), non_blocking=True)
+
+    for w in range(3):
+        e2e_step(w % POOL)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for k in range(E):
+        e2e_step(k % POOL)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / E
+
+    if world > 1:
+        t = torch.tensor([total_ms, e2e_ms, enc_ms, dec_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms, enc_ms, dec_ms = [float(v) for v in t.cpu()]
+
+    if rank == 0:
+        ms_per_step = total_ms / K
+        value = world * BYTES_STEP / (ms_per_step * 1e-3) / 1e9
+        peak, peak_kind = load_peaks()
+        # dominant kernel: the decode launch (1 B read + 4 B written per element, one kernel per call)
+        dec_gbs = BYTES_DECODE / (dec_ms * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "u8", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "elements": N_EL, "rounding": "TA", "target_exp": 14,
+                       "l2": f"inputs rotate over {POOL} buffer sets ({POOL * N_EL * 4 >> 20} MiB of sources) > 126 MB L2",
+                       "bytes_per_step": BYTES_STEP, "elements_per_s": world * N_EL / (ms_per_step * 1e-3)},
+            "clocks": clk.summary(),
+            "e2e": {"value": world * BYTES_STEP / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
+                    "h2d_bytes_per_step": 4 * N_EL, "d2h_bytes_per_step": 5 * N_EL},
+            "gpu_launches": int(launches),
+            "roofline": {"bound": "hbm", "kernel": "decode_kernel<f32>", "achieved": dec_gbs, "peak": peak,
+                         "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": dec_gbs / peak, "traffic": None,
+                         "algorithmic_bytes_per_launch": BYTES_DECODE, "avg_launch_ms": dec_ms},
+            "calls": {"amax_scale_encode_ms": enc_ms, "amax_scale_encode_GBps": BYTES_ENCODE / (enc_ms * 1e-3) / 1e9,
+                      "decode_ms": dec_ms, "decode_GBps": dec_gbs},
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(1 << 23)
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
