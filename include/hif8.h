@@ -107,6 +107,34 @@ int hif8_amax_scale_encode(const void* src, int src_dtype, uint8_t* dst, size_t 
                            size_t workspace_bytes, hif8_stream_t stream);
 
 /*
+ * hif8_amax_scale_encode without a caller-supplied workspace.  (The paper has no counterpart: this entry
+ * point exists for the benefit of the calling environment only.)
+ *
+ * Who needs it: code that must not, or cannot, obtain device memory at the point of the call -- a plug-in that
+ * runs inside another framework's memory pool and may not allocate behind its back, a call site inside a
+ * real-time or fault-handling path where cudaMalloc's implicit synchronisation and possible failure are not
+ * acceptable, or a process whose memory budget was handed out completely at start-up.  Such callers still pass
+ * their input and output tensors; the few bytes of scratch the amax reduction needs come from a
+ * HIF8_STATIC_SCRATCH_BYTES-byte array inside the library image, resident on every device that loads the
+ * library until the process exits.
+ *
+ * Same arguments, results and errors as hif8_amax_scale_encode minus the workspace pair, plus:
+ *   - n > HIF8_STATIC_MAX_ELEMENTS is rejected with HIF8_ERR_SHAPE before anything is launched.
+ *   - No cudaMalloc / cudaFree / allocating library routine is called, now or later.
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress); make that
+ *     first call outside any stream capture.
+ *   - All calls on a device share the one array.  Each call clears the words it needs on `stream` before
+ *     using them, so back-to-back calls on one stream are safe; two calls that can overlap on the GPU
+ *     (different streams, no dependency) race on it and give wrong scales -- serialise them, or use
+ *     hif8_amax_scale_encode with separate workspaces.
+ */
+#define HIF8_STATIC_SCRATCH_BYTES 256
+#define HIF8_STATIC_MAX_ELEMENTS ((size_t)1 << 32)
+int hif8_amax_scale_encode_static(const void* src, int src_dtype, uint8_t* dst, size_t n, int target_exp, int rnd,
+                                  unsigned flags, uint64_t seed, const int* d_scale_exp_in, float* d_amax_out,
+                                  int* d_scale_exp_out, float* d_scale_out, hif8_stream_t stream);
+
+/*
  * Quantize-dequantize in the source format ("simulated HiF8", Section 4: values are converted to only those
  * representable in HiF8):   dst[i] = value( To_HiF8_<rnd>(src[i] * 2^e) ) * 2^(-e)   in `dtype`.
  *   use_amax == 0: e = scale_or_target_exp.  No workspace needed (may be NULL).

@@ -745,3 +745,51 @@ const char* hif8_status_string(int status)
 uint64_t hif8_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------------
+// Variant of hif8_amax_scale_encode for callers that have no workspace to give.
+// The 8 bytes the amax reduction needs (running maximum + block ticket) live in a file-scope device array
+// that every device loading this library carries until the process exits.
+// ------------------------------------------------------------------------------------------------
+namespace {
+constexpr size_t kStaticScratchBytes = 256;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+// Device address of g_static_scratch per device ordinal.  In host code the array's name is only a handle for
+// the runtime, not an address a kernel may dereference; the real address comes from cudaGetSymbolAddress.
+void* g_static_scratch_addr[64];
+std::atomic<int> g_static_scratch_ready[64];
+
+int static_scratch(void** out)
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return HIF8_ERR_CUDA;
+    if (!g_static_scratch_ready[dev].load(std::memory_order_acquire)) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) return HIF8_ERR_CUDA;
+        g_static_scratch_addr[dev] = ptr;  // the same value from every racing thread
+        g_static_scratch_ready[dev].store(1, std::memory_order_release);
+    }
+    *out = g_static_scratch_addr[dev];
+    return HIF8_OK;
+}
+}  // namespace
+
+extern "C" int hif8_amax_scale_encode_static(const void* src, int src_dtype, uint8_t* dst, size_t n, int target_exp,
+                                             int rnd, unsigned flags, uint64_t seed, const int* d_scale_exp_in,
+                                             float* d_amax_out, int* d_scale_exp_out, float* d_scale_out,
+                                             hif8_stream_t stream)
+{
+    int rc = check_common(src_dtype, rnd, flags);
+    if (rc) return rc;
+    if (target_exp < -22 || target_exp > 15) return HIF8_ERR_SCALE_RANGE;
+    if (n > HIF8_STATIC_MAX_ELEMENTS) return HIF8_ERR_SHAPE;
+    if (n && (!src || !dst)) return HIF8_ERR_NULL;
+    void* scratch = nullptr;
+    rc = static_scratch(&scratch);
+    if (rc) return rc;
+    bool jit = d_scale_exp_in == nullptr;
+    // scaled_convert clears the two words that must start at zero before the first kernel reads them
+    return scaled_convert(false, src, dst, src_dtype, n, jit, target_exp, d_scale_exp_in, 0, rnd, flags, seed,
+                          d_amax_out, d_scale_exp_out, d_scale_out, scratch, kStaticScratchBytes, !jit,
+                          (cudaStream_t)stream);
+}
