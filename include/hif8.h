@@ -154,12 +154,21 @@ int hif8_fake_quant(const void* src, void* dst, int dtype, size_t n, int use_ama
  *   Aq: [M,K] row-major bytes, leading dimension lda.  Wq: [K,N] (w_is_nk = 0) or [N,K] (w_is_nk = 1)
  *   row-major bytes, leading dimension ldw.  C: [M,N] row-major, `c_dtype` HIF8_BF16 or HIF8_F32, ldc.
  *   d_scale_exp_a / d_scale_exp_w: device ints sa, sw (NULL = 0).
- * Pointers and leading dimensions must be multiples of 16 bytes (HIF8_ERR_ALIGN); K must be a multiple of
- * 16.  workspace: hif8_workspace_bytes(HIF8_WS_GEMM, 0) bytes (may be 0 -> NULL allowed).
+ * Pointers and leading dimensions (in bytes) must be multiples of 16 (HIF8_ERR_ALIGN); K must be a positive
+ * multiple of 16 (HIF8_ERR_SHAPE).  NaN / Inf codes propagate as in IEEE arithmetic.
+ * workspace: hif8_workspace_bytes(HIF8_WS_GEMM, 0) bytes, 16-byte aligned; its first int is a device status word
+ * that the call clears and the kernel sets if one of its bounded waits ever gives up (see hif8_gemm_status).
  */
 int hif8_gemm(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int64_t ldw, int w_is_nk, void* C,
               int64_t ldc, int c_dtype, int M, int N, int K, const int* d_scale_exp_a,
               const int* d_scale_exp_w, void* workspace, size_t workspace_bytes, hif8_stream_t stream);
+
+/*
+ * Host-side query of the status word of a finished hif8_gemm: copies it from `workspace`, SYNCHRONISES `stream`,
+ * and returns HIF8_OK or HIF8_ERR_DEVICE_TIMEOUT (the output tile of the CTA that gave up is then undefined).
+ * The only entry point that blocks the host.
+ */
+int hif8_gemm_status(const void* workspace, hif8_stream_t stream);
 
 /* bytes of device workspace a call needs (which = HIF8_WS_*; n = element count, ignored for GEMM) */
 size_t hif8_workspace_bytes(int which, size_t n);

@@ -17,7 +17,7 @@ OK = 0
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libhif8.so")
-EXPORTS = ["hif8_encode", "hif8_decode", "hif8_amax_scale_encode", "hif8_fake_quant", "hif8_gemm",
+EXPORTS = ["hif8_encode", "hif8_decode", "hif8_amax_scale_encode", "hif8_fake_quant", "hif8_gemm", "hif8_gemm_status",
            "hif8_amax_scale_encode_static", "hif8_workspace_bytes", "hif8_status_string", "hif8_launch_count"]
 
 if not os.path.exists(LIB_PATH):
@@ -32,6 +32,8 @@ lib.hif8_amax_scale_encode_static.argtypes = [_vp, _i, _vp, _sz, _i, _i, _u, _u6
 lib.hif8_amax_scale_encode_static.restype = _i
 lib.hif8_fake_quant.argtypes = [_vp, _vp, _i, _sz, _i, _i, _i, _u, _u64, _vp, _vp, _vp, _sz, _vp]
 lib.hif8_gemm.argtypes = [_vp, _i64, _vp, _i64, _i, _vp, _i64, _i, _i, _i, _i, _vp, _vp, _vp, _sz, _vp]
+lib.hif8_gemm_status.argtypes = [_vp, _vp]
+lib.hif8_gemm_status.restype = _i
 lib.hif8_workspace_bytes.argtypes = [_i, _sz]
 lib.hif8_workspace_bytes.restype = _sz
 lib.hif8_status_string.argtypes = [_i]
@@ -118,3 +120,7 @@ def hif8_gemm(Aq, lda, Wq, ldw, w_is_nk, Cmat, ldc, c_dtype, M, N, K, d_scale_ex
     return _check(lib.hif8_gemm(_ptr(Aq), lda, _ptr(Wq), ldw, w_is_nk, _ptr(Cmat), ldc, c_dtype, M, N, K,
                                 _ptr(d_scale_exp_a), _ptr(d_scale_exp_w), _ptr(workspace), workspace_bytes,
                                 _stream(stream)), check)
+
+
+def hif8_gemm_status(workspace, stream=None):
+    return int(lib.hif8_gemm_status(_ptr(workspace), _stream(stream)))

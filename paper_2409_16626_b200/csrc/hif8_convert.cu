@@ -737,6 +737,7 @@ size_t hif8_workspace_bytes(int which, size_t n)
     switch (which) {
         case HIF8_WS_AMAX_SCALE_ENCODE:
         case HIF8_WS_FAKE_QUANT: return kConvWorkspaceBytes;
+        case HIF8_WS_GEMM: return 256;
         default: return 0;
     }
 }

@@ -1,7 +1,505 @@
-// placeholder until the tcgen05 kernel lands
+// GEMM with HiF8 operands decoded in-kernel, for sm_100a (tcgen05 + TMEM + TMA).
+//
+//   C[m,n] = 2^-(sa+sw) * sum_k value(Aq[m,k]) * value(Wq[k,n])       (Algorithm 1, "MatMul & Restore")
+//
+// Every HiF8 value has at most 4 significant bits and an exponent in [-22, 15], so it is exact in BF16 and every
+// product of two of them is exact in the FP32 accumulator of the tensor core.
+//
+// One CTA computes one 128 x 256 tile of C.  Warp roles:
+//   warps 0-3  epilogue: TMEM -> registers -> descale -> BF16 / FP32 -> global
+//   warp  4    TMA producer: HiF8 byte tiles (A: 128 x 64, W: 256 x 64 or 64 x 256) into a 4-stage staging ring
+//   warp  5    MMA issuer: one elected thread issues tcgen05.mma (128 x 256 x 16, BF16 x BF16 -> FP32 in TMEM)
+//   warps 6-13 decode: staging bytes -> BF16 in the canonical 128-byte-swizzled operand layout (2-stage ring)
+// The operand layout follows the shared-memory matrix descriptor of tcgen05: K-major operands are rows of 64 BF16
+// (128 bytes), eight rows form a 1024-byte swizzle atom, 16-byte chunk j of row r is stored at chunk j ^ (r % 8).
+// W given as [K, N] is decoded in place as an MN-major operand (atoms of 8 k-rows x 64 n), so no transpose is needed.
+//
+// Every wait on an mbarrier is bounded; a wait that runs out records a status word, makes all roles leave their
+// loops, lets outstanding TMA copies land, frees TMEM and returns.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdint>
+#include <mutex>
+
 #include "hif8.h"
-extern "C" int hif8_gemm(const uint8_t*, int64_t, const uint8_t*, int64_t, int, void*, int64_t, int, int, int, int,
-                         const int*, const int*, void*, size_t, hif8_stream_t)
+
+namespace hif8 {
+extern std::atomic<uint64_t> g_launches;
+
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int kStages8 = 4;    // staging ring of HiF8 byte tiles
+constexpr int kStagesBf = 2;   // ring of decoded BF16 operand tiles
+constexpr int kEpiWarps = 4, kDecodeWarps = 8;
+constexpr int kThreads = (kEpiWarps + 2 + kDecodeWarps) * 32;  // 448
+constexpr int kTmaWarp = 4, kMmaWarp = 5, kFirstDecodeWarp = 6;
+constexpr uint32_t kA8Bytes = BM * BK, kB8Bytes = BN * BK;              // 8 KiB + 16 KiB
+constexpr uint32_t kABfBytes = BM * BK * 2, kBBfBytes = BN * BK * 2;    // 16 KiB + 32 KiB
+constexpr uint32_t kTmemCols = 256;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
+
+struct SmemLayout {
+    static constexpr uint32_t bf = 0;                                                  // 1024-byte aligned atoms
+    static constexpr uint32_t u8 = bf + kStagesBf * (kABfBytes + kBBfBytes);           // 96 KiB
+    static constexpr uint32_t lut = u8 + kStages8 * (kA8Bytes + kB8Bytes);             // + 96 KiB
+    static constexpr uint32_t bars = lut + 512;
+    static constexpr uint32_t n_bars = 2 * kStages8 + 2 * kStagesBf + 1;
+    static constexpr uint32_t tmem_slot = bars + n_bars * 8;
+    static constexpr uint32_t abort_flag = tmem_slot + 4;
+    static constexpr uint32_t total = abort_flag + 4;
+};
+constexpr uint32_t kSmemBytes = SmemLayout::total + 1024;  // slack for manual 1024-byte alignment
+
+// ---------------------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
-    return HIF8_ERR_SHAPE;
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait.  Returns false when the barrier did not complete in time or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int where)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (uint32_t it = 1;; it++) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 0) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                atomicCAS(status, 0, where);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+// D[tmem] (+)= A[smem] * B[smem], 128 x 256 x 16, BF16 inputs, FP32 accumulate
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// shared-memory matrix descriptor: start address, leading / stride byte offsets (16-byte units), version 1,
+// 128-byte swizzle
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;  // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;  // layout type: 128-byte swizzle
+    return d;
+}
+
+// BF16 bits of one HiF8 byte (Eq. 1, Eq. 2, specials); used to fill the shared lookup table
+__device__ __forceinline__ uint32_t hif8_to_bf16_bits(uint32_t c)
+{
+    uint32_t sign = (c & 0x80u) << 8, m = c & 0x7Fu;
+    if (m == 0) return sign ? 0x7FC0u : 0u;
+    if (m == 0x6F) return sign | 0x7F80u;
+    if (m < 8) return sign | ((m + 104u) << 7);
+    int E; uint32_t M, w;
+    if (m < 0x10)      { E = 0; M = m & 7; w = 3; }
+    else if (m < 0x20) { E = 1; M = m & 7; w = 3; if (m & 0x08) E = -E; }
+    else if (m < 0x40) { E = 2 | ((m >> 3) & 1); M = m & 7; w = 3; if (m & 0x10) E = -E; }
+    else if (m < 0x60) { E = 4 | ((m >> 2) & 3); M = m & 3; w = 2; if (m & 0x10) E = -E; }
+    else               { E = 8 | ((m >> 1) & 7); M = m & 1; w = 1; if (m & 0x10) E = -E; }
+    return sign | ((uint32_t)(E + 127) << 7) | (M << (7 - w));
+}
+
+// eight HiF8 bytes -> eight BF16 (one 16-byte operand chunk)
+__device__ __forceinline__ uint4 decode8(uint2 v, const unsigned short* lut)
+{
+    uint32_t o[4];
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+        uint32_t w = i < 2 ? v.x : v.y;
+        uint32_t c0 = (w >> (16 * (i & 1))) & 0xFFu, c1 = (w >> (16 * (i & 1) + 8)) & 0xFFu;
+        o[i] = (uint32_t)lut[c0] | ((uint32_t)lut[c1] << 16);
+    }
+    return make_uint4(o[0], o[1], o[2], o[3]);
+}
+
+struct GemmParams {
+    void* C;
+    long long ldc;
+    int c_is_f32;
+    int M, N, K;
+    const int* d_sa;
+    const int* d_sw;
+    int* status;
+    int tiles_m, tiles_n;
+};
+
+template <bool W_IS_NK>
+__global__ void __launch_bounds__(kThreads, 1)
+hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const GemmParams p)
+{
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* sm = smem_raw + (base - smem_u32(smem_raw));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    const uint32_t bars = base + SmemLayout::bars;
+    auto bar_u8_full = [&](int s) { return bars + 8u * s; };
+    auto bar_u8_empty = [&](int s) { return bars + 8u * (kStages8 + s); };
+    auto bar_bf_full = [&](int s) { return bars + 8u * (2 * kStages8 + s); };
+    auto bar_bf_empty = [&](int s) { return bars + 8u * (2 * kStages8 + kStagesBf + s); };
+    const uint32_t bar_acc_full = bars + 8u * (2 * kStages8 + 2 * kStagesBf);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + SmemLayout::abort_flag);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + SmemLayout::tmem_slot);
+    unsigned short* lut = reinterpret_cast<unsigned short*>(sm + SmemLayout::lut);
+
+    // tile of this CTA: groups of 8 tile-rows share their W tiles in L2
+    constexpr int kGroupM = 8;
+    const int t = blockIdx.x;
+    const int per_group = kGroupM * p.tiles_n;
+    const int g = t / per_group, first_m = g * kGroupM;
+    const int rows_in_group = min(kGroupM, p.tiles_m - first_m);
+    const int tile_m = first_m + (t % per_group) % rows_in_group;
+    const int tile_n = (t % per_group) / rows_in_group;
+    const int m0 = tile_m * BM, n0 = tile_n * BN;
+    const int num_kb = (p.K + BK - 1) / BK;
+
+    // ---- set-up
+    if (threadIdx.x < 256) lut[threadIdx.x] = (unsigned short)hif8_to_bf16_bits(threadIdx.x);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages8; s++) { mbar_init(bar_u8_full(s), 1); mbar_init(bar_u8_empty(s), kDecodeWarps); }
+        for (int s = 0; s < kStagesBf; s++) { mbar_init(bar_bf_full(s), kDecodeWarps); mbar_init(bar_bf_empty(s), 1); }
+        mbar_init(bar_acc_full, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == kMmaWarp) {  // this warp owns the TMEM allocation
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(base + SmemLayout::tmem_slot), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == kTmaWarp) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            int issued = 0;
+            for (int kb = 0; kb < num_kb; kb++) {
+                const int s = kb % kStages8, round = kb / kStages8;
+                if (round > 0 && !mbar_wait(bar_u8_empty(s), (round - 1) & 1, abort_flag, p.status, 1)) break;
+                if (*abort_flag) break;
+                const uint32_t dst_a = base + SmemLayout::u8 + s * (kA8Bytes + kB8Bytes), dst_b = dst_a + kA8Bytes;
+                mbar_arrive_expect_tx(bar_u8_full(s), kA8Bytes + kB8Bytes);
+                tma_load_2d(dst_a, &map_a, kb * BK, m0, bar_u8_full(s));
+                if (W_IS_NK) tma_load_2d(dst_b, &map_w, kb * BK, n0, bar_u8_full(s));
+                else tma_load_2d(dst_b, &map_w, n0, kb * BK, bar_u8_full(s));
+                issued = kb + 1;
+            }
+            if (*abort_flag) {
+                // let the copies already issued land before this CTA's shared memory goes away
+                for (int kb = max(0, issued - kStages8); kb < issued; kb++) {
+                    const int s = kb % kStages8;
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(bar_u8_full(s), (kb / kStages8) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+                }
+            }
+        }
+    } else if (warp == kMmaWarp) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            // instruction descriptor: FP32 accumulator, BF16 A and B, A K-major, B K- or MN-major, N, M
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((W_IS_NK ? 0u : 1u) << 16) |
+                                   ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+            bool ok = true;
+            for (int kb = 0; kb < num_kb && ok; kb++) {
+                const int s = kb % kStagesBf, round = kb / kStagesBf;
+                ok = mbar_wait(bar_bf_full(s), round & 1, abort_flag, p.status, 2);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a_addr = base + SmemLayout::bf + s * (kABfBytes + kBBfBytes), b_addr = a_addr + kABfBytes;
+#pragma unroll
+                for (int kk = 0; kk < BK / 16; kk++) {
+                    // K-major: 16 k = 32 bytes inside the 128-byte row; MN-major: 16 k = two 1024-byte atoms
+                    const uint64_t da = make_smem_desc(a_addr + kk * 32, 16, 1024);
+                    const uint64_t db = W_IS_NK ? make_smem_desc(b_addr + kk * 32, 16, 1024)
+                                                : make_smem_desc(b_addr + kk * 2048, 8192, 1024);
+                    tc_mma_bf16(tmem_base, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+                }
+                tc_commit(bar_bf_empty(s));  // frees this operand stage once the MMAs above have read it
+            }
+            if (ok) tc_commit(bar_acc_full);
+        }
+    } else if (warp >= kFirstDecodeWarp) {
+        // ------------------------------------------------------------------ decode warps
+        const int dt = threadIdx.x - kFirstDecodeWarp * 32;  // 0..255
+        bool ok = true;
+        for (int kb = 0; kb < num_kb && ok; kb++) {
+            const int s8 = kb % kStages8, r8 = kb / kStages8, sb = kb % kStagesBf, rb = kb / kStagesBf;
+            ok = mbar_wait(bar_u8_full(s8), r8 & 1, abort_flag, p.status, 3);
+            if (ok && rb > 0) ok = mbar_wait(bar_bf_empty(sb), (rb - 1) & 1, abort_flag, p.status, 4);
+            if (!ok) break;
+            const unsigned char* a8 = sm + SmemLayout::u8 + s8 * (kA8Bytes + kB8Bytes);
+            const unsigned char* b8 = a8 + kA8Bytes;
+            unsigned char* abf = sm + SmemLayout::bf + sb * (kABfBytes + kBBfBytes);
+            unsigned char* bbf = abf + kABfBytes;
+            // A: 128 rows x 8 chunks of 8 codes; chunk j of row r -> atom r/8, row r%8, chunk j ^ (r%8)
+#pragma unroll
+            for (int it = 0; it < (BM * BK / 8) / 256; it++) {
+                const int q = it * 256 + dt, r = q >> 3, j = q & 7;
+                const uint2 v = *reinterpret_cast<const uint2*>(a8 + r * BK + j * 8);
+                *reinterpret_cast<uint4*>(abf + (r >> 3) * 1024 + (r & 7) * 128 + ((j ^ (r & 7)) << 4)) = decode8(v, lut);
+            }
+            if (W_IS_NK) {
+#pragma unroll
+                for (int it = 0; it < (BN * BK / 8) / 256; it++) {
+                    const int q = it * 256 + dt, r = q >> 3, j = q & 7;
+                    const uint2 v = *reinterpret_cast<const uint2*>(b8 + r * BK + j * 8);
+                    *reinterpret_cast<uint4*>(bbf + (r >> 3) * 1024 + (r & 7) * 128 + ((j ^ (r & 7)) << 4)) = decode8(v, lut);
+                }
+            } else {
+                // W tile is [64 k][256 n]: chunk (k, n/8) -> atom (n/64) * 8 + k/8, row k%8, chunk (n/8)%8 ^ (k%8)
+#pragma unroll
+                for (int it = 0; it < (BN * BK / 8) / 256; it++) {
+                    const int q = it * 256 + dt, k = q >> 5, jn = q & 31;
+                    const uint2 v = *reinterpret_cast<const uint2*>(b8 + k * BN + jn * 8);
+                    const int atom = (jn >> 3) * 8 + (k >> 3);
+                    *reinterpret_cast<uint4*>(bbf + atom * 1024 + (k & 7) * 128 + (((jn & 7) ^ (k & 7)) << 4)) = decode8(v, lut);
+                }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // make the stores visible to the tensor core
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(bar_u8_empty(s8));
+                mbar_arrive(bar_bf_full(sb));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue warps 0-3
+        const bool ok = mbar_wait(bar_acc_full, 0, abort_flag, p.status, 5);
+        if (ok) {
+            tc_fence_after();
+            const int s = -((p.d_sa ? *p.d_sa : 0) + (p.d_sw ? *p.d_sw : 0));
+            const int s1 = s / 2, s2 = s - s1;  // |s1|, |s2| <= 126: two exact power-of-two factors
+            const float f1 = __uint_as_float((uint32_t)(s1 + 127) << 23), f2 = __uint_as_float((uint32_t)(s2 + 127) << 23);
+            const int row = m0 + warp * 32 + lane;
+#pragma unroll 1
+            for (int c = 0; c < BN; c += 32) {
+                uint32_t r[32];
+                tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(warp * 32) << 16) + c, r);
+                tmem_ld_wait();
+                const int col = n0 + c;
+                if (row < p.M && col < p.N) {
+                    const bool full = col + 32 <= p.N;
+                    if (p.c_is_f32) {
+                        float* out = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + col;
+                        if (full) {
+#pragma unroll
+                            for (int i = 0; i < 32; i += 4)
+                                *reinterpret_cast<float4*>(out + i) =
+                                    make_float4(__uint_as_float(r[i]) * f1 * f2, __uint_as_float(r[i + 1]) * f1 * f2,
+                                                __uint_as_float(r[i + 2]) * f1 * f2, __uint_as_float(r[i + 3]) * f1 * f2);
+                        } else {
+                            for (int i = 0; i < 32 && col + i < p.N; i++) out[i] = __uint_as_float(r[i]) * f1 * f2;
+                        }
+                    } else {
+                        unsigned short* out = reinterpret_cast<unsigned short*>(p.C) + (long long)row * p.ldc + col;
+                        uint32_t h[32];
+#pragma unroll
+                        for (int i = 0; i < 32; i++) {
+                            float v = __uint_as_float(r[i]) * f1 * f2;
+                            uint32_t u = __float_as_uint(v);
+                            h[i] = (v != v) ? 0x7FC0u : ((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);  // round to nearest even
+                        }
+                        if (full) {
+#pragma unroll
+                            for (int i = 0; i < 32; i += 8)
+                                *reinterpret_cast<uint4*>(out + i) =
+                                    make_uint4(h[i] | (h[i + 1] << 16), h[i + 2] | (h[i + 3] << 16),
+                                               h[i + 4] | (h[i + 5] << 16), h[i + 6] | (h[i + 7] << 16));
+                        } else {
+                            for (int i = 0; i < 32 && col + i < p.N; i++) out[i] = (unsigned short)h[i];
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    // ---- teardown: everybody arrives here (all waits are bounded), then the allocating warp frees TMEM
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kMmaWarp) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    });
+    return fn;
+}
+
+// 2-D byte tensor [rows][ld] with a box of box_inner x box_rows bytes, no swizzle, zero fill out of bounds
+bool make_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t rows, uint64_t ld, uint32_t box_inner, uint32_t box_rows)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {inner, rows};
+    cuuint64_t strides[1] = {ld};
+    cuuint32_t box[2] = {box_inner, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+constexpr size_t kGemmWorkspaceBytes = 256;
+
+}  // namespace
+
+size_t gemm_workspace_bytes() { return kGemmWorkspaceBytes; }
+
+}  // namespace hif8
+
+using namespace hif8;
+
+extern "C" int hif8_gemm(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int64_t ldw, int w_is_nk, void* C, int64_t ldc,
+                         int c_dtype, int M, int N, int K, const int* d_scale_exp_a, const int* d_scale_exp_w,
+                         void* workspace, size_t workspace_bytes, hif8_stream_t stream)
+{
+    if (c_dtype != HIF8_BF16 && c_dtype != HIF8_F32) return HIF8_ERR_DTYPE;
+    if (M < 0 || N < 0 || K < 0 || (K & 15)) return HIF8_ERR_SHAPE;
+    if (lda < K || ldc < N || ldw < (w_is_nk ? K : N)) return HIF8_ERR_SHAPE;
+    if (M == 0 || N == 0) return HIF8_OK;
+    if (!Aq || !Wq || !C) return HIF8_ERR_NULL;
+    const size_t c_item = c_dtype == HIF8_F32 ? 4 : 2;
+    if ((reinterpret_cast<uintptr_t>(Aq) & 15) || (reinterpret_cast<uintptr_t>(Wq) & 15) || (reinterpret_cast<uintptr_t>(C) & 15) ||
+        (lda & 15) || (ldw & 15) || ((ldc * c_item) & 15))
+        return HIF8_ERR_ALIGN;
+    if (!workspace || workspace_bytes < kGemmWorkspaceBytes || (reinterpret_cast<uintptr_t>(workspace) & 15))
+        return HIF8_ERR_WORKSPACE;
+    if (K == 0) return HIF8_ERR_SHAPE;
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return HIF8_ERR_CUDA;
+    cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (major != 10) return HIF8_ERR_CUDA;
+
+    CUtensorMap map_a, map_w;
+    if (!make_map(&map_a, Aq, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BK, BM)) return HIF8_ERR_CUDA;
+    const bool ok_w = w_is_nk ? make_map(&map_w, Wq, (uint64_t)K, (uint64_t)N, (uint64_t)ldw, BK, BN)
+                              : make_map(&map_w, Wq, (uint64_t)N, (uint64_t)K, (uint64_t)ldw, BN, BK);
+    if (!ok_w) return HIF8_ERR_CUDA;
+
+    GemmParams p{};
+    p.C = C; p.ldc = ldc; p.c_is_f32 = c_dtype == HIF8_F32; p.M = M; p.N = N; p.K = K;
+    p.d_sa = d_scale_exp_a; p.d_sw = d_scale_exp_w; p.status = reinterpret_cast<int*>(workspace);
+    p.tiles_m = (M + BM - 1) / BM; p.tiles_n = (N + BN - 1) / BN;
+    const long long tiles = (long long)p.tiles_m * p.tiles_n;
+    if (tiles > 0x7FFFFFFF) return HIF8_ERR_SHAPE;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemsetAsync(workspace, 0, 4, st) != cudaSuccess) return HIF8_ERR_CUDA;
+
+    static std::once_flag attr_once;
+    static cudaError_t attr_rc = cudaSuccess;
+    std::call_once(attr_once, [] {
+        attr_rc = cudaFuncSetAttribute(hif8_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (attr_rc == cudaSuccess)
+            attr_rc = cudaFuncSetAttribute(hif8_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+    });
+    if (attr_rc != cudaSuccess) return HIF8_ERR_CUDA;
+    if (w_is_nk) hif8_gemm_kernel<true><<<(unsigned)tiles, kThreads, kSmemBytes, st>>>(map_a, map_w, p);
+    else hif8_gemm_kernel<false><<<(unsigned)tiles, kThreads, kSmemBytes, st>>>(map_a, map_w, p);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
+}
+
+extern "C" int hif8_gemm_status(const void* workspace, hif8_stream_t stream)
+{
+    if (!workspace) return HIF8_ERR_NULL;
+    int v = 0;
+    if (cudaMemcpyAsync(&v, workspace, sizeof v, cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess) return HIF8_ERR_CUDA;
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return HIF8_ERR_CUDA;
+    return v == 0 ? HIF8_OK : HIF8_ERR_DEVICE_TIMEOUT;
 }

@@ -46,3 +46,18 @@ def test_argument_errors_before_any_launch():
     assert H.hif8_fake_quant(0, 0, H.BF16, 16, use_amax=1, scale_or_target_exp=14, stream=0, check=False) == 8
     assert H.hif8_fake_quant(0, 0, H.BF16, 16, use_amax=0, scale_or_target_exp=200, stream=0, check=False) == 5
     assert H.hif8_launch_count() == before
+
+
+def test_gemm_argument_errors_before_any_launch():
+    before = H.hif8_launch_count()
+    g = lambda **kw: H.hif8_gemm(kw.get("A", 16), kw.get("lda", 64), kw.get("W", 16), kw.get("ldw", 64), 0, kw.get("C", 16),
+                                 kw.get("ldc", 64), kw.get("cdt", H.F32), kw.get("M", 64), kw.get("N", 64), kw.get("K", 64),
+                                 None, None, kw.get("ws", 256), kw.get("wsb", 256), stream=0, check=False)
+    assert g(cdt=H.F16) == 2
+    assert g(K=40) == 6 and g(K=0) == 6 and g(M=-1) == 6 and g(lda=32) == 6 and g(ldc=32) == 6
+    assert g(A=0) == 1
+    assert g(A=24) == 7 and g(ldw=72) == 7 and g(ldc=66) == 7
+    assert g(ws=0) == 8 and g(wsb=8) == 8
+    assert g(M=0) == 0
+    assert H.hif8_workspace_bytes(H.WS_GEMM) == 256
+    assert H.hif8_launch_count() == before

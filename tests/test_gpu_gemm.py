@@ -1,0 +1,123 @@
+"""GPU parity of hif8_gemm (through the C ABI) against the FP64 oracle.
+
+Tolerance (per output, from the method's statement): FP32 output |C - C*| <= 1e-5 * S with
+S = 2^-(sa+sw) * sum_k |a_k w_k|; BF16 output additionally gets the BF16 unit roundoff (8-bit significand:
+half an ulp is at most 2^-8 * |C*|).
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2409_16626_b200 as H
+import workloads as W
+from oracle import hif8_oracle as O
+
+from gpu_util import to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def run_gemm(Aq, Wq, w_is_nk, c_dtype, sa=None, sw=None, M=None, N=None, K=None, lda=None, ldw=None):
+    M = Aq.shape[0] if M is None else M
+    K = Aq.shape[1] if K is None else K
+    N = (Wq.shape[0] if w_is_nk else Wq.shape[1]) if N is None else N
+    dA, dW = to_dev(Aq), to_dev(Wq)
+    ldc = (N + 7) // 8 * 8
+    C = torch.full((M, ldc), float("nan"), dtype=torch.float32 if c_dtype == H.F32 else torch.bfloat16, device="cuda")
+    ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+    dsa = torch.tensor([sa], dtype=torch.int32, device="cuda") if sa is not None else None
+    dsw = torch.tensor([sw], dtype=torch.int32, device="cuda") if sw is not None else None
+    H.hif8_gemm(dA, Aq.shape[1] if lda is None else lda, dW, Wq.shape[1] if ldw is None else ldw, int(w_is_nk), C, ldc,
+                c_dtype, M, N, K, dsa, dsw, ws, 256)
+    assert H.hif8_gemm_status(ws) == 0
+    out = C.float().cpu().numpy().astype(np.float64)
+    assert np.all(np.isnan(out[:, N:]))                      # padding columns untouched
+    return out[:, :N]
+
+
+def check(C, Cstar, S, c_dtype):
+    tol = 1e-5 * S + (2.0 ** -8 * np.abs(Cstar) if c_dtype == H.BF16 else 0.0)
+    err = np.abs(C - Cstar)
+    bad = err > tol
+    assert not bad.any(), f"{bad.sum()} of {bad.size} outside tolerance; worst ratio {np.max(err / np.maximum(tol, 1e-300)):.3g}"
+
+
+@pytest.mark.parametrize("w_is_nk", [0, 1])
+@pytest.mark.parametrize("c_dtype", [H.F32, H.BF16])
+@pytest.mark.parametrize("shape", [(128, 256, 64), (128, 256, 256), (256, 512, 192), (130, 264, 208), (77, 40, 16),
+                                   (300, 1000, 1040)])
+def test_gemm_small_full_compare(shape, c_dtype, w_is_nk):
+    M, N, K = shape
+    Aq = W.random_codes((M, K), seed=M + K)
+    Wkn = W.random_codes((K, N), seed=N + K + 1)
+    Wq = np.ascontiguousarray(Wkn.T) if w_is_nk else Wkn
+    if (Wq.shape[1] % 16) != 0:                              # leading dimension must be a multiple of 16 bytes
+        pad = 16 - Wq.shape[1] % 16
+        Wq = np.ascontiguousarray(np.pad(Wq, ((0, 0), (0, pad))))
+    Cs, S = O.gemm_full(Aq, Wkn, False, 0, 0)
+    C = run_gemm(Aq, Wq, w_is_nk, c_dtype, N=N)
+    check(C, Cs, S, c_dtype)
+
+
+@pytest.mark.parametrize("w_is_nk", [0, 1])
+def test_gemm_one_hot_rows_pin_tile_and_k_indexing(w_is_nk):
+    # A picks one k per row (value 1.0): C[m, :] must equal row perm[m] of W exactly
+    M, N, K = 384, 768, 512
+    rng = np.random.default_rng(5)
+    perm = rng.integers(0, K, M)
+    Aq = np.zeros((M, K), dtype=np.uint8)
+    Aq[np.arange(M), perm] = 0x08
+    Wkn = W.random_codes((K, N), seed=9)
+    tab = np.array([O.value(c) for c in range(256)])
+    C = run_gemm(Aq, np.ascontiguousarray(Wkn.T) if w_is_nk else Wkn, w_is_nk, H.F32)
+    assert np.array_equal(C, tab[Wkn][perm, :])
+    # and the mirror: W picks one k per column
+    permn = rng.integers(0, K, N)
+    Wsel = np.zeros((K, N), dtype=np.uint8)
+    Wsel[permn, np.arange(N)] = 0x90                          # -2.0
+    Aq2 = W.random_codes((M, K), seed=10)
+    C = run_gemm(Aq2, np.ascontiguousarray(Wsel.T) if w_is_nk else Wsel, w_is_nk, H.F32)
+    assert np.array_equal(C, -2.0 * tab[Aq2][:, permn])
+
+
+def test_gemm_small_integers_exact_and_descale():
+    M, N, K = 256, 256, 1024
+    ints = np.array([0x00, 0x08, 0x10, 0x14, 0x20, 0x88, 0x90, 0x94], dtype=np.uint8)   # 0, 1, 2, 3, 4, -1, -2, -3
+    rng = np.random.default_rng(3)
+    Aq = ints[rng.integers(0, len(ints), (M, K))]
+    Wq = ints[rng.integers(0, len(ints), (K, N))]
+    tab = np.array([O.value(c) for c in range(256)])
+    want = (tab[Aq].astype(np.int64) @ tab[Wq].astype(np.int64)).astype(np.float64)
+    assert np.array_equal(run_gemm(Aq, Wq, 0, H.F32), want)
+    assert np.array_equal(run_gemm(Aq, Wq, 0, H.F32, sa=3, sw=-1), want / 4.0)
+    assert np.array_equal(run_gemm(Aq, Wq, 0, H.F32, sa=60, sw=55), want * 2.0 ** -115)
+
+
+def test_gemm_specials_propagate():
+    M, N, K = 128, 256, 64
+    Aq = np.full((M, K), 0x08, dtype=np.uint8)
+    Wq = np.full((K, N), 0x08, dtype=np.uint8)
+    Aq[3, 5] = 0x80                                           # NaN
+    Aq[7, 9] = 0x6F                                           # +Inf
+    C = run_gemm(Aq, Wq, 0, H.F32)
+    assert np.all(np.isnan(C[3])) and np.all(np.isposinf(C[7]))
+    ok = np.ones(M, bool); ok[[3, 7]] = False
+    assert np.all(C[ok] == K)
+
+
+@pytest.mark.parametrize("w_is_nk", [0, 1])
+def test_gemm_medium_scaled_operands_sampled(w_is_nk):
+    # operands produced the way the method uses them: BF16 tensors, per-tensor scaled, encoded on the device
+    M, N, K = 1024, 1536, 4096
+    a = W.normal_bf16((M, K), seed=4567)
+    w = W.normal_bf16((K, N), seed=5678, std=0.02)
+    sa, sw = O.amax_scale(a, O.BF16, 14)[1], O.amax_scale(w, O.BF16, 14)[1]
+    Aq = O.encode(a, O.BF16, sa, O.TA, 0, quick=True)
+    Wkn = O.encode(w, O.BF16, sw, O.TA, 0, quick=True)
+    rng = np.random.default_rng(1)
+    rows = np.concatenate([rng.integers(0, M, 20000), np.repeat(np.arange(128), 256), np.repeat(np.arange(M - 128, M), 256)])
+    cols = np.concatenate([rng.integers(0, N, 20000), np.tile(np.arange(256), 128), np.tile(np.arange(N - 256, N), 128)])
+    Cs, S = O.gemm_entries(Aq, Wkn, False, sa, sw, rows, cols)
+    for c_dtype in (H.F32, H.BF16):
+        C = run_gemm(Aq, np.ascontiguousarray(Wkn.T) if w_is_nk else Wkn, w_is_nk, c_dtype, sa=sa, sw=sw)
+        check(C[rows, cols], Cs, S, c_dtype)
