@@ -156,8 +156,12 @@ int hif8_fake_quant(const void* src, void* dst, int dtype, size_t n, int use_ama
  *   d_scale_exp_a / d_scale_exp_w: device ints sa, sw (NULL = 0).
  * Pointers and leading dimensions (in bytes) must be multiples of 16 (HIF8_ERR_ALIGN); K must be a positive
  * multiple of 16 (HIF8_ERR_SHAPE).  NaN / Inf codes propagate as in IEEE arithmetic.
- * workspace: hif8_workspace_bytes(HIF8_WS_GEMM, 0) bytes, 16-byte aligned; its first int is a device status word
- * that the call clears and the kernel sets if one of its bounded waits ever gives up (see hif8_gemm_status).
+ * workspace: at least hif8_workspace_bytes(HIF8_WS_GEMM, 0) = 256 bytes, 16-byte aligned; its first int is a device
+ * status word that the call clears and the kernel sets if one of its bounded waits ever gives up (see
+ * hif8_gemm_status).  With only that, the fused kernel decodes the HiF8 tiles of every CTA in shared memory.
+ * With hif8_workspace_bytes(HIF8_WS_GEMM, M*K + K*N) bytes, 256-byte aligned, and contiguous operands (lda = K,
+ * ldw = row length of Wq), each operand byte is instead decoded once into the workspace (BF16, exact) and the
+ * tensor-core kernel streams BF16 tiles: several times faster for compute-bound shapes, same results.
  */
 int hif8_gemm(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int64_t ldw, int w_is_nk, void* C,
               int64_t ldc, int c_dtype, int M, int N, int K, const int* d_scale_exp_a,
@@ -170,7 +174,8 @@ int hif8_gemm(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int64_t ldw, in
  */
 int hif8_gemm_status(const void* workspace, hif8_stream_t stream);
 
-/* bytes of device workspace a call needs (which = HIF8_WS_*; n = element count, ignored for GEMM) */
+/* bytes of device workspace a call needs (which = HIF8_WS_*; n = element count; for HIF8_WS_GEMM: 0 for the
+ * minimum, or M*K + K*N for the decode-once path) */
 size_t hif8_workspace_bytes(int which, size_t n);
 
 /* static, NUL-terminated description of a status code */

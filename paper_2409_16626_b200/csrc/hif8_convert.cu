@@ -733,11 +733,10 @@ int hif8_fake_quant(const void* src, void* dst, int dtype, size_t n, int use_ama
 
 size_t hif8_workspace_bytes(int which, size_t n)
 {
-    (void)n;
     switch (which) {
         case HIF8_WS_AMAX_SCALE_ENCODE:
         case HIF8_WS_FAKE_QUANT: return kConvWorkspaceBytes;
-        case HIF8_WS_GEMM: return 256;
+        case HIF8_WS_GEMM: return n ? 256 + 512 + 2 * n : 256;  // status word (+ both operands as BF16)
         default: return 0;
     }
 }

@@ -2,6 +2,11 @@
 //
 //   C[m,n] = 2^-(sa+sw) * sum_k value(Aq[m,k]) * value(Wq[k,n])       (Algorithm 1, "MatMul & Restore")
 //
+// Two paths behind one entry point.  The fused kernel (described next) needs no memory beyond its operands and
+// decodes the byte tiles of every CTA in shared memory; because every operand element is then decoded once per
+// tile that uses it, it is bound by the decode rate.  With a workspace large enough for both operands in BF16 the
+// call decodes each byte once (conversion kernel) and runs the BF16 tensor-core kernel further down.
+//
 // Every HiF8 value has at most 4 significant bits and an exponent in [-22, 15], so it is exact in BF16 and every
 // product of two of them is exact in the FP32 accumulator of the tensor core.
 //
@@ -401,6 +406,201 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 }
 
 // ---------------------------------------------------------------------------------------------------------
+// Decode-once path: operands already decoded to BF16 (by the conversion kernel of this library, into the caller's
+// workspace).  Persistent kernel, one CTA per SM, 128 x 256 tiles, 64-wide k-blocks.
+//   warps 0-3  epilogue (TMEM -> global), overlapped with the next tile through two TMEM accumulators
+//   warp  4    TMA producer: BF16 tiles land directly in the 128-byte-swizzled operand layout (4-stage ring)
+//   warp  5    MMA issuer
+// ---------------------------------------------------------------------------------------------------------
+constexpr int kStagesP = 4;
+constexpr int kThreadsP = 6 * 32;
+constexpr uint32_t kStageBytesP = kABfBytes + kBBfBytes;  // 48 KiB
+struct SmemLayoutP {
+    static constexpr uint32_t ops = 0;
+    static constexpr uint32_t bars = kStagesP * kStageBytesP;           // 192 KiB
+    static constexpr uint32_t n_bars = 2 * kStagesP + 4;
+    static constexpr uint32_t tmem_slot = bars + n_bars * 8;
+    static constexpr uint32_t abort_flag = tmem_slot + 4;
+    static constexpr uint32_t total = abort_flag + 4;
+};
+constexpr uint32_t kSmemBytesP = SmemLayoutP::total + 1024;
+
+__device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int& tile_m, int& tile_n)
+{
+    constexpr int kGroupM = 8;  // groups of 8 tile-rows sweep N together: their W tiles stay in L2
+    const int per_group = kGroupM * tiles_n;
+    const int g = t / per_group, first_m = g * kGroupM;
+    const int rows_in_group = min(kGroupM, tiles_m - first_m);
+    tile_m = first_m + (t % per_group) % rows_in_group;
+    tile_n = (t % per_group) / rows_in_group;
+}
+
+template <bool W_IS_NK>
+__global__ void __launch_bounds__(kThreadsP, 1)
+bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const GemmParams p)
+{
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* sm = smem_raw + (base - smem_u32(smem_raw));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t bars = base + SmemLayoutP::bars;
+    auto bar_full = [&](int s) { return bars + 8u * s; };
+    auto bar_empty = [&](int s) { return bars + 8u * (kStagesP + s); };
+    auto bar_acc_full = [&](int a) { return bars + 8u * (2 * kStagesP + a); };
+    auto bar_acc_empty = [&](int a) { return bars + 8u * (2 * kStagesP + 2 + a); };
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + SmemLayoutP::abort_flag);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + SmemLayoutP::tmem_slot);
+    const int num_kb = (p.K + BK - 1) / BK;
+    const int tiles = p.tiles_m * p.tiles_n;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStagesP; s++) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
+        for (int a = 0; a < 2; a++) { mbar_init(bar_acc_full(a), 1); mbar_init(bar_acc_empty(a), kEpiWarps); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == kMmaWarp) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(base + SmemLayoutP::tmem_slot), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == kTmaWarp) {
+        if (lane == 0) {
+            long long it = 0, issued = 0;  // running k-block counter over all tiles of this CTA
+            bool ok = true;
+            for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x) {
+                int tile_m, tile_n;
+                tile_coords(t, p.tiles_m, p.tiles_n, tile_m, tile_n);
+                const int m0 = tile_m * BM, n0 = tile_n * BN;
+                for (int kb = 0; kb < num_kb; kb++, it++) {
+                    const int s = (int)(it % kStagesP);
+                    const long long round = it / kStagesP;
+                    if (round > 0) ok = mbar_wait(bar_empty(s), (uint32_t)((round - 1) & 1), abort_flag, p.status, 11);
+                    if (!ok || *abort_flag) { ok = false; break; }
+                    const uint32_t dst_a = base + s * kStageBytesP, dst_b = dst_a + kABfBytes;
+                    mbar_arrive_expect_tx(bar_full(s), kStageBytesP);
+                    tma_load_2d(dst_a, &map_a, kb * BK, m0, bar_full(s));
+                    if (W_IS_NK) tma_load_2d(dst_b, &map_w, kb * BK, n0, bar_full(s));
+                    else {
+#pragma unroll
+                        for (int c = 0; c < BN / 64; c++)  // four boxes of 64 k x 64 n: one 8-atom column each
+                            tma_load_2d(dst_b + c * 8192, &map_w, n0 + c * 64, kb * BK, bar_full(s));
+                    }
+                    issued = it + 1;
+                }
+            }
+            if (*abort_flag) {
+                for (long long j = issued > kStagesP ? issued - kStagesP : 0; j < issued; j++) {
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(bar_full((int)(j % kStagesP)), (uint32_t)((j / kStagesP) & 1)) &&
+                           global_ns() - t0 < kWaitLimitNs) {}
+                }
+            }
+        }
+    } else if (warp == kMmaWarp) {
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((W_IS_NK ? 0u : 1u) << 16) |
+                                   ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+            long long it = 0;
+            int local = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x, local++) {
+                const int acc = local & 1, use = local >> 1;
+                if (use > 0) ok = mbar_wait(bar_acc_empty(acc), (uint32_t)((use - 1) & 1), abort_flag, p.status, 12);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * 256;
+                for (int kb = 0; kb < num_kb; kb++, it++) {
+                    const int s = (int)(it % kStagesP);
+                    ok = mbar_wait(bar_full(s), (uint32_t)((it / kStagesP) & 1), abort_flag, p.status, 13);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a_addr = base + s * kStageBytesP, b_addr = a_addr + kABfBytes;
+#pragma unroll
+                    for (int kk = 0; kk < BK / 16; kk++) {
+                        const uint64_t da = make_smem_desc(a_addr + kk * 32, 16, 1024);
+                        const uint64_t db = W_IS_NK ? make_smem_desc(b_addr + kk * 32, 16, 1024)
+                                                    : make_smem_desc(b_addr + kk * 2048, 8192, 1024);
+                        tc_mma_bf16(d_tmem, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    tc_commit(bar_empty(s));
+                }
+                if (ok) tc_commit(bar_acc_full(acc));
+            }
+        }
+    } else if (warp < kEpiWarps) {
+        const int s = -((p.d_sa ? *p.d_sa : 0) + (p.d_sw ? *p.d_sw : 0));
+        const int s1 = s / 2, s2 = s - s1;
+        const float f1 = __uint_as_float((uint32_t)(s1 + 127) << 23), f2 = __uint_as_float((uint32_t)(s2 + 127) << 23);
+        int local = 0;
+        for (int t = blockIdx.x; t < tiles; t += gridDim.x, local++) {
+            const int acc = local & 1, use = local >> 1;
+            if (!mbar_wait(bar_acc_full(acc), (uint32_t)(use & 1), abort_flag, p.status, 14)) break;
+            tc_fence_after();
+            int tile_m, tile_n;
+            tile_coords(t, p.tiles_m, p.tiles_n, tile_m, tile_n);
+            const int row = tile_m * BM + warp * 32 + lane, n0 = tile_n * BN;
+#pragma unroll 1
+            for (int c = 0; c < BN; c += 32) {
+                uint32_t r[32];
+                tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(warp * 32) << 16) + acc * 256 + c, r);
+                tmem_ld_wait();
+                const int col = n0 + c;
+                if (row < p.M && col < p.N) {
+                    const bool full = col + 32 <= p.N;
+                    if (p.c_is_f32) {
+                        float* out = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + col;
+                        if (full) {
+#pragma unroll
+                            for (int i = 0; i < 32; i += 4)
+                                *reinterpret_cast<float4*>(out + i) =
+                                    make_float4(__uint_as_float(r[i]) * f1 * f2, __uint_as_float(r[i + 1]) * f1 * f2,
+                                                __uint_as_float(r[i + 2]) * f1 * f2, __uint_as_float(r[i + 3]) * f1 * f2);
+                        } else {
+                            for (int i = 0; i < 32 && col + i < p.N; i++) out[i] = __uint_as_float(r[i]) * f1 * f2;
+                        }
+                    } else {
+                        unsigned short* out = reinterpret_cast<unsigned short*>(p.C) + (long long)row * p.ldc + col;
+                        uint32_t h[32];
+#pragma unroll
+                        for (int i = 0; i < 32; i++) {
+                            float v = __uint_as_float(r[i]) * f1 * f2;
+                            uint32_t u = __float_as_uint(v);
+                            h[i] = (v != v) ? 0x7FC0u : ((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);
+                        }
+                        if (full) {
+#pragma unroll
+                            for (int i = 0; i < 32; i += 8)
+                                *reinterpret_cast<uint4*>(out + i) =
+                                    make_uint4(h[i] | (h[i + 1] << 16), h[i + 2] | (h[i + 3] << 16),
+                                               h[i + 4] | (h[i + 5] << 16), h[i + 6] | (h[i + 7] << 16));
+                        } else {
+                            for (int i = 0; i < 32 && col + i < p.N; i++) out[i] = (unsigned short)h[i];
+                        }
+                    }
+                }
+            }
+            // this accumulator may be overwritten by the tile after next
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_acc_empty(acc));
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kMmaWarp) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------------------
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -421,18 +621,20 @@ EncodeTiledFn encode_tiled_fn()
     return fn;
 }
 
-// 2-D byte tensor [rows][ld] with a box of box_inner x box_rows bytes, no swizzle, zero fill out of bounds
-bool make_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t rows, uint64_t ld, uint32_t box_inner, uint32_t box_rows)
+// 2-D tensor [rows][ld elements] with a box of box_inner x box_rows elements, zero fill out of bounds.
+// bf16 = false: bytes, no swizzle.  bf16 = true: 16-bit elements, 128-byte swizzle (box_inner must be 64).
+bool make_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t rows, uint64_t ld, uint32_t box_inner, uint32_t box_rows,
+              bool bf16 = false)
 {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     cuuint64_t dims[2] = {inner, rows};
-    cuuint64_t strides[1] = {ld};
+    cuuint64_t strides[1] = {ld * (bf16 ? 2u : 1u)};
     cuuint32_t box[2] = {box_inner, box_rows};
     cuuint32_t estr[2] = {1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    return fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims,
+              strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, bf16 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 constexpr size_t kGemmWorkspaceBytes = 256;
@@ -483,12 +685,42 @@ extern "C" int hif8_gemm(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int6
 
     static std::once_flag attr_once;
     static cudaError_t attr_rc = cudaSuccess;
-    std::call_once(attr_once, [] {
+    static int sm_count = 0;
+    std::call_once(attr_once, [dev] {
         attr_rc = cudaFuncSetAttribute(hif8_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (attr_rc == cudaSuccess)
             attr_rc = cudaFuncSetAttribute(hif8_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (attr_rc == cudaSuccess)
+            attr_rc = cudaFuncSetAttribute(bf16_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytesP);
+        if (attr_rc == cudaSuccess)
+            attr_rc = cudaFuncSetAttribute(bf16_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytesP);
+        if (attr_rc == cudaSuccess) attr_rc = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
     });
-    if (attr_rc != cudaSuccess) return HIF8_ERR_CUDA;
+    if (attr_rc != cudaSuccess || sm_count <= 0) return HIF8_ERR_CUDA;
+
+    // Decode-once path: with room for both operands as BF16 in the workspace (and contiguous operands), each HiF8
+    // byte is decoded exactly once by the conversion kernel and the tensor-core kernel reads BF16 tiles through TMA.
+    // Otherwise the fused kernel decodes the byte tiles of every CTA in shared memory.
+    const size_t bytes_a = (((size_t)M * K * 2) + 255) & ~(size_t)255, bytes_w = (((size_t)K * N * 2) + 255) & ~(size_t)255;
+    const bool contiguous = lda == K && ldw == (w_is_nk ? K : N);
+    if (contiguous && workspace_bytes >= kGemmWorkspaceBytes + bytes_a + bytes_w && !(reinterpret_cast<uintptr_t>(workspace) & 255)) {
+        unsigned char* a_bf = reinterpret_cast<unsigned char*>(workspace) + kGemmWorkspaceBytes;
+        unsigned char* w_bf = a_bf + bytes_a;
+        int rc = hif8_decode(Aq, a_bf, HIF8_BF16, (size_t)M * K, 0, stream);
+        if (rc == HIF8_OK) rc = hif8_decode(Wq, w_bf, HIF8_BF16, (size_t)K * N, 0, stream);
+        if (rc != HIF8_OK) return rc;
+        CUtensorMap ma, mw;
+        if (!make_map(&ma, a_bf, (uint64_t)K, (uint64_t)M, (uint64_t)K, BK, BM, true)) return HIF8_ERR_CUDA;
+        const bool okw = w_is_nk ? make_map(&mw, w_bf, (uint64_t)K, (uint64_t)N, (uint64_t)K, BK, BN, true)
+                                 : make_map(&mw, w_bf, (uint64_t)N, (uint64_t)K, (uint64_t)N, 64, BK, true);
+        if (!okw) return HIF8_ERR_CUDA;
+        const unsigned grid = (unsigned)(tiles < sm_count ? tiles : sm_count);
+        if (w_is_nk) bf16_gemm_kernel<true><<<grid, kThreadsP, kSmemBytesP, st>>>(ma, mw, p);
+        else bf16_gemm_kernel<false><<<grid, kThreadsP, kSmemBytesP, st>>>(ma, mw, p);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
+    }
+
     if (w_is_nk) hif8_gemm_kernel<true><<<(unsigned)tiles, kThreads, kSmemBytes, st>>>(map_a, map_w, p);
     else hif8_gemm_kernel<false><<<(unsigned)tiles, kThreads, kSmemBytes, st>>>(map_a, map_w, p);
     g_launches.fetch_add(1, std::memory_order_relaxed);

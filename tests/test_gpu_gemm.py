@@ -17,18 +17,20 @@ from gpu_util import to_dev
 pytestmark = pytest.mark.gpu
 
 
-def run_gemm(Aq, Wq, w_is_nk, c_dtype, sa=None, sw=None, M=None, N=None, K=None, lda=None, ldw=None):
+def run_gemm(Aq, Wq, w_is_nk, c_dtype, sa=None, sw=None, M=None, N=None, K=None, lda=None, ldw=None, staged=False):
     M = Aq.shape[0] if M is None else M
     K = Aq.shape[1] if K is None else K
     N = (Wq.shape[0] if w_is_nk else Wq.shape[1]) if N is None else N
     dA, dW = to_dev(Aq), to_dev(Wq)
     ldc = (N + 7) // 8 * 8
     C = torch.full((M, ldc), float("nan"), dtype=torch.float32 if c_dtype == H.F32 else torch.bfloat16, device="cuda")
-    ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+    # staged: workspace with room for both operands in BF16 -> decode-once path; else the fused kernel
+    wsb = H.hif8_workspace_bytes(H.WS_GEMM, M * K + K * N) if staged else H.hif8_workspace_bytes(H.WS_GEMM, 0)
+    ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
     dsa = torch.tensor([sa], dtype=torch.int32, device="cuda") if sa is not None else None
     dsw = torch.tensor([sw], dtype=torch.int32, device="cuda") if sw is not None else None
     H.hif8_gemm(dA, Aq.shape[1] if lda is None else lda, dW, Wq.shape[1] if ldw is None else ldw, int(w_is_nk), C, ldc,
-                c_dtype, M, N, K, dsa, dsw, ws, 256)
+                c_dtype, M, N, K, dsa, dsw, ws, wsb)
     assert H.hif8_gemm_status(ws) == 0
     out = C.float().cpu().numpy().astype(np.float64)
     assert np.all(np.isnan(out[:, N:]))                      # padding columns untouched
@@ -42,11 +44,12 @@ def check(C, Cstar, S, c_dtype):
     assert not bad.any(), f"{bad.sum()} of {bad.size} outside tolerance; worst ratio {np.max(err / np.maximum(tol, 1e-300)):.3g}"
 
 
+@pytest.mark.parametrize("staged", [False, True])
 @pytest.mark.parametrize("w_is_nk", [0, 1])
 @pytest.mark.parametrize("c_dtype", [H.F32, H.BF16])
 @pytest.mark.parametrize("shape", [(128, 256, 64), (128, 256, 256), (256, 512, 192), (130, 264, 208), (77, 40, 16),
                                    (300, 1000, 1040)])
-def test_gemm_small_full_compare(shape, c_dtype, w_is_nk):
+def test_gemm_small_full_compare(shape, c_dtype, w_is_nk, staged):
     M, N, K = shape
     Aq = W.random_codes((M, K), seed=M + K)
     Wkn = W.random_codes((K, N), seed=N + K + 1)
@@ -55,12 +58,13 @@ def test_gemm_small_full_compare(shape, c_dtype, w_is_nk):
         pad = 16 - Wq.shape[1] % 16
         Wq = np.ascontiguousarray(np.pad(Wq, ((0, 0), (0, pad))))
     Cs, S = O.gemm_full(Aq, Wkn, False, 0, 0)
-    C = run_gemm(Aq, Wq, w_is_nk, c_dtype, N=N)
+    C = run_gemm(Aq, Wq, w_is_nk, c_dtype, N=N, staged=staged)
     check(C, Cs, S, c_dtype)
 
 
+@pytest.mark.parametrize("staged", [False, True])
 @pytest.mark.parametrize("w_is_nk", [0, 1])
-def test_gemm_one_hot_rows_pin_tile_and_k_indexing(w_is_nk):
+def test_gemm_one_hot_rows_pin_tile_and_k_indexing(w_is_nk, staged):
     # A picks one k per row (value 1.0): C[m, :] must equal row perm[m] of W exactly
     M, N, K = 384, 768, 512
     rng = np.random.default_rng(5)
@@ -69,14 +73,14 @@ def test_gemm_one_hot_rows_pin_tile_and_k_indexing(w_is_nk):
     Aq[np.arange(M), perm] = 0x08
     Wkn = W.random_codes((K, N), seed=9)
     tab = np.array([O.value(c) for c in range(256)])
-    C = run_gemm(Aq, np.ascontiguousarray(Wkn.T) if w_is_nk else Wkn, w_is_nk, H.F32)
+    C = run_gemm(Aq, np.ascontiguousarray(Wkn.T) if w_is_nk else Wkn, w_is_nk, H.F32, staged=staged)
     assert np.array_equal(C, tab[Wkn][perm, :])
     # and the mirror: W picks one k per column
     permn = rng.integers(0, K, N)
     Wsel = np.zeros((K, N), dtype=np.uint8)
     Wsel[permn, np.arange(N)] = 0x90                          # -2.0
     Aq2 = W.random_codes((M, K), seed=10)
-    C = run_gemm(Aq2, np.ascontiguousarray(Wsel.T) if w_is_nk else Wsel, w_is_nk, H.F32)
+    C = run_gemm(Aq2, np.ascontiguousarray(Wsel.T) if w_is_nk else Wsel, w_is_nk, H.F32, staged=staged)
     assert np.array_equal(C, -2.0 * tab[Aq2][:, permn])
 
 
@@ -89,6 +93,8 @@ def test_gemm_small_integers_exact_and_descale():
     tab = np.array([O.value(c) for c in range(256)])
     want = (tab[Aq].astype(np.int64) @ tab[Wq].astype(np.int64)).astype(np.float64)
     assert np.array_equal(run_gemm(Aq, Wq, 0, H.F32), want)
+    assert np.array_equal(run_gemm(Aq, Wq, 0, H.F32, staged=True), want)
+    assert np.array_equal(run_gemm(Aq, Wq, 0, H.F32, sa=-7, sw=2, staged=True), want * 32.0)
     assert np.array_equal(run_gemm(Aq, Wq, 0, H.F32, sa=3, sw=-1), want / 4.0)
     assert np.array_equal(run_gemm(Aq, Wq, 0, H.F32, sa=60, sw=55), want * 2.0 ** -115)
 
@@ -99,10 +105,11 @@ def test_gemm_specials_propagate():
     Wq = np.full((K, N), 0x08, dtype=np.uint8)
     Aq[3, 5] = 0x80                                           # NaN
     Aq[7, 9] = 0x6F                                           # +Inf
-    C = run_gemm(Aq, Wq, 0, H.F32)
-    assert np.all(np.isnan(C[3])) and np.all(np.isposinf(C[7]))
-    ok = np.ones(M, bool); ok[[3, 7]] = False
-    assert np.all(C[ok] == K)
+    for staged in (False, True):
+        C = run_gemm(Aq, Wq, 0, H.F32, staged=staged)
+        assert np.all(np.isnan(C[3])) and np.all(np.isposinf(C[7]))
+        ok = np.ones(M, bool); ok[[3, 7]] = False
+        assert np.all(C[ok] == K)
 
 
 @pytest.mark.parametrize("w_is_nk", [0, 1])
@@ -119,5 +126,6 @@ def test_gemm_medium_scaled_operands_sampled(w_is_nk):
     cols = np.concatenate([rng.integers(0, N, 20000), np.tile(np.arange(256), 128), np.tile(np.arange(N - 256, N), 128)])
     Cs, S = O.gemm_entries(Aq, Wkn, False, sa, sw, rows, cols)
     for c_dtype in (H.F32, H.BF16):
-        C = run_gemm(Aq, np.ascontiguousarray(Wkn.T) if w_is_nk else Wkn, w_is_nk, c_dtype, sa=sa, sw=sw)
-        check(C[rows, cols], Cs, S, c_dtype)
+        for staged in (False, True):
+            C = run_gemm(Aq, np.ascontiguousarray(Wkn.T) if w_is_nk else Wkn, w_is_nk, c_dtype, sa=sa, sw=sw, staged=staged)
+            check(C[rows, cols], Cs, S, c_dtype)
