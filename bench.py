@@ -120,6 +120,103 @@ def cpu_baseline(sample_elems):
             "elements_per_s": sample_elems / dt}
 
 
+def extra_results(H, torch, hbm_peak, peak_kind):
+    """Secondary workloads (each with its own roofline fraction): BF16 fake-quant of an LLM-activation tensor,
+    gradient-range FP32 encode/decode, and the HiF8-operand GEMM.  Inputs are generated on the device from a
+    seeded torch generator with the same recipes as workloads/ (shapes and distributions, not the same bytes)."""
+    out = {}
+    g = torch.Generator(device="cuda")
+    g.manual_seed(2345)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    wsb = H.hif8_workspace_bytes(H.WS_FAKE_QUANT, 0)
+    ws = torch.empty(max(wsb, 256), dtype=torch.uint8, device="cuda")
+
+    def timed(fn, reps):
+        for _ in range(3):
+            fn(0)
+        torch.cuda.synchronize()
+        ev0.record()
+        for r in range(reps):
+            fn(r)
+        ev1.record()
+        torch.cuda.synchronize()
+        return ev0.elapsed_time(ev1) / reps
+
+    # ---- LLM-activation fake-quant: BF16 [8192 x 8192], Student-t(3) body, 0.1 % of channels x100
+    T = Hd = 8192
+    n = T * Hd
+    xs = []
+    for _ in range(2):
+        z = torch.randn(T, Hd, generator=g, device="cuda")
+        chi = torch.zeros_like(z)
+        for _ in range(3):
+            chi += torch.randn(T, Hd, generator=g, device="cuda") ** 2
+        x = z / torch.sqrt(chi / 3.0)
+        cols = torch.randperm(Hd, generator=g, device="cuda")[:8]
+        x[:, cols] *= 100.0
+        xs.append(x.to(torch.bfloat16))
+        del z, chi, x
+    ys = [torch.empty_like(x) for x in xs]
+    fq = {}
+    for name, mode in (("TA", H.RND_TA), ("HR", H.RND_HR), ("SSR", H.RND_SSR), ("TE", H.RND_TE), ("SR", H.RND_SR)):
+        ms = timed(lambda r: H.hif8_fake_quant(xs[r & 1], ys[r & 1], H.BF16, n, 1, 14, mode, 0, 7, None, None, ws, wsb), 20)
+        fq[name] = {"ms": ms, "GBps": 6 * n / ms / 1e6, "frac": 6 * n / ms / 1e6 / hbm_peak}
+    ms = timed(lambda r: H.hif8_fake_quant(xs[r & 1], ys[r & 1], H.BF16, n, 0, 3, H.RND_TA, 0, 0), 20)
+    fq["TA_given_scale"] = {"ms": ms, "GBps": 4 * n / ms / 1e6, "frac": 4 * n / ms / 1e6 / hbm_peak}
+    out["fake_quant_bf16_8192x8192"] = {"bytes_per_element": {"fused_amax": 6, "given_scale": 4}, "modes": fq,
+                                        "peak": hbm_peak, "peak_kind": f"of {peak_kind}"}
+    del xs, ys
+
+    # ---- gradient-range stress: FP32 2^28 elements, log-uniform magnitudes 2^-40 .. 2^20, random signs
+    n = 1 << 28
+    e = torch.randint(-40, 20, (n,), generator=g, device="cuda", dtype=torch.int32) + 127
+    m = torch.randint(0, 1 << 23, (n,), generator=g, device="cuda", dtype=torch.int32)
+    sg = torch.randint(0, 2, (n,), generator=g, device="cuda", dtype=torch.int32)
+    bits = (sg << 31) | (e << 23) | m
+    del e, m, sg
+    codes = torch.empty(n, dtype=torch.uint8, device="cuda")
+    back = torch.empty(n, dtype=torch.float32, device="cuda")
+    res = {}
+    for name, mode in (("encode_TA", H.RND_TA), ("encode_HR", H.RND_HR)):
+        ms = timed(lambda r: H.hif8_encode(bits, H.F32, codes, n, 0, mode), 10)
+        res[name] = {"ms": ms, "GBps": 5 * n / ms / 1e6, "frac": 5 * n / ms / 1e6 / hbm_peak}
+    ms = timed(lambda r: H.hif8_decode(codes, back, H.F32, n, 0), 10)
+    res["decode"] = {"ms": ms, "GBps": 5 * n / ms / 1e6, "frac": 5 * n / ms / 1e6 / hbm_peak}
+    out["loguniform_f32_2^28"] = {"bytes_per_element": 5, "calls": res, "peak": hbm_peak, "peak_kind": f"of {peak_kind}"}
+    del bits, codes, back
+
+    # ---- GEMM: A BF16 8192x8192 N(0,1), W BF16 8192x28672 N(0,0.02), per-tensor scaled to HiF8, C = dec(A) dec(W)
+    M, N, K = 8192, 28672, 8192
+    a = torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16)
+    w = (torch.randn(K, N, generator=g, device="cuda") * 0.02).to(torch.bfloat16)
+    Aq = torch.empty(M * K, dtype=torch.uint8, device="cuda")
+    Wq = torch.empty(K * N, dtype=torch.uint8, device="cuda")
+    se = torch.zeros(2, dtype=torch.int32, device="cuda")
+    H.hif8_amax_scale_encode(a, H.BF16, Aq, M * K, 14, H.RND_TA, 0, 0, None, None, se[0:1], None, ws, wsb)
+    H.hif8_amax_scale_encode(w, H.BF16, Wq, K * N, 14, H.RND_TA, 0, 0, None, None, se[1:2], None, ws, wsb)
+    del a, w
+    C = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
+    gws_b = H.hif8_workspace_bytes(H.WS_GEMM, M * K + K * N)
+    gws = torch.empty(gws_b, dtype=torch.uint8, device="cuda")
+    tf_peak, tf_kind = 1590.0, "fallback"
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        tf_peak, tf_kind = float(json.load(open(path))["bf16_tflops"]), "measured"
+    flops = 2.0 * M * N * K
+    ms = timed(lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, C, N, H.BF16, M, N, K, se[0:1], se[1:2], gws, gws_b), 10)
+    st1 = H.hif8_gemm_status(gws)
+    ms_f = timed(lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, C, N, H.BF16, M, N, K, se[0:1], se[1:2], gws, 256), 3)
+    st2 = H.hif8_gemm_status(gws)
+    out["gemm_8192x28672x8192"] = {
+        "decode_once": {"ms": ms, "TFLOPs": flops / ms / 1e9, "frac": flops / ms / 1e9 / tf_peak, "device_status": st1,
+                        "note": "whole call: decode of both operands to BF16 workspace + tcgen05 kernel"},
+        "fused": {"ms": ms_f, "TFLOPs": flops / ms_f / 1e9, "frac": flops / ms_f / 1e9 / tf_peak, "device_status": st2,
+                  "note": "no workspace: byte tiles decoded per CTA in shared memory"},
+        "bound": "tensor", "peak": tf_peak, "peak_kind": f"of {tf_kind} (cuBLAS BF16 burst)", "unit": "TFLOP/s",
+        "scale_exps": [int(v) for v in se.cpu()], "output": "bf16"}
+    return out
+
+
 def run_reference(args, rank):
     if rank != 0:
         return
@@ -158,6 +255,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extra", action="store_true", help="skip the secondary workloads (fake-quant, 2^28 stress, GEMM)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     rank, world, local = env_int("RANK", 0), env_int("WORLD_SIZE", 1), env_int("LOCAL_RANK", 0)
@@ -306,6 +404,10 @@ def main():
             "calls": {"amax_scale_encode_ms": enc_ms, "amax_scale_encode_GBps": BYTES_ENCODE / (enc_ms * 1e-3) / 1e9,
                       "decode_ms": dec_ms, "decode_GBps": dec_gbs},
         }
+        if world == 1 and not args.no_extra:
+            del srcs, codes, backs
+            torch.cuda.empty_cache()
+            line["extra"] = extra_results(H, torch, peak, peak_kind)
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(1 << 23)
         print(json.dumps(line))
