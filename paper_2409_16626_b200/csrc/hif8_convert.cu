@@ -37,7 +37,6 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kUnroll = 4;
 constexpr int kBlocksPerSM = 8;
-constexpr uint32_t kShSlow = 255;  // marks binades below 2^-22 in the shift table
 
 // ------------------------------------------------------------------------------------------------
 // Field packing (Table 1: sign | dot | exponent | mantissa; Table 2 prefix code; Table 3 exponent ranges)
@@ -203,32 +202,31 @@ __device__ __forceinline__ uint32_t encode_one(float x, uint32_t raw, float scal
                                                const uint8_t* s_sh, uint32_t word)
 {
     const float y = x * scale;
-    const uint32_t t = __float_as_uint(y);
+    uint32_t t = __float_as_uint(y);
     if (MODE == HIF8_RND_TA) return s_ta[t >> 19];
 
-    const uint32_t a = t & 0x7FFFFFFFu;
-    const uint32_t sh = s_sh[a >> 23];  // number of discarded mantissa bits (23 - width); 0: nothing to round
     // threshold T of Section 3.2 (with the guard that a zero fraction never rounds up: compare with max(T,1))
     constexpr int kSrBits = (SRC == HIF8_F32) ? 24 : 16;
-    if (sh == kShSlow) {
-        // |y| < 2^-22: kept bits are zero, the fraction is F = |y| / 2^-22 and the result is 0 or 2^-22
-        const float ya = fabsf(y);
-        bool up;
-        if (MODE == HIF8_RND_TE) up = ya > 1.1920928955078125e-07f;  // above 2^-23; the tie goes to the even 0
-        else {
-            float fn; uint32_t T;
-            if (MODE == HIF8_RND_SR) { fn = floorf(ya * exp2f(22.f + kSrBits)); T = word >> (32 - kSrBits); }
-            else if (SRC == HIF8_F32) { fn = floorf(ya * 68719476736.f); T = raw & 0x3FFFu; }  // F14 = floor(F 2^14)
-            else { fn = floorf(ya * 16777216.f); T = 2u * (raw & 1u) + 1u; }                // F2 = floor(F 2^2)
-            up = fn >= (float)max(T, 1u);
-        }
-        return up ? (((t >> 24) & 0x80u) | 0x01u) : 0u;
+    const uint32_t sign7 = (t >> 24) & 0x80u;
+    const bool sub = (t & 0x7FFFFFFFu) < 0x34800000u;  // |y| < 2^-22 (zero included): result is 0 or 2^-22
+    if (MODE == HIF8_RND_SR && SRC == HIF8_F32 && sub) {
+        // the 24-bit threshold is wider than a binary32 fraction: compare F24 = floor(|y| 2^46) directly
+        const uint32_t f24 = __float2uint_rz(fabsf(y) * 70368744177664.f);
+        return f24 >= max(word >> 8, 1u) ? (sign7 | 0x01u) : 0u;
     }
+    // Below 2^-22 the kept bits are zero and the fraction is F = |y| / 2^-22.  Adding 2^-22 with truncation puts
+    // floor(F 2^23) into the mantissa field of a value in the binade of 2^-22, so the common code below rounds it
+    // like a 0-bit-mantissa binade; one step of 2^-22 is taken off the result afterwards.
+    const uint32_t tz = __float_as_uint(__fadd_rz(fabsf(y), 2.384185791015625e-07f)) | (t & 0x80000000u);
+    t = sub ? tz : t;
+    const uint32_t sh = s_sh[(t >> 23) & 0xFFu];  // discarded mantissa bits (23 - width); 0: nothing to round
     const uint32_t s = sh ? sh : 23u;
     uint32_t inc;
     if (MODE == HIF8_RND_TE) {
-        // add half-1, plus one when the kept significand is odd (implicit one when no mantissa bit is kept)
+        // add half-1, plus one when the kept significand is odd (the implicit one when no mantissa bit is kept,
+        // zero below 2^-22)
         uint32_t lsb = (s == 23u) ? 1u : ((t >> s) & 1u);
+        if (sub) lsb = 0u;
         inc = (1u << (s - 1)) - 1u + lsb;
     } else {
         uint32_t inc_ssr;
@@ -236,19 +234,25 @@ __device__ __forceinline__ uint32_t encode_one(float x, uint32_t raw, float scal
         else inc_ssr = (3u - 2u * (raw & 1u)) << (s - 2);                                // SR2: 4 - T2
         if (MODE == HIF8_RND_SSR) inc = inc_ssr;
         else if (MODE == HIF8_RND_HR) {
-            int E = (int)(a >> 23) - 127;                                                // Eq. 3
+            const int E = (int)((t >> 23) & 0xFFu) - 127;                                // Eq. 3
             inc = (E > -4 && E < 4) ? (1u << (s - 1)) : inc_ssr;
         } else {  // standard SR
-            uint32_t T = max(word >> (32 - kSrBits), 1u);
+            const uint32_t T = max(word >> (32 - kSrBits), 1u);
             if (SRC == HIF8_F32) {
-                uint32_t k = 24u - s;  // F24 = discarded << k; up iff discarded >= ceil(T / 2^k)
+                const uint32_t k = 24u - s;  // F24 = discarded << k; up iff discarded >= ceil(T / 2^k)
                 inc = (1u << s) - ((T + (1u << k) - 1u) >> k);
             } else inc = (0x10000u - T) << (s - 16);
         }
     }
     if (sh == 0) inc = 0;
-    const uint32_t tr = (t + inc) & ~((1u << sh) - 1u);
-    return s_ta[tr >> 19];
+    const uint32_t tr = (t + inc) & (0xFFFFFFFFu << sh);
+    uint32_t code = s_ta[tr >> 19];
+    if (sub) {
+        if (MODE == HIF8_RND_TE)  // nearest: up iff above the midpoint 2^-23 (the tie goes to the even value, zero)
+            code = (__float_as_uint(y) & 0x7FFFFFFFu) > 0x34000000u ? (sign7 | 0x01u) : 0u;
+        else code = ((code & 0x7Fu) == 0x02u) ? (sign7 | 0x01u) : 0u;  // 2^-21 -> 2^-22, 2^-22 -> the single zero
+    }
+    return code;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -298,7 +302,7 @@ __device__ __forceinline__ void setup_tables(SmemTables& s, unsigned flags)
     if (NEED_SH) {
         int e = threadIdx.x;  // kThreads == 256 biased exponents
         int E = e - 127;
-        s.sh[e] = (E >= 16 || e == 255) ? 0 : (E <= -23 ? kShSlow : (uint8_t)(23 - mant_width(E)));
+        s.sh[e] = (E >= 16 || E < -22) ? 0 : (uint8_t)(23 - mant_width(E));
     }
     if (NEED_DEC) s.dec[threadIdx.x] = __uint_as_float(decode_bits_f32(threadIdx.x));
     __syncthreads();
@@ -428,6 +432,124 @@ __global__ void __launch_bounds__(kThreads) convert_kernel(const ConvParams p, u
                 if (p.d_amax_out) *p.d_amax_out = __uint_as_float(ab);
             }
         }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Fake-quant, round-half-away, FP32 and BF16: rounding done on the source bit pattern itself.
+// A power-of-two scale only moves which HiF8 binade (hence mantissa width) a source exponent falls into, so
+// quantize-dequantize is "add half of the discarded field, clear it" with an increment and a mask looked up by the
+// source exponent (table rebuilt per block for the scale in force).  No multiply, no code byte, no value table.
+// Exponents whose result is not of that form (overflow and the binade below it, Inf / NaN, subnormal sources under
+// a very large scale) are flagged in the table and take a table-free per-element routine.
+// ------------------------------------------------------------------------------------------------
+constexpr uint32_t kRareMask = 1u;  // never a legitimate mask: legitimate ones are 0 or end in at least four zero bits
+
+// one element, any input: value-level round-half-away through the scaled binary32 value
+template <int SRC>
+__device__ __noinline__ uint32_t fq_ta_rare(uint32_t raw, int se, unsigned flags)
+{
+    const float x = __uint_as_float(SRC == HIF8_F32 ? raw : raw << 16);
+    const uint32_t t = __float_as_uint(x * pow2f(se));
+    const uint32_t a = t & 0x7FFFFFFFu, sign = t & 0x80000000u;
+    if (a > 0x7F800000u) return (flags & HIF8_FLAG_NAN_TO_ZERO) ? 0u : (SRC == HIF8_F32 ? 0x7FC00000u : 0x7FC0u);
+    uint32_t r;
+    if (a >= 0x47200000u) r = (flags & HIF8_FLAG_SATURATE) ? 0x47000000u : 0x7F800000u;  // >= 1.25 * 2^15
+    else if (a < 0x34000000u) return 0u;                                                   // < 2^-23: the single zero
+    else {
+        const int E = (int)(a >> 23) - 127;
+        if (E < -22) r = 0x34800000u;                                                      // [2^-23, 2^-22) -> 2^-22
+        else { const uint32_t k = 23u - (uint32_t)mant_width(E); r = (a + (1u << (k - 1))) & (0xFFFFFFFFu << k); }
+    }
+    const int da = (-se) / 2, db = -se - da;
+    return to_bits<SRC>(__uint_as_float(r | sign) * pow2f(da) * pow2f(db));
+}
+
+template <int SRC>
+__global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, unsigned long long n_vec)
+{
+    constexpr int MB = SRC == HIF8_F32 ? 23 : 7;      // mantissa bits of the source format
+    constexpr int PV = SrcTraits<SRC>::kPerVec;
+    __shared__ uint32_t s_inc[256];                   // BF16: mask16 | inc16 << 16
+    __shared__ uint32_t s_mask[SRC == HIF8_F32 ? 256 : 1];
+    const int se = resolve_scale_exp(p);
+    {
+        const int e = threadIdx.x, E = e - 127 + se;
+        uint32_t inc = 0, mask = 0;
+        if (e == 255 || (e == 0 && se > 100) || (e > 0 && E >= 15)) mask = kRareMask;
+        else if (e == 0 || E <= -24) { inc = 0; mask = 0; }                                 // underflow to +0
+        else if (E == -23) { inc = 1u << MB; mask = 0xFFFFFFFFu << MB; }                    // up to 2^-22
+        else { const uint32_t k = (uint32_t)(MB - mant_width(E)); inc = 1u << (k - 1); mask = 0xFFFFFFFFu << k; }
+        if (SRC == HIF8_F32) { s_inc[e] = inc; s_mask[e] = mask; }
+        else s_inc[e] = (mask & 0xFFFFu) | (inc << 16);
+    }
+    __syncthreads();
+
+    const uint4* src = reinterpret_cast<const uint4*>(p.src);
+    const unsigned long long stride = (unsigned long long)gridDim.x * kThreads * kUnroll;
+    for (unsigned long long base = (unsigned long long)blockIdx.x * kThreads * kUnroll; base < n_vec; base += stride) {
+        uint4 v[kUnroll];
+#pragma unroll
+        for (int j = 0; j < kUnroll; j++) {
+            unsigned long long u = base + (unsigned long long)j * kThreads + threadIdx.x;
+            v[j] = (u < n_vec) ? __ldcs(src + u) : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int j = 0; j < kUnroll; j++) {
+            unsigned long long u = base + (unsigned long long)j * kThreads + threadIdx.x;
+            if (u >= n_vec) continue;
+            uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w}, o[4], rare = 0;
+            if (SRC == HIF8_F32) {
+                uint32_t m[4];
+#pragma unroll
+                for (int k = 0; k < 4; k++) {
+                    const uint32_t e = (w[k] >> 23) & 0xFFu;
+                    m[k] = s_mask[e];
+                    o[k] = (w[k] + s_inc[e]) & m[k];
+                    rare |= m[k];
+                }
+                if (rare & kRareMask) {
+#pragma unroll
+                    for (int k = 0; k < 4; k++)
+                        if (m[k] == kRareMask) o[k] = fq_ta_rare<SRC>(w[k], se, p.flags);
+                }
+            } else {
+                uint32_t tl[4], th[4];
+#pragma unroll
+                for (int k = 0; k < 4; k++) {
+                    tl[k] = s_inc[(w[k] >> 7) & 0xFFu];
+                    th[k] = s_inc[(w[k] >> 23) & 0xFFu];
+                    const uint32_t mask2 = __byte_perm(tl[k], th[k], 0x5410), inc2 = __byte_perm(tl[k], th[k], 0x7632);
+                    o[k] = (w[k] + inc2) & mask2;  // no carry between the halves: flagged exponents add nothing
+                    rare |= tl[k] | th[k];
+                }
+                if (rare & kRareMask) {
+#pragma unroll
+                    for (int k = 0; k < 4; k++) {
+                        if (tl[k] & kRareMask) o[k] = (o[k] & 0xFFFF0000u) | fq_ta_rare<SRC>(w[k] & 0xFFFFu, se, p.flags);
+                        if (th[k] & kRareMask) o[k] = (o[k] & 0x0000FFFFu) | (fq_ta_rare<SRC>(w[k] >> 16, se, p.flags) << 16);
+                    }
+                }
+            }
+            __stcs(reinterpret_cast<uint4*>(p.dst) + u, make_uint4(o[0], o[1], o[2], o[3]));
+        }
+    }
+    {   // tail / unaligned elements
+        const unsigned long long tid = (unsigned long long)blockIdx.x * kThreads + threadIdx.x;
+        for (unsigned long long i = n_vec * PV + tid; i < p.n; i += (unsigned long long)gridDim.x * kThreads) {
+            if (SRC == HIF8_F32) {
+                const uint32_t raw = reinterpret_cast<const uint32_t*>(p.src)[i];
+                reinterpret_cast<uint32_t*>(p.dst)[i] = fq_ta_rare<SRC>(raw, se, p.flags);
+            } else {
+                const uint32_t raw = reinterpret_cast<const unsigned short*>(p.src)[i];
+                reinterpret_cast<unsigned short*>(p.dst)[i] = (unsigned short)fq_ta_rare<SRC>(raw, se, p.flags);
+            }
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        if (p.d_scale_exp_out) *p.d_scale_exp_out = se;
+        if (p.d_scale_out) *p.d_scale_out = pow2f(se);
+        if (p.d_amax_out && p.d_amax_bits) *p.d_amax_out = __uint_as_float(*p.d_amax_bits);
     }
 }
 
@@ -590,6 +712,17 @@ int dispatch_convert(int dtype, int rnd, const ConvParams& p, bool vec_ok, int s
     }
 }
 
+int launch_fq_ta(int dtype, const ConvParams& p, bool vec_ok, int sms, cudaStream_t st)
+{
+    const unsigned long long pv = dtype == HIF8_F32 ? 4 : 8;
+    const unsigned long long n_vec = vec_ok ? p.n / pv : 0;
+    const unsigned grid = grid_for(n_vec, p.n, sms);
+    if (dtype == HIF8_F32) fq_ta_kernel<HIF8_F32><<<grid, kThreads, 0, st>>>(p, n_vec);
+    else fq_ta_kernel<HIF8_BF16><<<grid, kThreads, 0, st>>>(p, n_vec);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
+}
+
 int launch_amax(const void* src, int dtype, unsigned long long n, uint32_t* accum, int sms, cudaStream_t st)
 {
     bool vec_ok = aligned16(src);
@@ -680,13 +813,16 @@ static int scaled_convert(bool fq, const void* src, void* dst, int dtype, size_t
         if (!ws || workspace_bytes < kConvWorkspaceBytes || (reinterpret_cast<uintptr_t>(ws) & 255u)) return HIF8_ERR_WORKSPACE;
         if (cudaMemsetAsync(ws, 0, 8, st) != cudaSuccess) return HIF8_ERR_CUDA;
     }
+    const bool inplace_fq = fq && rnd == HIF8_RND_TA && (dtype == HIF8_F32 || dtype == HIF8_BF16) && !want_amax;
     if (jit) {
         rc = launch_amax(src, dtype, n, ws, sms, st);
         if (rc) return rc;
         p.d_amax_bits = ws;
+        if (inplace_fq) return launch_fq_ta(dtype, p, vec_ok, sms, st);
         return fq ? dispatch_convert<true, false>(dtype, rnd, p, vec_ok, sms, st)
                   : dispatch_convert<false, false>(dtype, rnd, p, vec_ok, sms, st);
     }
+    if (inplace_fq) return launch_fq_ta(dtype, p, vec_ok, sms, st);
     if (want_amax) {
         p.amax_accum = ws;
         return fq ? dispatch_convert<true, true>(dtype, rnd, p, vec_ok, sms, st)

@@ -1,0 +1,67 @@
+"""Run one named workload a few times, for use under a profiler:
+
+    python -m paper_2409_16626_b200.profile_cases <case> [repeats]
+
+cases: convert_f32 (FP32 4096^2: per-tensor scaled encode + decode), fq_bf16 (BF16 4096x8192 fake-quant, TA and HR,
+fused amax and given scale), encode_modes_f32 (FP32 2^25 log-uniform, every rounding mode), gemm (HiF8 GEMM
+4096 x 7168 x 4096, fused and decode-once paths).  Inputs are seeded device-side random tensors.
+"""
+import sys
+
+import torch
+
+from . import binding as H
+
+
+def main():
+    case = sys.argv[1] if len(sys.argv) > 1 else "convert_f32"
+    reps = int(sys.argv[2]) if len(sys.argv) > 2 else 3
+    g = torch.Generator(device="cuda")
+    g.manual_seed(1)
+    ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+    if case == "convert_f32":
+        n = 4096 * 4096
+        xs = [torch.randn(n, generator=g, device="cuda") for _ in range(3)]
+        codes = torch.empty(n, dtype=torch.uint8, device="cuda")
+        back = torch.empty(n, dtype=torch.float32, device="cuda")
+        se = torch.zeros(1, dtype=torch.int32, device="cuda")
+        for r in range(reps):
+            H.hif8_amax_scale_encode(xs[r % 3], H.F32, codes, n, 14, H.RND_TA, 0, 0, None, None, se, None, ws, 256)
+            H.hif8_decode(codes, back, H.F32, n, 12)
+    elif case == "fq_bf16":
+        n = 4096 * 8192
+        xs = [torch.randn(n, generator=g, device="cuda").to(torch.bfloat16) for _ in range(3)]
+        y = torch.empty_like(xs[0])
+        for r in range(reps):
+            for mode in (H.RND_TA, H.RND_HR):
+                H.hif8_fake_quant(xs[r % 3], y, H.BF16, n, 1, 14, mode, 0, 7, None, None, ws, 256)
+                H.hif8_fake_quant(xs[r % 3], y, H.BF16, n, 0, 12, mode, 0, 7)
+    elif case == "encode_modes_f32":
+        n = 1 << 25
+        e = torch.randint(-40, 20, (n,), generator=g, device="cuda", dtype=torch.int32) + 127
+        m = torch.randint(0, 1 << 23, (n,), generator=g, device="cuda", dtype=torch.int32)
+        bits = (e << 23) | m
+        codes = torch.empty(n, dtype=torch.uint8, device="cuda")
+        for r in range(reps):
+            for mode in (H.RND_TA, H.RND_HR, H.RND_SSR, H.RND_TE, H.RND_SR):
+                H.hif8_encode(bits, H.F32, codes, n, 0, mode, 0, 5)
+    elif case == "gemm":
+        M, N, K = 4096, 7168, 4096
+        A = torch.randint(0, 256, (M, K), dtype=torch.uint8, device="cuda", generator=g)
+        W = torch.randint(0, 256, (K, N), dtype=torch.uint8, device="cuda", generator=g)
+        for t in (A, W):                                   # keep the operands finite
+            t[(t == 0x80) | ((t & 0x7F) == 0x6F)] = 0x08
+        C = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
+        big = H.hif8_workspace_bytes(H.WS_GEMM, M * K + K * N)
+        gws = torch.empty(big, dtype=torch.uint8, device="cuda")
+        for r in range(reps):
+            H.hif8_gemm(A, K, W, N, 0, C, N, H.BF16, M, N, K, None, None, gws, big)
+            H.hif8_gemm(A, K, W, N, 0, C, N, H.BF16, M, N, K, None, None, gws, 256)
+    else:
+        raise SystemExit(f"unknown case {case}")
+    torch.cuda.synchronize()
+    print("done", case, H.hif8_launch_count())
+
+
+if __name__ == "__main__":
+    main()
