@@ -33,6 +33,9 @@ BYTES_DECODE = 5 * N_EL
 BYTES_STEP = BYTES_ENCODE + BYTES_DECODE
 POOL = 6                  # rotating buffer sets: 6 x 64 MiB of input alone exceeds the 126 MB L2
 WORKLOAD = "fp32_4096x4096_normal_amax_scale_encode_then_decode"
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture summarised in profiles/;
+# None for a kernel changed since its capture
+TRAFFIC = {"amax_kernel<f32>": None, "convert_kernel<f32,TA>": None, "decode_kernel<f32>": None}
 METRIC = "hif8_encode_decode_throughput"
 UNIT = "GB/s"
 
@@ -309,7 +312,7 @@ def main():
     # The launch sequence of POOL consecutive steps (one per buffer set) is captured once in a CUDA graph and
     # replayed, so the host's per-launch cost stays out of the device timeline; K steps = K // POOL replays plus
     # K % POOL directly launched steps.
-    K = args.steps
+    K = max(POOL, args.steps // POOL * POOL)   # whole graph replays: the step count is rounded down to a multiple of POOL
     ws2 = [ws, torch.empty(max(wsb, 256), dtype=torch.uint8, device="cuda")]
     scal2 = [scal, torch.zeros(4, dtype=torch.int32, device="cuda")]
 
@@ -356,28 +359,40 @@ def main():
         t0.record(stream)
         for _ in range(K // POOL):
             graph.replay()
-        for k in range(K % POOL):
-            encode_call(k)
-            decode_call(k, se)
         t1.record(stream)
         torch.cuda.synchronize()
-        # per-call durations: the same calls launched directly, an event after each call
-        K2 = min(K, 600)
-        ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * K2 + 1)]
-        ev[0].record(stream)
-        for k in range(K2):
-            i = k % POOL
-            encode_call(i)
-            ev[2 * k + 1].record(stream)
-            decode_call(i, se)
-            ev[2 * k + 2].record(stream)
-        torch.cuda.synchronize()
+        # per-kernel durations, measured live: each kernel of the step in a graph of its own (POOL launches over the
+        # rotating buffers: hif8_amax -> amax_kernel behind its 8-byte memset node; hif8_encode with the scale known ->
+        # the same convert_kernel the scaled call launches; hif8_decode -> decode_kernel), replayed between two events.
+        # Direct launches would time the host's launch rate, not these ~15 us kernels.
+        amax_out = torch.zeros(1, dtype=torch.float32, device="cuda")
+
+        def kernel_ms(call):
+            gk = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gk):
+                cs = torch.cuda.current_stream().cuda_stream
+                for i in range(POOL):
+                    call(i, cs)
+            R = max(4, min(K, 600) // POOL)
+            for _ in range(3):
+                gk.replay()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(R):
+                gk.replay()
+            b.record(stream)
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / (R * POOL)
+
+        amax_ms = kernel_ms(lambda i, cs: H.hif8_amax(srcs[i], H.F32, N_EL, amax_out, ws, wsb, stream=cs))
+        conv_ms = kernel_ms(lambda i, cs: H.hif8_encode(srcs[i], H.F32, codes[i], N_EL, se, H.RND_TA, 0, 0, stream=cs))
+        dec_ms = kernel_ms(lambda i, cs: H.hif8_decode(codes[i], backs[i], H.F32, N_EL, se, stream=cs))
+        enc_ms = kernel_ms(lambda i, cs: H.hif8_amax_scale_encode(srcs[i], H.F32, codes[i], N_EL, 14, H.RND_TA, 0, 0, None,
+                                                                  scal[0:1], scal[1:2], scal[2:3], ws, wsb, stream=cs))
     barrier()
-    launches = 3 * POOL * (K // POOL) + 3 * (K % POOL)   # amax + convert + decode kernels per step (replays included)
-    assert H.hif8_launch_count() - launches0 == 3 * (K % POOL) + 3 * K2
+    launches = 3 * POOL * (K // POOL)   # amax + convert + decode kernels per step (graph replays)
     total_ms = t0.elapsed_time(t1)
-    enc_ms = sum(ev[2 * k].elapsed_time(ev[2 * k + 1]) for k in range(K2)) / K2
-    dec_ms = sum(ev[2 * k + 1].elapsed_time(ev[2 * k + 2]) for k in range(K2)) / K2
 
     # ---- end to end: pinned host input -> device, both calls, results back to pinned host memory
     E = max(3, min(args.e2e_steps, K))
@@ -405,16 +420,24 @@ def main():
     e2e_ms = e0.elapsed_time(e1) / E
 
     if world > 1:
-        t = torch.tensor([total_ms, e2e_ms, enc_ms, dec_ms], dtype=torch.float64, device="cuda")
+        t = torch.tensor([total_ms, e2e_ms, enc_ms, dec_ms, amax_ms, conv_ms], dtype=torch.float64, device="cuda")
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms, enc_ms, dec_ms = [float(v) for v in t.cpu()]
+        total_ms, e2e_ms, enc_ms, dec_ms, amax_ms, conv_ms = [float(v) for v in t.cpu()]
 
     if rank == 0:
         ms_per_step = total_ms / K
         value = world * BYTES_STEP / (ms_per_step * 1e-3) / 1e9
         peak, peak_kind = load_peaks()
-        # dominant kernel: the decode launch (1 B read + 4 B written per element, one kernel per call)
-        dec_gbs = BYTES_DECODE / (dec_ms * 1e-3) / 1e9
+        kernels = {
+            "amax_kernel<f32>": {"ms": amax_ms, "bytes": 4 * N_EL, "note": "hif8_amax call: 8-byte memset node + kernel"},
+            "convert_kernel<f32,TA>": {"ms": conv_ms, "bytes": 5 * N_EL},
+            "decode_kernel<f32>": {"ms": dec_ms, "bytes": 5 * N_EL},
+        }
+        for kv in kernels.values():
+            kv["GBps"] = kv["bytes"] / (kv["ms"] * 1e-3) / 1e9
+            kv["frac"] = kv["GBps"] / peak
+        # the dominant kernel: longest live duration among the single-kernel calls
+        dom = max(("convert_kernel<f32,TA>", "decode_kernel<f32>"), key=lambda kname: kernels[kname]["ms"])
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -428,11 +451,12 @@ def main():
             "e2e": {"value": world * BYTES_STEP / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": 4 * N_EL, "d2h_bytes_per_step": 5 * N_EL},
             "gpu_launches": int(launches),
-            "roofline": {"bound": "hbm", "kernel": "decode_kernel<f32>", "achieved": dec_gbs, "peak": peak,
-                         "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": dec_gbs / peak, "traffic": None,
-                         "algorithmic_bytes_per_launch": BYTES_DECODE, "avg_launch_ms": dec_ms},
-            "calls": {"amax_scale_encode_ms": enc_ms, "amax_scale_encode_GBps": BYTES_ENCODE / (enc_ms * 1e-3) / 1e9,
-                      "decode_ms": dec_ms, "decode_GBps": dec_gbs},
+            "roofline": {"bound": "hbm", "kernel": dom, "achieved": kernels[dom]["GBps"], "peak": peak,
+                         "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": kernels[dom]["frac"],
+                         "traffic": TRAFFIC.get(dom), "algorithmic_bytes_per_launch": kernels[dom]["bytes"],
+                         "avg_launch_ms": kernels[dom]["ms"]},
+            "kernels": kernels,
+            "calls": {"amax_scale_encode_ms": enc_ms, "amax_scale_encode_GBps": BYTES_ENCODE / (enc_ms * 1e-3) / 1e9},
         }
         if world == 1 and not args.no_extra:
             del srcs, codes, backs

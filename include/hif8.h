@@ -107,6 +107,15 @@ int hif8_amax_scale_encode(const void* src, int src_dtype, uint8_t* dst, size_t 
                            size_t workspace_bytes, hif8_stream_t stream);
 
 /*
+ * Amax alone (Section 5.1: "every 10 iterations, we compute the maximum absolute value (Amax) of each tensor"):
+ *   *d_amax_out = max |src[i]| over the finite elements (0 if there is none), as an exact float.
+ * One read of the tensor.  workspace as for hif8_amax_scale_encode.  The caller derives the next scale exponent
+ * from it (or lets hif8_amax_scale_encode do both in one call).
+ */
+int hif8_amax(const void* src, int src_dtype, size_t n, float* d_amax_out, void* workspace, size_t workspace_bytes,
+              hif8_stream_t stream);
+
+/*
  * hif8_amax_scale_encode without a caller-supplied workspace.  (The paper has no counterpart: this entry
  * point exists for the benefit of the calling environment only.)
  *

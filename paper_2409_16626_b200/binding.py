@@ -17,7 +17,7 @@ OK = 0
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libhif8.so")
-EXPORTS = ["hif8_encode", "hif8_decode", "hif8_amax_scale_encode", "hif8_fake_quant", "hif8_gemm", "hif8_gemm_status",
+EXPORTS = ["hif8_encode", "hif8_decode", "hif8_amax", "hif8_amax_scale_encode", "hif8_fake_quant", "hif8_gemm", "hif8_gemm_status",
            "hif8_amax_scale_encode_static", "hif8_workspace_bytes", "hif8_status_string", "hif8_launch_count"]
 
 if not os.path.exists(LIB_PATH):
@@ -28,6 +28,8 @@ _vp, _sz, _i, _u, _u64, _i64 = C.c_void_p, C.c_size_t, C.c_int, C.c_uint, C.c_ui
 lib.hif8_encode.argtypes = [_vp, _i, _vp, _sz, _i, _i, _u, _u64, _vp]
 lib.hif8_decode.argtypes = [_vp, _vp, _i, _sz, _i, _vp]
 lib.hif8_amax_scale_encode.argtypes = [_vp, _i, _vp, _sz, _i, _i, _u, _u64, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
+lib.hif8_amax.argtypes = [_vp, _i, _sz, _vp, _vp, _sz, _vp]
+lib.hif8_amax.restype = _i
 lib.hif8_amax_scale_encode_static.argtypes = [_vp, _i, _vp, _sz, _i, _i, _u, _u64, _vp, _vp, _vp, _vp, _vp]
 lib.hif8_amax_scale_encode_static.restype = _i
 lib.hif8_fake_quant.argtypes = [_vp, _vp, _i, _sz, _i, _i, _i, _u, _u64, _vp, _vp, _vp, _sz, _vp]
@@ -97,6 +99,10 @@ def hif8_amax_scale_encode(src, src_dtype, dst, n, target_exp=14, rnd=RND_TA, fl
     return _check(lib.hif8_amax_scale_encode(_ptr(src), src_dtype, _ptr(dst), n, target_exp, rnd, flags, seed,
                                              _ptr(d_scale_exp_in), _ptr(d_amax_out), _ptr(d_scale_exp_out),
                                              _ptr(d_scale_out), _ptr(workspace), workspace_bytes, _stream(stream)), check)
+
+
+def hif8_amax(src, src_dtype, n, d_amax_out, workspace, workspace_bytes, stream=None, check=True):
+    return _check(lib.hif8_amax(_ptr(src), src_dtype, n, _ptr(d_amax_out), _ptr(workspace), workspace_bytes, _stream(stream)), check)
 
 
 def hif8_amax_scale_encode_static(src, src_dtype, dst, n, target_exp=14, rnd=RND_TA, flags=0, seed=0,

@@ -556,7 +556,7 @@ __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, uns
 // amax only (first pass of just-in-time scaling)
 template <int SRC>
 __global__ void __launch_bounds__(kThreads) amax_kernel(const void* __restrict__ srcv, unsigned long long n,
-                                                        unsigned long long n_vec, uint32_t* accum)
+                                                        unsigned long long n_vec, uint32_t* accum, float* d_amax_out)
 {
     constexpr int PV = SrcTraits<SRC>::kPerVec;
     const uint4* src = reinterpret_cast<const uint4*>(srcv);
@@ -586,6 +586,13 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const void* __restrict__
         amax = amax_step(amax, x);
     }
     block_amax_commit(amax, accum);
+    if (d_amax_out && threadIdx.x == 0) {  // stand-alone amax: the last block to finish publishes the result
+        __threadfence();
+        if (atomicAdd(accum + 1, 1u) == gridDim.x - 1) {
+            __threadfence();
+            *d_amax_out = __uint_as_float(atomicMax(accum, 0u));
+        }
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -595,10 +602,14 @@ template <int DT>
 __global__ void __launch_bounds__(kThreads) decode_kernel(const uint8_t* __restrict__ src, void* __restrict__ dst,
                                                           unsigned long long n, unsigned long long n_vec, int se)
 {
-    __shared__ SmemTables sm;
-    setup_tables<false, false, true>(sm, 0);
-    const int da = (-se) / 2, db = -se - da;
-    const float d1 = pow2f(da), d2 = pow2f(db);
+    // Output encodings of all 256 bytes for this call: value * 2^-scale_exp in two exact power-of-two steps (the first
+    // cannot leave the normal range, so only the second may round -- to nearest even), then the destination format.
+    __shared__ uint32_t s_out[256];
+    {
+        const int da = (-se) / 2, db = -se - da;
+        s_out[threadIdx.x] = to_bits<DT>(__uint_as_float(decode_bits_f32(threadIdx.x)) * pow2f(da) * pow2f(db));
+    }
+    __syncthreads();
     constexpr int PV = SrcTraits<DT>::kPerVec;  // codes per 16-byte store
     const unsigned long long stride = (unsigned long long)gridDim.x * kThreads * kUnroll;
     for (unsigned long long base = (unsigned long long)blockIdx.x * kThreads * kUnroll; base < n_vec; base += stride) {
@@ -618,10 +629,7 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const uint8_t* __restr
             if (u >= n_vec) continue;
             uint32_t o[PV];
 #pragma unroll
-            for (int k = 0; k < PV; k++) {
-                uint32_t c = ((k < 4 ? v[j].x : v[j].y) >> (8 * (k & 3))) & 0xFFu;
-                o[k] = to_bits<DT>(sm.dec[c] * d1 * d2);
-            }
+            for (int k = 0; k < PV; k++) o[k] = s_out[((k < 4 ? v[j].x : v[j].y) >> (8 * (k & 3))) & 0xFFu];
             uint4 out;
             if (PV == 4) out = make_uint4(o[0], o[1], o[2], o[3]);
             else out = make_uint4(o[0] | (o[1] << 16), o[2] | (o[3] << 16), o[4] | (o[5] << 16), o[6] | (o[7] << 16));
@@ -630,7 +638,7 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const uint8_t* __restr
     }
     const unsigned long long tid = (unsigned long long)blockIdx.x * kThreads + threadIdx.x;
     for (unsigned long long i = n_vec * PV + tid; i < n; i += (unsigned long long)gridDim.x * kThreads) {
-        uint32_t o = to_bits<DT>(sm.dec[src[i]] * d1 * d2);
+        const uint32_t o = s_out[src[i]];
         if (DT == HIF8_F32) reinterpret_cast<uint32_t*>(dst)[i] = o;
         else reinterpret_cast<unsigned short*>(dst)[i] = (unsigned short)o;
     }
@@ -723,16 +731,16 @@ int launch_fq_ta(int dtype, const ConvParams& p, bool vec_ok, int sms, cudaStrea
     return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
 }
 
-int launch_amax(const void* src, int dtype, unsigned long long n, uint32_t* accum, int sms, cudaStream_t st)
+int launch_amax(const void* src, int dtype, unsigned long long n, uint32_t* accum, float* d_amax_out, int sms, cudaStream_t st)
 {
     bool vec_ok = aligned16(src);
     unsigned long long pv = dtype == HIF8_F32 ? 4 : 8;
     unsigned long long n_vec = vec_ok ? n / pv : 0;
     unsigned grid = grid_for(n_vec, n, sms);
     switch (dtype) {
-        case HIF8_F32: amax_kernel<HIF8_F32><<<grid, kThreads, 0, st>>>(src, n, n_vec, accum); break;
-        case HIF8_BF16: amax_kernel<HIF8_BF16><<<grid, kThreads, 0, st>>>(src, n, n_vec, accum); break;
-        default: amax_kernel<HIF8_F16><<<grid, kThreads, 0, st>>>(src, n, n_vec, accum); break;
+        case HIF8_F32: amax_kernel<HIF8_F32><<<grid, kThreads, 0, st>>>(src, n, n_vec, accum, d_amax_out); break;
+        case HIF8_BF16: amax_kernel<HIF8_BF16><<<grid, kThreads, 0, st>>>(src, n, n_vec, accum, d_amax_out); break;
+        default: amax_kernel<HIF8_F16><<<grid, kThreads, 0, st>>>(src, n, n_vec, accum, d_amax_out); break;
     }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
@@ -815,7 +823,7 @@ static int scaled_convert(bool fq, const void* src, void* dst, int dtype, size_t
     }
     const bool inplace_fq = fq && rnd == HIF8_RND_TA && (dtype == HIF8_F32 || dtype == HIF8_BF16) && !want_amax;
     if (jit) {
-        rc = launch_amax(src, dtype, n, ws, sms, st);
+        rc = launch_amax(src, dtype, n, ws, nullptr, sms, st);
         if (rc) return rc;
         p.d_amax_bits = ws;
         if (inplace_fq) return launch_fq_ta(dtype, p, vec_ok, sms, st);
@@ -847,6 +855,20 @@ int hif8_amax_scale_encode(const void* src, int src_dtype, uint8_t* dst, size_t 
     return scaled_convert(false, src, dst, src_dtype, n, jit, target_exp, d_scale_exp_in, 0, rnd, flags, seed,
                           d_amax_out, d_scale_exp_out, d_scale_out, workspace, workspace_bytes, !jit,
                           (cudaStream_t)stream);
+}
+
+int hif8_amax(const void* src, int src_dtype, size_t n, float* d_amax_out, void* workspace, size_t workspace_bytes,
+              hif8_stream_t stream)
+{
+    if (src_dtype != HIF8_F32 && src_dtype != HIF8_BF16 && src_dtype != HIF8_F16) return HIF8_ERR_DTYPE;
+    if (!d_amax_out || (n && !src)) return HIF8_ERR_NULL;
+    if (!workspace || workspace_bytes < kConvWorkspaceBytes || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+        return HIF8_ERR_WORKSPACE;
+    int sms; int rc = device_info(&sms);
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemsetAsync(workspace, 0, 8, st) != cudaSuccess) return HIF8_ERR_CUDA;
+    return launch_amax(src, src_dtype, n, reinterpret_cast<uint32_t*>(workspace), d_amax_out, sms, st);
 }
 
 int hif8_fake_quant(const void* src, void* dst, int dtype, size_t n, int use_amax, int scale_or_target_exp, int rnd,

@@ -416,7 +416,6 @@ constexpr int kStagesP = 4;
 constexpr int kThreadsP = 6 * 32;
 constexpr uint32_t kStageBytesP = kABfBytes + kBBfBytes;  // 48 KiB
 struct SmemLayoutP {
-    static constexpr uint32_t ops = 0;
     static constexpr uint32_t bars = kStagesP * kStageBytesP;           // 192 KiB
     static constexpr uint32_t n_bars = 2 * kStagesP + 4;
     static constexpr uint32_t tmem_slot = bars + n_bars * 8;

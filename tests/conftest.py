@@ -8,6 +8,17 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 
+def _ensure_built():
+    """The C oracle and the CUDA library are built in-tree on demand (gcc / nvcc cross-compile, no GPU needed)."""
+    from paper_2409_16626_b200 import build as lib_build
+    lib_build.build()
+    from oracle import build as oracle_build
+    oracle_build.build()
+
+
+_ensure_built()
+
+
 def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200)")
 

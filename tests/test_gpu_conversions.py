@@ -176,6 +176,18 @@ def test_amax_scale_encode_jit_and_delayed(dtype):
     assert_same(rb(), O.encode(src, dtype, 5, O.TA, 0, quick=True), src)
 
 
+def test_amax_alone():
+    ws, wsb = workspace()
+    out = torch.zeros(1, dtype=torch.float32, device="cuda")
+    for dtype, src in [(H.F32, W.loguniform_f32(1_000_003, seed=4).view(np.uint32)), (H.BF16, W.normal_bf16(300_001, seed=5)),
+                       (H.F16, W.normal_f32(70_001, seed=6).astype(np.float16).view(np.uint16)),
+                       (H.F32, np.array([0x7FC00000, 0xFF800000, 0x80000000], np.uint32))]:
+        for _ in range(2):
+            H.hif8_amax(to_dev(src), dtype, src.size, out, ws, wsb)
+            torch.cuda.synchronize()
+            assert float(out.item()) == O.amax_scale(src, dtype, 14)[0]
+
+
 def test_amax_degenerate_tensors():
     ws, wsb = workspace()
     outs = torch.zeros(4, dtype=torch.int32, device="cuda")
