@@ -101,6 +101,21 @@ class ClockSampler:
         return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+def max_over_ranks(values, dist=None, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks (identity without an initialised process group)."""
+    if dist is None or not dist.is_available() or not dist.is_initialized() or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    import torch
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.cpu()]
+
+
+def job_throughput(world, bytes_per_rank_step, ms_per_step):
+    """Whole-job GB/s: every rank converts its own tensor (weak scaling), time is the slowest rank's."""
+    return world * bytes_per_rank_step / (ms_per_step * 1e-3) / 1e9
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -419,14 +434,12 @@ def main():
     barrier()
     e2e_ms = e0.elapsed_time(e1) / E
 
-    if world > 1:
-        t = torch.tensor([total_ms, e2e_ms, enc_ms, dec_ms, amax_ms, conv_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms, enc_ms, dec_ms, amax_ms, conv_ms = [float(v) for v in t.cpu()]
+    total_ms, e2e_ms, enc_ms, dec_ms, amax_ms, conv_ms = max_over_ranks(
+        [total_ms, e2e_ms, enc_ms, dec_ms, amax_ms, conv_ms], dist if world > 1 else None, "cuda")
 
     if rank == 0:
         ms_per_step = total_ms / K
-        value = world * BYTES_STEP / (ms_per_step * 1e-3) / 1e9
+        value = job_throughput(world, BYTES_STEP, ms_per_step)
         peak, peak_kind = load_peaks()
         kernels = {
             "amax_kernel<f32>": {"ms": amax_ms, "bytes": 4 * N_EL, "note": "hif8_amax call: 8-byte memset node + kernel"},
@@ -448,7 +461,7 @@ def main():
                        "l2": f"inputs rotate over {POOL} buffer sets ({POOL * N_EL * 4 >> 20} MiB of sources) > 126 MB L2",
                        "bytes_per_step": BYTES_STEP, "elements_per_s": world * N_EL / (ms_per_step * 1e-3)},
             "clocks": clk.summary(),
-            "e2e": {"value": world * BYTES_STEP / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
+            "e2e": {"value": job_throughput(world, BYTES_STEP, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": 4 * N_EL, "d2h_bytes_per_step": 5 * N_EL},
             "gpu_launches": int(launches),
             "roofline": {"bound": "hbm", "kernel": dom, "achieved": kernels[dom]["GBps"], "peak": peak,
