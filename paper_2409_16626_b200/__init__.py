@@ -5,8 +5,12 @@ The binding (and with it libhif8.so) is loaded on first attribute access, so tha
 """
 import importlib
 
+_SUBMODULES = ("build", "binding", "profile_cases")
+
 
 def __getattr__(name):
+    if name in _SUBMODULES:
+        return importlib.import_module("." + name, __name__)
     binding = importlib.import_module(".binding", __name__)
     try:
         return getattr(binding, name)
