@@ -436,7 +436,8 @@ __global__ void __launch_bounds__(kThreads) convert_kernel(const ConvParams p, u
 }
 
 // ------------------------------------------------------------------------------------------------
-// Fake-quant, round-half-away, FP32 and BF16: rounding done on the source bit pattern itself.
+// Fake-quant with the rounding done on the source bit pattern itself: round half away (FP32, BF16), and hybrid /
+// simplified stochastic rounding (BF16).
 // A power-of-two scale only moves which HiF8 binade (hence mantissa width) a source exponent falls into, so
 // quantize-dequantize is "add half of the discarded field, clear it" with an increment and a mask looked up by the
 // source exponent (table rebuilt per block for the scale in force).  No multiply, no code byte, no value table.
@@ -445,29 +446,47 @@ __global__ void __launch_bounds__(kThreads) convert_kernel(const ConvParams p, u
 // ------------------------------------------------------------------------------------------------
 constexpr uint32_t kRareMask = 1u;  // never a legitimate mask: legitimate ones are 0 or end in at least four zero bits
 
-// one element, any input: value-level round-half-away through the scaled binary32 value
-template <int SRC>
-__device__ __noinline__ uint32_t fq_ta_rare(uint32_t raw, int se, unsigned flags)
+// one element, any input: value-level rounding through the scaled binary32 value.
+// MODE: round half away, or (BF16 sources) the 2-bit simplified stochastic rounding SR2 / hybrid rounding of Eq. 3.
+template <int SRC, int MODE>
+__device__ __noinline__ uint32_t fq_rare(uint32_t raw, int se, unsigned flags)
 {
     const float x = __uint_as_float(SRC == HIF8_F32 ? raw : raw << 16);
-    const uint32_t t = __float_as_uint(x * pow2f(se));
+    const float y = x * pow2f(se);
+    const uint32_t t = __float_as_uint(y);
     const uint32_t a = t & 0x7FFFFFFFu, sign = t & 0x80000000u;
     if (a > 0x7F800000u) return (flags & HIF8_FLAG_NAN_TO_ZERO) ? 0u : (SRC == HIF8_F32 ? 0x7FC00000u : 0x7FC0u);
+    const uint32_t top = (flags & HIF8_FLAG_SATURATE) ? 0x47000000u : 0x7F800000u;  // 2^15 or Inf
+    const int E = (int)(a >> 23) - 127;
     uint32_t r;
-    if (a >= 0x47200000u) r = (flags & HIF8_FLAG_SATURATE) ? 0x47000000u : 0x7F800000u;  // >= 1.25 * 2^15
-    else if (a < 0x34000000u) return 0u;                                                   // < 2^-23: the single zero
-    else {
-        const int E = (int)(a >> 23) - 127;
-        if (E < -22) r = 0x34800000u;                                                      // [2^-23, 2^-22) -> 2^-22
+    if (MODE == HIF8_RND_TA || (MODE == HIF8_RND_HR && E > -4 && E < 4)) {
+        if (a >= 0x47200000u) r = top;                                                     // >= 1.25 * 2^15
+        else if (a < 0x34000000u) return 0u;                                               // < 2^-23: the single zero
+        else if (E < -22) r = 0x34800000u;                                                 // [2^-23, 2^-22) -> 2^-22
         else { const uint32_t k = 23u - (uint32_t)mant_width(E); r = (a + (1u << (k - 1))) & (0xFFFFFFFFu << k); }
+    } else {
+        const uint32_t T2 = 2u * (raw & 1u) + 1u;                                          // {source LSB, fixed 1}
+        if (a >= 0x47400000u) r = top;                                                     // >= 1.5 * 2^15
+        else if (E < -22) {                                                                // F = |y| / 2^-22, F2 = floor(4 F)
+            if ((uint32_t)floorf(fabsf(y) * 16777216.f) < T2) return 0u;
+            r = 0x34800000u;
+        } else {
+            const uint32_t k = 23u - (uint32_t)mant_width(E);
+            const uint32_t f2 = (a & ((1u << k) - 1u)) >> (k - 2);
+            r = (a & (0xFFFFFFFFu << k)) + ((f2 >= T2 ? 1u : 0u) << k);
+            if (r >= 0x47400000u) r = top;
+        }
     }
     const int da = (-se) / 2, db = -se - da;
     return to_bits<SRC>(__uint_as_float(r | sign) * pow2f(da) * pow2f(db));
 }
 
-template <int SRC>
+// MODE = round half away (FP32, BF16), or hybrid / simplified stochastic rounding (BF16 only: SR2 adds half * (3 - 2 lsb),
+// i.e. thresholds 0.25 / 0.75, where round-half-away adds half)
+template <int SRC, int MODE>
 __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, unsigned long long n_vec)
 {
+    static_assert(MODE == HIF8_RND_TA || SRC == HIF8_BF16, "threshold modes are done in place for BF16 only");
     constexpr int MB = SRC == HIF8_F32 ? 23 : 7;      // mantissa bits of the source format
     constexpr int PV = SrcTraits<SRC>::kPerVec;
     __shared__ uint32_t s_inc[256];                   // BF16: mask16 | inc16 << 16
@@ -477,9 +496,17 @@ __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, uns
         const int e = threadIdx.x, E = e - 127 + se;
         uint32_t inc = 0, mask = 0;
         if (e == 255 || (e == 0 && se > 100) || (e > 0 && E >= 15)) mask = kRareMask;
+        else if (MODE != HIF8_RND_TA && e > 0 && (E == -23 || E == -24)) mask = kRareMask;  // result is 0 or 2^-22
         else if (e == 0 || E <= -24) { inc = 0; mask = 0; }                                 // underflow to +0
         else if (E == -23) { inc = 1u << MB; mask = 0xFFFFFFFFu << MB; }                    // up to 2^-22
-        else { const uint32_t k = (uint32_t)(MB - mant_width(E)); inc = 1u << (k - 1); mask = 0xFFFFFFFFu << k; }
+        else {
+            const uint32_t k = (uint32_t)(MB - mant_width(E));
+            inc = 1u << (k - 1);
+            mask = 0xFFFFFFFFu << k;
+            // SR2 binades (every binade for SSR, |E| >= 4 for HR) hold a quarter of the discarded field instead of
+            // half of it, marked by bit 15: the increment is quarter * (4 - T2) = quarter * (3 - 2 lsb)
+            if (MODE == HIF8_RND_SSR || (MODE == HIF8_RND_HR && (E <= -4 || E >= 4))) inc = (1u << (k - 2)) | 0x8000u;
+        }
         if (SRC == HIF8_F32) { s_inc[e] = inc; s_mask[e] = mask; }
         else s_inc[e] = (mask & 0xFFFFu) | (inc << 16);
     }
@@ -511,7 +538,7 @@ __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, uns
                 if (rare & kRareMask) {
 #pragma unroll
                     for (int k = 0; k < 4; k++)
-                        if (m[k] == kRareMask) o[k] = fq_ta_rare<SRC>(w[k], se, p.flags);
+                        if (m[k] == kRareMask) o[k] = fq_rare<SRC, MODE>(w[k], se, p.flags);
                 }
             } else {
                 uint32_t tl[4], th[4];
@@ -519,15 +546,22 @@ __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, uns
                 for (int k = 0; k < 4; k++) {
                     tl[k] = s_inc[(w[k] >> 7) & 0xFFu];
                     th[k] = s_inc[(w[k] >> 23) & 0xFFu];
-                    const uint32_t mask2 = __byte_perm(tl[k], th[k], 0x5410), inc2 = __byte_perm(tl[k], th[k], 0x7632);
+                    const uint32_t mask2 = __byte_perm(tl[k], th[k], 0x5410);
+                    uint32_t inc2 = __byte_perm(tl[k], th[k], 0x7632);
+                    if (MODE != HIF8_RND_TA) {
+                        // SR2 lanes: increment = quarter * (3 - 2 lsb) = quarter + (2 quarter where the source LSB is 0)
+                        const uint32_t half2 = inc2 & 0x7FFF7FFFu;
+                        const uint32_t sr = ((inc2 >> 15) & 0x00010001u) * 0xFFFFu, odd = (w[k] & 0x00010001u) * 0xFFFFu;
+                        inc2 = half2 + ((half2 << 1) & sr & ~odd);
+                    }
                     o[k] = (w[k] + inc2) & mask2;  // no carry between the halves: flagged exponents add nothing
                     rare |= tl[k] | th[k];
                 }
                 if (rare & kRareMask) {
 #pragma unroll
                     for (int k = 0; k < 4; k++) {
-                        if (tl[k] & kRareMask) o[k] = (o[k] & 0xFFFF0000u) | fq_ta_rare<SRC>(w[k] & 0xFFFFu, se, p.flags);
-                        if (th[k] & kRareMask) o[k] = (o[k] & 0x0000FFFFu) | (fq_ta_rare<SRC>(w[k] >> 16, se, p.flags) << 16);
+                        if (tl[k] & kRareMask) o[k] = (o[k] & 0xFFFF0000u) | fq_rare<SRC, MODE>(w[k] & 0xFFFFu, se, p.flags);
+                        if (th[k] & kRareMask) o[k] = (o[k] & 0x0000FFFFu) | (fq_rare<SRC, MODE>(w[k] >> 16, se, p.flags) << 16);
                     }
                 }
             }
@@ -539,10 +573,10 @@ __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, uns
         for (unsigned long long i = n_vec * PV + tid; i < p.n; i += (unsigned long long)gridDim.x * kThreads) {
             if (SRC == HIF8_F32) {
                 const uint32_t raw = reinterpret_cast<const uint32_t*>(p.src)[i];
-                reinterpret_cast<uint32_t*>(p.dst)[i] = fq_ta_rare<SRC>(raw, se, p.flags);
+                reinterpret_cast<uint32_t*>(p.dst)[i] = fq_rare<SRC, MODE>(raw, se, p.flags);
             } else {
                 const uint32_t raw = reinterpret_cast<const unsigned short*>(p.src)[i];
-                reinterpret_cast<unsigned short*>(p.dst)[i] = (unsigned short)fq_ta_rare<SRC>(raw, se, p.flags);
+                reinterpret_cast<unsigned short*>(p.dst)[i] = (unsigned short)fq_rare<SRC, MODE>(raw, se, p.flags);
             }
         }
     }
@@ -720,13 +754,15 @@ int dispatch_convert(int dtype, int rnd, const ConvParams& p, bool vec_ok, int s
     }
 }
 
-int launch_fq_ta(int dtype, const ConvParams& p, bool vec_ok, int sms, cudaStream_t st)
+int launch_fq_ta(int dtype, int rnd, const ConvParams& p, bool vec_ok, int sms, cudaStream_t st)
 {
     const unsigned long long pv = dtype == HIF8_F32 ? 4 : 8;
     const unsigned long long n_vec = vec_ok ? p.n / pv : 0;
     const unsigned grid = grid_for(n_vec, p.n, sms);
-    if (dtype == HIF8_F32) fq_ta_kernel<HIF8_F32><<<grid, kThreads, 0, st>>>(p, n_vec);
-    else fq_ta_kernel<HIF8_BF16><<<grid, kThreads, 0, st>>>(p, n_vec);
+    if (dtype == HIF8_F32) fq_ta_kernel<HIF8_F32, HIF8_RND_TA><<<grid, kThreads, 0, st>>>(p, n_vec);
+    else if (rnd == HIF8_RND_TA) fq_ta_kernel<HIF8_BF16, HIF8_RND_TA><<<grid, kThreads, 0, st>>>(p, n_vec);
+    else if (rnd == HIF8_RND_HR) fq_ta_kernel<HIF8_BF16, HIF8_RND_HR><<<grid, kThreads, 0, st>>>(p, n_vec);
+    else fq_ta_kernel<HIF8_BF16, HIF8_RND_SSR><<<grid, kThreads, 0, st>>>(p, n_vec);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
 }
@@ -821,16 +857,17 @@ static int scaled_convert(bool fq, const void* src, void* dst, int dtype, size_t
         if (!ws || workspace_bytes < kConvWorkspaceBytes || (reinterpret_cast<uintptr_t>(ws) & 255u)) return HIF8_ERR_WORKSPACE;
         if (cudaMemsetAsync(ws, 0, 8, st) != cudaSuccess) return HIF8_ERR_CUDA;
     }
-    const bool inplace_fq = fq && rnd == HIF8_RND_TA && (dtype == HIF8_F32 || dtype == HIF8_BF16) && !want_amax;
+    const bool inplace_fq = fq && !want_amax && ((rnd == HIF8_RND_TA && (dtype == HIF8_F32 || dtype == HIF8_BF16)) ||
+                                                ((rnd == HIF8_RND_HR || rnd == HIF8_RND_SSR) && dtype == HIF8_BF16));
     if (jit) {
         rc = launch_amax(src, dtype, n, ws, nullptr, sms, st);
         if (rc) return rc;
         p.d_amax_bits = ws;
-        if (inplace_fq) return launch_fq_ta(dtype, p, vec_ok, sms, st);
+        if (inplace_fq) return launch_fq_ta(dtype, rnd, p, vec_ok, sms, st);
         return fq ? dispatch_convert<true, false>(dtype, rnd, p, vec_ok, sms, st)
                   : dispatch_convert<false, false>(dtype, rnd, p, vec_ok, sms, st);
     }
-    if (inplace_fq) return launch_fq_ta(dtype, p, vec_ok, sms, st);
+    if (inplace_fq) return launch_fq_ta(dtype, rnd, p, vec_ok, sms, st);
     if (want_amax) {
         p.amax_accum = ws;
         return fq ? dispatch_convert<true, true>(dtype, rnd, p, vec_ok, sms, st)
