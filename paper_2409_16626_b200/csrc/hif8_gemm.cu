@@ -12,9 +12,9 @@
 //
 // One CTA computes one 128 x 256 tile of C.  Warp roles:
 //   warps 0-3  epilogue: TMEM -> registers -> descale -> BF16 / FP32 -> global
-//   warp  4    TMA producer: HiF8 byte tiles (A: 128 x 64, W: 256 x 64 or 64 x 256) into a 4-stage staging ring
+//   warp  4    TMA producer: HiF8 byte tiles (A: 128 x 64, W: 256 x 64 or 64 x 256) into a 3-stage staging ring
 //   warp  5    MMA issuer: one elected thread issues tcgen05.mma (128 x 256 x 16, BF16 x BF16 -> FP32 in TMEM)
-//   warps 6-13 decode: staging bytes -> BF16 in the canonical 128-byte-swizzled operand layout (2-stage ring)
+//   warps 6-21 decode: staging bytes -> BF16 in the canonical 128-byte-swizzled operand layout (2-stage ring)
 // The operand layout follows the shared-memory matrix descriptor of tcgen05: K-major operands are rows of 64 BF16
 // (128 bytes), eight rows form a 1024-byte swizzle atom, 16-byte chunk j of row r is stored at chunk j ^ (r % 8).
 // W given as [K, N] is decoded in place as an MN-major operand (atoms of 8 k-rows x 64 n), so no transpose is needed.
@@ -36,10 +36,11 @@ extern std::atomic<uint64_t> g_launches;
 namespace {
 
 constexpr int BM = 128, BN = 256, BK = 64;
-constexpr int kStages8 = 4;    // staging ring of HiF8 byte tiles
+constexpr int kStages8 = 3;    // staging ring of HiF8 byte tiles
 constexpr int kStagesBf = 2;   // ring of decoded BF16 operand tiles
-constexpr int kEpiWarps = 4, kDecodeWarps = 8;
-constexpr int kThreads = (kEpiWarps + 2 + kDecodeWarps) * 32;  // 448
+constexpr int kEpiWarps = 4, kDecodeWarps = 16;
+constexpr int kDecodeThreads = kDecodeWarps * 32;
+constexpr int kThreads = (kEpiWarps + 2 + kDecodeWarps) * 32;  // 704
 constexpr int kTmaWarp = 4, kMmaWarp = 5, kFirstDecodeWarp = 6;
 constexpr uint32_t kA8Bytes = BM * BK, kB8Bytes = BN * BK;              // 8 KiB + 16 KiB
 constexpr uint32_t kABfBytes = BM * BK * 2, kBBfBytes = BN * BK * 2;    // 16 KiB + 32 KiB
@@ -50,7 +51,7 @@ struct SmemLayout {
     static constexpr uint32_t bf = 0;                                                  // 1024-byte aligned atoms
     static constexpr uint32_t u8 = bf + kStagesBf * (kABfBytes + kBBfBytes);           // 96 KiB
     static constexpr uint32_t lut = u8 + kStages8 * (kA8Bytes + kB8Bytes);             // + 96 KiB
-    static constexpr uint32_t bars = lut + 512;
+    static constexpr uint32_t bars = lut + 256 * 32 * 4;                                // lane-replicated table, 32 KiB
     static constexpr uint32_t n_bars = 2 * kStages8 + 2 * kStagesBf + 1;
     static constexpr uint32_t tmem_slot = bars + n_bars * 8;
     static constexpr uint32_t abort_flag = tmem_slot + 4;
@@ -178,15 +179,17 @@ __device__ __forceinline__ uint32_t hif8_to_bf16_bits(uint32_t c)
     return sign | ((uint32_t)(E + 127) << 7) | (M << (7 - w));
 }
 
-// eight HiF8 bytes -> eight BF16 (one 16-byte operand chunk)
-__device__ __forceinline__ uint4 decode8(uint2 v, const unsigned short* lut)
+// eight HiF8 bytes -> eight BF16 (one 16-byte operand chunk).  `lut_lane` points at this lane's column of the
+// lane-replicated table: entry of byte c is the 32-bit word at lut_lane[c * 32], so lane L only ever touches
+// shared-memory bank L and the eight lookups of a warp instruction never conflict.
+__device__ __forceinline__ uint4 decode8(uint2 v, const uint32_t* lut_lane)
 {
     uint32_t o[4];
 #pragma unroll
     for (int i = 0; i < 4; i++) {
-        uint32_t w = i < 2 ? v.x : v.y;
-        uint32_t c0 = (w >> (16 * (i & 1))) & 0xFFu, c1 = (w >> (16 * (i & 1) + 8)) & 0xFFu;
-        o[i] = (uint32_t)lut[c0] | ((uint32_t)lut[c1] << 16);
+        const uint32_t w = i < 2 ? v.x : v.y;
+        const uint32_t c0 = (w >> (16 * (i & 1))) & 0xFFu, c1 = (w >> (16 * (i & 1) + 8)) & 0xFFu;
+        o[i] = __byte_perm(lut_lane[c0 * 32], lut_lane[c1 * 32], 0x5410);
     }
     return make_uint4(o[0], o[1], o[2], o[3]);
 }
@@ -219,7 +222,8 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     const uint32_t bar_acc_full = bars + 8u * (2 * kStages8 + 2 * kStagesBf);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + SmemLayout::abort_flag);
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + SmemLayout::tmem_slot);
-    unsigned short* lut = reinterpret_cast<unsigned short*>(sm + SmemLayout::lut);
+    uint32_t* lut_all = reinterpret_cast<uint32_t*>(sm + SmemLayout::lut);
+    const uint32_t* lut = lut_all + lane;
 
     // tile of this CTA: groups of 8 tile-rows share their W tiles in L2
     constexpr int kGroupM = 8;
@@ -233,7 +237,7 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     const int num_kb = (p.K + BK - 1) / BK;
 
     // ---- set-up
-    if (threadIdx.x < 256) lut[threadIdx.x] = (unsigned short)hif8_to_bf16_bits(threadIdx.x);
+    for (int i = threadIdx.x; i < 256 * 32; i += kThreads) lut_all[i] = hif8_to_bf16_bits(i >> 5);
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages8; s++) { mbar_init(bar_u8_full(s), 1); mbar_init(bar_u8_empty(s), kDecodeWarps); }
         for (int s = 0; s < kStagesBf; s++) { mbar_init(bar_bf_full(s), kDecodeWarps); mbar_init(bar_bf_empty(s), 1); }
@@ -302,7 +306,7 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         }
     } else if (warp >= kFirstDecodeWarp) {
         // ------------------------------------------------------------------ decode warps
-        const int dt = threadIdx.x - kFirstDecodeWarp * 32;  // 0..255
+        const int dt = threadIdx.x - kFirstDecodeWarp * 32;  // 0..kDecodeThreads-1
         bool ok = true;
         for (int kb = 0; kb < num_kb && ok; kb++) {
             const int s8 = kb % kStages8, r8 = kb / kStages8, sb = kb % kStagesBf, rb = kb / kStagesBf;
@@ -315,23 +319,23 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             unsigned char* bbf = abf + kABfBytes;
             // A: 128 rows x 8 chunks of 8 codes; chunk j of row r -> atom r/8, row r%8, chunk j ^ (r%8)
 #pragma unroll
-            for (int it = 0; it < (BM * BK / 8) / 256; it++) {
-                const int q = it * 256 + dt, r = q >> 3, j = q & 7;
+            for (int it = 0; it < (BM * BK / 8) / kDecodeThreads; it++) {
+                const int q = it * kDecodeThreads + dt, r = q >> 3, j = q & 7;
                 const uint2 v = *reinterpret_cast<const uint2*>(a8 + r * BK + j * 8);
                 *reinterpret_cast<uint4*>(abf + (r >> 3) * 1024 + (r & 7) * 128 + ((j ^ (r & 7)) << 4)) = decode8(v, lut);
             }
             if (W_IS_NK) {
 #pragma unroll
-                for (int it = 0; it < (BN * BK / 8) / 256; it++) {
-                    const int q = it * 256 + dt, r = q >> 3, j = q & 7;
+                for (int it = 0; it < (BN * BK / 8) / kDecodeThreads; it++) {
+                    const int q = it * kDecodeThreads + dt, r = q >> 3, j = q & 7;
                     const uint2 v = *reinterpret_cast<const uint2*>(b8 + r * BK + j * 8);
                     *reinterpret_cast<uint4*>(bbf + (r >> 3) * 1024 + (r & 7) * 128 + ((j ^ (r & 7)) << 4)) = decode8(v, lut);
                 }
             } else {
                 // W tile is [64 k][256 n]: chunk (k, n/8) -> atom (n/64) * 8 + k/8, row k%8, chunk (n/8)%8 ^ (k%8)
 #pragma unroll
-                for (int it = 0; it < (BN * BK / 8) / 256; it++) {
-                    const int q = it * 256 + dt, k = q >> 5, jn = q & 31;
+                for (int it = 0; it < (BN * BK / 8) / kDecodeThreads; it++) {
+                    const int q = it * kDecodeThreads + dt, k = q >> 5, jn = q & 31;
                     const uint2 v = *reinterpret_cast<const uint2*>(b8 + k * BN + jn * 8);
                     const int atom = (jn >> 3) * 8 + (k >> 3);
                     *reinterpret_cast<uint4*>(bbf + atom * 1024 + (k & 7) * 128 + (((jn & 7) ^ (k & 7)) << 4)) = decode8(v, lut);
