@@ -5,7 +5,7 @@
 // Two paths behind one entry point.  The fused kernel (described next) needs no memory beyond its operands and
 // decodes the byte tiles of every CTA in shared memory; because every operand element is then decoded once per
 // tile that uses it, it is bound by the decode rate.  With a workspace large enough for both operands in BF16 the
-// call decodes each byte once (conversion kernel) and runs the BF16 tensor-core kernel further down.
+// call decodes each byte once (conversion kernel) and runs the BF16 CTA-pair tensor-core kernel further down.
 //
 // Every HiF8 value has at most 4 significant bits and an exponent in [-22, 15], so it is exact in BF16 and every
 // product of two of them is exact in the FP32 accumulator of the tensor core.
@@ -411,22 +411,12 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 
 // ---------------------------------------------------------------------------------------------------------
 // Decode-once path: operands already decoded to BF16 (by the conversion kernel of this library, into the caller's
-// workspace).  Persistent kernel, one CTA per SM, 128 x 256 tiles, 64-wide k-blocks.
+// workspace).  Persistent kernel, 64-wide k-blocks.
 //   warps 0-3  epilogue (TMEM -> global), overlapped with the next tile through two TMEM accumulators
-//   warp  4    TMA producer: BF16 tiles land directly in the 128-byte-swizzled operand layout (4-stage ring)
+//   warp  4    TMA producer: BF16 tiles land directly in the 128-byte-swizzled operand layout
 //   warp  5    MMA issuer
 // ---------------------------------------------------------------------------------------------------------
-constexpr int kStagesP = 4;
 constexpr int kThreadsP = 6 * 32;
-constexpr uint32_t kStageBytesP = kABfBytes + kBBfBytes;  // 48 KiB
-struct SmemLayoutP {
-    static constexpr uint32_t bars = kStagesP * kStageBytesP;           // 192 KiB
-    static constexpr uint32_t n_bars = 2 * kStagesP + 4;
-    static constexpr uint32_t tmem_slot = bars + n_bars * 8;
-    static constexpr uint32_t abort_flag = tmem_slot + 4;
-    static constexpr uint32_t total = abort_flag + 4;
-};
-constexpr uint32_t kSmemBytesP = SmemLayoutP::total + 1024;
 
 __device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int& tile_m, int& tile_n)
 {
@@ -438,116 +428,183 @@ __device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int
     tile_n = (t % per_group) / rows_in_group;
 }
 
+// ---------------------------------------------------------------------------------------------------------
+// Decode-once path, CTA pairs (cta_group::2).  A cluster of two CTAs on two SMs computes one 256 x 256 tile: each
+// CTA stages its own 128 rows of A and its own 128 columns of W (so the tensor core reads half as many operand bytes
+// per SM and flop as with one CTA per tile, which is what bounds the one-CTA kernel), both accumulate their 128 rows
+// in their own TMEM.  The even CTA of the pair (the leader) issues every tcgen05.mma; its commits arrive on the
+// barriers of both CTAs.  TMA copies of both CTAs complete on the leader's "full" barrier (no multicast loads).
+// ---------------------------------------------------------------------------------------------------------
+constexpr int kStages2 = 6;
+constexpr uint32_t kHalfBBytes = (BN / 2) * BK * 2;                   // 16 KiB: this CTA's half of the W tile
+constexpr uint32_t kStageBytes2 = kABfBytes + kHalfBBytes;            // 32 KiB per CTA and stage
+struct SmemLayout2 {
+    static constexpr uint32_t bars = kStages2 * kStageBytes2;         // 192 KiB
+    static constexpr uint32_t n_bars = 2 * kStages2 + 4;
+    static constexpr uint32_t tmem_slot = bars + n_bars * 8;
+    static constexpr uint32_t abort_flag = tmem_slot + 4;
+    static constexpr uint32_t total = abort_flag + 4;
+};
+constexpr uint32_t kSmemBytes2 = SmemLayout2::total + 1024;
+
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of `addr` (a shared::cta address of this CTA) in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// TMA tile load of a CTA pair: data into this CTA's shared memory, completion on a barrier that may live in the peer
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar_cluster)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar)  // arrives on `bar` in both CTAs of the pair
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
 template <bool W_IS_NK>
 __global__ void __launch_bounds__(kThreadsP, 1)
-bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const GemmParams p)
+bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const GemmParams p)
 {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* sm = smem_raw + (base - smem_u32(smem_raw));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t bars = base + SmemLayoutP::bars;
-    auto bar_full = [&](int s) { return bars + 8u * s; };
-    auto bar_empty = [&](int s) { return bars + 8u * (kStagesP + s); };
-    auto bar_acc_full = [&](int a) { return bars + 8u * (2 * kStagesP + a); };
-    auto bar_acc_empty = [&](int a) { return bars + 8u * (2 * kStagesP + 2 + a); };
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + SmemLayoutP::abort_flag);
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + SmemLayoutP::tmem_slot);
+    const uint32_t rank = cluster_ctarank();          // 0: leader (issues the MMAs), 1: peer
+    const bool leader = rank == 0;
+    const uint32_t bars = base + SmemLayout2::bars;
+    auto bar_full = [&](int s) { return bars + 8u * s; };                       // used in the leader only
+    auto bar_empty = [&](int s) { return bars + 8u * (kStages2 + s); };         // per CTA, released by the leader's commits
+    auto bar_acc_full = [&](int a) { return bars + 8u * (2 * kStages2 + a); };  // per CTA
+    auto bar_acc_empty = [&](int a) { return bars + 8u * (2 * kStages2 + 2 + a); };  // leader: both epilogues arrive
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + SmemLayout2::abort_flag);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + SmemLayout2::tmem_slot);
     const int num_kb = (p.K + BK - 1) / BK;
-    const int tiles = p.tiles_m * p.tiles_n;
+    const int tiles_m2 = (p.M + 2 * BM - 1) / (2 * BM), tiles_n2 = p.tiles_n;
+    const int tiles = tiles_m2 * tiles_n2, pairs = gridDim.x >> 1, pair_id = blockIdx.x >> 1;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStagesP; s++) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
-        for (int a = 0; a < 2; a++) { mbar_init(bar_acc_full(a), 1); mbar_init(bar_acc_empty(a), kEpiWarps); }
+        for (int s = 0; s < kStages2; s++) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
+        for (int a = 0; a < 2; a++) { mbar_init(bar_acc_full(a), 1); mbar_init(bar_acc_empty(a), 2 * kEpiWarps); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == kMmaWarp) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(base + SmemLayoutP::tmem_slot), "r"(512u) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(base + SmemLayout2::tmem_slot), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();   // barriers of both CTAs are initialised before anyone signals across
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == kTmaWarp) {
         if (lane == 0) {
-            long long it = 0, issued = 0;  // running k-block counter over all tiles of this CTA
+            long long it = 0, issued = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x) {
+            for (int t = pair_id; t < tiles && ok; t += pairs) {
                 int tile_m, tile_n;
-                tile_coords(t, p.tiles_m, p.tiles_n, tile_m, tile_n);
-                const int m0 = tile_m * BM, n0 = tile_n * BN;
+                tile_coords(t, tiles_m2, tiles_n2, tile_m, tile_n);
+                const int m0 = tile_m * 2 * BM + (int)rank * BM, n0 = tile_n * BN + (int)rank * (BN / 2);
                 for (int kb = 0; kb < num_kb; kb++, it++) {
-                    const int s = (int)(it % kStagesP);
-                    const long long round = it / kStagesP;
-                    if (round > 0) ok = mbar_wait(bar_empty(s), (uint32_t)((round - 1) & 1), abort_flag, p.status, 11);
+                    const int s = (int)(it % kStages2);
+                    const long long round = it / kStages2;
+                    if (round > 0) ok = mbar_wait(bar_empty(s), (uint32_t)((round - 1) & 1), abort_flag, p.status, 21);
                     if (!ok || *abort_flag) { ok = false; break; }
-                    const uint32_t dst_a = base + s * kStageBytesP, dst_b = dst_a + kABfBytes;
-                    mbar_arrive_expect_tx(bar_full(s), kStageBytesP);
-                    tma_load_2d(dst_a, &map_a, kb * BK, m0, bar_full(s));
-                    if (W_IS_NK) tma_load_2d(dst_b, &map_w, kb * BK, n0, bar_full(s));
+                    const uint32_t dst_a = base + s * kStageBytes2, dst_b = dst_a + kABfBytes;
+                    const uint32_t full = map_to_cta(bar_full(s), 0);
+                    if (leader) mbar_arrive_expect_tx(bar_full(s), 2 * kStageBytes2);  // bytes of both CTAs
+                    tma_load_2d_pair(dst_a, &map_a, kb * BK, m0, full);
+                    if (W_IS_NK) tma_load_2d_pair(dst_b, &map_w, kb * BK, n0, full);
                     else {
 #pragma unroll
-                        for (int c = 0; c < BN / 64; c++)  // four boxes of 64 k x 64 n: one 8-atom column each
-                            tma_load_2d(dst_b + c * 8192, &map_w, n0 + c * 64, kb * BK, bar_full(s));
+                        for (int c = 0; c < BN / 2 / 64; c++)
+                            tma_load_2d_pair(dst_b + c * 8192, &map_w, n0 + c * 64, kb * BK, full);
                     }
                     issued = it + 1;
                 }
             }
-            if (*abort_flag) {
-                for (long long j = issued > kStagesP ? issued - kStagesP : 0; j < issued; j++) {
+            if (*abort_flag && leader) {  // let copies in flight land (their completions are counted on the leader)
+                for (long long j = issued > kStages2 ? issued - kStages2 : 0; j < issued; j++) {
                     const unsigned long long t0 = global_ns();
-                    while (!mbar_try_wait(bar_full((int)(j % kStagesP)), (uint32_t)((j / kStagesP) & 1)) &&
+                    while (!mbar_try_wait(bar_full((int)(j % kStages2)), (uint32_t)((j / kStages2) & 1)) &&
                            global_ns() - t0 < kWaitLimitNs) {}
                 }
             }
         }
     } else if (warp == kMmaWarp) {
-        if (lane == 0) {
+        if (lane == 0 && leader) {
+            // M = 256 over the pair, N = 256
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((W_IS_NK ? 0u : 1u) << 16) |
-                                   ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+                                   ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
             long long it = 0;
             int local = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < tiles && ok; t += gridDim.x, local++) {
+            for (int t = pair_id; t < tiles && ok; t += pairs, local++) {
                 const int acc = local & 1, use = local >> 1;
-                if (use > 0) ok = mbar_wait(bar_acc_empty(acc), (uint32_t)((use - 1) & 1), abort_flag, p.status, 12);
+                if (use > 0) ok = mbar_wait(bar_acc_empty(acc), (uint32_t)((use - 1) & 1), abort_flag, p.status, 22);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * 256;
                 for (int kb = 0; kb < num_kb; kb++, it++) {
-                    const int s = (int)(it % kStagesP);
-                    ok = mbar_wait(bar_full(s), (uint32_t)((it / kStagesP) & 1), abort_flag, p.status, 13);
+                    const int s = (int)(it % kStages2);
+                    ok = mbar_wait(bar_full(s), (uint32_t)((it / kStages2) & 1), abort_flag, p.status, 23);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t a_addr = base + s * kStageBytesP, b_addr = a_addr + kABfBytes;
+                    const uint32_t a_addr = base + s * kStageBytes2, b_addr = a_addr + kABfBytes;
 #pragma unroll
                     for (int kk = 0; kk < BK / 16; kk++) {
                         const uint64_t da = make_smem_desc(a_addr + kk * 32, 16, 1024);
                         const uint64_t db = W_IS_NK ? make_smem_desc(b_addr + kk * 32, 16, 1024)
                                                     : make_smem_desc(b_addr + kk * 2048, 8192, 1024);
-                        tc_mma_bf16(d_tmem, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+                        tc_mma_bf16_pair(d_tmem, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
                     }
-                    tc_commit(bar_empty(s));
+                    tc_commit_pair(bar_empty(s));
                 }
-                if (ok) tc_commit(bar_acc_full(acc));
+                if (ok) tc_commit_pair(bar_acc_full(acc));
             }
         }
     } else if (warp < kEpiWarps) {
-        const int s = -((p.d_sa ? *p.d_sa : 0) + (p.d_sw ? *p.d_sw : 0));
-        const int s1 = s / 2, s2 = s - s1;
+        const int sdesc = -((p.d_sa ? *p.d_sa : 0) + (p.d_sw ? *p.d_sw : 0));
+        const int s1 = sdesc / 2, s2 = sdesc - s1;
         const float f1 = __uint_as_float((uint32_t)(s1 + 127) << 23), f2 = __uint_as_float((uint32_t)(s2 + 127) << 23);
         int local = 0;
-        for (int t = blockIdx.x; t < tiles; t += gridDim.x, local++) {
+        for (int t = pair_id; t < tiles; t += pairs, local++) {
             const int acc = local & 1, use = local >> 1;
-            if (!mbar_wait(bar_acc_full(acc), (uint32_t)(use & 1), abort_flag, p.status, 14)) break;
+            if (!mbar_wait(bar_acc_full(acc), (uint32_t)(use & 1), abort_flag, p.status, 24)) break;
             tc_fence_after();
             int tile_m, tile_n;
-            tile_coords(t, p.tiles_m, p.tiles_n, tile_m, tile_n);
-            const int row = tile_m * BM + warp * 32 + lane, n0 = tile_n * BN;
+            tile_coords(t, tiles_m2, tiles_n2, tile_m, tile_n);
+            const int row = tile_m * 2 * BM + (int)rank * BM + warp * 32 + lane, n0 = tile_n * BN;
 #pragma unroll 1
             for (int c = 0; c < BN; c += 32) {
                 uint32_t r[32];
@@ -588,18 +645,19 @@ bf16_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     }
                 }
             }
-            // this accumulator may be overwritten by the tile after next
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(bar_acc_empty(acc));
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(bar_acc_empty(acc), 0));  // tell the leader: accumulator drained
         }
     }
 
+    // nobody leaves while the other CTA may still read this CTA's shared memory or signal its barriers
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();
     if (warp == kMmaWarp) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
     }
 }
 
@@ -694,9 +752,9 @@ extern "C" int hif8_gemm(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int6
         if (attr_rc == cudaSuccess)
             attr_rc = cudaFuncSetAttribute(hif8_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (attr_rc == cudaSuccess)
-            attr_rc = cudaFuncSetAttribute(bf16_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytesP);
+            attr_rc = cudaFuncSetAttribute(bf16_gemm_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
         if (attr_rc == cudaSuccess)
-            attr_rc = cudaFuncSetAttribute(bf16_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytesP);
+            attr_rc = cudaFuncSetAttribute(bf16_gemm_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
         if (attr_rc == cudaSuccess) attr_rc = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
     });
     if (attr_rc != cudaSuccess || sm_count <= 0) return HIF8_ERR_CUDA;
@@ -717,11 +775,25 @@ extern "C" int hif8_gemm(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int6
         const bool okw = w_is_nk ? make_map(&mw, w_bf, (uint64_t)K, (uint64_t)N, (uint64_t)K, BK, BN, true)
                                  : make_map(&mw, w_bf, (uint64_t)N, (uint64_t)K, (uint64_t)N, 64, BK, true);
         if (!okw) return HIF8_ERR_CUDA;
-        const unsigned grid = (unsigned)(tiles < sm_count ? tiles : sm_count);
-        if (w_is_nk) bf16_gemm_kernel<true><<<grid, kThreadsP, kSmemBytesP, st>>>(ma, mw, p);
-        else bf16_gemm_kernel<false><<<grid, kThreadsP, kSmemBytesP, st>>>(ma, mw, p);
+        // CTA pairs: 256 x 256 tiles; W boxes are this CTA's half (128 columns / rows)
+        CUtensorMap mw2;
+        const bool okw2 = w_is_nk ? make_map(&mw2, w_bf, (uint64_t)K, (uint64_t)N, (uint64_t)K, BK, BN / 2, true) : true;
+        if (!okw2) return HIF8_ERR_CUDA;
+        const long long tiles2 = (long long)((M + 2 * BM - 1) / (2 * BM)) * p.tiles_n;
+        const int pairs = (int)(tiles2 < sm_count / 2 ? tiles2 : sm_count / 2);
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3(2u * (unsigned)pairs);
+        cfg.blockDim = dim3(kThreadsP);
+        cfg.dynamicSmemBytes = kSmemBytes2;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        cudaError_t lrc = w_is_nk ? cudaLaunchKernelEx(&cfg, bf16_gemm_pair_kernel<true>, ma, mw2, p)
+                                  : cudaLaunchKernelEx(&cfg, bf16_gemm_pair_kernel<false>, ma, mw, p);
         g_launches.fetch_add(1, std::memory_order_relaxed);
-        return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
+        return (lrc == cudaSuccess && cudaGetLastError() == cudaSuccess) ? HIF8_OK : HIF8_ERR_CUDA;
     }
 
     if (w_is_nk) hif8_gemm_kernel<true><<<(unsigned)tiles, kThreads, kSmemBytes, st>>>(map_a, map_w, p);
