@@ -10,11 +10,13 @@
 // Every HiF8 value has at most 4 significant bits and an exponent in [-22, 15], so it is exact in BF16 and every
 // product of two of them is exact in the FP32 accumulator of the tensor core.
 //
-// One CTA computes one 128 x 256 tile of C.  Warp roles:
+// A pair of CTAs (cluster of two, cta_group::2) computes one 256 x 256 tile of C: each CTA stages and decodes its
+// own 128 rows of A and 128 columns of W, the even CTA issues the MMAs for both.  Warp roles per CTA:
 //   warps 0-3  epilogue: TMEM -> registers -> descale -> BF16 / FP32 -> global
-//   warp  4    TMA producer: HiF8 byte tiles (A: 128 x 64, W: 256 x 64 or 64 x 256) into a 3-stage staging ring
-//   warp  5    MMA issuer: one elected thread issues tcgen05.mma (128 x 256 x 16, BF16 x BF16 -> FP32 in TMEM)
-//   warps 6-21 decode: staging bytes -> BF16 in the canonical 128-byte-swizzled operand layout (2-stage ring)
+//   warp  4    TMA producer: HiF8 byte tiles (A: 128 x 64, W: 128 x 64 or 64 x 128) into a 4-stage staging ring
+//   warp  5    MMA issuer: one elected thread of the even CTA issues tcgen05.mma (256 x 256 x 16 over the pair,
+//              BF16 x BF16 -> FP32 in the TMEM of both CTAs)
+//   warps 6-21 decode: staging bytes -> BF16 in the canonical 128-byte-swizzled operand layout (3-stage ring)
 // The operand layout follows the shared-memory matrix descriptor of tcgen05: K-major operands are rows of 64 BF16
 // (128 bytes), eight rows form a 1024-byte swizzle atom, 16-byte chunk j of row r is stored at chunk j ^ (r % 8).
 // W given as [K, N] is decoded in place as an MN-major operand (atoms of 8 k-rows x 64 n), so no transpose is needed.
@@ -36,21 +38,22 @@ extern std::atomic<uint64_t> g_launches;
 namespace {
 
 constexpr int BM = 128, BN = 256, BK = 64;
-constexpr int kStages8 = 3;    // staging ring of HiF8 byte tiles
-constexpr int kStagesBf = 2;   // ring of decoded BF16 operand tiles
+constexpr int kStages8 = 4;    // staging ring of HiF8 byte tiles
+constexpr int kStagesBf = 3;   // ring of decoded BF16 operand tiles
 constexpr int kEpiWarps = 4, kDecodeWarps = 16;
 constexpr int kDecodeThreads = kDecodeWarps * 32;
 constexpr int kThreads = (kEpiWarps + 2 + kDecodeWarps) * 32;  // 704
 constexpr int kTmaWarp = 4, kMmaWarp = 5, kFirstDecodeWarp = 6;
-constexpr uint32_t kA8Bytes = BM * BK, kB8Bytes = BN * BK;              // 8 KiB + 16 KiB
-constexpr uint32_t kABfBytes = BM * BK * 2, kBBfBytes = BN * BK * 2;    // 16 KiB + 32 KiB
+// per CTA of a pair: 128 rows of A and 128 of the 256 columns of W
+constexpr uint32_t kA8Bytes = BM * BK, kB8Bytes = (BN / 2) * BK;            // 8 KiB + 8 KiB
+constexpr uint32_t kABfBytes = BM * BK * 2, kBBfBytes = (BN / 2) * BK * 2;  // 16 KiB + 16 KiB
 constexpr uint32_t kTmemCols = 256;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
 
 struct SmemLayout {
     static constexpr uint32_t bf = 0;                                                  // 1024-byte aligned atoms
     static constexpr uint32_t u8 = bf + kStagesBf * (kABfBytes + kBBfBytes);           // 96 KiB
-    static constexpr uint32_t lut = u8 + kStages8 * (kA8Bytes + kB8Bytes);             // + 96 KiB
+    static constexpr uint32_t lut = u8 + kStages8 * (kA8Bytes + kB8Bytes);             // + 64 KiB
     static constexpr uint32_t bars = lut + 256 * 32 * 4;                                // lane-replicated table, 32 KiB
     static constexpr uint32_t n_bars = 2 * kStages8 + 2 * kStagesBf + 1;
     static constexpr uint32_t tmem_slot = bars + n_bars * 8;
@@ -150,6 +153,50 @@ __device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t (&r)
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// ---- CTA pairs (cluster of two CTAs, cta_group::2)
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of `addr` (a shared::cta address of this CTA) in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// TMA tile load of a CTA pair: data into this CTA's shared memory, completion on a barrier that may live in the peer
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar_cluster)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar)  // arrives on `bar` in both CTAs of the pair
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+
 // shared-memory matrix descriptor: start address, leading / stride byte offsets (16-byte units), version 1,
 // 128-byte swizzle
 __device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes)
@@ -194,6 +241,16 @@ __device__ __forceinline__ uint4 decode8(uint2 v, const uint32_t* lut_lane)
     return make_uint4(o[0], o[1], o[2], o[3]);
 }
 
+__device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int& tile_m, int& tile_n)
+{
+    constexpr int kGroupM = 8;  // groups of 8 tile-rows sweep N together: their W tiles stay in L2
+    const int per_group = kGroupM * tiles_n;
+    const int g = t / per_group, first_m = g * kGroupM;
+    const int rows_in_group = min(kGroupM, tiles_m - first_m);
+    tile_m = first_m + (t % per_group) % rows_in_group;
+    tile_n = (t % per_group) / rows_in_group;
+}
+
 struct GemmParams {
     void* C;
     long long ldc;
@@ -213,50 +270,48 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* sm = smem_raw + (base - smem_u32(smem_raw));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();  // 0: leader of the pair (issues the MMAs), 1: peer
+    const bool leader = rank == 0;
 
     const uint32_t bars = base + SmemLayout::bars;
-    auto bar_u8_full = [&](int s) { return bars + 8u * s; };
-    auto bar_u8_empty = [&](int s) { return bars + 8u * (kStages8 + s); };
-    auto bar_bf_full = [&](int s) { return bars + 8u * (2 * kStages8 + s); };
-    auto bar_bf_empty = [&](int s) { return bars + 8u * (2 * kStages8 + kStagesBf + s); };
-    const uint32_t bar_acc_full = bars + 8u * (2 * kStages8 + 2 * kStagesBf);
+    auto bar_u8_full = [&](int s) { return bars + 8u * s; };                                   // per CTA
+    auto bar_u8_empty = [&](int s) { return bars + 8u * (kStages8 + s); };                     // per CTA
+    auto bar_bf_full = [&](int s) { return bars + 8u * (2 * kStages8 + s); };                  // leader: both CTAs' decode warps
+    auto bar_bf_empty = [&](int s) { return bars + 8u * (2 * kStages8 + kStagesBf + s); };     // per CTA, leader's commits
+    const uint32_t bar_acc_full = bars + 8u * (2 * kStages8 + 2 * kStagesBf);                  // per CTA, leader's commit
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + SmemLayout::abort_flag);
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + SmemLayout::tmem_slot);
     uint32_t* lut_all = reinterpret_cast<uint32_t*>(sm + SmemLayout::lut);
     const uint32_t* lut = lut_all + lane;
 
-    // tile of this CTA: groups of 8 tile-rows share their W tiles in L2
-    constexpr int kGroupM = 8;
-    const int t = blockIdx.x;
-    const int per_group = kGroupM * p.tiles_n;
-    const int g = t / per_group, first_m = g * kGroupM;
-    const int rows_in_group = min(kGroupM, p.tiles_m - first_m);
-    const int tile_m = first_m + (t % per_group) % rows_in_group;
-    const int tile_n = (t % per_group) / rows_in_group;
-    const int m0 = tile_m * BM, n0 = tile_n * BN;
+    // 256 x 256 tile of this pair (groups of 8 tile-rows share their W tiles in L2); this CTA: 128 rows, 128 columns of W
+    int tile_m, tile_n;
+    tile_coords((int)(blockIdx.x >> 1), (p.M + 2 * BM - 1) / (2 * BM), p.tiles_n, tile_m, tile_n);
+    const int m0 = tile_m * 2 * BM + (int)rank * BM, n0 = tile_n * BN, nh = n0 + (int)rank * (BN / 2);
     const int num_kb = (p.K + BK - 1) / BK;
 
     // ---- set-up
     for (int i = threadIdx.x; i < 256 * 32; i += kThreads) lut_all[i] = hif8_to_bf16_bits(i >> 5);
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages8; s++) { mbar_init(bar_u8_full(s), 1); mbar_init(bar_u8_empty(s), kDecodeWarps); }
-        for (int s = 0; s < kStagesBf; s++) { mbar_init(bar_bf_full(s), kDecodeWarps); mbar_init(bar_bf_empty(s), 1); }
+        for (int s = 0; s < kStagesBf; s++) { mbar_init(bar_bf_full(s), 2 * kDecodeWarps); mbar_init(bar_bf_empty(s), 1); }
         mbar_init(bar_acc_full, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == kMmaWarp) {  // this warp owns the TMEM allocation
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+    if (warp == kMmaWarp) {  // this warp owns the TMEM allocation (both CTAs of the pair take part)
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(base + SmemLayout::tmem_slot), "r"(kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();  // barriers of both CTAs exist before anyone signals across
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == kTmaWarp) {
-        // ------------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------------ TMA producer (each CTA feeds itself)
         if (lane == 0) {
             int issued = 0;
             for (int kb = 0; kb < num_kb; kb++) {
@@ -266,8 +321,8 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 const uint32_t dst_a = base + SmemLayout::u8 + s * (kA8Bytes + kB8Bytes), dst_b = dst_a + kA8Bytes;
                 mbar_arrive_expect_tx(bar_u8_full(s), kA8Bytes + kB8Bytes);
                 tma_load_2d(dst_a, &map_a, kb * BK, m0, bar_u8_full(s));
-                if (W_IS_NK) tma_load_2d(dst_b, &map_w, kb * BK, n0, bar_u8_full(s));
-                else tma_load_2d(dst_b, &map_w, n0, kb * BK, bar_u8_full(s));
+                if (W_IS_NK) tma_load_2d(dst_b, &map_w, kb * BK, nh, bar_u8_full(s));
+                else tma_load_2d(dst_b, &map_w, nh, kb * BK, bar_u8_full(s));
                 issued = kb + 1;
             }
             if (*abort_flag) {
@@ -280,11 +335,11 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             }
         }
     } else if (warp == kMmaWarp) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            // instruction descriptor: FP32 accumulator, BF16 A and B, A K-major, B K- or MN-major, N, M
+        // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (lane == 0 && leader) {
+            // instruction descriptor: FP32 accumulator, BF16 A and B, A K-major, B K- or MN-major, N = 256, M = 256 (pair)
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((W_IS_NK ? 0u : 1u) << 16) |
-                                   ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+                                   ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
             bool ok = true;
             for (int kb = 0; kb < num_kb && ok; kb++) {
                 const int s = kb % kStagesBf, round = kb / kStagesBf;
@@ -298,11 +353,11 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     const uint64_t da = make_smem_desc(a_addr + kk * 32, 16, 1024);
                     const uint64_t db = W_IS_NK ? make_smem_desc(b_addr + kk * 32, 16, 1024)
                                                 : make_smem_desc(b_addr + kk * 2048, 8192, 1024);
-                    tc_mma_bf16(tmem_base, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+                    tc_mma_bf16_pair(tmem_base, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
                 }
-                tc_commit(bar_bf_empty(s));  // frees this operand stage once the MMAs above have read it
+                tc_commit_pair(bar_bf_empty(s));  // frees this operand stage in both CTAs once the MMAs have read it
             }
-            if (ok) tc_commit(bar_acc_full);
+            if (ok) tc_commit_pair(bar_acc_full);
         }
     } else if (warp >= kFirstDecodeWarp) {
         // ------------------------------------------------------------------ decode warps
@@ -326,17 +381,17 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             }
             if (W_IS_NK) {
 #pragma unroll
-                for (int it = 0; it < (BN * BK / 8) / kDecodeThreads; it++) {
+                for (int it = 0; it < ((BN / 2) * BK / 8) / kDecodeThreads; it++) {
                     const int q = it * kDecodeThreads + dt, r = q >> 3, j = q & 7;
                     const uint2 v = *reinterpret_cast<const uint2*>(b8 + r * BK + j * 8);
                     *reinterpret_cast<uint4*>(bbf + (r >> 3) * 1024 + (r & 7) * 128 + ((j ^ (r & 7)) << 4)) = decode8(v, lut);
                 }
             } else {
-                // W tile is [64 k][256 n]: chunk (k, n/8) -> atom (n/64) * 8 + k/8, row k%8, chunk (n/8)%8 ^ (k%8)
+                // W tile is [64 k][128 n]: chunk (k, n/8) -> atom (n/64) * 8 + k/8, row k%8, chunk (n/8)%8 ^ (k%8)
 #pragma unroll
-                for (int it = 0; it < (BN * BK / 8) / kDecodeThreads; it++) {
-                    const int q = it * kDecodeThreads + dt, k = q >> 5, jn = q & 31;
-                    const uint2 v = *reinterpret_cast<const uint2*>(b8 + k * BN + jn * 8);
+                for (int it = 0; it < ((BN / 2) * BK / 8) / kDecodeThreads; it++) {
+                    const int q = it * kDecodeThreads + dt, k = q >> 4, jn = q & 15;
+                    const uint2 v = *reinterpret_cast<const uint2*>(b8 + k * (BN / 2) + jn * 8);
                     const int atom = (jn >> 3) * 8 + (k >> 3);
                     *reinterpret_cast<uint4*>(bbf + atom * 1024 + (k & 7) * 128 + (((jn & 7) ^ (k & 7)) << 4)) = decode8(v, lut);
                 }
@@ -345,11 +400,11 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(bar_u8_empty(s8));
-                mbar_arrive(bar_bf_full(sb));
+                mbar_arrive_cluster(map_to_cta(bar_bf_full(sb), 0));  // the leader's MMAs read both CTAs' operands
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue warps 0-3
+        // ------------------------------------------------------------------ epilogue warps 0-3 (each CTA drains its rows)
         const bool ok = mbar_wait(bar_acc_full, 0, abort_flag, p.status, 5);
         if (ok) {
             tc_fence_after();
@@ -400,12 +455,14 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         }
     }
 
-    // ---- teardown: everybody arrives here (all waits are bounded), then the allocating warp frees TMEM
+    // ---- teardown: all waits are bounded, so everybody arrives; nobody leaves while the peer may still read this
+    // CTA's operands or signal its barriers; then the allocating warps free TMEM
     tc_fence_before();
     __syncthreads();
+    cluster_sync_all();
     if (warp == kMmaWarp) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
 }
 
@@ -418,15 +475,6 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 // ---------------------------------------------------------------------------------------------------------
 constexpr int kThreadsP = 6 * 32;
 
-__device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int& tile_m, int& tile_n)
-{
-    constexpr int kGroupM = 8;  // groups of 8 tile-rows sweep N together: their W tiles stay in L2
-    const int per_group = kGroupM * tiles_n;
-    const int g = t / per_group, first_m = g * kGroupM;
-    const int rows_in_group = min(kGroupM, tiles_m - first_m);
-    tile_m = first_m + (t % per_group) % rows_in_group;
-    tile_n = (t % per_group) / rows_in_group;
-}
 
 // ---------------------------------------------------------------------------------------------------------
 // Decode-once path, CTA pairs (cta_group::2).  A cluster of two CTAs on two SMs computes one 256 x 256 tile: each
@@ -436,8 +484,7 @@ __device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int
 // barriers of both CTAs.  TMA copies of both CTAs complete on the leader's "full" barrier (no multicast loads).
 // ---------------------------------------------------------------------------------------------------------
 constexpr int kStages2 = 6;
-constexpr uint32_t kHalfBBytes = (BN / 2) * BK * 2;                   // 16 KiB: this CTA's half of the W tile
-constexpr uint32_t kStageBytes2 = kABfBytes + kHalfBBytes;            // 32 KiB per CTA and stage
+constexpr uint32_t kStageBytes2 = kABfBytes + kBBfBytes;            // 32 KiB per CTA and stage
 struct SmemLayout2 {
     static constexpr uint32_t bars = kStages2 * kStageBytes2;         // 192 KiB
     static constexpr uint32_t n_bars = 2 * kStages2 + 4;
@@ -446,48 +493,6 @@ struct SmemLayout2 {
     static constexpr uint32_t total = abort_flag + 4;
 };
 constexpr uint32_t kSmemBytes2 = SmemLayout2::total + 1024;
-
-__device__ __forceinline__ uint32_t cluster_ctarank()
-{
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-// shared::cluster address of `addr` (a shared::cta address of this CTA) in CTA `rank` of the cluster
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank)
-{
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
-{
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
-__device__ __forceinline__ void cluster_sync_all()
-{
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// TMA tile load of a CTA pair: data into this CTA's shared memory, completion on a barrier that may live in the peer
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar_cluster)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(c0), "r"(c1) : "memory");
-}
-__device__ __forceinline__ void tc_commit_pair(uint32_t bar)  // arrives on `bar` in both CTAs of the pair
-{
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 ::"r"(bar), "h"((unsigned short)3) : "memory");
-}
-__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
 
 template <bool W_IS_NK>
 __global__ void __launch_bounds__(kThreadsP, 1)
@@ -731,16 +736,18 @@ extern "C" int hif8_gemm(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int6
 
     CUtensorMap map_a, map_w;
     if (!make_map(&map_a, Aq, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BK, BM)) return HIF8_ERR_CUDA;
-    const bool ok_w = w_is_nk ? make_map(&map_w, Wq, (uint64_t)K, (uint64_t)N, (uint64_t)ldw, BK, BN)
-                              : make_map(&map_w, Wq, (uint64_t)N, (uint64_t)K, (uint64_t)ldw, BN, BK);
+    // byte tiles of one CTA of a pair: 128 rows of A, 128 of the 256 columns of W
+    const bool ok_w = w_is_nk ? make_map(&map_w, Wq, (uint64_t)K, (uint64_t)N, (uint64_t)ldw, BK, BN / 2)
+                              : make_map(&map_w, Wq, (uint64_t)N, (uint64_t)K, (uint64_t)ldw, BN / 2, BK);
     if (!ok_w) return HIF8_ERR_CUDA;
 
     GemmParams p{};
     p.C = C; p.ldc = ldc; p.c_is_f32 = c_dtype == HIF8_F32; p.M = M; p.N = N; p.K = K;
     p.d_sa = d_scale_exp_a; p.d_sw = d_scale_exp_w; p.status = reinterpret_cast<int*>(workspace);
     p.tiles_m = (M + BM - 1) / BM; p.tiles_n = (N + BN - 1) / BN;
-    const long long tiles = (long long)p.tiles_m * p.tiles_n;
-    if (tiles > 0x7FFFFFFF) return HIF8_ERR_SHAPE;
+    // both kernels work on 256 x 256 tiles, one per pair of CTAs
+    const long long tiles2 = (long long)((M + 2 * BM - 1) / (2 * BM)) * p.tiles_n;
+    if (tiles2 > 0x3FFFFFFF) return HIF8_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMemsetAsync(workspace, 0, 4, st) != cudaSuccess) return HIF8_ERR_CUDA;
 
@@ -779,7 +786,6 @@ extern "C" int hif8_gemm(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int6
         CUtensorMap mw2;
         const bool okw2 = w_is_nk ? make_map(&mw2, w_bf, (uint64_t)K, (uint64_t)N, (uint64_t)K, BK, BN / 2, true) : true;
         if (!okw2) return HIF8_ERR_CUDA;
-        const long long tiles2 = (long long)((M + 2 * BM - 1) / (2 * BM)) * p.tiles_n;
         const int pairs = (int)(tiles2 < sm_count / 2 ? tiles2 : sm_count / 2);
         cudaLaunchConfig_t cfg{};
         cfg.gridDim = dim3(2u * (unsigned)pairs);
@@ -796,10 +802,19 @@ extern "C" int hif8_gemm(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int6
         return (lrc == cudaSuccess && cudaGetLastError() == cudaSuccess) ? HIF8_OK : HIF8_ERR_CUDA;
     }
 
-    if (w_is_nk) hif8_gemm_kernel<true><<<(unsigned)tiles, kThreads, kSmemBytes, st>>>(map_a, map_w, p);
-    else hif8_gemm_kernel<false><<<(unsigned)tiles, kThreads, kSmemBytes, st>>>(map_a, map_w, p);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(2u * (unsigned)tiles2);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    const cudaError_t lrc = w_is_nk ? cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<true>, map_a, map_w, p)
+                                    : cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<false>, map_a, map_w, p);
     g_launches.fetch_add(1, std::memory_order_relaxed);
-    return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
+    return (lrc == cudaSuccess && cudaGetLastError() == cudaSuccess) ? HIF8_OK : HIF8_ERR_CUDA;
 }
 
 extern "C" int hif8_gemm_status(const void* workspace, hif8_stream_t stream)
