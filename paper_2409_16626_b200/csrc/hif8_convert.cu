@@ -123,6 +123,15 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
 }
 
 // ------------------------------------------------------------------------------------------------
+// Programmatic dependent launch.  Every kernel here is launched so that it may be scheduled while the previous
+// kernel of the stream is still draining: it signals its own dependents at once (they can only start after all of
+// this grid's blocks have started), does the work that touches no global input (table set-up), and waits for the
+// previous grid to have completed and flushed before its first global read or write.
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait_prior_grid() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// ------------------------------------------------------------------------------------------------
 // Scale handling
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ int clamp_exp(int e) { return e < -126 ? -126 : (e > 126 ? 126 : e); }
@@ -339,7 +348,9 @@ template <int SRC, int MODE, bool FQ, bool AMAX>
 __global__ void __launch_bounds__(kThreads) convert_kernel(const ConvParams p, unsigned long long n_vec)
 {
     __shared__ SmemTables sm;
-    setup_tables<true, MODE != HIF8_RND_TA, FQ>(sm, p.flags);
+    pdl_launch_dependents();
+    setup_tables<true, MODE != HIF8_RND_TA, FQ>(sm, p.flags);  // reads only the constant table
+    pdl_wait_prior_grid();
     const int se = resolve_scale_exp(p);
     const float scale = pow2f(se);
     const int da = (-se) / 2, db = -se - da;  // descale in two exact steps (the first cannot leave the normal range)
@@ -491,6 +502,8 @@ __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, uns
     constexpr int PV = SrcTraits<SRC>::kPerVec;
     __shared__ uint32_t s_inc[256];                   // BF16: mask16 | inc16 << 16
     __shared__ uint32_t s_mask[SRC == HIF8_F32 ? 256 : 1];
+    pdl_launch_dependents();
+    pdl_wait_prior_grid();  // the scale may come from the previous kernel
     const int se = resolve_scale_exp(p);
     {
         const int e = threadIdx.x, E = e - 127 + se;
@@ -595,6 +608,8 @@ __global__ void __launch_bounds__(kThreads) amax_kernel(const void* __restrict__
     constexpr int PV = SrcTraits<SRC>::kPerVec;
     const uint4* src = reinterpret_cast<const uint4*>(srcv);
     float amax = 0.f;
+    pdl_launch_dependents();
+    pdl_wait_prior_grid();
     const unsigned long long stride = (unsigned long long)gridDim.x * kThreads * kUnroll;
     for (unsigned long long base = (unsigned long long)blockIdx.x * kThreads * kUnroll; base < n_vec; base += stride) {
         uint4 v[kUnroll];
@@ -639,11 +654,13 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const uint8_t* __restr
     // Output encodings of all 256 bytes for this call: value * 2^-scale_exp in two exact power-of-two steps (the first
     // cannot leave the normal range, so only the second may round -- to nearest even), then the destination format.
     __shared__ uint32_t s_out[256];
+    pdl_launch_dependents();
     {
         const int da = (-se) / 2, db = -se - da;
         s_out[threadIdx.x] = to_bits<DT>(__uint_as_float(decode_bits_f32(threadIdx.x)) * pow2f(da) * pow2f(db));
     }
     __syncthreads();
+    pdl_wait_prior_grid();
     constexpr int PV = SrcTraits<DT>::kPerVec;  // codes per 16-byte store
     const unsigned long long stride = (unsigned long long)gridDim.x * kThreads * kUnroll;
     for (unsigned long long base = (unsigned long long)blockIdx.x * kThreads * kUnroll; base < n_vec; base += stride) {
@@ -701,6 +718,23 @@ int device_info(int* sms)
     return HIF8_OK;
 }
 
+// launch with programmatic stream serialization (see pdl_* above)
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), unsigned grid, cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 unsigned grid_for(unsigned long long n_vec, unsigned long long n, int sms)
@@ -727,7 +761,7 @@ int launch_convert(const ConvParams& p, bool vec_ok, int sms, cudaStream_t st)
     constexpr int PV = SrcTraits<SRC>::kPerVec;
     unsigned long long n_vec = vec_ok ? p.n / PV : 0;
     unsigned grid = grid_for(n_vec, p.n, sms);
-    convert_kernel<SRC, MODE, FQ, AMAX><<<grid, kThreads, 0, st>>>(p, n_vec);
+    launch_pdl(convert_kernel<SRC, MODE, FQ, AMAX>, grid, st, p, n_vec);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
 }
@@ -759,10 +793,10 @@ int launch_fq_ta(int dtype, int rnd, const ConvParams& p, bool vec_ok, int sms, 
     const unsigned long long pv = dtype == HIF8_F32 ? 4 : 8;
     const unsigned long long n_vec = vec_ok ? p.n / pv : 0;
     const unsigned grid = grid_for(n_vec, p.n, sms);
-    if (dtype == HIF8_F32) fq_ta_kernel<HIF8_F32, HIF8_RND_TA><<<grid, kThreads, 0, st>>>(p, n_vec);
-    else if (rnd == HIF8_RND_TA) fq_ta_kernel<HIF8_BF16, HIF8_RND_TA><<<grid, kThreads, 0, st>>>(p, n_vec);
-    else if (rnd == HIF8_RND_HR) fq_ta_kernel<HIF8_BF16, HIF8_RND_HR><<<grid, kThreads, 0, st>>>(p, n_vec);
-    else fq_ta_kernel<HIF8_BF16, HIF8_RND_SSR><<<grid, kThreads, 0, st>>>(p, n_vec);
+    if (dtype == HIF8_F32) launch_pdl(fq_ta_kernel<HIF8_F32, HIF8_RND_TA>, grid, st, p, n_vec);
+    else if (rnd == HIF8_RND_TA) launch_pdl(fq_ta_kernel<HIF8_BF16, HIF8_RND_TA>, grid, st, p, n_vec);
+    else if (rnd == HIF8_RND_HR) launch_pdl(fq_ta_kernel<HIF8_BF16, HIF8_RND_HR>, grid, st, p, n_vec);
+    else launch_pdl(fq_ta_kernel<HIF8_BF16, HIF8_RND_SSR>, grid, st, p, n_vec);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
 }
@@ -774,9 +808,9 @@ int launch_amax(const void* src, int dtype, unsigned long long n, uint32_t* accu
     unsigned long long n_vec = vec_ok ? n / pv : 0;
     unsigned grid = grid_for(n_vec, n, sms);
     switch (dtype) {
-        case HIF8_F32: amax_kernel<HIF8_F32><<<grid, kThreads, 0, st>>>(src, n, n_vec, accum, d_amax_out); break;
-        case HIF8_BF16: amax_kernel<HIF8_BF16><<<grid, kThreads, 0, st>>>(src, n, n_vec, accum, d_amax_out); break;
-        default: amax_kernel<HIF8_F16><<<grid, kThreads, 0, st>>>(src, n, n_vec, accum, d_amax_out); break;
+        case HIF8_F32: launch_pdl(amax_kernel<HIF8_F32>, grid, st, src, n, n_vec, accum, d_amax_out); break;
+        case HIF8_BF16: launch_pdl(amax_kernel<HIF8_BF16>, grid, st, src, n, n_vec, accum, d_amax_out); break;
+        default: launch_pdl(amax_kernel<HIF8_F16>, grid, st, src, n, n_vec, accum, d_amax_out); break;
     }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
@@ -830,9 +864,9 @@ int hif8_decode(const uint8_t* src, void* dst, int dst_dtype, size_t n, int scal
     unsigned grid = grid_for(n_vec, n, sms);
     cudaStream_t st = (cudaStream_t)stream;
     switch (dst_dtype) {
-        case HIF8_F32: decode_kernel<HIF8_F32><<<grid, kThreads, 0, st>>>(src, dst, n, n_vec, scale_exp); break;
-        case HIF8_BF16: decode_kernel<HIF8_BF16><<<grid, kThreads, 0, st>>>(src, dst, n, n_vec, scale_exp); break;
-        default: decode_kernel<HIF8_F16><<<grid, kThreads, 0, st>>>(src, dst, n, n_vec, scale_exp); break;
+        case HIF8_F32: launch_pdl(decode_kernel<HIF8_F32>, grid, st, src, dst, n, n_vec, scale_exp); break;
+        case HIF8_BF16: launch_pdl(decode_kernel<HIF8_BF16>, grid, st, src, dst, n, n_vec, scale_exp); break;
+        default: launch_pdl(decode_kernel<HIF8_F16>, grid, st, src, dst, n, n_vec, scale_exp); break;
     }
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
