@@ -206,29 +206,50 @@ template <int DT> __device__ __forceinline__ uint32_t to_bits(float v)
 // ------------------------------------------------------------------------------------------------
 // One element: scaled value -> HiF8 byte
 // ------------------------------------------------------------------------------------------------
+// Per-exponent entry of the rounding table (indexed by the biased exponent of the scaled magnitude):
+//   bits 0-4   number of discarded mantissa bits (23 - width); 0: nothing to round (overflow, Inf, NaN)
+//   bits 8-12  left shift that aligns an N-bit threshold complement with the top of the discarded field
+//   bit  7     this binade rounds stochastically (the complement comes from the source bits)
+//   bits 16-31 otherwise: the constant to shift instead (half of 2^N for round-half-away binades, 0 for none)
+constexpr uint32_t kThrStochastic = 0x80u;
+
 template <int MODE, int SRC>
 __device__ __forceinline__ uint32_t encode_one(float x, uint32_t raw, float scale, const uint8_t* s_ta,
-                                               const uint8_t* s_sh, uint32_t word)
+                                               const uint32_t* s_thr, uint32_t word)
 {
     const float y = x * scale;
     uint32_t t = __float_as_uint(y);
     if (MODE == HIF8_RND_TA) return s_ta[t >> 19];
 
-    // threshold T of Section 3.2 (with the guard that a zero fraction never rounds up: compare with max(T,1))
+    const bool sub = (t & 0x7FFFFFFFu) < 0x34800000u;  // |y| < 2^-22 (zero included): result is 0 or 2^-22
+    // Below 2^-22 the kept bits are zero and the fraction is F = |y| / 2^-22.  Adding 2^-22 with truncation puts
+    // floor(F 2^23) into the mantissa field of a value in the binade of 2^-22, so the common code rounds it like a
+    // 0-bit-mantissa binade (result 2^-22 or 2^-21); it is moved down again afterwards.
+    const uint32_t tz = __float_as_uint(__fadd_rz(fabsf(y), 2.384185791015625e-07f));
+
+    if (MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR) {
+        // hybrid / simplified stochastic rounding: the carry of (magnitude + (2^N - T) << k) does the rounding
+        const uint32_t u = sub ? tz : (t & 0x7FFFFFFFu);
+        const uint32_t ent = s_thr[u >> 23];
+        const uint32_t d_ssr = (SRC == HIF8_F32) ? 0x4000u - max(raw & 0x3FFFu, 1u)   // SR14: 2^14 - max(T14, 1)
+                                                 : 3u - 2u * (raw & 1u);               // SR2:  4 - {source LSB, 1}
+        const uint32_t d = (ent & kThrStochastic) ? d_ssr : (ent >> 16);
+        uint32_t tr = (u + (d << ((ent >> 8) & 31u))) & (0xFFFFFFFFu << (ent & 31u));
+        // below 2^-22: two binades down, so that 2^-21 packs as 2^-22 and 2^-22 as the single zero
+        tr -= sub ? 0x01000000u : 0u;
+        return s_ta[(tr >> 19) | ((t >> 19) & 0x1000u)];
+    }
+
+    // TE and standard SR
     constexpr int kSrBits = (SRC == HIF8_F32) ? 24 : 16;
     const uint32_t sign7 = (t >> 24) & 0x80u;
-    const bool sub = (t & 0x7FFFFFFFu) < 0x34800000u;  // |y| < 2^-22 (zero included): result is 0 or 2^-22
     if (MODE == HIF8_RND_SR && SRC == HIF8_F32 && sub) {
         // the 24-bit threshold is wider than a binary32 fraction: compare F24 = floor(|y| 2^46) directly
         const uint32_t f24 = __float2uint_rz(fabsf(y) * 70368744177664.f);
         return f24 >= max(word >> 8, 1u) ? (sign7 | 0x01u) : 0u;
     }
-    // Below 2^-22 the kept bits are zero and the fraction is F = |y| / 2^-22.  Adding 2^-22 with truncation puts
-    // floor(F 2^23) into the mantissa field of a value in the binade of 2^-22, so the common code below rounds it
-    // like a 0-bit-mantissa binade; one step of 2^-22 is taken off the result afterwards.
-    const uint32_t tz = __float_as_uint(__fadd_rz(fabsf(y), 2.384185791015625e-07f)) | (t & 0x80000000u);
-    t = sub ? tz : t;
-    const uint32_t sh = s_sh[(t >> 23) & 0xFFu];  // discarded mantissa bits (23 - width); 0: nothing to round
+    t = sub ? (tz | (t & 0x80000000u)) : t;
+    const uint32_t sh = s_thr[(t >> 23) & 0xFFu] & 31u;  // discarded mantissa bits (23 - width); 0: nothing to round
     const uint32_t s = sh ? sh : 23u;
     uint32_t inc;
     if (MODE == HIF8_RND_TE) {
@@ -237,21 +258,12 @@ __device__ __forceinline__ uint32_t encode_one(float x, uint32_t raw, float scal
         uint32_t lsb = (s == 23u) ? 1u : ((t >> s) & 1u);
         if (sub) lsb = 0u;
         inc = (1u << (s - 1)) - 1u + lsb;
-    } else {
-        uint32_t inc_ssr;
-        if (SRC == HIF8_F32) inc_ssr = (0x4000u - max(raw & 0x3FFFu, 1u)) << (s - 14);  // SR14
-        else inc_ssr = (3u - 2u * (raw & 1u)) << (s - 2);                                // SR2: 4 - T2
-        if (MODE == HIF8_RND_SSR) inc = inc_ssr;
-        else if (MODE == HIF8_RND_HR) {
-            const int E = (int)((t >> 23) & 0xFFu) - 127;                                // Eq. 3
-            inc = (E > -4 && E < 4) ? (1u << (s - 1)) : inc_ssr;
-        } else {  // standard SR
-            const uint32_t T = max(word >> (32 - kSrBits), 1u);
-            if (SRC == HIF8_F32) {
-                const uint32_t k = 24u - s;  // F24 = discarded << k; up iff discarded >= ceil(T / 2^k)
-                inc = (1u << s) - ((T + (1u << k) - 1u) >> k);
-            } else inc = (0x10000u - T) << (s - 16);
-        }
+    } else {  // standard SR (threshold T of Section 3.2, compared as max(T,1) so that a zero fraction never rounds up)
+        const uint32_t T = max(word >> (32 - kSrBits), 1u);
+        if (SRC == HIF8_F32) {
+            const uint32_t k = 24u - s;  // F24 = discarded << k; up iff discarded >= ceil(T / 2^k)
+            inc = (1u << s) - ((T + (1u << k) - 1u) >> k);
+        } else inc = (0x10000u - T) << (s - 16);
     }
     if (sh == 0) inc = 0;
     const uint32_t tr = (t + inc) & (0xFFFFFFFFu << sh);
@@ -269,11 +281,11 @@ __device__ __forceinline__ uint32_t encode_one(float x, uint32_t raw, float scal
 // ------------------------------------------------------------------------------------------------
 struct __align__(16) SmemTables {
     uint8_t ta[8192];
-    uint8_t sh[256];
+    uint32_t thr[256];
     float dec[256];
 };
 
-template <bool NEED_TA, bool NEED_SH, bool NEED_DEC>
+template <bool NEED_TA, bool NEED_SH, bool NEED_DEC, int MODE = HIF8_RND_TA, int SRC = HIF8_F32>
 __device__ __forceinline__ void setup_tables(SmemTables& s, unsigned flags)
 {
     if (NEED_TA) {
@@ -309,9 +321,16 @@ __device__ __forceinline__ void setup_tables(SmemTables& s, unsigned flags)
         }
     }
     if (NEED_SH) {
-        int e = threadIdx.x;  // kThreads == 256 biased exponents
-        int E = e - 127;
-        s.sh[e] = (E >= 16 || E < -22) ? 0 : (uint8_t)(23 - mant_width(E));
+        const int e = threadIdx.x, E = e - 127;  // kThreads == 256 biased exponents
+        uint32_t ent = 0;
+        if (E < 16 && E >= -22) {
+            constexpr uint32_t N = (SRC == HIF8_F32) ? 14u : 2u;  // threshold bits of the simplified SR
+            const uint32_t sh = 23u - (uint32_t)mant_width(E);
+            ent = sh | ((sh - N) << 8);
+            if (MODE == HIF8_RND_SSR || (MODE == HIF8_RND_HR && (E <= -4 || E >= 4))) ent |= kThrStochastic;
+            else ent |= (1u << (N - 1)) << 16;  // round half away = threshold one half
+        }
+        s.thr[e] = ent;
     }
     if (NEED_DEC) s.dec[threadIdx.x] = __uint_as_float(decode_bits_f32(threadIdx.x));
     __syncthreads();
@@ -349,7 +368,7 @@ __global__ void __launch_bounds__(kThreads) convert_kernel(const ConvParams p, u
 {
     __shared__ SmemTables sm;
     pdl_launch_dependents();
-    setup_tables<true, MODE != HIF8_RND_TA, FQ>(sm, p.flags);  // reads only the constant table
+    setup_tables<true, MODE != HIF8_RND_TA, FQ, MODE, SRC>(sm, p.flags);  // reads only the constant table
     pdl_wait_prior_grid();
     const int se = resolve_scale_exp(p);
     const float scale = pow2f(se);
@@ -384,7 +403,7 @@ __global__ void __launch_bounds__(kThreads) convert_kernel(const ConvParams p, u
                 float x; uint32_t raw;
                 unpack<SRC>(v[j], k, x, raw);
                 if (AMAX) amax = amax_step(amax, x);
-                codes[k] = encode_one<MODE, SRC>(x, raw, scale, sm.ta, sm.sh, rw[k]);
+                codes[k] = encode_one<MODE, SRC>(x, raw, scale, sm.ta, sm.thr, rw[k]);
             }
             if (!FQ) {
                 uint32_t w0 = codes[0] | (codes[1] << 8) | (codes[2] << 16) | (codes[3] << 24);
@@ -418,7 +437,7 @@ __global__ void __launch_bounds__(kThreads) convert_kernel(const ConvParams p, u
                 const uint32_t rr[4] = {r.x, r.y, r.z, r.w};
                 word = rr[i & 3];
             }
-            uint32_t c = encode_one<MODE, SRC>(x, raw, scale, sm.ta, sm.sh, word);
+            uint32_t c = encode_one<MODE, SRC>(x, raw, scale, sm.ta, sm.thr, word);
             if (!FQ) reinterpret_cast<uint8_t*>(p.dst)[i] = (uint8_t)c;
             else {
                 uint32_t o = to_bits<SRC>(sm.dec[c] * d1 * d2);
