@@ -492,3 +492,53 @@ void hif8o_gemm_full(const uint8_t* Aq, long long lda, const uint8_t* Wq, long l
             S[m * N + n] = ldexp(sab, -(sa + sw));
         }
 }
+
+/* Algorithm 1 (HiF8 Calibration with Per-Tensor Scaling), the search of one layer:
+ *   for Ea in [e_min, e_max], Ew in [e_min, e_max]:
+ *     A_q = To_HiF8_TA(A * 2^Ea), W_q = To_HiF8_TA(W * 2^Ew)          ("Scale & Cast")
+ *     O_q = (A_q x W_q) * 2^-(Ea+Ew)                                   ("MatMul & Restore")
+ *     err[Ea][Ew] = mean over all outputs of (O_q - O)^2               ("Quantization Error": MSE)
+ *   best = argmin err (READING: the first minimum in row-major (Ea, Ew) order on exact ties).
+ * A is [M,K] row-major, W is [K,N] or (w_is_nk) [N,K], both of `dtype`; O is the high-precision output [M,N] float.
+ * Everything after the cast is computed in double. */
+void hif8o_pts_search(const void* A, const void* W, int dtype, int w_is_nk, const float* O, int M, int N, int K,
+                      int e_min, int e_max, int quick, double* err, int* best)
+{
+    int nE = e_max - e_min + 1;
+    size_t na = (size_t)M * K, nw = (size_t)K * N;
+    double* da = (double*)malloc(sizeof(double) * na * nE);
+    double* dw = (double*)malloc(sizeof(double) * nw * nE);
+    for (int i = 0; i < nE; i++) {
+        int e = e_min + i;
+#pragma omp parallel for schedule(static)
+        for (long long j = 0; j < (long long)na; j++) {
+            uint32_t raw; double x = src_to_double(A, (size_t)j, dtype, &raw);
+            da[(size_t)i * na + j] = hif8o_value(encode_value(x, raw, dtype, e, O_TA, 0, 0, 0, quick));
+        }
+#pragma omp parallel for schedule(static)
+        for (long long j = 0; j < (long long)nw; j++) {
+            uint32_t raw; double x = src_to_double(W, (size_t)j, dtype, &raw);
+            dw[(size_t)i * nw + j] = hif8o_value(encode_value(x, raw, dtype, e, O_TA, 0, 0, 0, quick));
+        }
+    }
+    for (int ia = 0; ia < nE; ia++)
+        for (int iw = 0; iw < nE; iw++) {
+            const double* a = da + (size_t)ia * na;
+            const double* w = dw + (size_t)iw * nw;
+            double sum = 0.0;
+#pragma omp parallel for reduction(+ : sum) schedule(static)
+            for (long long m = 0; m < M; m++)
+                for (long long n = 0; n < N; n++) {
+                    double acc = 0.0;
+                    for (int k = 0; k < K; k++)
+                        acc += a[m * K + k] * (w_is_nk ? w[n * K + k] : w[(long long)k * N + n]);
+                    double d = ldexp(acc, -((e_min + ia) + (e_min + iw))) - (double)O[m * N + n];
+                    sum += d * d;
+                }
+            err[ia * nE + iw] = sum / ((double)M * (double)N);
+        }
+    int bi = 0;
+    for (int i = 1; i < nE * nE; i++) if (err[i] < err[bi]) bi = i;
+    best[0] = e_min + bi / nE; best[1] = e_min + bi % nE;
+    free(da); free(dw);
+}

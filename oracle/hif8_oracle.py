@@ -30,6 +30,7 @@ _lib.hif8o_decode.argtypes = [_vp, _vp, _i, _sz, _i]
 _lib.hif8o_amax_scale.argtypes = [_vp, _i, _sz, _i, C.POINTER(C.c_float), C.POINTER(C.c_int)]
 _lib.hif8o_fake_quant.argtypes = [_vp, _vp, _i, _sz, _i, _i, _u, _u64, _i]
 _lib.hif8o_gemm_entries.argtypes = [_vp, _ll, _vp, _ll, _i, _i, _i, _i, _vp, _vp, _sz, _vp, _vp]
+_lib.hif8o_pts_search.argtypes = [_vp, _vp, _i, _i, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp]
 _lib.hif8o_gemm_full.argtypes = [_vp, _ll, _vp, _ll, _i, _i, _i, _i, _i, _i, _vp, _vp]
 
 
@@ -144,3 +145,19 @@ def gemm_full(Aq, Wq, w_is_nk, sa, sw):
     s = np.empty((M, N), dtype=np.float64)
     _lib.hif8o_gemm_full(_ptr(Aq), K, _ptr(Wq), Wq.shape[1], int(w_is_nk), M, N, K, sa, sw, _ptr(cs), _ptr(s))
     return cs, s
+
+
+def pts_search(A, W, dtype, w_is_nk, O_ref, e_min=-4, e_max=5, quick=False):
+    """Algorithm 1 for one layer: (err[nE, nE] float64 MSE table indexed [Ea - e_min, Ew - e_min], (best Ea, best Ew)).
+    A [M,K], W [K,N] or [N,K] raw encodings of `dtype`; O_ref [M,N] float32."""
+    A = _src(A, dtype)
+    W = _src(W, dtype)
+    O_ref = np.ascontiguousarray(O_ref, dtype=np.float32)
+    M, K = A.shape
+    N = W.shape[0] if w_is_nk else W.shape[1]
+    nE = e_max - e_min + 1
+    err = np.empty((nE, nE), dtype=np.float64)
+    best = np.zeros(2, dtype=np.int32)
+    _lib.hif8o_pts_search(_ptr(A), _ptr(W), dtype, int(w_is_nk), _ptr(O_ref), M, N, K, e_min, e_max, int(quick),
+                          _ptr(err), _ptr(best))
+    return err, (int(best[0]), int(best[1]))

@@ -465,3 +465,33 @@ def test_gemm_oracle_against_numpy():
     Wi = ints[rng.integers(0, len(ints), (K, N))]
     ci, _ = O.gemm_full(Ai, Wi, False, 0, 0)
     assert np.array_equal(ci, (tab[Ai].astype(np.int64) @ tab[Wi].astype(np.int64)).astype(np.float64))
+
+
+def test_pts_search_against_definition_and_scale_shift_property():
+    # Algorithm 1: the error table recomputed from the pinned pieces (cast, decode) with numpy's matmul, and two
+    # properties of power-of-two scaling: a tensor pre-multiplied by 2^s shifts the table by s along its axis, and
+    # an operand that is exactly representable at every scale contributes no error
+    M, N, K = 24, 20, 48
+    a = W.normal_bf16((M, K), seed=41)
+    w = W.normal_bf16((K, N), seed=42, std=0.05)
+    af, wf = W.bf16_bits_to_f32(a).astype(np.float64), W.bf16_bits_to_f32(w).astype(np.float64)
+    Oref = (af @ wf).astype(np.float32)
+    err, best = O.pts_search(a, w, O.BF16, False, Oref, -4, 5)
+    tab = np.array([O.value(c) for c in range(256)])
+    for ea, ew in [(-4, -4), (0, 3), (5, 5), (2, -1)]:
+        aq, wq = tab[O.encode(a, O.BF16, ea)], tab[O.encode(w, O.BF16, ew)]
+        want = np.mean(((aq @ wq) * 2.0 ** -(ea + ew) - Oref.astype(np.float64)) ** 2)
+        assert np.isclose(err[ea + 4, ew + 4], want, rtol=1e-12)
+    assert err[best[0] + 4, best[1] + 4] == err.min()
+    a2 = W.f32_to_bf16_bits(W.bf16_bits_to_f32(a) * np.float32(4.0))           # A * 2^2: exact in BF16
+    O2 = (af * 4.0 @ wf).astype(np.float32)
+    err2, _ = O.pts_search(a2, w, O.BF16, False, O2, -4, 5)
+    assert np.allclose(err2[:8, :], 16.0 * err[2:, :], rtol=1e-6)              # Ea' = Ea - 2, errors scale by 4^2
+    ones = np.full((M, K), 0x3F80, dtype=np.uint16)                            # all-ones A: exact at every Ea
+    O3 = (np.ones((M, K)) @ wf).astype(np.float32)
+    err3, _ = O.pts_search(ones, w, O.BF16, False, O3, -4, 5)
+    assert np.allclose(err3, err3[0:1, :], rtol=1e-9)                          # no dependence on Ea
+    errq, bestq = O.pts_search(a, w, O.BF16, False, Oref, -4, 5, quick=True)
+    assert np.allclose(errq, err, rtol=1e-12) and bestq == best      # (the parallel sum order is not fixed)
+    errt, _ = O.pts_search(a, np.ascontiguousarray(w.T), O.BF16, True, Oref, -4, 5)
+    assert np.allclose(errt, err, rtol=1e-12)
