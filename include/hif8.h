@@ -183,6 +183,24 @@ int hif8_gemm(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int64_t ldw, in
  */
 int hif8_gemm_status(const void* workspace, hif8_stream_t stream);
 
+/*
+ * Per-layer search of Algorithm 1 ("HiF8 Calibration with Per-Tensor Scaling"): for every (Ea, Ew) with both
+ * exponents in [e_min, e_max] (the paper searches [-4, 5]):
+ *     A_q = To_HiF8_TA(A * 2^Ea), W_q = To_HiF8_TA(W * 2^Ew);  O_q = (A_q x W_q) * 2^-(Ea+Ew);
+ *     d_err[(Ea - e_min) * n + (Ew - e_min)] = MSE(O_q, O_ref) over all M*N outputs      (n = e_max - e_min + 1 <= 16)
+ * and d_best[0], d_best[1] = the (Ea, Ew) of the smallest error (first one in that order on exact ties).
+ * A: [M,K] row-major; W: [K,N] (w_is_nk = 0) or [N,K]; both contiguous, of `dtype`; O_ref: the layer's high-precision
+ * output [M,N] as float, leading dimension ldo.  K and the row length of W must be multiples of 16.
+ * All device memory; 2n encodes, n*n GEMMs with FP32 output and n*n reductions are enqueued on `stream`, nothing
+ * returns to the host.  workspace: hif8_pts_workspace_bytes(M, N, K, n) bytes, 256-byte aligned; its first int is a
+ * device status word as for hif8_gemm (hif8_pts_status reads it, synchronising the stream).
+ */
+int hif8_pts_search(const void* A, const void* W, int dtype, int w_is_nk, const float* O_ref, int64_t ldo, int M, int N,
+                    int K, int e_min, int e_max, float* d_err, int* d_best, void* workspace, size_t workspace_bytes,
+                    hif8_stream_t stream);
+size_t hif8_pts_workspace_bytes(int M, int N, int K, int n_exp);
+int hif8_pts_status(const void* workspace, hif8_stream_t stream);
+
 /* bytes of device workspace a call needs (which = HIF8_WS_*; n = element count; for HIF8_WS_GEMM: 0 for the
  * minimum, or M*K + K*N for the decode-once path) */
 size_t hif8_workspace_bytes(int which, size_t n);

@@ -17,7 +17,8 @@ OK = 0
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libhif8.so")
-EXPORTS = ["hif8_encode", "hif8_decode", "hif8_amax", "hif8_amax_scale_encode", "hif8_fake_quant", "hif8_gemm", "hif8_gemm_status",
+EXPORTS = ["hif8_encode", "hif8_decode", "hif8_amax", "hif8_amax_scale_encode", "hif8_fake_quant", "hif8_gemm", "hif8_gemm_status", "hif8_pts_search", "hif8_pts_workspace_bytes",
+           "hif8_pts_status",
            "hif8_amax_scale_encode_static", "hif8_workspace_bytes", "hif8_status_string", "hif8_launch_count"]
 
 if not os.path.exists(LIB_PATH):
@@ -36,6 +37,12 @@ lib.hif8_fake_quant.argtypes = [_vp, _vp, _i, _sz, _i, _i, _i, _u, _u64, _vp, _v
 lib.hif8_gemm.argtypes = [_vp, _i64, _vp, _i64, _i, _vp, _i64, _i, _i, _i, _i, _vp, _vp, _vp, _sz, _vp]
 lib.hif8_gemm_status.argtypes = [_vp, _vp]
 lib.hif8_gemm_status.restype = _i
+lib.hif8_pts_search.argtypes = [_vp, _vp, _i, _i, _vp, _i64, _i, _i, _i, _i, _i, _vp, _vp, _vp, _sz, _vp]
+lib.hif8_pts_search.restype = _i
+lib.hif8_pts_workspace_bytes.argtypes = [_i, _i, _i, _i]
+lib.hif8_pts_workspace_bytes.restype = _sz
+lib.hif8_pts_status.argtypes = [_vp, _vp]
+lib.hif8_pts_status.restype = _i
 lib.hif8_workspace_bytes.argtypes = [_i, _sz]
 lib.hif8_workspace_bytes.restype = _sz
 lib.hif8_status_string.argtypes = [_i]
@@ -130,3 +137,17 @@ def hif8_gemm(Aq, lda, Wq, ldw, w_is_nk, Cmat, ldc, c_dtype, M, N, K, d_scale_ex
 
 def hif8_gemm_status(workspace, stream=None):
     return int(lib.hif8_gemm_status(_ptr(workspace), _stream(stream)))
+
+
+def hif8_pts_workspace_bytes(M, N, K, n_exp):
+    return int(lib.hif8_pts_workspace_bytes(M, N, K, n_exp))
+
+
+def hif8_pts_search(A, W, dtype, w_is_nk, O_ref, ldo, M, N, K, e_min, e_max, d_err, d_best, workspace, workspace_bytes,
+                    stream=None, check=True):
+    return _check(lib.hif8_pts_search(_ptr(A), _ptr(W), dtype, int(w_is_nk), _ptr(O_ref), ldo, M, N, K, e_min, e_max,
+                                      _ptr(d_err), _ptr(d_best), _ptr(workspace), workspace_bytes, _stream(stream)), check)
+
+
+def hif8_pts_status(workspace, stream=None):
+    return int(lib.hif8_pts_status(_ptr(workspace), _stream(stream)))
