@@ -232,6 +232,21 @@ def extra_results(H, torch, hbm_peak, peak_kind):
                   "note": "no workspace: byte tiles decoded per CTA in shared memory"},
         "bound": "tensor", "peak": tf_peak, "peak_kind": f"of {tf_kind} (cuBLAS BF16 burst)", "unit": "TFLOP/s",
         "scale_exps": [int(v) for v in se.cpu()], "output": "bf16"}
+    del C, gws, Aq, Wq
+
+    # ---- Algorithm 1, one layer: 10 x 10 grid of scale exponents, 4096^3 (20 casts, 100 GEMMs, 100 MSE reductions)
+    M = N = K = 4096
+    a = torch.randn(M, K, generator=g, device="cuda").to(torch.bfloat16)
+    w = (torch.randn(K, N, generator=g, device="cuda") * 0.02).to(torch.bfloat16)
+    o_ref = torch.matmul(a.float(), w.float())
+    pb = H.hif8_pts_workspace_bytes(M, N, K, 10)
+    pws = torch.empty(pb, dtype=torch.uint8, device="cuda")
+    d_err = torch.zeros(100, dtype=torch.float32, device="cuda")
+    d_best = torch.zeros(2, dtype=torch.int32, device="cuda")
+    ms = timed(lambda r: H.hif8_pts_search(a, w, H.BF16, 0, o_ref, N, M, N, K, -4, 5, d_err, d_best, pws, pb), 3)
+    out["pts_search_4096^3"] = {"ms": ms, "TFLOPs_of_100_gemms": 100 * 2.0 * M * N * K / ms / 1e9,
+                                "best_exponents": [int(v) for v in d_best.cpu()], "device_status": H.hif8_pts_status(pws),
+                                "min_mse": float(d_err.min().item())}
     return out
 
 
