@@ -184,6 +184,14 @@ int hif8_gemm(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int64_t ldw, in
 int hif8_gemm_status(const void* workspace, hif8_stream_t stream);
 
 /*
+ * Self-test of the device-side failure detection: launches one warp that waits, with a limit of `limit_ms`
+ * milliseconds (1..1000), on a barrier that is never completed.  The wait gives up, the kernel records the status
+ * word in `workspace` (first int, cleared by the call) and ends normally; hif8_gemm_status(workspace, stream) then
+ * returns HIF8_ERR_DEVICE_TIMEOUT and the device stays usable.  No fault, trap or unbounded loop is involved.
+ */
+int hif8_selftest_wait_timeout(void* workspace, unsigned limit_ms, hif8_stream_t stream);
+
+/*
  * Per-layer search of Algorithm 1 ("HiF8 Calibration with Per-Tensor Scaling"): for every (Ea, Ew) with both
  * exponents in [e_min, e_max] (the paper searches [-4, 5]):
  *     A_q = To_HiF8_TA(A * 2^Ea), W_q = To_HiF8_TA(W * 2^Ew);  O_q = (A_q x W_q) * 2^-(Ea+Ew);

@@ -18,7 +18,7 @@ OK = 0
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libhif8.so")
 EXPORTS = ["hif8_encode", "hif8_decode", "hif8_amax", "hif8_amax_scale_encode", "hif8_fake_quant", "hif8_gemm", "hif8_gemm_status", "hif8_pts_search", "hif8_pts_workspace_bytes",
-           "hif8_pts_status",
+           "hif8_pts_status", "hif8_selftest_wait_timeout",
            "hif8_amax_scale_encode_static", "hif8_workspace_bytes", "hif8_status_string", "hif8_launch_count"]
 
 if not os.path.exists(LIB_PATH):
@@ -43,6 +43,8 @@ lib.hif8_pts_workspace_bytes.argtypes = [_i, _i, _i, _i]
 lib.hif8_pts_workspace_bytes.restype = _sz
 lib.hif8_pts_status.argtypes = [_vp, _vp]
 lib.hif8_pts_status.restype = _i
+lib.hif8_selftest_wait_timeout.argtypes = [_vp, _u, _vp]
+lib.hif8_selftest_wait_timeout.restype = _i
 lib.hif8_workspace_bytes.argtypes = [_i, _sz]
 lib.hif8_workspace_bytes.restype = _sz
 lib.hif8_status_string.argtypes = [_i]
@@ -151,3 +153,7 @@ def hif8_pts_search(A, W, dtype, w_is_nk, O_ref, ldo, M, N, K, e_min, e_max, d_e
 
 def hif8_pts_status(workspace, stream=None):
     return int(lib.hif8_pts_status(_ptr(workspace), _stream(stream)))
+
+
+def hif8_selftest_wait_timeout(workspace, limit_ms, stream=None, check=True):
+    return _check(lib.hif8_selftest_wait_timeout(_ptr(workspace), limit_ms, _stream(stream)), check)

@@ -97,7 +97,8 @@ __device__ __forceinline__ unsigned long long global_ns()
 }
 
 // Bounded wait.  Returns false when the barrier did not complete in time or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int where)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int where,
+                                          unsigned long long limit_ns = kWaitLimitNs)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_ns();
@@ -105,7 +106,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 63u) == 0) {
             if (*abort_flag) return false;
-            if (global_ns() - t0 > kWaitLimitNs) {
+            if (global_ns() - t0 > limit_ns) {
                 *abort_flag = 1;
                 atomicCAS(status, 0, where);
                 return false;
@@ -666,6 +667,22 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     }
 }
 
+// Self-test of the bounded wait: one warp waits on a barrier that nothing will ever complete, with a short limit.
+// The wait must give up, record its status word and let the kernel finish normally.
+__global__ void wait_selftest_kernel(int* status, unsigned long long limit_ns)
+{
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) (void)mbar_wait(smem_u32(&bar), 0, &abort_flag, status, 99, limit_ns);
+    __syncthreads();
+}
+
 // ---------------------------------------------------------------------------------------------------------
 // Host side
 // ---------------------------------------------------------------------------------------------------------
@@ -824,4 +841,15 @@ extern "C" int hif8_gemm_status(const void* workspace, hif8_stream_t stream)
     if (cudaMemcpyAsync(&v, workspace, sizeof v, cudaMemcpyDeviceToHost, (cudaStream_t)stream) != cudaSuccess) return HIF8_ERR_CUDA;
     if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return HIF8_ERR_CUDA;
     return v == 0 ? HIF8_OK : HIF8_ERR_DEVICE_TIMEOUT;
+}
+
+extern "C" int hif8_selftest_wait_timeout(void* workspace, unsigned limit_ms, hif8_stream_t stream)
+{
+    if (!workspace) return HIF8_ERR_NULL;
+    if (limit_ms == 0 || limit_ms > 1000) return HIF8_ERR_SHAPE;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemsetAsync(workspace, 0, 4, st) != cudaSuccess) return HIF8_ERR_CUDA;
+    wait_selftest_kernel<<<1, 32, 0, st>>>(reinterpret_cast<int*>(workspace), (unsigned long long)limit_ms * 1000000ull);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
 }

@@ -129,3 +129,16 @@ def test_gemm_medium_scaled_operands_sampled(w_is_nk):
         for staged in (False, True):
             C = run_gemm(Aq, np.ascontiguousarray(Wkn.T) if w_is_nk else Wkn, w_is_nk, c_dtype, sa=sa, sw=sw, staged=staged)
             check(C[rows, cols], Cs, S, c_dtype)
+
+
+def test_bounded_wait_gives_up_and_reports_without_disturbing_the_device():
+    # failure detection: a wait that nothing satisfies runs out after its limit (50 ms here), the status word says so,
+    # and the next GEMM on the same device works
+    ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+    H.hif8_selftest_wait_timeout(ws, 50)
+    assert H.hif8_gemm_status(ws) == 10                      # HIF8_ERR_DEVICE_TIMEOUT
+    assert int(ws[:4].view(torch.int32).item()) == 99        # where it gave up
+    M, N, K = 128, 256, 64
+    Aq = np.full((M, K), 0x08, dtype=np.uint8)
+    Wq = np.full((K, N), 0x10, dtype=np.uint8)
+    assert np.all(run_gemm(Aq, Wq, 0, H.F32) == 2.0 * K)
