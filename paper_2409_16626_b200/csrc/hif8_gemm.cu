@@ -31,6 +31,7 @@
 #include <mutex>
 
 #include "hif8.h"
+#include "hif8_internal.cuh"
 
 namespace hif8 {
 extern std::atomic<uint64_t> g_launches;
@@ -124,21 +125,6 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-// D[tmem] (+)= A[smem] * B[smem], 128 x 256 x 16, BF16 inputs, FP32 accumulate
-__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
 
 __device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t (&r)[32])
 {
@@ -252,16 +238,6 @@ __device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int
     tile_n = (t % per_group) / rows_in_group;
 }
 
-struct GemmParams {
-    void* C;
-    long long ldc;
-    int c_is_f32;
-    int M, N, K;
-    const int* d_sa;
-    const int* d_sw;
-    int* status;
-    int tiles_m, tiles_n;
-};
 
 template <bool W_IS_NK>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -604,6 +580,8 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
         const int s1 = sdesc / 2, s2 = sdesc - s1;
         const float f1 = __uint_as_float((uint32_t)(s1 + 127) << 23), f2 = __uint_as_float((uint32_t)(s2 + 127) << 23);
         int local = 0;
+        double err_acc = 0.0;  // squared-error variant: this thread's share over all its tiles
+        const bool ref_vec = !(reinterpret_cast<uintptr_t>(p.err_ref) & 15) && !(p.ld_ref & 3);
         for (int t = pair_id; t < tiles; t += pairs, local++) {
             const int acc = local & 1, use = local >> 1;
             if (!mbar_wait(bar_acc_full(acc), (uint32_t)(use & 1), abort_flag, p.status, 24)) break;
@@ -617,7 +595,28 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                 tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(warp * 32) << 16) + acc * 256 + c, r);
                 tmem_ld_wait();
                 const int col = n0 + c;
-                if (row < p.M && col < p.N) {
+                if (p.err_sum) {
+                    if (row < p.M && col < p.N) {
+                        // exact differences of the FP32 result and the FP32 reference, squared and summed in double
+                        const float* ref = p.err_ref + (long long)row * p.ld_ref + col;
+                        if (col + 32 <= p.N && ref_vec) {
+#pragma unroll
+                            for (int i = 0; i < 32; i += 4) {
+                                const float4 o = __ldg(reinterpret_cast<const float4*>(ref + i));
+                                const double d0 = (double)(__uint_as_float(r[i]) * f1 * f2) - (double)o.x;
+                                const double d1 = (double)(__uint_as_float(r[i + 1]) * f1 * f2) - (double)o.y;
+                                const double d2 = (double)(__uint_as_float(r[i + 2]) * f1 * f2) - (double)o.z;
+                                const double d3 = (double)(__uint_as_float(r[i + 3]) * f1 * f2) - (double)o.w;
+                                err_acc += d0 * d0 + d1 * d1 + d2 * d2 + d3 * d3;
+                            }
+                        } else {
+                            for (int i = 0; i < 32 && col + i < p.N; i++) {
+                                const double d = (double)(__uint_as_float(r[i]) * f1 * f2) - (double)__ldg(ref + i);
+                                err_acc += d * d;
+                            }
+                        }
+                    }
+                } else if (row < p.M && col < p.N) {
                     const bool full = col + 32 <= p.N;
                     if (p.c_is_f32) {
                         float* out = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + col;
@@ -654,6 +653,10 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(bar_acc_empty(acc), 0));  // tell the leader: accumulator drained
+        }
+        if (p.err_sum) {
+            for (int off = 16; off > 0; off >>= 1) err_acc += __shfl_xor_sync(0xFFFFFFFFu, err_acc, off);
+            if (lane == 0 && err_acc != 0.0) atomicAdd(p.err_sum, err_acc);
         }
     }
 
@@ -720,11 +723,60 @@ bool make_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t rows, 
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// one-time kernel attributes (dynamic shared memory) and the SM count of the device
+bool gemm_kernels_ready(int dev, int* sm_count_out)
+{
+    static std::once_flag attr_once;
+    static cudaError_t attr_rc = cudaSuccess;
+    static int sm_count = 0;
+    std::call_once(attr_once, [dev] {
+        attr_rc = cudaFuncSetAttribute(hif8_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (attr_rc == cudaSuccess)
+            attr_rc = cudaFuncSetAttribute(hif8_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (attr_rc == cudaSuccess)
+            attr_rc = cudaFuncSetAttribute(bf16_gemm_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
+        if (attr_rc == cudaSuccess)
+            attr_rc = cudaFuncSetAttribute(bf16_gemm_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
+        if (attr_rc == cudaSuccess) attr_rc = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+    });
+    *sm_count_out = sm_count;
+    return attr_rc == cudaSuccess && sm_count > 0;
+}
+
 constexpr size_t kGemmWorkspaceBytes = 256;
 
 }  // namespace
 
-size_t gemm_workspace_bytes() { return kGemmWorkspaceBytes; }
+int launch_bf16_pair_gemm(const void* a_bf, const void* w_bf, int w_is_nk, GemmParams p, cudaStream_t st)
+{
+    int dev = 0, sm_count = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || !gemm_kernels_ready(dev, &sm_count)) return HIF8_ERR_CUDA;
+    const int M = p.M, N = p.N, K = p.K;
+    p.tiles_m = (M + BM - 1) / BM;
+    p.tiles_n = (N + BN - 1) / BN;
+    const long long tiles2 = (long long)((M + 2 * BM - 1) / (2 * BM)) * p.tiles_n;
+    if (M <= 0 || N <= 0 || K <= 0 || tiles2 > 0x3FFFFFFF) return HIF8_ERR_SHAPE;
+    CUtensorMap ma, mw;
+    if (!make_map(&ma, a_bf, (uint64_t)K, (uint64_t)M, (uint64_t)K, BK, BM, true)) return HIF8_ERR_CUDA;
+    // W boxes are one CTA's half of the 256-column tile: 128 rows of [N,K], or two boxes of 64 columns of [K,N]
+    const bool okw = w_is_nk ? make_map(&mw, w_bf, (uint64_t)K, (uint64_t)N, (uint64_t)K, BK, BN / 2, true)
+                             : make_map(&mw, w_bf, (uint64_t)N, (uint64_t)K, (uint64_t)N, 64, BK, true);
+    if (!okw) return HIF8_ERR_CUDA;
+    const int pairs = (int)(tiles2 < sm_count / 2 ? tiles2 : sm_count / 2);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(2u * (unsigned)pairs);
+    cfg.blockDim = dim3(kThreadsP);
+    cfg.dynamicSmemBytes = kSmemBytes2;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    const cudaError_t lrc = w_is_nk ? cudaLaunchKernelEx(&cfg, bf16_gemm_pair_kernel<true>, ma, mw, p)
+                                    : cudaLaunchKernelEx(&cfg, bf16_gemm_pair_kernel<false>, ma, mw, p);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return (lrc == cudaSuccess && cudaGetLastError() == cudaSuccess) ? HIF8_OK : HIF8_ERR_CUDA;
+}
 
 }  // namespace hif8
 
@@ -768,20 +820,8 @@ extern "C" int hif8_gemm(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int6
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMemsetAsync(workspace, 0, 4, st) != cudaSuccess) return HIF8_ERR_CUDA;
 
-    static std::once_flag attr_once;
-    static cudaError_t attr_rc = cudaSuccess;
-    static int sm_count = 0;
-    std::call_once(attr_once, [dev] {
-        attr_rc = cudaFuncSetAttribute(hif8_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        if (attr_rc == cudaSuccess)
-            attr_rc = cudaFuncSetAttribute(hif8_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        if (attr_rc == cudaSuccess)
-            attr_rc = cudaFuncSetAttribute(bf16_gemm_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
-        if (attr_rc == cudaSuccess)
-            attr_rc = cudaFuncSetAttribute(bf16_gemm_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
-        if (attr_rc == cudaSuccess) attr_rc = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-    });
-    if (attr_rc != cudaSuccess || sm_count <= 0) return HIF8_ERR_CUDA;
+    int sm_count = 0;
+    if (!gemm_kernels_ready(dev, &sm_count)) return HIF8_ERR_CUDA;
 
     // Decode-once path: with room for both operands as BF16 in the workspace (and contiguous operands), each HiF8
     // byte is decoded exactly once by the conversion kernel and the tensor-core kernel reads BF16 tiles through TMA.
@@ -794,29 +834,7 @@ extern "C" int hif8_gemm(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int6
         int rc = hif8_decode(Aq, a_bf, HIF8_BF16, (size_t)M * K, 0, stream);
         if (rc == HIF8_OK) rc = hif8_decode(Wq, w_bf, HIF8_BF16, (size_t)K * N, 0, stream);
         if (rc != HIF8_OK) return rc;
-        CUtensorMap ma, mw;
-        if (!make_map(&ma, a_bf, (uint64_t)K, (uint64_t)M, (uint64_t)K, BK, BM, true)) return HIF8_ERR_CUDA;
-        const bool okw = w_is_nk ? make_map(&mw, w_bf, (uint64_t)K, (uint64_t)N, (uint64_t)K, BK, BN, true)
-                                 : make_map(&mw, w_bf, (uint64_t)N, (uint64_t)K, (uint64_t)N, 64, BK, true);
-        if (!okw) return HIF8_ERR_CUDA;
-        // CTA pairs: 256 x 256 tiles; W boxes are this CTA's half (128 columns / rows)
-        CUtensorMap mw2;
-        const bool okw2 = w_is_nk ? make_map(&mw2, w_bf, (uint64_t)K, (uint64_t)N, (uint64_t)K, BK, BN / 2, true) : true;
-        if (!okw2) return HIF8_ERR_CUDA;
-        const int pairs = (int)(tiles2 < sm_count / 2 ? tiles2 : sm_count / 2);
-        cudaLaunchConfig_t cfg{};
-        cfg.gridDim = dim3(2u * (unsigned)pairs);
-        cfg.blockDim = dim3(kThreadsP);
-        cfg.dynamicSmemBytes = kSmemBytes2;
-        cfg.stream = st;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr; cfg.numAttrs = 1;
-        cudaError_t lrc = w_is_nk ? cudaLaunchKernelEx(&cfg, bf16_gemm_pair_kernel<true>, ma, mw2, p)
-                                  : cudaLaunchKernelEx(&cfg, bf16_gemm_pair_kernel<false>, ma, mw, p);
-        g_launches.fetch_add(1, std::memory_order_relaxed);
-        return (lrc == cudaSuccess && cudaGetLastError() == cudaSuccess) ? HIF8_OK : HIF8_ERR_CUDA;
+        return launch_bf16_pair_gemm(a_bf, w_bf, w_is_nk, p, st);
     }
 
     cudaLaunchConfig_t cfg{};

@@ -1,0 +1,26 @@
+// Declarations shared between the translation units of the library (not part of the C ABI).
+#pragma once
+#include <cuda_runtime.h>
+
+namespace hif8 {
+
+struct GemmParams {
+    void* C;
+    long long ldc;
+    int c_is_f32;
+    int M, N, K;
+    const int* d_sa;
+    const int* d_sw;
+    int* status;
+    int tiles_m, tiles_n;
+    // when err_sum is set the epilogue stores nothing: it adds sum (result - err_ref)^2 of its tile to *err_sum
+    const float* err_ref;
+    long long ld_ref;
+    double* err_sum;
+};
+
+// C (or the squared error) from operands that are already BF16 in device memory: a_bf [M,K], w_bf [K,N] or [N,K],
+// both contiguous.  Fills in the tile counts of `p`; p.status must point at a zeroed device int.
+int launch_bf16_pair_gemm(const void* a_bf, const void* w_bf, int w_is_nk, GemmParams p, cudaStream_t st);
+
+}  // namespace hif8

@@ -2,16 +2,18 @@
 // scale exponents (Ea, Ew) of a grid, cast activation and weight to HiF8 with round-half-away, multiply, restore, and
 // measure the mean squared error against the layer's high-precision output; keep the pair with the smallest error.
 //
-// Built from the library's own entry points: each operand is encoded once per exponent (hif8_encode), each pair is one
-// hif8_gemm (FP32 output, descale by the device-resident exponents), followed by a squared-error reduction in double
-// precision; a last one-block kernel turns the sums into the MSE table and takes the argmin.  Nothing returns to the
-// host in between.
+// Each operand is cast once per exponent (hif8_encode into a scratch byte buffer) and expanded once to BF16
+// (hif8_decode, exact), so the n*n multiplications read ready BF16 operands.  Each pair is one launch of the
+// tensor-core kernel whose epilogue restores the scale (2^-(Ea+Ew), device-resident exponents) and, instead of storing
+// the product, adds the squared differences to the layer's output into one double per pair; a last one-block kernel
+// turns the sums into the MSE table and takes the argmin.  Nothing returns to the host in between.
 #include <cuda_runtime.h>
 
 #include <atomic>
 #include <cstdint>
 
 #include "hif8.h"
+#include "hif8_internal.cuh"
 
 namespace hif8 {
 extern std::atomic<uint64_t> g_launches;
@@ -35,29 +37,6 @@ __global__ void pts_init_kernel(PtsCtl* ctl, int e_min, int n_exp)
     if (i == 0) ctl->status = 0;
     if (i < n_exp) ctl->exps[i] = e_min + i;
     if (i < kMaxExps * kMaxExps) ctl->sums[i] = 0.0;
-}
-
-// sums[slot] += sum over the tile of (C - O)^2; also latches a GEMM device status into ctl->status
-__global__ void __launch_bounds__(256) pts_sqerr_kernel(const float* __restrict__ C, const float* __restrict__ O, long long ldo,
-                                                        int M, int N, PtsCtl* ctl, int slot, const int* gemm_status)
-{
-    double acc = 0.0;
-    const long long total = (long long)M * N;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
-        const long long m = i / N, n = i - m * N;
-        const double d = (double)C[i] - (double)O[m * ldo + n];
-        acc += d * d;
-    }
-    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
-    __shared__ double s_part[8];
-    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = acc;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        double t = 0.0;
-        for (int w = 0; w < 8; w++) t += s_part[w];
-        atomicAdd(&ctl->sums[slot], t);
-        if (blockIdx.x == 0 && *gemm_status) atomicCAS(&ctl->status, 0, *gemm_status);
-    }
 }
 
 __global__ void pts_finish_kernel(const PtsCtl* ctl, int e_min, int n_exp, double inv_count, float* d_err, int* d_best)
@@ -85,8 +64,8 @@ extern "C" size_t hif8_pts_workspace_bytes(int M, int N, int K, int n_exp)
 {
     if (M <= 0 || N <= 0 || K <= 0 || n_exp <= 0 || n_exp > kMaxExps) return 0;
     const size_t mk = (size_t)M * K, kn = (size_t)K * N;
-    return kCtlBytes + align256(mk) * n_exp + align256(kn) * n_exp + align256((size_t)M * N * 4) +
-           align256(hif8_workspace_bytes(HIF8_WS_GEMM, mk + kn));
+    // control block, one scratch byte tensor, n BF16 copies of each operand
+    return kCtlBytes + align256(mk > kn ? mk : kn) + (align256(mk * 2) + align256(kn * 2)) * (size_t)n_exp;
 }
 
 extern "C" int hif8_pts_search(const void* A, const void* W, int dtype, int w_is_nk, const float* O_ref, int64_t ldo, int M,
@@ -100,33 +79,38 @@ extern "C" int hif8_pts_search(const void* A, const void* W, int dtype, int w_is
     if (!A || !W || !O_ref || !d_err || !d_best) return HIF8_ERR_NULL;
     if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < hif8_pts_workspace_bytes(M, N, K, n_exp))
         return HIF8_ERR_WORKSPACE;
+    int dev = 0, major = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return HIF8_ERR_CUDA;
+    cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (major != 10) return HIF8_ERR_CUDA;
     cudaStream_t st = (cudaStream_t)stream;
     const size_t mk = (size_t)M * K, kn = (size_t)K * N;
     unsigned char* base = reinterpret_cast<unsigned char*>(workspace);
     PtsCtl* ctl = reinterpret_cast<PtsCtl*>(base);
-    unsigned char* aq = base + kCtlBytes;
-    unsigned char* wq = aq + align256(mk) * n_exp;
-    float* C = reinterpret_cast<float*>(wq + align256(kn) * n_exp);
-    unsigned char* gws = reinterpret_cast<unsigned char*>(C) + align256((size_t)M * N * 4);
-    const size_t gws_bytes = hif8_workspace_bytes(HIF8_WS_GEMM, mk + kn);
+    unsigned char* q_tmp = base + kCtlBytes;
+    unsigned char* a_bf = q_tmp + align256(mk > kn ? mk : kn);
+    unsigned char* w_bf = a_bf + align256(mk * 2) * n_exp;
 
     pts_init_kernel<<<1, 256, 0, st>>>(ctl, e_min, n_exp);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     if (cudaGetLastError() != cudaSuccess) return HIF8_ERR_CUDA;
-    for (int i = 0; i < n_exp; i++) {  // "Scale & Cast", once per exponent and operand
-        int rc = hif8_encode(A, dtype, aq + align256(mk) * i, mk, e_min + i, HIF8_RND_TA, 0, 0, stream);
-        if (rc == HIF8_OK) rc = hif8_encode(W, dtype, wq + align256(kn) * i, kn, e_min + i, HIF8_RND_TA, 0, 0, stream);
+    for (int i = 0; i < n_exp; i++) {  // "Scale & Cast", once per exponent and operand; the HiF8 values as BF16
+        int rc = hif8_encode(A, dtype, q_tmp, mk, e_min + i, HIF8_RND_TA, 0, 0, stream);
+        if (rc == HIF8_OK) rc = hif8_decode(q_tmp, a_bf + align256(mk * 2) * i, HIF8_BF16, mk, 0, stream);
+        if (rc == HIF8_OK) rc = hif8_encode(W, dtype, q_tmp, kn, e_min + i, HIF8_RND_TA, 0, 0, stream);
+        if (rc == HIF8_OK) rc = hif8_decode(q_tmp, w_bf + align256(kn * 2) * i, HIF8_BF16, kn, 0, stream);
         if (rc != HIF8_OK) return rc;
     }
-    const long long total = (long long)M * N;
-    const unsigned grid = (unsigned)(total / 1024 + 1 < 1184 ? total / 1024 + 1 : 1184);
+    GemmParams p{};
+    p.M = M; p.N = N; p.K = K;
+    p.status = &ctl->status;
+    p.err_ref = O_ref; p.ld_ref = ldo;
     for (int ia = 0; ia < n_exp; ia++)
-        for (int iw = 0; iw < n_exp; iw++) {  // "MatMul & Restore", "Quantization Error"
-            int rc = hif8_gemm(aq + align256(mk) * ia, K, wq + align256(kn) * iw, w_is_nk ? K : N, w_is_nk, C, N, HIF8_F32, M, N, K,
-                               &ctl->exps[ia], &ctl->exps[iw], gws, gws_bytes, stream);
+        for (int iw = 0; iw < n_exp; iw++) {  // "MatMul & Restore" and "Quantization Error" in one launch
+            p.d_sa = &ctl->exps[ia]; p.d_sw = &ctl->exps[iw];
+            p.err_sum = &ctl->sums[ia * n_exp + iw];
+            const int rc = launch_bf16_pair_gemm(a_bf + align256(mk * 2) * ia, w_bf + align256(kn * 2) * iw, w_is_nk, p, st);
             if (rc != HIF8_OK) return rc;
-            pts_sqerr_kernel<<<grid, 256, 0, st>>>(C, O_ref, ldo, M, N, ctl, ia * n_exp + iw, reinterpret_cast<const int*>(gws));
-            g_launches.fetch_add(1, std::memory_order_relaxed);
         }
     pts_finish_kernel<<<1, 32, 0, st>>>(ctl, e_min, n_exp, 1.0 / ((double)M * (double)N), d_err, d_best);
     g_launches.fetch_add(1, std::memory_order_relaxed);
