@@ -24,7 +24,8 @@
  *   options                  Section 3: saturation on overflow, NaN to zero.
  *   scaling                  Section 4.2 / 5.1: power-of-two per-tensor scale,
  *                            amax, descale (Algorithm 1, "Scale & Cast" and
- *                            "MatMul & Restore" steps).
+ *                            "MatMul & Restore" steps); per-channel weight
+ *                            scales; the every-N-iterations amax cadence.
  *
  * Readings taken where the paper is silent are marked "READING" below.
  * Pin status: every function here is pinned by tests/test_oracle_pins.py
@@ -413,6 +414,19 @@ void hif8o_decode(const uint8_t* src, void* dst, int dtype, size_t n, int scale_
     }
 }
 
+/* the scale rule of the READING below, for one amax */
+static int scale_exp_for(double amax, int target_exp)
+{
+    int se = 0;
+    if (amax > 0.0) {
+        int ex; (void)frexp(amax, &ex);
+        se = target_exp - (ex - 1);
+        if (se > 126) se = 126;
+        if (se < -126) se = -126;
+    }
+    return se;
+}
+
 /* amax over the finite elements and the power-of-two scale that brings it into
  * [2^target_exp, 2^(target_exp+1)).  READING of "update the scale factor by a
  * certain algorithm": scale_exp = target_exp - floor(log2 amax), clamped to
@@ -426,13 +440,7 @@ void hif8o_amax_scale(const void* src, int dtype, size_t n, int target_exp, floa
         uint32_t raw; double x = fabs(src_to_double(src, (size_t)i, dtype, &raw));
         if (isfinite(x) && x > amax) amax = x;
     }
-    int se = 0;
-    if (amax > 0.0) {
-        int ex; (void)frexp(amax, &ex);
-        se = target_exp - (ex - 1);
-        if (se > 126) se = 126;
-        if (se < -126) se = -126;
-    }
+    int se = scale_exp_for(amax, target_exp);
     *amax_out = (float)amax; /* exact: amax is a source value */
     *scale_exp_out = se;
 }
@@ -541,4 +549,97 @@ void hif8o_pts_search(const void* A, const void* W, int dtype, int w_is_nk, cons
     for (int i = 1; i < nE * nE; i++) if (err[i] < err[bi]) bi = i;
     best[0] = e_min + bi / nE; best[1] = e_min + bi % nE;
     free(da); free(dw);
+}
+
+/* ------------------------------------------------------------------------- *
+ * Section 5.1 / 5.3 outlook: "per-tensor scaling for activations and per-channel
+ * scaling for weights".  A weight matrix W [rows, cols] (row-major) gets one
+ * power-of-two scale per output channel: channel = row (axis 0, weights stored
+ * [N,K]) or channel = column (axis 1, weights stored [K,N]).  Each channel's
+ * amax and scale exponent follow the per-tensor rule applied to the elements of
+ * that channel alone.
+ * ------------------------------------------------------------------------- */
+void hif8o_channel_amax_scale(const void* W, int dtype, long long rows, long long cols, int axis, int target_exp,
+                              float* amax_out, int* scale_exp_out)
+{
+    long long channels = axis == 0 ? rows : cols, len = axis == 0 ? cols : rows;
+#pragma omp parallel for schedule(static)
+    for (long long c = 0; c < channels; c++) {
+        double amax = 0.0;
+        for (long long j = 0; j < len; j++) {
+            long long idx = axis == 0 ? c * cols + j : j * cols + c;
+            uint32_t raw; double x = fabs(src_to_double(W, (size_t)idx, dtype, &raw));
+            if (isfinite(x) && x > amax) amax = x;
+        }
+        amax_out[c] = (float)amax;
+        scale_exp_out[c] = scale_exp_for(amax, target_exp);
+    }
+}
+
+/* dst[r, c] = To_HiF8( W[r, c] * 2^scale_exp[channel of (r, c)] ); the stochastic word of element (r, c) is the one
+ * of flat index r * cols + c, as for a flat tensor */
+void hif8o_channel_encode(const void* W, int dtype, uint8_t* dst, long long rows, long long cols, int axis,
+                          const int* scale_exp, int rnd, unsigned flags, uint64_t seed, int quick)
+{
+#pragma omp parallel for schedule(static)
+    for (long long r = 0; r < rows; r++)
+        for (long long c = 0; c < cols; c++) {
+            long long idx = r * cols + c;
+            uint32_t raw; double x = src_to_double(W, (size_t)idx, dtype, &raw);
+            dst[idx] = (uint8_t)encode_value(x, raw, dtype, scale_exp[axis == 0 ? r : c], rnd, flags, seed,
+                                             (uint64_t)idx, quick);
+        }
+}
+
+/* "MatMul & Restore" with a per-tensor activation scale and per-channel weight scales:
+ * C*[m,n] = 2^-(sa + sw[n]) * sum_k dec(A[m,k]) dec(W[k,n]);  S likewise with |.| */
+void hif8o_gemm_entries_channel(const uint8_t* Aq, long long lda, const uint8_t* Wq, long long ldw, int w_is_nk,
+                                int K, int sa, const int* sw, const long long* rows, const long long* cols,
+                                size_t count, double* Cstar, double* S)
+{
+#pragma omp parallel for schedule(dynamic, 64)
+    for (long long t = 0; t < (long long)count; t++) {
+        long long m = rows[t], n = cols[t];
+        double acc = 0.0, sab = 0.0;
+        for (int k = 0; k < K; k++) {
+            double a = hif8o_value(Aq[m * lda + k]);
+            double w = hif8o_value(w_is_nk ? Wq[n * ldw + k] : Wq[(long long)k * ldw + n]);
+            acc += a * w; sab += fabs(a * w);
+        }
+        Cstar[t] = ldexp(acc, -(sa + sw[n]));
+        S[t] = ldexp(sab, -(sa + sw[n]));
+    }
+}
+
+/* ------------------------------------------------------------------------- *
+ * Section 5.1, the cadence of per-tensor scaling in training: "the initial scale
+ * factors are all set to 1.  Then every 10 iterations, we compute [Amax] of each
+ * tensor, and update the corresponding scale factor by a certain algorithm ...
+ * in each iteration, whether the scale factors are updated or not, they will
+ * scale the corresponding tensors".
+ * READING (the update algorithm is not given; the text likens the scheme to FP8
+ * delayed scaling): the state is the exponent in force (initially 0) and a ring
+ * of the last `hist_len` measured amax values (initially empty).  Iteration t
+ * converts its tensor with the exponent in force.  If t is a multiple of
+ * `interval`, the amax of that same tensor is measured, pushed into the ring
+ * (replacing the oldest entry once full) and the exponent becomes
+ * scale_exp_for(max of the ring, target_exp) from iteration t + 1 on.
+ * amax[t] is read only for t % interval == 0.  used[t] = exponent of iteration t.
+ * ------------------------------------------------------------------------- */
+void hif8o_delayed_scale_run(const float* amax, int T, int interval, int hist_len, int target_exp, int* used)
+{
+    double ring[64];
+    int filled = 0, pos = 0, se = 0;
+    if (hist_len > 64) hist_len = 64;
+    for (int t = 0; t < T; t++) {
+        used[t] = se;
+        if (t % interval == 0) {
+            ring[pos] = (double)amax[t];
+            pos = (pos + 1) % hist_len;
+            if (filled < hist_len) filled++;
+            double m = 0.0;
+            for (int j = 0; j < filled; j++) if (ring[j] > m) m = ring[j];
+            se = scale_exp_for(m, target_exp);
+        }
+    }
 }

@@ -31,6 +31,10 @@ _lib.hif8o_amax_scale.argtypes = [_vp, _i, _sz, _i, C.POINTER(C.c_float), C.POIN
 _lib.hif8o_fake_quant.argtypes = [_vp, _vp, _i, _sz, _i, _i, _u, _u64, _i]
 _lib.hif8o_gemm_entries.argtypes = [_vp, _ll, _vp, _ll, _i, _i, _i, _i, _vp, _vp, _sz, _vp, _vp]
 _lib.hif8o_pts_search.argtypes = [_vp, _vp, _i, _i, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp]
+_lib.hif8o_channel_amax_scale.argtypes = [_vp, _i, _ll, _ll, _i, _i, _vp, _vp]
+_lib.hif8o_channel_encode.argtypes = [_vp, _i, _vp, _ll, _ll, _i, _vp, _i, _u, _u64, _i]
+_lib.hif8o_gemm_entries_channel.argtypes = [_vp, _ll, _vp, _ll, _i, _i, _i, _vp, _vp, _vp, _sz, _vp, _vp]
+_lib.hif8o_delayed_scale_run.argtypes = [_vp, _i, _i, _i, _i, _vp]
 _lib.hif8o_gemm_full.argtypes = [_vp, _ll, _vp, _ll, _i, _i, _i, _i, _i, _i, _vp, _vp]
 
 
@@ -161,3 +165,48 @@ def pts_search(A, W, dtype, w_is_nk, O_ref, e_min=-4, e_max=5, quick=False):
     _lib.hif8o_pts_search(_ptr(A), _ptr(W), dtype, int(w_is_nk), _ptr(O_ref), M, N, K, e_min, e_max, int(quick),
                           _ptr(err), _ptr(best))
     return err, (int(best[0]), int(best[1]))
+
+
+def channel_amax_scale(W, dtype, axis, target_exp=14):
+    """Per-channel amax (float32) and scale exponents (int32) of W [rows, cols]; axis 0: channel = row, 1: column."""
+    W = _src(W, dtype)
+    rows, cols = W.shape
+    ch = rows if axis == 0 else cols
+    amax = np.empty(ch, dtype=np.float32)
+    se = np.empty(ch, dtype=np.int32)
+    _lib.hif8o_channel_amax_scale(_ptr(W), dtype, rows, cols, axis, target_exp, _ptr(amax), _ptr(se))
+    return amax, se
+
+
+def channel_encode(W, dtype, axis, scale_exp, rnd=TA, flags=0, seed=0, quick=False):
+    W = _src(W, dtype)
+    rows, cols = W.shape
+    se = np.ascontiguousarray(scale_exp, dtype=np.int32)
+    assert se.size == (rows if axis == 0 else cols)
+    out = np.empty((rows, cols), dtype=np.uint8)
+    _lib.hif8o_channel_encode(_ptr(W), dtype, _ptr(out), rows, cols, axis, _ptr(se), rnd, flags, seed, int(quick))
+    return out
+
+
+def gemm_entries_channel(Aq, Wq, w_is_nk, sa, sw, rows, cols):
+    """As gemm_entries with one weight exponent per output column: sw int32 [N]."""
+    Aq = np.ascontiguousarray(Aq, dtype=np.uint8)
+    Wq = np.ascontiguousarray(Wq, dtype=np.uint8)
+    K = Aq.shape[1]
+    sw = np.ascontiguousarray(sw, dtype=np.int32)
+    assert sw.size == (Wq.shape[0] if w_is_nk else Wq.shape[1])
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    cols = np.ascontiguousarray(cols, dtype=np.int64)
+    cs = np.empty(rows.size, dtype=np.float64)
+    s = np.empty(rows.size, dtype=np.float64)
+    _lib.hif8o_gemm_entries_channel(_ptr(Aq), Aq.shape[1], _ptr(Wq), Wq.shape[1], int(w_is_nk), K, sa, _ptr(sw),
+                                    _ptr(rows), _ptr(cols), rows.size, _ptr(cs), _ptr(s))
+    return cs, s
+
+
+def delayed_scale_run(amax, interval, hist_len, target_exp=14):
+    """Exponent in force at each iteration of the every-`interval`-iterations amax cadence (int32 [T])."""
+    amax = np.ascontiguousarray(amax, dtype=np.float32)
+    used = np.empty(amax.size, dtype=np.int32)
+    _lib.hif8o_delayed_scale_run(_ptr(amax), amax.size, interval, hist_len, target_exp, _ptr(used))
+    return used

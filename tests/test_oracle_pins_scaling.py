@@ -1,0 +1,127 @@
+"""Pins for the oracle's per-channel weight scaling (Section 5.1: per-tensor scaling for activations and per-channel
+scaling for weights) and for the every-N-iterations amax cadence of Section 5.1.  Each check compares the oracle
+with something it does not compute itself: the already pinned per-tensor routines on extracted slices, properties
+that hold for any correct implementation, or sequences worked out by hand."""
+import numpy as np
+import pytest
+
+import workloads as W
+from oracle import hif8_oracle as O
+
+
+def weight(rows, cols, seed, dtype):
+    x = W.normal_f32(rows * cols, seed).reshape(rows, cols)
+    x *= np.exp2(np.random.default_rng(seed).integers(-12, 12, size=(1, cols))).astype(np.float32)  # channels differ
+    x[3, 5] = np.inf
+    x[4, 7] = np.nan
+    x[:, 2] = 0.0  # an all-zero column
+    return x if dtype == O.F32 else W.f32_to_bf16_bits(x)
+
+
+@pytest.mark.parametrize("dtype", [O.F32, O.BF16])
+@pytest.mark.parametrize("axis", [0, 1])
+def test_channel_scale_is_the_per_tensor_rule_on_each_slice(dtype, axis):
+    x = weight(37, 29, 11, dtype)
+    amax, se = O.channel_amax_scale(x, dtype, axis, target_exp=9)
+    for c in range(x.shape[axis]):
+        sl = np.ascontiguousarray(x[c, :] if axis == 0 else x[:, c])
+        a1, s1 = O.amax_scale(sl, dtype, 9)  # pinned in test_oracle_pins.py::test_amax_scale_closed_form
+        assert (amax[c], se[c]) == (np.float32(a1), s1)
+        if a1 > 0:
+            assert 2.0 ** 9 <= a1 * 2.0 ** s1 < 2.0 ** 10
+    if axis == 1:
+        assert amax[2] == 0 and se[2] == 0  # the all-zero column keeps exponent 0
+
+
+@pytest.mark.parametrize("mode", [O.TA, O.HR, O.SR])
+@pytest.mark.parametrize("axis", [0, 1])
+def test_channel_encode_against_slices_transpose_and_uniform_case(mode, axis):
+    dtype = O.BF16
+    x = weight(24, 40, 5, dtype)
+    _, se = O.channel_amax_scale(x, dtype, axis)
+    q = O.channel_encode(x, dtype, axis, se, rnd=mode, seed=9)
+    if mode != O.SR:
+        # deterministic given the source bits: every channel equals the flat encoder on that slice ...
+        for c in range(x.shape[axis]):
+            sl = np.ascontiguousarray(x[c, :] if axis == 0 else x[:, c])
+            assert np.array_equal(q[c, :] if axis == 0 else q[:, c], O.encode(sl, dtype, int(se[c]), mode))
+        # ... and the transposed matrix with the other axis gives the transposed codes
+        qt = O.channel_encode(np.ascontiguousarray(x.T), dtype, 1 - axis, se, rnd=mode)
+        assert np.array_equal(qt.T, q)
+    # one common exponent: the flat per-tensor encoder, stochastic words included (flat index r * cols + c)
+    same = np.full(x.shape[axis], 3, dtype=np.int32)
+    assert np.array_equal(O.channel_encode(x, dtype, axis, same, rnd=mode, seed=9).ravel(),
+                          O.encode(x.ravel(), dtype, 3, mode, seed=9))
+
+
+def test_channel_scale_shift_property():
+    # multiplying one channel by 2^j moves that channel's exponent by -j and changes no code anywhere
+    x = W.normal_f32(32 * 16, 3).reshape(32, 16)
+    _, se = O.channel_amax_scale(x, O.F32, 1)
+    q = O.channel_encode(x, O.F32, 1, se)
+    y = x.copy()
+    y[:, 4] *= 2.0 ** 7
+    _, se2 = O.channel_amax_scale(y, O.F32, 1)
+    d = se2 - se
+    assert d[4] == -7 and not d[np.arange(16) != 4].any()
+    assert np.array_equal(O.channel_encode(y, O.F32, 1, se2), q)
+
+
+def test_channel_roundtrip_error_bound():
+    # TA keeps >= 1 mantissa bit over the whole normal range: |w - dec| <= 2^-2 |w| at worst, 2^-4 |w| near amax
+    x = W.normal_f32(64 * 48, 8).reshape(64, 48) * np.exp2(np.arange(48) - 24).astype(np.float32)
+    _, se = O.channel_amax_scale(x, O.F32, 1, 14)
+    q = O.channel_encode(x, O.F32, 1, se)
+    back = np.stack([O.decode(q[:, c], O.F32, int(se[c])).view(np.float32) for c in range(48)], axis=1).astype(np.float64)
+    big = np.abs(x) * np.exp2(se)[None, :] >= 2.0 ** -15
+    assert np.all(np.abs(back - x)[big] <= 2.0 ** -2 * np.abs(x)[big])
+    top = np.abs(x) * np.exp2(se)[None, :] >= 2.0 ** 8       # scaled exponent in [8, 15]: 1 or 2 mantissa bits
+    assert np.all(np.abs(back - x)[top] <= 2.0 ** -2 * np.abs(x)[top])
+    mid = (np.abs(x) * np.exp2(se)[None, :] >= 2.0 ** -3) & (np.abs(x) * np.exp2(se)[None, :] < 2.0 ** 3)
+    assert mid.any() and np.all(np.abs(back - x)[mid] <= 2.0 ** -4 * np.abs(x)[mid] * (1 + 1e-12))
+
+
+@pytest.mark.parametrize("w_is_nk", [0, 1])
+def test_gemm_channel_is_the_per_tensor_product_times_column_powers(w_is_nk):
+    M, N, K = 9, 12, 48
+    Aq = W.random_codes(M * K, 1).reshape(M, K)
+    Wq = W.random_codes(K * N, 2).reshape((N, K) if w_is_nk else (K, N))
+    for t in (Aq, Wq):
+        t[(t == 0x80) | ((t & 0x7F) == 0x6F)] = 0x10
+    sw = np.random.default_rng(4).integers(-20, 20, size=N).astype(np.int32)
+    rows, cols = np.divmod(np.arange(M * N), N)
+    c0, s0 = O.gemm_entries(Aq, Wq, w_is_nk, 0, 0, rows, cols)  # pinned against numpy in test_oracle_pins.py
+    c1, s1 = O.gemm_entries_channel(Aq, Wq, w_is_nk, 5, sw, rows, cols)
+    f = np.exp2(-(5.0 + sw[cols]))
+    assert np.array_equal(c1, c0 * f) and np.array_equal(s1, s0 * f)
+    # a column's exponent must not leak into its neighbours
+    sw2 = sw.copy()
+    sw2[3] += 1
+    c2, _ = O.gemm_entries_channel(Aq, Wq, w_is_nk, 5, sw2, rows, cols)
+    assert np.array_equal(c2[cols != 3], c1[cols != 3]) and np.array_equal(c2[cols == 3] * 2, c1[cols == 3])
+
+
+def test_delayed_scale_sequences_worked_by_hand():
+    # history of one, update every iteration: iteration t uses the exponent of the amax seen at t-1; the first uses 0
+    amax = np.array([3.0, 0.4, 100.0, 100.0, 0.0, 7.0], dtype=np.float32)
+    #    floor(log2):   1    -2     6      6     -    2         target 14 ->  13, 16, 8, 8, 0(amax 0), 12
+    assert O.delayed_scale_run(amax, 1, 1, 14).tolist() == [0, 13, 16, 8, 8, 0]
+    # history of three: the exponent follows the largest of the last three measurements
+    #   rings: [3] [3,.4] [3,.4,100] [.4,100,100] [100,100,0] [100,0,7]   max: 3 3 100 100 100 100
+    assert O.delayed_scale_run(amax, 1, 3, 14).tolist() == [0, 13, 13, 8, 8, 8]
+    # a spike leaves the ring after hist_len further measurements
+    spike = np.array([1, 1, 64, 1, 1, 1, 1], dtype=np.float32)
+    assert O.delayed_scale_run(spike, 1, 2, 14).tolist() == [0, 14, 14, 8, 8, 14, 14]
+    # measurements only at multiples of the interval; values in between are never read
+    seq = np.array([2.0, 999, 999, 0.5, 999, 999, 32.0, 999], dtype=np.float32)
+    assert O.delayed_scale_run(seq, 3, 1, 10).tolist() == [0, 9, 9, 9, 11, 11, 11, 5]
+
+
+def test_delayed_scale_with_history_one_matches_the_per_tensor_rule():
+    rng = np.random.default_rng(2)
+    tensors = [W.normal_f32(257, 100 + t) * np.float32(2.0 ** rng.integers(-30, 30)) for t in range(12)]
+    amax = np.array([np.max(np.abs(x)) for x in tensors], dtype=np.float32)
+    used = O.delayed_scale_run(amax, 1, 1, 12)
+    assert used[0] == 0
+    for t in range(1, 12):
+        assert used[t] == O.amax_scale(tensors[t - 1], O.F32, 12)[1]
