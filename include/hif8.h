@@ -144,6 +144,47 @@ int hif8_amax_scale_encode_static(const void* src, int src_dtype, uint8_t* dst, 
                                   int* d_scale_exp_out, float* d_scale_out, hif8_stream_t stream);
 
 /*
+ * Per-channel scaled conversion of a weight matrix (Section 5.1, end: "per-tensor scaling for activations and
+ * per-channel scaling for weights"; repeated in the outlook of Section 5.3).  W is [rows, cols] row-major and
+ * contiguous; every output channel has its own power-of-two scale:
+ *   channel_axis = 0: channel = row    (weights stored [N,K]);   channel_axis = 1: channel = column (stored [K,N]).
+ *   d_scale_exp_in == NULL: per channel, amax over the channel's finite elements and
+ *        scale_exp = clamp(target_exp - floor(log2 amax), -126, 126) (0 for an all-zero channel), the per-tensor rule
+ *        of hif8_amax_scale_encode applied to the channel alone; d_amax [channels] receives the amax values (it is also
+ *        the accumulator of the reduction and must not be NULL).
+ *   d_scale_exp_in != NULL: the exponents are read from that device array [channels]; d_amax is not touched.
+ *   dst[r, c] = To_HiF8_<rnd>( W[r, c] * 2^scale_exp[channel(r, c)] ), same layout as W, one byte per element.
+ * d_scale_exp_out [channels] (may be NULL; may equal d_scale_exp_in): the exponents used, ready for
+ * hif8_gemm_channel_scaled.  HIF8_RND_SR draws the word of flat index r * cols + c, as hif8_encode would.
+ * Needs no workspace.  The fast path wants 16-byte aligned pointers and rows (cols * element size a multiple of 16);
+ * anything else takes a slower element-wise path with identical results.
+ */
+int hif8_channel_amax_scale_encode(const void* W, int src_dtype, uint8_t* dst, int64_t rows, int64_t cols,
+                                   int channel_axis, int target_exp, int rnd, unsigned flags, uint64_t seed,
+                                   const int* d_scale_exp_in, float* d_amax, int* d_scale_exp_out,
+                                   hif8_stream_t stream);
+
+/*
+ * The every-N-iterations cadence of per-tensor scaling in training (Section 5.1: scale factors start at 1; "every 10
+ * iterations" the amax of each tensor is computed and its scale updated; the scale in force is applied in every
+ * iteration, updated or not).  The paper does not give the update rule; this library keeps, per tensor, the exponent
+ * in force and a ring of the last `hist_len` measured amax values, and after a measurement sets
+ *   scale_exp = clamp(target_exp - floor(log2 max(ring)), -126, 126)      (0 while every entry is 0)
+ * which takes effect from the next conversion on.  The state lives in HIF8_SCALE_STATE_BYTES of device memory
+ * (256-byte aligned) owned by the caller; nothing returns to the host.
+ *   hif8_scale_state_init:      exponent 0, empty ring of hist_len entries (1..HIF8_SCALE_HISTORY_MAX).
+ *   hif8_delayed_scale_encode:  dst = To_HiF8_<rnd>(src * 2^(exponent in force)) in one pass over src.  With
+ *        measure != 0 (the caller's "iteration % N == 0") the same pass also reduces amax of src, and a one-thread
+ *        kernel then pushes it into the ring and updates the exponent.  The first int of the state is the exponent
+ *        in force (readable as the d_scale_exp_a / d_scale_exp_w of hif8_gemm), the float at byte 16 the last amax.
+ */
+#define HIF8_SCALE_STATE_BYTES 1024
+#define HIF8_SCALE_HISTORY_MAX 32
+int hif8_scale_state_init(void* d_state, int hist_len, hif8_stream_t stream);
+int hif8_delayed_scale_encode(const void* src, int src_dtype, uint8_t* dst, size_t n, int rnd, unsigned flags,
+                              uint64_t seed, void* d_state, int measure, int target_exp, hif8_stream_t stream);
+
+/*
  * Quantize-dequantize in the source format ("simulated HiF8", Section 4: values are converted to only those
  * representable in HiF8):   dst[i] = value( To_HiF8_<rnd>(src[i] * 2^e) ) * 2^(-e)   in `dtype`.
  *   use_amax == 0: e = scale_or_target_exp.  No workspace needed (may be NULL).
@@ -175,6 +216,16 @@ int hif8_fake_quant(const void* src, void* dst, int dtype, size_t n, int use_ama
 int hif8_gemm(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int64_t ldw, int w_is_nk, void* C,
               int64_t ldc, int c_dtype, int M, int N, int K, const int* d_scale_exp_a,
               const int* d_scale_exp_w, void* workspace, size_t workspace_bytes, hif8_stream_t stream);
+
+/*
+ * hif8_gemm with one weight exponent per output channel (per-tensor activation scale, per-channel weight scales):
+ *   C[m,n] = 2^-(sa + sw[n]) * sum_k value(Aq[m,k]) * value(Wq[k,n]),   d_scale_exp_w_channel: device int [N], not NULL.
+ * Everything else as hif8_gemm.
+ */
+int hif8_gemm_channel_scaled(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int64_t ldw, int w_is_nk, void* C,
+                             int64_t ldc, int c_dtype, int M, int N, int K, const int* d_scale_exp_a,
+                             const int* d_scale_exp_w_channel, void* workspace, size_t workspace_bytes,
+                             hif8_stream_t stream);
 
 /*
  * Host-side query of the status word of a finished hif8_gemm: copies it from `workspace`, SYNCHRONISES `stream`,

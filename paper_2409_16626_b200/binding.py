@@ -14,11 +14,13 @@ RND_TA, RND_HR, RND_SSR, RND_TE, RND_SR = 0, 1, 2, 3, 4
 FLAG_SATURATE, FLAG_NAN_TO_ZERO = 1, 2
 WS_AMAX_SCALE_ENCODE, WS_FAKE_QUANT, WS_GEMM = 0, 1, 2
 OK = 0
+SCALE_STATE_BYTES, SCALE_HISTORY_MAX = 1024, 32
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libhif8.so")
 EXPORTS = ["hif8_encode", "hif8_decode", "hif8_amax", "hif8_amax_scale_encode", "hif8_fake_quant", "hif8_gemm", "hif8_gemm_status", "hif8_pts_search", "hif8_pts_workspace_bytes",
-           "hif8_pts_status", "hif8_selftest_wait_timeout",
+           "hif8_pts_status", "hif8_selftest_wait_timeout", "hif8_channel_amax_scale_encode", "hif8_gemm_channel_scaled",
+           "hif8_scale_state_init", "hif8_delayed_scale_encode",
            "hif8_amax_scale_encode_static", "hif8_workspace_bytes", "hif8_status_string", "hif8_launch_count"]
 
 if not os.path.exists(LIB_PATH):
@@ -45,6 +47,14 @@ lib.hif8_pts_status.argtypes = [_vp, _vp]
 lib.hif8_pts_status.restype = _i
 lib.hif8_selftest_wait_timeout.argtypes = [_vp, _u, _vp]
 lib.hif8_selftest_wait_timeout.restype = _i
+lib.hif8_channel_amax_scale_encode.argtypes = [_vp, _i, _vp, _i64, _i64, _i, _i, _i, _u, _u64, _vp, _vp, _vp, _vp]
+lib.hif8_channel_amax_scale_encode.restype = _i
+lib.hif8_gemm_channel_scaled.argtypes = lib.hif8_gemm.argtypes
+lib.hif8_gemm_channel_scaled.restype = _i
+lib.hif8_scale_state_init.argtypes = [_vp, _i, _vp]
+lib.hif8_scale_state_init.restype = _i
+lib.hif8_delayed_scale_encode.argtypes = [_vp, _i, _vp, _sz, _i, _u, _u64, _vp, _i, _i, _vp]
+lib.hif8_delayed_scale_encode.restype = _i
 lib.hif8_workspace_bytes.argtypes = [_i, _sz]
 lib.hif8_workspace_bytes.restype = _sz
 lib.hif8_status_string.argtypes = [_i]
@@ -157,3 +167,27 @@ def hif8_pts_status(workspace, stream=None):
 
 def hif8_selftest_wait_timeout(workspace, limit_ms, stream=None, check=True):
     return _check(lib.hif8_selftest_wait_timeout(_ptr(workspace), limit_ms, _stream(stream)), check)
+
+
+def hif8_channel_amax_scale_encode(W, src_dtype, dst, rows, cols, channel_axis, target_exp=14, rnd=RND_TA, flags=0, seed=0,
+                                   d_scale_exp_in=None, d_amax=None, d_scale_exp_out=None, stream=None, check=True):
+    return _check(lib.hif8_channel_amax_scale_encode(_ptr(W), src_dtype, _ptr(dst), rows, cols, channel_axis, target_exp, rnd,
+                                                     flags, seed, _ptr(d_scale_exp_in), _ptr(d_amax), _ptr(d_scale_exp_out),
+                                                     _stream(stream)), check)
+
+
+def hif8_gemm_channel_scaled(Aq, lda, Wq, ldw, w_is_nk, Cmat, ldc, c_dtype, M, N, K, d_scale_exp_a=None,
+                             d_scale_exp_w_channel=None, workspace=None, workspace_bytes=0, stream=None, check=True):
+    return _check(lib.hif8_gemm_channel_scaled(_ptr(Aq), lda, _ptr(Wq), ldw, w_is_nk, _ptr(Cmat), ldc, c_dtype, M, N, K,
+                                               _ptr(d_scale_exp_a), _ptr(d_scale_exp_w_channel), _ptr(workspace),
+                                               workspace_bytes, _stream(stream)), check)
+
+
+def hif8_scale_state_init(d_state, hist_len, stream=None, check=True):
+    return _check(lib.hif8_scale_state_init(_ptr(d_state), hist_len, _stream(stream)), check)
+
+
+def hif8_delayed_scale_encode(src, src_dtype, dst, n, rnd, flags, seed, d_state, measure, target_exp=14, stream=None,
+                              check=True):
+    return _check(lib.hif8_delayed_scale_encode(_ptr(src), src_dtype, _ptr(dst), n, rnd, flags, seed, _ptr(d_state),
+                                                int(measure), target_exp, _stream(stream)), check)

@@ -27,337 +27,14 @@
 #include <cstdint>
 
 #include "hif8.h"
+#include "hif8_device.cuh"
+#include "hif8_internal.cuh"
 
 namespace hif8 {
 
 std::atomic<uint64_t> g_launches{0};
 
 namespace {
-
-constexpr int kThreads = 256;
-constexpr int kUnroll = 4;
-constexpr int kBlocksPerSM = 8;
-
-// ------------------------------------------------------------------------------------------------
-// Field packing (Table 1: sign | dot | exponent | mantissa; Table 2 prefix code; Table 3 exponent ranges)
-// ------------------------------------------------------------------------------------------------
-__host__ __device__ constexpr int mant_width(int E)
-{
-    int a = E < 0 ? -E : E;
-    return (E <= -16) ? 0 : (a <= 3 ? 3 : (a <= 7 ? 2 : 1));
-}
-
-// magnitude byte (bit 7 clear) of 2^E * 1.M, E in [-22, 15], M already `mant_width(E)` bits wide
-__host__ __device__ constexpr uint32_t pack_magnitude(int E, uint32_t M)
-{
-    if (E <= -16) return (uint32_t)(E + 23);  // Eq. 2: denormal, mantissa field = E + 23
-    uint32_t a = (uint32_t)(E < 0 ? -E : E), se = E < 0 ? 1u : 0u;
-    if (a == 0) return 0x08u | M;                                     // dot 0001
-    if (a == 1) return 0x10u | (se << 3) | M;                         // dot 001, Em = {Se}
-    if (a <= 3) return 0x20u | (se << 4) | ((a & 1u) << 3) | M;       // dot 01,  Em = {Se, Mag[2]}
-    if (a <= 7) return 0x40u | (se << 4) | ((a & 3u) << 2) | M;       // dot 10,  Em = {Se, Mag[2:3]}
-    return 0x60u | (se << 4) | ((a & 7u) << 1) | M;                   // dot 11,  Em = {Se, Mag[2:4]}
-}
-
-// Round-half-away result for the binary32 patterns whose top 13 bits are `idx`
-// (1 sign, 8 exponent, 4 mantissa bits).
-__host__ __device__ constexpr uint8_t ta_entry(uint32_t idx)
-{
-    uint32_t sign = (idx >> 12) << 7;
-    int e = (int)((idx >> 4) & 0xFF);
-    uint32_t m4 = idx & 0xF;
-    if (e == 255) return m4 ? (uint8_t)0x80 : (uint8_t)(sign | 0x6F);   // NaN (canonical has m4 = 15) / Inf
-    int E = e - 127;
-    if (E >= 16) return (uint8_t)(sign | 0x6F);
-    if (E <= -24) return 0;                       // below half of 2^-22: the single zero pattern
-    if (E == -23) return (uint8_t)(sign | 0x01);  // [2^-23, 2^-22) rounds up to 2^-22 (tie away)
-    int w = mant_width(E);
-    uint32_t M = m4 >> (4 - w);
-    uint32_t rbit = (m4 >> (3 - w)) & 1u;         // MSB of the discarded bits
-    M += rbit;
-    if (M == (1u << w)) { M = 0; E += 1; }        // carry into the exponent; the mantissa is then zero
-    if (E >= 16) return (uint8_t)(sign | 0x6F);
-    return (uint8_t)(sign | pack_magnitude(E, M));  // E = 15, M = 1 is the Inf pattern by construction
-}
-
-struct TaTable { uint8_t v[8192]; };
-constexpr TaTable make_ta_table()
-{
-    TaTable t{};
-    for (uint32_t i = 0; i < 8192; i++) t.v[i] = ta_entry(i);
-    return t;
-}
-__device__ const TaTable g_ta_table = make_ta_table();
-
-// value of one byte as binary32 bits (Eq. 1 / Eq. 2 / specials)
-__device__ __forceinline__ uint32_t decode_bits_f32(uint32_t c)
-{
-    uint32_t sign = (c & 0x80u) << 24, m = c & 0x7Fu;
-    if (m == 0) return sign ? 0x7FC00000u : 0u;
-    if (m == 0x6F) return sign | 0x7F800000u;
-    if (m < 8) return sign | ((m + 104u) << 23);  // 2^(m-23)
-    int E; uint32_t M, w;
-    if (m < 0x10)      { E = 0; M = m & 7; w = 3; }
-    else if (m < 0x20) { E = 1; M = m & 7; w = 3; if (m & 0x08) E = -E; }
-    else if (m < 0x40) { E = 2 | ((m >> 3) & 1); M = m & 7; w = 3; if (m & 0x10) E = -E; }
-    else if (m < 0x60) { E = 4 | ((m >> 2) & 3); M = m & 3; w = 2; if (m & 0x10) E = -E; }
-    else               { E = 8 | ((m >> 1) & 7); M = m & 1; w = 1; if (m & 0x10) E = -E; }
-    return sign | ((uint32_t)(E + 127) << 23) | (M << (23 - w));
-}
-
-// ------------------------------------------------------------------------------------------------
-// Philox4x32-10 (Salmon et al., SC'11): counter (c0, c1, 0, 0), key (k0, k1)
-// ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t k0, uint32_t k1)
-{
-    uint32_t x0 = c0, x1 = c1, x2 = 0, x3 = 0;
-#pragma unroll
-    for (int r = 0; r < 10; r++) {
-        uint32_t hi0 = __umulhi(0xD2511F53u, x0), lo0 = 0xD2511F53u * x0;
-        uint32_t hi1 = __umulhi(0xCD9E8D57u, x2), lo1 = 0xCD9E8D57u * x2;
-        uint32_t n0 = hi1 ^ x1 ^ k0, n2 = hi0 ^ x3 ^ k1;
-        x0 = n0; x1 = lo1; x2 = n2; x3 = lo0;
-        k0 += 0x9E3779B9u; k1 += 0xBB67AE85u;
-    }
-    return make_uint4(x0, x1, x2, x3);
-}
-
-// ------------------------------------------------------------------------------------------------
-// Programmatic dependent launch.  Every kernel here is launched so that it may be scheduled while the previous
-// kernel of the stream is still draining: it signals its own dependents at once (they can only start after all of
-// this grid's blocks have started), does the work that touches no global input (table set-up), and waits for the
-// previous grid to have completed and flushed before its first global read or write.
-// ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void pdl_wait_prior_grid() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
-// ------------------------------------------------------------------------------------------------
-// Scale handling
-// ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ int clamp_exp(int e) { return e < -126 ? -126 : (e > 126 ? 126 : e); }
-__device__ __forceinline__ float pow2f(int e) { return __uint_as_float((uint32_t)(e + 127) << 23); }  // |e| <= 126
-
-// scale exponent from the bits of amax (a non-negative finite binary32)
-__device__ __forceinline__ int scale_exp_from_amax(uint32_t ab, int target_exp)
-{
-    if (ab == 0) return 0;
-    int e = (ab >> 23) ? (int)(ab >> 23) - 127 : (31 - __clz(ab)) - 149;  // floor(log2 amax)
-    return clamp_exp(target_exp - e);
-}
-
-struct ConvParams {
-    const void* src;
-    void* dst;
-    unsigned long long n;
-    int scale_exp;                // used when neither pointer below is set
-    const int* d_scale_exp;       // delayed scaling: exponent read from the device
-    const uint32_t* d_amax_bits;  // just-in-time scaling: exponent derived from this amax
-    int target_exp;
-    unsigned flags;
-    unsigned long long seed;
-    uint32_t* amax_accum;         // when the kernel also reduces amax: accumulator and ticket (2 words)
-    float* d_amax_out;
-    int* d_scale_exp_out;
-    float* d_scale_out;
-};
-
-template <int SRC> struct SrcTraits;
-template <> struct SrcTraits<HIF8_F32>  { static constexpr int kPerVec = 4; };
-template <> struct SrcTraits<HIF8_BF16> { static constexpr int kPerVec = 8; };
-template <> struct SrcTraits<HIF8_F16>  { static constexpr int kPerVec = 8; };
-
-// element k of a 16-byte source vector: its value as binary32 and its raw encoding
-template <int SRC>
-__device__ __forceinline__ void unpack(const uint4& v, int k, float& x, uint32_t& raw)
-{
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-    if (SRC == HIF8_F32) { raw = w[k]; x = __uint_as_float(raw); }
-    else {
-        uint32_t word = w[k >> 1];
-        raw = (k & 1) ? (word >> 16) : (word & 0xFFFFu);
-        if (SRC == HIF8_BF16) x = __uint_as_float(raw << 16);
-        else x = __half2float(__ushort_as_half((unsigned short)raw));
-    }
-}
-
-template <int SRC>
-__device__ __forceinline__ void load_scalar(const void* p, unsigned long long i, float& x, uint32_t& raw)
-{
-    if (SRC == HIF8_F32) { raw = reinterpret_cast<const uint32_t*>(p)[i]; x = __uint_as_float(raw); }
-    else {
-        raw = reinterpret_cast<const unsigned short*>(p)[i];
-        if (SRC == HIF8_BF16) x = __uint_as_float(raw << 16);
-        else x = __half2float(__ushort_as_half((unsigned short)raw));
-    }
-}
-
-// binary32 value -> encoding of the destination format, round to nearest even
-template <int DT> __device__ __forceinline__ uint32_t to_bits(float v)
-{
-    if (DT == HIF8_F32) return (v != v) ? 0x7FC00000u : __float_as_uint(v);
-    if (DT == HIF8_BF16) {
-        if (v != v) return 0x7FC0u;
-        return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v));
-    }
-    if (v != v) return 0x7E00u;
-    return (uint32_t)__half_as_ushort(__float2half_rn(v));
-}
-
-// ------------------------------------------------------------------------------------------------
-// One element: scaled value -> HiF8 byte
-// ------------------------------------------------------------------------------------------------
-// Per-exponent entry of the rounding table (indexed by the biased exponent of the scaled magnitude):
-//   bits 0-4   number of discarded mantissa bits (23 - width); 0: nothing to round (overflow, Inf, NaN)
-//   bits 8-12  left shift that aligns an N-bit threshold complement with the top of the discarded field
-//   bit  7     this binade rounds stochastically (the complement comes from the source bits)
-//   bits 16-31 otherwise: the constant to shift instead (half of 2^N for round-half-away binades, 0 for none)
-constexpr uint32_t kThrStochastic = 0x80u;
-
-template <int MODE, int SRC>
-__device__ __forceinline__ uint32_t encode_one(float x, uint32_t raw, float scale, const uint8_t* s_ta,
-                                               const uint32_t* s_thr, uint32_t word)
-{
-    const float y = x * scale;
-    uint32_t t = __float_as_uint(y);
-    if (MODE == HIF8_RND_TA) return s_ta[t >> 19];
-
-    const bool sub = (t & 0x7FFFFFFFu) < 0x34800000u;  // |y| < 2^-22 (zero included): result is 0 or 2^-22
-    // Below 2^-22 the kept bits are zero and the fraction is F = |y| / 2^-22.  Adding 2^-22 with truncation puts
-    // floor(F 2^23) into the mantissa field of a value in the binade of 2^-22, so the common code rounds it like a
-    // 0-bit-mantissa binade (result 2^-22 or 2^-21); it is moved down again afterwards.
-    const uint32_t tz = __float_as_uint(__fadd_rz(fabsf(y), 2.384185791015625e-07f));
-
-    if (MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR) {
-        // hybrid / simplified stochastic rounding: the carry of (magnitude + (2^N - T) << k) does the rounding
-        const uint32_t u = sub ? tz : (t & 0x7FFFFFFFu);
-        const uint32_t ent = s_thr[u >> 23];
-        const uint32_t d_ssr = (SRC == HIF8_F32) ? 0x4000u - max(raw & 0x3FFFu, 1u)   // SR14: 2^14 - max(T14, 1)
-                                                 : 3u - 2u * (raw & 1u);               // SR2:  4 - {source LSB, 1}
-        const uint32_t d = (ent & kThrStochastic) ? d_ssr : (ent >> 16);
-        uint32_t tr = (u + (d << ((ent >> 8) & 31u))) & (0xFFFFFFFFu << (ent & 31u));
-        // below 2^-22: two binades down, so that 2^-21 packs as 2^-22 and 2^-22 as the single zero
-        tr -= sub ? 0x01000000u : 0u;
-        return s_ta[(tr >> 19) | ((t >> 19) & 0x1000u)];
-    }
-
-    // TE and standard SR
-    constexpr int kSrBits = (SRC == HIF8_F32) ? 24 : 16;
-    const uint32_t sign7 = (t >> 24) & 0x80u;
-    if (MODE == HIF8_RND_SR && SRC == HIF8_F32 && sub) {
-        // the 24-bit threshold is wider than a binary32 fraction: compare F24 = floor(|y| 2^46) directly
-        const uint32_t f24 = __float2uint_rz(fabsf(y) * 70368744177664.f);
-        return f24 >= max(word >> 8, 1u) ? (sign7 | 0x01u) : 0u;
-    }
-    t = sub ? (tz | (t & 0x80000000u)) : t;
-    const uint32_t sh = s_thr[(t >> 23) & 0xFFu] & 31u;  // discarded mantissa bits (23 - width); 0: nothing to round
-    const uint32_t s = sh ? sh : 23u;
-    uint32_t inc;
-    if (MODE == HIF8_RND_TE) {
-        // add half-1, plus one when the kept significand is odd (the implicit one when no mantissa bit is kept,
-        // zero below 2^-22)
-        uint32_t lsb = (s == 23u) ? 1u : ((t >> s) & 1u);
-        if (sub) lsb = 0u;
-        inc = (1u << (s - 1)) - 1u + lsb;
-    } else {  // standard SR (threshold T of Section 3.2, compared as max(T,1) so that a zero fraction never rounds up)
-        const uint32_t T = max(word >> (32 - kSrBits), 1u);
-        if (SRC == HIF8_F32) {
-            const uint32_t k = 24u - s;  // F24 = discarded << k; up iff discarded >= ceil(T / 2^k)
-            inc = (1u << s) - ((T + (1u << k) - 1u) >> k);
-        } else inc = (0x10000u - T) << (s - 16);
-    }
-    if (sh == 0) inc = 0;
-    const uint32_t tr = (t + inc) & (0xFFFFFFFFu << sh);
-    uint32_t code = s_ta[tr >> 19];
-    if (sub) {
-        if (MODE == HIF8_RND_TE)  // nearest: up iff above the midpoint 2^-23 (the tie goes to the even value, zero)
-            code = (__float_as_uint(y) & 0x7FFFFFFFu) > 0x34000000u ? (sign7 | 0x01u) : 0u;
-        else code = ((code & 0x7Fu) == 0x02u) ? (sign7 | 0x01u) : 0u;  // 2^-21 -> 2^-22, 2^-22 -> the single zero
-    }
-    return code;
-}
-
-// ------------------------------------------------------------------------------------------------
-// Block set-up: tables into shared memory, scale
-// ------------------------------------------------------------------------------------------------
-struct __align__(16) SmemTables {
-    uint8_t ta[8192];
-    uint32_t thr[256];
-    float dec[256];
-};
-
-template <bool NEED_TA, bool NEED_SH, bool NEED_DEC, int MODE = HIF8_RND_TA, int SRC = HIF8_F32>
-__device__ __forceinline__ void setup_tables(SmemTables& s, unsigned flags)
-{
-    if (NEED_TA) {
-        // Only binades 2^-24 .. 2^16 differ from their neighbours: those 41 x 16 entries per sign come from the
-        // compile-time table (1.3 KiB of global reads per block); everything below is zero, everything above is
-        // Inf (or NaN in the all-ones exponent), written straight into shared memory.
-        const uint4* g = reinterpret_cast<const uint4*>(g_ta_table.v);
-        uint4* d = reinterpret_cast<uint4*>(s.ta);
-        for (int i = threadIdx.x; i < 512; i += kThreads) {
-            const uint32_t e = i & 255, inf = ((uint32_t)(i >> 8) << 7) | 0x6Fu;
-            uint4 v;
-            if (e < 103) v = make_uint4(0, 0, 0, 0);
-            else if (e <= 143) v = g[i];
-            else if (e < 255) { uint32_t w = inf * 0x01010101u; v = make_uint4(w, w, w, w); }
-            else v = make_uint4(0x80808000u | inf, 0x80808080u, 0x80808080u, 0x80808080u);
-            if (flags) {  // Section 3 options: patch the Inf / NaN entries
-                uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                for (int j = 0; j < 4; j++) {
-                    uint32_t o = 0;
-#pragma unroll
-                    for (int b = 0; b < 4; b++) {
-                        uint32_t c = (w[j] >> (8 * b)) & 0xFFu;
-                        if ((flags & HIF8_FLAG_SATURATE) && (c & 0x7Fu) == 0x6Fu) c &= 0xFEu;
-                        if ((flags & HIF8_FLAG_NAN_TO_ZERO) && c == 0x80u) c = 0;
-                        o |= c << (8 * b);
-                    }
-                    w[j] = o;
-                }
-                v = make_uint4(w[0], w[1], w[2], w[3]);
-            }
-            d[i] = v;
-        }
-    }
-    if (NEED_SH) {
-        const int e = threadIdx.x, E = e - 127;  // kThreads == 256 biased exponents
-        uint32_t ent = 0;
-        if (E < 16 && E >= -22) {
-            constexpr uint32_t N = (SRC == HIF8_F32) ? 14u : 2u;  // threshold bits of the simplified SR
-            const uint32_t sh = 23u - (uint32_t)mant_width(E);
-            ent = sh | ((sh - N) << 8);
-            if (MODE == HIF8_RND_SSR || (MODE == HIF8_RND_HR && (E <= -4 || E >= 4))) ent |= kThrStochastic;
-            else ent |= (1u << (N - 1)) << 16;  // round half away = threshold one half
-        }
-        s.thr[e] = ent;
-    }
-    if (NEED_DEC) s.dec[threadIdx.x] = __uint_as_float(decode_bits_f32(threadIdx.x));
-    __syncthreads();
-}
-
-__device__ __forceinline__ int resolve_scale_exp(const ConvParams& p)
-{
-    if (p.d_amax_bits) return scale_exp_from_amax(*p.d_amax_bits, p.target_exp);
-    if (p.d_scale_exp) return clamp_exp(*p.d_scale_exp);
-    return p.scale_exp;
-}
-
-// amax contribution of a value: |x| for finite x, ignored (NaN) otherwise; fmaxf drops NaN operands
-__device__ __forceinline__ float amax_step(float acc, float x) { return fmaxf(acc, fmaf(x, 0.0f, fabsf(x))); }
-
-__device__ __forceinline__ void block_amax_commit(float acc, uint32_t* accum)
-{
-    __shared__ uint32_t s_part[kThreads / 32];
-    uint32_t v = __reduce_max_sync(0xFFFFFFFFu, __float_as_uint(acc));  // non-negative floats order as integers
-    if ((threadIdx.x & 31) == 0) s_part[threadIdx.x >> 5] = v;
-    __syncthreads();
-    if (threadIdx.x < 32) {
-        v = threadIdx.x < kThreads / 32 ? s_part[threadIdx.x] : 0u;
-        v = __reduce_max_sync(0xFFFFFFFFu, v);
-        if (threadIdx.x == 0 && v) atomicMax(accum, v);
-    }
-}
 
 // ------------------------------------------------------------------------------------------------
 // Encode / fake-quant kernel.  FQ = false: bytes out.  FQ = true: dequantized values in the source format.
@@ -737,23 +414,6 @@ int device_info(int* sms)
     return HIF8_OK;
 }
 
-// launch with programmatic stream serialization (see pdl_* above)
-template <typename... KArgs, typename... Args>
-cudaError_t launch_pdl(void (*kernel)(KArgs...), unsigned grid, cudaStream_t st, Args... args)
-{
-    cudaLaunchConfig_t cfg{};
-    cfg.gridDim = dim3(grid);
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = 0;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
-}
-
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 unsigned grid_for(unsigned long long n_vec, unsigned long long n, int sms)
@@ -846,6 +506,9 @@ int check_common(int dtype, int rnd, unsigned flags)
 constexpr size_t kConvWorkspaceBytes = 256;
 
 }  // namespace
+
+int checked_device(int* sms) { return device_info(sms); }
+
 }  // namespace hif8
 
 using namespace hif8;
@@ -1057,4 +720,79 @@ extern "C" int hif8_amax_scale_encode_static(const void* src, int src_dtype, uin
     return scaled_convert(false, src, dst, src_dtype, n, jit, target_exp, d_scale_exp_in, 0, rnd, flags, seed,
                           d_amax_out, d_scale_exp_out, d_scale_out, scratch, kStaticScratchBytes, !jit,
                           (cudaStream_t)stream);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Delayed scaling: the every-N-iterations amax cadence of Section 5.1 with a ring of past amax values.
+// State (device memory, HIF8_SCALE_STATE_BYTES): bytes 0-255 the record below, bytes 256-511 the scratch of the
+// conversion kernel's amax reduction.
+// ------------------------------------------------------------------------------------------------
+namespace hif8 {
+namespace {
+struct ScaleState {
+    int scale_exp;  // exponent in force
+    int pos;        // next ring slot
+    int filled;     // valid ring entries
+    int hist_len;
+    float amax_last;
+    int pad[3];
+    float ring[HIF8_SCALE_HISTORY_MAX];
+};
+static_assert(sizeof(ScaleState) <= 256, "state record too large");
+
+__global__ void scale_state_init_kernel(ScaleState* st, int hist_len)
+{
+    const int i = threadIdx.x;
+    if (i == 0) { st->scale_exp = 0; st->pos = 0; st->filled = 0; st->hist_len = hist_len; st->amax_last = 0.f; }
+    if (i < HIF8_SCALE_HISTORY_MAX) st->ring[i] = 0.f;
+}
+
+// push the amax just measured, then exponent = rule(max of the ring); one thread
+__global__ void scale_state_update_kernel(ScaleState* st, int target_exp)
+{
+    if (threadIdx.x != 0) return;
+    const int n = st->hist_len;
+    st->ring[st->pos] = st->amax_last;
+    st->pos = (st->pos + 1) % n;
+    if (st->filled < n) st->filled++;
+    uint32_t m = 0;
+    for (int j = 0; j < st->filled; j++) m = max(m, __float_as_uint(st->ring[j]));  // non-negative floats order as integers
+    st->scale_exp = scale_exp_from_amax(m, target_exp);
+}
+}  // namespace
+}  // namespace hif8
+
+extern "C" int hif8_scale_state_init(void* d_state, int hist_len, hif8_stream_t stream)
+{
+    if (!d_state) return HIF8_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(d_state) & 255u) return HIF8_ERR_WORKSPACE;
+    if (hist_len < 1 || hist_len > HIF8_SCALE_HISTORY_MAX) return HIF8_ERR_SHAPE;
+    int sms; int rc = device_info(&sms);
+    if (rc) return rc;
+    scale_state_init_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(reinterpret_cast<ScaleState*>(d_state), hist_len);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
+}
+
+extern "C" int hif8_delayed_scale_encode(const void* src, int src_dtype, uint8_t* dst, size_t n, int rnd, unsigned flags,
+                                         uint64_t seed, void* d_state, int measure, int target_exp, hif8_stream_t stream)
+{
+    int rc = check_common(src_dtype, rnd, flags);
+    if (rc) return rc;
+    if (target_exp < -22 || target_exp > 15) return HIF8_ERR_SCALE_RANGE;
+    if (!d_state || (n && (!src || !dst))) return HIF8_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(d_state) & 255u) return HIF8_ERR_WORKSPACE;
+    ScaleState* state = reinterpret_cast<ScaleState*>(d_state);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!measure)  // conversion alone, exponent read from the state on the device
+        return scaled_convert(false, src, dst, src_dtype, n, false, target_exp, &state->scale_exp, 0, rnd, flags, seed, nullptr,
+                              nullptr, nullptr, nullptr, 0, false, st);
+    // one pass: convert with the exponent in force and reduce amax; then the one-thread update
+    rc = scaled_convert(false, src, dst, src_dtype, n, false, target_exp, &state->scale_exp, 0, rnd, flags, seed,
+                        &state->amax_last, nullptr, nullptr, reinterpret_cast<unsigned char*>(d_state) + 256, kConvWorkspaceBytes,
+                        true, st);
+    if (rc) return rc;
+    scale_state_update_kernel<<<1, 32, 0, st>>>(state, target_exp);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
 }

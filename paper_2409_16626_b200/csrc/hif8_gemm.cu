@@ -239,6 +239,58 @@ __device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int
 }
 
 
+// Epilogue of one 32-column chunk of one accumulator row: descale by f1 * f2 (two exact powers of two) and store as
+// FP32 or BF16 (round to nearest even); rows / columns outside the matrix are skipped.
+__device__ __forceinline__ void store_chunk(const GemmParams& p, int row, int col, const uint32_t (&r)[32], float f1, float f2)
+{
+    if (row >= p.M || col >= p.N) return;
+    const bool full = col + 32 <= p.N;
+    if (p.c_is_f32) {
+        float* out = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + col;
+        if (full) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 4)
+                *reinterpret_cast<float4*>(out + i) =
+                    make_float4(__uint_as_float(r[i]) * f1 * f2, __uint_as_float(r[i + 1]) * f1 * f2,
+                                __uint_as_float(r[i + 2]) * f1 * f2, __uint_as_float(r[i + 3]) * f1 * f2);
+        } else {
+            for (int i = 0; i < 32 && col + i < p.N; i++) out[i] = __uint_as_float(r[i]) * f1 * f2;
+        }
+    } else {
+        unsigned short* out = reinterpret_cast<unsigned short*>(p.C) + (long long)row * p.ldc + col;
+        uint32_t h[32];
+#pragma unroll
+        for (int i = 0; i < 32; i++) {
+            float v = __uint_as_float(r[i]) * f1 * f2;
+            uint32_t u = __float_as_uint(v);
+            h[i] = (v != v) ? 0x7FC0u : ((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);  // round to nearest even
+        }
+        if (full) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 8)
+                *reinterpret_cast<uint4*>(out + i) =
+                    make_uint4(h[i] | (h[i + 1] << 16), h[i + 2] | (h[i + 3] << 16),
+                               h[i + 4] | (h[i + 5] << 16), h[i + 6] | (h[i + 7] << 16));
+        } else {
+            for (int i = 0; i < 32 && col + i < p.N; i++) out[i] = (unsigned short)h[i];
+        }
+    }
+}
+
+// Per-channel weight scales: multiply column col + i of the chunk by 2^-(sa + sw[col + i]).  Lane L fetches the
+// exponent of column col + L once; every lane then walks the 32 columns of its own row.
+__device__ __forceinline__ void apply_channel_scale(const GemmParams& p, int col, int lane, int sa, uint32_t (&r)[32])
+{
+    const int mine = (col + lane < p.N) ? -(sa + __ldg(p.d_sw_channel + col + lane)) : 0;
+#pragma unroll
+    for (int i = 0; i < 32; i++) {
+        const int s = __shfl_sync(0xFFFFFFFFu, mine, i);
+        const int s1 = s / 2, s2 = s - s1;
+        r[i] = __float_as_uint(__uint_as_float(r[i]) * __uint_as_float((uint32_t)(s1 + 127) << 23) *
+                               __uint_as_float((uint32_t)(s2 + 127) << 23));
+    }
+}
+
 template <bool W_IS_NK>
 __global__ void __launch_bounds__(kThreads, 1)
 hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const GemmParams p)
@@ -385,7 +437,8 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         const bool ok = mbar_wait(bar_acc_full, 0, abort_flag, p.status, 5);
         if (ok) {
             tc_fence_after();
-            const int s = -((p.d_sa ? *p.d_sa : 0) + (p.d_sw ? *p.d_sw : 0));
+            const int sa = p.d_sa ? *p.d_sa : 0;
+            const int s = p.d_sw_channel ? 0 : -(sa + (p.d_sw ? *p.d_sw : 0));
             const int s1 = s / 2, s2 = s - s1;  // |s1|, |s2| <= 126: two exact power-of-two factors
             const float f1 = __uint_as_float((uint32_t)(s1 + 127) << 23), f2 = __uint_as_float((uint32_t)(s2 + 127) << 23);
             const int row = m0 + warp * 32 + lane;
@@ -394,40 +447,8 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 uint32_t r[32];
                 tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(warp * 32) << 16) + c, r);
                 tmem_ld_wait();
-                const int col = n0 + c;
-                if (row < p.M && col < p.N) {
-                    const bool full = col + 32 <= p.N;
-                    if (p.c_is_f32) {
-                        float* out = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + col;
-                        if (full) {
-#pragma unroll
-                            for (int i = 0; i < 32; i += 4)
-                                *reinterpret_cast<float4*>(out + i) =
-                                    make_float4(__uint_as_float(r[i]) * f1 * f2, __uint_as_float(r[i + 1]) * f1 * f2,
-                                                __uint_as_float(r[i + 2]) * f1 * f2, __uint_as_float(r[i + 3]) * f1 * f2);
-                        } else {
-                            for (int i = 0; i < 32 && col + i < p.N; i++) out[i] = __uint_as_float(r[i]) * f1 * f2;
-                        }
-                    } else {
-                        unsigned short* out = reinterpret_cast<unsigned short*>(p.C) + (long long)row * p.ldc + col;
-                        uint32_t h[32];
-#pragma unroll
-                        for (int i = 0; i < 32; i++) {
-                            float v = __uint_as_float(r[i]) * f1 * f2;
-                            uint32_t u = __float_as_uint(v);
-                            h[i] = (v != v) ? 0x7FC0u : ((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);  // round to nearest even
-                        }
-                        if (full) {
-#pragma unroll
-                            for (int i = 0; i < 32; i += 8)
-                                *reinterpret_cast<uint4*>(out + i) =
-                                    make_uint4(h[i] | (h[i + 1] << 16), h[i + 2] | (h[i + 3] << 16),
-                                               h[i + 4] | (h[i + 5] << 16), h[i + 6] | (h[i + 7] << 16));
-                        } else {
-                            for (int i = 0; i < 32 && col + i < p.N; i++) out[i] = (unsigned short)h[i];
-                        }
-                    }
-                }
+                if (p.d_sw_channel) apply_channel_scale(p, n0 + c, lane, sa, r);
+                store_chunk(p, row, n0 + c, r, f1, f2);
             }
         }
     }
@@ -576,7 +597,8 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
             }
         }
     } else if (warp < kEpiWarps) {
-        const int sdesc = -((p.d_sa ? *p.d_sa : 0) + (p.d_sw ? *p.d_sw : 0));
+        const int sa = p.d_sa ? *p.d_sa : 0;
+        const int sdesc = p.d_sw_channel ? 0 : -(sa + (p.d_sw ? *p.d_sw : 0));
         const int s1 = sdesc / 2, s2 = sdesc - s1;
         const float f1 = __uint_as_float((uint32_t)(s1 + 127) << 23), f2 = __uint_as_float((uint32_t)(s2 + 127) << 23);
         int local = 0;
@@ -595,6 +617,7 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                 tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(warp * 32) << 16) + acc * 256 + c, r);
                 tmem_ld_wait();
                 const int col = n0 + c;
+                if (p.d_sw_channel) apply_channel_scale(p, col, lane, sa, r);
                 if (p.err_sum) {
                     if (row < p.M && col < p.N) {
                         // exact differences of the FP32 result and the FP32 reference, squared and summed in double
@@ -616,39 +639,7 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                             }
                         }
                     }
-                } else if (row < p.M && col < p.N) {
-                    const bool full = col + 32 <= p.N;
-                    if (p.c_is_f32) {
-                        float* out = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + col;
-                        if (full) {
-#pragma unroll
-                            for (int i = 0; i < 32; i += 4)
-                                *reinterpret_cast<float4*>(out + i) =
-                                    make_float4(__uint_as_float(r[i]) * f1 * f2, __uint_as_float(r[i + 1]) * f1 * f2,
-                                                __uint_as_float(r[i + 2]) * f1 * f2, __uint_as_float(r[i + 3]) * f1 * f2);
-                        } else {
-                            for (int i = 0; i < 32 && col + i < p.N; i++) out[i] = __uint_as_float(r[i]) * f1 * f2;
-                        }
-                    } else {
-                        unsigned short* out = reinterpret_cast<unsigned short*>(p.C) + (long long)row * p.ldc + col;
-                        uint32_t h[32];
-#pragma unroll
-                        for (int i = 0; i < 32; i++) {
-                            float v = __uint_as_float(r[i]) * f1 * f2;
-                            uint32_t u = __float_as_uint(v);
-                            h[i] = (v != v) ? 0x7FC0u : ((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);
-                        }
-                        if (full) {
-#pragma unroll
-                            for (int i = 0; i < 32; i += 8)
-                                *reinterpret_cast<uint4*>(out + i) =
-                                    make_uint4(h[i] | (h[i + 1] << 16), h[i + 2] | (h[i + 3] << 16),
-                                               h[i + 4] | (h[i + 5] << 16), h[i + 6] | (h[i + 7] << 16));
-                        } else {
-                            for (int i = 0; i < 32 && col + i < p.N; i++) out[i] = (unsigned short)h[i];
-                        }
-                    }
-                }
+                } else store_chunk(p, row, col, r, f1, f2);
             }
             tc_fence_before();
             __syncwarp();
@@ -782,9 +773,9 @@ int launch_bf16_pair_gemm(const void* a_bf, const void* w_bf, int w_is_nk, GemmP
 
 using namespace hif8;
 
-extern "C" int hif8_gemm(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int64_t ldw, int w_is_nk, void* C, int64_t ldc,
-                         int c_dtype, int M, int N, int K, const int* d_scale_exp_a, const int* d_scale_exp_w,
-                         void* workspace, size_t workspace_bytes, hif8_stream_t stream)
+static int gemm_entry(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int64_t ldw, int w_is_nk, void* C, int64_t ldc,
+                      int c_dtype, int M, int N, int K, const int* d_scale_exp_a, const int* d_scale_exp_w,
+                      const int* d_scale_exp_w_channel, void* workspace, size_t workspace_bytes, hif8_stream_t stream)
 {
     if (c_dtype != HIF8_BF16 && c_dtype != HIF8_F32) return HIF8_ERR_DTYPE;
     if (M < 0 || N < 0 || K < 0 || (K & 15)) return HIF8_ERR_SHAPE;
@@ -812,7 +803,8 @@ extern "C" int hif8_gemm(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int6
 
     GemmParams p{};
     p.C = C; p.ldc = ldc; p.c_is_f32 = c_dtype == HIF8_F32; p.M = M; p.N = N; p.K = K;
-    p.d_sa = d_scale_exp_a; p.d_sw = d_scale_exp_w; p.status = reinterpret_cast<int*>(workspace);
+    p.d_sa = d_scale_exp_a; p.d_sw = d_scale_exp_w; p.d_sw_channel = d_scale_exp_w_channel;
+    p.status = reinterpret_cast<int*>(workspace);
     p.tiles_m = (M + BM - 1) / BM; p.tiles_n = (N + BN - 1) / BN;
     // both kernels work on 256 x 256 tiles, one per pair of CTAs
     const long long tiles2 = (long long)((M + 2 * BM - 1) / (2 * BM)) * p.tiles_n;
@@ -850,6 +842,24 @@ extern "C" int hif8_gemm(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int6
                                     : cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<false>, map_a, map_w, p);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return (lrc == cudaSuccess && cudaGetLastError() == cudaSuccess) ? HIF8_OK : HIF8_ERR_CUDA;
+}
+
+extern "C" int hif8_gemm(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int64_t ldw, int w_is_nk, void* C, int64_t ldc,
+                         int c_dtype, int M, int N, int K, const int* d_scale_exp_a, const int* d_scale_exp_w,
+                         void* workspace, size_t workspace_bytes, hif8_stream_t stream)
+{
+    return gemm_entry(Aq, lda, Wq, ldw, w_is_nk, C, ldc, c_dtype, M, N, K, d_scale_exp_a, d_scale_exp_w, nullptr, workspace,
+                      workspace_bytes, stream);
+}
+
+extern "C" int hif8_gemm_channel_scaled(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int64_t ldw, int w_is_nk, void* C,
+                                        int64_t ldc, int c_dtype, int M, int N, int K, const int* d_scale_exp_a,
+                                        const int* d_scale_exp_w_channel, void* workspace, size_t workspace_bytes,
+                                        hif8_stream_t stream)
+{
+    if (!d_scale_exp_w_channel && M > 0 && N > 0) return HIF8_ERR_NULL;
+    return gemm_entry(Aq, lda, Wq, ldw, w_is_nk, C, ldc, c_dtype, M, N, K, d_scale_exp_a, nullptr, d_scale_exp_w_channel,
+                      workspace, workspace_bytes, stream);
 }
 
 extern "C" int hif8_gemm_status(const void* workspace, hif8_stream_t stream)
