@@ -212,6 +212,39 @@ def extra_results(H, torch, hbm_peak, peak_kind):
     se = torch.zeros(2, dtype=torch.int32, device="cuda")
     H.hif8_amax_scale_encode(a, H.BF16, Aq, M * K, 14, H.RND_TA, 0, 0, None, None, se[0:1], None, ws, wsb)
     H.hif8_amax_scale_encode(w, H.BF16, Wq, K * N, 14, H.RND_TA, 0, 0, None, None, se[1:2], None, ws, wsb)
+    # per-channel weight scaling of the same weight (one exponent per output column / per row of the [N,K] view) and
+    # the delayed-scaling cadence on the activation; bytes per element: source reads + code byte
+    ch_amax = torch.empty(N, dtype=torch.float32, device="cuda")
+    ch_se = torch.empty(N, dtype=torch.int32, device="cuda")
+    ch_amax2 = torch.empty(2 * N, dtype=torch.float32, device="cuda")
+    ch_se2 = torch.empty(2 * N, dtype=torch.int32, device="cuda")
+    chan = {}
+    ms = timed(lambda r: H.hif8_channel_amax_scale_encode(w, H.BF16, Wq, K, N, 1, 14, H.RND_TA, 0, 0, None, ch_amax, ch_se), 10)
+    chan["columns_[K,N]"] = {"ms": ms, "bytes_per_element": 5, "GBps": 5 * K * N / ms / 1e6, "frac": 5 * K * N / ms / 1e6 / hbm_peak,
+                             "note": "amax kernel (2 B) + encode kernel (2 + 1 B)"}
+    ms = timed(lambda r: H.hif8_channel_amax_scale_encode(w, H.BF16, Wq, N, K, 0, 14, H.RND_TA, 0, 0, None, ch_amax, ch_se), 10)
+    chan["rows_[N,K]"] = {"ms": ms, "bytes_per_element": 3, "GBps": 3 * K * N / ms / 1e6, "frac": 3 * K * N / ms / 1e6 / hbm_peak,
+                          "note": "one kernel, a block per row; the second read of the row hits L1/L2"}
+    ms = timed(lambda r: H.hif8_channel_amax_scale_encode(w, H.BF16, Wq, 2 * N, K // 2, 0, 14, H.RND_TA, 0, 0, None, ch_amax2, ch_se2), 10)
+    chan["rows_[2N,K/2]"] = {"ms": ms, "bytes_per_element": 3, "GBps": 3 * K * N / ms / 1e6, "frac": 3 * K * N / ms / 1e6 / hbm_peak,
+                             "note": "rows of 4096: two rows per block"}
+    ms = timed(lambda r: H.hif8_channel_amax_scale_encode(w, H.BF16, Wq, N // 2, 2 * K, 0, 14, H.RND_TA, 0, 0, None, ch_amax2, ch_se2), 10)
+    chan["rows_[N/2,2K]"] = {"ms": ms, "bytes_per_element": 3, "GBps": 3 * K * N / ms / 1e6, "frac": 3 * K * N / ms / 1e6 / hbm_peak,
+                             "note": "rows of 16384: held in registers, read once"}
+    ms = timed(lambda r: H.hif8_channel_amax_scale_encode(w, H.BF16, Wq, K, N, 1, 14, H.RND_TA, 0, 0, ch_se, None, None), 10)
+    chan["columns_given_exponents"] = {"ms": ms, "bytes_per_element": 3, "GBps": 3 * K * N / ms / 1e6,
+                                       "frac": 3 * K * N / ms / 1e6 / hbm_peak}
+    out["channel_scaled_encode_bf16_8192x28672"] = {"calls": chan, "peak": hbm_peak, "peak_kind": f"of {peak_kind}"}
+    state = torch.empty(H.SCALE_STATE_BYTES, dtype=torch.uint8, device="cuda")
+    H.hif8_scale_state_init(state, 4)
+    dl = {}
+    for name, measure in (("measuring_iteration", 1), ("plain_iteration", 0)):
+        ms = timed(lambda r: H.hif8_delayed_scale_encode(a, H.BF16, Aq, M * K, H.RND_TA, 0, 0, state, measure, 14), 20)
+        dl[name] = {"ms": ms, "GBps": 3 * M * K / ms / 1e6, "frac": 3 * M * K / ms / 1e6 / hbm_peak}
+    out["delayed_scale_encode_bf16_8192x8192"] = {"bytes_per_element": 3, "calls": dl, "peak": hbm_peak,
+                                                  "peak_kind": f"of {peak_kind}"}
+    H.hif8_amax_scale_encode(a, H.BF16, Aq, M * K, 14, H.RND_TA, 0, 0, None, None, se[0:1], None, ws, wsb)
+    H.hif8_amax_scale_encode(w, H.BF16, Wq, K * N, 14, H.RND_TA, 0, 0, None, None, se[1:2], None, ws, wsb)
     del a, w
     C = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
     gws_b = H.hif8_workspace_bytes(H.WS_GEMM, M * K + K * N)
@@ -225,7 +258,12 @@ def extra_results(H, torch, hbm_peak, peak_kind):
     st1 = H.hif8_gemm_status(gws)
     ms_f = timed(lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, C, N, H.BF16, M, N, K, se[0:1], se[1:2], gws, 256), 3)
     st2 = H.hif8_gemm_status(gws)
+    ch_se.fill_(int(se[1]))
+    ms_c = timed(lambda r: H.hif8_gemm_channel_scaled(Aq, K, Wq, N, 0, C, N, H.BF16, M, N, K, se[0:1], ch_se, gws, gws_b), 10)
+    st3 = H.hif8_gemm_status(gws)
     out["gemm_8192x28672x8192"] = {
+        "decode_once_channel_scaled": {"ms": ms_c, "TFLOPs": flops / ms_c / 1e9, "frac": flops / ms_c / 1e9 / tf_peak,
+                                       "device_status": st3, "note": "one weight exponent per output column"},
         "decode_once": {"ms": ms, "TFLOPs": flops / ms / 1e9, "frac": flops / ms / 1e9 / tf_peak, "device_status": st1,
                         "note": "whole call: decode of both operands to BF16 workspace + tcgen05 kernel"},
         "fused": {"ms": ms_f, "TFLOPs": flops / ms_f / 1e9, "frac": flops / ms_f / 1e9 / tf_peak, "device_status": st2,

@@ -53,13 +53,24 @@ def run_channel(x, dtype, axis, rnd=H.RND_TA, flags=0, seed=0, target=14, given=
 
 @pytest.mark.parametrize("dtype", [H.F32, H.BF16, H.F16])
 @pytest.mark.parametrize("axis", [0, 1])
-@pytest.mark.parametrize("shape", [(300, 520), (64, 4096), (1031, 264), (9, 8), (257, 40)])
+@pytest.mark.parametrize("shape", [(300, 520), (64, 4096), (1031, 264), (9, 8), (257, 40), (12, 20480)])
 def test_channel_encode_ta_matches_oracle(shape, axis, dtype):
     x = weight(*shape, seed=shape[0] + axis, dtype=dtype)
     q, amax, se = run_channel(x, dtype, axis)
     amax_o, se_o = O.channel_amax_scale(x, dtype, axis, 14)
     assert np.array_equal(amax, amax_o) and np.array_equal(se, se_o)
     assert np.array_equal(q, O.channel_encode(x, dtype, axis, se_o, quick=True))
+
+
+@pytest.mark.parametrize("dtype,shape", [(H.F32, (2400, 8192)), (H.BF16, (4096, 7168)), (H.BF16, (1216, 16384))])
+@pytest.mark.parametrize("axis", [0, 1])
+def test_channel_encode_large(axis, dtype, shape):
+    # large enough for the widest column strips (8 and 4 warps across) and for rows of exactly one register tile
+    x = weight(*shape, seed=21, dtype=dtype)
+    q, amax, se = run_channel(x, dtype, axis, rnd=H.RND_HR)
+    amax_o, se_o = O.channel_amax_scale(x, dtype, axis, 14)
+    assert np.array_equal(amax, amax_o) and np.array_equal(se, se_o)
+    assert np.array_equal(q, O.channel_encode(x, dtype, axis, se_o, rnd=H.RND_HR, quick=True))
 
 
 @pytest.mark.parametrize("mode", MODES)
