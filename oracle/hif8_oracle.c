@@ -643,3 +643,46 @@ void hif8o_delayed_scale_run(const float* amax, int T, int interval, int hist_le
         }
     }
 }
+
+/* ------------------------------------------------------------------------- *
+ * Backward-pass operand forms (Section 3: TA or hybrid rounding in the backward
+ * pass; Section 4.1: activation gradients are GEMM inputs too).  For Y = X W the
+ * backward GEMMs are dX = dY W^T and dW = X^T dY: the same "MatMul & Restore"
+ * with an operand read through its transpose, and dW may be summed into an
+ * existing buffer.  Nothing new is computed; only the indexing differs.
+ * ------------------------------------------------------------------------- */
+
+/* dst[c, r] = To_HiF8( src[r, c] * 2^scale_exp ): the converted tensor, stored transposed ([cols, rows]).  The
+ * stochastic word of an element is the one of its flat index in the SOURCE, r * cols + c. */
+void hif8o_encode_transpose(const void* src, int dtype, uint8_t* dst, long long rows, long long cols, int scale_exp,
+                            int rnd, unsigned flags, uint64_t seed, int quick)
+{
+#pragma omp parallel for schedule(static)
+    for (long long r = 0; r < rows; r++)
+        for (long long c = 0; c < cols; c++) {
+            long long idx = r * cols + c;
+            uint32_t raw; double x = src_to_double(src, (size_t)idx, dtype, &raw);
+            dst[c * rows + r] = (uint8_t)encode_value(x, raw, dtype, scale_exp, rnd, flags, seed, (uint64_t)idx, quick);
+        }
+}
+
+/* C*[m,n] = 2^-(sa + sw_n) * sum_k dec(A(m,k)) dec(W(k,n)) with A stored [M,K] or (a_is_km) [K,M], W stored [K,N] or
+ * (w_is_nk) [N,K]; sw_n = sw_channel[n] if sw_channel is given, else sw.  S likewise with |.|. */
+void hif8o_gemm_entries_ex(const uint8_t* Aq, long long lda, int a_is_km, const uint8_t* Wq, long long ldw, int w_is_nk,
+                           int K, int sa, int sw, const int* sw_channel, const long long* rows, const long long* cols,
+                           size_t count, double* Cstar, double* S)
+{
+#pragma omp parallel for schedule(dynamic, 64)
+    for (long long t = 0; t < (long long)count; t++) {
+        long long m = rows[t], n = cols[t];
+        double acc = 0.0, sab = 0.0;
+        for (long long k = 0; k < K; k++) {
+            double a = hif8o_value(a_is_km ? Aq[k * lda + m] : Aq[m * lda + k]);
+            double w = hif8o_value(w_is_nk ? Wq[n * ldw + k] : Wq[k * ldw + n]);
+            acc += a * w; sab += fabs(a * w);
+        }
+        int s = sa + (sw_channel ? sw_channel[n] : sw);
+        Cstar[t] = ldexp(acc, -s);
+        S[t] = ldexp(sab, -s);
+    }
+}

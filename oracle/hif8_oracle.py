@@ -35,6 +35,8 @@ _lib.hif8o_channel_amax_scale.argtypes = [_vp, _i, _ll, _ll, _i, _i, _vp, _vp]
 _lib.hif8o_channel_encode.argtypes = [_vp, _i, _vp, _ll, _ll, _i, _vp, _i, _u, _u64, _i]
 _lib.hif8o_gemm_entries_channel.argtypes = [_vp, _ll, _vp, _ll, _i, _i, _i, _vp, _vp, _vp, _sz, _vp, _vp]
 _lib.hif8o_delayed_scale_run.argtypes = [_vp, _i, _i, _i, _i, _vp]
+_lib.hif8o_encode_transpose.argtypes = [_vp, _i, _vp, _ll, _ll, _i, _i, _u, _u64, _i]
+_lib.hif8o_gemm_entries_ex.argtypes = [_vp, _ll, _i, _vp, _ll, _i, _i, _i, _i, _vp, _vp, _vp, _sz, _vp, _vp]
 _lib.hif8o_gemm_full.argtypes = [_vp, _ll, _vp, _ll, _i, _i, _i, _i, _i, _i, _vp, _vp]
 
 
@@ -210,3 +212,28 @@ def delayed_scale_run(amax, interval, hist_len, target_exp=14):
     used = np.empty(amax.size, dtype=np.int32)
     _lib.hif8o_delayed_scale_run(_ptr(amax), amax.size, interval, hist_len, target_exp, _ptr(used))
     return used
+
+
+def encode_transpose(src, dtype, scale_exp=0, rnd=TA, flags=0, seed=0, quick=False):
+    """Codes of src [rows, cols], stored transposed: uint8 [cols, rows]."""
+    a = _src(src, dtype)
+    rows, cols = a.shape
+    out = np.empty((cols, rows), dtype=np.uint8)
+    _lib.hif8o_encode_transpose(_ptr(a), dtype, _ptr(out), rows, cols, scale_exp, rnd, flags, seed, int(quick))
+    return out
+
+
+def gemm_entries_ex(Aq, a_is_km, Wq, w_is_nk, sa, sw, rows, cols):
+    """(C*, S) for listed entries; Aq [M,K] or (a_is_km) [K,M]; Wq [K,N] or (w_is_nk) [N,K]; sw an int or an int32 [N]."""
+    Aq = np.ascontiguousarray(Aq, dtype=np.uint8)
+    Wq = np.ascontiguousarray(Wq, dtype=np.uint8)
+    K = Aq.shape[0] if a_is_km else Aq.shape[1]
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    cols = np.ascontiguousarray(cols, dtype=np.int64)
+    cs = np.empty(rows.size, dtype=np.float64)
+    s = np.empty(rows.size, dtype=np.float64)
+    ch = None if np.isscalar(sw) else np.ascontiguousarray(sw, dtype=np.int32)
+    _lib.hif8o_gemm_entries_ex(_ptr(Aq), Aq.shape[1], int(a_is_km), _ptr(Wq), Wq.shape[1], int(w_is_nk), K, sa,
+                               int(sw) if ch is None else 0, None if ch is None else _ptr(ch), _ptr(rows), _ptr(cols),
+                               rows.size, _ptr(cs), _ptr(s))
+    return cs, s

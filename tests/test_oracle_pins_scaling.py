@@ -125,3 +125,40 @@ def test_delayed_scale_with_history_one_matches_the_per_tensor_rule():
     assert used[0] == 0
     for t in range(1, 12):
         assert used[t] == O.amax_scale(tensors[t - 1], O.F32, 12)[1]
+
+
+# ----------------------------------------------------------------------------- backward-pass operand forms
+@pytest.mark.parametrize("mode", [O.TA, O.HR, O.SR])
+def test_encode_transpose_is_the_flat_encoder_followed_by_a_transpose(mode):
+    x = W.f32_to_bf16_bits(W.normal_f32(33 * 20, 6).reshape(33, 20) * np.float32(300.0))
+    q = O.encode(x.ravel(), O.BF16, -2, mode, seed=4).reshape(33, 20)   # pinned flat encoder, source-order words
+    qt = O.encode_transpose(x, O.BF16, -2, mode, seed=4)
+    assert qt.shape == (20, 33) and np.array_equal(qt, q.T)
+    if mode != O.SR:  # deterministic modes: transposing twice is the identity on the codes' values
+        back = O.decode(qt, O.BF16, -2)
+        assert np.array_equal(O.encode_transpose(back, O.BF16, -2, O.TA), q)
+
+
+def test_gemm_ex_equals_the_plain_gemm_on_explicitly_transposed_operands():
+    M, N, K = 7, 10, 32
+    A = W.random_codes(M * K, 11).reshape(M, K)
+    Wk = W.random_codes(K * N, 12).reshape(K, N)
+    for t in (A, Wk):
+        t[(t == 0x80) | ((t & 0x7F) == 0x6F)] = 0x21
+    rows, cols = np.divmod(np.arange(M * N), N)
+    ref = O.gemm_entries(A, Wk, 0, 3, -2, rows, cols)  # pinned against numpy in test_oracle_pins.py
+    for a_km in (0, 1):
+        for w_nk in (0, 1):
+            got = O.gemm_entries_ex(np.ascontiguousarray(A.T) if a_km else A, a_km,
+                                    np.ascontiguousarray(Wk.T) if w_nk else Wk, w_nk, 3, -2, rows, cols)
+            assert np.array_equal(got[0], ref[0]) and np.array_equal(got[1], ref[1])
+    sw = np.arange(N, dtype=np.int32) - 4
+    ch = O.gemm_entries_ex(np.ascontiguousarray(A.T), 1, Wk, 0, 3, sw, rows, cols)
+    ref_ch = O.gemm_entries_channel(A, Wk, 0, 3, sw, rows, cols)
+    assert np.array_equal(ch[0], ref_ch[0]) and np.array_equal(ch[1], ref_ch[1])
+    # a non-square case where a wrong leading dimension or swapped index cannot cancel: one-hot operands
+    A1 = np.zeros((M, K), dtype=np.uint8); A1[2, 5] = 0x08          # value 1 at (m=2, k=5)
+    W1 = np.zeros((K, N), dtype=np.uint8); W1[5, 7] = 0x10          # value 2 at (k=5, n=7)
+    c, _ = O.gemm_entries_ex(np.ascontiguousarray(A1.T), 1, np.ascontiguousarray(W1.T), 1, 0, 0, rows, cols)
+    expect = np.zeros(M * N); expect[2 * N + 7] = 2.0
+    assert np.array_equal(c, expect)
