@@ -228,6 +228,36 @@ int hif8_gemm_channel_scaled(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, 
                              hif8_stream_t stream);
 
 /*
+ * The general form of the HiF8 GEMM, covering the backward pass of Y = X W (Section 3: the activation gradient is
+ * converted with TA or hybrid rounding; Section 4.1: activation, weight and activation gradient are the GEMM inputs):
+ *   dgrad  dX[M,K'] = dY[M,N'] W^T :  Aq = dYq [M,N'],           Wq = the forward weight bytes [K',N'], w_is_nk = 1
+ *   wgrad  dW[K',N'] = X^T dY      :  Aq = Xq [M',K'], a_is_km = 1 (A is read as [K,M] = [M',K']), Wq = dYq [M',N'], w_is_nk = 0
+ * so neither backward GEMM needs a transposed copy of a byte tensor.
+ *   C[m,n] (+)= 2^-(sa + sw_n) * sum_k value(A(m,k)) * value(W(k,n))
+ *   a_is_km = 0: Aq is [M,K] row-major (lda >= K);  a_is_km = 1: Aq is [K,M] row-major (lda >= M).
+ *   w_is_nk as in hif8_gemm.  sw_n = d_scale_exp_w_channel[n] if that pointer is given, else *d_scale_exp_w (or 0).
+ *   accumulate != 0: the product is added to the existing contents of C (FP32 C: one rounding per element per call;
+ *   BF16 C: sum formed in FP32, then rounded to nearest even) -- gradient accumulation over micro-batches.
+ * Alignment, K, workspace and status conventions as in hif8_gemm (the decode-once path needs contiguous operands).
+ */
+int hif8_gemm_ex(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t* Wq, int64_t ldw, int w_is_nk, void* C,
+                 int64_t ldc, int c_dtype, int M, int N, int K, const int* d_scale_exp_a, const int* d_scale_exp_w,
+                 const int* d_scale_exp_w_channel, int accumulate, void* workspace, size_t workspace_bytes,
+                 hif8_stream_t stream);
+
+/*
+ * Conversion with transposed store: dst[c, r] = To_HiF8_<rnd>( src[r, c] * 2^e ), src [rows, cols] row-major of
+ * `src_dtype`, dst [cols, rows] bytes.  For frameworks that keep a second, transposed byte copy of a GEMM operand
+ * (the backward GEMMs contract over the other dimension); hif8_gemm_ex does not need it.
+ *   e = *d_scale_exp if that device pointer is given (delayed scaling), else scale_exp.
+ *   HIF8_RND_SR draws the word of the SOURCE flat index r * cols + c, so the codes equal those of hif8_encode, moved.
+ * The fast path wants 16-byte aligned pointers, cols a multiple of the 16-byte vector (4 FP32 / 8 16-bit elements) and
+ * rows a multiple of 16; anything else takes an element-wise path with identical results.
+ */
+int hif8_encode_transpose(const void* src, int src_dtype, uint8_t* dst, int64_t rows, int64_t cols, int scale_exp,
+                          const int* d_scale_exp, int rnd, unsigned flags, uint64_t seed, hif8_stream_t stream);
+
+/*
  * Host-side query of the status word of a finished hif8_gemm: copies it from `workspace`, SYNCHRONISES `stream`,
  * and returns HIF8_OK or HIF8_ERR_DEVICE_TIMEOUT (the output tile of the CTA that gave up is then undefined).
  * The only entry point that blocks the host.

@@ -20,7 +20,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libhif8.so")
 EXPORTS = ["hif8_encode", "hif8_decode", "hif8_amax", "hif8_amax_scale_encode", "hif8_fake_quant", "hif8_gemm", "hif8_gemm_status", "hif8_pts_search", "hif8_pts_workspace_bytes",
            "hif8_pts_status", "hif8_selftest_wait_timeout", "hif8_channel_amax_scale_encode", "hif8_gemm_channel_scaled",
-           "hif8_scale_state_init", "hif8_delayed_scale_encode",
+           "hif8_scale_state_init", "hif8_delayed_scale_encode", "hif8_gemm_ex", "hif8_encode_transpose",
            "hif8_amax_scale_encode_static", "hif8_workspace_bytes", "hif8_status_string", "hif8_launch_count"]
 
 if not os.path.exists(LIB_PATH):
@@ -55,6 +55,10 @@ lib.hif8_scale_state_init.argtypes = [_vp, _i, _vp]
 lib.hif8_scale_state_init.restype = _i
 lib.hif8_delayed_scale_encode.argtypes = [_vp, _i, _vp, _sz, _i, _u, _u64, _vp, _i, _i, _vp]
 lib.hif8_delayed_scale_encode.restype = _i
+lib.hif8_gemm_ex.argtypes = [_vp, _i64, _i, _vp, _i64, _i, _vp, _i64, _i, _i, _i, _i, _vp, _vp, _vp, _i, _vp, _sz, _vp]
+lib.hif8_gemm_ex.restype = _i
+lib.hif8_encode_transpose.argtypes = [_vp, _i, _vp, _i64, _i64, _i, _vp, _i, _u, _u64, _vp]
+lib.hif8_encode_transpose.restype = _i
 lib.hif8_workspace_bytes.argtypes = [_i, _sz]
 lib.hif8_workspace_bytes.restype = _sz
 lib.hif8_status_string.argtypes = [_i]
@@ -191,3 +195,16 @@ def hif8_delayed_scale_encode(src, src_dtype, dst, n, rnd, flags, seed, d_state,
                               check=True):
     return _check(lib.hif8_delayed_scale_encode(_ptr(src), src_dtype, _ptr(dst), n, rnd, flags, seed, _ptr(d_state),
                                                 int(measure), target_exp, _stream(stream)), check)
+
+
+def hif8_gemm_ex(Aq, lda, a_is_km, Wq, ldw, w_is_nk, Cmat, ldc, c_dtype, M, N, K, d_scale_exp_a=None, d_scale_exp_w=None,
+                 d_scale_exp_w_channel=None, accumulate=0, workspace=None, workspace_bytes=0, stream=None, check=True):
+    return _check(lib.hif8_gemm_ex(_ptr(Aq), lda, int(a_is_km), _ptr(Wq), ldw, int(w_is_nk), _ptr(Cmat), ldc, c_dtype, M, N, K,
+                                   _ptr(d_scale_exp_a), _ptr(d_scale_exp_w), _ptr(d_scale_exp_w_channel), int(accumulate),
+                                   _ptr(workspace), workspace_bytes, _stream(stream)), check)
+
+
+def hif8_encode_transpose(src, src_dtype, dst, rows, cols, scale_exp=0, d_scale_exp=None, rnd=RND_TA, flags=0, seed=0,
+                          stream=None, check=True):
+    return _check(lib.hif8_encode_transpose(_ptr(src), src_dtype, _ptr(dst), rows, cols, scale_exp, _ptr(d_scale_exp), rnd,
+                                            flags, seed, _stream(stream)), check)

@@ -249,19 +249,38 @@ __device__ __forceinline__ void store_chunk(const GemmParams& p, int row, int co
         float* out = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + col;
         if (full) {
 #pragma unroll
-            for (int i = 0; i < 32; i += 4)
-                *reinterpret_cast<float4*>(out + i) =
-                    make_float4(__uint_as_float(r[i]) * f1 * f2, __uint_as_float(r[i + 1]) * f1 * f2,
-                                __uint_as_float(r[i + 2]) * f1 * f2, __uint_as_float(r[i + 3]) * f1 * f2);
+            for (int i = 0; i < 32; i += 4) {
+                float4 o = make_float4(__uint_as_float(r[i]) * f1 * f2, __uint_as_float(r[i + 1]) * f1 * f2,
+                                       __uint_as_float(r[i + 2]) * f1 * f2, __uint_as_float(r[i + 3]) * f1 * f2);
+                if (p.accumulate) {
+                    const float4 c = *reinterpret_cast<const float4*>(out + i);
+                    o.x += c.x; o.y += c.y; o.z += c.z; o.w += c.w;
+                }
+                *reinterpret_cast<float4*>(out + i) = o;
+            }
         } else {
-            for (int i = 0; i < 32 && col + i < p.N; i++) out[i] = __uint_as_float(r[i]) * f1 * f2;
+            for (int i = 0; i < 32 && col + i < p.N; i++) out[i] = __uint_as_float(r[i]) * f1 * f2 + (p.accumulate ? out[i] : 0.f);
         }
     } else {
         unsigned short* out = reinterpret_cast<unsigned short*>(p.C) + (long long)row * p.ldc + col;
         uint32_t h[32];
+        if (p.accumulate) {  // previous contents of C, widened exactly
+            if (full) {
+#pragma unroll
+                for (int i = 0; i < 32; i += 8) {
+                    const uint4 c = *reinterpret_cast<const uint4*>(out + i);
+                    h[i] = c.x << 16; h[i + 1] = c.x & 0xFFFF0000u; h[i + 2] = c.y << 16; h[i + 3] = c.y & 0xFFFF0000u;
+                    h[i + 4] = c.z << 16; h[i + 5] = c.z & 0xFFFF0000u; h[i + 6] = c.w << 16; h[i + 7] = c.w & 0xFFFF0000u;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < 32; i++) h[i] = (col + i < p.N) ? (uint32_t)out[i] << 16 : 0u;
+            }
+        }
 #pragma unroll
         for (int i = 0; i < 32; i++) {
             float v = __uint_as_float(r[i]) * f1 * f2;
+            if (p.accumulate) v += __uint_as_float(h[i]);
             uint32_t u = __float_as_uint(v);
             h[i] = (v != v) ? 0x7FC0u : ((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);  // round to nearest even
         }
@@ -291,7 +310,30 @@ __device__ __forceinline__ void apply_channel_scale(const GemmParams& p, int col
     }
 }
 
-template <bool W_IS_NK>
+// Fused kernel, decode warps: one 128 x 64 tile of HiF8 bytes -> BF16 in the 128-byte-swizzled operand layout.
+// K-major source tile [128 rows][64 k]: chunk j (8 codes) of row r -> atom r/8, row r%8, chunk j ^ (r%8).
+__device__ __forceinline__ void decode_tile_k_major(const unsigned char* src8, unsigned char* dst, int dt, const uint32_t* lut)
+{
+#pragma unroll
+    for (int it = 0; it < (BM * BK / 8) / kDecodeThreads; it++) {
+        const int q = it * kDecodeThreads + dt, r = q >> 3, j = q & 7;
+        const uint2 v = *reinterpret_cast<const uint2*>(src8 + r * BK + j * 8);
+        *reinterpret_cast<uint4*>(dst + (r >> 3) * 1024 + (r & 7) * 128 + ((j ^ (r & 7)) << 4)) = decode8(v, lut);
+    }
+}
+// MN-major source tile [64 k][128 mn]: chunk (k, mn/8) -> atom (mn/64) * 8 + k/8, row k%8, chunk (mn/8)%8 ^ (k%8).
+__device__ __forceinline__ void decode_tile_mn_major(const unsigned char* src8, unsigned char* dst, int dt, const uint32_t* lut)
+{
+#pragma unroll
+    for (int it = 0; it < (BM * BK / 8) / kDecodeThreads; it++) {
+        const int q = it * kDecodeThreads + dt, k = q >> 4, jn = q & 15;
+        const uint2 v = *reinterpret_cast<const uint2*>(src8 + k * BM + jn * 8);
+        const int atom = (jn >> 3) * 8 + (k >> 3);
+        *reinterpret_cast<uint4*>(dst + atom * 1024 + (k & 7) * 128 + (((jn & 7) ^ (k & 7)) << 4)) = decode8(v, lut);
+    }
+}
+
+template <bool A_IS_KM, bool W_IS_NK>
 __global__ void __launch_bounds__(kThreads, 1)
 hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const GemmParams p)
 {
@@ -349,7 +391,8 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 if (*abort_flag) break;
                 const uint32_t dst_a = base + SmemLayout::u8 + s * (kA8Bytes + kB8Bytes), dst_b = dst_a + kA8Bytes;
                 mbar_arrive_expect_tx(bar_u8_full(s), kA8Bytes + kB8Bytes);
-                tma_load_2d(dst_a, &map_a, kb * BK, m0, bar_u8_full(s));
+                if (A_IS_KM) tma_load_2d(dst_a, &map_a, m0, kb * BK, bar_u8_full(s));
+                else tma_load_2d(dst_a, &map_a, kb * BK, m0, bar_u8_full(s));
                 if (W_IS_NK) tma_load_2d(dst_b, &map_w, kb * BK, nh, bar_u8_full(s));
                 else tma_load_2d(dst_b, &map_w, nh, kb * BK, bar_u8_full(s));
                 issued = kb + 1;
@@ -367,7 +410,7 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         // ------------------------------------------------------------------ MMA issuer (leader CTA only)
         if (lane == 0 && leader) {
             // instruction descriptor: FP32 accumulator, BF16 A and B, A K-major, B K- or MN-major, N = 256, M = 256 (pair)
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((W_IS_NK ? 0u : 1u) << 16) |
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_IS_KM ? 1u : 0u) << 15) | ((W_IS_NK ? 0u : 1u) << 16) |
                                    ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
             bool ok = true;
             for (int kb = 0; kb < num_kb && ok; kb++) {
@@ -379,7 +422,8 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 #pragma unroll
                 for (int kk = 0; kk < BK / 16; kk++) {
                     // K-major: 16 k = 32 bytes inside the 128-byte row; MN-major: 16 k = two 1024-byte atoms
-                    const uint64_t da = make_smem_desc(a_addr + kk * 32, 16, 1024);
+                    const uint64_t da = A_IS_KM ? make_smem_desc(a_addr + kk * 2048, 8192, 1024)
+                                                : make_smem_desc(a_addr + kk * 32, 16, 1024);
                     const uint64_t db = W_IS_NK ? make_smem_desc(b_addr + kk * 32, 16, 1024)
                                                 : make_smem_desc(b_addr + kk * 2048, 8192, 1024);
                     tc_mma_bf16_pair(tmem_base, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
@@ -401,30 +445,8 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             const unsigned char* b8 = a8 + kA8Bytes;
             unsigned char* abf = sm + SmemLayout::bf + sb * (kABfBytes + kBBfBytes);
             unsigned char* bbf = abf + kABfBytes;
-            // A: 128 rows x 8 chunks of 8 codes; chunk j of row r -> atom r/8, row r%8, chunk j ^ (r%8)
-#pragma unroll
-            for (int it = 0; it < (BM * BK / 8) / kDecodeThreads; it++) {
-                const int q = it * kDecodeThreads + dt, r = q >> 3, j = q & 7;
-                const uint2 v = *reinterpret_cast<const uint2*>(a8 + r * BK + j * 8);
-                *reinterpret_cast<uint4*>(abf + (r >> 3) * 1024 + (r & 7) * 128 + ((j ^ (r & 7)) << 4)) = decode8(v, lut);
-            }
-            if (W_IS_NK) {
-#pragma unroll
-                for (int it = 0; it < ((BN / 2) * BK / 8) / kDecodeThreads; it++) {
-                    const int q = it * kDecodeThreads + dt, r = q >> 3, j = q & 7;
-                    const uint2 v = *reinterpret_cast<const uint2*>(b8 + r * BK + j * 8);
-                    *reinterpret_cast<uint4*>(bbf + (r >> 3) * 1024 + (r & 7) * 128 + ((j ^ (r & 7)) << 4)) = decode8(v, lut);
-                }
-            } else {
-                // W tile is [64 k][128 n]: chunk (k, n/8) -> atom (n/64) * 8 + k/8, row k%8, chunk (n/8)%8 ^ (k%8)
-#pragma unroll
-                for (int it = 0; it < ((BN / 2) * BK / 8) / kDecodeThreads; it++) {
-                    const int q = it * kDecodeThreads + dt, k = q >> 4, jn = q & 15;
-                    const uint2 v = *reinterpret_cast<const uint2*>(b8 + k * (BN / 2) + jn * 8);
-                    const int atom = (jn >> 3) * 8 + (k >> 3);
-                    *reinterpret_cast<uint4*>(bbf + atom * 1024 + (k & 7) * 128 + (((jn & 7) ^ (k & 7)) << 4)) = decode8(v, lut);
-                }
-            }
+            if (A_IS_KM) decode_tile_mn_major(a8, abf, dt, lut); else decode_tile_k_major(a8, abf, dt, lut);
+            if (W_IS_NK) decode_tile_k_major(b8, bbf, dt, lut); else decode_tile_mn_major(b8, bbf, dt, lut);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // make the stores visible to the tensor core
             __syncwarp();
             if (lane == 0) {
@@ -492,7 +514,7 @@ struct SmemLayout2 {
 };
 constexpr uint32_t kSmemBytes2 = SmemLayout2::total + 1024;
 
-template <bool W_IS_NK>
+template <bool A_IS_KM, bool W_IS_NK>
 __global__ void __launch_bounds__(kThreadsP, 1)
 bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const GemmParams p)
 {
@@ -546,7 +568,10 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                     const uint32_t dst_a = base + s * kStageBytes2, dst_b = dst_a + kABfBytes;
                     const uint32_t full = map_to_cta(bar_full(s), 0);
                     if (leader) mbar_arrive_expect_tx(bar_full(s), 2 * kStageBytes2);  // bytes of both CTAs
-                    tma_load_2d_pair(dst_a, &map_a, kb * BK, m0, full);
+                    if (A_IS_KM) {
+#pragma unroll
+                        for (int c = 0; c < BM / 64; c++) tma_load_2d_pair(dst_a + c * 8192, &map_a, m0 + c * 64, kb * BK, full);
+                    } else tma_load_2d_pair(dst_a, &map_a, kb * BK, m0, full);
                     if (W_IS_NK) tma_load_2d_pair(dst_b, &map_w, kb * BK, n0, full);
                     else {
 #pragma unroll
@@ -567,7 +592,7 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     } else if (warp == kMmaWarp) {
         if (lane == 0 && leader) {
             // M = 256 over the pair, N = 256
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((W_IS_NK ? 0u : 1u) << 16) |
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_IS_KM ? 1u : 0u) << 15) | ((W_IS_NK ? 0u : 1u) << 16) |
                                    ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
             long long it = 0;
             int local = 0;
@@ -586,7 +611,8 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                     const uint32_t a_addr = base + s * kStageBytes2, b_addr = a_addr + kABfBytes;
 #pragma unroll
                     for (int kk = 0; kk < BK / 16; kk++) {
-                        const uint64_t da = make_smem_desc(a_addr + kk * 32, 16, 1024);
+                        const uint64_t da = A_IS_KM ? make_smem_desc(a_addr + kk * 2048, 8192, 1024)
+                                                    : make_smem_desc(a_addr + kk * 32, 16, 1024);
                         const uint64_t db = W_IS_NK ? make_smem_desc(b_addr + kk * 32, 16, 1024)
                                                     : make_smem_desc(b_addr + kk * 2048, 8192, 1024);
                         tc_mma_bf16_pair(d_tmem, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
@@ -721,13 +747,14 @@ bool gemm_kernels_ready(int dev, int* sm_count_out)
     static cudaError_t attr_rc = cudaSuccess;
     static int sm_count = 0;
     std::call_once(attr_once, [dev] {
-        attr_rc = cudaFuncSetAttribute(hif8_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        if (attr_rc == cudaSuccess)
-            attr_rc = cudaFuncSetAttribute(hif8_gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        if (attr_rc == cudaSuccess)
-            attr_rc = cudaFuncSetAttribute(bf16_gemm_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
-        if (attr_rc == cudaSuccess)
-            attr_rc = cudaFuncSetAttribute(bf16_gemm_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
+        const void* fused[4] = {(const void*)hif8_gemm_kernel<false, false>, (const void*)hif8_gemm_kernel<false, true>,
+                                (const void*)hif8_gemm_kernel<true, false>, (const void*)hif8_gemm_kernel<true, true>};
+        const void* pair[4] = {(const void*)bf16_gemm_pair_kernel<false, false>, (const void*)bf16_gemm_pair_kernel<false, true>,
+                               (const void*)bf16_gemm_pair_kernel<true, false>, (const void*)bf16_gemm_pair_kernel<true, true>};
+        for (int i = 0; i < 4 && attr_rc == cudaSuccess; i++) {
+            attr_rc = cudaFuncSetAttribute(fused[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+            if (attr_rc == cudaSuccess) attr_rc = cudaFuncSetAttribute(pair[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
+        }
         if (attr_rc == cudaSuccess) attr_rc = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
     });
     *sm_count_out = sm_count;
@@ -738,7 +765,7 @@ constexpr size_t kGemmWorkspaceBytes = 256;
 
 }  // namespace
 
-int launch_bf16_pair_gemm(const void* a_bf, const void* w_bf, int w_is_nk, GemmParams p, cudaStream_t st)
+int launch_bf16_pair_gemm(const void* a_bf, int a_is_km, const void* w_bf, int w_is_nk, GemmParams p, cudaStream_t st)
 {
     int dev = 0, sm_count = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || !gemm_kernels_ready(dev, &sm_count)) return HIF8_ERR_CUDA;
@@ -748,7 +775,10 @@ int launch_bf16_pair_gemm(const void* a_bf, const void* w_bf, int w_is_nk, GemmP
     const long long tiles2 = (long long)((M + 2 * BM - 1) / (2 * BM)) * p.tiles_n;
     if (M <= 0 || N <= 0 || K <= 0 || tiles2 > 0x3FFFFFFF) return HIF8_ERR_SHAPE;
     CUtensorMap ma, mw;
-    if (!make_map(&ma, a_bf, (uint64_t)K, (uint64_t)M, (uint64_t)K, BK, BM, true)) return HIF8_ERR_CUDA;
+    // A boxes: this CTA's 128 rows of [M,K], or two boxes of 64 columns of [K,M]
+    const bool oka = a_is_km ? make_map(&ma, a_bf, (uint64_t)M, (uint64_t)K, (uint64_t)M, 64, BK, true)
+                             : make_map(&ma, a_bf, (uint64_t)K, (uint64_t)M, (uint64_t)K, BK, BM, true);
+    if (!oka) return HIF8_ERR_CUDA;
     // W boxes are one CTA's half of the 256-column tile: 128 rows of [N,K], or two boxes of 64 columns of [K,N]
     const bool okw = w_is_nk ? make_map(&mw, w_bf, (uint64_t)K, (uint64_t)N, (uint64_t)K, BK, BN / 2, true)
                              : make_map(&mw, w_bf, (uint64_t)N, (uint64_t)K, (uint64_t)N, 64, BK, true);
@@ -763,8 +793,11 @@ int launch_bf16_pair_gemm(const void* a_bf, const void* w_bf, int w_is_nk, GemmP
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    const cudaError_t lrc = w_is_nk ? cudaLaunchKernelEx(&cfg, bf16_gemm_pair_kernel<true>, ma, mw, p)
-                                    : cudaLaunchKernelEx(&cfg, bf16_gemm_pair_kernel<false>, ma, mw, p);
+    cudaError_t lrc;
+    if (a_is_km) lrc = w_is_nk ? cudaLaunchKernelEx(&cfg, bf16_gemm_pair_kernel<true, true>, ma, mw, p)
+                               : cudaLaunchKernelEx(&cfg, bf16_gemm_pair_kernel<true, false>, ma, mw, p);
+    else lrc = w_is_nk ? cudaLaunchKernelEx(&cfg, bf16_gemm_pair_kernel<false, true>, ma, mw, p)
+                       : cudaLaunchKernelEx(&cfg, bf16_gemm_pair_kernel<false, false>, ma, mw, p);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return (lrc == cudaSuccess && cudaGetLastError() == cudaSuccess) ? HIF8_OK : HIF8_ERR_CUDA;
 }
@@ -773,13 +806,14 @@ int launch_bf16_pair_gemm(const void* a_bf, const void* w_bf, int w_is_nk, GemmP
 
 using namespace hif8;
 
-static int gemm_entry(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int64_t ldw, int w_is_nk, void* C, int64_t ldc,
-                      int c_dtype, int M, int N, int K, const int* d_scale_exp_a, const int* d_scale_exp_w,
-                      const int* d_scale_exp_w_channel, void* workspace, size_t workspace_bytes, hif8_stream_t stream)
+static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t* Wq, int64_t ldw, int w_is_nk, void* C,
+                      int64_t ldc, int c_dtype, int M, int N, int K, const int* d_scale_exp_a, const int* d_scale_exp_w,
+                      const int* d_scale_exp_w_channel, int accumulate, void* workspace, size_t workspace_bytes,
+                      hif8_stream_t stream)
 {
     if (c_dtype != HIF8_BF16 && c_dtype != HIF8_F32) return HIF8_ERR_DTYPE;
     if (M < 0 || N < 0 || K < 0 || (K & 15)) return HIF8_ERR_SHAPE;
-    if (lda < K || ldc < N || ldw < (w_is_nk ? K : N)) return HIF8_ERR_SHAPE;
+    if (lda < (a_is_km ? M : K) || ldc < N || ldw < (w_is_nk ? K : N)) return HIF8_ERR_SHAPE;
     if (M == 0 || N == 0) return HIF8_OK;
     if (!Aq || !Wq || !C) return HIF8_ERR_NULL;
     const size_t c_item = c_dtype == HIF8_F32 ? 4 : 2;
@@ -795,7 +829,9 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int64_t
     if (major != 10) return HIF8_ERR_CUDA;
 
     CUtensorMap map_a, map_w;
-    if (!make_map(&map_a, Aq, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BK, BM)) return HIF8_ERR_CUDA;
+    const bool ok_a = a_is_km ? make_map(&map_a, Aq, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BM, BK)
+                              : make_map(&map_a, Aq, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BK, BM);
+    if (!ok_a) return HIF8_ERR_CUDA;
     // byte tiles of one CTA of a pair: 128 rows of A, 128 of the 256 columns of W
     const bool ok_w = w_is_nk ? make_map(&map_w, Wq, (uint64_t)K, (uint64_t)N, (uint64_t)ldw, BK, BN / 2)
                               : make_map(&map_w, Wq, (uint64_t)N, (uint64_t)K, (uint64_t)ldw, BN / 2, BK);
@@ -804,6 +840,7 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int64_t
     GemmParams p{};
     p.C = C; p.ldc = ldc; p.c_is_f32 = c_dtype == HIF8_F32; p.M = M; p.N = N; p.K = K;
     p.d_sa = d_scale_exp_a; p.d_sw = d_scale_exp_w; p.d_sw_channel = d_scale_exp_w_channel;
+    p.accumulate = accumulate ? 1 : 0;
     p.status = reinterpret_cast<int*>(workspace);
     p.tiles_m = (M + BM - 1) / BM; p.tiles_n = (N + BN - 1) / BN;
     // both kernels work on 256 x 256 tiles, one per pair of CTAs
@@ -819,14 +856,14 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int64_t
     // byte is decoded exactly once by the conversion kernel and the tensor-core kernel reads BF16 tiles through TMA.
     // Otherwise the fused kernel decodes the byte tiles of every CTA in shared memory.
     const size_t bytes_a = (((size_t)M * K * 2) + 255) & ~(size_t)255, bytes_w = (((size_t)K * N * 2) + 255) & ~(size_t)255;
-    const bool contiguous = lda == K && ldw == (w_is_nk ? K : N);
+    const bool contiguous = lda == (a_is_km ? M : K) && ldw == (w_is_nk ? K : N);
     if (contiguous && workspace_bytes >= kGemmWorkspaceBytes + bytes_a + bytes_w && !(reinterpret_cast<uintptr_t>(workspace) & 255)) {
         unsigned char* a_bf = reinterpret_cast<unsigned char*>(workspace) + kGemmWorkspaceBytes;
         unsigned char* w_bf = a_bf + bytes_a;
         int rc = hif8_decode(Aq, a_bf, HIF8_BF16, (size_t)M * K, 0, stream);
         if (rc == HIF8_OK) rc = hif8_decode(Wq, w_bf, HIF8_BF16, (size_t)K * N, 0, stream);
         if (rc != HIF8_OK) return rc;
-        return launch_bf16_pair_gemm(a_bf, w_bf, w_is_nk, p, st);
+        return launch_bf16_pair_gemm(a_bf, a_is_km, w_bf, w_is_nk, p, st);
     }
 
     cudaLaunchConfig_t cfg{};
@@ -838,8 +875,11 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int64_t
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    const cudaError_t lrc = w_is_nk ? cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<true>, map_a, map_w, p)
-                                    : cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<false>, map_a, map_w, p);
+    cudaError_t lrc;
+    if (a_is_km) lrc = w_is_nk ? cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<true, true>, map_a, map_w, p)
+                               : cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<true, false>, map_a, map_w, p);
+    else lrc = w_is_nk ? cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<false, true>, map_a, map_w, p)
+                       : cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<false, false>, map_a, map_w, p);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return (lrc == cudaSuccess && cudaGetLastError() == cudaSuccess) ? HIF8_OK : HIF8_ERR_CUDA;
 }
@@ -848,7 +888,7 @@ extern "C" int hif8_gemm(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int6
                          int c_dtype, int M, int N, int K, const int* d_scale_exp_a, const int* d_scale_exp_w,
                          void* workspace, size_t workspace_bytes, hif8_stream_t stream)
 {
-    return gemm_entry(Aq, lda, Wq, ldw, w_is_nk, C, ldc, c_dtype, M, N, K, d_scale_exp_a, d_scale_exp_w, nullptr, workspace,
+    return gemm_entry(Aq, lda, 0, Wq, ldw, w_is_nk, C, ldc, c_dtype, M, N, K, d_scale_exp_a, d_scale_exp_w, nullptr, 0, workspace,
                       workspace_bytes, stream);
 }
 
@@ -858,8 +898,18 @@ extern "C" int hif8_gemm_channel_scaled(const uint8_t* Aq, int64_t lda, const ui
                                         hif8_stream_t stream)
 {
     if (!d_scale_exp_w_channel && M > 0 && N > 0) return HIF8_ERR_NULL;
-    return gemm_entry(Aq, lda, Wq, ldw, w_is_nk, C, ldc, c_dtype, M, N, K, d_scale_exp_a, nullptr, d_scale_exp_w_channel,
+    return gemm_entry(Aq, lda, 0, Wq, ldw, w_is_nk, C, ldc, c_dtype, M, N, K, d_scale_exp_a, nullptr, d_scale_exp_w_channel, 0,
                       workspace, workspace_bytes, stream);
+}
+
+extern "C" int hif8_gemm_ex(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t* Wq, int64_t ldw, int w_is_nk, void* C,
+                            int64_t ldc, int c_dtype, int M, int N, int K, const int* d_scale_exp_a, const int* d_scale_exp_w,
+                            const int* d_scale_exp_w_channel, int accumulate, void* workspace, size_t workspace_bytes,
+                            hif8_stream_t stream)
+{
+    return gemm_entry(Aq, lda, a_is_km ? 1 : 0, Wq, ldw, w_is_nk ? 1 : 0, C, ldc, c_dtype, M, N, K, d_scale_exp_a,
+                      d_scale_exp_w_channel ? nullptr : d_scale_exp_w, d_scale_exp_w_channel, accumulate, workspace,
+                      workspace_bytes, stream);
 }
 
 extern "C" int hif8_gemm_status(const void* workspace, hif8_stream_t stream)

@@ -11,6 +11,7 @@ struct GemmParams {
     int M, N, K;
     const int* d_sa;
     const int* d_sw;
+    int accumulate;           // nonzero: C += result instead of C = result
     const int* d_sw_channel;  // when set: one weight exponent per output column [N]; d_sw is then ignored
     int* status;
     int tiles_m, tiles_n;
@@ -20,9 +21,9 @@ struct GemmParams {
     double* err_sum;
 };
 
-// C (or the squared error) from operands that are already BF16 in device memory: a_bf [M,K], w_bf [K,N] or [N,K],
+// C (or the squared error) from operands that are already BF16 in device memory: a_bf [M,K] or (a_is_km) [K,M], w_bf [K,N] or (w_is_nk) [N,K],
 // both contiguous.  Fills in the tile counts of `p`; p.status must point at a zeroed device int.
-int launch_bf16_pair_gemm(const void* a_bf, const void* w_bf, int w_is_nk, GemmParams p, cudaStream_t st);
+int launch_bf16_pair_gemm(const void* a_bf, int a_is_km, const void* w_bf, int w_is_nk, GemmParams p, cudaStream_t st);
 
 // SM count of the current device; HIF8_ERR_CUDA unless it is a compute-capability-10.0 device
 int checked_device(int* sms);

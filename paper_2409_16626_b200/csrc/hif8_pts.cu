@@ -109,7 +109,7 @@ extern "C" int hif8_pts_search(const void* A, const void* W, int dtype, int w_is
         for (int iw = 0; iw < n_exp; iw++) {  // "MatMul & Restore" and "Quantization Error" in one launch
             p.d_sa = &ctl->exps[ia]; p.d_sw = &ctl->exps[iw];
             p.err_sum = &ctl->sums[ia * n_exp + iw];
-            const int rc = launch_bf16_pair_gemm(a_bf + align256(mk * 2) * ia, w_bf + align256(kn * 2) * iw, w_is_nk, p, st);
+            const int rc = launch_bf16_pair_gemm(a_bf + align256(mk * 2) * ia, 0, w_bf + align256(kn * 2) * iw, w_is_nk, p, st);
             if (rc != HIF8_OK) return rc;
         }
     pts_finish_kernel<<<1, 32, 0, st>>>(ctl, e_min, n_exp, 1.0 / ((double)M * (double)N), d_err, d_best);

@@ -1,0 +1,182 @@
+// Conversion with transposed store: dst[c, r] = To_HiF8(src[r, c] * 2^e).  (Backward-pass operand form: the GEMMs of
+// the backward pass contract over the other dimension of the activation / gradient tensors.)
+//
+// A block converts a tile of 128 source rows by 8 source vectors (32 FP32 or 64 16-bit columns).  Thread (rq, cv)
+// loads the four vectors of rows 4 rq .. 4 rq + 3 in vector-column cv (four independent 16-byte loads; a warp covers
+// four full 128-byte lines per instruction), converts them, and packs the four bytes of each of its columns into one
+// 32-bit word of a shared tile held transposed ([column][row / 4], row stride 33 words: conflict-free for FP32,
+// two-way for 16-bit sources).  The block then writes each column of the tile as 128 contiguous bytes of a dst row.
+// Traffic is that of the flat encoder: one read of the source, one byte written per element.
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cstdint>
+
+#include "hif8.h"
+#include "hif8_device.cuh"
+#include "hif8_internal.cuh"
+
+namespace hif8 {
+extern std::atomic<uint64_t> g_launches;
+namespace {
+
+struct TrParams {
+    const void* src;
+    uint8_t* dst;
+    long long rows, cols;
+    int scale_exp;
+    const int* d_scale_exp;
+    unsigned flags;
+    unsigned long long seed;
+};
+
+constexpr int kTileRows = 128;
+constexpr int kTileVecs = 8;          // vector-columns per tile
+constexpr int kTileStride = kTileRows / 4 + 1;  // words per tile column
+
+template <int SRC, int MODE>
+__global__ void __launch_bounds__(kThreads) encode_transpose_kernel(const TrParams p)
+{
+    constexpr int PV = SrcTraits<SRC>::kPerVec;
+    constexpr int TC = kTileVecs * PV;  // source columns per tile
+    __shared__ SmemTables sm;
+    __shared__ uint32_t tile[TC * kTileStride];
+    setup_tables<true, MODE != HIF8_RND_TA, false, MODE, SRC>(sm, p.flags);
+    const float scale = pow2f(p.d_scale_exp ? clamp_exp(*p.d_scale_exp) : p.scale_exp);
+    const uint32_t k0 = (uint32_t)p.seed, k1 = (uint32_t)(p.seed >> 32);
+    const long long nvc = p.cols / PV;                        // vectors per source row
+    const long long tiles_c = (nvc + kTileVecs - 1) / kTileVecs;
+    const long long tiles_r = (p.rows + kTileRows - 1) / kTileRows;
+    const int cv = threadIdx.x % kTileVecs, rq = threadIdx.x / kTileVecs;
+    const uint4* src = reinterpret_cast<const uint4*>(p.src);
+
+    for (long long tix = blockIdx.x; tix < tiles_c * tiles_r; tix += gridDim.x) {
+        // consecutive blocks take consecutive row-tiles of one column strip: their dst segments are adjacent
+        const long long tc = tix / tiles_r, tr = tix % tiles_r;
+        const long long r0 = tr * kTileRows, v0 = tc * kTileVecs;
+        const long long vcol = v0 + cv;
+        uint4 v[4];
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+            const long long r = r0 + rq * 4 + j;
+            v[j] = (r < p.rows && vcol < nvc) ? __ldcs(src + r * nvc + vcol) : make_uint4(0, 0, 0, 0);
+        }
+        uint32_t packed[PV];
+#pragma unroll
+        for (int k = 0; k < PV; k++) packed[k] = 0;
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+            const long long r = r0 + rq * 4 + j;
+            uint32_t rw[8];
+            uint4 q0 = make_uint4(0, 0, 0, 0), q1 = q0;
+            if (MODE == HIF8_RND_SR) {
+                const unsigned long long u = (unsigned long long)r * nvc + vcol;  // flat vector index in the source
+                q0 = philox4x32_10((uint32_t)(u * (PV / 4)), (uint32_t)((u * (PV / 4)) >> 32), k0, k1);
+                if (PV == 8) q1 = philox4x32_10((uint32_t)(u * 2 + 1), (uint32_t)((u * 2 + 1) >> 32), k0, k1);
+            }
+            rw[0] = q0.x; rw[1] = q0.y; rw[2] = q0.z; rw[3] = q0.w; rw[4] = q1.x; rw[5] = q1.y; rw[6] = q1.z; rw[7] = q1.w;
+#pragma unroll
+            for (int k = 0; k < PV; k++) {
+                float x; uint32_t raw;
+                unpack<SRC>(v[j], k, x, raw);
+                packed[k] |= encode_one<MODE, SRC>(x, raw, scale, sm.ta, sm.thr, rw[k]) << (8 * j);
+            }
+        }
+        __syncthreads();  // the previous tile has been written out
+#pragma unroll
+        for (int k = 0; k < PV; k++) tile[(cv * PV + k) * kTileStride + rq] = packed[k];
+        __syncthreads();
+        // column c of the tile = 128 bytes of dst row (v0 * PV + c), starting at byte r0; 16 bytes per thread
+        for (int o = threadIdx.x; o < TC * (kTileRows / 16); o += kThreads) {
+            const int c = o / (kTileRows / 16), seg = o % (kTileRows / 16);
+            const long long col = v0 * PV + c, r = r0 + seg * 16;
+            if (col < p.cols && r < p.rows) {  // rows is a multiple of 16 on this path: a segment is all in or all out
+                const uint32_t* w = tile + c * kTileStride + seg * 4;
+                __stcs(reinterpret_cast<uint4*>(p.dst + col * p.rows + r), make_uint4(w[0], w[1], w[2], w[3]));
+            }
+        }
+    }
+}
+
+// any shape and alignment: one thread per source element
+template <int SRC, int MODE>
+__global__ void __launch_bounds__(kThreads) encode_transpose_scalar_kernel(const TrParams p)
+{
+    __shared__ SmemTables sm;
+    setup_tables<true, MODE != HIF8_RND_TA, false, MODE, SRC>(sm, p.flags);
+    const float scale = pow2f(p.d_scale_exp ? clamp_exp(*p.d_scale_exp) : p.scale_exp);
+    const uint32_t k0 = (uint32_t)p.seed, k1 = (uint32_t)(p.seed >> 32);
+    const unsigned long long n = (unsigned long long)p.rows * (unsigned long long)p.cols;
+    for (unsigned long long i = (unsigned long long)blockIdx.x * kThreads + threadIdx.x; i < n; i += (unsigned long long)gridDim.x * kThreads) {
+        const unsigned long long r = i / (unsigned long long)p.cols, c = i - r * (unsigned long long)p.cols;
+        float x; uint32_t raw;
+        load_scalar<SRC>(p.src, i, x, raw);
+        uint32_t word = 0;
+        if (MODE == HIF8_RND_SR) {
+            const uint4 q = philox4x32_10((uint32_t)(i >> 2), (uint32_t)(i >> 34), k0, k1);
+            const uint32_t qq[4] = {q.x, q.y, q.z, q.w};
+            word = qq[i & 3];
+        }
+        p.dst[c * (unsigned long long)p.rows + r] = (uint8_t)encode_one<MODE, SRC>(x, raw, scale, sm.ta, sm.thr, word);
+    }
+}
+
+template <int SRC, int MODE>
+int launch(const TrParams& p, bool vec, int sms, cudaStream_t st)
+{
+    if (vec) {
+        constexpr int PV = SrcTraits<SRC>::kPerVec;
+        const long long nvc = p.cols / PV;
+        const long long tiles = ((nvc + kTileVecs - 1) / kTileVecs) * ((p.rows + kTileRows - 1) / kTileRows);
+        encode_transpose_kernel<SRC, MODE><<<(unsigned)(tiles < 0x7FFFFFFFll ? tiles : 0x7FFFFFFFll), kThreads, 0, st>>>(p);
+    } else {
+        const unsigned long long n = (unsigned long long)p.rows * (unsigned long long)p.cols;
+        const unsigned long long need = (n + kThreads - 1) / kThreads, cap = (unsigned long long)sms * 32;
+        encode_transpose_scalar_kernel<SRC, MODE><<<(unsigned)(need < cap ? need : cap), kThreads, 0, st>>>(p);
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
+}
+
+template <int SRC>
+int launch_mode(int rnd, const TrParams& p, bool vec, int sms, cudaStream_t st)
+{
+    switch (rnd) {
+        case HIF8_RND_TA: return launch<SRC, HIF8_RND_TA>(p, vec, sms, st);
+        case HIF8_RND_HR: return launch<SRC, HIF8_RND_HR>(p, vec, sms, st);
+        case HIF8_RND_SSR: return launch<SRC, HIF8_RND_SSR>(p, vec, sms, st);
+        case HIF8_RND_TE: return launch<SRC, HIF8_RND_TE>(p, vec, sms, st);
+        default: return launch<SRC, HIF8_RND_SR>(p, vec, sms, st);
+    }
+}
+
+}  // namespace
+}  // namespace hif8
+
+using namespace hif8;
+
+extern "C" int hif8_encode_transpose(const void* src, int src_dtype, uint8_t* dst, int64_t rows, int64_t cols, int scale_exp,
+                                     const int* d_scale_exp, int rnd, unsigned flags, uint64_t seed, hif8_stream_t stream)
+{
+    if (src_dtype != HIF8_F32 && src_dtype != HIF8_BF16 && src_dtype != HIF8_F16) return HIF8_ERR_DTYPE;
+    if (rnd < HIF8_RND_TA || rnd > HIF8_RND_SR) return HIF8_ERR_ROUND;
+    if (flags & ~(unsigned)(HIF8_FLAG_SATURATE | HIF8_FLAG_NAN_TO_ZERO)) return HIF8_ERR_FLAGS;
+    if (scale_exp < -126 || scale_exp > 126) return HIF8_ERR_SCALE_RANGE;
+    if (rows < 0 || cols < 0) return HIF8_ERR_SHAPE;
+    if (rows == 0 || cols == 0) return HIF8_OK;
+    if (!src || !dst) return HIF8_ERR_NULL;
+    int sms; int rc = checked_device(&sms);
+    if (rc) return rc;
+    const int pv = src_dtype == HIF8_F32 ? 4 : 8;
+    const bool vec = !(reinterpret_cast<uintptr_t>(src) & 15u) && !(reinterpret_cast<uintptr_t>(dst) & 15u) && cols % pv == 0 &&
+                     rows % 16 == 0;
+    TrParams p{};
+    p.src = src; p.dst = dst; p.rows = rows; p.cols = cols; p.scale_exp = scale_exp; p.d_scale_exp = d_scale_exp;
+    p.flags = flags; p.seed = seed;
+    cudaStream_t st = (cudaStream_t)stream;
+    switch (src_dtype) {
+        case HIF8_F32: return launch_mode<HIF8_F32>(rnd, p, vec, sms, st);
+        case HIF8_BF16: return launch_mode<HIF8_BF16>(rnd, p, vec, sms, st);
+        default: return launch_mode<HIF8_F16>(rnd, p, vec, sms, st);
+    }
+}
