@@ -241,6 +241,10 @@ def extra_results(H, torch, hbm_peak, peak_kind):
     for name, measure in (("measuring_iteration", 1), ("plain_iteration", 0)):
         ms = timed(lambda r: H.hif8_delayed_scale_encode(a, H.BF16, Aq, M * K, H.RND_TA, 0, 0, state, measure, 14), 20)
         dl[name] = {"ms": ms, "GBps": 3 * M * K / ms / 1e6, "frac": 3 * M * K / ms / 1e6 / hbm_peak}
+    ms = timed(lambda r: H.hif8_encode_transpose(a, H.BF16, Aq, M, K, 3, None, H.RND_HR), 20)
+    out["encode_transpose_bf16_8192x8192_HR"] = {"ms": ms, "bytes_per_element": 3, "GBps": 3 * M * K / ms / 1e6,
+                                                 "frac": 3 * M * K / ms / 1e6 / hbm_peak, "peak": hbm_peak,
+                                                 "peak_kind": f"of {peak_kind}"}
     out["delayed_scale_encode_bf16_8192x8192"] = {"bytes_per_element": 3, "calls": dl, "peak": hbm_peak,
                                                   "peak_kind": f"of {peak_kind}"}
     H.hif8_amax_scale_encode(a, H.BF16, Aq, M * K, 14, H.RND_TA, 0, 0, None, None, se[0:1], None, ws, wsb)
@@ -261,7 +265,18 @@ def extra_results(H, torch, hbm_peak, peak_kind):
     ch_se.fill_(int(se[1]))
     ms_c = timed(lambda r: H.hif8_gemm_channel_scaled(Aq, K, Wq, N, 0, C, N, H.BF16, M, N, K, se[0:1], ch_se, gws, gws_b), 10)
     st3 = H.hif8_gemm_status(gws)
+    # backward-pass forms of the same size: dgrad reads the weight as [N,K], wgrad reads A as [K,M] and accumulates in FP32
+    bw = {}
+    ms_d = timed(lambda r: H.hif8_gemm_ex(Aq, K, 0, Wq, K, 1, C, N, H.BF16, M, N, K, se[0:1], se[1:2], None, 0, gws, gws_b), 10)
+    bw["dgrad_form_w_as_[N,K]"] = {"ms": ms_d, "TFLOPs": flops / ms_d / 1e9, "frac": flops / ms_d / 1e9 / tf_peak,
+                                   "device_status": H.hif8_gemm_status(gws)}
+    C32 = torch.zeros(M, N, dtype=torch.float32, device="cuda")
+    ms_w = timed(lambda r: H.hif8_gemm_ex(Aq, M, 1, Wq, N, 0, C32, N, H.F32, M, N, K, se[0:1], se[1:2], None, 1, gws, gws_b), 10)
+    bw["wgrad_form_a_as_[K,M]_fp32_accumulate"] = {"ms": ms_w, "TFLOPs": flops / ms_w / 1e9, "frac": flops / ms_w / 1e9 / tf_peak,
+                                                   "device_status": H.hif8_gemm_status(gws)}
+    del C32
     out["gemm_8192x28672x8192"] = {
+        "backward_forms": bw,
         "decode_once_channel_scaled": {"ms": ms_c, "TFLOPs": flops / ms_c / 1e9, "frac": flops / ms_c / 1e9 / tf_peak,
                                        "device_status": st3, "note": "one weight exponent per output column"},
         "decode_once": {"ms": ms, "TFLOPs": flops / ms / 1e9, "frac": flops / ms / 1e9 / tf_peak, "device_status": st1,

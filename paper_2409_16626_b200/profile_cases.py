@@ -4,7 +4,8 @@
 
 cases: convert_f32 (FP32 4096^2: per-tensor scaled encode + decode), fq_bf16 (BF16 4096x8192 fake-quant, TA and HR,
 fused amax and given scale), encode_modes_f32 (FP32 2^25 log-uniform, every rounding mode), gemm (HiF8 GEMM
-4096 x 7168 x 4096, fused and decode-once paths).  Inputs are seeded device-side random tensors.
+4096 x 7168 x 4096, fused and decode-once paths), gemm_forms (same size, decode-once path, the four operand layouts:
+forward, dgrad form, wgrad form with FP32 accumulation, both transposed).  Inputs are seeded device-side random tensors.
 """
 import sys
 
@@ -57,6 +58,19 @@ def main():
         for r in range(reps):
             H.hif8_gemm(A, K, W, N, 0, C, N, H.BF16, M, N, K, None, None, gws, big)
             H.hif8_gemm(A, K, W, N, 0, C, N, H.BF16, M, N, K, None, None, gws, 256)
+    elif case == "gemm_forms":
+        M, N, K = 4096, 7168, 4096
+        A = torch.randint(8, 100, (M * K,), dtype=torch.uint8, device="cuda", generator=g)
+        W = torch.randint(8, 100, (K * N,), dtype=torch.uint8, device="cuda", generator=g)
+        Cb = torch.zeros(M, N, dtype=torch.bfloat16, device="cuda")
+        Cf = torch.zeros(M, N, dtype=torch.float32, device="cuda")
+        big = H.hif8_workspace_bytes(H.WS_GEMM, M * K + K * N)
+        gws = torch.empty(big, dtype=torch.uint8, device="cuda")
+        for r in range(reps):
+            H.hif8_gemm_ex(A, K, 0, W, N, 0, Cb, N, H.BF16, M, N, K, None, None, None, 0, gws, big)
+            H.hif8_gemm_ex(A, K, 0, W, K, 1, Cb, N, H.BF16, M, N, K, None, None, None, 0, gws, big)
+            H.hif8_gemm_ex(A, M, 1, W, N, 0, Cf, N, H.F32, M, N, K, None, None, None, 1, gws, big)
+            H.hif8_gemm_ex(A, M, 1, W, K, 1, Cb, N, H.BF16, M, N, K, None, None, None, 0, gws, big)
     else:
         raise SystemExit(f"unknown case {case}")
     torch.cuda.synchronize()
