@@ -686,3 +686,47 @@ void hif8o_gemm_entries_ex(const uint8_t* Aq, long long lda, int a_is_km, const 
         S[t] = ldexp(sab, -s);
     }
 }
+
+/* ------------------------------------------------------------------------- *
+ * Section 5.1, "Adaptive Loss-Scaling (ALS)": backward loss scaling whose scale
+ * window (growth interval) moves along the list {1, 20, 50, 100, 200, 500, 1000}.
+ * "The initial scale value and scale window are set to 2^32 and 20.  During
+ * training, if the scale value increases three times, the scale window will
+ * increase once as per the list order.  If the scale value decreases three times
+ * in a row, scale window will decrease once."
+ * The scale itself follows the usual dynamic loss scaling the paper builds on
+ * (growth factor 2, backoff factor 1/2, so the scale stays a power of two):
+ *   overflow seen in this iteration's gradients -> scale / 2, clean-step counter = 0
+ *   otherwise clean-step counter + 1; when it reaches the window -> scale * 2, counter = 0.
+ * READINGS: "increases three times" counts increases since the last window change
+ * (decreases in between do not cancel them); "decreases three times in a row" is a run
+ * of decreases not interrupted by an increase; a window change clears both counts; the
+ * window stops at the ends of the list; the exponent is kept within [-126, 126].
+ * found_inf[t] != 0: the gradients of iteration t held an Inf or NaN.
+ * scale_exp[t], window[t]: log2 of the scale, and the window, in force DURING iteration t.
+ * ------------------------------------------------------------------------- */
+static const int k_als_windows[7] = {1, 20, 50, 100, 200, 500, 1000};
+
+void hif8o_als_run(const int* found_inf, int T, int init_scale_exp, int init_window_index, int* scale_exp, int* window)
+{
+    int se = init_scale_exp, wi = init_window_index, clean = 0, ups = 0, downs = 0;
+    for (int t = 0; t < T; t++) {
+        scale_exp[t] = se;
+        window[t] = k_als_windows[wi];
+        if (found_inf[t]) {
+            if (se > -126) se -= 1;
+            clean = 0;
+            downs += 1;
+            if (downs == 3) { if (wi > 0) wi -= 1; ups = 0; downs = 0; }
+        } else {
+            clean += 1;
+            if (clean >= k_als_windows[wi]) {
+                if (se < 126) se += 1;
+                clean = 0;
+                ups += 1;
+                downs = 0;
+                if (ups == 3) { if (wi < 6) wi += 1; ups = 0; downs = 0; }
+            }
+        }
+    }
+}

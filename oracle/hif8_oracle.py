@@ -37,6 +37,7 @@ _lib.hif8o_gemm_entries_channel.argtypes = [_vp, _ll, _vp, _ll, _i, _i, _i, _vp,
 _lib.hif8o_delayed_scale_run.argtypes = [_vp, _i, _i, _i, _i, _vp]
 _lib.hif8o_encode_transpose.argtypes = [_vp, _i, _vp, _ll, _ll, _i, _i, _u, _u64, _i]
 _lib.hif8o_gemm_entries_ex.argtypes = [_vp, _ll, _i, _vp, _ll, _i, _i, _i, _i, _vp, _vp, _vp, _sz, _vp, _vp]
+_lib.hif8o_als_run.argtypes = [_vp, _i, _i, _i, _vp, _vp]
 _lib.hif8o_gemm_full.argtypes = [_vp, _ll, _vp, _ll, _i, _i, _i, _i, _i, _i, _vp, _vp]
 
 
@@ -237,3 +238,15 @@ def gemm_entries_ex(Aq, a_is_km, Wq, w_is_nk, sa, sw, rows, cols):
                                int(sw) if ch is None else 0, None if ch is None else _ptr(ch), _ptr(rows), _ptr(cols),
                                rows.size, _ptr(cs), _ptr(s))
     return cs, s
+
+
+ALS_WINDOWS = (1, 20, 50, 100, 200, 500, 1000)
+
+
+def als_run(found_inf, init_scale_exp=32, init_window_index=1):
+    """Adaptive loss scaling over a sequence of overflow flags: (log2 scale, window) in force during each iteration."""
+    f = np.ascontiguousarray(found_inf, dtype=np.int32)
+    se = np.empty(f.size, dtype=np.int32)
+    win = np.empty(f.size, dtype=np.int32)
+    _lib.hif8o_als_run(_ptr(f), f.size, init_scale_exp, init_window_index, _ptr(se), _ptr(win))
+    return se, win

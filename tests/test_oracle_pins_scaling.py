@@ -4,6 +4,7 @@ with something it does not compute itself: the already pinned per-tensor routine
 that hold for any correct implementation, or sequences worked out by hand."""
 import numpy as np
 import pytest
+import torch
 
 import workloads as W
 from oracle import hif8_oracle as O
@@ -162,3 +163,49 @@ def test_gemm_ex_equals_the_plain_gemm_on_explicitly_transposed_operands():
     c, _ = O.gemm_entries_ex(np.ascontiguousarray(A1.T), 1, np.ascontiguousarray(W1.T), 1, 0, 0, rows, cols)
     expect = np.zeros(M * N); expect[2 * N + 7] = 2.0
     assert np.array_equal(c, expect)
+
+
+# ----------------------------------------------------------------------------- adaptive loss scaling (Section 5.1)
+def test_als_initial_state_and_window_walk_worked_by_hand():
+    # the paper's start: scale 2^32, window 20.  60 clean iterations = three increases -> window 50
+    se, win = O.als_run(np.zeros(60 + 150 + 1, dtype=np.int32))
+    assert se[0] == 32 and win[0] == 20
+    assert se[19] == 32 and se[20] == 33 and se[40] == 34 and se[60] == 35   # an increase after every 20 clean steps
+    assert win[59] == 20 and win[60] == 50                                      # third increase moves the window up
+    assert se[60 + 49] == 35 and se[60 + 50] == 36 and se[60 + 100] == 37 and se[60 + 150] == 38
+    assert win[60 + 149] == 50 and win[60 + 150] == 100
+    # three overflows in a row: three halvings, then the window steps down the list (20 -> 1)
+    se, win = O.als_run(np.array([1, 1, 1, 0, 0, 0, 0], dtype=np.int32))
+    assert se.tolist() == [32, 31, 30, 29, 30, 31, 32] and win.tolist() == [20, 20, 20, 1, 1, 1, 20]
+    # (with window 1 every clean step doubles, so the third clean step is the third increase: back up to 20)
+    se, win = O.als_run(np.array([1, 1, 1, 0, 0, 0, 0, 0], dtype=np.int32))
+    assert win.tolist() == [20, 20, 20, 1, 1, 1, 20, 20] and se[7] == 32 and se[6] == 32
+    # an increase between overflows breaks the run of decreases: two overflows, 20 clean steps (one increase), one more
+    f = np.array([1, 1] + [0] * 20 + [1, 0], dtype=np.int32)
+    se, win = O.als_run(f)
+    assert np.all(win == 20) and se[22] == 31 and se[23] == 30
+    # clean steps that do not change the scale do not break it (window 20: 5 clean steps change nothing)
+    f = np.array([1] + [0] * 5 + [1] + [0] * 5 + [1, 0], dtype=np.int32)
+    se, win = O.als_run(f)
+    assert win[12] == 20 and win[13] == 1 and se[13] == 29
+    # the list ends: the window stays at 1 / at 1000
+    se, win = O.als_run(np.ones(40, dtype=np.int32), init_window_index=0)
+    assert np.all(win == 1) and se[39] == 32 - 39
+    se, win = O.als_run(np.zeros(1000 * 7, dtype=np.int32), init_window_index=6)
+    assert np.all(win == 1000) and se[-1] == 32 + 6
+    assert O.ALS_WINDOWS == (1, 20, 50, 100, 200, 500, 1000)
+
+
+def test_als_scale_rule_against_the_library_loss_scaler():
+    # given the oracle's windows, the scale must follow torch's dynamic loss-scale update (growth 2, backoff 1/2)
+    rng = np.random.default_rng(7)
+    f = (rng.random(4000) < 0.02).astype(np.int32)
+    f[100:103] = 1
+    f[900:906] = 1
+    se, win = O.als_run(f, init_scale_exp=16)
+    scale = torch.tensor(2.0 ** 16)
+    tracker = torch.tensor(0, dtype=torch.int32)
+    for t in range(f.size):
+        assert float(scale) == 2.0 ** int(se[t]), t
+        torch._amp_update_scale_(scale, tracker, torch.tensor(float(f[t])), 2.0, 0.5, int(win[t]))
+    assert len(set(win.tolist())) >= 3      # the walk visited several windows
