@@ -185,6 +185,29 @@ int hif8_delayed_scale_encode(const void* src, int src_dtype, uint8_t* dst, size
                               uint64_t seed, void* d_state, int measure, int target_exp, hif8_stream_t stream);
 
 /*
+ * Adaptive loss scaling (Section 5.1, "Adaptive Loss-Scaling (ALS)"), resident on the device.
+ * The loss scale is 2^scale_exp.  After each backward pass: hif8_check_finite over the (scaled) gradient tensors ORs
+ * "holds an Inf or NaN" into *d_found_inf (a device int the caller zeroes once; hif8_als_update clears it again), then
+ * hif8_als_update advances the controller:
+ *   overflow          -> scale / 2, clean-iteration count = 0
+ *   no overflow       -> count + 1; when it reaches the scale window -> scale * 2, count = 0
+ *   scale window      : walks the list {1, 20, 50, 100, 200, 500, 1000}: three increases of the scale since the last
+ *                       window change move it up one entry; three decreases not interrupted by an increase move it
+ *                       down one entry; a window change clears both counts; it stops at the ends of the list.
+ * The paper starts from scale 2^32 and window 20 (init_scale_exp = 32, init_window_index = 1).
+ * State: HIF8_ALS_STATE_BYTES of device memory, 16-byte aligned, eight ints the caller may read at any time:
+ *   [0] scale_exp  [1] window  [2] window index  [3] clean iterations  [4] increases counted  [5] decreases in a row
+ *   [6] iterations seen  [7] iterations that overflowed.
+ * The optimizer step of an overflowed iteration is the caller's to skip (it can test the flag on the device before
+ * hif8_als_update clears it).  Nothing here returns to the host or synchronises.
+ */
+#define HIF8_ALS_STATE_BYTES 64
+int hif8_als_state_init(void* d_state, int init_scale_exp, int init_window_index, hif8_stream_t stream);
+int hif8_als_update(void* d_state, int* d_found_inf, hif8_stream_t stream);
+/* *d_found_inf |= (some src[i] is +-Inf or NaN); one read of the tensor; src must be aligned to its element size */
+int hif8_check_finite(const void* src, int dtype, size_t n, int* d_found_inf, hif8_stream_t stream);
+
+/*
  * Quantize-dequantize in the source format ("simulated HiF8", Section 4: values are converted to only those
  * representable in HiF8):   dst[i] = value( To_HiF8_<rnd>(src[i] * 2^e) ) * 2^(-e)   in `dtype`.
  *   use_amax == 0: e = scale_or_target_exp.  No workspace needed (may be NULL).

@@ -15,12 +15,13 @@ FLAG_SATURATE, FLAG_NAN_TO_ZERO = 1, 2
 WS_AMAX_SCALE_ENCODE, WS_FAKE_QUANT, WS_GEMM = 0, 1, 2
 OK = 0
 SCALE_STATE_BYTES, SCALE_HISTORY_MAX = 1024, 32
+ALS_STATE_BYTES = 64
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libhif8.so")
 EXPORTS = ["hif8_encode", "hif8_decode", "hif8_amax", "hif8_amax_scale_encode", "hif8_fake_quant", "hif8_gemm", "hif8_gemm_status", "hif8_pts_search", "hif8_pts_workspace_bytes",
            "hif8_pts_status", "hif8_selftest_wait_timeout", "hif8_channel_amax_scale_encode", "hif8_gemm_channel_scaled",
-           "hif8_scale_state_init", "hif8_delayed_scale_encode", "hif8_gemm_ex", "hif8_encode_transpose",
+           "hif8_scale_state_init", "hif8_delayed_scale_encode", "hif8_gemm_ex", "hif8_encode_transpose", "hif8_als_state_init", "hif8_als_update", "hif8_check_finite",
            "hif8_amax_scale_encode_static", "hif8_workspace_bytes", "hif8_status_string", "hif8_launch_count"]
 
 if not os.path.exists(LIB_PATH):
@@ -59,6 +60,12 @@ lib.hif8_gemm_ex.argtypes = [_vp, _i64, _i, _vp, _i64, _i, _vp, _i64, _i, _i, _i
 lib.hif8_gemm_ex.restype = _i
 lib.hif8_encode_transpose.argtypes = [_vp, _i, _vp, _i64, _i64, _i, _vp, _i, _u, _u64, _vp]
 lib.hif8_encode_transpose.restype = _i
+lib.hif8_als_state_init.argtypes = [_vp, _i, _i, _vp]
+lib.hif8_als_state_init.restype = _i
+lib.hif8_als_update.argtypes = [_vp, _vp, _vp]
+lib.hif8_als_update.restype = _i
+lib.hif8_check_finite.argtypes = [_vp, _i, _sz, _vp, _vp]
+lib.hif8_check_finite.restype = _i
 lib.hif8_workspace_bytes.argtypes = [_i, _sz]
 lib.hif8_workspace_bytes.restype = _sz
 lib.hif8_status_string.argtypes = [_i]
@@ -208,3 +215,15 @@ def hif8_encode_transpose(src, src_dtype, dst, rows, cols, scale_exp=0, d_scale_
                           stream=None, check=True):
     return _check(lib.hif8_encode_transpose(_ptr(src), src_dtype, _ptr(dst), rows, cols, scale_exp, _ptr(d_scale_exp), rnd,
                                             flags, seed, _stream(stream)), check)
+
+
+def hif8_als_state_init(d_state, init_scale_exp=32, init_window_index=1, stream=None, check=True):
+    return _check(lib.hif8_als_state_init(_ptr(d_state), init_scale_exp, init_window_index, _stream(stream)), check)
+
+
+def hif8_als_update(d_state, d_found_inf, stream=None, check=True):
+    return _check(lib.hif8_als_update(_ptr(d_state), _ptr(d_found_inf), _stream(stream)), check)
+
+
+def hif8_check_finite(src, dtype, n, d_found_inf, stream=None, check=True):
+    return _check(lib.hif8_check_finite(_ptr(src), dtype, n, _ptr(d_found_inf), _stream(stream)), check)
