@@ -116,6 +116,18 @@ int hif8_amax(const void* src, int src_dtype, size_t n, float* d_amax_out, void*
               hif8_stream_t stream);
 
 /*
+ * The second half of the just-in-time form on its own: the scale exponent is derived on the device from an amax the
+ * caller already has in device memory, scale_exp = clamp(target_exp - floor(log2 *d_amax), -126, 126) (0 if it is 0),
+ * then dst = To_HiF8_<rnd>(src * 2^scale_exp).  *d_amax must be a non-negative float.  Together with hif8_amax this
+ * splits hif8_amax_scale_encode where a tensor is sharded over several GPUs: each rank reduces its shard, the ranks
+ * combine the 4-byte values with a max all-reduce, and each converts its shard with the common exponent (Section 5.1:
+ * one scale factor per GEMM input tensor).  Optional outputs as in hif8_amax_scale_encode.  No workspace.
+ */
+int hif8_encode_from_amax(const void* src, int src_dtype, uint8_t* dst, size_t n, int target_exp, int rnd, unsigned flags,
+                          uint64_t seed, const float* d_amax, int* d_scale_exp_out, float* d_scale_out,
+                          hif8_stream_t stream);
+
+/*
  * hif8_amax_scale_encode without a caller-supplied workspace.  (The paper has no counterpart: this entry
  * point exists for the benefit of the calling environment only.)
  *

@@ -21,7 +21,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libhif8.so")
 EXPORTS = ["hif8_encode", "hif8_decode", "hif8_amax", "hif8_amax_scale_encode", "hif8_fake_quant", "hif8_gemm", "hif8_gemm_status", "hif8_pts_search", "hif8_pts_workspace_bytes",
            "hif8_pts_status", "hif8_selftest_wait_timeout", "hif8_channel_amax_scale_encode", "hif8_gemm_channel_scaled",
-           "hif8_scale_state_init", "hif8_delayed_scale_encode", "hif8_gemm_ex", "hif8_encode_transpose", "hif8_als_state_init", "hif8_als_update", "hif8_check_finite",
+           "hif8_scale_state_init", "hif8_delayed_scale_encode", "hif8_gemm_ex", "hif8_encode_transpose", "hif8_als_state_init", "hif8_als_update", "hif8_check_finite", "hif8_encode_from_amax",
            "hif8_amax_scale_encode_static", "hif8_workspace_bytes", "hif8_status_string", "hif8_launch_count"]
 
 if not os.path.exists(LIB_PATH):
@@ -66,6 +66,8 @@ lib.hif8_als_update.argtypes = [_vp, _vp, _vp]
 lib.hif8_als_update.restype = _i
 lib.hif8_check_finite.argtypes = [_vp, _i, _sz, _vp, _vp]
 lib.hif8_check_finite.restype = _i
+lib.hif8_encode_from_amax.argtypes = [_vp, _i, _vp, _sz, _i, _i, _u, _u64, _vp, _vp, _vp, _vp]
+lib.hif8_encode_from_amax.restype = _i
 lib.hif8_workspace_bytes.argtypes = [_i, _sz]
 lib.hif8_workspace_bytes.restype = _sz
 lib.hif8_status_string.argtypes = [_i]
@@ -227,3 +229,9 @@ def hif8_als_update(d_state, d_found_inf, stream=None, check=True):
 
 def hif8_check_finite(src, dtype, n, d_found_inf, stream=None, check=True):
     return _check(lib.hif8_check_finite(_ptr(src), dtype, n, _ptr(d_found_inf), _stream(stream)), check)
+
+
+def hif8_encode_from_amax(src, src_dtype, dst, n, target_exp, rnd, flags, seed, d_amax, d_scale_exp_out=None, d_scale_out=None,
+                          stream=None, check=True):
+    return _check(lib.hif8_encode_from_amax(_ptr(src), src_dtype, _ptr(dst), n, target_exp, rnd, flags, seed, _ptr(d_amax),
+                                            _ptr(d_scale_exp_out), _ptr(d_scale_out), _stream(stream)), check)

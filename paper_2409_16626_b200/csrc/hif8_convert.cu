@@ -624,6 +624,24 @@ int hif8_amax(const void* src, int src_dtype, size_t n, float* d_amax_out, void*
     return launch_amax(src, src_dtype, n, reinterpret_cast<uint32_t*>(workspace), d_amax_out, sms, st);
 }
 
+int hif8_encode_from_amax(const void* src, int src_dtype, uint8_t* dst, size_t n, int target_exp, int rnd, unsigned flags,
+                          uint64_t seed, const float* d_amax, int* d_scale_exp_out, float* d_scale_out, hif8_stream_t stream)
+{
+    int rc = check_common(src_dtype, rnd, flags);
+    if (rc) return rc;
+    if (target_exp < -22 || target_exp > 15) return HIF8_ERR_SCALE_RANGE;
+    if (!d_amax || (n && (!src || !dst))) return HIF8_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(d_amax) & 3u) return HIF8_ERR_ALIGN;
+    int sms; rc = device_info(&sms);
+    if (rc) return rc;
+    ConvParams p{};
+    p.src = src; p.dst = dst; p.n = n; p.flags = flags; p.seed = seed; p.target_exp = target_exp;
+    p.d_amax_bits = reinterpret_cast<const uint32_t*>(d_amax);  // a non-negative float: its bits order as the value
+    p.d_scale_exp_out = d_scale_exp_out; p.d_scale_out = d_scale_out;
+    const bool vec_ok = aligned16(src) && (reinterpret_cast<uintptr_t>(dst) % (src_dtype == HIF8_F32 ? 4 : 8)) == 0;
+    return dispatch_convert<false, false>(src_dtype, rnd, p, vec_ok, sms, (cudaStream_t)stream);
+}
+
 int hif8_fake_quant(const void* src, void* dst, int dtype, size_t n, int use_amax, int scale_or_target_exp, int rnd,
                     unsigned flags, uint64_t seed, float* d_amax_out, int* d_scale_exp_out, void* workspace,
                     size_t workspace_bytes, hif8_stream_t stream)
