@@ -496,7 +496,9 @@ extern "C" int hif8_channel_amax_scale_encode(const void* W, int src_dtype, uint
         const long long strips = (nvc + 32 * wx - 1) / (32 * wx);
         const int wy = 8 / wx;
         while (rpt > 4 && strips * ((rows + rpt * wy - 1) / (rpt * wy)) < (long long)pl.sms * 8) rpt >>= 1;
-        const int rpb_e = rpt * wy, rpb_a = 4 * rpb_e;
+        int rpt_a = 4 * rpt;  // the reduction likes longer walks, as long as every SM still gets eight blocks
+        while (rpt_a > rpt && strips * ((rows + rpt_a * wy - 1) / (rpt_a * wy)) < (long long)pl.sms * 8) rpt_a >>= 1;
+        const int rpb_e = rpt * wy, rpb_a = rpt_a * wy;
         const long long gy_e = (rows + rpb_e - 1) / rpb_e, gy_a = (rows + rpb_a - 1) / rpb_a;
         if (strips > 0x7FFFFFFFll || gy_e > 65535) pl.vec = false;  // outside the launch limits: element-wise path
         pl.wx = wx; pl.rpb_encode = rpb_e; pl.rpb_amax = rpb_a;

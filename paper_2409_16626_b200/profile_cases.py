@@ -5,7 +5,8 @@
 cases: convert_f32 (FP32 4096^2: per-tensor scaled encode + decode), fq_bf16 (BF16 4096x8192 fake-quant, TA and HR,
 fused amax and given scale), encode_modes_f32 (FP32 2^25 log-uniform, every rounding mode), gemm (HiF8 GEMM
 4096 x 7168 x 4096, fused and decode-once paths), gemm_forms (same size, decode-once path, the four operand layouts:
-forward, dgrad form, wgrad form with FP32 accumulation, both transposed).  Inputs are seeded device-side random tensors.
+forward, dgrad form, wgrad form with FP32 accumulation, both transposed), channel_bf16 (per-channel scaled encode of a
+BF16 8192 x 14336 weight, channel = column and channel = row, plus the overflow check of the same tensor).  Inputs are seeded device-side random tensors.
 """
 import sys
 
@@ -71,6 +72,17 @@ def main():
             H.hif8_gemm_ex(A, K, 0, W, K, 1, Cb, N, H.BF16, M, N, K, None, None, None, 0, gws, big)
             H.hif8_gemm_ex(A, M, 1, W, N, 0, Cf, N, H.F32, M, N, K, None, None, None, 1, gws, big)
             H.hif8_gemm_ex(A, M, 1, W, K, 1, Cb, N, H.BF16, M, N, K, None, None, None, 0, gws, big)
+    elif case == "channel_bf16":
+        K, N = 8192, 14336
+        w = (torch.randn(K, N, generator=g, device="cuda") * 0.02).to(torch.bfloat16)
+        q = torch.empty(K * N, dtype=torch.uint8, device="cuda")
+        amax = torch.empty(N, dtype=torch.float32, device="cuda")
+        se = torch.empty(N, dtype=torch.int32, device="cuda")
+        flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+        for r in range(reps):
+            H.hif8_channel_amax_scale_encode(w, H.BF16, q, K, N, 1, 14, H.RND_TA, 0, 0, None, amax, se)
+            H.hif8_channel_amax_scale_encode(w, H.BF16, q, N, K, 0, 14, H.RND_TA, 0, 0, None, amax, se)
+            H.hif8_check_finite(w, H.BF16, K * N, flag)
     else:
         raise SystemExit(f"unknown case {case}")
     torch.cuda.synchronize()
