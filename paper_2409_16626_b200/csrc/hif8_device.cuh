@@ -60,6 +60,23 @@ __host__ __device__ constexpr uint8_t ta_entry(uint32_t idx)
     return (uint8_t)(sign | pack_magnitude(E, M));  // E = 15, M = 1 is the Inf pattern by construction
 }
 
+// Truncating companion of ta_entry, for patterns that a threshold-based rounding has already rounded: the mantissa bits
+// beyond the binade's width are ignored instead of rounded.  Two binades below the format's range keep the meaning the
+// threshold modes give them after their own carry trick: 2^-23 stands for "reached the threshold" (-> 2^-22), anything
+// smaller for zero.
+__host__ __device__ constexpr uint8_t trunc_entry(uint32_t idx)
+{
+    uint32_t sign = (idx >> 12) << 7;
+    int e = (int)((idx >> 4) & 0xFF);
+    uint32_t m4 = idx & 0xF;
+    if (e == 255) return m4 ? (uint8_t)0x80 : (uint8_t)(sign | 0x6F);
+    int E = e - 127;
+    if (E >= 16) return (uint8_t)(sign | 0x6F);
+    if (E <= -24) return 0;
+    if (E == -23) return (uint8_t)(sign | 0x01);
+    return (uint8_t)(sign | pack_magnitude(E, m4 >> (4 - mant_width(E))));  // E = 15, M = 1 is the Inf pattern by construction
+}
+
 struct TaTable { uint8_t v[8192]; };
 constexpr TaTable make_ta_table()
 {
@@ -68,6 +85,13 @@ constexpr TaTable make_ta_table()
     return t;
 }
 __device__ const TaTable g_ta_table = make_ta_table();
+constexpr TaTable make_trunc_table()
+{
+    TaTable t{};
+    for (uint32_t i = 0; i < 8192; i++) t.v[i] = trunc_entry(i);
+    return t;
+}
+__device__ const TaTable g_trunc_table = make_trunc_table();
 
 // value of one byte as binary32 bits (Eq. 1 / Eq. 2 / specials)
 __device__ __forceinline__ uint32_t decode_bits_f32(uint32_t c)
@@ -186,13 +210,21 @@ template <int DT> __device__ __forceinline__ uint32_t to_bits(float v)
 // ------------------------------------------------------------------------------------------------
 // One element: scaled value -> HiF8 byte
 // ------------------------------------------------------------------------------------------------
-// Per-exponent entry of the rounding table (indexed by the biased exponent of the scaled magnitude):
-//   bits 0-4   number of discarded mantissa bits (23 - width); 0: nothing to round (overflow, Inf, NaN)
-//   bits 8-12  left shift that aligns an N-bit threshold complement with the top of the discarded field
-//   bit  7     this binade rounds stochastically (the complement comes from the source bits)
-//   bits 16-31 otherwise: the constant to shift instead (half of 2^N for round-half-away binades, 0 for none)
-constexpr uint32_t kThrStochastic = 0x80u;
-
+// Rounding tables, indexed by the biased exponent of the scaled value: thr[i] = A, thr[256 + i] = B.
+//  * TE / SR tables hold only B = sh, the number of discarded mantissa bits (23 - width; 0: nothing to round).
+//  * Hybrid / simplified stochastic rounding is one multiply-add on the bit pattern, t' = t + B + A * v, whose carry out
+//    of the discarded field rounds up (also across binade and width boundaries); the discarded bits of the old binade are
+//    cleared (mask ~0 << sh, with sh kept in spare bits of B: bits 27-31 for FP32 sources, bits 0-4 for 16-bit sources,
+//    whose widened patterns have zeros there) and the code is read from the truncating table.
+//       FP32 sources   v = 2^14 - max(T14, 1);  stochastic binade: A = 2^(sh-14), B = 0;  round-half-away binade: A = 0, B = 2^(sh-1)
+//       16-bit sources v = source LSB (T2 = 2 v + 1, complement 3 - 2 v);  stochastic: A = -2 * 2^(sh-2), B = 3 * 2^(sh-2);
+//                      round-half-away: A = 0, B = 2^(sh-1)
+//    Below 2^-22 (result 0 or 2^-22, F = |y| / 2^-22):
+//       FP32: the element is first moved into the binade of 2^-24 (see encode_one), whose entry rounds it like a
+//             0-bit-mantissa binade: no carry leaves 2^-24 (-> 0), a carry gives 2^-23 (-> 2^-22 in the truncating table).
+//       16-bit: only the binades of 2^-23 and 2^-24 can reach the threshold; their entries add the complement at the top
+//             of the pattern and step the exponent down by one / two, which leaves 2^-23 or 2^-22 when the threshold is
+//             reached and something below 2^-23 when not.
 template <int MODE, int SRC>
 __device__ __forceinline__ uint32_t encode_one(float x, uint32_t raw, float scale, const uint8_t* s_ta,
                                                const uint32_t* s_thr, uint32_t word)
@@ -201,24 +233,28 @@ __device__ __forceinline__ uint32_t encode_one(float x, uint32_t raw, float scal
     uint32_t t = __float_as_uint(y);
     if (MODE == HIF8_RND_TA) return s_ta[t >> 19];
 
+    if (MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR) {  // s_ta is the truncating table here
+        if (SRC == HIF8_F32) {
+            // below 2^-22: |y| / 4 + 2^-24 with truncation puts floor(F 2^23) into the mantissa of a value in the binade
+            // of 2^-24 (sign kept)
+            const float z = __fmaf_rz(y, 0.25f, __uint_as_float((t & 0x80000000u) | 0x33800000u));
+            const uint32_t u = fabsf(y) < 2.384185791015625e-07f ? __float_as_uint(z) : t;
+            const uint32_t i = (u >> 23) & 0xFFu;  // without the sign: values of either sign share the entry (and its bank)
+            const uint32_t v = 0x4000u - max(raw & 0x3FFFu, 1u);  // SR14: 2^14 - max(T14, 1)
+            const uint32_t B = s_thr[256 + i];                    // constant in bits 0-26, sh in bits 27-31
+            return s_ta[((u + (B & 0x07FFFFFFu) + s_thr[i] * v) & (0xFFFFFFFFu << (B >> 27))) >> 19];
+        } else {
+            const uint32_t i = (t >> 23) & 0xFFu;
+            const uint32_t B = s_thr[256 + i];                    // sh in bits 0-4, below anything a 16-bit source sets
+            return s_ta[((t + B + s_thr[i] * (raw & 1u)) & (0xFFFFFFFFu << (B & 31u))) >> 19];  // SR2: complement 3 - 2 LSB
+        }
+    }
+
     const bool sub = (t & 0x7FFFFFFFu) < 0x34800000u;  // |y| < 2^-22 (zero included): result is 0 or 2^-22
     // Below 2^-22 the kept bits are zero and the fraction is F = |y| / 2^-22.  Adding 2^-22 with truncation puts
     // floor(F 2^23) into the mantissa field of a value in the binade of 2^-22, so the common code rounds it like a
     // 0-bit-mantissa binade (result 2^-22 or 2^-21); it is moved down again afterwards.
     const uint32_t tz = __float_as_uint(__fadd_rz(fabsf(y), 2.384185791015625e-07f));
-
-    if (MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR) {
-        // hybrid / simplified stochastic rounding: the carry of (magnitude + (2^N - T) << k) does the rounding
-        const uint32_t u = sub ? tz : (t & 0x7FFFFFFFu);
-        const uint32_t ent = s_thr[u >> 23];
-        const uint32_t d_ssr = (SRC == HIF8_F32) ? 0x4000u - max(raw & 0x3FFFu, 1u)   // SR14: 2^14 - max(T14, 1)
-                                                 : 3u - 2u * (raw & 1u);               // SR2:  4 - {source LSB, 1}
-        const uint32_t d = (ent & kThrStochastic) ? d_ssr : (ent >> 16);
-        uint32_t tr = (u + (d << ((ent >> 8) & 31u))) & (0xFFFFFFFFu << (ent & 31u));
-        // below 2^-22: two binades down, so that 2^-21 packs as 2^-22 and 2^-22 as the single zero
-        tr -= sub ? 0x01000000u : 0u;
-        return s_ta[(tr >> 19) | ((t >> 19) & 0x1000u)];
-    }
 
     // TE and standard SR
     constexpr int kSrBits = (SRC == HIF8_F32) ? 24 : 16;
@@ -229,7 +265,7 @@ __device__ __forceinline__ uint32_t encode_one(float x, uint32_t raw, float scal
         return f24 >= max(word >> 8, 1u) ? (sign7 | 0x01u) : 0u;
     }
     t = sub ? (tz | (t & 0x80000000u)) : t;
-    const uint32_t sh = s_thr[(t >> 23) & 0xFFu] & 31u;  // discarded mantissa bits (23 - width); 0: nothing to round
+    const uint32_t sh = s_thr[256 + ((t >> 23) & 0xFFu)] & 31u;  // discarded mantissa bits (23 - width); 0: nothing to round
     const uint32_t s = sh ? sh : 23u;
     uint32_t inc;
     if (MODE == HIF8_RND_TE) {
@@ -261,7 +297,7 @@ __device__ __forceinline__ uint32_t encode_one(float x, uint32_t raw, float scal
 // ------------------------------------------------------------------------------------------------
 struct __align__(16) SmemTables {
     uint8_t ta[8192];
-    uint32_t thr[256];
+    uint32_t thr[512];
     float dec[256];
 };
 
@@ -272,7 +308,7 @@ __device__ __forceinline__ void setup_tables(SmemTables& s, unsigned flags)
         // Only binades 2^-24 .. 2^16 differ from their neighbours: those 41 x 16 entries per sign come from the
         // compile-time table (1.3 KiB of global reads per block); everything below is zero, everything above is
         // Inf (or NaN in the all-ones exponent), written straight into shared memory.
-        const uint4* g = reinterpret_cast<const uint4*>(g_ta_table.v);
+        const uint4* g = reinterpret_cast<const uint4*>((MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR) ? g_trunc_table.v : g_ta_table.v);
         uint4* d = reinterpret_cast<uint4*>(s.ta);
         for (int i = threadIdx.x; i < 512; i += kThreads) {
             const uint32_t e = i & 255, inf = ((uint32_t)(i >> 8) << 7) | 0x6Fu;
@@ -302,15 +338,25 @@ __device__ __forceinline__ void setup_tables(SmemTables& s, unsigned flags)
     }
     if (NEED_SH) {
         const int e = threadIdx.x, E = e - 127;  // kThreads == 256 biased exponents
-        uint32_t ent = 0;
+        constexpr bool kF32 = SRC == HIF8_F32;
+        constexpr bool kThreshold = MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR;
+        uint32_t A = 0, B = 0;
         if (E < 16 && E >= -22) {
-            constexpr uint32_t N = (SRC == HIF8_F32) ? 14u : 2u;  // threshold bits of the simplified SR
             const uint32_t sh = 23u - (uint32_t)mant_width(E);
-            ent = sh | ((sh - N) << 8);
-            if (MODE == HIF8_RND_SSR || (MODE == HIF8_RND_HR && (E <= -4 || E >= 4))) ent |= kThrStochastic;
-            else ent |= (1u << (N - 1)) << 16;  // round half away = threshold one half
+            if (!kThreshold) B = sh;  // TE / SR: only the width is read
+            else if (MODE == HIF8_RND_SSR || E <= -4 || E >= 4) {
+                if (kF32) A = 1u << (sh - 14u);
+                else { A = 0u - (2u << (sh - 2u)); B = 3u << (sh - 2u); }
+                B |= kF32 ? sh << 27 : sh;
+            } else B = (1u << (sh - 1u)) | (kF32 ? sh << 27 : sh);  // Eq. 3: round half away in the binades |E| < 4
+        } else if (kThreshold && kF32 && E == -24) {
+            A = 1u << 9; B = 23u << 27;  // where encode_one parks FP32 elements below 2^-22
+        } else if (kThreshold && !kF32 && (E == -23 || E == -24)) {
+            const uint32_t j = (uint32_t)(-23 - E);  // complement << (22 + j), then j + 1 binades down
+            A = 0u - (2u << (22u + j));
+            B = ((3u << (22u + j)) - ((j + 1u) << 23)) | 23u;
         }
-        s.thr[e] = ent;
+        s.thr[e] = A; s.thr[256 + e] = B;
     }
     if (NEED_DEC) s.dec[threadIdx.x] = __uint_as_float(decode_bits_f32(threadIdx.x));
     __syncthreads();

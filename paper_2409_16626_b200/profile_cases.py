@@ -3,7 +3,7 @@
     python -m paper_2409_16626_b200.profile_cases <case> [repeats]
 
 cases: convert_f32 (FP32 4096^2: per-tensor scaled encode + decode), fq_bf16 (BF16 4096x8192 fake-quant, TA and HR,
-fused amax and given scale), encode_modes_f32 (FP32 2^25 log-uniform, every rounding mode), gemm (HiF8 GEMM
+fused amax and given scale), encode_modes_f32 / encode_modes_bf16 (2^25 log-uniform values, every rounding mode), gemm (HiF8 GEMM
 4096 x 7168 x 4096, fused and decode-once paths), gemm_forms (same size, decode-once path, the four operand layouts:
 forward, dgrad form, wgrad form with FP32 accumulation, both transposed), channel_bf16 (per-channel scaled encode of a
 BF16 8192 x 14336 weight, channel = column and channel = row, plus the overflow check of the same tensor).  Inputs are seeded device-side random tensors.
@@ -47,6 +47,15 @@ def main():
         for r in range(reps):
             for mode in (H.RND_TA, H.RND_HR, H.RND_SSR, H.RND_TE, H.RND_SR):
                 H.hif8_encode(bits, H.F32, codes, n, 0, mode, 0, 5)
+    elif case == "encode_modes_bf16":
+        n = 1 << 25
+        e = torch.randint(-40, 20, (n,), generator=g, device="cuda", dtype=torch.int32) + 127
+        m = torch.randint(0, 1 << 7, (n,), generator=g, device="cuda", dtype=torch.int32)
+        bits = ((e << 7) | m).to(torch.int16)
+        codes = torch.empty(n, dtype=torch.uint8, device="cuda")
+        for r in range(reps):
+            for mode in (H.RND_TA, H.RND_HR, H.RND_SSR, H.RND_TE, H.RND_SR):
+                H.hif8_encode(bits, H.BF16, codes, n, 0, mode, 0, 5)
     elif case == "gemm":
         M, N, K = 4096, 7168, 4096
         A = torch.randint(0, 256, (M, K), dtype=torch.uint8, device="cuda", generator=g)
