@@ -181,6 +181,14 @@ def extra_results(H, torch, hbm_peak, peak_kind):
         fq[name] = {"ms": ms, "GBps": 6 * n / ms / 1e6, "frac": 6 * n / ms / 1e6 / hbm_peak}
     ms = timed(lambda r: H.hif8_fake_quant(xs[r & 1], ys[r & 1], H.BF16, n, 0, 3, H.RND_TA, 0, 0), 20)
     fq["TA_given_scale"] = {"ms": ms, "GBps": 4 * n / ms / 1e6, "frac": 4 * n / ms / 1e6 / hbm_peak}
+    # the same tensors to HiF8 bytes with a given scale (2 B read + 1 B written): forward (TA) and backward (HR) rounding
+    cq = torch.empty(n, dtype=torch.uint8, device="cuda")
+    enc = {}
+    for name, mode in (("TA", H.RND_TA), ("HR", H.RND_HR)):
+        ms = timed(lambda r: H.hif8_encode(xs[r & 1], H.BF16, cq, n, 3, mode), 20)
+        enc[name] = {"ms": ms, "GBps": 3 * n / ms / 1e6, "frac": 3 * n / ms / 1e6 / hbm_peak}
+    out["encode_bf16_8192x8192"] = {"bytes_per_element": 3, "modes": enc, "peak": hbm_peak, "peak_kind": f"of {peak_kind}"}
+    del cq
     out["fake_quant_bf16_8192x8192"] = {"bytes_per_element": {"fused_amax": 6, "given_scale": 4}, "modes": fq,
                                         "peak": hbm_peak, "peak_kind": f"of {peak_kind}"}
     del xs, ys
