@@ -162,12 +162,13 @@ __device__ __forceinline__ void cluster_sync_all()
 {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-// TMA tile load of a CTA pair: data into this CTA's shared memory, completion on a barrier that may live in the peer
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar_cluster)
+// TMA tile load of a CTA pair: data into this CTA's shared memory, completion on a barrier that may live in the peer.
+// The tile comes from matrix c2 of a stack of matrices (three-dimensional tensor map, box one matrix deep).
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar_cluster)
 {
     asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(c0), "r"(c1) : "memory");
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar)  // arrives on `bar` in both CTAs of the pair
 {
@@ -533,7 +534,10 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + SmemLayout2::tmem_slot);
     const int num_kb = (p.K + BK - 1) / BK;
     const int tiles_m2 = (p.M + 2 * BM - 1) / (2 * BM), tiles_n2 = p.tiles_n;
-    const int tiles = tiles_m2 * tiles_n2, pairs = gridDim.x >> 1, pair_id = blockIdx.x >> 1;
+    // a batch of n x n products (A variant ia, W variant iw) is one list of tiles: product b = ia * n + iw owns tiles
+    // [b * tiles_one, (b + 1) * tiles_one)
+    const int tiles_one = tiles_m2 * tiles_n2, nb = p.batch_n > 0 ? p.batch_n : 1;
+    const int tiles = tiles_one * nb * nb, pairs = gridDim.x >> 1, pair_id = blockIdx.x >> 1;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages2; s++) { mbar_init(bar_full(s), 1); mbar_init(bar_empty(s), 1); }
@@ -558,7 +562,8 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
             bool ok = true;
             for (int t = pair_id; t < tiles && ok; t += pairs) {
                 int tile_m, tile_n;
-                tile_coords(t, tiles_m2, tiles_n2, tile_m, tile_n);
+                const int b = t / tiles_one, ia = b / nb, iw = b - ia * nb;
+                tile_coords(t - b * tiles_one, tiles_m2, tiles_n2, tile_m, tile_n);
                 const int m0 = tile_m * 2 * BM + (int)rank * BM, n0 = tile_n * BN + (int)rank * (BN / 2);
                 for (int kb = 0; kb < num_kb; kb++, it++) {
                     const int s = (int)(it % kStages2);
@@ -570,13 +575,13 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                     if (leader) mbar_arrive_expect_tx(bar_full(s), 2 * kStageBytes2);  // bytes of both CTAs
                     if (A_IS_KM) {
 #pragma unroll
-                        for (int c = 0; c < BM / 64; c++) tma_load_2d_pair(dst_a + c * 8192, &map_a, m0 + c * 64, kb * BK, full);
-                    } else tma_load_2d_pair(dst_a, &map_a, kb * BK, m0, full);
-                    if (W_IS_NK) tma_load_2d_pair(dst_b, &map_w, kb * BK, n0, full);
+                        for (int c = 0; c < BM / 64; c++) tma_load_3d_pair(dst_a + c * 8192, &map_a, m0 + c * 64, kb * BK, ia, full);
+                    } else tma_load_3d_pair(dst_a, &map_a, kb * BK, m0, ia, full);
+                    if (W_IS_NK) tma_load_3d_pair(dst_b, &map_w, kb * BK, n0, iw, full);
                     else {
 #pragma unroll
                         for (int c = 0; c < BN / 2 / 64; c++)
-                            tma_load_2d_pair(dst_b + c * 8192, &map_w, n0 + c * 64, kb * BK, full);
+                            tma_load_3d_pair(dst_b + c * 8192, &map_w, n0 + c * 64, kb * BK, iw, full);
                     }
                     issued = it + 1;
                 }
@@ -623,19 +628,27 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
             }
         }
     } else if (warp < kEpiWarps) {
-        const int sa = p.d_sa ? *p.d_sa : 0;
-        const int sdesc = p.d_sw_channel ? 0 : -(sa + (p.d_sw ? *p.d_sw : 0));
-        const int s1 = sdesc / 2, s2 = sdesc - s1;
-        const float f1 = __uint_as_float((uint32_t)(s1 + 127) << 23), f2 = __uint_as_float((uint32_t)(s2 + 127) << 23);
-        int local = 0;
-        double err_acc = 0.0;  // squared-error variant: this thread's share over all its tiles
+        int local = 0, b_held = -1;
+        double err_acc = 0.0;  // squared-error variant: this thread's share of product b_held
         const bool ref_vec = !(reinterpret_cast<uintptr_t>(p.err_ref) & 15) && !(p.ld_ref & 3);
+        auto flush_error = [&]() {  // all lanes of the warp
+            for (int off = 16; off > 0; off >>= 1) err_acc += __shfl_xor_sync(0xFFFFFFFFu, err_acc, off);
+            if (lane == 0 && err_acc != 0.0 && b_held >= 0) atomicAdd(p.err_sum + b_held, err_acc);
+            err_acc = 0.0;
+        };
         for (int t = pair_id; t < tiles; t += pairs, local++) {
             const int acc = local & 1, use = local >> 1;
             if (!mbar_wait(bar_acc_full(acc), (uint32_t)(use & 1), abort_flag, p.status, 24)) break;
             tc_fence_after();
             int tile_m, tile_n;
-            tile_coords(t, tiles_m2, tiles_n2, tile_m, tile_n);
+            const int b = t / tiles_one, ia = b / nb, iw = b - ia * nb;
+            if (p.err_sum && b != b_held) { flush_error(); b_held = b; }
+            // exponents of this product (in a batch: entry ia / iw of the two device arrays)
+            const int sa = p.d_sa ? p.d_sa[ia] : 0;
+            const int sdesc = p.d_sw_channel ? 0 : -(sa + (p.d_sw ? p.d_sw[iw] : 0));
+            const int s1 = sdesc / 2, s2 = sdesc - s1;
+            const float f1 = __uint_as_float((uint32_t)(s1 + 127) << 23), f2 = __uint_as_float((uint32_t)(s2 + 127) << 23);
+            tile_coords(t - b * tiles_one, tiles_m2, tiles_n2, tile_m, tile_n);
             const int row = tile_m * 2 * BM + (int)rank * BM + warp * 32 + lane, n0 = tile_n * BN;
 #pragma unroll 1
             for (int c = 0; c < BN; c += 32) {
@@ -671,10 +684,7 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(bar_acc_empty(acc), 0));  // tell the leader: accumulator drained
         }
-        if (p.err_sum) {
-            for (int off = 16; off > 0; off >>= 1) err_acc += __shfl_xor_sync(0xFFFFFFFFu, err_acc, off);
-            if (lane == 0 && err_acc != 0.0) atomicAdd(p.err_sum, err_acc);
-        }
+        if (p.err_sum) flush_error();
     }
 
     // nobody leaves while the other CTA may still read this CTA's shared memory or signal its barriers
@@ -740,6 +750,20 @@ bool make_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t rows, 
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// BF16 stack of `count` matrices [rows, inner], `stack_stride` elements apart (box: one matrix deep)
+bool make_map3(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t rows, uint64_t count, uint64_t stack_stride,
+               uint32_t box_inner, uint32_t box_rows)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {inner, rows, count};
+    cuuint64_t strides[2] = {inner * 2u, (count > 1 ? stack_stride : inner * rows) * 2u};
+    cuuint32_t box[3] = {box_inner, box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // one-time kernel attributes (dynamic shared memory) and the SM count of the device
 bool gemm_kernels_ready(int dev, int* sm_count_out)
 {
@@ -765,23 +789,26 @@ constexpr size_t kGemmWorkspaceBytes = 256;
 
 }  // namespace
 
-int launch_bf16_pair_gemm(const void* a_bf, int a_is_km, const void* w_bf, int w_is_nk, GemmParams p, cudaStream_t st)
+int launch_bf16_pair_gemm(const void* a_bf, int a_is_km, const void* w_bf, int w_is_nk, GemmParams p, cudaStream_t st,
+                          long long a_stack_stride, long long w_stack_stride)
 {
     int dev = 0, sm_count = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || !gemm_kernels_ready(dev, &sm_count)) return HIF8_ERR_CUDA;
     const int M = p.M, N = p.N, K = p.K;
+    const uint64_t nb = p.batch_n > 0 ? (uint64_t)p.batch_n : 1;
     p.tiles_m = (M + BM - 1) / BM;
     p.tiles_n = (N + BN - 1) / BN;
-    const long long tiles2 = (long long)((M + 2 * BM - 1) / (2 * BM)) * p.tiles_n;
+    const long long tiles2 = (long long)((M + 2 * BM - 1) / (2 * BM)) * p.tiles_n * (long long)(nb * nb);
     if (M <= 0 || N <= 0 || K <= 0 || tiles2 > 0x3FFFFFFF) return HIF8_ERR_SHAPE;
+    if (nb > 1 && ((a_stack_stride & 7) || (w_stack_stride & 7))) return HIF8_ERR_ALIGN;  // 16-byte strides
     CUtensorMap ma, mw;
     // A boxes: this CTA's 128 rows of [M,K], or two boxes of 64 columns of [K,M]
-    const bool oka = a_is_km ? make_map(&ma, a_bf, (uint64_t)M, (uint64_t)K, (uint64_t)M, 64, BK, true)
-                             : make_map(&ma, a_bf, (uint64_t)K, (uint64_t)M, (uint64_t)K, BK, BM, true);
+    const bool oka = a_is_km ? make_map3(&ma, a_bf, (uint64_t)M, (uint64_t)K, nb, (uint64_t)a_stack_stride, 64, BK)
+                             : make_map3(&ma, a_bf, (uint64_t)K, (uint64_t)M, nb, (uint64_t)a_stack_stride, BK, BM);
     if (!oka) return HIF8_ERR_CUDA;
     // W boxes are one CTA's half of the 256-column tile: 128 rows of [N,K], or two boxes of 64 columns of [K,N]
-    const bool okw = w_is_nk ? make_map(&mw, w_bf, (uint64_t)K, (uint64_t)N, (uint64_t)K, BK, BN / 2, true)
-                             : make_map(&mw, w_bf, (uint64_t)N, (uint64_t)K, (uint64_t)N, 64, BK, true);
+    const bool okw = w_is_nk ? make_map3(&mw, w_bf, (uint64_t)K, (uint64_t)N, nb, (uint64_t)w_stack_stride, BK, BN / 2)
+                             : make_map3(&mw, w_bf, (uint64_t)N, (uint64_t)K, nb, (uint64_t)w_stack_stride, 64, BK);
     if (!okw) return HIF8_ERR_CUDA;
     const int pairs = (int)(tiles2 < sm_count / 2 ? tiles2 : sm_count / 2);
     cudaLaunchConfig_t cfg{};

@@ -19,11 +19,16 @@ struct GemmParams {
     const float* err_ref;
     long long ld_ref;
     double* err_sum;
+    // batch_n = n > 0: n x n products in one launch, A variant ia with W variant iw for product ia * n + iw; d_sa / d_sw
+    // are then arrays of n exponents and err_sum an array of n * n sums
+    int batch_n;
 };
 
 // C (or the squared error) from operands that are already BF16 in device memory: a_bf [M,K] or (a_is_km) [K,M], w_bf [K,N] or (w_is_nk) [N,K],
 // both contiguous.  Fills in the tile counts of `p`; p.status must point at a zeroed device int.
-int launch_bf16_pair_gemm(const void* a_bf, int a_is_km, const void* w_bf, int w_is_nk, GemmParams p, cudaStream_t st);
+// In a batch the variants of an operand are `*_stack_stride` elements apart (multiples of 8).
+int launch_bf16_pair_gemm(const void* a_bf, int a_is_km, const void* w_bf, int w_is_nk, GemmParams p, cudaStream_t st,
+                          long long a_stack_stride = 0, long long w_stack_stride = 0);
 
 // SM count of the current device; HIF8_ERR_CUDA unless it is a compute-capability-10.0 device
 int checked_device(int* sms);

@@ -3,8 +3,8 @@
 // measure the mean squared error against the layer's high-precision output; keep the pair with the smallest error.
 //
 // Each operand is cast once per exponent (hif8_encode into a scratch byte buffer) and expanded once to BF16
-// (hif8_decode, exact), so the n*n multiplications read ready BF16 operands.  Each pair is one launch of the
-// tensor-core kernel whose epilogue restores the scale (2^-(Ea+Ew), device-resident exponents) and, instead of storing
+// (hif8_decode, exact), so the n*n multiplications read ready BF16 operands.  All pairs are one launch of the
+// tensor-core kernel (their tiles form one list for the persistent CTA pairs), whose epilogue restores the scale (2^-(Ea+Ew), device-resident exponents) and, instead of storing
 // the product, adds the squared differences to the layer's output into one double per pair; a last one-block kernel
 // turns the sums into the MSE table and takes the argmin.  Nothing returns to the host in between.
 #include <cuda_runtime.h>
@@ -105,13 +105,15 @@ extern "C" int hif8_pts_search(const void* A, const void* W, int dtype, int w_is
     p.M = M; p.N = N; p.K = K;
     p.status = &ctl->status;
     p.err_ref = O_ref; p.ld_ref = ldo;
-    for (int ia = 0; ia < n_exp; ia++)
-        for (int iw = 0; iw < n_exp; iw++) {  // "MatMul & Restore" and "Quantization Error" in one launch
-            p.d_sa = &ctl->exps[ia]; p.d_sw = &ctl->exps[iw];
-            p.err_sum = &ctl->sums[ia * n_exp + iw];
-            const int rc = launch_bf16_pair_gemm(a_bf + align256(mk * 2) * ia, 0, w_bf + align256(kn * 2) * iw, w_is_nk, p, st);
-            if (rc != HIF8_OK) return rc;
-        }
+    // "MatMul & Restore" and "Quantization Error" of all n * n pairs in one launch: the tiles of every product form one
+    // list that the persistent CTA pairs walk through, so only the very last wave of the whole search is ragged
+    p.d_sa = ctl->exps; p.d_sw = ctl->exps;
+    p.err_sum = ctl->sums;
+    p.batch_n = n_exp;
+    {
+        const int rc = launch_bf16_pair_gemm(a_bf, 0, w_bf, w_is_nk, p, st, (long long)(align256(mk * 2) / 2), (long long)(align256(kn * 2) / 2));
+        if (rc != HIF8_OK) return rc;
+    }
     pts_finish_kernel<<<1, 32, 0, st>>>(ctl, e_min, n_exp, 1.0 / ((double)M * (double)N), d_err, d_best);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
