@@ -176,3 +176,43 @@ def test_backward_pass_of_a_linear_layer():
         S_acc += S.reshape(K, N)
     got = dW.cpu().numpy().astype(np.float64)
     assert np.all(np.abs(got - dW_ref) <= 1e-5 * S_acc + 2.0 ** -23 * np.abs(dW_ref))
+
+
+@pytest.mark.parametrize("shape", [(200, 72, 16), (56, 264, 80), (129, 8, 1040)])
+@pytest.mark.parametrize("w_is_nk", [0, 1])
+def test_gemm_ex_transposed_a_ragged_shapes_and_padded_leading_dimensions(shape, w_is_nk):
+    # A stored [K, M] with lda > M, M not a multiple of anything convenient, tiny K / N: the fused kernel (operands not
+    # contiguous), out-of-range parts of the TMA boxes must read as zero
+    M, N, K = shape
+    lda = (M + 15) // 16 * 16 + 16
+    ldw = ((K if w_is_nk else N) + 15) // 16 * 16 + 16
+    Amk, Wkn = codes((M, K), 21), codes((K, N), 22)
+    Aq = np.full((K, lda), 0x7B, dtype=np.uint8)            # padding holds a large finite value: it must never be read in
+    Aq[:, :M] = Amk.T
+    Wsrc = Wkn.T if w_is_nk else Wkn
+    Wq = np.full((Wsrc.shape[0], ldw), 0x7B, dtype=np.uint8)
+    Wq[:, :Wsrc.shape[1]] = Wsrc
+    ldc = (N + 7) // 8 * 8
+    C = torch.full((M, ldc), float("nan"), dtype=torch.float32, device="cuda")
+    ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+    H.hif8_gemm_ex(to_dev(Aq), lda, 1, to_dev(Wq), ldw, w_is_nk, C, ldc, H.F32, M, N, K, None, None, None, 0, ws, 256)
+    assert H.hif8_gemm_status(ws) == 0
+    out = C.cpu().numpy().astype(np.float64)
+    assert np.all(np.isnan(out[:, N:]))
+    rows, cols = np.divmod(np.arange(M * N), N)
+    P, S = O.gemm_entries_ex(np.ascontiguousarray(Amk.T), 1, np.ascontiguousarray(Wsrc), w_is_nk, 0, 0, rows, cols)
+    assert np.all(np.abs(out[:, :N].ravel() - P) <= 1e-5 * S)
+
+
+def test_gemm_ex_argument_checks():
+    A = torch.zeros(64 * 64, dtype=torch.uint8, device="cuda")
+    C = torch.zeros(64 * 64, dtype=torch.float32, device="cuda")
+    ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+    ok = dict(workspace=ws, workspace_bytes=256, check=False)
+    assert H.hif8_gemm_ex(A, 64, 1, A, 64, 0, C, 64, H.F32, 64, 64, 64, **ok) == 0
+    assert H.hif8_gemm_ex(A, 48, 1, A, 64, 0, C, 64, H.F32, 64, 64, 64, **ok) == 6    # lda < M for a [K,M] operand
+    assert H.hif8_gemm_ex(A, 64, 1, A, 64, 0, C, 64, H.F32, 64, 64, 24, **ok) == 6    # K not a multiple of 16
+    assert H.hif8_gemm_ex(A, 72, 1, A, 64, 0, C, 64, H.F32, 64, 64, 64, **ok) == 7    # lda not a multiple of 16
+    assert H.hif8_gemm_ex(A, 64, 1, A, 64, 0, C, 64, 5, 64, 64, 64, **ok) == 2
+    assert H.hif8_gemm_ex(A, 64, 1, A, 64, 0, C, 64, H.F32, 64, 64, 64, workspace=None, workspace_bytes=0, check=False) == 8
+    assert H.hif8_gemm_ex(A, 64, 1, A, 64, 0, C, 64, H.F32, 0, 64, 64, **ok) == 0     # empty output
