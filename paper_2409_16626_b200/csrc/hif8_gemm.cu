@@ -515,7 +515,7 @@ struct SmemLayout2 {
 };
 constexpr uint32_t kSmemBytes2 = SmemLayout2::total + 1024;
 
-template <bool A_IS_KM, bool W_IS_NK>
+template <bool W_IS_NK>
 __global__ void __launch_bounds__(kThreadsP, 1)
 bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const GemmParams p)
 {
@@ -573,10 +573,7 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                     const uint32_t dst_a = base + s * kStageBytes2, dst_b = dst_a + kABfBytes;
                     const uint32_t full = map_to_cta(bar_full(s), 0);
                     if (leader) mbar_arrive_expect_tx(bar_full(s), 2 * kStageBytes2);  // bytes of both CTAs
-                    if (A_IS_KM) {
-#pragma unroll
-                        for (int c = 0; c < BM / 64; c++) tma_load_3d_pair(dst_a + c * 8192, &map_a, m0 + c * 64, kb * BK, ia, full);
-                    } else tma_load_3d_pair(dst_a, &map_a, kb * BK, m0, ia, full);
+                    tma_load_3d_pair(dst_a, &map_a, kb * BK, m0, ia, full);
                     if (W_IS_NK) tma_load_3d_pair(dst_b, &map_w, kb * BK, n0, iw, full);
                     else {
 #pragma unroll
@@ -597,7 +594,7 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     } else if (warp == kMmaWarp) {
         if (lane == 0 && leader) {
             // M = 256 over the pair, N = 256
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_IS_KM ? 1u : 0u) << 15) | ((W_IS_NK ? 0u : 1u) << 16) |
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((W_IS_NK ? 0u : 1u) << 16) |
                                    ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
             long long it = 0;
             int local = 0;
@@ -616,8 +613,7 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                     const uint32_t a_addr = base + s * kStageBytes2, b_addr = a_addr + kABfBytes;
 #pragma unroll
                     for (int kk = 0; kk < BK / 16; kk++) {
-                        const uint64_t da = A_IS_KM ? make_smem_desc(a_addr + kk * 2048, 8192, 1024)
-                                                    : make_smem_desc(a_addr + kk * 32, 16, 1024);
+                        const uint64_t da = make_smem_desc(a_addr + kk * 32, 16, 1024);
                         const uint64_t db = W_IS_NK ? make_smem_desc(b_addr + kk * 32, 16, 1024)
                                                     : make_smem_desc(b_addr + kk * 2048, 8192, 1024);
                         tc_mma_bf16_pair(d_tmem, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
@@ -773,12 +769,11 @@ bool gemm_kernels_ready(int dev, int* sm_count_out)
     std::call_once(attr_once, [dev] {
         const void* fused[4] = {(const void*)hif8_gemm_kernel<false, false>, (const void*)hif8_gemm_kernel<false, true>,
                                 (const void*)hif8_gemm_kernel<true, false>, (const void*)hif8_gemm_kernel<true, true>};
-        const void* pair[4] = {(const void*)bf16_gemm_pair_kernel<false, false>, (const void*)bf16_gemm_pair_kernel<false, true>,
-                               (const void*)bf16_gemm_pair_kernel<true, false>, (const void*)bf16_gemm_pair_kernel<true, true>};
-        for (int i = 0; i < 4 && attr_rc == cudaSuccess; i++) {
+        const void* pair[2] = {(const void*)bf16_gemm_pair_kernel<false>, (const void*)bf16_gemm_pair_kernel<true>};
+        for (int i = 0; i < 4 && attr_rc == cudaSuccess; i++)
             attr_rc = cudaFuncSetAttribute(fused[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-            if (attr_rc == cudaSuccess) attr_rc = cudaFuncSetAttribute(pair[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
-        }
+        for (int i = 0; i < 2 && attr_rc == cudaSuccess; i++)
+            attr_rc = cudaFuncSetAttribute(pair[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
         if (attr_rc == cudaSuccess) attr_rc = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
     });
     *sm_count_out = sm_count;
@@ -789,7 +784,7 @@ constexpr size_t kGemmWorkspaceBytes = 256;
 
 }  // namespace
 
-int launch_bf16_pair_gemm(const void* a_bf, int a_is_km, const void* w_bf, int w_is_nk, GemmParams p, cudaStream_t st,
+int launch_bf16_pair_gemm(const void* a_bf, const void* w_bf, int w_is_nk, GemmParams p, cudaStream_t st,
                           long long a_stack_stride, long long w_stack_stride)
 {
     int dev = 0, sm_count = 0;
@@ -802,10 +797,8 @@ int launch_bf16_pair_gemm(const void* a_bf, int a_is_km, const void* w_bf, int w
     if (M <= 0 || N <= 0 || K <= 0 || tiles2 > 0x3FFFFFFF) return HIF8_ERR_SHAPE;
     if (nb > 1 && ((a_stack_stride & 7) || (w_stack_stride & 7))) return HIF8_ERR_ALIGN;  // 16-byte strides
     CUtensorMap ma, mw;
-    // A boxes: this CTA's 128 rows of [M,K], or two boxes of 64 columns of [K,M]
-    const bool oka = a_is_km ? make_map3(&ma, a_bf, (uint64_t)M, (uint64_t)K, nb, (uint64_t)a_stack_stride, 64, BK)
-                             : make_map3(&ma, a_bf, (uint64_t)K, (uint64_t)M, nb, (uint64_t)a_stack_stride, BK, BM);
-    if (!oka) return HIF8_ERR_CUDA;
+    // A boxes: this CTA's 128 rows of [M,K]
+    if (!make_map3(&ma, a_bf, (uint64_t)K, (uint64_t)M, nb, (uint64_t)a_stack_stride, BK, BM)) return HIF8_ERR_CUDA;
     // W boxes are one CTA's half of the 256-column tile: 128 rows of [N,K], or two boxes of 64 columns of [K,N]
     const bool okw = w_is_nk ? make_map3(&mw, w_bf, (uint64_t)K, (uint64_t)N, nb, (uint64_t)w_stack_stride, BK, BN / 2)
                              : make_map3(&mw, w_bf, (uint64_t)N, (uint64_t)K, nb, (uint64_t)w_stack_stride, 64, BK);
@@ -820,11 +813,8 @@ int launch_bf16_pair_gemm(const void* a_bf, int a_is_km, const void* w_bf, int w
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    cudaError_t lrc;
-    if (a_is_km) lrc = w_is_nk ? cudaLaunchKernelEx(&cfg, bf16_gemm_pair_kernel<true, true>, ma, mw, p)
-                               : cudaLaunchKernelEx(&cfg, bf16_gemm_pair_kernel<true, false>, ma, mw, p);
-    else lrc = w_is_nk ? cudaLaunchKernelEx(&cfg, bf16_gemm_pair_kernel<false, true>, ma, mw, p)
-                       : cudaLaunchKernelEx(&cfg, bf16_gemm_pair_kernel<false, false>, ma, mw, p);
+    const cudaError_t lrc = w_is_nk ? cudaLaunchKernelEx(&cfg, bf16_gemm_pair_kernel<true>, ma, mw, p)
+                                    : cudaLaunchKernelEx(&cfg, bf16_gemm_pair_kernel<false>, ma, mw, p);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return (lrc == cudaSuccess && cudaGetLastError() == cudaSuccess) ? HIF8_OK : HIF8_ERR_CUDA;
 }
@@ -887,10 +877,11 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t
     if (contiguous && workspace_bytes >= kGemmWorkspaceBytes + bytes_a + bytes_w && !(reinterpret_cast<uintptr_t>(workspace) & 255)) {
         unsigned char* a_bf = reinterpret_cast<unsigned char*>(workspace) + kGemmWorkspaceBytes;
         unsigned char* w_bf = a_bf + bytes_a;
-        int rc = hif8_decode(Aq, a_bf, HIF8_BF16, (size_t)M * K, 0, stream);
+        // an A given as [K,M] is written as [M,K] while it is expanded: the tensor-core kernel streams a K-major A fastest
+        int rc = a_is_km ? decode_transpose_bf16(Aq, a_bf, K, M, st) : hif8_decode(Aq, a_bf, HIF8_BF16, (size_t)M * K, 0, stream);
         if (rc == HIF8_OK) rc = hif8_decode(Wq, w_bf, HIF8_BF16, (size_t)K * N, 0, stream);
         if (rc != HIF8_OK) return rc;
-        return launch_bf16_pair_gemm(a_bf, a_is_km, w_bf, w_is_nk, p, st);
+        return launch_bf16_pair_gemm(a_bf, w_bf, w_is_nk, p, st);
     }
 
     cudaLaunchConfig_t cfg{};

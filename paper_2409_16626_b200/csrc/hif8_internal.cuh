@@ -2,6 +2,8 @@
 #pragma once
 #include <cuda_runtime.h>
 
+#include <cstdint>
+
 namespace hif8 {
 
 struct GemmParams {
@@ -24,11 +26,15 @@ struct GemmParams {
     int batch_n;
 };
 
-// C (or the squared error) from operands that are already BF16 in device memory: a_bf [M,K] or (a_is_km) [K,M], w_bf [K,N] or (w_is_nk) [N,K],
+// C (or the squared error) from operands that are already BF16 in device memory: a_bf [M,K], w_bf [K,N] or (w_is_nk) [N,K],
 // both contiguous.  Fills in the tile counts of `p`; p.status must point at a zeroed device int.
 // In a batch the variants of an operand are `*_stack_stride` elements apart (multiples of 8).
-int launch_bf16_pair_gemm(const void* a_bf, int a_is_km, const void* w_bf, int w_is_nk, GemmParams p, cudaStream_t st,
+int launch_bf16_pair_gemm(const void* a_bf, const void* w_bf, int w_is_nk, GemmParams p, cudaStream_t st,
                           long long a_stack_stride = 0, long long w_stack_stride = 0);
+
+// dst[c][r] = BF16 value of the HiF8 byte src[r][c]; src [rows, cols] contiguous (rows a multiple of 8, cols of 16), both
+// pointers 16-byte aligned
+int decode_transpose_bf16(const uint8_t* src, void* dst, long long rows, long long cols, cudaStream_t st);
 
 // SM count of the current device; HIF8_ERR_CUDA unless it is a compute-capability-10.0 device
 int checked_device(int* sms);

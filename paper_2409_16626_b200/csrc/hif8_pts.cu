@@ -111,7 +111,7 @@ extern "C" int hif8_pts_search(const void* A, const void* W, int dtype, int w_is
     p.err_sum = ctl->sums;
     p.batch_n = n_exp;
     {
-        const int rc = launch_bf16_pair_gemm(a_bf, 0, w_bf, w_is_nk, p, st, (long long)(align256(mk * 2) / 2), (long long)(align256(kn * 2) / 2));
+        const int rc = launch_bf16_pair_gemm(a_bf, w_bf, w_is_nk, p, st, (long long)(align256(mk * 2) / 2), (long long)(align256(kn * 2) / 2));
         if (rc != HIF8_OK) return rc;
     }
     pts_finish_kernel<<<1, 32, 0, st>>>(ctl, e_min, n_exp, 1.0 / ((double)M * (double)N), d_err, d_best);

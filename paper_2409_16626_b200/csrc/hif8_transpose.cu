@@ -121,6 +121,48 @@ __global__ void __launch_bounds__(kThreads) encode_transpose_scalar_kernel(const
     }
 }
 
+// HiF8 bytes [rows, cols] -> BF16 [cols, rows] (exact).  Used by the GEMM's decode-once path for an A operand given as
+// [K, M]: the tensor-core kernel then always streams a K-major A.  A block stages a 64 x 256 byte tile in shared memory
+// (rows padded by one word: a column walk then touches successive banks), then eight lanes write the 64 values of one
+// output row segment as 128 contiguous bytes.
+constexpr int kDtRows = 64, kDtCols = 256, kDtStride = kDtCols + 4;
+
+__global__ void __launch_bounds__(kThreads) decode_transpose_bf16_kernel(const uint8_t* __restrict__ src, unsigned short* __restrict__ dst,
+                                                                         long long rows, long long cols)
+{
+    __shared__ uint32_t tile[kDtRows * kDtStride / 4];
+    __shared__ unsigned short lut[256];
+    lut[threadIdx.x] = (unsigned short)(decode_bits_f32(threadIdx.x) >> 16);  // every HiF8 value is exact in BF16
+    const long long tiles_c = (cols + kDtCols - 1) / kDtCols, tiles_r = (rows + kDtRows - 1) / kDtRows;
+    const uint8_t* tb = reinterpret_cast<const uint8_t*>(tile);
+    for (long long tix = blockIdx.x; tix < tiles_c * tiles_r; tix += gridDim.x) {
+        const long long tc = tix / tiles_r, tr = tix % tiles_r;
+        const long long r0 = tr * kDtRows, c0 = tc * kDtCols;
+        __syncthreads();  // the previous tile has been read out (and the table is complete)
+        // 64 rows x 16 chunks of 16 bytes
+#pragma unroll
+        for (int i = 0; i < kDtRows * (kDtCols / 16) / kThreads; i++) {
+            const int v = i * kThreads + threadIdx.x, r = v / (kDtCols / 16), ch = v % (kDtCols / 16);
+            uint4 q = make_uint4(0, 0, 0, 0);
+            if (r0 + r < rows && c0 + ch * 16 < cols) q = __ldcs(reinterpret_cast<const uint4*>(src + (r0 + r) * cols + c0 + ch * 16));
+            uint32_t* d = tile + (r * kDtStride + ch * 16) / 4;
+            d[0] = q.x; d[1] = q.y; d[2] = q.z; d[3] = q.w;
+        }
+        __syncthreads();
+        // output row c (a source column), eight source rows per lane: 16 bytes of BF16
+#pragma unroll
+        for (int i = 0; i < kDtCols * (kDtRows / 8) / kThreads; i++) {
+            const int v = i * kThreads + threadIdx.x, c = v / (kDtRows / 8), seg = v % (kDtRows / 8);
+            if (c0 + c >= cols || r0 + seg * 8 >= rows) continue;  // rows is a multiple of 8: a segment is all in or all out
+            uint32_t h[8];
+#pragma unroll
+            for (int k = 0; k < 8; k++) h[k] = lut[tb[(seg * 8 + k) * kDtStride + c]];
+            __stcs(reinterpret_cast<uint4*>(dst + (c0 + c) * rows + r0 + seg * 8),
+                   make_uint4(h[0] | (h[1] << 16), h[2] | (h[3] << 16), h[4] | (h[5] << 16), h[6] | (h[7] << 16)));
+        }
+    }
+}
+
 template <int SRC, int MODE>
 int launch(const TrParams& p, bool vec, int sms, cudaStream_t st)
 {
@@ -151,6 +193,18 @@ int launch_mode(int rnd, const TrParams& p, bool vec, int sms, cudaStream_t st)
 }
 
 }  // namespace
+
+int decode_transpose_bf16(const uint8_t* src, void* dst, long long rows, long long cols, cudaStream_t st)
+{
+    if (rows <= 0 || cols <= 0 || (rows & 7) || (cols & 15)) return HIF8_ERR_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(src) & 15u) || (reinterpret_cast<uintptr_t>(dst) & 15u)) return HIF8_ERR_ALIGN;
+    const long long tiles = ((cols + kDtCols - 1) / kDtCols) * ((rows + kDtRows - 1) / kDtRows);
+    decode_transpose_bf16_kernel<<<(unsigned)(tiles < 0x7FFFFFFFll ? tiles : 0x7FFFFFFFll), kThreads, 0, st>>>(
+        src, reinterpret_cast<unsigned short*>(dst), rows, cols);
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
+}
+
 }  // namespace hif8
 
 using namespace hif8;
