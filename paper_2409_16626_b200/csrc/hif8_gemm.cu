@@ -249,16 +249,16 @@ __device__ __forceinline__ void store_chunk(const GemmParams& p, int row, int co
     if (p.c_is_f32) {
         float* out = reinterpret_cast<float*>(p.C) + (long long)row * p.ldc + col;
         if (full) {
+            // C is touched once: streaming loads and stores, so that it does not push operand tiles out of L2; all the
+            // loads of the chunk are issued before the first store (they cannot be moved across it by the compiler)
+            float4 c[8];
 #pragma unroll
-            for (int i = 0; i < 32; i += 4) {
-                float4 o = make_float4(__uint_as_float(r[i]) * f1 * f2, __uint_as_float(r[i + 1]) * f1 * f2,
-                                       __uint_as_float(r[i + 2]) * f1 * f2, __uint_as_float(r[i + 3]) * f1 * f2);
-                if (p.accumulate) {
-                    const float4 c = *reinterpret_cast<const float4*>(out + i);
-                    o.x += c.x; o.y += c.y; o.z += c.z; o.w += c.w;
-                }
-                *reinterpret_cast<float4*>(out + i) = o;
-            }
+            for (int i = 0; i < 8; i++) c[i] = p.accumulate ? __ldcs(reinterpret_cast<const float4*>(out) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int i = 0; i < 8; i++)
+                __stcs(reinterpret_cast<float4*>(out) + i,
+                       make_float4(__uint_as_float(r[4 * i]) * f1 * f2 + c[i].x, __uint_as_float(r[4 * i + 1]) * f1 * f2 + c[i].y,
+                                   __uint_as_float(r[4 * i + 2]) * f1 * f2 + c[i].z, __uint_as_float(r[4 * i + 3]) * f1 * f2 + c[i].w));
         } else {
             for (int i = 0; i < 32 && col + i < p.N; i++) out[i] = __uint_as_float(r[i]) * f1 * f2 + (p.accumulate ? out[i] : 0.f);
         }
@@ -269,7 +269,7 @@ __device__ __forceinline__ void store_chunk(const GemmParams& p, int row, int co
             if (full) {
 #pragma unroll
                 for (int i = 0; i < 32; i += 8) {
-                    const uint4 c = *reinterpret_cast<const uint4*>(out + i);
+                    const uint4 c = __ldcs(reinterpret_cast<const uint4*>(out + i));
                     h[i] = c.x << 16; h[i + 1] = c.x & 0xFFFF0000u; h[i + 2] = c.y << 16; h[i + 3] = c.y & 0xFFFF0000u;
                     h[i + 4] = c.z << 16; h[i + 5] = c.z & 0xFFFF0000u; h[i + 6] = c.w << 16; h[i + 7] = c.w & 0xFFFF0000u;
                 }
@@ -288,9 +288,9 @@ __device__ __forceinline__ void store_chunk(const GemmParams& p, int row, int co
         if (full) {
 #pragma unroll
             for (int i = 0; i < 32; i += 8)
-                *reinterpret_cast<uint4*>(out + i) =
-                    make_uint4(h[i] | (h[i + 1] << 16), h[i + 2] | (h[i + 3] << 16),
-                               h[i + 4] | (h[i + 5] << 16), h[i + 6] | (h[i + 7] << 16));
+                __stcs(reinterpret_cast<uint4*>(out + i),
+                       make_uint4(h[i] | (h[i + 1] << 16), h[i + 2] | (h[i + 3] << 16),
+                                  h[i + 4] | (h[i + 5] << 16), h[i + 6] | (h[i + 7] << 16)));
         } else {
             for (int i = 0; i < 32 && col + i < p.N; i++) out[i] = (unsigned short)h[i];
         }
