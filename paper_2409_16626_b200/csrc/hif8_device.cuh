@@ -210,15 +210,17 @@ template <int DT> __device__ __forceinline__ uint32_t to_bits(float v)
 // ------------------------------------------------------------------------------------------------
 // One element: scaled value -> HiF8 byte
 // ------------------------------------------------------------------------------------------------
-// Rounding tables, indexed by the biased exponent of the scaled value: thr[i] = A, thr[256 + i] = B.
-//  * TE / SR tables hold only B = sh, the number of discarded mantissa bits (23 - width; 0: nothing to round).
-//  * Hybrid / simplified stochastic rounding is one multiply-add on the bit pattern, t' = t + B + A * v, whose carry out
-//    of the discarded field rounds up (also across binade and width boundaries); the discarded bits of the old binade are
-//    cleared (mask ~0 << sh, with sh kept in spare bits of B: bits 27-31 for FP32 sources, bits 0-4 for 16-bit sources,
-//    whose widened patterns have zeros there) and the code is read from the truncating table.
-//       FP32 sources   v = 2^14 - max(T14, 1);  stochastic binade: A = 2^(sh-14), B = 0;  round-half-away binade: A = 0, B = 2^(sh-1)
-//       16-bit sources v = source LSB (T2 = 2 v + 1, complement 3 - 2 v);  stochastic: A = -2 * 2^(sh-2), B = 3 * 2^(sh-2);
-//                      round-half-away: A = 0, B = 2^(sh-1)
+// Rounding table thr[], indexed by the biased exponent of the scaled value (never by its sign: values of either sign would
+// otherwise hit different words of the same bank).
+//  * TE / SR: thr[e] = sh, the number of discarded mantissa bits (23 - width; 0: nothing to round).
+//  * Hybrid / simplified stochastic rounding adds an increment to the bit pattern so that the carry out of the discarded
+//    field rounds up (also across binade and width boundaries), clears the old binade's discarded bits (~0 << sh) and
+//    reads the code from the truncating table.
+//       FP32 sources: t' = t + B + A * v with v = 2^14 - max(T14, 1); stochastic binade: A = 2^(sh-14), B = 0; round-half-away
+//                     binade of Eq. 3: A = 0, B = 2^(sh-1).  thr[e] = A, thr[256 + e] = B with sh in bits 27-31.  (One
+//                     merged entry with a select on a flag measured slower: 156 against 143 us per 2^27 elements.)
+//       16-bit sources (T2 = 2 LSB + 1, complement 3 - 2 LSB): the increment itself, thr[2e + LSB] = (3 - 2 LSB) * 2^(sh-2)
+//                     or one half, with sh in bits 0-4: a widened 16-bit pattern has zeros there, so they cannot carry.
 //    Below 2^-22 (result 0 or 2^-22, F = |y| / 2^-22):
 //       FP32: the element is first moved into the binade of 2^-24 (see encode_one), whose entry rounds it like a
 //             0-bit-mantissa binade: no carry leaves 2^-24 (-> 0), a carry gives 2^-23 (-> 2^-22 in the truncating table).
@@ -244,9 +246,10 @@ __device__ __forceinline__ uint32_t encode_one(float x, uint32_t raw, float scal
             const uint32_t B = s_thr[256 + i];                    // constant in bits 0-26, sh in bits 27-31
             return s_ta[((u + (B & 0x07FFFFFFu) + s_thr[i] * v) & (0xFFFFFFFFu << (B >> 27))) >> 19];
         } else {
-            const uint32_t i = (t >> 23) & 0xFFu;
-            const uint32_t B = s_thr[256 + i];                    // sh in bits 0-4, below anything a 16-bit source sets
-            return s_ta[((t + B + s_thr[i] * (raw & 1u)) & (0xFFFFFFFFu << (B & 31u))) >> 19];  // SR2: complement 3 - 2 LSB
+            // two entries per exponent, chosen by the source LSB: B + A * LSB, with sh in bits 0-4 (a widened 16-bit
+            // pattern has zeros there, so they cannot carry)
+            const uint32_t ent = s_thr[((t >> 22) & 0x1FEu) | (raw & 1u)];
+            return s_ta[((t + ent) & (0xFFFFFFFFu << (ent & 31u))) >> 19];
         }
     }
 
@@ -265,7 +268,7 @@ __device__ __forceinline__ uint32_t encode_one(float x, uint32_t raw, float scal
         return f24 >= max(word >> 8, 1u) ? (sign7 | 0x01u) : 0u;
     }
     t = sub ? (tz | (t & 0x80000000u)) : t;
-    const uint32_t sh = s_thr[256 + ((t >> 23) & 0xFFu)] & 31u;  // discarded mantissa bits (23 - width); 0: nothing to round
+    const uint32_t sh = s_thr[(t >> 23) & 0xFFu];  // discarded mantissa bits (23 - width); 0: nothing to round
     const uint32_t s = sh ? sh : 23u;
     uint32_t inc;
     if (MODE == HIF8_RND_TE) {
@@ -340,23 +343,28 @@ __device__ __forceinline__ void setup_tables(SmemTables& s, unsigned flags)
         const int e = threadIdx.x, E = e - 127;  // kThreads == 256 biased exponents
         constexpr bool kF32 = SRC == HIF8_F32;
         constexpr bool kThreshold = MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR;
-        uint32_t A = 0, B = 0;
+        // TE / SR: thr[e] = e0.  FP32 threshold modes: thr[e] = e0 (A), thr[256 + e] = e1 (B).  16-bit threshold modes:
+        // thr[2e] = e0 (source LSB 0), thr[2e + 1] = e1 (LSB 1).
+        uint32_t e0 = 0, e1 = 0;
         if (E < 16 && E >= -22) {
             const uint32_t sh = 23u - (uint32_t)mant_width(E);
-            if (!kThreshold) B = sh;  // TE / SR: only the width is read
-            else if (MODE == HIF8_RND_SSR || E <= -4 || E >= 4) {
-                if (kF32) A = 1u << (sh - 14u);
-                else { A = 0u - (2u << (sh - 2u)); B = 3u << (sh - 2u); }
-                B |= kF32 ? sh << 27 : sh;
-            } else B = (1u << (sh - 1u)) | (kF32 ? sh << 27 : sh);  // Eq. 3: round half away in the binades |E| < 4
+            const bool stochastic = MODE == HIF8_RND_SSR || E <= -4 || E >= 4;  // Eq. 3 for HR
+            if (!kThreshold) e0 = sh;  // TE / SR: only the width is read
+            else if (kF32) {
+                if (stochastic) e0 = 1u << (sh - 14u); else e1 = 1u << (sh - 1u);
+                e1 |= sh << 27;
+            }
+            else if (stochastic) { e0 = (3u << (sh - 2u)) | sh; e1 = (1u << (sh - 2u)) | sh; }  // complement 3 - 2 LSB
+            else e0 = e1 = (1u << (sh - 1u)) | sh;
         } else if (kThreshold && kF32 && E == -24) {
-            A = 1u << 9; B = 23u << 27;  // where encode_one parks FP32 elements below 2^-22
+            e0 = 1u << 9; e1 = 23u << 27;  // where encode_one parks FP32 elements below 2^-22
         } else if (kThreshold && !kF32 && (E == -23 || E == -24)) {
             const uint32_t j = (uint32_t)(-23 - E);  // complement << (22 + j), then j + 1 binades down
-            A = 0u - (2u << (22u + j));
-            B = ((3u << (22u + j)) - ((j + 1u) << 23)) | 23u;
+            e0 = ((3u << (22u + j)) - ((j + 1u) << 23)) | 23u;
+            e1 = ((1u << (22u + j)) - ((j + 1u) << 23)) | 23u;
         }
-        s.thr[e] = A; s.thr[256 + e] = B;
+        if (kThreshold && !kF32) { s.thr[2 * e] = e0; s.thr[2 * e + 1] = e1; }
+        else { s.thr[e] = e0; s.thr[256 + e] = e1; }
     }
     if (NEED_DEC) s.dec[threadIdx.x] = __uint_as_float(decode_bits_f32(threadIdx.x));
     __syncthreads();
