@@ -186,8 +186,8 @@ int hif8_channel_amax_scale_encode(const void* W, int src_dtype, uint8_t* dst, i
  * (256-byte aligned) owned by the caller; nothing returns to the host.
  *   hif8_scale_state_init:      exponent 0, empty ring of hist_len entries (1..HIF8_SCALE_HISTORY_MAX).
  *   hif8_delayed_scale_encode:  dst = To_HiF8_<rnd>(src * 2^(exponent in force)) in one pass over src.  With
- *        measure != 0 (the caller's "iteration % N == 0") the same pass also reduces amax of src, and a one-thread
- *        kernel then pushes it into the ring and updates the exponent.  The first int of the state is the exponent
+ *        measure != 0 (the caller's "iteration % N == 0") the same pass also reduces amax of src, and the last
+ *        thread block to finish pushes it into the ring and updates the exponent (one kernel launch either way).  The first int of the state is the exponent
  *        in force (readable as the d_scale_exp_a / d_scale_exp_w of hif8_gemm), the float at byte 16 the last amax.
  */
 #define HIF8_SCALE_STATE_BYTES 1024

@@ -137,6 +137,13 @@ __global__ void __launch_bounds__(kThreads) convert_kernel(const ConvParams p, u
                 __threadfence();
                 uint32_t ab = atomicMax(p.amax_accum, 0u);
                 if (p.d_amax_out) *p.d_amax_out = __uint_as_float(ab);
+                if (p.scale_state) {
+                    // delayed scaling: every block has read the exponent in force and finished, so the state can move on;
+                    // the accumulator and the ticket are left at zero for the next measuring pass
+                    scale_state_push(reinterpret_cast<ScaleState*>(p.scale_state), ab, p.target_exp);
+                    p.amax_accum[0] = 0u;
+                    p.amax_accum[1] = 0u;
+                }
             }
         }
     }
@@ -558,7 +565,7 @@ int hif8_decode(const uint8_t* src, void* dst, int dst_dtype, size_t n, int scal
 static int scaled_convert(bool fq, const void* src, void* dst, int dtype, size_t n, bool jit, int target_exp,
                           const int* d_scale_exp_in, int scale_exp, int rnd, unsigned flags, uint64_t seed,
                           float* d_amax_out, int* d_scale_exp_out, float* d_scale_out, void* workspace,
-                          size_t workspace_bytes, bool want_amax, cudaStream_t st)
+                          size_t workspace_bytes, bool want_amax, cudaStream_t st, void* scale_state = nullptr)
 {
     int sms; int rc = device_info(&sms);
     if (rc) return rc;
@@ -571,8 +578,10 @@ static int scaled_convert(bool fq, const void* src, void* dst, int dtype, size_t
     bool vec_ok = aligned16(src) && (reinterpret_cast<uintptr_t>(dst) % out_align) == 0;
     if (jit || want_amax) {
         if (!ws || workspace_bytes < kConvWorkspaceBytes || (reinterpret_cast<uintptr_t>(ws) & 255u)) return HIF8_ERR_WORKSPACE;
-        if (cudaMemsetAsync(ws, 0, 8, st) != cudaSuccess) return HIF8_ERR_CUDA;
+        // (a delayed-scaling state keeps its two words at zero between passes itself)
+        if (!scale_state && cudaMemsetAsync(ws, 0, 8, st) != cudaSuccess) return HIF8_ERR_CUDA;
     }
+    p.scale_state = scale_state;
     const bool inplace_fq = fq && !want_amax && ((rnd == HIF8_RND_TA && (dtype == HIF8_F32 || dtype == HIF8_BF16)) ||
                                                 ((rnd == HIF8_RND_HR || rnd == HIF8_RND_SSR) && dtype == HIF8_BF16));
     if (jit) {
@@ -742,41 +751,19 @@ extern "C" int hif8_amax_scale_encode_static(const void* src, int src_dtype, uin
 
 // ------------------------------------------------------------------------------------------------
 // Delayed scaling: the every-N-iterations amax cadence of Section 5.1 with a ring of past amax values.
-// State (device memory, HIF8_SCALE_STATE_BYTES): bytes 0-255 the record below, bytes 256-511 the scratch of the
-// conversion kernel's amax reduction.
+// State (device memory, HIF8_SCALE_STATE_BYTES): bytes 0-255 the ScaleState record, bytes 256-511 the scratch of the
+// conversion kernel's amax reduction (kept at zero between measuring passes by the kernel itself).
 // ------------------------------------------------------------------------------------------------
 namespace hif8 {
 namespace {
-struct ScaleState {
-    int scale_exp;  // exponent in force
-    int pos;        // next ring slot
-    int filled;     // valid ring entries
-    int hist_len;
-    float amax_last;
-    int pad[3];
-    float ring[HIF8_SCALE_HISTORY_MAX];
-};
-static_assert(sizeof(ScaleState) <= 256, "state record too large");
-
 __global__ void scale_state_init_kernel(ScaleState* st, int hist_len)
 {
     const int i = threadIdx.x;
     if (i == 0) { st->scale_exp = 0; st->pos = 0; st->filled = 0; st->hist_len = hist_len; st->amax_last = 0.f; }
     if (i < HIF8_SCALE_HISTORY_MAX) st->ring[i] = 0.f;
+    if (i < 2) reinterpret_cast<uint32_t*>(reinterpret_cast<unsigned char*>(st) + 256)[i] = 0u;  // amax accumulator, block ticket
 }
 
-// push the amax just measured, then exponent = rule(max of the ring); one thread
-__global__ void scale_state_update_kernel(ScaleState* st, int target_exp)
-{
-    if (threadIdx.x != 0) return;
-    const int n = st->hist_len;
-    st->ring[st->pos] = st->amax_last;
-    st->pos = (st->pos + 1) % n;
-    if (st->filled < n) st->filled++;
-    uint32_t m = 0;
-    for (int j = 0; j < st->filled; j++) m = max(m, __float_as_uint(st->ring[j]));  // non-negative floats order as integers
-    st->scale_exp = scale_exp_from_amax(m, target_exp);
-}
 }  // namespace
 }  // namespace hif8
 
@@ -805,12 +792,9 @@ extern "C" int hif8_delayed_scale_encode(const void* src, int src_dtype, uint8_t
     if (!measure)  // conversion alone, exponent read from the state on the device
         return scaled_convert(false, src, dst, src_dtype, n, false, target_exp, &state->scale_exp, 0, rnd, flags, seed, nullptr,
                               nullptr, nullptr, nullptr, 0, false, st);
-    // one pass: convert with the exponent in force and reduce amax; then the one-thread update
-    rc = scaled_convert(false, src, dst, src_dtype, n, false, target_exp, &state->scale_exp, 0, rnd, flags, seed,
-                        &state->amax_last, nullptr, nullptr, reinterpret_cast<unsigned char*>(d_state) + 256, kConvWorkspaceBytes,
-                        true, st);
-    if (rc) return rc;
-    scale_state_update_kernel<<<1, 32, 0, st>>>(state, target_exp);
-    g_launches.fetch_add(1, std::memory_order_relaxed);
-    return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
+    // one pass: convert with the exponent in force and reduce amax; the last block to finish pushes it into the ring and
+    // sets the exponent for the next conversion
+    return scaled_convert(false, src, dst, src_dtype, n, false, target_exp, &state->scale_exp, 0, rnd, flags, seed,
+                          &state->amax_last, nullptr, nullptr, reinterpret_cast<unsigned char*>(d_state) + 256, kConvWorkspaceBytes,
+                          true, st, d_state);
 }

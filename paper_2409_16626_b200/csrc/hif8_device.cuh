@@ -163,6 +163,7 @@ struct ConvParams {
     float* d_amax_out;
     int* d_scale_exp_out;
     float* d_scale_out;
+    void* scale_state;            // delayed scaling: ScaleState that the last block of an amax-reducing pass advances
 };
 
 template <int SRC> struct SrcTraits;
@@ -368,6 +369,31 @@ __device__ __forceinline__ void setup_tables(SmemTables& s, unsigned flags)
     }
     if (NEED_DEC) s.dec[threadIdx.x] = __uint_as_float(decode_bits_f32(threadIdx.x));
     __syncthreads();
+}
+
+// Delayed scaling (the every-N-iterations amax cadence of Section 5.1): exponent in force and a ring of past amax values
+struct ScaleState {
+    int scale_exp;  // exponent in force
+    int pos;        // next ring slot
+    int filled;     // valid ring entries
+    int hist_len;
+    float amax_last;
+    int pad[3];
+    float ring[HIF8_SCALE_HISTORY_MAX];
+};
+static_assert(sizeof(ScaleState) <= 256, "state record too large");
+
+// push the amax just measured (bit pattern of a non-negative float), then exponent = rule(max of the ring); one thread
+__device__ __forceinline__ void scale_state_push(ScaleState* st, uint32_t amax_bits, int target_exp)
+{
+    const int n = st->hist_len;
+    st->amax_last = __uint_as_float(amax_bits);
+    st->ring[st->pos] = __uint_as_float(amax_bits);
+    st->pos = (st->pos + 1) % n;
+    if (st->filled < n) st->filled++;
+    uint32_t m = 0;
+    for (int j = 0; j < st->filled; j++) m = max(m, __float_as_uint(st->ring[j]));  // non-negative floats order as integers
+    st->scale_exp = scale_exp_from_amax(m, target_exp);
 }
 
 __device__ __forceinline__ int resolve_scale_exp(const ConvParams& p)
