@@ -160,6 +160,24 @@ def extra_results(H, torch, hbm_peak, peak_kind):
         torch.cuda.synchronize()
         return ev0.elapsed_time(ev1) / reps
 
+    # ---- small and odd sizes (launch latency, tails): FP32 encode TA + decode, 20 call pairs per graph replay
+    small = {}
+    for n in (9408, 1000003, 4096 * 11008, 256 * 64 * 56 * 56):
+        xs_ = torch.randn(n, generator=g, device="cuda")
+        cq = torch.empty(n, dtype=torch.uint8, device="cuda")
+        bk = torch.empty(n, dtype=torch.float32, device="cuda")
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr):
+            cs = torch.cuda.current_stream().cuda_stream
+            for _ in range(20):
+                H.hif8_encode(xs_, H.F32, cq, n, 10, H.RND_TA, stream=cs)
+                H.hif8_decode(cq, bk, H.F32, n, 10, stream=cs)
+        ms = timed(lambda r: gr.replay(), 5) / 20
+        small[str(n)] = {"us_per_encode_decode_pair": ms * 1e3, "GBps": 10 * n / ms / 1e6, "frac": 10 * n / ms / 1e6 / hbm_peak}
+        del xs_, cq, bk, gr
+    out["small_and_odd_sizes_f32"] = {"bytes_per_element": 10, "sizes": small, "peak": hbm_peak, "peak_kind": f"of {peak_kind}",
+                                      "note": "tensors up to 45 M elements fit in L2 between the two calls; a pair is two launches"}
+
     # ---- LLM-activation fake-quant: BF16 [8192 x 8192], Student-t(3) body, 0.1 % of channels x100
     T = Hd = 8192
     n = T * Hd
