@@ -40,9 +40,12 @@ namespace {
 
 constexpr int BM = 128, BN = 256, BK = 64;
 constexpr int kStages8 = 4;    // staging ring of HiF8 byte tiles
-constexpr int kStagesBf = 3;   // ring of decoded BF16 operand tiles
+constexpr int kStagesBf = 4;   // ring of decoded BF16 operand tiles
 constexpr int kEpiWarps = 4, kDecodeWarps = 16;
-constexpr int kDecodeThreads = kDecodeWarps * 32;
+// The decode warps work in groups, group g on the k-blocks kb = g (mod kDecodeGroups): several k-blocks are in the
+// decode stage at once, which covers the latency of each one's lookups, proxy fence and barrier hand-over.
+constexpr int kDecodeGroups = 4, kGroupWarps = kDecodeWarps / kDecodeGroups, kGroupThreads = kGroupWarps * 32;
+static_assert(kStages8 == kDecodeGroups && kStagesBf == kDecodeGroups, "group g owns byte stage g and operand stage g");
 constexpr int kThreads = (kEpiWarps + 2 + kDecodeWarps) * 32;  // 704
 constexpr int kTmaWarp = 4, kMmaWarp = 5, kFirstDecodeWarp = 6;
 // per CTA of a pair: 128 rows of A and 128 of the 256 columns of W
@@ -316,8 +319,8 @@ __device__ __forceinline__ void apply_channel_scale(const GemmParams& p, int col
 __device__ __forceinline__ void decode_tile_k_major(const unsigned char* src8, unsigned char* dst, int dt, const uint32_t* lut)
 {
 #pragma unroll
-    for (int it = 0; it < (BM * BK / 8) / kDecodeThreads; it++) {
-        const int q = it * kDecodeThreads + dt, r = q >> 3, j = q & 7;
+    for (int it = 0; it < (BM * BK / 8) / kGroupThreads; it++) {
+        const int q = it * kGroupThreads + dt, r = q >> 3, j = q & 7;
         const uint2 v = *reinterpret_cast<const uint2*>(src8 + r * BK + j * 8);
         *reinterpret_cast<uint4*>(dst + (r >> 3) * 1024 + (r & 7) * 128 + ((j ^ (r & 7)) << 4)) = decode8(v, lut);
     }
@@ -326,8 +329,8 @@ __device__ __forceinline__ void decode_tile_k_major(const unsigned char* src8, u
 __device__ __forceinline__ void decode_tile_mn_major(const unsigned char* src8, unsigned char* dst, int dt, const uint32_t* lut)
 {
 #pragma unroll
-    for (int it = 0; it < (BM * BK / 8) / kDecodeThreads; it++) {
-        const int q = it * kDecodeThreads + dt, k = q >> 4, jn = q & 15;
+    for (int it = 0; it < (BM * BK / 8) / kGroupThreads; it++) {
+        const int q = it * kGroupThreads + dt, k = q >> 4, jn = q & 15;
         const uint2 v = *reinterpret_cast<const uint2*>(src8 + k * BM + jn * 8);
         const int atom = (jn >> 3) * 8 + (k >> 3);
         *reinterpret_cast<uint4*>(dst + atom * 1024 + (k & 7) * 128 + (((jn & 7) ^ (k & 7)) << 4)) = decode8(v, lut);
@@ -365,8 +368,8 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     // ---- set-up
     for (int i = threadIdx.x; i < 256 * 32; i += kThreads) lut_all[i] = hif8_to_bf16_bits(i >> 5);
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages8; s++) { mbar_init(bar_u8_full(s), 1); mbar_init(bar_u8_empty(s), kDecodeWarps); }
-        for (int s = 0; s < kStagesBf; s++) { mbar_init(bar_bf_full(s), 2 * kDecodeWarps); mbar_init(bar_bf_empty(s), 1); }
+        for (int s = 0; s < kStages8; s++) { mbar_init(bar_u8_full(s), 1); mbar_init(bar_u8_empty(s), kGroupWarps); }
+        for (int s = 0; s < kStagesBf; s++) { mbar_init(bar_bf_full(s), 2 * kGroupWarps); mbar_init(bar_bf_empty(s), 1); }
         mbar_init(bar_acc_full, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -435,10 +438,11 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         }
     } else if (warp >= kFirstDecodeWarp) {
         // ------------------------------------------------------------------ decode warps
-        const int dt = threadIdx.x - kFirstDecodeWarp * 32;  // 0..kDecodeThreads-1
+        const int group = (warp - kFirstDecodeWarp) / kGroupWarps;
+        const int dt = threadIdx.x - (kFirstDecodeWarp + group * kGroupWarps) * 32;  // 0..kGroupThreads-1
         bool ok = true;
-        for (int kb = 0; kb < num_kb && ok; kb++) {
-            const int s8 = kb % kStages8, r8 = kb / kStages8, sb = kb % kStagesBf, rb = kb / kStagesBf;
+        for (int kb = group; kb < num_kb && ok; kb += kDecodeGroups) {
+            const int s8 = group, r8 = kb / kStages8, sb = group, rb = kb / kStagesBf;
             ok = mbar_wait(bar_u8_full(s8), r8 & 1, abort_flag, p.status, 3);
             if (ok && rb > 0) ok = mbar_wait(bar_bf_empty(sb), (rb - 1) & 1, abort_flag, p.status, 4);
             if (!ok) break;
