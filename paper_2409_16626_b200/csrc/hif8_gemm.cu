@@ -43,7 +43,9 @@ constexpr int kStages8 = 4;    // staging ring of HiF8 byte tiles
 constexpr int kStagesBf = 4;   // ring of decoded BF16 operand tiles
 constexpr int kEpiWarps = 4, kDecodeWarps = 16;
 // The decode warps work in groups, group g on the k-blocks kb = g (mod kDecodeGroups): several k-blocks are in the
-// decode stage at once, which covers the latency of each one's lookups, proxy fence and barrier hand-over.
+// decode stage at once, which covers the latency of each one's lookups, proxy fence and barrier hand-over.  Group g
+// owns byte stage g and operand stage g, so every barrier is waited on by one party in program order (a waiter is never
+// more than one phase ahead of the barrier, which a parity wait could not tell apart).
 constexpr int kDecodeGroups = 4, kGroupWarps = kDecodeWarps / kDecodeGroups, kGroupThreads = kGroupWarps * 32;
 static_assert(kStages8 == kDecodeGroups && kStagesBf == kDecodeGroups, "group g owns byte stage g and operand stage g");
 constexpr int kThreads = (kEpiWarps + 2 + kDecodeWarps) * 32;  // 704
@@ -314,26 +316,35 @@ __device__ __forceinline__ void apply_channel_scale(const GemmParams& p, int col
     }
 }
 
-// Fused kernel, decode warps: one 128 x 64 tile of HiF8 bytes -> BF16 in the 128-byte-swizzled operand layout.
+// Fused kernel, decode warps: one 128 x 64 tile of HiF8 bytes -> BF16 in the 128-byte-swizzled operand layout, in two
+// steps so that the byte tile can be handed back to the TMA producer as soon as it has been read: first a thread's
+// eight 8-byte chunks into registers, then lookups and swizzled stores.
+constexpr int kChunksPerThread = (BM * BK / 8) / kGroupThreads;  // 8
 // K-major source tile [128 rows][64 k]: chunk j (8 codes) of row r -> atom r/8, row r%8, chunk j ^ (r%8).
-__device__ __forceinline__ void decode_tile_k_major(const unsigned char* src8, unsigned char* dst, int dt, const uint32_t* lut)
+// MN-major source tile [64 k][128 mn]: chunk (k, mn/8) -> atom (mn/64) * 8 + k/8, row k%8, chunk (mn/8)%8 ^ (k%8).
+template <bool MN_MAJOR>
+__device__ __forceinline__ void load_tile_chunks(const unsigned char* src8, int dt, uint2 (&v)[kChunksPerThread])
 {
 #pragma unroll
-    for (int it = 0; it < (BM * BK / 8) / kGroupThreads; it++) {
-        const int q = it * kGroupThreads + dt, r = q >> 3, j = q & 7;
-        const uint2 v = *reinterpret_cast<const uint2*>(src8 + r * BK + j * 8);
-        *reinterpret_cast<uint4*>(dst + (r >> 3) * 1024 + (r & 7) * 128 + ((j ^ (r & 7)) << 4)) = decode8(v, lut);
+    for (int it = 0; it < kChunksPerThread; it++) {
+        const int q = it * kGroupThreads + dt;
+        v[it] = MN_MAJOR ? *reinterpret_cast<const uint2*>(src8 + (q >> 4) * BM + (q & 15) * 8)
+                         : *reinterpret_cast<const uint2*>(src8 + (q >> 3) * BK + (q & 7) * 8);
     }
 }
-// MN-major source tile [64 k][128 mn]: chunk (k, mn/8) -> atom (mn/64) * 8 + k/8, row k%8, chunk (mn/8)%8 ^ (k%8).
-__device__ __forceinline__ void decode_tile_mn_major(const unsigned char* src8, unsigned char* dst, int dt, const uint32_t* lut)
+template <bool MN_MAJOR>
+__device__ __forceinline__ void decode_tile_chunks(const uint2 (&v)[kChunksPerThread], unsigned char* dst, int dt, const uint32_t* lut)
 {
 #pragma unroll
-    for (int it = 0; it < (BM * BK / 8) / kGroupThreads; it++) {
-        const int q = it * kGroupThreads + dt, k = q >> 4, jn = q & 15;
-        const uint2 v = *reinterpret_cast<const uint2*>(src8 + k * BM + jn * 8);
-        const int atom = (jn >> 3) * 8 + (k >> 3);
-        *reinterpret_cast<uint4*>(dst + atom * 1024 + (k & 7) * 128 + (((jn & 7) ^ (k & 7)) << 4)) = decode8(v, lut);
+    for (int it = 0; it < kChunksPerThread; it++) {
+        const int q = it * kGroupThreads + dt;
+        if (MN_MAJOR) {
+            const int k = q >> 4, jn = q & 15, atom = (jn >> 3) * 8 + (k >> 3);
+            *reinterpret_cast<uint4*>(dst + atom * 1024 + (k & 7) * 128 + (((jn & 7) ^ (k & 7)) << 4)) = decode8(v[it], lut);
+        } else {
+            const int r = q >> 3, j = q & 7;
+            *reinterpret_cast<uint4*>(dst + (r >> 3) * 1024 + (r & 7) * 128 + ((j ^ (r & 7)) << 4)) = decode8(v[it], lut);
+        }
     }
 }
 
@@ -450,14 +461,16 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             const unsigned char* b8 = a8 + kA8Bytes;
             unsigned char* abf = sm + SmemLayout::bf + sb * (kABfBytes + kBBfBytes);
             unsigned char* bbf = abf + kABfBytes;
-            if (A_IS_KM) decode_tile_mn_major(a8, abf, dt, lut); else decode_tile_k_major(a8, abf, dt, lut);
-            if (W_IS_NK) decode_tile_k_major(b8, bbf, dt, lut); else decode_tile_mn_major(b8, bbf, dt, lut);
+            uint2 va[kChunksPerThread], vw[kChunksPerThread];
+            load_tile_chunks<A_IS_KM>(a8, dt, va);
+            load_tile_chunks<!W_IS_NK>(b8, dt, vw);
+            __syncwarp();  // every lane's reads of the byte stage are done: the producer may refill it during the decode
+            if (lane == 0) mbar_arrive(bar_u8_empty(s8));
+            decode_tile_chunks<A_IS_KM>(va, abf, dt, lut);
+            decode_tile_chunks<!W_IS_NK>(vw, bbf, dt, lut);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // make the stores visible to the tensor core
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(bar_u8_empty(s8));
-                mbar_arrive_cluster(map_to_cta(bar_bf_full(sb), 0));  // the leader's MMAs read both CTAs' operands
-            }
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(bar_bf_full(sb), 0));  // the leader's MMAs read both CTAs' operands
         }
     } else {
         // ------------------------------------------------------------------ epilogue warps 0-3 (each CTA drains its rows)
