@@ -219,17 +219,36 @@ __device__ __forceinline__ uint32_t hif8_to_bf16_bits(uint32_t c)
     return sign | ((uint32_t)(E + 127) << 7) | (M << (7 - w));
 }
 
+// Shared-memory accesses by 32-bit shared-window address: the operand ring lives at a run-time offset inside the dynamic
+// allocation, and spelling the state space out keeps every one of these an LDS / STS (never a generic access).
+__device__ __forceinline__ uint32_t lds_u32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint2 lds_v2(uint32_t addr)
+{
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void sts_v4(uint32_t addr, uint4 v)
+{
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
 // eight HiF8 bytes -> eight BF16 (one 16-byte operand chunk).  `lut_lane` points at this lane's column of the
-// lane-replicated table: entry of byte c is the 32-bit word at lut_lane[c * 32], so lane L only ever touches
+// lane-replicated table: entry of byte c is the 32-bit word at lut_lane + 128 c, so lane L only ever touches
 // shared-memory bank L and the eight lookups of a warp instruction never conflict.
-__device__ __forceinline__ uint4 decode8(uint2 v, const uint32_t* lut_lane)
+__device__ __forceinline__ uint4 decode8(uint2 v, uint32_t lut_lane)  // lut_lane: shared address of this lane's column
 {
     uint32_t o[4];
 #pragma unroll
     for (int i = 0; i < 4; i++) {
         const uint32_t w = i < 2 ? v.x : v.y;
         const uint32_t c0 = (w >> (16 * (i & 1))) & 0xFFu, c1 = (w >> (16 * (i & 1) + 8)) & 0xFFu;
-        o[i] = __byte_perm(lut_lane[c0 * 32], lut_lane[c1 * 32], 0x5410);
+        o[i] = __byte_perm(lds_u32(lut_lane + c0 * 128), lds_u32(lut_lane + c1 * 128), 0x5410);
     }
     return make_uint4(o[0], o[1], o[2], o[3]);
 }
@@ -323,27 +342,26 @@ constexpr int kChunksPerThread = (BM * BK / 8) / kGroupThreads;  // 8
 // K-major source tile [128 rows][64 k]: chunk j (8 codes) of row r -> atom r/8, row r%8, chunk j ^ (r%8).
 // MN-major source tile [64 k][128 mn]: chunk (k, mn/8) -> atom (mn/64) * 8 + k/8, row k%8, chunk (mn/8)%8 ^ (k%8).
 template <bool MN_MAJOR>
-__device__ __forceinline__ void load_tile_chunks(const unsigned char* src8, int dt, uint2 (&v)[kChunksPerThread])
+__device__ __forceinline__ void load_tile_chunks(uint32_t src8, int dt, uint2 (&v)[kChunksPerThread])
 {
 #pragma unroll
     for (int it = 0; it < kChunksPerThread; it++) {
         const int q = it * kGroupThreads + dt;
-        v[it] = MN_MAJOR ? *reinterpret_cast<const uint2*>(src8 + (q >> 4) * BM + (q & 15) * 8)
-                         : *reinterpret_cast<const uint2*>(src8 + (q >> 3) * BK + (q & 7) * 8);
+        v[it] = MN_MAJOR ? lds_v2(src8 + (q >> 4) * BM + (q & 15) * 8) : lds_v2(src8 + (q >> 3) * BK + (q & 7) * 8);
     }
 }
 template <bool MN_MAJOR>
-__device__ __forceinline__ void decode_tile_chunks(const uint2 (&v)[kChunksPerThread], unsigned char* dst, int dt, const uint32_t* lut)
+__device__ __forceinline__ void decode_tile_chunks(const uint2 (&v)[kChunksPerThread], uint32_t dst, int dt, uint32_t lut)
 {
 #pragma unroll
     for (int it = 0; it < kChunksPerThread; it++) {
         const int q = it * kGroupThreads + dt;
         if (MN_MAJOR) {
             const int k = q >> 4, jn = q & 15, atom = (jn >> 3) * 8 + (k >> 3);
-            *reinterpret_cast<uint4*>(dst + atom * 1024 + (k & 7) * 128 + (((jn & 7) ^ (k & 7)) << 4)) = decode8(v[it], lut);
+            sts_v4(dst + atom * 1024 + (k & 7) * 128 + (((jn & 7) ^ (k & 7)) << 4), decode8(v[it], lut));
         } else {
             const int r = q >> 3, j = q & 7;
-            *reinterpret_cast<uint4*>(dst + (r >> 3) * 1024 + (r & 7) * 128 + ((j ^ (r & 7)) << 4)) = decode8(v[it], lut);
+            sts_v4(dst + (r >> 3) * 1024 + (r & 7) * 128 + ((j ^ (r & 7)) << 4), decode8(v[it], lut));
         }
     }
 }
@@ -368,7 +386,7 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + SmemLayout::abort_flag);
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + SmemLayout::tmem_slot);
     uint32_t* lut_all = reinterpret_cast<uint32_t*>(sm + SmemLayout::lut);
-    const uint32_t* lut = lut_all + lane;
+    const uint32_t lut = base + SmemLayout::lut + 4u * lane;  // this lane's column of the table
 
     // 256 x 256 tile of this pair (groups of 8 tile-rows share their W tiles in L2); this CTA: 128 rows, 128 columns of W
     int tile_m, tile_n;
@@ -457,10 +475,8 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             ok = mbar_wait(bar_u8_full(s8), r8 & 1, abort_flag, p.status, 3);
             if (ok && rb > 0) ok = mbar_wait(bar_bf_empty(sb), (rb - 1) & 1, abort_flag, p.status, 4);
             if (!ok) break;
-            const unsigned char* a8 = sm + SmemLayout::u8 + s8 * (kA8Bytes + kB8Bytes);
-            const unsigned char* b8 = a8 + kA8Bytes;
-            unsigned char* abf = sm + SmemLayout::bf + sb * (kABfBytes + kBBfBytes);
-            unsigned char* bbf = abf + kABfBytes;
+            const uint32_t a8 = base + SmemLayout::u8 + s8 * (kA8Bytes + kB8Bytes), b8 = a8 + kA8Bytes;
+            const uint32_t abf = base + SmemLayout::bf + sb * (kABfBytes + kBBfBytes), bbf = abf + kABfBytes;
             uint2 va[kChunksPerThread], vw[kChunksPerThread];
             load_tile_chunks<A_IS_KM>(a8, dt, va);
             load_tile_chunks<!W_IS_NK>(b8, dt, vw);
