@@ -175,6 +175,19 @@ __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap
         "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
         ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
+// one-CTA forms (the narrow kernel)
+__device__ __forceinline__ void tc_commit_cta(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_cta(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar)  // arrives on `bar` in both CTAs of the pair
 {
     asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
@@ -521,6 +534,191 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 }
 
 // ---------------------------------------------------------------------------------------------------------
+// Narrow products (M <= 64 rows of activations: the decode phase of inference).  The product is bound by reading the
+// weight bytes once, so the roles are swapped: a CTA streams a slab of 128 weight columns as the 128-row MMA operand and
+// the few activation rows are the narrow operand (MMA N = M rounded up to 16).  Same machinery as the fused kernel
+// (byte tiles by TMA, four decode groups on four k-blocks, operands in the 128-byte-swizzled layout), one CTA per slab,
+// no pairs.  The accumulator holds C transposed (row = weight column n, column = activation row m); the epilogue writes
+// C[m][n] with consecutive lanes on consecutive n.
+// ---------------------------------------------------------------------------------------------------------
+constexpr int kNarrowMaxM = 64;
+constexpr uint32_t kNwW8 = BM * BK, kNwA8 = kNarrowMaxM * BK;          // byte tiles per stage: 8 KiB weights, 4 KiB activations
+constexpr uint32_t kNwWBf = BM * BK * 2, kNwABf = kNarrowMaxM * BK * 2;  // operand tiles per stage: 16 KiB + 8 KiB
+struct SmemLayoutN {
+    static constexpr uint32_t bf = 0;
+    static constexpr uint32_t u8 = bf + kDecodeGroups * (kNwWBf + kNwABf);
+    static constexpr uint32_t lut = u8 + kDecodeGroups * (kNwW8 + kNwA8);
+    static constexpr uint32_t bars = lut + 256 * 32 * 4;
+    static constexpr uint32_t n_bars = 4 * kDecodeGroups + 1;
+    static constexpr uint32_t tmem_slot = bars + n_bars * 8;
+    static constexpr uint32_t abort_flag = tmem_slot + 4;
+    static constexpr uint32_t total = abort_flag + 4;
+};
+constexpr uint32_t kSmemBytesN = SmemLayoutN::total + 1024;
+constexpr uint32_t kTmemColsN = 64;
+
+template <bool W_IS_NK>
+__global__ void __launch_bounds__(kThreads, 1)
+hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_constant__ CUtensorMap map_w, const GemmParams p, int mp)
+{
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    unsigned char* sm = smem_raw + (base - smem_u32(smem_raw));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr int S = kDecodeGroups;  // stages of both rings: group g owns stage g
+    const uint32_t bars = base + SmemLayoutN::bars;
+    auto bar_u8_full = [&](int s) { return bars + 8u * s; };
+    auto bar_u8_empty = [&](int s) { return bars + 8u * (S + s); };
+    auto bar_bf_full = [&](int s) { return bars + 8u * (2 * S + s); };
+    auto bar_bf_empty = [&](int s) { return bars + 8u * (3 * S + s); };
+    const uint32_t bar_acc_full = bars + 8u * (4 * S);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + SmemLayoutN::abort_flag);
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + SmemLayoutN::tmem_slot);
+    uint32_t* lut_all = reinterpret_cast<uint32_t*>(sm + SmemLayoutN::lut);
+    const uint32_t lut = base + SmemLayoutN::lut + 4u * lane;
+    const int n0 = blockIdx.x * BM;  // this CTA's 128 weight columns
+    const int num_kb = (p.K + BK - 1) / BK;
+    const uint32_t act_bytes = (uint32_t)mp * BK;
+
+    for (int i = threadIdx.x; i < 256 * 32; i += kThreads) lut_all[i] = hif8_to_bf16_bits(i >> 5);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; s++) {
+            mbar_init(bar_u8_full(s), 1); mbar_init(bar_u8_empty(s), kGroupWarps);
+            mbar_init(bar_bf_full(s), kGroupWarps); mbar_init(bar_bf_empty(s), 1);
+        }
+        mbar_init(bar_acc_full, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == kMmaWarp) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(base + SmemLayoutN::tmem_slot), "r"(kTmemColsN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == kTmaWarp) {
+        if (lane == 0) {
+            int issued = 0;
+            for (int kb = 0; kb < num_kb; kb++) {
+                const int s = kb % S, round = kb / S;
+                if (round > 0 && !mbar_wait(bar_u8_empty(s), (round - 1) & 1, abort_flag, p.status, 31)) break;
+                if (*abort_flag) break;
+                const uint32_t dst_w = base + SmemLayoutN::u8 + s * (kNwW8 + kNwA8), dst_a = dst_w + kNwW8;
+                mbar_arrive_expect_tx(bar_u8_full(s), kNwW8 + act_bytes);
+                if (W_IS_NK) tma_load_2d(dst_w, &map_w, kb * BK, n0, bar_u8_full(s));
+                else tma_load_2d(dst_w, &map_w, n0, kb * BK, bar_u8_full(s));
+                tma_load_2d(dst_a, &map_act, kb * BK, 0, bar_u8_full(s));
+                issued = kb + 1;
+            }
+            if (*abort_flag) {  // let the copies already issued land before this CTA's shared memory goes away
+                for (int kb = max(0, issued - S); kb < issued; kb++) {
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(bar_u8_full(kb % S), (kb / S) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+                }
+            }
+        }
+    } else if (warp == kMmaWarp) {
+        if (lane == 0) {
+            // FP32 accumulator, BF16 operands; A = weight slab (K-major for [N,K] weights, MN-major for [K,N]), B = activations
+            // (K-major), N = mp, M = 128
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((W_IS_NK ? 0u : 1u) << 15) | ((uint32_t)(mp >> 3) << 17) |
+                                   ((uint32_t)(BM >> 4) << 24);
+            bool ok = true;
+            for (int kb = 0; kb < num_kb && ok; kb++) {
+                const int s = kb % S, round = kb / S;
+                ok = mbar_wait(bar_bf_full(s), round & 1, abort_flag, p.status, 32);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t w_addr = base + SmemLayoutN::bf + s * (kNwWBf + kNwABf), a_addr = w_addr + kNwWBf;
+#pragma unroll
+                for (int kk = 0; kk < BK / 16; kk++) {
+                    const uint64_t dw = W_IS_NK ? make_smem_desc(w_addr + kk * 32, 16, 1024) : make_smem_desc(w_addr + kk * 2048, 8192, 1024);
+                    const uint64_t da = make_smem_desc(a_addr + kk * 32, 16, 1024);
+                    tc_mma_bf16_cta(tmem_base, dw, da, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+                }
+                tc_commit_cta(bar_bf_empty(s));
+            }
+            if (ok) tc_commit_cta(bar_acc_full);
+        }
+    } else if (warp >= kFirstDecodeWarp) {
+        const int group = (warp - kFirstDecodeWarp) / kGroupWarps;
+        const int dt = threadIdx.x - (kFirstDecodeWarp + group * kGroupWarps) * 32;
+        const int act_chunks = mp * (BK / 8);  // 8-byte chunks of the activation tile
+        bool ok = true;
+        for (int kb = group; kb < num_kb && ok; kb += kDecodeGroups) {
+            const int s = group, r = kb / S;
+            ok = mbar_wait(bar_u8_full(s), r & 1, abort_flag, p.status, 33);
+            if (ok && r > 0) ok = mbar_wait(bar_bf_empty(s), (r - 1) & 1, abort_flag, p.status, 34);
+            if (!ok) break;
+            const uint32_t w8 = base + SmemLayoutN::u8 + s * (kNwW8 + kNwA8), a8 = w8 + kNwW8;
+            const uint32_t wbf = base + SmemLayoutN::bf + s * (kNwWBf + kNwABf), abf = wbf + kNwWBf;
+            uint2 vw[kChunksPerThread], va[kNarrowMaxM * (BK / 8) / kGroupThreads];
+            load_tile_chunks<!W_IS_NK>(w8, dt, vw);
+#pragma unroll
+            for (int it = 0; it < kNarrowMaxM * (BK / 8) / kGroupThreads; it++) {
+                const int q = it * kGroupThreads + dt;
+                if (q < act_chunks) va[it] = lds_v2(a8 + (q >> 3) * BK + (q & 7) * 8);
+            }
+            __syncwarp();  // the byte stage has been read: the producer may refill it during the decode
+            if (lane == 0) mbar_arrive(bar_u8_empty(s));
+            decode_tile_chunks<!W_IS_NK>(vw, wbf, dt, lut);
+#pragma unroll
+            for (int it = 0; it < kNarrowMaxM * (BK / 8) / kGroupThreads; it++) {
+                const int q = it * kGroupThreads + dt, row = q >> 3, j = q & 7;
+                if (q < act_chunks) sts_v4(abf + (row >> 3) * 1024 + (row & 7) * 128 + ((j ^ (row & 7)) << 4), decode8(va[it], lut));
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_bf_full(s));
+        }
+    } else {
+        // epilogue warps 0-3: TMEM lane = weight column n, TMEM column = activation row m
+        const bool ok = mbar_wait(bar_acc_full, 0, abort_flag, p.status, 35);
+        if (ok) {
+            tc_fence_after();
+            const int n = n0 + warp * 32 + lane;
+            const int sa = p.d_sa ? *p.d_sa : 0;
+            const int sw = p.d_sw_channel ? (n < p.N ? p.d_sw_channel[n] : 0) : (p.d_sw ? *p.d_sw : 0);
+            const int sc = -(sa + sw), s1 = sc / 2, s2 = sc - s1;
+            const float f1 = __uint_as_float((uint32_t)(s1 + 127) << 23), f2 = __uint_as_float((uint32_t)(s2 + 127) << 23);
+            for (int c = 0; c < mp; c += 32) {
+                uint32_t r[32];
+                tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(warp * 32) << 16) + c, r);
+                tmem_ld_wait();
+                if (n < p.N) {
+#pragma unroll
+                    for (int i = 0; i < 32; i++) {
+                        const int m = c + i;
+                        if (m >= p.M) break;
+                        float v = __uint_as_float(r[i]) * f1 * f2;
+                        if (p.c_is_f32) {
+                            float* out = reinterpret_cast<float*>(p.C) + (long long)m * p.ldc + n;
+                            *out = p.accumulate ? v + *out : v;
+                        } else {
+                            unsigned short* out = reinterpret_cast<unsigned short*>(p.C) + (long long)m * p.ldc + n;
+                            if (p.accumulate) v += __uint_as_float((uint32_t)*out << 16);
+                            const uint32_t u = __float_as_uint(v);
+                            *out = (unsigned short)((v != v) ? 0x7FC0u : ((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16));
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kMmaWarp) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemColsN) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------------
 // Decode-once path: operands already decoded to BF16 (by the conversion kernel of this library, into the caller's
 // workspace).  Persistent kernel, 64-wide k-blocks.
 //   warps 0-3  epilogue (TMEM -> global), overlapped with the next tile through two TMEM accumulators
@@ -807,6 +1005,10 @@ bool gemm_kernels_ready(int dev, int* sm_count_out)
             attr_rc = cudaFuncSetAttribute(fused[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         for (int i = 0; i < 2 && attr_rc == cudaSuccess; i++)
             attr_rc = cudaFuncSetAttribute(pair[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
+        if (attr_rc == cudaSuccess)
+            attr_rc = cudaFuncSetAttribute(hif8_gemm_narrow_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytesN);
+        if (attr_rc == cudaSuccess)
+            attr_rc = cudaFuncSetAttribute(hif8_gemm_narrow_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytesN);
         if (attr_rc == cudaSuccess) attr_rc = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
     });
     *sm_count_out = sm_count;
@@ -901,6 +1103,21 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t
 
     int sm_count = 0;
     if (!gemm_kernels_ready(dev, &sm_count)) return HIF8_ERR_CUDA;
+
+    // Narrow products: the weight-streaming kernel, whatever the workspace
+    if (!a_is_km && M <= kNarrowMaxM) {
+        const int mp = (M + 15) & ~15;
+        CUtensorMap map_act, map_ws;
+        if (!make_map(&map_act, Aq, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BK, (uint32_t)mp)) return HIF8_ERR_CUDA;
+        const bool okn = w_is_nk ? make_map(&map_ws, Wq, (uint64_t)K, (uint64_t)N, (uint64_t)ldw, BK, BM)
+                                 : make_map(&map_ws, Wq, (uint64_t)N, (uint64_t)K, (uint64_t)ldw, BM, BK);
+        if (!okn) return HIF8_ERR_CUDA;
+        const unsigned slabs = (unsigned)((N + BM - 1) / BM);
+        if (w_is_nk) hif8_gemm_narrow_kernel<true><<<slabs, kThreads, kSmemBytesN, st>>>(map_act, map_ws, p, mp);
+        else hif8_gemm_narrow_kernel<false><<<slabs, kThreads, kSmemBytesN, st>>>(map_act, map_ws, p, mp);
+        g_launches.fetch_add(1, std::memory_order_relaxed);
+        return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
+    }
 
     // Decode-once path: with room for both operands as BF16 in the workspace (and contiguous operands), each HiF8
     // byte is decoded exactly once by the conversion kernel and the tensor-core kernel reads BF16 tiles through TMA.

@@ -142,3 +142,43 @@ def test_bounded_wait_gives_up_and_reports_without_disturbing_the_device():
     Aq = np.full((M, K), 0x08, dtype=np.uint8)
     Wq = np.full((K, N), 0x10, dtype=np.uint8)
     assert np.all(run_gemm(Aq, Wq, 0, H.F32) == 2.0 * K)
+
+
+@pytest.mark.parametrize("w_is_nk", [0, 1])
+@pytest.mark.parametrize("c_dtype", [H.F32, H.BF16])
+@pytest.mark.parametrize("shape", [(1, 256, 64), (16, 1008, 272), (17, 640, 1040), (33, 128, 16), (64, 400, 208), (48, 2064, 4096)])
+def test_gemm_narrow_products(shape, c_dtype, w_is_nk):
+    # M <= 64: the weight-streaming kernel (weights as the 128-row tensor-core operand, C accumulated transposed)
+    M, N, K = shape
+    N16 = (N + 15) // 16 * 16
+    Aq = W.random_codes((M, K), seed=M + K)
+    Wkn = W.random_codes((K, N), seed=N + K + 3)
+    for t in (Aq, Wkn):
+        t[(t == 0x80) | ((t & 0x7F) == 0x6F)] = 0x33
+    if w_is_nk:
+        Wq = np.ascontiguousarray(Wkn.T)
+    else:
+        Wq = np.full((K, N16 + 16), 0x7B, dtype=np.uint8)     # padded leading dimension; the padding must not be read in
+        Wq[:, :N] = Wkn
+    Cs, S = O.gemm_full(Aq, Wkn, False, 3, -5)
+    out = run_gemm(Aq, Wq, w_is_nk, c_dtype, sa=3, sw=-5, M=M, N=N, K=K, ldw=Wq.shape[1])
+    check(out, Cs, S, c_dtype)
+
+
+def test_gemm_narrow_channel_scales_and_accumulate():
+    M, N, K = 24, 528, 272
+    Aq = W.random_codes((M, K), seed=1)
+    Wkn = W.random_codes((K, N), seed=2)
+    for t in (Aq, Wkn):
+        t[(t == 0x80) | ((t & 0x7F) == 0x6F)] = 0x33
+    sw = np.random.default_rng(3).integers(-20, 20, size=N).astype(np.int32)
+    c0 = (np.random.default_rng(4).standard_normal((M, N)) * 10).astype(np.float32)
+    C = torch.from_numpy(c0.copy()).cuda()
+    ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+    H.hif8_gemm_ex(to_dev(Aq), K, 0, to_dev(Wkn), N, 0, C, N, H.F32, M, N, K, torch.tensor([2], dtype=torch.int32, device="cuda"),
+                   None, to_dev(sw.view(np.uint32)), 1, ws, 256)
+    assert H.hif8_gemm_status(ws) == 0
+    rows, cols = np.divmod(np.arange(M * N), N)
+    P, S = O.gemm_entries_channel(Aq, Wkn, 0, 2, sw, rows, cols)
+    want = P.reshape(M, N) + c0
+    assert np.all(np.abs(C.cpu().numpy().astype(np.float64) - want) <= 1e-5 * S.reshape(M, N) + 2.0 ** -24 * np.abs(want))
