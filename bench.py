@@ -301,6 +301,17 @@ def extra_results(H, torch, hbm_peak, peak_kind):
     bw["wgrad_form_a_as_[K,M]_fp32_accumulate"] = {"ms": ms_w, "TFLOPs": flops / ms_w / 1e9, "frac": flops / ms_w / 1e9 / tf_peak,
                                                    "device_status": H.hif8_gemm_status(gws)}
     del C32
+    # inference-decode shapes: a few activation rows against the same weight (bound by reading the weight bytes once)
+    narrow = {}
+    for Mn in (16, 64):
+        Cn = torch.empty(Mn, N, dtype=torch.bfloat16, device="cuda")
+        ms_n = timed(lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, Cn, N, H.BF16, Mn, N, K, se[0:1], se[1:2], gws, 256), 20)
+        byt = K * N + Mn * K + 2 * Mn * N
+        narrow[f"M={Mn}"] = {"us": ms_n * 1e3, "GBps": byt / ms_n / 1e6, "frac_of_hbm": byt / ms_n / 1e6 / hbm_peak,
+                             "device_status": H.hif8_gemm_status(gws)}
+        del Cn
+    out["gemm_narrow_Mx28672x8192"] = {"bound": "hbm", "bytes": "K*N weight bytes + M*K + 2*M*N", "shapes": narrow,
+                                       "peak": hbm_peak, "peak_kind": f"of {peak_kind}"}
     out["gemm_8192x28672x8192"] = {
         "backward_forms": bw,
         "decode_once_channel_scaled": {"ms": ms_c, "TFLOPs": flops / ms_c / 1e9, "frac": flops / ms_c / 1e9 / tf_peak,
