@@ -28,7 +28,8 @@
  *                            scales; the every-N-iterations amax cadence.
  *
  * Readings taken where the paper is silent are marked "READING" below.
- * Pin status: every function here is pinned by tests/test_oracle_pins.py
+ * Pin status: the later additions (per-channel scaling, the amax cadence, backward-pass operand forms, adaptive loss
+ * scaling) are pinned by tests/test_oracle_pins_scaling.py; every other function here is pinned by tests/test_oracle_pins.py
  * against values the paper prints (Table 4 patterns, the abstract's counts,
  * the TE/TA worked example, the 0.5 / 0.75 / 1 ulp error bounds, the 2^-20 tie
  * probability, the SR expectation identity) and by closed forms.  The bit-level
