@@ -35,7 +35,7 @@ POOL = 6                  # rotating buffer sets: 6 x 64 MiB of input alone exce
 WORKLOAD = "fp32_4096x4096_normal_amax_scale_encode_then_decode"
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture summarised in profiles/;
 # None for a kernel changed since its capture
-TRAFFIC = {"amax_kernel<f32>": 67.46e6, "convert_kernel<f32,TA>": 69.12e6, "decode_kernel<f32>": 26.74e6}
+TRAFFIC = {"amax_kernel<f32>": 67.64e6, "convert_kernel<f32,TA>": 69.68e6, "decode_kernel<f32>": 26.26e6}
 METRIC = "hif8_encode_decode_throughput"
 UNIT = "GB/s"
 
