@@ -495,3 +495,24 @@ def test_pts_search_against_definition_and_scale_shift_property():
     assert np.allclose(errq, err, rtol=1e-12) and bestq == best      # (the parallel sum order is not fixed)
     errt, _ = O.pts_search(a, np.ascontiguousarray(w.T), O.BF16, True, Oref, -4, 5)
     assert np.allclose(errt, err, rtol=1e-12)
+
+
+def test_significand_bits_over_exponent_profile():
+    """The content of the paper's Fig. 1 (significand bits as a function of the exponent), recomputed from the decoded
+    values alone: in every binade the positive finite values are 2^E * (1 + j / 2^w), j = 0 .. 2^w - 1, which gives the
+    mantissa width w of that binade; the profile must be the tapered, symmetric one of Table 3 with the denormal tail."""
+    import math
+    vals = sorted({O.value(c) for c in range(128) if O.parse(c)["kind"] == 1})
+    by_exp = {}
+    for v in vals:
+        by_exp.setdefault(math.floor(math.log2(v)), []).append(v)
+    assert sorted(by_exp) == list(range(-22, 16))                          # 38 binades, none missing
+    profile = {}
+    for E, vs in by_exp.items():
+        w = round(math.log2(len(vs))) if E != 15 else 1                    # the top binade loses its second value to Inf
+        assert len(vs) == (2 ** w if E != 15 else 1)
+        assert vs == [2.0 ** E * (1 + j / 2 ** w) for j in range(len(vs))]  # equally spaced: Eq. 1 with a w-bit mantissa
+        profile[E] = w
+    expect = {E: (0 if E <= -16 else 3 if abs(E) <= 3 else 2 if abs(E) <= 7 else 1) for E in range(-22, 16)}
+    assert profile == expect
+    print("significand bits (1 + mantissa) by exponent:", {E: 1 + w for E, w in profile.items()})
