@@ -213,7 +213,9 @@ template <int DT> __device__ __forceinline__ uint32_t to_bits(float v)
 // ------------------------------------------------------------------------------------------------
 // Rounding table thr[], indexed by the biased exponent of the scaled value (never by its sign: values of either sign would
 // otherwise hit different words of the same bank).
-//  * TE / SR: thr[e] = sh, the number of discarded mantissa bits (23 - width; 0: nothing to round).
+//  * SR: thr[e] = sh, the number of discarded mantissa bits (23 - width; 0: nothing to round).
+//  * TE: thr[e] = half - 1 (bits 0-22; half itself where no mantissa bit is kept: the implicit one is odd), bit 26 "add
+//    the kept LSB", sh in bits 27-31; the binade of 2^-23 adds 2^23 - 1 (anything above the tie carries into 2^-22).
 //  * Hybrid / simplified stochastic rounding adds an increment to the bit pattern so that the carry out of the discarded
 //    field rounds up (also across binade and width boundaries), clears the old binade's discarded bits (~0 << sh) and
 //    reads the code from the truncating table.
@@ -254,16 +256,25 @@ __device__ __forceinline__ uint32_t encode_one(float x, uint32_t raw, float scal
         }
     }
 
+    if (MODE == HIF8_RND_TE) {
+        // round half to even as one increment: half - 1 plus the kept LSB (the carry rounds up exactly when the discarded
+        // field exceeds one half, or equals it with an odd kept significand); s_ta is the truncating table with 2^-23 -> 0
+        const uint32_t ent = s_thr[(t >> 23) & 0xFFu];  // bits 0-22 constant, bit 26 "add the kept LSB", bits 27-31 sh
+        const uint32_t sh = ent >> 27;
+        const uint32_t lsb = (t >> sh) & (ent >> 26) & 1u;
+        return s_ta[((t + (ent & 0x03FFFFFFu) + lsb) & (0xFFFFFFFFu << sh)) >> 19];
+    }
+
     const bool sub = (t & 0x7FFFFFFFu) < 0x34800000u;  // |y| < 2^-22 (zero included): result is 0 or 2^-22
     // Below 2^-22 the kept bits are zero and the fraction is F = |y| / 2^-22.  Adding 2^-22 with truncation puts
     // floor(F 2^23) into the mantissa field of a value in the binade of 2^-22, so the common code rounds it like a
     // 0-bit-mantissa binade (result 2^-22 or 2^-21); it is moved down again afterwards.
     const uint32_t tz = __float_as_uint(__fadd_rz(fabsf(y), 2.384185791015625e-07f));
 
-    // TE and standard SR
+    // standard SR
     constexpr int kSrBits = (SRC == HIF8_F32) ? 24 : 16;
     const uint32_t sign7 = (t >> 24) & 0x80u;
-    if (MODE == HIF8_RND_SR && SRC == HIF8_F32 && sub) {
+    if (SRC == HIF8_F32 && sub) {
         // the 24-bit threshold is wider than a binary32 fraction: compare F24 = floor(|y| 2^46) directly
         const uint32_t f24 = __float2uint_rz(fabsf(y) * 70368744177664.f);
         return f24 >= max(word >> 8, 1u) ? (sign7 | 0x01u) : 0u;
@@ -271,28 +282,17 @@ __device__ __forceinline__ uint32_t encode_one(float x, uint32_t raw, float scal
     t = sub ? (tz | (t & 0x80000000u)) : t;
     const uint32_t sh = s_thr[(t >> 23) & 0xFFu];  // discarded mantissa bits (23 - width); 0: nothing to round
     const uint32_t s = sh ? sh : 23u;
+    // threshold T of Section 3.2, compared as max(T,1) so that a zero fraction never rounds up
+    const uint32_t T = max(word >> (32 - kSrBits), 1u);
     uint32_t inc;
-    if (MODE == HIF8_RND_TE) {
-        // add half-1, plus one when the kept significand is odd (the implicit one when no mantissa bit is kept,
-        // zero below 2^-22)
-        uint32_t lsb = (s == 23u) ? 1u : ((t >> s) & 1u);
-        if (sub) lsb = 0u;
-        inc = (1u << (s - 1)) - 1u + lsb;
-    } else {  // standard SR (threshold T of Section 3.2, compared as max(T,1) so that a zero fraction never rounds up)
-        const uint32_t T = max(word >> (32 - kSrBits), 1u);
-        if (SRC == HIF8_F32) {
-            const uint32_t k = 24u - s;  // F24 = discarded << k; up iff discarded >= ceil(T / 2^k)
-            inc = (1u << s) - ((T + (1u << k) - 1u) >> k);
-        } else inc = (0x10000u - T) << (s - 16);
-    }
+    if (SRC == HIF8_F32) {
+        const uint32_t k = 24u - s;  // F24 = discarded << k; up iff discarded >= ceil(T / 2^k)
+        inc = (1u << s) - ((T + (1u << k) - 1u) >> k);
+    } else inc = (0x10000u - T) << (s - 16);
     if (sh == 0) inc = 0;
     const uint32_t tr = (t + inc) & (0xFFFFFFFFu << sh);
     uint32_t code = s_ta[tr >> 19];
-    if (sub) {
-        if (MODE == HIF8_RND_TE)  // nearest: up iff above the midpoint 2^-23 (the tie goes to the even value, zero)
-            code = (__float_as_uint(y) & 0x7FFFFFFFu) > 0x34000000u ? (sign7 | 0x01u) : 0u;
-        else code = ((code & 0x7Fu) == 0x02u) ? (sign7 | 0x01u) : 0u;  // 2^-21 -> 2^-22, 2^-22 -> the single zero
-    }
+    if (sub) code = ((code & 0x7Fu) == 0x02u) ? (sign7 | 0x01u) : 0u;  // 2^-21 -> 2^-22, 2^-22 -> the single zero
     return code;
 }
 
@@ -312,12 +312,14 @@ __device__ __forceinline__ void setup_tables(SmemTables& s, unsigned flags)
         // Only binades 2^-24 .. 2^16 differ from their neighbours: those 41 x 16 entries per sign come from the
         // compile-time table (1.3 KiB of global reads per block); everything below is zero, everything above is
         // Inf (or NaN in the all-ones exponent), written straight into shared memory.
-        const uint4* g = reinterpret_cast<const uint4*>((MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR) ? g_trunc_table.v : g_ta_table.v);
+        constexpr bool kTrunc = MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR || MODE == HIF8_RND_TE;  // modes that round before the lookup
+        const uint4* g = reinterpret_cast<const uint4*>(kTrunc ? g_trunc_table.v : g_ta_table.v);
         uint4* d = reinterpret_cast<uint4*>(s.ta);
         for (int i = threadIdx.x; i < 512; i += kThreads) {
             const uint32_t e = i & 255, inf = ((uint32_t)(i >> 8) << 7) | 0x6Fu;
             uint4 v;
             if (e < 103) v = make_uint4(0, 0, 0, 0);
+            else if (MODE == HIF8_RND_TE && e == 104) v = make_uint4(0, 0, 0, 0);  // TE: what is left in the binade of 2^-23 is the exact tie
             else if (e <= 143) v = g[i];
             else if (e < 255) { uint32_t w = inf * 0x01010101u; v = make_uint4(w, w, w, w); }
             else v = make_uint4(0x80808000u | inf, 0x80808080u, 0x80808080u, 0x80808080u);
@@ -350,13 +352,16 @@ __device__ __forceinline__ void setup_tables(SmemTables& s, unsigned flags)
         if (E < 16 && E >= -22) {
             const uint32_t sh = 23u - (uint32_t)mant_width(E);
             const bool stochastic = MODE == HIF8_RND_SSR || E <= -4 || E >= 4;  // Eq. 3 for HR
-            if (!kThreshold) e0 = sh;  // TE / SR: only the width is read
+            if (MODE == HIF8_RND_TE) e0 = (sh == 23u ? (1u << 22) : ((1u << (sh - 1u)) - 1u) | (1u << 26)) | (sh << 27);
+            else if (!kThreshold) e0 = sh;  // SR: only the width is read
             else if (kF32) {
                 if (stochastic) e0 = 1u << (sh - 14u); else e1 = 1u << (sh - 1u);
                 e1 |= sh << 27;
             }
             else if (stochastic) { e0 = (3u << (sh - 2u)) | sh; e1 = (1u << (sh - 2u)) | sh; }  // complement 3 - 2 LSB
             else e0 = e1 = (1u << (sh - 1u)) | sh;
+        } else if (MODE == HIF8_RND_TE && E == -23) {
+            e0 = ((1u << 23) - 1u) | (23u << 27);  // above 2^-23 -> carry -> 2^-22; exactly 2^-23 stays (-> 0 in TE's table)
         } else if (kThreshold && kF32 && E == -24) {
             e0 = 1u << 9; e1 = 23u << 27;  // where encode_one parks FP32 elements below 2^-22
         } else if (kThreshold && !kF32 && (E == -23 || E == -24)) {
