@@ -430,14 +430,15 @@ def main():
 
     # ---- timed region: device-resident inputs, CUDA events on the launching stream.
     # The launch sequence of POOL consecutive steps (one per buffer set) is captured once in a CUDA graph and
-    # replayed, so the host's per-launch cost stays out of the device timeline; K steps = K // POOL replays plus
-    # K % POOL directly launched steps.
-    K = max(POOL, args.steps // POOL * POOL)   # whole graph replays: the step count is rounded down to a multiple of POOL
+    # replayed, so the host's per-launch cost stays out of the device timeline; K steps = K // POOL replays of that
+    # graph plus one replay of a second graph holding the remaining K % POOL steps, so exactly K steps are timed.
+    K = max(1, args.steps)
+    W_REPLAYS = max(1, -(-args.warmup // POOL))   # warm-up in whole replays: at least args.warmup steps
     ws2 = [ws, torch.empty(max(wsb, 256), dtype=torch.uint8, device="cuda")]
     scal2 = [scal, torch.zeros(4, dtype=torch.int32, device="cuda")]
 
-    def capture(two_streams):
-        """POOL consecutive steps in one graph.  With two_streams, even and odd steps (independent tensors, separate
+    def capture(two_streams, nsteps=POOL):
+        """nsteps consecutive steps in one graph.  With two_streams, even and odd steps (independent tensors, separate
         workspaces) are enqueued on two streams, so the ramp and drain of one step's kernels overlap the other's."""
         gr = torch.cuda.CUDAGraph()
         with torch.cuda.graph(gr):
@@ -445,7 +446,7 @@ def main():
             side_s = torch.cuda.Stream() if two_streams else main_s
             if two_streams:
                 side_s.wait_stream(main_s)
-            for i in range(POOL):
+            for i in range(nsteps):
                 st = (main_s, side_s)[i & 1]
                 cs = st.cuda_stream
                 H.hif8_amax_scale_encode(srcs[i], H.F32, codes[i], N_EL, 14, H.RND_TA, 0, 0, None, scal2[i & 1][0:1],
@@ -455,30 +456,39 @@ def main():
                 main_s.wait_stream(side_s)
         return gr
 
-    def time_graph(gr):
-        for _ in range(max(1, args.warmup // POOL)):
+    def replay_steps(gr, tail):
+        for _ in range(K // POOL):
             gr.replay()
+        if tail is not None:
+            tail.replay()
+
+    def time_graph(gr, tail):
+        for _ in range(W_REPLAYS):
+            gr.replay()
+        if tail is not None:
+            tail.replay()
         torch.cuda.synchronize()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record(stream)
-        for _ in range(K // POOL):
-            gr.replay()
+        replay_steps(gr, tail)
         b.record(stream)
         torch.cuda.synchronize()
-        return a.elapsed_time(b) / max(1, (K // POOL) * POOL)
+        return a.elapsed_time(b) / K
 
-    serial_ms = time_graph(capture(False))     # one stream: every kernel waits for the previous one to drain
+    # one stream: every kernel waits for the previous one to drain
+    serial_ms = time_graph(capture(False), capture(False, K % POOL) if K % POOL else None)
     graph = capture(True)
-    for _ in range(max(1, args.warmup // POOL)):
+    graph_tail = capture(True, K % POOL) if K % POOL else None
+    for _ in range(W_REPLAYS):
         graph.replay()
+    if graph_tail is not None:
+        graph_tail.replay()
     torch.cuda.synchronize()
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    launches0 = H.hif8_launch_count()
     barrier()
     with ClockSampler(local) as clk:
         t0.record(stream)
-        for _ in range(K // POOL):
-            graph.replay()
+        replay_steps(graph, graph_tail)
         t1.record(stream)
         torch.cuda.synchronize()
         # per-kernel durations, measured live: each kernel of the step in a graph of its own (POOL launches over the
@@ -493,7 +503,7 @@ def main():
                 cs = torch.cuda.current_stream().cuda_stream
                 for i in range(POOL):
                     call(i, cs)
-            R = max(4, min(K, 600) // POOL)
+            R = max(4, min(K, 600) // POOL)   # own repeat count: these are per-kernel figures, not the timed K steps
             for _ in range(3):
                 gk.replay()
             torch.cuda.synchronize()
@@ -511,7 +521,7 @@ def main():
         enc_ms = kernel_ms(lambda i, cs: H.hif8_amax_scale_encode(srcs[i], H.F32, codes[i], N_EL, 14, H.RND_TA, 0, 0, None,
                                                                   scal[0:1], scal[1:2], scal[2:3], ws, wsb, stream=cs))
     barrier()
-    launches = 3 * POOL * (K // POOL)   # amax + convert + decode kernels per step (graph replays)
+    launches = 3 * K   # amax + convert + decode kernels per step (graph replays)
     total_ms = t0.elapsed_time(t1)
 
     # ---- end to end: pinned host input -> device, both calls, results back to pinned host memory.  Consecutive
@@ -578,7 +588,8 @@ def main():
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "u8", "data": "synthetic",
             "config": {"workload": WORKLOAD, "elements": N_EL, "rounding": "TA", "target_exp": 14,
-                       "launch": "CUDA graph of 6 steps replayed; even/odd steps (independent tensors) on two streams",
+                       "launch": f"CUDA graph of {POOL} steps replayed (+ one graph of steps % {POOL}); even/odd steps "
+                                 "(independent tensors) on two streams",
                        "ms_per_step_single_stream": serial_ms,
                        "l2": f"inputs rotate over {POOL} buffer sets ({POOL * N_EL * 4 >> 20} MiB of sources) > 126 MB L2",
                        "bytes_per_step": BYTES_STEP, "elements_per_s": world * N_EL / (ms_per_step * 1e-3)},
