@@ -4,8 +4,8 @@
 // A block converts a tile of 128 source rows by 8 source vectors (32 FP32 or 64 16-bit columns).  Thread (rq, cv)
 // loads the four vectors of rows 4 rq .. 4 rq + 3 in vector-column cv (four independent 16-byte loads; a warp covers
 // four full 128-byte lines per instruction), converts them, and packs the four bytes of each of its columns into one
-// 32-bit word of a shared tile held transposed ([column][row / 4], row stride 33 words: conflict-free for FP32,
-// two-way for 16-bit sources).  The block then writes each column of the tile as 128 contiguous bytes of a dst row.
+// 32-bit word of a shared tile held transposed ([column][row / 4], 16-byte chunks XOR-swizzled by the column's vector
+// index: conflict-free both ways).  The block then writes each column of the tile as 128 contiguous bytes of a dst row.
 // Traffic is that of the flat encoder: one read of the source, one byte written per element.
 #include <cuda_runtime.h>
 
@@ -32,69 +32,88 @@ struct TrParams {
 
 constexpr int kTileRows = 128;
 constexpr int kTileVecs = 8;          // vector-columns per tile
-constexpr int kTileStride = kTileRows / 4 + 1;  // words per tile column
+constexpr int kTileWords = kTileRows / 4;  // words per tile column (128 code bytes)
 
+// Grid: x = tile of 128 source rows, y = strip of 8 source vectors (looped when there are more strips than the grid's
+// y extent).  Blocks with consecutive x write adjacent 128-byte segments of the same dst rows.
 template <int SRC, int MODE>
-__global__ void __launch_bounds__(kThreads) encode_transpose_kernel(const TrParams p)
+__global__ void __launch_bounds__(kThreads, MODE == HIF8_RND_SR ? 4 : 6) encode_transpose_kernel(const TrParams p)
 {
     constexpr int PV = SrcTraits<SRC>::kPerVec;
     constexpr int TC = kTileVecs * PV;  // source columns per tile
     __shared__ SmemTables sm;
-    __shared__ uint32_t tile[TC * kTileStride];
+    // tile[c][w]: code bytes of source column c, rows 4w .. 4w+3 in word w; the 16-byte chunk index (w / 4) is XORed
+    // with the column's vector index so that both the word stores below and the 16-byte reads are conflict-free
+    __shared__ __align__(16) uint32_t tile[TC * kTileWords];
     setup_tables<true, MODE != HIF8_RND_TA, false, MODE, SRC>(sm, p.flags);
     const float scale = pow2f(p.d_scale_exp ? clamp_exp(*p.d_scale_exp) : p.scale_exp);
     const uint32_t k0 = (uint32_t)p.seed, k1 = (uint32_t)(p.seed >> 32);
     const long long nvc = p.cols / PV;                        // vectors per source row
-    const long long tiles_c = (nvc + kTileVecs - 1) / kTileVecs;
-    const long long tiles_r = (p.rows + kTileRows - 1) / kTileRows;
+    const long long strips = (nvc + kTileVecs - 1) / kTileVecs;
     const int cv = threadIdx.x % kTileVecs, rq = threadIdx.x / kTileVecs;
-    const uint4* src = reinterpret_cast<const uint4*>(p.src);
+    const long long r0 = (long long)blockIdx.x * kTileRows;
+    const bool rows_full = r0 + kTileRows <= p.rows;
+    uint32_t* const my_words = tile + cv * PV * kTileWords + (((rq >> 2) ^ cv) << 2) + (rq & 3);
 
-    for (long long tix = blockIdx.x; tix < tiles_c * tiles_r; tix += gridDim.x) {
-        // consecutive blocks take consecutive row-tiles of one column strip: their dst segments are adjacent
-        const long long tc = tix / tiles_r, tr = tix % tiles_r;
-        const long long r0 = tr * kTileRows, v0 = tc * kTileVecs;
-        const long long vcol = v0 + cv;
+    for (long long tc = blockIdx.y; tc < strips; tc += gridDim.y) {
+        const long long v0 = tc * kTileVecs, vcol = v0 + cv;
+        const bool full = rows_full && v0 + kTileVecs <= nvc;
+        const uint4* sp = reinterpret_cast<const uint4*>(p.src) + (r0 + rq * 4) * nvc + vcol;
         uint4 v[4];
+        if (full) {
 #pragma unroll
-        for (int j = 0; j < 4; j++) {
-            const long long r = r0 + rq * 4 + j;
-            v[j] = (r < p.rows && vcol < nvc) ? __ldcs(src + r * nvc + vcol) : make_uint4(0, 0, 0, 0);
+            for (int j = 0; j < 4; j++) v[j] = __ldcs(sp + j * nvc);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; j++)
+                v[j] = (r0 + rq * 4 + j < p.rows && vcol < nvc) ? __ldcs(sp + j * nvc) : make_uint4(0, 0, 0, 0);
         }
-        uint32_t packed[PV];
+        if (MODE == HIF8_RND_SR) {
+            // one generator call serves a whole source vector: rows outermost, the words of all columns accumulate
+            uint32_t packed[PV];
 #pragma unroll
-        for (int k = 0; k < PV; k++) packed[k] = 0;
-#pragma unroll
-        for (int j = 0; j < 4; j++) {
-            const long long r = r0 + rq * 4 + j;
-            uint32_t rw[8];
-            uint4 q0 = make_uint4(0, 0, 0, 0), q1 = q0;
-            if (MODE == HIF8_RND_SR) {
-                const unsigned long long u = (unsigned long long)r * nvc + vcol;  // flat vector index in the source
-                q0 = philox4x32_10((uint32_t)(u * (PV / 4)), (uint32_t)((u * (PV / 4)) >> 32), k0, k1);
+            for (int j = 0; j < 4; j++) {
+                const unsigned long long u = (unsigned long long)(r0 + rq * 4 + j) * nvc + vcol;  // flat vector index in the source
+                uint4 q0 = philox4x32_10((uint32_t)(u * (PV / 4)), (uint32_t)((u * (PV / 4)) >> 32), k0, k1), q1 = q0;
                 if (PV == 8) q1 = philox4x32_10((uint32_t)(u * 2 + 1), (uint32_t)((u * 2 + 1) >> 32), k0, k1);
+                const uint32_t rw[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+#pragma unroll
+                for (int k = 0; k < PV; k++) {
+                    float x; uint32_t raw;
+                    unpack<SRC>(v[j], k, x, raw);
+                    const uint32_t c = encode_one<MODE, SRC>(x, raw, scale, sm.ta, sm.thr, rw[k]) << (8 * j);
+                    packed[k] = j ? (packed[k] | c) : c;
+                }
             }
-            rw[0] = q0.x; rw[1] = q0.y; rw[2] = q0.z; rw[3] = q0.w; rw[4] = q1.x; rw[5] = q1.y; rw[6] = q1.z; rw[7] = q1.w;
+#pragma unroll
+            for (int k = 0; k < PV; k++) my_words[k * kTileWords] = packed[k];
+        } else {
+            // columns outermost: the four codes of a column are packed and stored at once
 #pragma unroll
             for (int k = 0; k < PV; k++) {
-                float x; uint32_t raw;
-                unpack<SRC>(v[j], k, x, raw);
-                packed[k] |= encode_one<MODE, SRC>(x, raw, scale, sm.ta, sm.thr, rw[k]) << (8 * j);
+                uint32_t c[4];
+#pragma unroll
+                for (int j = 0; j < 4; j++) {
+                    float x; uint32_t raw;
+                    unpack<SRC>(v[j], k, x, raw);
+                    c[j] = encode_one<MODE, SRC>(x, raw, scale, sm.ta, sm.thr, 0u);
+                }
+                my_words[k * kTileWords] = c[0] | (c[1] << 8) | (c[2] << 16) | (c[3] << 24);
             }
         }
-        __syncthreads();  // the previous tile has been written out
-#pragma unroll
-        for (int k = 0; k < PV; k++) tile[(cv * PV + k) * kTileStride + rq] = packed[k];
         __syncthreads();
         // column c of the tile = 128 bytes of dst row (v0 * PV + c), starting at byte r0; 16 bytes per thread
-        for (int o = threadIdx.x; o < TC * (kTileRows / 16); o += kThreads) {
-            const int c = o / (kTileRows / 16), seg = o % (kTileRows / 16);
-            const long long col = v0 * PV + c, r = r0 + seg * 16;
-            if (col < p.cols && r < p.rows) {  // rows is a multiple of 16 on this path: a segment is all in or all out
-                const uint32_t* w = tile + c * kTileStride + seg * 4;
-                __stcs(reinterpret_cast<uint4*>(p.dst + col * p.rows + r), make_uint4(w[0], w[1], w[2], w[3]));
-            }
+        constexpr int kSegs = kTileRows / 16;
+        const int seg = threadIdx.x % kSegs, c_lo = threadIdx.x / kSegs;
+        uint8_t* dp = p.dst + (v0 * PV + c_lo) * p.rows + r0 + seg * 16;
+#pragma unroll
+        for (int i = 0; i < TC * kSegs / kThreads; i++) {
+            const int c = c_lo + i * (kThreads / kSegs);
+            const uint4 q = *reinterpret_cast<const uint4*>(tile + c * kTileWords + ((seg ^ ((c / PV) & 7)) << 2));
+            // rows is a multiple of 16 on this path: a segment is all in or all out
+            if (full || (v0 * PV + c < p.cols && r0 + seg * 16 < p.rows)) __stcs(reinterpret_cast<uint4*>(dp + (long long)i * (kThreads / kSegs) * p.rows), q);
         }
+        if (tc + gridDim.y < strips) __syncthreads();  // (block-uniform) the tile is read out before the next one is stored
     }
 }
 
@@ -169,8 +188,10 @@ int launch(const TrParams& p, bool vec, int sms, cudaStream_t st)
     if (vec) {
         constexpr int PV = SrcTraits<SRC>::kPerVec;
         const long long nvc = p.cols / PV;
-        const long long tiles = ((nvc + kTileVecs - 1) / kTileVecs) * ((p.rows + kTileRows - 1) / kTileRows);
-        encode_transpose_kernel<SRC, MODE><<<(unsigned)(tiles < 0x7FFFFFFFll ? tiles : 0x7FFFFFFFll), kThreads, 0, st>>>(p);
+        const long long strips = (nvc + kTileVecs - 1) / kTileVecs, row_tiles = (p.rows + kTileRows - 1) / kTileRows;
+        if (row_tiles > 0x7FFFFFFFll) return HIF8_ERR_SHAPE;
+        const dim3 grid((unsigned)row_tiles, (unsigned)(strips < 65535 ? strips : 65535));
+        encode_transpose_kernel<SRC, MODE><<<grid, kThreads, 0, st>>>(p);
     } else {
         const unsigned long long n = (unsigned long long)p.rows * (unsigned long long)p.cols;
         const unsigned long long need = (n + kThreads - 1) / kThreads, cap = (unsigned long long)sms * 32;

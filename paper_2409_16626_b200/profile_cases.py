@@ -6,7 +6,8 @@ cases: convert_f32 (FP32 4096^2: per-tensor scaled encode + decode), fq_bf16 (BF
 fused amax and given scale), encode_modes_f32 / encode_modes_bf16 (2^25 log-uniform values, every rounding mode), gemm (HiF8 GEMM
 4096 x 7168 x 4096, fused and decode-once paths), gemm_forms (same size, decode-once path, the four operand layouts:
 forward, dgrad form, wgrad form with FP32 accumulation, both transposed), channel_bf16 (per-channel scaled encode of a
-BF16 8192 x 14336 weight, channel = column and channel = row, plus the overflow check of the same tensor).  Inputs are seeded device-side random tensors.
+BF16 8192 x 14336 weight, channel = column and channel = row, plus the overflow check of the same tensor), transpose_bf16
+(BF16 8192 x 8192 to HiF8 bytes, flat and with transposed store, round half away and hybrid rounding).  Inputs are seeded device-side random tensors.
 """
 import sys
 
@@ -56,6 +57,14 @@ def main():
         for r in range(reps):
             for mode in (H.RND_TA, H.RND_HR, H.RND_SSR, H.RND_TE, H.RND_SR):
                 H.hif8_encode(bits, H.BF16, codes, n, 0, mode, 0, 5)
+    elif case == "transpose_bf16":
+        R, C = 8192, 8192
+        xs = [torch.randn(R * C, generator=g, device="cuda").to(torch.bfloat16) for _ in range(2)]
+        codes = torch.empty(R * C, dtype=torch.uint8, device="cuda")
+        for r in range(reps):
+            for mode in (H.RND_TA, H.RND_HR):
+                H.hif8_encode(xs[r & 1], H.BF16, codes, R * C, 3, mode, 0, 5)
+                H.hif8_encode_transpose(xs[r & 1], H.BF16, codes, R, C, 3, None, mode)
     elif case == "gemm":
         M, N, K = 4096, 7168, 4096
         A = torch.randint(0, 256, (M, K), dtype=torch.uint8, device="cuda", generator=g)
