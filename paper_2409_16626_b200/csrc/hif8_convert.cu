@@ -36,6 +36,57 @@ std::atomic<uint64_t> g_launches{0};
 
 namespace {
 
+// One group of kUnroll vectors per thread starting at vector index `base`.  FULL: the whole group lies inside the
+// tensor, so no bounds are checked.
+template <int SRC, int MODE, bool FQ, bool AMAX, bool FULL>
+__device__ __forceinline__ void convert_group(const ConvParams& p, const SmemTables& sm, unsigned long long base, unsigned long long n_vec,
+                                              float scale, float d1, float d2, uint32_t k0, uint32_t k1, float& amax)
+{
+    constexpr int PV = SrcTraits<SRC>::kPerVec;
+    const uint4* src = reinterpret_cast<const uint4*>(p.src);
+    uint4 v[kUnroll];
+#pragma unroll
+    for (int j = 0; j < kUnroll; j++) {
+        unsigned long long u = base + (unsigned long long)j * kThreads + threadIdx.x;
+        if (FULL || u < n_vec) v[j] = __ldcs(src + u); else v[j] = make_uint4(0, 0, 0, 0);
+    }
+#pragma unroll
+    for (int j = 0; j < kUnroll; j++) {
+        unsigned long long u = base + (unsigned long long)j * kThreads + threadIdx.x;
+        if (!FULL && u >= n_vec) continue;
+        uint32_t codes[PV];
+        uint4 r0 = make_uint4(0, 0, 0, 0), r1 = r0;
+        if (MODE == HIF8_RND_SR) {
+            r0 = philox4x32_10((uint32_t)(u * (PV / 4)), (uint32_t)((u * (PV / 4)) >> 32), k0, k1);
+            if (PV == 8) r1 = philox4x32_10((uint32_t)(u * 2 + 1), (uint32_t)((u * 2 + 1) >> 32), k0, k1);
+        }
+        const uint32_t rw[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
+#pragma unroll
+        for (int k = 0; k < PV; k++) {
+            float x; uint32_t raw;
+            unpack<SRC>(v[j], k, x, raw);
+            if (AMAX) amax = amax_step(amax, x);
+            codes[k] = encode_one<MODE, SRC>(x, raw, scale, sm.ta, sm.thr, rw[k]);
+        }
+        if (!FQ) {
+            uint32_t w0 = codes[0] | (codes[1] << 8) | (codes[2] << 16) | (codes[3] << 24);
+            if (PV == 4) __stcs(reinterpret_cast<uint32_t*>(p.dst) + u, w0);
+            else {
+                uint32_t w1 = codes[4] | (codes[5] << 8) | (codes[6] << 16) | (codes[7] << 24);
+                __stcs(reinterpret_cast<uint2*>(p.dst) + u, make_uint2(w0, w1));
+            }
+        } else {
+            uint32_t o[PV];
+#pragma unroll
+            for (int k = 0; k < PV; k++) o[k] = to_bits<SRC>(sm.dec[codes[k]] * d1 * d2);
+            uint4 out;
+            if (PV == 4) out = make_uint4(o[0], o[1], o[2], o[3]);
+            else out = make_uint4(o[0] | (o[1] << 16), o[2] | (o[3] << 16), o[4] | (o[5] << 16), o[6] | (o[7] << 16));
+            __stcs(reinterpret_cast<uint4*>(p.dst) + u, out);
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // Encode / fake-quant kernel.  FQ = false: bytes out.  FQ = true: dequantized values in the source format.
 // AMAX = true: also reduce amax of the source into p.amax_accum[0]; the last block publishes it.
@@ -55,50 +106,12 @@ __global__ void __launch_bounds__(kThreads) convert_kernel(const ConvParams p, u
     const uint32_t k0 = (uint32_t)p.seed, k1 = (uint32_t)(p.seed >> 32);
     float amax = 0.f;
 
-    const uint4* src = reinterpret_cast<const uint4*>(p.src);
     const unsigned long long stride = (unsigned long long)gridDim.x * kThreads * kUnroll;
     for (unsigned long long base = (unsigned long long)blockIdx.x * kThreads * kUnroll; base < n_vec; base += stride) {
-        uint4 v[kUnroll];
-#pragma unroll
-        for (int j = 0; j < kUnroll; j++) {
-            unsigned long long u = base + (unsigned long long)j * kThreads + threadIdx.x;
-            if (u < n_vec) v[j] = __ldcs(src + u); else v[j] = make_uint4(0, 0, 0, 0);
-        }
-#pragma unroll
-        for (int j = 0; j < kUnroll; j++) {
-            unsigned long long u = base + (unsigned long long)j * kThreads + threadIdx.x;
-            if (u >= n_vec) continue;
-            uint32_t codes[PV];
-            uint4 r0 = make_uint4(0, 0, 0, 0), r1 = r0;
-            if (MODE == HIF8_RND_SR) {
-                r0 = philox4x32_10((uint32_t)(u * (PV / 4)), (uint32_t)((u * (PV / 4)) >> 32), k0, k1);
-                if (PV == 8) r1 = philox4x32_10((uint32_t)(u * 2 + 1), (uint32_t)((u * 2 + 1) >> 32), k0, k1);
-            }
-            const uint32_t rw[8] = {r0.x, r0.y, r0.z, r0.w, r1.x, r1.y, r1.z, r1.w};
-#pragma unroll
-            for (int k = 0; k < PV; k++) {
-                float x; uint32_t raw;
-                unpack<SRC>(v[j], k, x, raw);
-                if (AMAX) amax = amax_step(amax, x);
-                codes[k] = encode_one<MODE, SRC>(x, raw, scale, sm.ta, sm.thr, rw[k]);
-            }
-            if (!FQ) {
-                uint32_t w0 = codes[0] | (codes[1] << 8) | (codes[2] << 16) | (codes[3] << 24);
-                if (PV == 4) __stcs(reinterpret_cast<uint32_t*>(p.dst) + u, w0);
-                else {
-                    uint32_t w1 = codes[4] | (codes[5] << 8) | (codes[6] << 16) | (codes[7] << 24);
-                    __stcs(reinterpret_cast<uint2*>(p.dst) + u, make_uint2(w0, w1));
-                }
-            } else {
-                uint32_t o[PV];
-#pragma unroll
-                for (int k = 0; k < PV; k++) o[k] = to_bits<SRC>(sm.dec[codes[k]] * d1 * d2);
-                uint4 out;
-                if (PV == 4) out = make_uint4(o[0], o[1], o[2], o[3]);
-                else out = make_uint4(o[0] | (o[1] << 16), o[2] | (o[3] << 16), o[4] | (o[5] << 16), o[6] | (o[7] << 16));
-                __stcs(reinterpret_cast<uint4*>(p.dst) + u, out);
-            }
-        }
+        if (base + (unsigned long long)kThreads * kUnroll <= n_vec)
+            convert_group<SRC, MODE, FQ, AMAX, true>(p, sm, base, n_vec, scale, d1, d2, k0, k1, amax);
+        else
+            convert_group<SRC, MODE, FQ, AMAX, false>(p, sm, base, n_vec, scale, d1, d2, k0, k1, amax);
     }
     // elements not covered by whole vectors (tail, or everything when the pointers are not 16-byte aligned)
     {
@@ -425,15 +438,24 @@ int device_info(int* sms)
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-unsigned grid_for(unsigned long long n_vec, unsigned long long n, int sms, int unroll = kUnroll)
+constexpr int kGroupsConvert = 4;  // encode / fake-quant kernels: groups per block on large tensors
+
+unsigned grid_for(unsigned long long n_vec, unsigned long long n, int sms, int unroll = kUnroll, int max_groups = 1)
 {
-    // One block per kThreads * kUnroll vectors, no persistent loop: blocks are handed to SMs as they free up, which
+    // Many more blocks than the SMs can hold, no persistent loop: blocks are handed to SMs as they free up, which
     // balances the load between SMs near to and far from a memory partition (measured 10-20 % faster than a static
     // grid-stride split).  The scalar fallback (unaligned pointers) keeps a bounded grid-stride grid.
     unsigned long long per_block = (unsigned long long)kThreads * unroll;
     unsigned long long need;
-    if (n_vec) need = (n_vec + per_block - 1) / per_block;
-    else {
+    if (n_vec) {
+        need = (n_vec + per_block - 1) / per_block;
+        // Large tensors: up to max_groups groups per block (grid-stride), as long as at least one full wave of resident
+        // blocks remains for the scheduler to balance.  The per-block prologue (table set-up, scale) is then paid
+        // once per 64 KiB instead of once per 16 KiB, which the arithmetic-bound rounding modes feel most.
+        const unsigned long long wave = (unsigned long long)sms * kBlocksPerSM;
+        const unsigned long long groups = need / wave < (unsigned long long)max_groups ? need / wave : (unsigned long long)max_groups;
+        if (groups > 1) need = (need + groups - 1) / groups;
+    } else {
         need = (n + kThreads - 1) / kThreads;
         unsigned long long cap = (unsigned long long)sms * kBlocksPerSM * 4;
         if (need > cap) need = cap;
@@ -448,7 +470,7 @@ int launch_convert(const ConvParams& p, bool vec_ok, int sms, cudaStream_t st)
 {
     constexpr int PV = SrcTraits<SRC>::kPerVec;
     unsigned long long n_vec = vec_ok ? p.n / PV : 0;
-    unsigned grid = grid_for(n_vec, p.n, sms);
+    unsigned grid = grid_for(n_vec, p.n, sms, kUnroll, kGroupsConvert);
     launch_pdl(convert_kernel<SRC, MODE, FQ, AMAX>, grid, st, p, n_vec);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
@@ -480,7 +502,7 @@ int launch_fq_ta(int dtype, int rnd, const ConvParams& p, bool vec_ok, int sms, 
 {
     const unsigned long long pv = dtype == HIF8_F32 ? 4 : 8;
     const unsigned long long n_vec = vec_ok ? p.n / pv : 0;
-    const unsigned grid = grid_for(n_vec, p.n, sms);
+    const unsigned grid = grid_for(n_vec, p.n, sms, kUnroll, kGroupsConvert);
     if (dtype == HIF8_F32) launch_pdl(fq_ta_kernel<HIF8_F32, HIF8_RND_TA>, grid, st, p, n_vec);
     else if (rnd == HIF8_RND_TA) launch_pdl(fq_ta_kernel<HIF8_BF16, HIF8_RND_TA>, grid, st, p, n_vec);
     else if (rnd == HIF8_RND_HR) launch_pdl(fq_ta_kernel<HIF8_BF16, HIF8_RND_HR>, grid, st, p, n_vec);
