@@ -190,7 +190,14 @@ int launch(const TrParams& p, bool vec, int sms, cudaStream_t st)
         const long long nvc = p.cols / PV;
         const long long strips = (nvc + kTileVecs - 1) / kTileVecs, row_tiles = (p.rows + kTileRows - 1) / kTileRows;
         if (row_tiles > 0x7FFFFFFFll) return HIF8_ERR_SHAPE;
-        const dim3 grid((unsigned)row_tiles, (unsigned)(strips < 65535 ? strips : 65535));
+        // up to four strips per block while at least one full wave of resident blocks remains (the per-block table
+        // set-up is then shared by several tiles)
+        const long long wave = (long long)sms * 6;
+        long long per_block = row_tiles * strips / wave;
+        per_block = per_block < 1 ? 1 : per_block > 4 ? 4 : per_block;
+        long long gy = (strips + per_block - 1) / per_block;
+        if (gy > 65535) gy = 65535;
+        const dim3 grid((unsigned)row_tiles, (unsigned)gy);
         encode_transpose_kernel<SRC, MODE><<<grid, kThreads, 0, st>>>(p);
     } else {
         const unsigned long long n = (unsigned long long)p.rows * (unsigned long long)p.cols;
