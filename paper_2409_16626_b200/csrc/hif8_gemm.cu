@@ -544,49 +544,67 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 constexpr int kNarrowMaxM = 64;
 constexpr uint32_t kNwW8 = BM * BK, kNwA8 = kNarrowMaxM * BK;          // byte tiles per stage: 8 KiB weights, 4 KiB activations
 constexpr uint32_t kNwWBf = BM * BK * 2, kNwABf = kNarrowMaxM * BK * 2;  // operand tiles per stage: 16 KiB + 8 KiB
+constexpr int kNwByteStages = 8;  // byte ring deeper than the operand ring: 8 x 8 KiB of weights in flight per SM
 struct SmemLayoutN {
     static constexpr uint32_t bf = 0;
     static constexpr uint32_t u8 = bf + kDecodeGroups * (kNwWBf + kNwABf);
-    static constexpr uint32_t lut = u8 + kDecodeGroups * (kNwW8 + kNwA8);
+    static constexpr uint32_t lut = u8 + kNwByteStages * (kNwW8 + kNwA8);
     static constexpr uint32_t bars = lut + 256 * 32 * 4;
-    static constexpr uint32_t n_bars = 4 * kDecodeGroups + 1;
+    static constexpr uint32_t n_bars = 2 * kNwByteStages + 2 * kDecodeGroups + 4;
     static constexpr uint32_t tmem_slot = bars + n_bars * 8;
     static constexpr uint32_t abort_flag = tmem_slot + 4;
     static constexpr uint32_t total = abort_flag + 4;
 };
 constexpr uint32_t kSmemBytesN = SmemLayoutN::total + 1024;
-constexpr uint32_t kTmemColsN = 64;
+constexpr uint32_t kTmemColsN = 2 * kNarrowMaxM;  // two accumulators: the epilogue of one segment overlaps the next segment's MMAs
+
+// Work split of the narrow kernel.  The (slab, k-block) pairs are numbered slab-major, total = slabs * k-blocks, and CTA c
+// of G takes the contiguous range [total c / G, total (c + 1) / G): every SM streams the same number of weight bytes
+// whatever the number of slabs.  A range cuts slabs into segments.  A segment that covers its whole slab is finished by
+// its CTA; otherwise the CTA stores its FP32 partial sums as slice (slab, its position among the slab's contributors),
+// and the last contributor to arrive (one ticket per slab and epilogue warp) adds the slices in position order - so the
+// result does not depend on arrival order - and writes C.
+struct NarrowPlan {
+    long long total;     // slabs * k-blocks
+    float* part;         // [slab][pmax][mp][128] partial sums, or nullptr when every range is made of whole slabs
+    unsigned* tickets;   // [slab][4], zero at launch
+    int pmax;            // slices per slab
+};
 
 template <bool W_IS_NK>
 __global__ void __launch_bounds__(kThreads, 1)
-hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_constant__ CUtensorMap map_w, const GemmParams p, int mp)
+hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_constant__ CUtensorMap map_w, const GemmParams p, int mp,
+                        const NarrowPlan plan)
 {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* sm = smem_raw + (base - smem_u32(smem_raw));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    constexpr int S = kDecodeGroups;  // stages of both rings: group g owns stage g
+    constexpr int S = kDecodeGroups;    // operand ring: group g owns stage g
+    constexpr int S8 = kNwByteStages;   // byte ring: the it-th k-block of this CTA lands in stage it % S8
+    static_assert(S8 % kDecodeGroups == 0, "a byte stage is always read by the same group");
     const uint32_t bars = base + SmemLayoutN::bars;
     auto bar_u8_full = [&](int s) { return bars + 8u * s; };
-    auto bar_u8_empty = [&](int s) { return bars + 8u * (S + s); };
-    auto bar_bf_full = [&](int s) { return bars + 8u * (2 * S + s); };
-    auto bar_bf_empty = [&](int s) { return bars + 8u * (3 * S + s); };
-    const uint32_t bar_acc_full = bars + 8u * (4 * S);
+    auto bar_u8_empty = [&](int s) { return bars + 8u * (S8 + s); };
+    auto bar_bf_full = [&](int s) { return bars + 8u * (2 * S8 + s); };
+    auto bar_bf_empty = [&](int s) { return bars + 8u * (2 * S8 + S + s); };
+    auto bar_acc_full = [&](int b) { return bars + 8u * (2 * S8 + 2 * S + b); };
+    auto bar_acc_empty = [&](int b) { return bars + 8u * (2 * S8 + 2 * S + 2 + b); };
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + SmemLayoutN::abort_flag);
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + SmemLayoutN::tmem_slot);
     uint32_t* lut_all = reinterpret_cast<uint32_t*>(sm + SmemLayoutN::lut);
     const uint32_t lut = base + SmemLayoutN::lut + 4u * lane;
-    const int n0 = blockIdx.x * BM;  // this CTA's 128 weight columns
     const int num_kb = (p.K + BK - 1) / BK;
+    const long long G = gridDim.x;
+    const long long lin0 = plan.total * blockIdx.x / G, lin1 = plan.total * (blockIdx.x + 1) / G;  // this CTA's (slab, k-block) range
+    const int n_it = (int)(lin1 - lin0);
     const uint32_t act_bytes = (uint32_t)mp * BK;
 
     for (int i = threadIdx.x; i < 256 * 32; i += kThreads) lut_all[i] = hif8_to_bf16_bits(i >> 5);
     if (threadIdx.x == 0) {
-        for (int s = 0; s < S; s++) {
-            mbar_init(bar_u8_full(s), 1); mbar_init(bar_u8_empty(s), kGroupWarps);
-            mbar_init(bar_bf_full(s), kGroupWarps); mbar_init(bar_bf_empty(s), 1);
-        }
-        mbar_init(bar_acc_full, 1);
+        for (int s = 0; s < S8; s++) { mbar_init(bar_u8_full(s), 1); mbar_init(bar_u8_empty(s), kGroupWarps); }
+        for (int s = 0; s < S; s++) { mbar_init(bar_bf_full(s), kGroupWarps); mbar_init(bar_bf_empty(s), 1); }
+        for (int b = 0; b < 2; b++) { mbar_init(bar_acc_full(b), 1); mbar_init(bar_acc_empty(b), kEpiWarps); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -603,21 +621,23 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
     if (warp == kTmaWarp) {
         if (lane == 0) {
             int issued = 0;
-            for (int kb = 0; kb < num_kb; kb++) {
-                const int s = kb % S, round = kb / S;
+            int j = (int)(lin0 / num_kb), kb = (int)(lin0 % num_kb);
+            for (int it = 0; it < n_it; it++) {
+                const int s = it % S8, round = it / S8;
                 if (round > 0 && !mbar_wait(bar_u8_empty(s), (round - 1) & 1, abort_flag, p.status, 31)) break;
                 if (*abort_flag) break;
                 const uint32_t dst_w = base + SmemLayoutN::u8 + s * (kNwW8 + kNwA8), dst_a = dst_w + kNwW8;
                 mbar_arrive_expect_tx(bar_u8_full(s), kNwW8 + act_bytes);
-                if (W_IS_NK) tma_load_2d(dst_w, &map_w, kb * BK, n0, bar_u8_full(s));
-                else tma_load_2d(dst_w, &map_w, n0, kb * BK, bar_u8_full(s));
+                if (W_IS_NK) tma_load_2d(dst_w, &map_w, kb * BK, j * BM, bar_u8_full(s));
+                else tma_load_2d(dst_w, &map_w, j * BM, kb * BK, bar_u8_full(s));
                 tma_load_2d(dst_a, &map_act, kb * BK, 0, bar_u8_full(s));
-                issued = kb + 1;
+                issued = it + 1;
+                if (++kb == num_kb) { kb = 0; j++; }
             }
             if (*abort_flag) {  // let the copies already issued land before this CTA's shared memory goes away
-                for (int kb = max(0, issued - S); kb < issued; kb++) {
+                for (int it = max(0, issued - S8); it < issued; it++) {
                     const unsigned long long t0 = global_ns();
-                    while (!mbar_try_wait(bar_u8_full(kb % S), (kb / S) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+                    while (!mbar_try_wait(bar_u8_full(it % S8), (it / S8) & 1) && global_ns() - t0 < kWaitLimitNs) {}
                 }
             }
         }
@@ -627,10 +647,13 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
             // (K-major), N = mp, M = 128
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((W_IS_NK ? 0u : 1u) << 15) | ((uint32_t)(mp >> 3) << 17) |
                                    ((uint32_t)(BM >> 4) << 24);
-            bool ok = true;
-            for (int kb = 0; kb < num_kb && ok; kb++) {
-                const int s = kb % S, round = kb / S;
-                ok = mbar_wait(bar_bf_full(s), round & 1, abort_flag, p.status, 32);
+            bool ok = true, first = true;
+            int kb = (int)(lin0 % num_kb), seg = 0;
+            for (int it = 0; it < n_it && ok; it++) {
+                const int s = it % S, round = it / S, buf = seg & 1;
+                // a segment's first MMA overwrites the accumulator: the epilogue must have read its previous contents
+                if (first && seg >= 2) ok = mbar_wait(bar_acc_empty(buf), ((seg >> 1) - 1) & 1, abort_flag, p.status, 36);
+                if (ok) ok = mbar_wait(bar_bf_full(s), round & 1, abort_flag, p.status, 32);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t w_addr = base + SmemLayoutN::bf + s * (kNwWBf + kNwABf), a_addr = w_addr + kNwWBf;
@@ -638,38 +661,42 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
                 for (int kk = 0; kk < BK / 16; kk++) {
                     const uint64_t dw = W_IS_NK ? make_smem_desc(w_addr + kk * 32, 16, 1024) : make_smem_desc(w_addr + kk * 2048, 8192, 1024);
                     const uint64_t da = make_smem_desc(a_addr + kk * 32, 16, 1024);
-                    tc_mma_bf16_cta(tmem_base, dw, da, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+                    tc_mma_bf16_cta(tmem_base + (uint32_t)(buf * kNarrowMaxM), dw, da, idesc, (!first || kk > 0) ? 1u : 0u);
                 }
                 tc_commit_cta(bar_bf_empty(s));
+                first = false;
+                if (++kb == num_kb || it == n_it - 1) {  // the segment ends with its slab or with this CTA's range
+                    tc_commit_cta(bar_acc_full(buf));
+                    kb = 0; seg++; first = true;
+                }
             }
-            if (ok) tc_commit_cta(bar_acc_full);
         }
     } else if (warp >= kFirstDecodeWarp) {
         const int group = (warp - kFirstDecodeWarp) / kGroupWarps;
         const int dt = threadIdx.x - (kFirstDecodeWarp + group * kGroupWarps) * 32;
         const int act_chunks = mp * (BK / 8);  // 8-byte chunks of the activation tile
         bool ok = true;
-        for (int kb = group; kb < num_kb && ok; kb += kDecodeGroups) {
-            const int s = group, r = kb / S;
-            ok = mbar_wait(bar_u8_full(s), r & 1, abort_flag, p.status, 33);
+        for (int it = group; it < n_it && ok; it += kDecodeGroups) {
+            const int s = group, r = it / S, s8 = it % S8;
+            ok = mbar_wait(bar_u8_full(s8), (it / S8) & 1, abort_flag, p.status, 33);
             if (ok && r > 0) ok = mbar_wait(bar_bf_empty(s), (r - 1) & 1, abort_flag, p.status, 34);
             if (!ok) break;
-            const uint32_t w8 = base + SmemLayoutN::u8 + s * (kNwW8 + kNwA8), a8 = w8 + kNwW8;
+            const uint32_t w8 = base + SmemLayoutN::u8 + s8 * (kNwW8 + kNwA8), a8 = w8 + kNwW8;
             const uint32_t wbf = base + SmemLayoutN::bf + s * (kNwWBf + kNwABf), abf = wbf + kNwWBf;
             uint2 vw[kChunksPerThread], va[kNarrowMaxM * (BK / 8) / kGroupThreads];
             load_tile_chunks<!W_IS_NK>(w8, dt, vw);
 #pragma unroll
-            for (int it = 0; it < kNarrowMaxM * (BK / 8) / kGroupThreads; it++) {
-                const int q = it * kGroupThreads + dt;
-                if (q < act_chunks) va[it] = lds_v2(a8 + (q >> 3) * BK + (q & 7) * 8);
+            for (int i = 0; i < kNarrowMaxM * (BK / 8) / kGroupThreads; i++) {
+                const int q = i * kGroupThreads + dt;
+                if (q < act_chunks) va[i] = lds_v2(a8 + (q >> 3) * BK + (q & 7) * 8);
             }
             __syncwarp();  // the byte stage has been read: the producer may refill it during the decode
-            if (lane == 0) mbar_arrive(bar_u8_empty(s));
+            if (lane == 0) mbar_arrive(bar_u8_empty(s8));
             decode_tile_chunks<!W_IS_NK>(vw, wbf, dt, lut);
 #pragma unroll
-            for (int it = 0; it < kNarrowMaxM * (BK / 8) / kGroupThreads; it++) {
-                const int q = it * kGroupThreads + dt, row = q >> 3, j = q & 7;
-                if (q < act_chunks) sts_v4(abf + (row >> 3) * 1024 + (row & 7) * 128 + ((j ^ (row & 7)) << 4), decode8(va[it], lut));
+            for (int i = 0; i < kNarrowMaxM * (BK / 8) / kGroupThreads; i++) {
+                const int q = i * kGroupThreads + dt, row = q >> 3, jc = q & 7;
+                if (q < act_chunks) sts_v4(abf + (row >> 3) * 1024 + (row & 7) * 128 + ((jc ^ (row & 7)) << 4), decode8(va[i], lut));
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
@@ -677,36 +704,86 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
         }
     } else {
         // epilogue warps 0-3: TMEM lane = weight column n, TMEM column = activation row m
-        const bool ok = mbar_wait(bar_acc_full, 0, abort_flag, p.status, 35);
-        if (ok) {
+        const int sa = p.d_sa ? *p.d_sa : 0;
+        long long lin = lin0;
+        for (int seg = 0; lin < lin1; seg++) {
+            const int j = (int)(lin / num_kb), kb_a = (int)(lin % num_kb), buf = seg & 1;
+            const long long slab_end = (long long)(j + 1) * num_kb, seg_end = slab_end < lin1 ? slab_end : lin1;
+            const bool whole = kb_a == 0 && seg_end == slab_end;
+            if (!mbar_wait(bar_acc_full(buf), (seg >> 1) & 1, abort_flag, p.status, 35)) break;
             tc_fence_after();
-            const int n = n0 + warp * 32 + lane;
-            const int sa = p.d_sa ? *p.d_sa : 0;
+            const int n = j * BM + warp * 32 + lane;
             const int sw = p.d_sw_channel ? (n < p.N ? p.d_sw_channel[n] : 0) : (p.d_sw ? *p.d_sw : 0);
             const int sc = -(sa + sw), s1 = sc / 2, s2 = sc - s1;
             const float f1 = __uint_as_float((uint32_t)(s1 + 127) << 23), f2 = __uint_as_float((uint32_t)(s2 + 127) << 23);
+            auto finish = [&](int m, float acc) {  // C[m][n] from the complete sum
+                float v = acc * f1 * f2;
+                if (p.c_is_f32) {
+                    float* out = reinterpret_cast<float*>(p.C) + (long long)m * p.ldc + n;
+                    *out = p.accumulate ? v + *out : v;
+                } else {
+                    unsigned short* out = reinterpret_cast<unsigned short*>(p.C) + (long long)m * p.ldc + n;
+                    if (p.accumulate) v += __uint_as_float((uint32_t)*out << 16);
+                    const uint32_t u = __float_as_uint(v);
+                    *out = (unsigned short)((v != v) ? 0x7FC0u : ((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16));
+                }
+            };
+            // contributors of slab j are the CTAs owner(first k-block) .. owner(last k-block);
+            // owner(x) = the largest c with total c / G <= x
+            const long long c_first = ((slab_end - num_kb + 1) * G - 1) / plan.total, c_last = (slab_end * G - 1) / plan.total;
+            const int pos = (int)(blockIdx.x - c_first), count = (int)(c_last - c_first + 1);
+            float* slab_part = whole ? nullptr : plan.part + (size_t)j * plan.pmax * mp * BM + warp * 32 + lane;
+            float* mine = whole ? nullptr : slab_part + (size_t)pos * mp * BM;
+            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * kNarrowMaxM);
             for (int c = 0; c < mp; c += 32) {
-                uint32_t r[32];
-                tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(warp * 32) << 16) + c, r);
+                uint32_t r[32];  // this lane's row of the accumulator, columns c .. c + 31
+                tmem_ld_32x32b_x32(taddr + c, r);
                 tmem_ld_wait();
-                if (n < p.N) {
+                if (whole) {
+                    if (n < p.N) {
 #pragma unroll
-                    for (int i = 0; i < 32; i++) {
-                        const int m = c + i;
-                        if (m >= p.M) break;
-                        float v = __uint_as_float(r[i]) * f1 * f2;
-                        if (p.c_is_f32) {
-                            float* out = reinterpret_cast<float*>(p.C) + (long long)m * p.ldc + n;
-                            *out = p.accumulate ? v + *out : v;
-                        } else {
-                            unsigned short* out = reinterpret_cast<unsigned short*>(p.C) + (long long)m * p.ldc + n;
-                            if (p.accumulate) v += __uint_as_float((uint32_t)*out << 16);
-                            const uint32_t u = __float_as_uint(v);
-                            *out = (unsigned short)((v != v) ? 0x7FC0u : ((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16));
+                        for (int i = 0; i < 32; i++)
+                            if (c + i < p.M) finish(c + i, __uint_as_float(r[i]));
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; i++)
+                        if (c + i < mp) __stcg(mine + (c + i) * BM, __uint_as_float(r[i]));
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_acc_empty(buf));  // the accumulator has been read: it may be overwritten
+            if (!whole) {
+                __threadfence();
+                __syncwarp();
+                unsigned prior = 0;
+                if (lane == 0) prior = atomicAdd(plan.tickets + j * kEpiWarps + warp, 1u);
+                prior = __shfl_sync(0xFFFFFFFFu, prior, 0);
+                if (prior == (unsigned)(count - 1)) {  // every slice of this quarter slab is complete
+                    __threadfence();
+                    if (n < p.N) {
+                        // sixteen rows at a time: their loads are independent, so the L2 latency is paid once per slice
+                        for (int m0 = 0; m0 < p.M; m0 += 16) {
+                            float acc[16];
+#pragma unroll
+                            for (int u = 0; u < 16; u++) acc[u] = 0.f;
+                            for (int i = 0; i < count; i++) {
+                                const float* sl = slab_part + ((size_t)i * mp + m0) * BM;  // m0 + 15 < mp: mp is a multiple of 16
+                                float v[16];
+#pragma unroll
+                                for (int u = 0; u < 16; u++) v[u] = __ldcg(sl + u * BM);
+#pragma unroll
+                                for (int u = 0; u < 16; u++) acc[u] += v[u];
+                            }
+#pragma unroll
+                            for (int u = 0; u < 16; u++)
+                                if (m0 + u < p.M) finish(m0 + u, acc[u]);
                         }
                     }
                 }
             }
+            lin = seg_end;
         }
     }
 
@@ -1112,9 +1189,33 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t
         const bool okn = w_is_nk ? make_map(&map_ws, Wq, (uint64_t)K, (uint64_t)N, (uint64_t)ldw, BK, BM)
                                  : make_map(&map_ws, Wq, (uint64_t)N, (uint64_t)K, (uint64_t)ldw, BM, BK);
         if (!okn) return HIF8_ERR_CUDA;
-        const unsigned slabs = (unsigned)((N + BM - 1) / BM);
-        if (w_is_nk) hif8_gemm_narrow_kernel<true><<<slabs, kThreads, kSmemBytesN, st>>>(map_act, map_ws, p, mp);
-        else hif8_gemm_narrow_kernel<false><<<slabs, kThreads, kSmemBytesN, st>>>(map_act, map_ws, p, mp);
+        const long long slabs = (N + BM - 1) / BM, num_kb = (K + BK - 1) / BK;
+        NarrowPlan plan{};
+        plan.total = slabs * num_kb;
+        // One CTA per SM, equal k-block ranges, when the workspace holds the partial sums of the slabs that a range
+        // boundary cuts; otherwise one CTA per slab.
+        long long grid = slabs;
+        {
+            // aim at eight or more k-blocks per CTA, but never fewer CTAs than the per-slab grid would keep busy
+            long long g = plan.total / 8 < sm_count ? plan.total / 8 : sm_count;
+            const long long floor_g = slabs < sm_count ? slabs : sm_count;
+            if (g < floor_g) g = floor_g;
+            const long long per = plan.total / g;
+            const long long pmax = (num_kb + per - 1) / per + 1;
+            const size_t ticket_bytes = (((size_t)slabs * kEpiWarps * 4) + 255) & ~(size_t)255;
+            const size_t part_bytes = (size_t)slabs * pmax * mp * BM * 4;
+            if (g != slabs && workspace_bytes >= kGemmWorkspaceBytes + ticket_bytes + part_bytes && !(reinterpret_cast<uintptr_t>(workspace) & 255)) {
+                unsigned char* wsb = reinterpret_cast<unsigned char*>(workspace) + kGemmWorkspaceBytes;
+                plan.tickets = reinterpret_cast<unsigned*>(wsb);
+                plan.part = reinterpret_cast<float*>(wsb + ticket_bytes);
+                plan.pmax = (int)pmax;
+                grid = g;
+                if (cudaMemsetAsync(plan.tickets, 0, ticket_bytes, st) != cudaSuccess) return HIF8_ERR_CUDA;
+            }
+        }
+        if (grid > 0x7FFFFFFFll) return HIF8_ERR_SHAPE;
+        if (w_is_nk) hif8_gemm_narrow_kernel<true><<<(unsigned)grid, kThreads, kSmemBytesN, st>>>(map_act, map_ws, p, mp, plan);
+        else hif8_gemm_narrow_kernel<false><<<(unsigned)grid, kThreads, kSmemBytesN, st>>>(map_act, map_ws, p, mp, plan);
         g_launches.fetch_add(1, std::memory_order_relaxed);
         return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
     }

@@ -5,7 +5,8 @@
 cases: convert_f32 (FP32 4096^2: per-tensor scaled encode + decode), fq_bf16 (BF16 4096x8192 fake-quant, TA and HR,
 fused amax and given scale), encode_modes_f32 / encode_modes_bf16 (2^25 log-uniform values, every rounding mode), gemm (HiF8 GEMM
 4096 x 7168 x 4096, fused and decode-once paths), gemm_forms (same size, decode-once path, the four operand layouts:
-forward, dgrad form, wgrad form with FP32 accumulation, both transposed), channel_bf16 (per-channel scaled encode of a
+forward, dgrad form, wgrad form with FP32 accumulation, both transposed), gemm_narrow (16 x 8192 x 8192, the
+weight-streaming kernel, weights as [K,N] and as [N,K]), channel_bf16 (per-channel scaled encode of a
 BF16 8192 x 14336 weight, channel = column and channel = row, plus the overflow check of the same tensor), transpose_bf16
 (BF16 8192 x 8192 to HiF8 bytes, flat and with transposed store, round half away and hybrid rounding).  Inputs are seeded device-side random tensors.
 """
@@ -77,6 +78,14 @@ def main():
         for r in range(reps):
             H.hif8_gemm(A, K, W, N, 0, C, N, H.BF16, M, N, K, None, None, gws, big)
             H.hif8_gemm(A, K, W, N, 0, C, N, H.BF16, M, N, K, None, None, gws, 256)
+    elif case == "gemm_narrow":
+        M, N, K = 16, 8192, 8192
+        A = torch.randint(8, 100, (M * K,), dtype=torch.uint8, device="cuda", generator=g)
+        W = torch.randint(8, 100, (K * N,), dtype=torch.uint8, device="cuda", generator=g)
+        C = torch.zeros(M, N, dtype=torch.bfloat16, device="cuda")
+        for r in range(reps):
+            H.hif8_gemm(A, K, W, N, 0, C, N, H.BF16, M, N, K, None, None, ws, 256)
+            H.hif8_gemm(A, K, W, K, 1, C, N, H.BF16, M, N, K, None, None, ws, 256)
     elif case == "gemm_forms":
         M, N, K = 4096, 7168, 4096
         A = torch.randint(8, 100, (M * K,), dtype=torch.uint8, device="cuda", generator=g)

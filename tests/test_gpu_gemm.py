@@ -146,9 +146,13 @@ def test_bounded_wait_gives_up_and_reports_without_disturbing_the_device():
 
 @pytest.mark.parametrize("w_is_nk", [0, 1])
 @pytest.mark.parametrize("c_dtype", [H.F32, H.BF16])
-@pytest.mark.parametrize("shape", [(1, 256, 64), (16, 1008, 272), (17, 640, 1040), (33, 128, 16), (64, 400, 208), (48, 2064, 4096)])
-def test_gemm_narrow_products(shape, c_dtype, w_is_nk):
-    # M <= 64: the weight-streaming kernel (weights as the 128-row tensor-core operand, C accumulated transposed)
+@pytest.mark.parametrize("staged", [False, True])
+@pytest.mark.parametrize("shape", [(1, 256, 64), (16, 1008, 272), (17, 640, 1040), (33, 128, 16), (64, 400, 208), (48, 2064, 4096),
+                                   (8, 304, 8192), (20, 912, 1472), (64, 1296, 2048)])
+def test_gemm_narrow_products(shape, c_dtype, w_is_nk, staged):
+    # M <= 64: the weight-streaming kernel (weights as the 128-row tensor-core operand, C accumulated transposed).
+    # staged: with a workspace for partial sums the (slab, k-block) pairs are dealt out in equal contiguous ranges, so
+    # slabs are cut (the last three shapes: 16, ~3 and 4 contributors per slab) and summed from per-contributor slices
     M, N, K = shape
     N16 = (N + 15) // 16 * 16
     Aq = W.random_codes((M, K), seed=M + K)
@@ -161,12 +165,17 @@ def test_gemm_narrow_products(shape, c_dtype, w_is_nk):
         Wq = np.full((K, N16 + 16), 0x7B, dtype=np.uint8)     # padded leading dimension; the padding must not be read in
         Wq[:, :N] = Wkn
     Cs, S = O.gemm_full(Aq, Wkn, False, 3, -5)
-    out = run_gemm(Aq, Wq, w_is_nk, c_dtype, sa=3, sw=-5, M=M, N=N, K=K, ldw=Wq.shape[1])
+    out = run_gemm(Aq, Wq, w_is_nk, c_dtype, sa=3, sw=-5, M=M, N=N, K=K, ldw=Wq.shape[1], staged=staged)
     check(out, Cs, S, c_dtype)
+    if staged:  # slices are added in contributor order: the result does not depend on which CTA arrives last
+        again = run_gemm(Aq, Wq, w_is_nk, c_dtype, sa=3, sw=-5, M=M, N=N, K=K, ldw=Wq.shape[1], staged=staged)
+        assert np.array_equal(out, again)
 
 
-def test_gemm_narrow_channel_scales_and_accumulate():
-    M, N, K = 24, 528, 272
+@pytest.mark.parametrize("K", [272, 2112])
+def test_gemm_narrow_channel_scales_and_accumulate(K):
+    # K = 2112 with the large workspace: slabs cut between CTAs, finished by whichever contributor arrives last
+    M, N = 24, 528
     Aq = W.random_codes((M, K), seed=1)
     Wkn = W.random_codes((K, N), seed=2)
     for t in (Aq, Wkn):
@@ -174,9 +183,10 @@ def test_gemm_narrow_channel_scales_and_accumulate():
     sw = np.random.default_rng(3).integers(-20, 20, size=N).astype(np.int32)
     c0 = (np.random.default_rng(4).standard_normal((M, N)) * 10).astype(np.float32)
     C = torch.from_numpy(c0.copy()).cuda()
-    ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+    wsb = H.hif8_workspace_bytes(H.WS_GEMM, M * K + K * N) if K > 1000 else 256
+    ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
     H.hif8_gemm_ex(to_dev(Aq), K, 0, to_dev(Wkn), N, 0, C, N, H.F32, M, N, K, torch.tensor([2], dtype=torch.int32, device="cuda"),
-                   None, to_dev(sw.view(np.uint32)), 1, ws, 256)
+                   None, to_dev(sw.view(np.uint32)), 1, ws, wsb)
     assert H.hif8_gemm_status(ws) == 0
     rows, cols = np.divmod(np.arange(M * N), N)
     P, S = O.gemm_entries_channel(Aq, Wkn, 0, 2, sw, rows, cols)
