@@ -35,7 +35,7 @@ POOL = 6                  # rotating buffer sets: 6 x 64 MiB of input alone exce
 WORKLOAD = "fp32_4096x4096_normal_amax_scale_encode_then_decode"
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture summarised in profiles/;
 # None for a kernel changed since its capture
-TRAFFIC = {"amax_kernel<f32>": 67.64e6, "convert_kernel<f32,TA>": 69.68e6, "decode_kernel<f32>": 26.26e6}
+TRAFFIC = {"amax_kernel<f32>": 67.57e6, "convert_kernel<f32,TA>": 69.53e6, "decode_kernel<f32>": 26.10e6}
 METRIC = "hif8_encode_decode_throughput"
 UNIT = "GB/s"
 
@@ -305,10 +305,12 @@ def extra_results(H, torch, hbm_peak, peak_kind):
     narrow = {}
     for Mn in (16, 64):
         Cn = torch.empty(Mn, N, dtype=torch.bfloat16, device="cuda")
-        ms_n = timed(lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, Cn, N, H.BF16, Mn, N, K, se[0:1], se[1:2], gws, 256), 20)
+        # with the workspace: equal (slab, k-block) ranges per SM; with the 256-byte minimum: one CTA per slab
+        ms_n = timed(lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, Cn, N, H.BF16, Mn, N, K, se[0:1], se[1:2], gws, gws_b), 20)
+        ms_s = timed(lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, Cn, N, H.BF16, Mn, N, K, se[0:1], se[1:2], gws, 256), 20)
         byt = K * N + Mn * K + 2 * Mn * N
         narrow[f"M={Mn}"] = {"us": ms_n * 1e3, "GBps": byt / ms_n / 1e6, "frac_of_hbm": byt / ms_n / 1e6 / hbm_peak,
-                             "device_status": H.hif8_gemm_status(gws)}
+                             "us_one_cta_per_slab": ms_s * 1e3, "device_status": H.hif8_gemm_status(gws)}
         del Cn
     out["gemm_narrow_Mx28672x8192"] = {"bound": "hbm", "bytes": "K*N weight bytes + M*K + 2*M*N", "shapes": narrow,
                                        "peak": hbm_peak, "peak_kind": f"of {peak_kind}"}

@@ -247,7 +247,9 @@ int hif8_fake_quant(const void* src, void* dst, int dtype, size_t n, int use_ama
  * With hif8_workspace_bytes(HIF8_WS_GEMM, M*K + K*N) bytes, 256-byte aligned, and contiguous operands (lda = K,
  * ldw = row length of Wq), each operand byte is instead decoded once into the workspace (BF16, exact) and the
  * tensor-core kernel streams BF16 tiles: several times faster for compute-bound shapes, same results.
- * Products with at most 64 rows of A (and A given as [M,K]) take a weight-streaming kernel whatever the workspace.
+ * Products with at most 64 rows of A (and A given as [M,K]) take a weight-streaming kernel whatever the workspace;
+ * with the workspace size above it spreads the weight bytes evenly over all SMs (partial sums of a column slab that
+ * two SMs share go through the workspace and are added in a fixed order: results are reproducible run to run).
  */
 int hif8_gemm(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int64_t ldw, int w_is_nk, void* C,
               int64_t ldc, int c_dtype, int M, int N, int K, const int* d_scale_exp_a,
