@@ -796,22 +796,18 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
 }
 
 // ---------------------------------------------------------------------------------------------------------
-// Decode-once path: operands already decoded to BF16 (by the conversion kernel of this library, into the caller's
-// workspace).  Persistent kernel, 64-wide k-blocks.
+// Decode-once path: operands already decoded to BF16 (by the conversion kernels of this library, into the caller's
+// workspace).  Persistent kernel on CTA pairs (cta_group::2), 64-wide k-blocks.
 //   warps 0-3  epilogue (TMEM -> global), overlapped with the next tile through two TMEM accumulators
 //   warp  4    TMA producer: BF16 tiles land directly in the 128-byte-swizzled operand layout
 //   warp  5    MMA issuer
+// A cluster of two CTAs on two SMs computes one 256 x 256 tile: each CTA stages its own 128 rows of A and its own 128
+// columns of W (so the tensor core reads half as many operand bytes per SM and flop as with one CTA per tile, which is
+// what bounds a one-CTA kernel), both accumulate their 128 rows in their own TMEM.  The even CTA of the pair (the
+// leader) issues every tcgen05.mma; its commits arrive on the barriers of both CTAs.  TMA copies of both CTAs complete
+// on the leader's "full" barrier (no multicast loads).
 // ---------------------------------------------------------------------------------------------------------
 constexpr int kThreadsP = 6 * 32;
-
-
-// ---------------------------------------------------------------------------------------------------------
-// Decode-once path, CTA pairs (cta_group::2).  A cluster of two CTAs on two SMs computes one 256 x 256 tile: each
-// CTA stages its own 128 rows of A and its own 128 columns of W (so the tensor core reads half as many operand bytes
-// per SM and flop as with one CTA per tile, which is what bounds the one-CTA kernel), both accumulate their 128 rows
-// in their own TMEM.  The even CTA of the pair (the leader) issues every tcgen05.mma; its commits arrive on the
-// barriers of both CTAs.  TMA copies of both CTAs complete on the leader's "full" barrier (no multicast loads).
-// ---------------------------------------------------------------------------------------------------------
 constexpr int kStages2 = 6;
 constexpr uint32_t kStageBytes2 = kABfBytes + kBBfBytes;            // 32 KiB per CTA and stage
 struct SmemLayout2 {

@@ -41,8 +41,9 @@ def run_transpose(x, dtype, scale_exp=0, rnd=H.RND_TA, flags=0, seed=0, dev_exp=
 
 
 @pytest.mark.parametrize("dtype", [H.F32, H.BF16, H.F16])
-@pytest.mark.parametrize("shape", [(256, 128), (144, 72), (1040, 520), (16, 8), (130, 50), (48, 4096)])
+@pytest.mark.parametrize("shape", [(256, 128), (144, 72), (1040, 520), (16, 8), (130, 50), (48, 4096), (2064, 7048), (4112, 14360)])
 def test_encode_transpose_matches_oracle(shape, dtype):
+    # the last two shapes are large enough for two and for four column strips per block (ragged in both directions)
     x = source(*shape, seed=shape[0], dtype=dtype)
     se = 30 if dtype != H.F16 else 3
     q = run_transpose(x, dtype, scale_exp=se, rnd=H.RND_HR)

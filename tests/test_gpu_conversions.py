@@ -127,6 +127,33 @@ def test_encode_ragged_sizes_and_misaligned_pointers(mode):
     assert H.hif8_encode(0, H.F32, 0, 0) == 0
 
 
+def test_encode_sizes_around_the_groups_per_block_steps():
+    # Large tensors give a block two, three or four groups of vectors (grid-stride) and skip the bounds checks of groups
+    # that lie wholly inside the tensor: sizes just below and above each step, with ragged vector and element tails,
+    # every element compared
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    wave, per_group = sms * 8, 256 * 4 * 4                    # resident blocks per wave; FP32 elements per group
+    base = W.loguniform_f32(1 << 22, seed=77, lo_exp=-26, hi_exp=17).view(np.uint32)
+    for groups in (2, 3, 4):
+        for n in (groups * wave * per_group - 4099, groups * wave * per_group + 3 * per_group + 1027):
+            bits = np.resize(base, n)
+            d_src = to_dev(bits)
+            for mode in (H.RND_TA, H.RND_HR) + ((H.RND_SR,) if groups == 2 else ()):
+                _, dptr, rb = dev_empty(n, np.uint8)
+                H.hif8_encode(d_src, H.F32, dptr, n, 3, mode, 0, 21)
+                torch.cuda.synchronize()
+                assert np.array_equal(rb(), O.encode(bits, O.F32, 3, mode, 0, seed=21, quick=True))
+    # the BF16 fake-quant kernels (rounding on the bit pattern) take the same grid rule
+    n = 4 * wave * 256 * 4 * 8 + 8 * 1024 + 13
+    b16 = np.resize(W.llm_activation_bf16(512, 4096, seed=5).reshape(-1), n)
+    d = to_dev(b16)
+    for mode in (H.RND_TA, H.RND_HR):
+        _, dptr, rb = dev_empty(n, np.uint16)
+        H.hif8_fake_quant(d, dptr, H.BF16, n, 0, 4, mode, 0, 9)
+        torch.cuda.synchronize()
+        assert np.array_equal(rb(), O.fake_quant(b16, O.BF16, 4, mode, 0, seed=9, quick=True))
+
+
 def test_encode_sr_index_is_the_element_offset():
     # the threshold of element i depends on (seed, i) only: a long tensor and a slice of it differ
     bits = np.full(100_000, np.float32(1.03).view(np.uint32), dtype=np.uint32)
