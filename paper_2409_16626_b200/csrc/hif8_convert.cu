@@ -25,6 +25,7 @@
 
 #include <atomic>
 #include <cstdint>
+#include <type_traits>
 
 #include "hif8.h"
 #include "hif8_device.cuh"
@@ -243,17 +244,19 @@ __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, uns
 
     const uint4* src = reinterpret_cast<const uint4*>(p.src);
     const unsigned long long stride = (unsigned long long)gridDim.x * kThreads * kUnroll;
-    for (unsigned long long base = (unsigned long long)blockIdx.x * kThreads * kUnroll; base < n_vec; base += stride) {
+    // one group of kUnroll vectors per thread; a group wholly inside the tensor runs without bounds checks
+    auto group = [&](unsigned long long base, auto full_tag) {
+        constexpr bool FULL = decltype(full_tag)::value;
         uint4 v[kUnroll];
 #pragma unroll
         for (int j = 0; j < kUnroll; j++) {
             unsigned long long u = base + (unsigned long long)j * kThreads + threadIdx.x;
-            v[j] = (u < n_vec) ? __ldcs(src + u) : make_uint4(0, 0, 0, 0);
+            v[j] = (FULL || u < n_vec) ? __ldcs(src + u) : make_uint4(0, 0, 0, 0);
         }
 #pragma unroll
         for (int j = 0; j < kUnroll; j++) {
             unsigned long long u = base + (unsigned long long)j * kThreads + threadIdx.x;
-            if (u >= n_vec) continue;
+            if (!FULL && u >= n_vec) continue;
             uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w}, o[4], rare = 0;
             if (SRC == HIF8_F32) {
                 uint32_t m[4];
@@ -296,6 +299,10 @@ __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, uns
             }
             __stcs(reinterpret_cast<uint4*>(p.dst) + u, make_uint4(o[0], o[1], o[2], o[3]));
         }
+    };
+    for (unsigned long long base = (unsigned long long)blockIdx.x * kThreads * kUnroll; base < n_vec; base += stride) {
+        if (base + (unsigned long long)kThreads * kUnroll <= n_vec) group(base, std::true_type{});
+        else group(base, std::false_type{});
     }
     {   // tail / unaligned elements
         const unsigned long long tid = (unsigned long long)blockIdx.x * kThreads + threadIdx.x;
@@ -381,13 +388,15 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const uint8_t* __restr
     pdl_wait_prior_grid();
     constexpr int PV = SrcTraits<DT>::kPerVec;  // codes per 16-byte store
     const unsigned long long stride = (unsigned long long)gridDim.x * kThreads * kUnroll;
-    for (unsigned long long base = (unsigned long long)blockIdx.x * kThreads * kUnroll; base < n_vec; base += stride) {
+    // one group of kUnroll vectors per thread; a group wholly inside the tensor runs without bounds checks
+    auto group = [&](unsigned long long base, auto full_tag) {
+        constexpr bool FULL = decltype(full_tag)::value;
         uint2 v[kUnroll];
 #pragma unroll
         for (int j = 0; j < kUnroll; j++) {
             unsigned long long u = base + (unsigned long long)j * kThreads + threadIdx.x;
             v[j] = make_uint2(0, 0);
-            if (u < n_vec) {
+            if (FULL || u < n_vec) {
                 if (PV == 4) v[j].x = __ldcs(reinterpret_cast<const uint32_t*>(src) + u);
                 else v[j] = __ldcs(reinterpret_cast<const uint2*>(src) + u);
             }
@@ -395,7 +404,7 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const uint8_t* __restr
 #pragma unroll
         for (int j = 0; j < kUnroll; j++) {
             unsigned long long u = base + (unsigned long long)j * kThreads + threadIdx.x;
-            if (u >= n_vec) continue;
+            if (!FULL && u >= n_vec) continue;
             uint32_t o[PV];
 #pragma unroll
             for (int k = 0; k < PV; k++) o[k] = s_out[((k < 4 ? v[j].x : v[j].y) >> (8 * (k & 3))) & 0xFFu];
@@ -404,6 +413,10 @@ __global__ void __launch_bounds__(kThreads) decode_kernel(const uint8_t* __restr
             else out = make_uint4(o[0] | (o[1] << 16), o[2] | (o[3] << 16), o[4] | (o[5] << 16), o[6] | (o[7] << 16));
             __stcs(reinterpret_cast<uint4*>(dst) + u, out);
         }
+    };
+    for (unsigned long long base = (unsigned long long)blockIdx.x * kThreads * kUnroll; base < n_vec; base += stride) {
+        if (base + (unsigned long long)kThreads * kUnroll <= n_vec) group(base, std::true_type{});
+        else group(base, std::false_type{});
     }
     const unsigned long long tid = (unsigned long long)blockIdx.x * kThreads + threadIdx.x;
     for (unsigned long long i = n_vec * PV + tid; i < n; i += (unsigned long long)gridDim.x * kThreads) {
