@@ -55,6 +55,25 @@ __device__ __forceinline__ void convert_group(const ConvParams& p, const SmemTab
     for (int j = 0; j < kUnroll; j++) {
         unsigned long long u = base + (unsigned long long)j * kThreads + threadIdx.x;
         if (!FULL && u >= n_vec) continue;
+        if constexpr (SRC == HIF8_BF16 && (MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR) && !FQ) {
+            // two elements per word (see encode_pair16); sm.ta holds the 16-bit neighbour-pair words
+            const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w}, ns2 = neg_scale_bf16x2(scale);
+            uint32_t y[4], c[4];
+#pragma unroll
+            for (int k = 0; k < 4; k++) {
+                if (AMAX) {
+                    amax = amax_step(amax, __uint_as_float(w[k] << 16));
+                    amax = amax_step(amax, __uint_as_float(w[k] & 0xFFFF0000u));
+                }
+                y[k] = mul_bf16x2(w[k], ns2);
+                c[k] = encode_pair16(w[k], y[k], reinterpret_cast<const uint32_t*>(sm.ta));
+            }
+            // gather the codes and the sign bytes of four elements; a set (inverted) sign clears bit 7
+            const uint32_t c0 = __byte_perm(c[0], c[1], 0x5410), c1 = __byte_perm(c[2], c[3], 0x5410);
+            const uint32_t s0 = __byte_perm(y[0], y[1], 0x7531), s1 = __byte_perm(y[2], y[3], 0x7531);
+            __stcs(reinterpret_cast<uint2*>(p.dst) + u, make_uint2(c0 & (~s0 | 0x7F7F7F7Fu), c1 & (~s1 | 0x7F7F7F7Fu)));
+            continue;
+        }
         uint32_t codes[PV];
         uint4 r0 = make_uint4(0, 0, 0, 0), r1 = r0;
         if (MODE == HIF8_RND_SR) {
@@ -97,7 +116,9 @@ __global__ void __launch_bounds__(kThreads) convert_kernel(const ConvParams p, u
 {
     __shared__ SmemTables sm;
     pdl_launch_dependents();
-    setup_tables<true, MODE != HIF8_RND_TA, FQ, MODE, SRC>(sm, p.flags);  // reads only the constant table
+    constexpr bool kPair16 = SRC == HIF8_BF16 && (MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR) && !FQ;
+    if (kPair16) setup_pair16<MODE>(reinterpret_cast<uint32_t*>(sm.ta), p.flags);
+    else setup_tables<true, MODE != HIF8_RND_TA, FQ, MODE, SRC>(sm, p.flags);  // reads only the constant table
     pdl_wait_prior_grid();
     const int se = resolve_scale_exp(p);
     const float scale = pow2f(se);
@@ -128,7 +149,11 @@ __global__ void __launch_bounds__(kThreads) convert_kernel(const ConvParams p, u
                 const uint32_t rr[4] = {r.x, r.y, r.z, r.w};
                 word = rr[i & 3];
             }
-            uint32_t c = encode_one<MODE, SRC>(x, raw, scale, sm.ta, sm.thr, word);
+            uint32_t c;
+            if constexpr (kPair16) {
+                const uint32_t y = mul_bf16x2(raw, neg_scale_bf16x2(scale));  // the element as the low half of a word
+                c = encode_pair16(raw, y, reinterpret_cast<const uint32_t*>(sm.ta)) & (~(y >> 8) | 0x7Fu) & 0xFFu;
+            } else c = encode_one<MODE, SRC>(x, raw, scale, sm.ta, sm.thr, word);
             if (!FQ) reinterpret_cast<uint8_t*>(p.dst)[i] = (uint8_t)c;
             else {
                 uint32_t o = to_bits<SRC>(sm.dec[c] * d1 * d2);

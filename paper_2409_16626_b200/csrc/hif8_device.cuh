@@ -93,6 +93,38 @@ constexpr TaTable make_trunc_table()
 }
 __device__ const TaTable g_trunc_table = make_trunc_table();
 
+// Hybrid / simplified stochastic rounding (Section 3.2, Eq. 3): both neighbours of a scaled magnitude in one word.  Index =
+// (biased exponent, top three mantissa bits) of the magnitude, no sign: 2^-23 .. 2^16 are the binades that differ.
+//   bits 0-4   left shift that puts the discarded field of this binade at the top of a word (9 + mantissa width)
+//   bits 8-15  the neighbour below (truncation), bits 16-23 the neighbour above; bit 7 of either byte says "takes the
+//              sign" (clear for the single zero; the NaN pattern 0x80 reads as a zero magnitude that takes a sign which
+//              the caller arranges to be set)
+//   bits 30-31 are filled in at set-up (stochastic or round-half-away binade)
+// The binade of 2^-23 stands for everything below 2^-22 (see encode_one): neighbours 0 and 2^-22, no mantissa bit kept.
+__host__ __device__ constexpr uint32_t pair_entry(uint32_t idx)
+{
+    int e = (int)(idx >> 3);
+    uint32_t m3 = idx & 7u;
+    if (e == 255) return m3 ? 0x00808009u : 0x00EFEF09u;  // NaN / Inf
+    int E = e - 127;
+    if (E >= 16) return 0x00EFEF09u;
+    if (E < -23) return 0u;
+    if (E == -23) return 0x00810009u;
+    int w = mant_width(E);
+    uint32_t M = m3 >> (3 - w);
+    uint32_t down = pack_magnitude(E, M);  // E = 15, M = 1 is the Inf pattern by construction
+    uint32_t up = (M + 1u == (1u << w)) ? (E + 1 >= 16 ? 0x6Fu : pack_magnitude(E + 1, 0u)) : pack_magnitude(E, M + 1u);
+    return (uint32_t)(9 + w) | ((down | 0x80u) << 8) | ((up | 0x80u) << 16);
+}
+struct PairTable { uint32_t v[2048]; };
+constexpr PairTable make_pair_table()
+{
+    PairTable t{};
+    for (uint32_t i = 0; i < 2048; i++) t.v[i] = pair_entry(i);
+    return t;
+}
+__device__ const PairTable g_pair_table = make_pair_table();
+
 // value of one byte as binary32 bits (Eq. 1 / Eq. 2 / specials)
 __device__ __forceinline__ uint32_t decode_bits_f32(uint32_t c)
 {
@@ -216,44 +248,50 @@ template <int DT> __device__ __forceinline__ uint32_t to_bits(float v)
 //  * SR: thr[e] = sh, the number of discarded mantissa bits (23 - width; 0: nothing to round).
 //  * TE: thr[e] = half - 1 (bits 0-22; half itself where no mantissa bit is kept: the implicit one is odd), bit 26 "add
 //    the kept LSB", sh in bits 27-31; the binade of 2^-23 adds 2^23 - 1 (anything above the tie carries into 2^-22).
-//  * Hybrid / simplified stochastic rounding adds an increment to the bit pattern so that the carry out of the discarded
-//    field rounds up (also across binade and width boundaries), clears the old binade's discarded bits (~0 << sh) and
-//    reads the code from the truncating table.
-//       FP32 sources: t' = t + B + A * v with v = 2^14 - max(T14, 1); stochastic binade: A = 2^(sh-14), B = 0; round-half-away
-//                     binade of Eq. 3: A = 0, B = 2^(sh-1).  thr[e] = A, thr[256 + e] = B with sh in bits 27-31.  (One
-//                     merged entry with a select on a flag measured slower: 156 against 143 us per 2^27 elements.)
-//       16-bit sources (T2 = 2 LSB + 1, complement 3 - 2 LSB): the increment itself, thr[2e + LSB] = (3 - 2 LSB) * 2^(sh-2)
-//                     or one half, with sh in bits 0-4: a widened 16-bit pattern has zeros there, so they cannot carry.
-//    Below 2^-22 (result 0 or 2^-22, F = |y| / 2^-22):
-//       FP32: the element is first moved into the binade of 2^-24 (see encode_one), whose entry rounds it like a
-//             0-bit-mantissa binade: no carry leaves 2^-24 (-> 0), a carry gives 2^-23 (-> 2^-22 in the truncating table).
-//       16-bit: only the binades of 2^-23 and 2^-24 can reach the threshold; their entries add the complement at the top
-//             of the pattern and step the exponent down by one / two, which leaves 2^-23 or 2^-22 when the threshold is
-//             reached and something below 2^-23 when not.
+//  * Hybrid / simplified stochastic rounding, FP32 sources: thr[] is not used.  One word per (exponent, top three
+//    mantissa bits) holds both neighbours and the binade's shift (pair_entry); the discarded field, left-aligned, is
+//    compared with the threshold (SR14: the source's low 14 bits; one half in the round-half-away binades of Eq. 3) and
+//    the comparison picks the byte: one 4-byte lookup per element.  (The same form measured slower than the one below
+//    for 16-bit sources: 54.7 against 41.7 us per 2^26 BF16 elements.)
+//  * Hybrid / simplified stochastic rounding, 16-bit sources (T2 = 2 LSB + 1, complement 3 - 2 LSB): an increment is added
+//    to the bit pattern so that the carry out of the discarded field rounds up (also across binade and width boundaries),
+//    the old binade's discarded bits are cleared (~0 << sh) and the code is read from the truncating table.
+//    thr[2e + LSB] = (3 - 2 LSB) * 2^(sh-2), or one half in a round-half-away binade, with sh in bits 0-4.  Below 2^-22
+//    (result 0 or 2^-22, F = |y| / 2^-22) only the binades of 2^-23 and 2^-24 can reach the threshold; their entries add
+//    the complement at the top of the pattern and step the exponent down by one / two, which leaves 2^-23 or 2^-22 when
+//    the threshold is reached and something below 2^-23 when not.
 template <int MODE, int SRC>
 __device__ __forceinline__ uint32_t encode_one(float x, uint32_t raw, float scale, const uint8_t* s_ta,
                                                const uint32_t* s_thr, uint32_t word)
 {
-    const float y = x * scale;
+    constexpr bool kPair = (MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR) && SRC == HIF8_F32;
+    const float y = kPair ? x * -scale : x * scale;
     uint32_t t = __float_as_uint(y);
     if (MODE == HIF8_RND_TA) return s_ta[t >> 19];
 
-    if (MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR) {  // s_ta is the truncating table here
-        if (SRC == HIF8_F32) {
-            // below 2^-22: |y| / 4 + 2^-24 with truncation puts floor(F 2^23) into the mantissa of a value in the binade
-            // of 2^-24 (sign kept)
-            const float z = __fmaf_rz(y, 0.25f, __uint_as_float((t & 0x80000000u) | 0x33800000u));
-            const uint32_t u = fabsf(y) < 2.384185791015625e-07f ? __float_as_uint(z) : t;
-            const uint32_t i = (u >> 23) & 0xFFu;  // without the sign: values of either sign share the entry (and its bank)
-            const uint32_t v = 0x4000u - max(raw & 0x3FFFu, 1u);  // SR14: 2^14 - max(T14, 1)
-            const uint32_t B = s_thr[256 + i];                    // constant in bits 0-26, sh in bits 27-31
-            return s_ta[((u + (B & 0x07FFFFFFu) + s_thr[i] * v) & (0xFFFFFFFFu << (B >> 27))) >> 19];
-        } else {
-            // two entries per exponent, chosen by the source LSB: B + A * LSB, with sh in bits 0-4 (a widened 16-bit
-            // pattern has zeros there, so they cannot carry)
-            const uint32_t ent = s_thr[((t >> 22) & 0x1FEu) | (raw & 1u)];
-            return s_ta[((t + ent) & (0xFFFFFFFFu << (ent & 31u))) >> 19];
+    if ((MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR) && SRC == HIF8_F32) {
+        // s_ta holds the neighbour-pair words here (see pair_entry).  The scale was negated above: every sign is then
+        // inverted except that of the canonical NaN the multiply produces, so "bit 7 of the code AND NOT the sign" gives
+        // the sign of every finite / infinite result, a set bit for NaN and nothing for the single zero.
+        const float a = fabsf(y);
+        // below 2^-22 the result is 0 or 2^-22 with F = |y| / 2^-22: |y| / 2 + 2^-23 with truncation puts floor(F 2^23)
+        // into the mantissa of a value in the binade of 2^-23, and exceeds |y| exactly when |y| < 2^-22
+        const uint32_t w = __float_as_uint(fmaxf(a, __fmaf_rz(a, 0.5f, 1.1920928955078125e-07f)));
+        const uint32_t ent = reinterpret_cast<const uint32_t*>(s_ta)[w >> 20];
+        const uint32_t u = __funnelshift_l(0u, w, ent);  // discarded field, left-aligned (shift = low five bits of ent)
+        uint32_t thr = max(raw << 18, 0x40000u);         // SR14: round up iff F14 >= max(T14, 1), T14 = low 14 source bits
+        if (MODE == HIF8_RND_HR) {                       // round-half-away binades of Eq. 3 (bit 31): the top discarded bit decides
+            const uint32_t m = (uint32_t)((int32_t)ent >> 31);
+            thr = (thr & ~m) | (m & 0x80000000u);
         }
+        const uint32_t c = __byte_perm(ent, 0u, u >= thr ? 0x4442u : 0x4441u);
+        return c & (~(t >> 24) | 0x7Fu);
+    }
+    if (MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR) {  // 16-bit sources; s_ta is the truncating table here
+        // two entries per exponent, chosen by the source LSB, with sh in bits 0-4 (a widened 16-bit pattern has zeros
+        // there, so they cannot carry)
+        const uint32_t ent = s_thr[((t >> 22) & 0x1FEu) | (raw & 1u)];
+        return s_ta[((t + ent) & (0xFFFFFFFFu << (ent & 31u))) >> 19];
     }
 
     if (MODE == HIF8_RND_TE) {
@@ -297,6 +335,72 @@ __device__ __forceinline__ uint32_t encode_one(float x, uint32_t raw, float scal
 }
 
 // ------------------------------------------------------------------------------------------------
+// BF16 sources, hybrid / simplified stochastic rounding, two elements per 32-bit word.
+// The scale is applied with one packed BF16 multiply (exact for a power of two wherever the result matters: BF16 has the
+// binary32 exponent range; NaN comes out as the canonical positive pattern), by the negated scale as in encode_one.  Each
+// half then takes one neighbour-pair word, indexed by (exponent, top three mantissa bits) of the scaled magnitude:
+//   bits 0-4   left shift that puts the discarded field of the 16-bit pattern at the top of a word (25 + mantissa width)
+//   bits 8-15 / 16-23  neighbour below / above (bit 7: takes the sign), bits 24-29 zero
+//   bits 31-30 01 in an SR2 binade, 10 in a round-half-away binade of Eq. 3
+// Round up iff u >= thr with u = pattern << shift, filled with ones from below, and thr = entry with the source LSB
+// OR-ed into bit 31: the top two bits compare F2 with T2 = 2 LSB + 1 (or the top discarded bit with one half), and
+// whenever they are equal the ones below make u the larger.  Below 2^-22 (F = |y| / 2^-22, F2 = floor(4 F)) only two
+// binades can reach a threshold; their shifts put exponent bits that spell F2 at the top: 2^-23 (exponent 01101000) with
+// top mantissa bit 0 has F2 = 2 and shift 19 (bits "10"), with top mantissa bit 1 F2 = 3 reaches every threshold (both
+// neighbours 2^-22); 2^-24 (exponent 01100111) has F2 = 1 and shift 17 (bits "011").
+// ------------------------------------------------------------------------------------------------
+template <int MODE>
+__device__ __forceinline__ void setup_pair16(uint32_t* d, unsigned flags)
+{
+    for (int i = threadIdx.x; i < 2048; i += kThreads) {
+        const int e = i >> 3, E = e - 127;
+        uint32_t v = 0u;
+        if (e == 103) v = 0x00810011u;
+        else if (e == 104) v = (i & 4) ? 0x00818119u : 0x00810013u;
+        else if (e <= 142 && e > 104) v = g_pair_table.v[i] + 16u;
+        else if (e > 142) v = (e == 255 && (i & 7)) ? 0x00808019u : 0x00EFEF19u;
+        if (flags) {  // Section 3 options: patch the Inf / NaN bytes
+            uint32_t lo = (v >> 8) & 0xFFu, hi = (v >> 16) & 0xFFu;
+            if (flags & HIF8_FLAG_SATURATE) {
+                if ((lo & 0x7Fu) == 0x6Fu) lo &= 0xFEu;
+                if ((hi & 0x7Fu) == 0x6Fu) hi &= 0xFEu;
+            }
+            if (flags & HIF8_FLAG_NAN_TO_ZERO) {
+                if (lo == 0x80u) lo = 0u;
+                if (hi == 0x80u) hi = 0u;
+            }
+            v = (v & 0xFF0000FFu) | (lo << 8) | (hi << 16);
+        }
+        v |= (MODE == HIF8_RND_HR && E > -4 && E < 4) ? 0x80000000u : 0x40000000u;
+        d[i] = v;
+    }
+    __syncthreads();
+}
+
+// the negated power-of-two scale as two BF16 values
+__device__ __forceinline__ uint32_t neg_scale_bf16x2(float scale) { return (0x8000u | (__float_as_uint(scale) >> 16)) * 0x00010001u; }
+
+__device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+
+// W: two source patterns, Y = W times the negated scale.  Returns the two codes before the sign step in bytes 0 and 1
+// (bytes 2 and 3 are not meaningful); the caller clears bit 7 of a code where bit 15 / 31 of Y is set.
+__device__ __forceinline__ uint32_t encode_pair16(uint32_t W, uint32_t Y, const uint32_t* tab)
+{
+    const uint32_t A = Y & 0x7FFF7FFFu, Ah = A >> 16;
+    const uint32_t el = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(tab) + ((A >> 2) & 0x3FFCu));
+    const uint32_t eh = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(tab) + ((Ah >> 2) & 0x3FFCu));
+    const uint32_t ul = __funnelshift_l(0xFFFFFFFFu, A, el), uh = __funnelshift_l(0xFFFFFFFFu, Ah, eh);
+    const uint32_t tl = el | ((W << 31) & 0x80000000u), th = eh | ((W << 15) & 0x80000000u);
+    const uint32_t sel = 0x4051u + (ul >= tl ? 0x01u : 0u) + (uh >= th ? 0x10u : 0u);
+    return __byte_perm(el, eh, sel);
+}
+
+// ------------------------------------------------------------------------------------------------
 // Block set-up: tables into shared memory, scale
 // ------------------------------------------------------------------------------------------------
 struct __align__(16) SmemTables {
@@ -308,7 +412,34 @@ struct __align__(16) SmemTables {
 template <bool NEED_TA, bool NEED_SH, bool NEED_DEC, int MODE = HIF8_RND_TA, int SRC = HIF8_F32>
 __device__ __forceinline__ void setup_tables(SmemTables& s, unsigned flags)
 {
-    if (NEED_TA) {
+    constexpr bool kPair = (MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR) && SRC == HIF8_F32;  // neighbour-pair words instead of code bytes
+    if (NEED_TA && kPair) {
+        // 2048 words indexed by (exponent, top three mantissa bits).  The magnitudes that reach the lookup lie in
+        // 2^-23 .. Inf / NaN; 2^-23 .. 2^15 come from the compile-time table, everything above is Inf.
+        uint32_t* d = reinterpret_cast<uint32_t*>(s.ta);
+        for (int i = threadIdx.x; i < 2048; i += kThreads) {
+            const int e = i >> 3, E = e - 127;
+            uint32_t v = 0u;
+            if (e >= 104 && e <= 142) v = g_pair_table.v[i];
+            else if (e > 142) v = (e == 255 && (i & 7)) ? 0x00808009u : 0x00EFEF09u;
+            if (flags) {  // Section 3 options: patch the Inf / NaN bytes
+                uint32_t lo = (v >> 8) & 0xFFu, hi = (v >> 16) & 0xFFu;
+                if (flags & HIF8_FLAG_SATURATE) {
+                    if ((lo & 0x7Fu) == 0x6Fu) lo &= 0xFEu;
+                    if ((hi & 0x7Fu) == 0x6Fu) hi &= 0xFEu;
+                }
+                if (flags & HIF8_FLAG_NAN_TO_ZERO) {
+                    if (lo == 0x80u) lo = 0u;
+                    if (hi == 0x80u) hi = 0u;
+                }
+                v = (v & 0xFF0000FFu) | (lo << 8) | (hi << 16);
+            }
+            // Eq. 3: round half away for |E| < 4 under hybrid rounding (bits 31-30 = 10), stochastic elsewhere (01)
+            v |= (MODE == HIF8_RND_HR && E > -4 && E < 4) ? 0x80000000u : 0x40000000u;
+            d[i] = v;
+        }
+    }
+    if (NEED_TA && !kPair) {
         // Only binades 2^-24 .. 2^16 differ from their neighbours: those 41 x 16 entries per sign come from the
         // compile-time table (1.3 KiB of global reads per block); everything below is zero, everything above is
         // Inf (or NaN in the all-ones exponent), written straight into shared memory.
@@ -342,35 +473,27 @@ __device__ __forceinline__ void setup_tables(SmemTables& s, unsigned flags)
             d[i] = v;
         }
     }
-    if (NEED_SH) {
+    if (NEED_SH && !kPair) {
         const int e = threadIdx.x, E = e - 127;  // kThreads == 256 biased exponents
-        constexpr bool kF32 = SRC == HIF8_F32;
         constexpr bool kThreshold = MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR;
-        // TE / SR: thr[e] = e0.  FP32 threshold modes: thr[e] = e0 (A), thr[256 + e] = e1 (B).  16-bit threshold modes:
-        // thr[2e] = e0 (source LSB 0), thr[2e + 1] = e1 (LSB 1).
+        // TE / SR: thr[e] = e0.  Threshold modes (16-bit sources): thr[2e] = e0 (source LSB 0), thr[2e + 1] = e1 (LSB 1).
         uint32_t e0 = 0, e1 = 0;
         if (E < 16 && E >= -22) {
             const uint32_t sh = 23u - (uint32_t)mant_width(E);
             const bool stochastic = MODE == HIF8_RND_SSR || E <= -4 || E >= 4;  // Eq. 3 for HR
             if (MODE == HIF8_RND_TE) e0 = (sh == 23u ? (1u << 22) : ((1u << (sh - 1u)) - 1u) | (1u << 26)) | (sh << 27);
             else if (!kThreshold) e0 = sh;  // SR: only the width is read
-            else if (kF32) {
-                if (stochastic) e0 = 1u << (sh - 14u); else e1 = 1u << (sh - 1u);
-                e1 |= sh << 27;
-            }
             else if (stochastic) { e0 = (3u << (sh - 2u)) | sh; e1 = (1u << (sh - 2u)) | sh; }  // complement 3 - 2 LSB
             else e0 = e1 = (1u << (sh - 1u)) | sh;
         } else if (MODE == HIF8_RND_TE && E == -23) {
             e0 = ((1u << 23) - 1u) | (23u << 27);  // above 2^-23 -> carry -> 2^-22; exactly 2^-23 stays (-> 0 in TE's table)
-        } else if (kThreshold && kF32 && E == -24) {
-            e0 = 1u << 9; e1 = 23u << 27;  // where encode_one parks FP32 elements below 2^-22
-        } else if (kThreshold && !kF32 && (E == -23 || E == -24)) {
+        } else if (kThreshold && (E == -23 || E == -24)) {
             const uint32_t j = (uint32_t)(-23 - E);  // complement << (22 + j), then j + 1 binades down
             e0 = ((3u << (22u + j)) - ((j + 1u) << 23)) | 23u;
             e1 = ((1u << (22u + j)) - ((j + 1u) << 23)) | 23u;
         }
-        if (kThreshold && !kF32) { s.thr[2 * e] = e0; s.thr[2 * e + 1] = e1; }
-        else { s.thr[e] = e0; s.thr[256 + e] = e1; }
+        if (kThreshold) { s.thr[2 * e] = e0; s.thr[2 * e + 1] = e1; }
+        else s.thr[e] = e0;
     }
     if (NEED_DEC) s.dec[threadIdx.x] = __uint_as_float(decode_bits_f32(threadIdx.x));
     __syncthreads();

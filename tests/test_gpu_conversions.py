@@ -75,7 +75,7 @@ def test_encode_exhaustive_16bit(dtype, mode):
     for flags in FLAGSETS:
         want = O.encode(bits, dtype, 0, mode, flags, seed=1, quick=False)
         assert_same(gpu_encode(bits, dtype, scale_exp=0, rnd=mode, flags=flags, seed=1), want, bits)
-    for se in (3, -9, 14, -30, 100, -100):
+    for se in (3, -9, 14, -30, 100, -100, 126, 110):  # the last two bring subnormal BF16 sources into range
         want = O.encode(bits, dtype, se, mode, 0, seed=7, quick=True)
         assert_same(gpu_encode(bits, dtype, scale_exp=se, rnd=mode, seed=7), want, bits)
 
@@ -112,7 +112,7 @@ def test_encode_f32_subnormal_sources_with_large_scale():
             assert_same(gpu_encode(bits, H.F32, scale_exp=se, rnd=mode, seed=3), want, bits)
 
 
-@pytest.mark.parametrize("mode", [H.RND_TA, H.RND_SR])
+@pytest.mark.parametrize("mode", [H.RND_TA, H.RND_SR, H.RND_HR, H.RND_SSR])
 def test_encode_ragged_sizes_and_misaligned_pointers(mode):
     base = W.loguniform_f32(5000, seed=5, lo_exp=-26, hi_exp=17).view(np.uint32)
     for n in (1, 3, 4, 15, 16, 17, 1023, 1024, 1025, 4097):
