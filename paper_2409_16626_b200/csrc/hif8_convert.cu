@@ -74,6 +74,25 @@ __device__ __forceinline__ void convert_group(const ConvParams& p, const SmemTab
             __stcs(reinterpret_cast<uint2*>(p.dst) + u, make_uint2(c0 & (~s0 | 0x7F7F7F7Fu), c1 & (~s1 | 0x7F7F7F7Fu)));
             continue;
         }
+        if constexpr (SRC == HIF8_F32 && (MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR) && !FQ) {
+            // four elements: neighbour-pair words, the comparisons pick the bytes pairwise, one sign step for all four
+            const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w};
+            uint32_t y[4], ent[4], sel[4];
+#pragma unroll
+            for (int k = 0; k < 4; k++) {
+                const float x = __uint_as_float(w[k]);
+                if (AMAX) amax = amax_step(amax, x);
+                const float ys = x * -scale;
+                y[k] = __float_as_uint(ys);
+                sel[k] = pair32_lookup<MODE>(ys, w[k], reinterpret_cast<const uint32_t*>(sm.ta), ent[k]) ? 1u : 0u;
+            }
+            const uint32_t c01 = __byte_perm(ent[0], ent[1], 0x4051u + sel[0] + (sel[1] << 4));
+            const uint32_t c23 = __byte_perm(ent[2], ent[3], 0x4051u + sel[2] + (sel[3] << 4));
+            const uint32_t s01 = __byte_perm(y[0], y[1], 0x7373), s23 = __byte_perm(y[2], y[3], 0x7373);
+            const uint32_t c = __byte_perm(c01, c23, 0x5410), s = __byte_perm(s01, s23, 0x5410);
+            __stcs(reinterpret_cast<uint32_t*>(p.dst) + u, c & (~s | 0x7F7F7F7Fu));  // a set (inverted) sign clears bit 7
+            continue;
+        }
         uint32_t codes[PV];
         uint4 r0 = make_uint4(0, 0, 0, 0), r1 = r0;
         if (MODE == HIF8_RND_SR) {

@@ -260,6 +260,25 @@ template <int DT> __device__ __forceinline__ uint32_t to_bits(float v)
 //    (result 0 or 2^-22, F = |y| / 2^-22) only the binades of 2^-23 and 2^-24 can reach the threshold; their entries add
 //    the complement at the top of the pattern and step the exponent down by one / two, which leaves 2^-23 or 2^-22 when
 //    the threshold is reached and something below 2^-23 when not.
+// FP32 sources, hybrid / simplified stochastic rounding: the neighbour-pair word of the scaled value y and whether the
+// upper neighbour is taken
+template <int MODE>
+__device__ __forceinline__ bool pair32_lookup(float y, uint32_t raw, const uint32_t* tab, uint32_t& ent)
+{
+    const float a = fabsf(y);
+    // below 2^-22 the result is 0 or 2^-22 with F = |y| / 2^-22: |y| / 2 + 2^-23 with truncation puts floor(F 2^23)
+    // into the mantissa of a value in the binade of 2^-23, and exceeds |y| exactly when |y| < 2^-22
+    const uint32_t w = __float_as_uint(fmaxf(a, __fmaf_rz(a, 0.5f, 1.1920928955078125e-07f)));
+    ent = tab[w >> 20];
+    const uint32_t u = __funnelshift_l(0u, w, ent);  // discarded field, left-aligned (shift = low five bits of ent)
+    uint32_t thr = max(raw << 18, 0x40000u);         // SR14: round up iff F14 >= max(T14, 1), T14 = low 14 source bits
+    if (MODE == HIF8_RND_HR) {                       // round-half-away binades of Eq. 3 (bit 31): the top discarded bit decides
+        const uint32_t m = (uint32_t)((int32_t)ent >> 31);
+        thr = (thr & ~m) | (m & 0x80000000u);
+    }
+    return u >= thr;
+}
+
 template <int MODE, int SRC>
 __device__ __forceinline__ uint32_t encode_one(float x, uint32_t raw, float scale, const uint8_t* s_ta,
                                                const uint32_t* s_thr, uint32_t word)
@@ -273,18 +292,9 @@ __device__ __forceinline__ uint32_t encode_one(float x, uint32_t raw, float scal
         // s_ta holds the neighbour-pair words here (see pair_entry).  The scale was negated above: every sign is then
         // inverted except that of the canonical NaN the multiply produces, so "bit 7 of the code AND NOT the sign" gives
         // the sign of every finite / infinite result, a set bit for NaN and nothing for the single zero.
-        const float a = fabsf(y);
-        // below 2^-22 the result is 0 or 2^-22 with F = |y| / 2^-22: |y| / 2 + 2^-23 with truncation puts floor(F 2^23)
-        // into the mantissa of a value in the binade of 2^-23, and exceeds |y| exactly when |y| < 2^-22
-        const uint32_t w = __float_as_uint(fmaxf(a, __fmaf_rz(a, 0.5f, 1.1920928955078125e-07f)));
-        const uint32_t ent = reinterpret_cast<const uint32_t*>(s_ta)[w >> 20];
-        const uint32_t u = __funnelshift_l(0u, w, ent);  // discarded field, left-aligned (shift = low five bits of ent)
-        uint32_t thr = max(raw << 18, 0x40000u);         // SR14: round up iff F14 >= max(T14, 1), T14 = low 14 source bits
-        if (MODE == HIF8_RND_HR) {                       // round-half-away binades of Eq. 3 (bit 31): the top discarded bit decides
-            const uint32_t m = (uint32_t)((int32_t)ent >> 31);
-            thr = (thr & ~m) | (m & 0x80000000u);
-        }
-        const uint32_t c = __byte_perm(ent, 0u, u >= thr ? 0x4442u : 0x4441u);
+        uint32_t ent;
+        const bool up = pair32_lookup<MODE>(y, raw, reinterpret_cast<const uint32_t*>(s_ta), ent);
+        const uint32_t c = __byte_perm(ent, 0u, up ? 0x4442u : 0x4441u);
         return c & (~(t >> 24) | 0x7Fu);
     }
     if (MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR) {  // 16-bit sources; s_ta is the truncating table here
