@@ -56,7 +56,7 @@ __device__ __forceinline__ void convert_group(const ConvParams& p, const SmemTab
         unsigned long long u = base + (unsigned long long)j * kThreads + threadIdx.x;
         if (!FULL && u >= n_vec) continue;
         if constexpr (SRC == HIF8_BF16 && (MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR) && !FQ) {
-            // two elements per word (see encode_pair16); sm.ta holds the 16-bit neighbour-pair words
+            // two elements per word (see encode_sum16)
             const uint32_t w[4] = {v[j].x, v[j].y, v[j].z, v[j].w}, ns2 = neg_scale_bf16x2(scale);
             uint32_t y[4], c[4];
 #pragma unroll
@@ -66,7 +66,7 @@ __device__ __forceinline__ void convert_group(const ConvParams& p, const SmemTab
                     amax = amax_step(amax, __uint_as_float(w[k] & 0xFFFF0000u));
                 }
                 y[k] = mul_bf16x2(w[k], ns2);
-                c[k] = encode_pair16(w[k], y[k], reinterpret_cast<const uint32_t*>(sm.ta));
+                c[k] = encode_sum16(w[k], y[k], sm.ta, sm.thr);
             }
             // gather the codes and the sign bytes of four elements; a set (inverted) sign clears bit 7
             const uint32_t c0 = __byte_perm(c[0], c[1], 0x5410), c1 = __byte_perm(c[2], c[3], 0x5410);
@@ -136,7 +136,7 @@ __global__ void __launch_bounds__(kThreads) convert_kernel(const ConvParams p, u
     __shared__ SmemTables sm;
     pdl_launch_dependents();
     constexpr bool kPair16 = SRC == HIF8_BF16 && (MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR) && !FQ;
-    if (kPair16) setup_pair16<MODE>(reinterpret_cast<uint32_t*>(sm.ta), p.flags);
+    if (kPair16) setup_sum16<MODE>(sm.ta, sm.thr, p.flags);
     else setup_tables<true, MODE != HIF8_RND_TA, FQ, MODE, SRC>(sm, p.flags);  // reads only the constant table
     pdl_wait_prior_grid();
     const int se = resolve_scale_exp(p);
@@ -171,7 +171,7 @@ __global__ void __launch_bounds__(kThreads) convert_kernel(const ConvParams p, u
             uint32_t c;
             if constexpr (kPair16) {
                 const uint32_t y = mul_bf16x2(raw, neg_scale_bf16x2(scale));  // the element as the low half of a word
-                c = encode_pair16(raw, y, reinterpret_cast<const uint32_t*>(sm.ta)) & (~(y >> 8) | 0x7Fu) & 0xFFu;
+                c = encode_sum16(raw, y, sm.ta, sm.thr) & (~(y >> 8) | 0x7Fu) & 0xFFu;
             } else c = encode_one<MODE, SRC>(x, raw, scale, sm.ta, sm.thr, word);
             if (!FQ) reinterpret_cast<uint8_t*>(p.dst)[i] = (uint8_t)c;
             else {

@@ -411,6 +411,69 @@ __device__ __forceinline__ uint32_t encode_pair16(uint32_t W, uint32_t Y, const 
 }
 
 // ------------------------------------------------------------------------------------------------
+// BF16 sources, hybrid / simplified stochastic rounding in packed BF16 arithmetic (two elements per instruction, on the
+// floating-point pipe).  SR2 rounds up iff F >= T2 / 4 with T2 = 2 LSB + 1, i.e. iff |y| + (1 - T2 / 4) ulp reaches the
+// upper neighbour: add 0.75 ulp minus LSB * 0.5 ulp (0.5 ulp in a round-half-away binade of Eq. 3) and let a truncating
+// code table drop what is left of the discarded bits.  The addend is a multiple of the 8-bit significand's grid, so the
+// sum is exact unless it carries into the next binade, where the leftover is below one unit of any mantissa width.
+//   inck[e] (by the biased exponent of |y|): low half the addend for LSB = 0, high half -(0.5 ulp) * 2^69
+//   LSB term: the source's LSB as the BF16 pattern 0x0001 (2^-133) times 2^64, times the high half
+//   Below 2^-22 (result 0 or 2^-22, F = |y| / 2^-22): the binades of 2^-23 and 2^-24 add 3 * 2^-24 - LSB * 2 * 2^-24 and
+//   reach 2^-22 exactly when floor(4 F) >= T2; smaller values add nothing.  Anything that ends below 2^-22 reads zero.
+//   code8[(e, top three mantissa bits)] is the truncated magnitude with bit 7 = "takes the sign" (see pair_entry).
+// ------------------------------------------------------------------------------------------------
+template <int MODE>
+__device__ __forceinline__ void setup_sum16(uint8_t* code8, uint32_t* inck, unsigned flags)
+{
+    for (int i = threadIdx.x; i < 512; i += kThreads) {  // four codes per word
+        uint32_t word = 0;
+#pragma unroll
+        for (int b = 0; b < 4; b++) {
+            const int idx = 4 * i + b, e = idx >> 3;
+            uint32_t c = 0;
+            if (e >= 105 && e <= 142) c = (g_pair_table.v[idx] >> 8) & 0xFFu;
+            else if (e > 142) c = (e == 255 && (idx & 7)) ? 0x80u : 0xEFu;
+            if ((flags & HIF8_FLAG_SATURATE) && (c & 0x7Fu) == 0x6Fu) c &= 0xFEu;
+            if ((flags & HIF8_FLAG_NAN_TO_ZERO) && c == 0x80u) c = 0u;
+            word |= c << (8 * b);
+        }
+        reinterpret_cast<uint32_t*>(code8)[i] = word;
+    }
+    {
+        const int e = threadIdx.x, E = e - 127;  // kThreads == 256 biased exponents
+        uint32_t v = 0u;
+        if (E >= -24 && E <= 15) {
+            // h = biased exponent of 0.5 ulp; below 2^-22 the unit is 2^-22 whatever the binade
+            const int h = (E < -22 ? -23 : E - mant_width(E) - 1) + 127;
+            if (MODE == HIF8_RND_HR && E > -4 && E < 4) v = (uint32_t)h << 7;                       // 0.5 ulp, no LSB term
+            else v = (((uint32_t)h << 7) | 0x40u) | ((0x8000u | ((uint32_t)(h + 69) << 7)) << 16);  // 0.75 ulp; -(0.5 ulp) 2^69
+        }
+        inck[e] = v;
+    }
+    __syncthreads();
+}
+
+__device__ __forceinline__ uint32_t fma_bf16x2(uint32_t a, uint32_t b, uint32_t c)
+{
+    uint32_t d;
+    asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
+// W: two source patterns, Y = W times the negated scale.  Returns the two codes before the sign step in bytes 0 and 1;
+// the caller clears bit 7 of a code where bit 15 / 31 of Y is set.
+__device__ __forceinline__ uint32_t encode_sum16(uint32_t W, uint32_t Y, const uint8_t* code8, const uint32_t* inck)
+{
+    const uint32_t A = Y & 0x7FFF7FFFu;
+    const uint32_t el = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(inck) + ((A >> 5) & 0x3FCu));
+    const uint32_t eh = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(inck) + ((A >> 21) & 0x3FCu));
+    const uint32_t lsb = mul_bf16x2(W & 0x00010001u, 0x5F805F80u);  // LSB * 2^-133 * 2^64
+    const uint32_t add = fma_bf16x2(lsb, __byte_perm(el, eh, 0x7632), __byte_perm(el, eh, 0x5410));
+    const uint32_t R = fma_bf16x2(A, 0x3F803F80u, add);  // |y| + addend, non-negative
+    return (uint32_t)code8[(R >> 4) & 0x7FFu] | ((uint32_t)code8[R >> 20] << 8);
+}
+
+// ------------------------------------------------------------------------------------------------
 // Block set-up: tables into shared memory, scale
 // ------------------------------------------------------------------------------------------------
 struct __align__(16) SmemTables {
