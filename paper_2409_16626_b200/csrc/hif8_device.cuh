@@ -345,72 +345,6 @@ __device__ __forceinline__ uint32_t encode_one(float x, uint32_t raw, float scal
 }
 
 // ------------------------------------------------------------------------------------------------
-// BF16 sources, hybrid / simplified stochastic rounding, two elements per 32-bit word.
-// The scale is applied with one packed BF16 multiply (exact for a power of two wherever the result matters: BF16 has the
-// binary32 exponent range; NaN comes out as the canonical positive pattern), by the negated scale as in encode_one.  Each
-// half then takes one neighbour-pair word, indexed by (exponent, top three mantissa bits) of the scaled magnitude:
-//   bits 0-4   left shift that puts the discarded field of the 16-bit pattern at the top of a word (25 + mantissa width)
-//   bits 8-15 / 16-23  neighbour below / above (bit 7: takes the sign), bits 24-29 zero
-//   bits 31-30 01 in an SR2 binade, 10 in a round-half-away binade of Eq. 3
-// Round up iff u >= thr with u = pattern << shift, filled with ones from below, and thr = entry with the source LSB
-// OR-ed into bit 31: the top two bits compare F2 with T2 = 2 LSB + 1 (or the top discarded bit with one half), and
-// whenever they are equal the ones below make u the larger.  Below 2^-22 (F = |y| / 2^-22, F2 = floor(4 F)) only two
-// binades can reach a threshold; their shifts put exponent bits that spell F2 at the top: 2^-23 (exponent 01101000) with
-// top mantissa bit 0 has F2 = 2 and shift 19 (bits "10"), with top mantissa bit 1 F2 = 3 reaches every threshold (both
-// neighbours 2^-22); 2^-24 (exponent 01100111) has F2 = 1 and shift 17 (bits "011").
-// ------------------------------------------------------------------------------------------------
-template <int MODE>
-__device__ __forceinline__ void setup_pair16(uint32_t* d, unsigned flags)
-{
-    for (int i = threadIdx.x; i < 2048; i += kThreads) {
-        const int e = i >> 3, E = e - 127;
-        uint32_t v = 0u;
-        if (e == 103) v = 0x00810011u;
-        else if (e == 104) v = (i & 4) ? 0x00818119u : 0x00810013u;
-        else if (e <= 142 && e > 104) v = g_pair_table.v[i] + 16u;
-        else if (e > 142) v = (e == 255 && (i & 7)) ? 0x00808019u : 0x00EFEF19u;
-        if (flags) {  // Section 3 options: patch the Inf / NaN bytes
-            uint32_t lo = (v >> 8) & 0xFFu, hi = (v >> 16) & 0xFFu;
-            if (flags & HIF8_FLAG_SATURATE) {
-                if ((lo & 0x7Fu) == 0x6Fu) lo &= 0xFEu;
-                if ((hi & 0x7Fu) == 0x6Fu) hi &= 0xFEu;
-            }
-            if (flags & HIF8_FLAG_NAN_TO_ZERO) {
-                if (lo == 0x80u) lo = 0u;
-                if (hi == 0x80u) hi = 0u;
-            }
-            v = (v & 0xFF0000FFu) | (lo << 8) | (hi << 16);
-        }
-        v |= (MODE == HIF8_RND_HR && E > -4 && E < 4) ? 0x80000000u : 0x40000000u;
-        d[i] = v;
-    }
-    __syncthreads();
-}
-
-// the negated power-of-two scale as two BF16 values
-__device__ __forceinline__ uint32_t neg_scale_bf16x2(float scale) { return (0x8000u | (__float_as_uint(scale) >> 16)) * 0x00010001u; }
-
-__device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b)
-{
-    uint32_t d;
-    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-    return d;
-}
-
-// W: two source patterns, Y = W times the negated scale.  Returns the two codes before the sign step in bytes 0 and 1
-// (bytes 2 and 3 are not meaningful); the caller clears bit 7 of a code where bit 15 / 31 of Y is set.
-__device__ __forceinline__ uint32_t encode_pair16(uint32_t W, uint32_t Y, const uint32_t* tab)
-{
-    const uint32_t A = Y & 0x7FFF7FFFu, Ah = A >> 16;
-    const uint32_t el = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(tab) + ((A >> 2) & 0x3FFCu));
-    const uint32_t eh = *reinterpret_cast<const uint32_t*>(reinterpret_cast<const char*>(tab) + ((Ah >> 2) & 0x3FFCu));
-    const uint32_t ul = __funnelshift_l(0xFFFFFFFFu, A, el), uh = __funnelshift_l(0xFFFFFFFFu, Ah, eh);
-    const uint32_t tl = el | ((W << 31) & 0x80000000u), th = eh | ((W << 15) & 0x80000000u);
-    const uint32_t sel = 0x4051u + (ul >= tl ? 0x01u : 0u) + (uh >= th ? 0x10u : 0u);
-    return __byte_perm(el, eh, sel);
-}
-
-// ------------------------------------------------------------------------------------------------
 // BF16 sources, hybrid / simplified stochastic rounding in packed BF16 arithmetic (two elements per instruction, on the
 // floating-point pipe).  SR2 rounds up iff F >= T2 / 4 with T2 = 2 LSB + 1, i.e. iff |y| + (1 - T2 / 4) ulp reaches the
 // upper neighbour: add 0.75 ulp minus LSB * 0.5 ulp (0.5 ulp in a round-half-away binade of Eq. 3) and let a truncating
@@ -451,6 +385,16 @@ __device__ __forceinline__ void setup_sum16(uint8_t* code8, uint32_t* inck, unsi
         inck[e] = v;
     }
     __syncthreads();
+}
+
+// the negated power-of-two scale as two BF16 values
+__device__ __forceinline__ uint32_t neg_scale_bf16x2(float scale) { return (0x8000u | (__float_as_uint(scale) >> 16)) * 0x00010001u; }
+
+__device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
 }
 
 __device__ __forceinline__ uint32_t fma_bf16x2(uint32_t a, uint32_t b, uint32_t c)

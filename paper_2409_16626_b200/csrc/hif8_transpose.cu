@@ -45,7 +45,9 @@ __global__ void __launch_bounds__(kThreads, MODE == HIF8_RND_SR ? 4 : 6) encode_
     // tile[c][w]: code bytes of source column c, rows 4w .. 4w+3 in word w; the 16-byte chunk index (w / 4) is XORed
     // with the column's vector index so that both the word stores below and the 16-byte reads are conflict-free
     __shared__ __align__(16) uint32_t tile[TC * kTileWords];
-    setup_tables<true, MODE != HIF8_RND_TA, false, MODE, SRC>(sm, p.flags);
+    constexpr bool kSum16 = SRC == HIF8_BF16 && (MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR);  // packed BF16 arithmetic
+    if (kSum16) setup_sum16<MODE>(sm.ta, sm.thr, p.flags);
+    else setup_tables<true, MODE != HIF8_RND_TA, false, MODE, SRC>(sm, p.flags);
     const float scale = pow2f(p.d_scale_exp ? clamp_exp(*p.d_scale_exp) : p.scale_exp);
     const uint32_t k0 = (uint32_t)p.seed, k1 = (uint32_t)(p.seed >> 32);
     const long long nvc = p.cols / PV;                        // vectors per source row
@@ -87,6 +89,24 @@ __global__ void __launch_bounds__(kThreads, MODE == HIF8_RND_SR ? 4 : 6) encode_
             }
 #pragma unroll
             for (int k = 0; k < PV; k++) my_words[k * kTileWords] = packed[k];
+        } else if constexpr (kSum16) {
+            // a source word holds two neighbouring columns: the codes of four rows are gathered into one word per column
+            const uint32_t ns2 = neg_scale_bf16x2(scale);
+#pragma unroll
+            for (int m = 0; m < 4; m++) {
+                uint32_t c[4], y[4];
+#pragma unroll
+                for (int j = 0; j < 4; j++) {
+                    const uint32_t w = m == 0 ? v[j].x : (m == 1 ? v[j].y : (m == 2 ? v[j].z : v[j].w));
+                    y[j] = mul_bf16x2(w, ns2);
+                    c[j] = encode_sum16(w, y[j], sm.ta, sm.thr);
+                }
+                const uint32_t c01 = __byte_perm(c[0], c[1], 0x5140), c23 = __byte_perm(c[2], c[3], 0x5140);
+                const uint32_t s01 = __byte_perm(y[0], y[1], 0x7351), s23 = __byte_perm(y[2], y[3], 0x7351);
+                // a set (inverted) sign clears bit 7
+                my_words[(2 * m) * kTileWords] = __byte_perm(c01, c23, 0x5410) & (~__byte_perm(s01, s23, 0x5410) | 0x7F7F7F7Fu);
+                my_words[(2 * m + 1) * kTileWords] = __byte_perm(c01, c23, 0x7632) & (~__byte_perm(s01, s23, 0x7632) | 0x7F7F7F7Fu);
+            }
         } else {
             // columns outermost: the four codes of a column are packed and stored at once
 #pragma unroll
