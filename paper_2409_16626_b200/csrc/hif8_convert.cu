@@ -219,7 +219,8 @@ __global__ void __launch_bounds__(kThreads) convert_kernel(const ConvParams p, u
 constexpr uint32_t kRareMask = 1u;  // never a legitimate mask: legitimate ones are 0 or end in at least four zero bits
 
 // one element, any input: value-level rounding through the scaled binary32 value.
-// MODE: round half away, or (BF16 sources) the 2-bit simplified stochastic rounding SR2 / hybrid rounding of Eq. 3.
+// MODE: round half away, round half to even, or (BF16 sources) the 2-bit simplified stochastic rounding SR2 / hybrid
+// rounding of Eq. 3.
 template <int SRC, int MODE>
 __device__ __noinline__ uint32_t fq_rare(uint32_t raw, int se, unsigned flags)
 {
@@ -231,7 +232,16 @@ __device__ __noinline__ uint32_t fq_rare(uint32_t raw, int se, unsigned flags)
     const uint32_t top = (flags & HIF8_FLAG_SATURATE) ? 0x47000000u : 0x7F800000u;  // 2^15 or Inf
     const int E = (int)(a >> 23) - 127;
     uint32_t r;
-    if (MODE == HIF8_RND_TA || (MODE == HIF8_RND_HR && E > -4 && E < 4)) {
+    if (MODE == HIF8_RND_TE) {
+        if (a <= 0x34000000u) return 0u;                                                   // up to the tie 2^-23 (kept significand 0 is even)
+        else if (E < -22) r = 0x34800000u;                                                 // (2^-23, 2^-22) -> 2^-22
+        else {
+            // half - 1 plus the kept LSB; where no mantissa bit is kept the bit above the field is the implicit one (odd)
+            const uint32_t k = 23u - (uint32_t)mant_width(E);
+            r = (a + (1u << (k - 1)) - 1u + (k == 23u ? 1u : (a >> k) & 1u)) & (0xFFFFFFFFu << k);
+            if (r >= 0x47400000u) r = top;                                                 // 1.5 * 2^15 and above
+        }
+    } else if (MODE == HIF8_RND_TA || (MODE == HIF8_RND_HR && E > -4 && E < 4)) {
         if (a >= 0x47200000u) r = top;                                                     // >= 1.25 * 2^15
         else if (a < 0x34000000u) return 0u;                                               // < 2^-23: the single zero
         else if (E < -22) r = 0x34800000u;                                                 // [2^-23, 2^-22) -> 2^-22
@@ -255,10 +265,14 @@ __device__ __noinline__ uint32_t fq_rare(uint32_t raw, int se, unsigned flags)
 
 // MODE = round half away (FP32, BF16), or hybrid / simplified stochastic rounding (BF16 only: SR2 adds half * (3 - 2 lsb),
 // i.e. thresholds 0.25 / 0.75, where round-half-away adds half)
+// MODE = round half to even (BF16 only) is done in packed BF16 arithmetic instead: (x + C) - C with C = 2^(7 - width) times
+// the element's own power of two and the element's sign.  The sum lies in the binade of C, whose spacing is the HiF8
+// spacing of the element's binade (2^-22 over the scale below the format's range), so the hardware's round-to-nearest-even
+// does the rounding, ties to the even kept significand (the implicit one counts), and x - x = +0 gives the single zero.
 template <int SRC, int MODE>
 __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, unsigned long long n_vec)
 {
-    static_assert(MODE == HIF8_RND_TA || SRC == HIF8_BF16, "threshold modes are done in place for BF16 only");
+    static_assert(MODE == HIF8_RND_TA || SRC == HIF8_BF16, "threshold modes and round half to even are done in place for BF16 only");
     constexpr int MB = SRC == HIF8_F32 ? 23 : 7;      // mantissa bits of the source format
     constexpr int PV = SrcTraits<SRC>::kPerVec;
     __shared__ uint32_t s_inc[256];                   // BF16: mask16 | inc16 << 16
@@ -270,7 +284,7 @@ __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, uns
         const int e = threadIdx.x, E = e - 127 + se;
         uint32_t inc = 0, mask = 0;
         if (e == 255 || (e == 0 && se > 100) || (e > 0 && E >= 15)) mask = kRareMask;
-        else if (MODE != HIF8_RND_TA && e > 0 && (E == -23 || E == -24)) mask = kRareMask;  // result is 0 or 2^-22
+        else if ((MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR) && e > 0 && (E == -23 || E == -24)) mask = kRareMask;  // result is 0 or 2^-22
         else if (e == 0 || E <= -24) { inc = 0; mask = 0; }                                 // underflow to +0
         else if (E == -23) { inc = 1u << MB; mask = 0xFFFFFFFFu << MB; }                    // up to 2^-22
         else {
@@ -281,7 +295,12 @@ __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, uns
             // half of it, marked by bit 15: the increment is quarter * (4 - T2) = quarter * (3 - 2 lsb)
             if (MODE == HIF8_RND_SSR || (MODE == HIF8_RND_HR && (E <= -4 || E >= 4))) inc = (1u << (k - 2)) | 0x8000u;
         }
-        if (SRC == HIF8_F32) { s_inc[e] = inc; s_mask[e] = mask; }
+        if (MODE == HIF8_RND_TE) {
+            // biased exponent of C: the element's plus 7 - width, or that of 2^(-22 - se + 7) below the format's range
+            const int cb = (e == 0 || E < -22) ? 112 - se : e + 7 - mant_width(E);
+            const bool rare = mask == kRareMask || cb < 1 || cb > 254;
+            s_inc[e] = rare ? kRareMask : (uint32_t)cb << 23;  // C in the high half
+        } else if (SRC == HIF8_F32) { s_inc[e] = inc; s_mask[e] = mask; }
         else s_inc[e] = (mask & 0xFFFFu) | (inc << 16);
     }
     __syncthreads();
@@ -322,6 +341,12 @@ __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, uns
                 for (int k = 0; k < 4; k++) {
                     tl[k] = s_inc[(w[k] >> 7) & 0xFFu];
                     th[k] = s_inc[(w[k] >> 23) & 0xFFu];
+                    if (MODE == HIF8_RND_TE) {
+                        const uint32_t cs = __byte_perm(tl[k], th[k], 0x7632) | (w[k] & 0x80008000u);  // C with the element's sign
+                        o[k] = fma_bf16x2(fma_bf16x2(w[k], 0x3F803F80u, cs), 0x3F803F80u, cs ^ 0x80008000u);
+                        rare |= tl[k] | th[k];
+                        continue;
+                    }
                     const uint32_t mask2 = __byte_perm(tl[k], th[k], 0x5410);
                     uint32_t inc2 = __byte_perm(tl[k], th[k], 0x7632);
                     if (MODE != HIF8_RND_TA) {
@@ -565,6 +590,7 @@ int launch_fq_ta(int dtype, int rnd, const ConvParams& p, bool vec_ok, int sms, 
     if (dtype == HIF8_F32) launch_pdl(fq_ta_kernel<HIF8_F32, HIF8_RND_TA>, grid, st, p, n_vec);
     else if (rnd == HIF8_RND_TA) launch_pdl(fq_ta_kernel<HIF8_BF16, HIF8_RND_TA>, grid, st, p, n_vec);
     else if (rnd == HIF8_RND_HR) launch_pdl(fq_ta_kernel<HIF8_BF16, HIF8_RND_HR>, grid, st, p, n_vec);
+    else if (rnd == HIF8_RND_TE) launch_pdl(fq_ta_kernel<HIF8_BF16, HIF8_RND_TE>, grid, st, p, n_vec);
     else launch_pdl(fq_ta_kernel<HIF8_BF16, HIF8_RND_SSR>, grid, st, p, n_vec);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
@@ -666,7 +692,7 @@ static int scaled_convert(bool fq, const void* src, void* dst, int dtype, size_t
     }
     p.scale_state = scale_state;
     const bool inplace_fq = fq && !want_amax && ((rnd == HIF8_RND_TA && (dtype == HIF8_F32 || dtype == HIF8_BF16)) ||
-                                                ((rnd == HIF8_RND_HR || rnd == HIF8_RND_SSR) && dtype == HIF8_BF16));
+                                                ((rnd == HIF8_RND_HR || rnd == HIF8_RND_SSR || rnd == HIF8_RND_TE) && dtype == HIF8_BF16));
     if (jit) {
         rc = launch_amax(src, dtype, n, ws, nullptr, sms, st);
         if (rc) return rc;
