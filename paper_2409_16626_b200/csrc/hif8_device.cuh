@@ -100,7 +100,7 @@ __device__ const TaTable g_trunc_table = make_trunc_table();
 //              sign" (clear for the single zero; the NaN pattern 0x80 reads as a zero magnitude that takes a sign which
 //              the caller arranges to be set)
 //   bits 30-31 are filled in at set-up (stochastic or round-half-away binade)
-// The binade of 2^-23 stands for everything below 2^-22 (see encode_one): neighbours 0 and 2^-22, no mantissa bit kept.
+// The binade of 2^-23 stands for everything below 2^-22 (see pair32_lookup): neighbours 0 and 2^-22, no mantissa bit kept.
 __host__ __device__ constexpr uint32_t pair_entry(uint32_t idx)
 {
     int e = (int)(idx >> 3);

@@ -177,7 +177,7 @@ def test_channel_pipeline_weight_to_gemm():
     assert rel < 0.06  # target exponent 2 puts each channel's bulk into the 3-bit-mantissa binades (|E| <= 3)
 
 
-@pytest.mark.parametrize("dtype,rnd", [(H.F32, H.RND_TA), (H.BF16, H.RND_HR)])
+@pytest.mark.parametrize("dtype,rnd", [(H.F32, H.RND_TA), (H.BF16, H.RND_HR), (H.F32, H.RND_HR), (H.BF16, H.RND_SSR)])
 @pytest.mark.parametrize("interval,hist", [(1, 1), (3, 2), (10, 4)])
 def test_delayed_scale_cadence(interval, hist, dtype, rnd):
     T, n = 24, 70001
