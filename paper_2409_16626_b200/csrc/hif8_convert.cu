@@ -263,8 +263,8 @@ __device__ __noinline__ uint32_t fq_rare(uint32_t raw, int se, unsigned flags)
     return to_bits<SRC>(__uint_as_float(r | sign) * pow2f(da) * pow2f(db));
 }
 
-// MODE = round half away (FP32, BF16), or hybrid / simplified stochastic rounding (BF16 only: SR2 adds half * (3 - 2 lsb),
-// i.e. thresholds 0.25 / 0.75, where round-half-away adds half)
+// MODE = round half away (FP32, BF16), or hybrid / simplified stochastic rounding (BF16 only, in packed BF16 arithmetic:
+// SR2 adds 0.75 ulp - LSB * 0.5 ulp to the magnitude, i.e. thresholds 0.25 / 0.75, where round-half-away adds half)
 // MODE = round half to even (BF16 only) is done in packed BF16 arithmetic instead: (x + C) - C with C = 2^(7 - width) times
 // the element's own power of two and the element's sign.  The sum lies in the binade of C, whose spacing is the HiF8
 // spacing of the element's binade (2^-22 over the scale below the format's range), so the hardware's round-to-nearest-even
@@ -275,14 +275,15 @@ __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, uns
     static_assert(MODE == HIF8_RND_TA || SRC == HIF8_BF16, "threshold modes and round half to even are done in place for BF16 only");
     constexpr int MB = SRC == HIF8_F32 ? 23 : 7;      // mantissa bits of the source format
     constexpr int PV = SrcTraits<SRC>::kPerVec;
-    __shared__ uint32_t s_inc[256];                   // BF16: mask16 | inc16 << 16
-    __shared__ uint32_t s_mask[SRC == HIF8_F32 ? 256 : 1];
+    constexpr bool kThr = MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR;  // packed BF16 arithmetic with an LSB term
+    __shared__ uint32_t s_inc[256];                   // BF16: mask16 | inc16 << 16 (threshold modes: mask16 | addend << 16)
+    __shared__ uint32_t s_mask[(SRC == HIF8_F32 || kThr) ? 256 : 1];  // threshold modes: the LSB term's factor
     pdl_launch_dependents();
     pdl_wait_prior_grid();  // the scale may come from the previous kernel
     const int se = resolve_scale_exp(p);
     {
         const int e = threadIdx.x, E = e - 127 + se;
-        uint32_t inc = 0, mask = 0;
+        uint32_t inc = 0, mask = 0, kfac = 0;
         if (e == 255 || (e == 0 && se > 100) || (e > 0 && E >= 15)) mask = kRareMask;
         else if ((MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR) && e > 0 && (E == -23 || E == -24)) mask = kRareMask;  // result is 0 or 2^-22
         else if (e == 0 || E <= -24) { inc = 0; mask = 0; }                                 // underflow to +0
@@ -291,9 +292,15 @@ __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, uns
             const uint32_t k = (uint32_t)(MB - mant_width(E));
             inc = 1u << (k - 1);
             mask = 0xFFFFFFFFu << k;
-            // SR2 binades (every binade for SSR, |E| >= 4 for HR) hold a quarter of the discarded field instead of
-            // half of it, marked by bit 15: the increment is quarter * (4 - T2) = quarter * (3 - 2 lsb)
-            if (MODE == HIF8_RND_SSR || (MODE == HIF8_RND_HR && (E <= -4 || E >= 4))) inc = (1u << (k - 2)) | 0x8000u;
+            if (kThr) {
+                // BF16 values in the source's own scale: the addend 0.75 ulp (0.5 ulp in a round-half-away binade of
+                // Eq. 3: every binade with |E| < 4 under hybrid rounding) and the factor -2^(6 - width) that turns the
+                // element's own LSB (2^-7 of its power of two) into LSB * 0.5 ulp
+                const int w = mant_width(E), hb = e - w - 1;  // biased exponent of 0.5 ulp
+                const bool sr2 = MODE == HIF8_RND_SSR || E <= -4 || E >= 4;
+                if (hb < 1) mask = kRareMask;
+                else { inc = ((uint32_t)hb << 7) | (sr2 ? 0x40u : 0u); kfac = sr2 ? (0x8000u | ((uint32_t)(133 - w) << 7)) : 0u; }
+            }
         }
         if (MODE == HIF8_RND_TE) {
             // biased exponent of C: the element's plus 7 - width, or that of 2^(-22 - se + 7) below the format's range
@@ -301,7 +308,10 @@ __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, uns
             const bool rare = mask == kRareMask || cb < 1 || cb > 254;
             s_inc[e] = rare ? kRareMask : (uint32_t)cb << 23;  // C in the high half
         } else if (SRC == HIF8_F32) { s_inc[e] = inc; s_mask[e] = mask; }
-        else s_inc[e] = (mask & 0xFFFFu) | (inc << 16);
+        else {
+            s_inc[e] = (mask & 0xFFFFu) | (inc << 16);
+            if (kThr) s_mask[e] = kfac;
+        }
     }
     __syncthreads();
 
@@ -348,14 +358,16 @@ __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, uns
                         continue;
                     }
                     const uint32_t mask2 = __byte_perm(tl[k], th[k], 0x5410);
-                    uint32_t inc2 = __byte_perm(tl[k], th[k], 0x7632);
-                    if (MODE != HIF8_RND_TA) {
-                        // SR2 lanes: increment = quarter * (3 - 2 lsb) = quarter + (2 quarter where the source LSB is 0)
-                        const uint32_t half2 = inc2 & 0x7FFF7FFFu;
-                        const uint32_t sr = ((inc2 >> 15) & 0x00010001u) * 0xFFFFu, odd = (w[k] & 0x00010001u) * 0xFFFFu;
-                        inc2 = half2 + ((half2 << 1) & sr & ~odd);
-                    }
-                    o[k] = (w[k] + inc2) & mask2;  // no carry between the halves: flagged exponents add nothing
+                    const uint32_t inc2 = __byte_perm(tl[k], th[k], 0x7632);
+                    if (kThr) {
+                        // SR2 rounds up iff F >= T2 / 4: x + sign * (0.75 ulp - LSB * 0.5 ulp), then the discarded bits
+                        // are cleared.  The addend lies on the significand's grid, so the sum is exact unless it carries
+                        // into the next binade, where what is left stays below the mask's cut.
+                        const uint32_t kl = s_mask[(w[k] >> 7) & 0xFFu], kh = s_mask[(w[k] >> 23) & 0xFFu];
+                        const uint32_t lsbval = fma_bf16x2(w[k] & 0xFFFEFFFEu, 0xBF80BF80u, w[k]);  // x minus x without its LSB
+                        const uint32_t adds = fma_bf16x2(lsbval, __byte_perm(kl, kh, 0x5410), inc2 | (w[k] & 0x80008000u));
+                        o[k] = fma_bf16x2(w[k], 0x3F803F80u, adds) & mask2;
+                    } else o[k] = (w[k] + inc2) & mask2;  // no carry between the halves: flagged exponents add nothing
                     rare |= tl[k] | th[k];
                 }
                 if (rare & kRareMask) {

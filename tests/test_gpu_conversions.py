@@ -262,26 +262,27 @@ def test_fake_quant(dtype, mode):
     assert_same(got, O.fake_quant(src, dtype, se, mode, 0, seed=9, quick=True), src)
 
 
-def test_fake_quant_bf16_half_even_scale_edges_and_tails():
-    # round half to even on BF16 is done in packed BF16 arithmetic with a per-exponent constant: scales at which that
-    # constant leaves the BF16 range or subnormal sources come into range, every pattern; then ragged, misaligned pieces
+@pytest.mark.parametrize("mode,omode", [(H.RND_TE, O.TE), (H.RND_HR, O.HR), (H.RND_SSR, O.SSR)])
+def test_fake_quant_bf16_packed_arithmetic_scale_edges_and_tails(mode, omode):
+    # these modes round BF16 in packed BF16 arithmetic with per-exponent constants: scales at which a constant leaves
+    # the BF16 range or subnormal sources come into range, every pattern; then ragged, misaligned pieces
     src = W.all_u16()
     d_src = to_dev(src)
-    for se in (14, -30, 100, 101, 104, 111, 112, 120, 126, -100, -105, -110, -120, -126):
+    for se in (14, -30, 100, 101, 104, 111, 112, 120, 122, 126, -100, -105, -110, -120, -126):
         _, dptr, rb = dev_empty(src.size, np.uint16)
-        H.hif8_fake_quant(d_src, dptr, H.BF16, src.size, 0, se, H.RND_TE, 0, 0)
+        H.hif8_fake_quant(d_src, dptr, H.BF16, src.size, 0, se, mode, 0, 0)
         torch.cuda.synchronize()
-        assert_same(rb(), O.fake_quant(src, O.BF16, se, O.TE, 0, quick=True), src)
+        assert_same(rb(), O.fake_quant(src, O.BF16, se, omode, 0, quick=True), src)
     part = W.llm_activation_bf16(7, 1000, seed=5).reshape(-1)
     for n, off in [(1, 0), (7, 0), (8, 0), (9, 2), (1025, 0), (4099, 6), (6999, 2)]:
         piece = part[:n]
         raw = torch.zeros(2 * n + 32, dtype=torch.uint8, device="cuda")
         raw[off:off + 2 * n] = torch.from_numpy(piece.view(np.uint8).copy()).cuda()
         out = torch.zeros(2 * n + 32, dtype=torch.uint8, device="cuda")
-        H.hif8_fake_quant(raw.data_ptr() + off, out.data_ptr() + off, H.BF16, n, 0, 5, H.RND_TE, 3, 0)
+        H.hif8_fake_quant(raw.data_ptr() + off, out.data_ptr() + off, H.BF16, n, 0, 5, mode, 3, 0)
         torch.cuda.synchronize()
         got = out[off:off + 2 * n].cpu().numpy().view(np.uint16)
-        assert_same(got, O.fake_quant(piece, O.BF16, 5, O.TE, 3, quick=True), piece)
+        assert_same(got, O.fake_quant(piece, O.BF16, 5, omode, 3, quick=True), piece)
 
 
 # ----------------------------------------------------------------------------- full sizes: sampled outputs
