@@ -2,7 +2,7 @@
 
     python -m paper_2409_16626_b200.profile_cases <case> [repeats]
 
-cases: convert_f32 (FP32 4096^2: per-tensor scaled encode + decode), fq_bf16 (BF16 4096x8192 fake-quant, TA and HR,
+cases: convert_f32 (FP32 4096^2: per-tensor scaled encode + decode), fq_bf16 (BF16 4096x8192 fake-quant, TA, HR and TE,
 fused amax and given scale), encode_modes_f32 / encode_modes_bf16 (2^25 log-uniform values, every rounding mode), gemm (HiF8 GEMM
 4096 x 7168 x 4096, fused and decode-once paths), gemm_forms (same size, decode-once path, the four operand layouts:
 forward, dgrad form, wgrad form with FP32 accumulation, both transposed), gemm_narrow (16 x 8192 x 8192, the
@@ -37,7 +37,7 @@ def main():
         xs = [torch.randn(n, generator=g, device="cuda").to(torch.bfloat16) for _ in range(3)]
         y = torch.empty_like(xs[0])
         for r in range(reps):
-            for mode in (H.RND_TA, H.RND_HR):
+            for mode in (H.RND_TA, H.RND_HR, H.RND_TE):
                 H.hif8_fake_quant(xs[r % 3], y, H.BF16, n, 1, 14, mode, 0, 7, None, None, ws, 256)
                 H.hif8_fake_quant(xs[r % 3], y, H.BF16, n, 0, 12, mode, 0, 7)
     elif case == "encode_modes_f32":
