@@ -262,10 +262,11 @@ def test_fake_quant(dtype, mode):
     assert_same(got, O.fake_quant(src, dtype, se, mode, 0, seed=9, quick=True), src)
 
 
-@pytest.mark.parametrize("mode,omode", [(H.RND_TE, O.TE), (H.RND_HR, O.HR), (H.RND_SSR, O.SSR)])
-def test_fake_quant_bf16_packed_arithmetic_scale_edges_and_tails(mode, omode):
-    # these modes round BF16 in packed BF16 arithmetic with per-exponent constants: scales at which a constant leaves
-    # the BF16 range or subnormal sources come into range, every pattern; then ragged, misaligned pieces
+@pytest.mark.parametrize("mode,omode", [(H.RND_TA, O.TA), (H.RND_TE, O.TE), (H.RND_HR, O.HR), (H.RND_SSR, O.SSR)])
+def test_fake_quant_bf16_in_place_scale_edges_and_tails(mode, omode):
+    # the in-place kernel rounds BF16 with per-exponent constants (packed BF16 arithmetic except for round half away):
+    # scales at which a constant leaves the BF16 range or subnormal sources come into range, every pattern; then ragged,
+    # misaligned pieces
     src = W.all_u16()
     d_src = to_dev(src)
     for se in (14, -30, 100, 101, 104, 111, 112, 120, 122, 126, -100, -105, -110, -120, -126):
