@@ -494,7 +494,7 @@ def main():
         t1.record(stream)
         torch.cuda.synchronize()
         # per-kernel durations, measured live: each kernel of the step in a graph of its own (POOL launches over the
-        # rotating buffers: hif8_amax -> amax_kernel behind its 8-byte memset node; hif8_encode with the scale known ->
+        # rotating buffers: hif8_amax -> the two-word clearing kernel + amax_kernel; hif8_encode with the scale known ->
         # the same convert_kernel the scaled call launches; hif8_decode -> decode_kernel), replayed between two events.
         # Direct launches would time the host's launch rate, not these ~15 us kernels.
         amax_out = torch.zeros(1, dtype=torch.float32, device="cuda")
@@ -523,7 +523,7 @@ def main():
         enc_ms = kernel_ms(lambda i, cs: H.hif8_amax_scale_encode(srcs[i], H.F32, codes[i], N_EL, 14, H.RND_TA, 0, 0, None,
                                                                   scal[0:1], scal[1:2], scal[2:3], ws, wsb, stream=cs))
     barrier()
-    launches = 3 * K   # amax + convert + decode kernels per step (graph replays)
+    launches = 4 * K   # accumulator clear + amax + convert + decode kernels per step (graph replays)
     total_ms = t0.elapsed_time(t1)
 
     # ---- end to end: pinned host input -> device, both calls, results back to pinned host memory.  Consecutive
@@ -576,7 +576,7 @@ def main():
         value = job_throughput(world, BYTES_STEP, ms_per_step)
         peak, peak_kind = load_peaks()
         kernels = {
-            "amax_kernel<f32>": {"ms": amax_ms, "bytes": 4 * N_EL, "note": "hif8_amax call: 8-byte memset node + kernel"},
+            "amax_kernel<f32>": {"ms": amax_ms, "bytes": 4 * N_EL, "note": "hif8_amax call: accumulator-clearing kernel + amax kernel"},
             "convert_kernel<f32,TA>": {"ms": conv_ms, "bytes": 5 * N_EL},
             "decode_kernel<f32>": {"ms": dec_ms, "bytes": 5 * N_EL},
         }

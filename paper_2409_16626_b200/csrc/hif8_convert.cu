@@ -404,6 +404,15 @@ __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, uns
     }
 }
 
+// Clears the amax accumulator and its ticket.  A kernel rather than a memset so that the amax kernel that follows can be
+// launched programmatically: its blocks become resident while this one drains and wait at their first global access.
+__global__ void clear_accum_kernel(uint32_t* accum)
+{
+    pdl_launch_dependents();
+    pdl_wait_prior_grid();
+    if (threadIdx.x < 2) accum[threadIdx.x] = 0u;
+}
+
 // amax only (first pass of just-in-time scaling).  A read-only pass: eight 16-byte loads in flight per thread (32 KiB per
 // block) measured 2 us faster on a 64 MiB tensor than the four of the converting kernels.
 constexpr int kUnrollAmax = 8;
@@ -700,7 +709,10 @@ static int scaled_convert(bool fq, const void* src, void* dst, int dtype, size_t
     if (jit || want_amax) {
         if (!ws || workspace_bytes < kConvWorkspaceBytes || (reinterpret_cast<uintptr_t>(ws) & 255u)) return HIF8_ERR_WORKSPACE;
         // (a delayed-scaling state keeps its two words at zero between passes itself)
-        if (!scale_state && cudaMemsetAsync(ws, 0, 8, st) != cudaSuccess) return HIF8_ERR_CUDA;
+        if (!scale_state) {
+            if (launch_pdl(clear_accum_kernel, 1u, st, ws) != cudaSuccess) return HIF8_ERR_CUDA;
+            g_launches.fetch_add(1, std::memory_order_relaxed);
+        }
     }
     p.scale_state = scale_state;
     const bool inplace_fq = fq && !want_amax && ((rnd == HIF8_RND_TA && (dtype == HIF8_F32 || dtype == HIF8_BF16)) ||
@@ -750,7 +762,8 @@ int hif8_amax(const void* src, int src_dtype, size_t n, float* d_amax_out, void*
     int sms; int rc = device_info(&sms);
     if (rc) return rc;
     cudaStream_t st = (cudaStream_t)stream;
-    if (cudaMemsetAsync(workspace, 0, 8, st) != cudaSuccess) return HIF8_ERR_CUDA;
+    if (launch_pdl(clear_accum_kernel, 1u, st, reinterpret_cast<uint32_t*>(workspace)) != cudaSuccess) return HIF8_ERR_CUDA;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
     return launch_amax(src, src_dtype, n, reinterpret_cast<uint32_t*>(workspace), d_amax_out, sms, st);
 }
 
