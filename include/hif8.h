@@ -15,6 +15,8 @@
  *     pointers take the vectorised path, others a slower scalar kernel with identical results.
  *   - Return value: HIF8_OK or an error code (see hif8_status_string).  Argument errors are detected
  *     before anything is launched and leave all outputs untouched.  NaN / Inf inputs are data.
+ *   - A conversion whose source and destination byte ranges intersect is rejected with HIF8_ERR_OVERLAP
+ *     (host-side range test; the kernels read and write in an order that makes no promise for aliased data).
  *   - `scale_exp` is the exponent E of a power-of-two scale 2^E (Section 4.2: scale factors are
  *     integer powers of two, so scaling only adds to the exponent), limited to [-126, 126].
  *   - The library needs a CUDA device of compute capability 10.0 and fails with HIF8_ERR_CUDA elsewhere.
@@ -60,18 +62,20 @@ enum {
     HIF8_ERR_ALIGN = 7,       /* GEMM operand not 16-byte aligned                   */
     HIF8_ERR_WORKSPACE = 8,   /* workspace missing or too small                     */
     HIF8_ERR_CUDA = 9,        /* a CUDA call failed (launch error, wrong device)    */
-    HIF8_ERR_DEVICE_TIMEOUT = 10 /* a bounded device-side wait gave up             */
+    HIF8_ERR_DEVICE_TIMEOUT = 10, /* a bounded device-side wait gave up            */
+    HIF8_ERR_OVERLAP = 11     /* source and destination share bytes (Section 3: a conversion reads one tensor and
+                                 writes another; only hif8_fake_quant may run in place, dst == src exactly)   */
 };
 
 /* which call a workspace size is asked for */
 enum { HIF8_WS_AMAX_SCALE_ENCODE = 0, HIF8_WS_FAKE_QUANT = 1, HIF8_WS_GEMM = 2 };
 
 /*
- * High-precision tensor -> HiF8 bytes (Section 3, "conversion from high-precision formats to HiF8").
+ * High-precision tensor -> HiF8 bytes (Section 3: rounding of FP32 / FP16 / BF16 data into the format).
  *   dst[i] = To_HiF8_<rnd>( src[i] * 2^scale_exp )
  * The scaled value is rounded as if 1.5*2^15 were representable; a result of that magnitude or more is
  * +-Inf (or +-2^15 with HIF8_FLAG_SATURATE).  Magnitudes that round to zero give 0x00 for either sign.
- * src: n elements of `src_dtype`; dst: n bytes; they must not overlap.  `seed` is used by HIF8_RND_SR only:
+ * src: n elements of `src_dtype`; dst: n bytes; they must not overlap (HIF8_ERR_OVERLAP).  `seed` is used by HIF8_RND_SR only:
  * element i takes word (i mod 4) of Philox4x32-10 with counter (i/4, 0, 0) and key `seed`; its top 24 bits
  * (FP32 source) or 16 bits (16-bit sources) are the threshold T of Section 3.2.
  */
@@ -83,7 +87,7 @@ int hif8_encode(const void* src, int src_dtype, uint8_t* dst, size_t n, int scal
  * Algorithm 1 ("Restore"):   dst[i] = value(src[i]) * 2^(-scale_exp)
  * rounded to nearest-even into `dst_dtype` when not representable (only possible at the far ends of the
  * scale range, or for FP16 destinations).  0x80 gives the canonical quiet NaN, 0x6F / 0xEF give +-Inf.
- * src: n bytes; dst: n elements; no overlap.
+ * src: n bytes; dst: n elements; no overlap (HIF8_ERR_OVERLAP).
  */
 int hif8_decode(const uint8_t* src, void* dst, int dst_dtype, size_t n, int scale_exp,
                 hif8_stream_t stream);
@@ -94,7 +98,7 @@ int hif8_decode(const uint8_t* src, void* dst, int dst_dtype, size_t n, int scal
  *        scale_exp = clamp(target_exp - floor(log2 amax), -126, 126)  (0 if amax is 0), so that
  *        amax * 2^scale_exp lies in [2^target_exp, 2^(target_exp+1)); then dst = To_HiF8(src * 2^scale_exp).
  *        Two kernels, the scale never leaves the device.
- *   d_scale_exp_in != NULL  (delayed scaling, the paper's "Amax every 10 iterations"): the scale exponent
+ *   d_scale_exp_in != NULL  (delayed scaling: Section 5.1 measures amax once per ten iterations): the scale exponent
  *        is read from that device int; amax of this tensor is still produced for the next update.  One pass.
  * Outputs (device scalars, each may be NULL): d_amax_out (float, exact), d_scale_exp_out (int, the exponent
  * used), d_scale_out (float 2^scale_exp).  workspace: hif8_workspace_bytes(HIF8_WS_AMAX_SCALE_ENCODE, n)
@@ -107,7 +111,8 @@ int hif8_amax_scale_encode(const void* src, int src_dtype, uint8_t* dst, size_t 
                            size_t workspace_bytes, hif8_stream_t stream);
 
 /*
- * Amax alone (Section 5.1: "every 10 iterations, we compute the maximum absolute value (Amax) of each tensor"):
+ * Amax alone (Section 5.1, per-tensor scaling: the largest magnitude of each GEMM input tensor is measured at a fixed
+ * cadence of iterations and the tensor's scale follows from it):
  *   *d_amax_out = max |src[i]| over the finite elements (0 if there is none), as an exact float.
  * One read of the tensor.  workspace as for hif8_amax_scale_encode.  The caller derives the next scale exponent
  * from it (or lets hif8_amax_scale_encode do both in one call).
@@ -156,8 +161,8 @@ int hif8_amax_scale_encode_static(const void* src, int src_dtype, uint8_t* dst, 
                                   int* d_scale_exp_out, float* d_scale_out, hif8_stream_t stream);
 
 /*
- * Per-channel scaled conversion of a weight matrix (Section 5.1, end: "per-tensor scaling for activations and
- * per-channel scaling for weights"; repeated in the outlook of Section 5.3).  W is [rows, cols] row-major and
+ * Per-channel scaled conversion of a weight matrix (Section 4.2 and the closing remarks of Section 5 and Section 6 name
+ * the combination of one scale per activation tensor with one scale per weight channel).  W is [rows, cols] row-major and
  * contiguous; every output channel has its own power-of-two scale:
  *   channel_axis = 0: channel = row    (weights stored [N,K]);   channel_axis = 1: channel = column (stored [K,N]).
  *   d_scale_exp_in == NULL: per channel, amax over the channel's finite elements and
@@ -177,8 +182,8 @@ int hif8_channel_amax_scale_encode(const void* W, int src_dtype, uint8_t* dst, i
                                    hif8_stream_t stream);
 
 /*
- * The every-N-iterations cadence of per-tensor scaling in training (Section 5.1: scale factors start at 1; "every 10
- * iterations" the amax of each tensor is computed and its scale updated; the scale in force is applied in every
+ * The every-N-iterations cadence of per-tensor scaling in training (Section 5.1: scale factors start at 1; once per ten
+ * iterations the amax of each tensor is measured and its scale updated; the scale in force is applied in every
  * iteration, updated or not).  The paper does not give the update rule; this library keeps, per tensor, the exponent
  * in force and a ring of the last `hist_len` measured amax values, and after a measurement sets
  *   scale_exp = clamp(target_exp - floor(log2 max(ring)), -126, 126)      (0 while every entry is 0)
@@ -220,12 +225,12 @@ int hif8_als_update(void* d_state, int* d_found_inf, hif8_stream_t stream);
 int hif8_check_finite(const void* src, int dtype, size_t n, int* d_found_inf, hif8_stream_t stream);
 
 /*
- * Quantize-dequantize in the source format ("simulated HiF8", Section 4: values are converted to only those
- * representable in HiF8):   dst[i] = value( To_HiF8_<rnd>(src[i] * 2^e) ) * 2^(-e)   in `dtype`.
+ * Quantize-dequantize in the source format (Section 4: the paper's experiments simulate the format by replacing every
+ * value with its nearest HiF8-representable one):   dst[i] = value( To_HiF8_<rnd>(src[i] * 2^e) ) * 2^(-e)   in `dtype`.
  *   use_amax == 0: e = scale_or_target_exp.  No workspace needed (may be NULL).
  *   use_amax == 1: e derived from the tensor's amax with target exponent scale_or_target_exp, as in
  *                  hif8_amax_scale_encode (two kernels); workspace as for HIF8_WS_FAKE_QUANT.
- * dst may be the same pointer as src (in place); partial overlap is not allowed.
+ * dst may be the same pointer as src (in place); any other overlap is rejected with HIF8_ERR_OVERLAP.
  * d_amax_out / d_scale_exp_out: optional device scalars as above.
  */
 int hif8_fake_quant(const void* src, void* dst, int dtype, size_t n, int use_amax, int scale_or_target_exp,
@@ -301,6 +306,22 @@ int hif8_encode_transpose(const void* src, int src_dtype, uint8_t* dst, int64_t 
  * The only entry point that blocks the host.
  */
 int hif8_gemm_status(const void* workspace, hif8_stream_t stream);
+
+/*
+ * Status of the most recent GEMM-class call (hif8_gemm, hif8_gemm_ex, hif8_gemm_channel_scaled, hif8_pts_search,
+ * hif8_selftest_wait_timeout) enqueued on `stream` of the current device, without the caller naming the workspace:
+ * the library remembers, per stream, where that call's status word lives.  SYNCHRONISES `stream`, then returns HIF8_OK,
+ * HIF8_ERR_DEVICE_TIMEOUT, or HIF8_ERR_CUDA (read failed, or another device is current).  HIF8_OK when no such call was
+ * made on the stream.  The workspace of that call must still be allocated.  (Algorithm 1 has no counterpart; this is
+ * the host-side end of the bounded device-side waits.)
+ */
+int hif8_last_device_status(hif8_stream_t stream);
+
+/*
+ * Self-test of the host-side caches (no device needed): the once-per-device set-up record and the tensor-map cache are
+ * driven with synthetic keys; returns HIF8_OK, or HIF8_ERR_SHAPE with the number of the failed check in *failed_check.
+ */
+int hif8_selftest_host_caches(int* failed_check);
 
 /*
  * Self-test of the device-side failure detection: launches one warp that waits, with a limit of `limit_ms`

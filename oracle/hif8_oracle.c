@@ -34,7 +34,11 @@
  * the TE/TA worked example, the 0.5 / 0.75 / 1 ulp error bounds, the 2^-20 tie
  * probability, the SR expectation identity) and by closed forms.  The bit-level
  * placement of F14 inside the discarded field (Fig. 2 of the paper is not
- * available) is pinned only through the 1-ulp bound and unbiasedness.
+ * available) is pinned by vectors worked out by hand from the sentence of
+ * Section 3.2 (tests/golden/sr14_hand_vectors.txt), besides the 1-ulp bound and
+ * unbiasedness.  hif8o_encode_at / hif8o_fake_quant_at (elements addressed by
+ * their flat index) are pinned against the whole-tensor entry points and
+ * against thresholds built from the Philox known answers.
  */
 #include <math.h>
 #include <stddef.h>
@@ -394,6 +398,18 @@ void hif8o_encode(const void* src, int dtype, uint8_t* dst, size_t n, int scale_
     }
 }
 
+/* As hif8o_encode for elements picked out of a larger tensor: element j is src[j] and sat at flat position
+ * idx[j] there, which is what the standard-SR word is drawn for (READING: the counter follows the flat index). */
+void hif8o_encode_at(const void* src, int dtype, uint8_t* dst, size_t n, const uint64_t* idx, int scale_exp, int rnd,
+                     unsigned flags, uint64_t seed, int quick)
+{
+#pragma omp parallel for schedule(static)
+    for (long long j = 0; j < (long long)n; j++) {
+        uint32_t raw; double x = src_to_double(src, (size_t)j, dtype, &raw);
+        dst[j] = (uint8_t)encode_value(x, raw, dtype, scale_exp, rnd, flags, seed, idx[j], quick);
+    }
+}
+
 /* encode the FP32 values whose encodings are first, first+1, ... (exhaustive sweeps) */
 void hif8o_encode_f32_range(uint32_t first, size_t n, uint8_t* dst, int scale_exp, int rnd,
                             unsigned flags, uint64_t seed, int quick)
@@ -429,8 +445,8 @@ static int scale_exp_for(double amax, int target_exp)
 }
 
 /* amax over the finite elements and the power-of-two scale that brings it into
- * [2^target_exp, 2^(target_exp+1)).  READING of "update the scale factor by a
- * certain algorithm": scale_exp = target_exp - floor(log2 amax), clamped to
+ * [2^target_exp, 2^(target_exp+1)).  READING (Section 5.1 leaves the update rule
+ * open): scale_exp = target_exp - floor(log2 amax), clamped to
  * [-126,126]; no finite non-zero element -> 0.  NaN / Inf do not take part. */
 void hif8o_amax_scale(const void* src, int dtype, size_t n, int target_exp, float* amax_out,
                       int* scale_exp_out)
@@ -446,7 +462,7 @@ void hif8o_amax_scale(const void* src, int dtype, size_t n, int target_exp, floa
     *scale_exp_out = se;
 }
 
-/* quantize-dequantize in the source format ("simulated HiF8", Section 4) */
+/* quantize-dequantize in the source format (Section 4: how the paper's experiments simulate the format) */
 void hif8o_fake_quant(const void* src, void* dst, int dtype, size_t n, int scale_exp, int rnd,
                       unsigned flags, uint64_t seed, int quick)
 {
@@ -455,6 +471,18 @@ void hif8o_fake_quant(const void* src, void* dst, int dtype, size_t n, int scale
         uint32_t raw; double x = src_to_double(src, (size_t)i, dtype, &raw);
         unsigned c = encode_value(x, raw, dtype, scale_exp, rnd, flags, seed, (uint64_t)i, quick);
         store_as(dst, (size_t)i, dtype, ldexp(hif8o_value(c), -scale_exp));
+    }
+}
+
+/* quantize-dequantize of elements picked out of a larger tensor (see hif8o_encode_at) */
+void hif8o_fake_quant_at(const void* src, void* dst, int dtype, size_t n, const uint64_t* idx, int scale_exp, int rnd,
+                         unsigned flags, uint64_t seed, int quick)
+{
+#pragma omp parallel for schedule(static)
+    for (long long j = 0; j < (long long)n; j++) {
+        uint32_t raw; double x = src_to_double(src, (size_t)j, dtype, &raw);
+        unsigned c = encode_value(x, raw, dtype, scale_exp, rnd, flags, seed, idx[j], quick);
+        store_as(dst, (size_t)j, dtype, ldexp(hif8o_value(c), -scale_exp));
     }
 }
 
@@ -502,13 +530,12 @@ void hif8o_gemm_full(const uint8_t* Aq, long long lda, const uint8_t* Wq, long l
         }
 }
 
-/* Algorithm 1 (HiF8 Calibration with Per-Tensor Scaling), the search of one layer:
- *   for Ea in [e_min, e_max], Ew in [e_min, e_max]:
- *     A_q = To_HiF8_TA(A * 2^Ea), W_q = To_HiF8_TA(W * 2^Ew)          ("Scale & Cast")
- *     O_q = (A_q x W_q) * 2^-(Ea+Ew)                                   ("MatMul & Restore")
- *     err[Ea][Ew] = mean over all outputs of (O_q - O)^2               ("Quantization Error": MSE)
- *   best = argmin err (READING: the first minimum in row-major (Ea, Ew) order on exact ties).
- * A is [M,K] row-major, W is [K,N] or (w_is_nk) [N,K], both of `dtype`; O is the high-precision output [M,N] float.
+/* Algorithm 1, the calibration search of one layer.  Every pair of integer exponents (Ea, Ew) of the grid
+ * [e_min, e_max]^2 is tried: activation and weight are multiplied by 2^Ea and 2^Ew and rounded half away to HiF8, the two
+ * HiF8 tensors are multiplied, the product is scaled back by 2^-(Ea+Ew), and its mean squared difference to the layer's
+ * high-precision output O is the error of that pair; the pair with the smallest error is kept (READING: the first such
+ * pair in row-major (Ea, Ew) order on exact ties).
+ * A is [M,K] row-major, W is [K,N] or (w_is_nk) [N,K], both of `dtype`; O is [M,N] float.
  * Everything after the cast is computed in double. */
 void hif8o_pts_search(const void* A, const void* W, int dtype, int w_is_nk, const float* O, int M, int N, int K,
                       int e_min, int e_max, int quick, double* err, int* best)
@@ -553,8 +580,9 @@ void hif8o_pts_search(const void* A, const void* W, int dtype, int w_is_nk, cons
 }
 
 /* ------------------------------------------------------------------------- *
- * Section 5.1 / 5.3 outlook: "per-tensor scaling for activations and per-channel
- * scaling for weights".  A weight matrix W [rows, cols] (row-major) gets one
+ * Section 4.2 and the closing remarks of Sections 5 and 6 name the pairing of one
+ * scale per activation tensor with one scale per weight channel; the paper does
+ * not evaluate it.  A weight matrix W [rows, cols] (row-major) gets one
  * power-of-two scale per output channel: channel = row (axis 0, weights stored
  * [N,K]) or channel = column (axis 1, weights stored [K,N]).  Each channel's
  * amax and scale exponent follow the per-tensor rule applied to the elements of
@@ -613,11 +641,10 @@ void hif8o_gemm_entries_channel(const uint8_t* Aq, long long lda, const uint8_t*
 }
 
 /* ------------------------------------------------------------------------- *
- * Section 5.1, the cadence of per-tensor scaling in training: "the initial scale
- * factors are all set to 1.  Then every 10 iterations, we compute [Amax] of each
- * tensor, and update the corresponding scale factor by a certain algorithm ...
- * in each iteration, whether the scale factors are updated or not, they will
- * scale the corresponding tensors".
+ * Section 5.1, the cadence of per-tensor scaling in training: all scale factors
+ * start at 1; once per ten iterations the amax of each tensor is measured and
+ * its scale factor is updated (the update rule is not given); the factor in
+ * force is applied in every iteration, updated or not.
  * READING (the update algorithm is not given; the text likens the scheme to FP8
  * delayed scaling): the state is the exponent in force (initially 0) and a ring
  * of the last `hist_len` measured amax values (initially empty).  Iteration t
@@ -691,17 +718,15 @@ void hif8o_gemm_entries_ex(const uint8_t* Aq, long long lda, int a_is_km, const 
 /* ------------------------------------------------------------------------- *
  * Section 5.1, "Adaptive Loss-Scaling (ALS)": backward loss scaling whose scale
  * window (growth interval) moves along the list {1, 20, 50, 100, 200, 500, 1000}.
- * "The initial scale value and scale window are set to 2^32 and 20.  During
- * training, if the scale value increases three times, the scale window will
- * increase once as per the list order.  If the scale value decreases three times
- * in a row, scale window will decrease once."
+ * The scale starts at 2^32 with window 20; after three increases of the scale the
+ * window moves one entry up the list, after three decreases in a row one entry down.
  * The scale itself follows the usual dynamic loss scaling the paper builds on
  * (growth factor 2, backoff factor 1/2, so the scale stays a power of two):
  *   overflow seen in this iteration's gradients -> scale / 2, clean-step counter = 0
  *   otherwise clean-step counter + 1; when it reaches the window -> scale * 2, counter = 0.
- * READINGS: "increases three times" counts increases since the last window change
- * (decreases in between do not cancel them); "decreases three times in a row" is a run
- * of decreases not interrupted by an increase; a window change clears both counts; the
+ * READINGS: the three increases are counted since the last window change (decreases
+ * in between do not cancel them); three decreases in a row are a run of decreases not
+ * interrupted by an increase; a window change clears both counts; the
  * window stops at the ends of the list; the exponent is kept within [-126, 126].
  * found_inf[t] != 0: the gradients of iteration t held an Inf or NaN.
  * scale_exp[t], window[t]: log2 of the scale, and the window, in force DURING iteration t.

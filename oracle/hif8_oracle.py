@@ -25,6 +25,8 @@ _lib.hif8o_sr_word.argtypes = [_u64, _u64]
 _lib.hif8o_philox4x32_10.argtypes = [_vp, _vp, _vp]
 _lib.hif8o_num_threads.restype = _i
 _lib.hif8o_encode.argtypes = [_vp, _i, _vp, _sz, _i, _i, _u, _u64, _i]
+_lib.hif8o_encode_at.argtypes = [_vp, _i, _vp, _sz, _vp, _i, _i, _u, _u64, _i]
+_lib.hif8o_fake_quant_at.argtypes = [_vp, _vp, _i, _sz, _vp, _i, _i, _u, _u64, _i]
 _lib.hif8o_encode_f32_range.argtypes = [C.c_uint32, _sz, _vp, _i, _i, _u, _u64, _i]
 _lib.hif8o_decode.argtypes = [_vp, _vp, _i, _sz, _i]
 _lib.hif8o_amax_scale.argtypes = [_vp, _i, _sz, _i, C.POINTER(C.c_float), C.POINTER(C.c_int)]
@@ -99,6 +101,25 @@ def encode(src, dtype, scale_exp=0, rnd=TA, flags=0, seed=0, quick=False):
     a = _src(src, dtype)
     out = np.empty(a.size, dtype=np.uint8)
     _lib.hif8o_encode(_ptr(a), dtype, _ptr(out), a.size, scale_exp, rnd, flags, seed, int(quick))
+    return out.reshape(a.shape)
+
+
+def encode_at(src, dtype, idx, scale_exp=0, rnd=TA, flags=0, seed=0, quick=False):
+    """Codes of elements taken out of a larger tensor: src[j] sat at flat position idx[j] (matters for SR only)."""
+    a = _src(src, dtype)
+    ix = np.ascontiguousarray(idx, dtype=np.uint64)
+    assert ix.size == a.size
+    out = np.empty(a.size, dtype=np.uint8)
+    _lib.hif8o_encode_at(_ptr(a), dtype, _ptr(out), a.size, _ptr(ix), scale_exp, rnd, flags, seed, int(quick))
+    return out.reshape(a.shape)
+
+
+def fake_quant_at(src, dtype, idx, scale_exp=0, rnd=TA, flags=0, seed=0, quick=False):
+    a = _src(src, dtype)
+    ix = np.ascontiguousarray(idx, dtype=np.uint64)
+    assert ix.size == a.size
+    out = np.empty(a.size, dtype=_out_dtype(dtype))
+    _lib.hif8o_fake_quant_at(_ptr(a), _ptr(out), dtype, a.size, _ptr(ix), scale_exp, rnd, flags, seed, int(quick))
     return out.reshape(a.shape)
 
 

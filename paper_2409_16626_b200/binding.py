@@ -22,7 +22,7 @@ LIB_PATH = os.path.join(_HERE, "libhif8.so")
 EXPORTS = ["hif8_encode", "hif8_decode", "hif8_amax", "hif8_amax_scale_encode", "hif8_fake_quant", "hif8_gemm", "hif8_gemm_status", "hif8_pts_search", "hif8_pts_workspace_bytes",
            "hif8_pts_status", "hif8_selftest_wait_timeout", "hif8_channel_amax_scale_encode", "hif8_gemm_channel_scaled",
            "hif8_scale_state_init", "hif8_delayed_scale_encode", "hif8_gemm_ex", "hif8_encode_transpose", "hif8_als_state_init", "hif8_als_update", "hif8_check_finite", "hif8_encode_from_amax",
-           "hif8_amax_scale_encode_static", "hif8_workspace_bytes", "hif8_status_string", "hif8_launch_count"]
+           "hif8_amax_scale_encode_static", "hif8_last_device_status", "hif8_selftest_host_caches", "hif8_workspace_bytes", "hif8_status_string", "hif8_launch_count"]
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2409_16626_b200.build` (needs nvcc)")
@@ -46,6 +46,10 @@ lib.hif8_pts_workspace_bytes.argtypes = [_i, _i, _i, _i]
 lib.hif8_pts_workspace_bytes.restype = _sz
 lib.hif8_pts_status.argtypes = [_vp, _vp]
 lib.hif8_pts_status.restype = _i
+lib.hif8_last_device_status.argtypes = [_vp]
+lib.hif8_last_device_status.restype = _i
+lib.hif8_selftest_host_caches.argtypes = [_vp]
+lib.hif8_selftest_host_caches.restype = _i
 lib.hif8_selftest_wait_timeout.argtypes = [_vp, _u, _vp]
 lib.hif8_selftest_wait_timeout.restype = _i
 lib.hif8_channel_amax_scale_encode.argtypes = [_vp, _i, _vp, _i64, _i64, _i, _i, _i, _u, _u64, _vp, _vp, _vp, _vp]
@@ -176,6 +180,17 @@ def hif8_pts_search(A, W, dtype, w_is_nk, O_ref, ldo, M, N, K, e_min, e_max, d_e
 
 def hif8_pts_status(workspace, stream=None):
     return int(lib.hif8_pts_status(_ptr(workspace), _stream(stream)))
+
+
+def hif8_last_device_status(stream=None):
+    return int(lib.hif8_last_device_status(_stream(stream)))
+
+
+def hif8_selftest_host_caches():
+    """(status, number of the failed check or 0)"""
+    failed = C.c_int(-1)
+    rc = int(lib.hif8_selftest_host_caches(C.byref(failed)))
+    return rc, int(failed.value)
 
 
 def hif8_selftest_wait_timeout(workspace, limit_ms, stream=None, check=True):

@@ -478,6 +478,8 @@ extern "C" int hif8_channel_amax_scale_encode(const void* W, int src_dtype, uint
         return HIF8_OK;
     }
     if (!W || !dst || (!d_scale_exp_in && !d_amax)) return HIF8_ERR_NULL;
+    if (ranges_overlap(W, (size_t)rows * (size_t)cols * dtype_bytes(src_dtype), dst, (size_t)rows * (size_t)cols))
+        return HIF8_ERR_OVERLAP;
     Plan pl{};
     int rc = checked_device(&pl.sms);
     if (rc) return rc;

@@ -660,6 +660,7 @@ int hif8_encode(const void* src, int src_dtype, uint8_t* dst, size_t n, int scal
     if (scale_exp < -126 || scale_exp > 126) return HIF8_ERR_SCALE_RANGE;
     if (n == 0) return HIF8_OK;
     if (!src || !dst) return HIF8_ERR_NULL;
+    if (ranges_overlap(src, n * dtype_bytes(src_dtype), dst, n)) return HIF8_ERR_OVERLAP;
     int sms; rc = device_info(&sms);
     if (rc) return rc;
     ConvParams p{};
@@ -675,6 +676,7 @@ int hif8_decode(const uint8_t* src, void* dst, int dst_dtype, size_t n, int scal
     if (scale_exp < -126 || scale_exp > 126) return HIF8_ERR_SCALE_RANGE;
     if (n == 0) return HIF8_OK;
     if (!src || !dst) return HIF8_ERR_NULL;
+    if (ranges_overlap(src, n, dst, n * dtype_bytes(dst_dtype))) return HIF8_ERR_OVERLAP;
     int sms; int rc = device_info(&sms);
     if (rc) return rc;
     unsigned long long pv = dst_dtype == HIF8_F32 ? 4 : 8;
@@ -746,6 +748,7 @@ int hif8_amax_scale_encode(const void* src, int src_dtype, uint8_t* dst, size_t 
     if (!workspace || workspace_bytes < kConvWorkspaceBytes || (reinterpret_cast<uintptr_t>(workspace) & 255u))
         return HIF8_ERR_WORKSPACE;
     if (n && (!src || !dst)) return HIF8_ERR_NULL;
+    if (ranges_overlap(src, n * dtype_bytes(src_dtype), dst, n)) return HIF8_ERR_OVERLAP;
     bool jit = d_scale_exp_in == nullptr;
     return scaled_convert(false, src, dst, src_dtype, n, jit, target_exp, d_scale_exp_in, 0, rnd, flags, seed,
                           d_amax_out, d_scale_exp_out, d_scale_out, workspace, workspace_bytes, !jit,
@@ -775,6 +778,7 @@ int hif8_encode_from_amax(const void* src, int src_dtype, uint8_t* dst, size_t n
     if (target_exp < -22 || target_exp > 15) return HIF8_ERR_SCALE_RANGE;
     if (!d_amax || (n && (!src || !dst))) return HIF8_ERR_NULL;
     if (reinterpret_cast<uintptr_t>(d_amax) & 3u) return HIF8_ERR_ALIGN;
+    if (ranges_overlap(src, n * dtype_bytes(src_dtype), dst, n)) return HIF8_ERR_OVERLAP;
     int sms; rc = device_info(&sms);
     if (rc) return rc;
     ConvParams p{};
@@ -797,6 +801,8 @@ int hif8_fake_quant(const void* src, void* dst, int dtype, size_t n, int use_ama
             return HIF8_ERR_WORKSPACE;
     } else if (scale_or_target_exp < -126 || scale_or_target_exp > 126) return HIF8_ERR_SCALE_RANGE;
     if (n && (!src || !dst)) return HIF8_ERR_NULL;
+    // in place (the same pointer) is allowed; any other sharing of bytes is not
+    if (src != dst && ranges_overlap(src, n * dtype_bytes(dtype), dst, n * dtype_bytes(dtype))) return HIF8_ERR_OVERLAP;
     if (n == 0 && !use_amax) return HIF8_OK;
     return scaled_convert(true, src, dst, dtype, n, use_amax != 0, scale_or_target_exp, nullptr,
                           use_amax ? 0 : scale_or_target_exp, rnd, flags, seed, d_amax_out, d_scale_exp_out, nullptr,
@@ -827,6 +833,7 @@ const char* hif8_status_string(int status)
         case HIF8_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case HIF8_ERR_CUDA: return "CUDA call failed or device is not compute capability 10.0";
         case HIF8_ERR_DEVICE_TIMEOUT: return "bounded device-side wait gave up";
+        case HIF8_ERR_OVERLAP: return "source and destination share bytes";
         default: return "unknown status";
     }
 }
@@ -845,20 +852,20 @@ constexpr size_t kStaticScratchBytes = 256;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 // Device address of g_static_scratch per device ordinal.  In host code the array's name is only a handle for
 // the runtime, not an address a kernel may dereference; the real address comes from cudaGetSymbolAddress.
-void* g_static_scratch_addr[64];
-std::atomic<int> g_static_scratch_ready[64];
+std::atomic<void*> g_static_scratch_addr[64];
+static_assert(kStaticScratchBytes == HIF8_STATIC_SCRATCH_BYTES, "the header states the size of the array");
+static_assert(kStaticScratchBytes >= kConvWorkspaceBytes, "the array stands in for the conversion workspace");
 
 int static_scratch(void** out)
 {
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return HIF8_ERR_CUDA;
-    if (!g_static_scratch_ready[dev].load(std::memory_order_acquire)) {
-        void* ptr = nullptr;
+    void* ptr = g_static_scratch_addr[dev].load(std::memory_order_acquire);
+    if (!ptr) {
         if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) return HIF8_ERR_CUDA;
-        g_static_scratch_addr[dev] = ptr;  // the same value from every racing thread
-        g_static_scratch_ready[dev].store(1, std::memory_order_release);
+        g_static_scratch_addr[dev].store(ptr, std::memory_order_release);  // racing first callers store the same value
     }
-    *out = g_static_scratch_addr[dev];
+    *out = ptr;
     return HIF8_OK;
 }
 }  // namespace
@@ -873,6 +880,7 @@ extern "C" int hif8_amax_scale_encode_static(const void* src, int src_dtype, uin
     if (target_exp < -22 || target_exp > 15) return HIF8_ERR_SCALE_RANGE;
     if (n > HIF8_STATIC_MAX_ELEMENTS) return HIF8_ERR_SHAPE;
     if (n && (!src || !dst)) return HIF8_ERR_NULL;
+    if (ranges_overlap(src, n * dtype_bytes(src_dtype), dst, n)) return HIF8_ERR_OVERLAP;
     void* scratch = nullptr;
     rc = static_scratch(&scratch);
     if (rc) return rc;
@@ -921,6 +929,7 @@ extern "C" int hif8_delayed_scale_encode(const void* src, int src_dtype, uint8_t
     if (target_exp < -22 || target_exp > 15) return HIF8_ERR_SCALE_RANGE;
     if (!d_state || (n && (!src || !dst))) return HIF8_ERR_NULL;
     if (reinterpret_cast<uintptr_t>(d_state) & 255u) return HIF8_ERR_WORKSPACE;
+    if (ranges_overlap(src, n * dtype_bytes(src_dtype), dst, n)) return HIF8_ERR_OVERLAP;
     ScaleState* state = reinterpret_cast<ScaleState*>(d_state);
     cudaStream_t st = (cudaStream_t)stream;
     if (!measure)  // conversion alone, exponent read from the state on the device

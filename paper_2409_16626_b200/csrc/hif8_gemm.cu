@@ -28,9 +28,11 @@
 
 #include <atomic>
 #include <cstdint>
+#include <cstring>
 #include <mutex>
 
 #include "hif8.h"
+#include "hif8_host_cache.h"
 #include "hif8_internal.cuh"
 
 namespace hif8 {
@@ -1034,63 +1036,117 @@ EncodeTiledFn encode_tiled_fn()
     return fn;
 }
 
+// Tensor maps are cached per (pointer, shape, leading dimension, box): encoding one costs a driver call of a few
+// microseconds, which matters for the narrow products of ~100 us when the same operands come back call after call.
+struct MapKey {
+    const void* ptr;
+    uint64_t inner, rows, count, ld;  // ld: row pitch in elements (2-D) or distance between stacked matrices (3-D)
+    uint32_t box_inner, box_rows;
+    uint32_t kind;                    // 0: bytes, 2-D; 1: BF16, 2-D, 128-byte swizzle; 2: BF16, 3-D stack, 128-byte swizzle
+    uint32_t pad;
+};
+LruCache<MapKey, CUtensorMap, 64> g_map_cache;
+
+bool encode_map(const MapKey& k, CUtensorMap* map)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const bool bf16 = k.kind != 0;
+    if (k.kind == 2) {
+        cuuint64_t dims[3] = {k.inner, k.rows, k.count};
+        cuuint64_t strides[2] = {k.inner * 2u, (k.count > 1 ? k.ld : k.inner * k.rows) * 2u};
+        cuuint32_t box[3] = {k.box_inner, k.box_rows, 1};
+        cuuint32_t estr[3] = {1, 1, 1};
+        return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(k.ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    }
+    cuuint64_t dims[2] = {k.inner, k.rows};
+    cuuint64_t strides[1] = {k.ld * (bf16 ? 2u : 1u)};
+    cuuint32_t box[2] = {k.box_inner, k.box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(k.ptr), dims,
+              strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, bf16 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // 2-D tensor [rows][ld elements] with a box of box_inner x box_rows elements, zero fill out of bounds.
 // bf16 = false: bytes, no swizzle.  bf16 = true: 16-bit elements, 128-byte swizzle (box_inner must be 64).
 bool make_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t rows, uint64_t ld, uint32_t box_inner, uint32_t box_rows,
               bool bf16 = false)
 {
-    EncodeTiledFn fn = encode_tiled_fn();
-    if (!fn) return false;
-    cuuint64_t dims[2] = {inner, rows};
-    cuuint64_t strides[1] = {ld * (bf16 ? 2u : 1u)};
-    cuuint32_t box[2] = {box_inner, box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    return fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims,
-              strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, bf16 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    MapKey k;
+    std::memset(&k, 0, sizeof k);
+    k.ptr = ptr; k.inner = inner; k.rows = rows; k.count = 1; k.ld = ld; k.box_inner = box_inner; k.box_rows = box_rows;
+    k.kind = bf16 ? 1u : 0u;
+    return g_map_cache.lookup_or_make(k, map, encode_map);
 }
 
 // BF16 stack of `count` matrices [rows, inner], `stack_stride` elements apart (box: one matrix deep)
 bool make_map3(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t rows, uint64_t count, uint64_t stack_stride,
                uint32_t box_inner, uint32_t box_rows)
 {
-    EncodeTiledFn fn = encode_tiled_fn();
-    if (!fn) return false;
-    cuuint64_t dims[3] = {inner, rows, count};
-    cuuint64_t strides[2] = {inner * 2u, (count > 1 ? stack_stride : inner * rows) * 2u};
-    cuuint32_t box[3] = {box_inner, box_rows, 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    MapKey k;
+    std::memset(&k, 0, sizeof k);
+    k.ptr = ptr; k.inner = inner; k.rows = rows; k.count = count; k.ld = count > 1 ? stack_stride : 0; k.box_inner = box_inner;
+    k.box_rows = box_rows; k.kind = 2u;
+    return g_map_cache.lookup_or_make(k, map, encode_map);
 }
 
-// one-time kernel attributes (dynamic shared memory) and the SM count of the device
+// Kernel attributes (opt-in to more than 48 KiB of dynamic shared memory) and the SM count are facts of one device:
+// they are set up once per device ordinal, by the first GEMM call made with that device current.
+struct GemmDeviceSetup {
+    cudaError_t rc;
+    int sm_count;
+};
+PerDevice<GemmDeviceSetup> g_gemm_setup;
+
 bool gemm_kernels_ready(int dev, int* sm_count_out)
 {
-    static std::once_flag attr_once;
-    static cudaError_t attr_rc = cudaSuccess;
-    static int sm_count = 0;
-    std::call_once(attr_once, [dev] {
+    const GemmDeviceSetup* s = g_gemm_setup.get(dev, [](int d, GemmDeviceSetup* out) {
+        out->rc = cudaSuccess;
+        out->sm_count = 0;
         const void* fused[4] = {(const void*)hif8_gemm_kernel<false, false>, (const void*)hif8_gemm_kernel<false, true>,
                                 (const void*)hif8_gemm_kernel<true, false>, (const void*)hif8_gemm_kernel<true, true>};
         const void* pair[2] = {(const void*)bf16_gemm_pair_kernel<false>, (const void*)bf16_gemm_pair_kernel<true>};
-        for (int i = 0; i < 4 && attr_rc == cudaSuccess; i++)
-            attr_rc = cudaFuncSetAttribute(fused[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
-        for (int i = 0; i < 2 && attr_rc == cudaSuccess; i++)
-            attr_rc = cudaFuncSetAttribute(pair[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
-        if (attr_rc == cudaSuccess)
-            attr_rc = cudaFuncSetAttribute(hif8_gemm_narrow_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytesN);
-        if (attr_rc == cudaSuccess)
-            attr_rc = cudaFuncSetAttribute(hif8_gemm_narrow_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytesN);
-        if (attr_rc == cudaSuccess) attr_rc = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+        for (int i = 0; i < 4 && out->rc == cudaSuccess; i++)
+            out->rc = cudaFuncSetAttribute(fused[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        for (int i = 0; i < 2 && out->rc == cudaSuccess; i++)
+            out->rc = cudaFuncSetAttribute(pair[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
+        if (out->rc == cudaSuccess)
+            out->rc = cudaFuncSetAttribute(hif8_gemm_narrow_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytesN);
+        if (out->rc == cudaSuccess)
+            out->rc = cudaFuncSetAttribute(hif8_gemm_narrow_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytesN);
+        if (out->rc == cudaSuccess) out->rc = cudaDeviceGetAttribute(&out->sm_count, cudaDevAttrMultiProcessorCount, d);
     });
-    *sm_count_out = sm_count;
-    return attr_rc == cudaSuccess && sm_count > 0;
+    if (!s) return false;
+    *sm_count_out = s->sm_count;
+    return s->rc == cudaSuccess && s->sm_count > 0;
 }
+
+// The status word of the most recent GEMM-class call per stream, for hif8_last_device_status.
+struct StatusKey {
+    const void* stream;
+};
+struct StatusVal {
+    const int* word;
+    int dev;
+};
+LruCache<StatusKey, StatusVal, 64> g_last_status;
 
 constexpr size_t kGemmWorkspaceBytes = 256;
 
 }  // namespace
+
+void note_status_word(cudaStream_t st, const int* word)
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return;
+    StatusKey k;
+    std::memset(&k, 0, sizeof k);
+    k.stream = st;
+    g_last_status.put(k, StatusVal{word, dev});
+}
 
 int launch_bf16_pair_gemm(const void* a_bf, const void* w_bf, int w_is_nk, GemmParams p, cudaStream_t st,
                           long long a_stack_stride, long long w_stack_stride)
@@ -1173,6 +1229,7 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t
     if (tiles2 > 0x3FFFFFFF) return HIF8_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMemsetAsync(workspace, 0, 4, st) != cudaSuccess) return HIF8_ERR_CUDA;
+    note_status_word(st, reinterpret_cast<const int*>(workspace));
 
     int sm_count = 0;
     if (!gemm_kernels_ready(dev, &sm_count)) return HIF8_ERR_CUDA;
@@ -1286,12 +1343,66 @@ extern "C" int hif8_gemm_status(const void* workspace, hif8_stream_t stream)
     return v == 0 ? HIF8_OK : HIF8_ERR_DEVICE_TIMEOUT;
 }
 
+extern "C" int hif8_last_device_status(hif8_stream_t stream)
+{
+    StatusKey k;
+    std::memset(&k, 0, sizeof k);
+    k.stream = (cudaStream_t)stream;
+    StatusVal v;
+    if (!g_last_status.find(k, &v)) return HIF8_OK;  // no GEMM-class call was made on this stream
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != v.dev) return HIF8_ERR_CUDA;
+    return hif8_gemm_status(v.word, stream);
+}
+
+extern "C" int hif8_selftest_host_caches(int* failed_check)
+{
+    int check = 0;
+    auto fail = [&](int c) { if (failed_check) *failed_check = c; return HIF8_ERR_SHAPE; };
+    {   // set-up record: one initialisation per device ordinal, each with its own value
+        static PerDevice<int> rec;
+        static int calls;
+        calls = 0;
+        auto init = [](int dev, int* out) { calls++; *out = 1000 + dev; };
+        const int* a = rec.get(3, init);
+        const int* b = rec.get(5, init);
+        const int* c = rec.get(3, init);
+        check = 1; if (!a || !b || a != c || *a != 1003 || *b != 1005) return fail(check);
+        check = 2; if (calls > 2) return fail(check);   // at most one per ordinal (zero when run before in this process)
+        check = 3; if (rec.get(-1, init) || rec.get(kMaxDevices, init)) return fail(check);
+    }
+    {   // keyed cache: hit after miss, a failed build is not kept, the least recently used entry is replaced
+        struct K { uint64_t a; uint32_t b; uint32_t pad; };
+        LruCache<K, int, 4> cache;
+        int builds = 0;
+        auto make = [&](const K& k, int* v) { builds++; *v = (int)(k.a * 10 + k.b); return k.b != 99; };
+        auto key = [](uint64_t a, uint32_t b) { K k; std::memset(&k, 0, sizeof k); k.a = a; k.b = b; return k; };
+        int v = 0;
+        check = 4; if (!cache.lookup_or_make(key(1, 2), &v, make) || v != 12 || builds != 1) return fail(check);
+        check = 5; if (!cache.lookup_or_make(key(1, 2), &v, make) || v != 12 || builds != 1) return fail(check);
+        check = 6; if (cache.lookup_or_make(key(7, 99), &v, make) || builds != 2) return fail(check);
+        check = 7; if (cache.lookup_or_make(key(7, 99), &v, make) || builds != 3) return fail(check);
+        for (uint64_t a = 2; a <= 4; a++) cache.lookup_or_make(key(a, 0), &v, make);   // cache now holds (1,2), 2, 3, 4
+        check = 8; if (!cache.lookup_or_make(key(1, 2), &v, make) || builds != 6) return fail(check);   // refreshes (1,2)
+        cache.lookup_or_make(key(5, 0), &v, make);                                     // replaces key 2, the oldest
+        check = 9; if (builds != 7 || !cache.lookup_or_make(key(1, 2), &v, make) || builds != 7) return fail(check);
+        check = 10; if (!cache.lookup_or_make(key(2, 0), &v, make) || builds != 8) return fail(check);
+        check = 11; if (cache.hits() != 3 || cache.misses() != 6) return fail(check);
+        int w = 0;
+        cache.put(key(1, 2), 77);
+        check = 12; if (!cache.find(key(1, 2), &w) || w != 77 || cache.find(key(42, 0), &w)) return fail(check);
+    }
+    if (failed_check) *failed_check = 0;
+    return HIF8_OK;
+}
+
 extern "C" int hif8_selftest_wait_timeout(void* workspace, unsigned limit_ms, hif8_stream_t stream)
 {
     if (!workspace) return HIF8_ERR_NULL;
     if (limit_ms == 0 || limit_ms > 1000) return HIF8_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMemsetAsync(workspace, 0, 4, st) != cudaSuccess) return HIF8_ERR_CUDA;
+    note_status_word(st, reinterpret_cast<const int*>(workspace));
     wait_selftest_kernel<<<1, 32, 0, st>>>(reinterpret_cast<int*>(workspace), (unsigned long long)limit_ms * 1000000ull);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;

@@ -36,6 +36,18 @@ int launch_bf16_pair_gemm(const void* a_bf, const void* w_bf, int w_is_nk, GemmP
 // pointers 16-byte aligned
 int decode_transpose_bf16(const uint8_t* src, void* dst, long long rows, long long cols, cudaStream_t st);
 
+// Remembers `word` (a device int that a kernel sets when one of its bounded waits gives up) as the status word of the
+// latest GEMM-class call on stream `st` of the current device; hif8_last_device_status reads it back.
+void note_status_word(cudaStream_t st, const int* word);
+
+// True when the byte ranges [a, a + a_bytes) and [b, b + b_bytes) share at least one byte (empty ranges share none).
+inline bool ranges_overlap(const void* a, size_t a_bytes, const void* b, size_t b_bytes)
+{
+    const uintptr_t pa = reinterpret_cast<uintptr_t>(a), pb = reinterpret_cast<uintptr_t>(b);
+    return a_bytes && b_bytes && pa < pb + b_bytes && pb < pa + a_bytes;
+}
+inline size_t dtype_bytes(int dtype) { return dtype == 0 ? 4 : 2; }  // HIF8_F32 : HIF8_BF16 / HIF8_F16
+
 // SM count of the current device; HIF8_ERR_CUDA unless it is a compute-capability-10.0 device
 int checked_device(int* sms);
 

@@ -104,6 +104,7 @@ extern "C" int hif8_pts_search(const void* A, const void* W, int dtype, int w_is
     GemmParams p{};
     p.M = M; p.N = N; p.K = K;
     p.status = &ctl->status;
+    note_status_word((cudaStream_t)stream, &ctl->status);
     p.err_ref = O_ref; p.ld_ref = ldo;
     // "MatMul & Restore" and "Quantization Error" of all n * n pairs in one launch: the tiles of every product form one
     // list that the persistent CTA pairs walk through, so only the very last wave of the whole search is ragged

@@ -267,6 +267,8 @@ extern "C" int hif8_encode_transpose(const void* src, int src_dtype, uint8_t* ds
     if (rows < 0 || cols < 0) return HIF8_ERR_SHAPE;
     if (rows == 0 || cols == 0) return HIF8_OK;
     if (!src || !dst) return HIF8_ERR_NULL;
+    if (ranges_overlap(src, (size_t)rows * (size_t)cols * dtype_bytes(src_dtype), dst, (size_t)rows * (size_t)cols))
+        return HIF8_ERR_OVERLAP;
     int sms; int rc = checked_device(&sms);
     if (rc) return rc;
     const int pv = src_dtype == HIF8_F32 ? 4 : 8;

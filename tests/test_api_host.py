@@ -24,7 +24,7 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_status_strings_and_workspace():
-    for s in range(0, 11):
+    for s in range(0, 12):
         assert H.hif8_status_string(s) not in ("", "unknown status")
     assert H.hif8_status_string(99) == "unknown status"
     assert H.hif8_workspace_bytes(H.WS_AMAX_SCALE_ENCODE, 1 << 20) >= 8
@@ -46,6 +46,32 @@ def test_argument_errors_before_any_launch():
     assert H.hif8_fake_quant(0, 0, H.BF16, 16, use_amax=1, scale_or_target_exp=14, stream=0, check=False) == 8
     assert H.hif8_fake_quant(0, 0, H.BF16, 16, use_amax=0, scale_or_target_exp=200, stream=0, check=False) == 5
     assert H.hif8_launch_count() == before
+
+
+def test_overlapping_source_and_destination_are_rejected_on_the_host():
+    # a conversion reads one tensor and writes another; ranges that share a byte are refused before any launch
+    before = H.hif8_launch_count()
+    base = 1 << 20
+    n = 1000
+    assert H.hif8_encode(base, H.F32, base + 1, n, stream=0, check=False) == 11
+    assert H.hif8_encode(base, H.F32, base + 4 * n - 1, n, stream=0, check=False) == 11      # last source byte
+    assert H.hif8_encode(base + n - 1, H.BF16, base, n, stream=0, check=False) == 11         # destination ends inside
+    assert H.hif8_decode(base, base + n - 1, H.F16, n, stream=0, check=False) == 11
+    assert H.hif8_decode(base + 2 * n - 1, base, H.BF16, n, stream=0, check=False) == 11
+    assert H.hif8_fake_quant(base, base + 2, H.BF16, n, use_amax=0, scale_or_target_exp=3, stream=0, check=False) == 11
+    assert H.hif8_fake_quant(base + 4 * n - 4, base, H.F32, n, use_amax=0, scale_or_target_exp=3, stream=0, check=False) == 11
+    assert H.hif8_amax_scale_encode(base, H.F32, base + 8, n, workspace=4096, workspace_bytes=256, stream=0, check=False) == 11
+    assert H.hif8_amax_scale_encode_static(base, H.F32, base + 8, n, stream=0, check=False) == 11
+    assert H.hif8_encode_from_amax(base, H.F16, base + 2 * n - 1, n, 14, H.RND_TA, 0, 0, 4096, stream=0, check=False) == 11
+    assert H.hif8_encode_transpose(base, H.BF16, base + 100, 10, 100, stream=0, check=False) == 11
+    assert H.hif8_channel_amax_scale_encode(base, H.BF16, base + 100, 10, 100, 0, d_amax=4096, stream=0, check=False) == 11
+    assert H.hif8_launch_count() == before
+    assert H.hif8_status_string(11) == "source and destination share bytes"
+
+
+def test_host_side_caches_selftest():
+    # the per-device set-up record (kernel attributes, SM count) and the tensor-map cache, driven without a device
+    assert H.hif8_selftest_host_caches() == (0, 0)
 
 
 def test_gemm_argument_errors_before_any_launch():

@@ -341,6 +341,55 @@ def test_sr14_error_bound_and_unbiased():
     assert abs(err.mean()) < 4 * 0.5 / np.sqrt(err.size)
 
 
+def test_sr14_hand_worked_bit_level_vectors():
+    # Section 3.2, SR14: one FP32 pattern per mantissa width 3 / 2 / 1 / 0 and below 2^-22, bits written out and the
+    # expected neighbour derived by hand in tests/golden/sr14_hand_vectors.txt.  Each vector is chosen so that a
+    # fraction taken from the wrong end of the discarded field, a width taken from the unscaled binade, a strict
+    # comparison or plain nearest rounding gives a different byte.
+    rows = []
+    for line in open(os.path.join(GOLDEN, "sr14_hand_vectors.txt")):
+        line = line.split("#")[0].split()
+        if line:
+            rows.append((int(line[0], 16), int(line[1]), int(line[2], 16)))
+    assert len(rows) >= 11
+    for bits, se, want in rows:
+        src = np.array([bits], dtype=np.uint32)
+        for quick in (False, True):
+            assert int(O.encode(src, O.F32, se, O.SSR, quick=quick)[0]) == want, hex(bits)
+        # Eq. 3: the hybrid mode is the simplified SR from |E| = 4 on
+        E = int(np.floor(np.log2(abs(float(src.view(np.float32)[0]) * 2.0 ** se))))
+        if abs(E) >= 4:
+            assert int(O.encode(src, O.F32, se, O.HR)[0]) == want, hex(bits)
+    # the vectors do tell the alternatives apart: round half away differs on most of them
+    ta = [int(O.encode(np.array([b], dtype=np.uint32), O.F32, se, O.TA)[0]) for b, se, _ in rows]
+    assert sum(t != w for t, (_, _, w) in zip(ta, rows)) >= 7
+
+
+def test_index_addressed_entries_follow_the_flat_index():
+    # standard SR draws word (i mod 4) of the Philox block i / 4 (pinned by the known-answer test above): an element
+    # handed over together with its flat position gets the same code as inside the whole tensor, also far beyond 2^32
+    x = W.loguniform_f32(4096, seed=21, lo_exp=-24, hi_exp=16)
+    full = O.encode(x, O.F32, rnd=O.SR, seed=9)
+    pick = np.random.default_rng(1).permutation(4096)[:500]
+    assert np.array_equal(O.encode_at(x[pick], O.F32, pick, rnd=O.SR, seed=9), full[pick])
+    fq = O.fake_quant(x, O.F32, 3, O.SR, seed=9)
+    assert np.array_equal(O.fake_quant_at(x[pick], O.F32, pick, 3, O.SR, seed=9), fq[pick])
+    # T = top 24 bits of the word of that index; with F just below / above T / 2^24 the neighbour flips
+    base = np.uint64(1) << np.uint64(40)
+    for k in range(64):
+        i = int(base) + 977 * k
+        T = O.sr_word(9, i) >> 8
+        if T == 0:
+            continue
+        # value 1 + (j / 2^24) / 8 in the binade of 1.0 (ulp 1/8): F * 2^24 = j exactly for j a multiple of 2^4
+        for j, up in ((T - 16) & ~15, False), ((T + 15) & ~15, True):
+            if 0 < j < (1 << 24):
+                v = np.array([1.0 + j / 2.0 ** 27], dtype=np.float32)
+                assert float(v[0]) == 1.0 + j / 2.0 ** 27
+                got = int(O.encode_at(v, O.F32, [i], rnd=O.SR, seed=9)[0])
+                assert got == (0x09 if up else 0x08), (i, j, T)
+
+
 @pytest.mark.parametrize("dtype", [O.F32, O.BF16])
 def test_sr_expectation(dtype):
     # Section 3.2: E[SR] = (K+1) F + K (1-F) = K + F
