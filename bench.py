@@ -4,9 +4,12 @@
 One step = per-tensor scaled encode (amax -> power-of-two scale -> HiF8 bytes, just-in-time form) followed
 by decode back to FP32 of one FP32 4096x4096 N(0,1) tensor (synthetic, seeded).  The metric is algorithmic
 bytes moved per second: 9 B/element for the encode call (4 read for amax, 4 read + 1 written for the
-conversion) plus 5 B/element for the decode call (1 read, 4 written).
+conversion) plus 5 B/element for the decode call (1 read, 4 written).  It is NOT a DRAM bandwidth: the second
+read of the source and the read of the codes can be served by the L2; `config.step_dram` gives the DRAM-based
+figure from profiler counters beside it, and `roofline` describes single kernels.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+  python bench.py --case NAME [--reps R]        one named workload a few times, for use under a profiler
 
 N > 1 is launched under torch.distributed.run, one rank per GPU; ranks convert independent tensors (no
 data-path collective, weak scaling) and rank 0 prints the single JSON line.
@@ -33,11 +36,15 @@ BYTES_DECODE = 5 * N_EL
 BYTES_STEP = BYTES_ENCODE + BYTES_DECODE
 POOL = 6                  # rotating buffer sets: 6 x 64 MiB of input alone exceeds the 126 MB L2
 WORKLOAD = "fp32_4096x4096_normal_amax_scale_encode_then_decode"
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture summarised in profiles/;
-# None for a kernel changed since its capture
-TRAFFIC = {"amax_kernel<f32>": 67.57e6, "convert_kernel<f32,TA>": 69.53e6, "decode_kernel<f32>": 26.10e6}
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from profiler captures of these kernels on this
+# workload.  "cold": every launch alone with the caches flushed in front of it.  "in_step": the same launches inside the
+# running amax -> convert -> decode sequence with the caches left as the previous kernel left them.  None: the kernel
+# has changed since its capture.
+TRAFFIC_COLD = {"amax_kernel<f32>": 67.57e6, "convert_kernel<f32,TA>": 69.53e6, "decode_kernel<f32>": 26.10e6}
+TRAFFIC_IN_STEP = {"amax_kernel<f32>": None, "convert_kernel<f32,TA>": None, "decode_kernel<f32>": None}
 METRIC = "hif8_encode_decode_throughput"
 UNIT = "GB/s"
+MIN_REPEATS = 7
 
 
 def env_int(name, default):
@@ -116,16 +123,32 @@ def job_throughput(world, bytes_per_rank_step, ms_per_step):
     return world * bytes_per_rank_step / (ms_per_step * 1e-3) / 1e9
 
 
+def spread(samples_ms):
+    """median / best / worst of a list of per-unit times (ms)."""
+    s = sorted(float(v) for v in samples_ms)
+    return {"ms": s[len(s) // 2] if len(s) % 2 else 0.5 * (s[len(s) // 2 - 1] + s[len(s) // 2]), "best_ms": s[0],
+            "worst_ms": s[-1], "repeats": len(s)}
+
+
+def repeats_for(region_ms):
+    """How often a timed region is repeated: at least MIN_REPEATS, more for short regions (about half a second of
+    device time in all, so that the clock sampler sees the run), never more than 200."""
+    return int(min(200, max(MIN_REPEATS, 500.0 / max(region_ms, 1e-3))))
+
+
 def load_peaks():
+    """(HBM GB/s, BF16 burst TFLOP/s, BF16 sustained TFLOP/s, kind)"""
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         p = json.load(open(path))
-        return float(p["hbm_gbs"]), "measured"
-    return 6650.0, "fallback"
+        return float(p["hbm_gbs"]), float(p["bf16_tflops"]), float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "measured"
+    return 6650.0, 1590.0, 1400.0, "fallback"
 
 
-def cpu_baseline(sample_elems):
-    """The oracle as it stands (brute-force nearest-of-256 encode), on a leading slice of the same tensor."""
+# --------------------------------------------------------------------------------------------------------------
+# CPU baseline: the oracle as it stands, on bounded samples of the workloads
+# --------------------------------------------------------------------------------------------------------------
+def cpu_baseline(sample_elems, legs=True):
     from oracle import hif8_oracle as O
     x = W.normal_f32((ROWS, COLS), seed=1234).reshape(-1)[:sample_elems]
     t0 = time.perf_counter()
@@ -133,32 +156,82 @@ def cpu_baseline(sample_elems):
     codes = O.encode(x, O.F32, se, O.TA, 0, quick=False)
     O.decode(codes, O.F32, se)
     dt = time.perf_counter() - t0
-    return {"value": 14 * sample_elems / dt / 1e9, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
-            "sample": f"first {sample_elems} of {N_EL} elements: amax + brute-force TA encode + decode, {dt:.2f} s",
-            "elements_per_s": sample_elems / dt}
+    out = {"value": 14 * sample_elems / dt / 1e9, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
+           "sample": f"first {sample_elems} of {N_EL} elements: amax + brute-force TA encode + decode, {dt:.2f} s",
+           "elements_per_s": sample_elems / dt}
+    if not legs:
+        return out
+    by = {}
+    # LLM-activation fake-quant (BF16, Student-t body with outlier channels), fused amax, round half away
+    xb = W.llm_activation_bf16(2048, 8192, seed=2345).reshape(-1)
+    t0 = time.perf_counter()
+    _, se = O.amax_scale(xb, O.BF16, 14)
+    O.fake_quant(xb, O.BF16, se, O.TA, 0, quick=False)
+    dt = time.perf_counter() - t0
+    by["bf16_activation_fake_quant_TA"] = {"elements_per_s": xb.size / dt, "GBps": 6 * xb.size / dt / 1e9, "kind": "oracle (scan of 256 codes)",
+                                           "sample": f"{xb.size} of {8192 * 8192} elements, {dt:.2f} s"}
+    t0 = time.perf_counter()
+    O.fake_quant(xb, O.BF16, se, O.HR, 0, quick=False)
+    dt = time.perf_counter() - t0
+    by["bf16_activation_fake_quant_HR"] = {"elements_per_s": xb.size / dt, "GBps": 4 * xb.size / dt / 1e9, "kind": "oracle (scale given)",
+                                           "sample": f"{xb.size} of {8192 * 8192} elements, {dt:.2f} s"}
+    # gradient-range FP32 encode: the neighbour-pair variant, which is the one the 2^32 sweep is checked with
+    g = W.loguniform_f32(1 << 24, seed=3456)
+    t0 = time.perf_counter()
+    O.encode(g, O.F32, 0, O.TA, 0, quick=True)
+    dt = time.perf_counter() - t0
+    by["loguniform_f32_encode_TA"] = {"elements_per_s": g.size / dt, "GBps": 5 * g.size / dt / 1e9,
+                                      "kind": "oracle, neighbour-pair (quick) variant", "sample": f"2^24 of 2^28 elements, {dt:.2f} s"}
+    # GEMM: FP64 oracle on a 128 x 128 block of outputs at K = 8192
+    Aq, Wq = W.random_codes((128, 8192), seed=4567), W.random_codes((8192, 128), seed=5678)
+    t0 = time.perf_counter()
+    O.gemm_full(Aq, Wq, False, 0, 0)
+    dt = time.perf_counter() - t0
+    by["gemm_fp64"] = {"TFLOPs": 2.0 * 128 * 128 * 8192 / dt / 1e12, "kind": "oracle (FP64, sum and sum of magnitudes), extrapolated",
+                       "sample": f"128 x 128 outputs of 8192 x 28672 at K = 8192, {dt:.2f} s"}
+    out["by_config"] = by
+    return out
 
 
-def extra_results(H, torch, hbm_peak, peak_kind):
+# --------------------------------------------------------------------------------------------------------------
+# Secondary workloads
+# --------------------------------------------------------------------------------------------------------------
+def extra_results(H, torch, hbm_peak, tf_peak, peak_kind):
     """Secondary workloads (each with its own roofline fraction): BF16 fake-quant of an LLM-activation tensor,
     gradient-range FP32 encode/decode, and the HiF8-operand GEMM.  Inputs are generated on the device from a
-    seeded torch generator with the same recipes as workloads/ (shapes and distributions, not the same bytes)."""
-    out = {}
+    seeded torch generator with the same recipes as workloads/ (shapes and distributions, not the same bytes).
+    Returns (detail, by_config): by_config is the compact table of the headline figure of every configuration."""
+    out, table = {}, {}
     g = torch.Generator(device="cuda")
     g.manual_seed(2345)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     wsb = H.hif8_workspace_bytes(H.WS_FAKE_QUANT, 0)
     ws = torch.empty(max(wsb, 256), dtype=torch.uint8, device="cuda")
 
-    def timed(fn, reps):
+    def timed(fn, reps, repeats=MIN_REPEATS):
+        """`repeats` timed regions of `reps` calls each; median / best / worst per call."""
         for _ in range(3):
             fn(0)
         torch.cuda.synchronize()
-        ev0.record()
-        for r in range(reps):
-            fn(r)
-        ev1.record()
-        torch.cuda.synchronize()
-        return ev0.elapsed_time(ev1) / reps
+        per_call = []
+        for _ in range(repeats):
+            ev0.record()
+            for r in range(reps):
+                fn(r)
+            ev1.record()
+            torch.cuda.synchronize()
+            per_call.append(ev0.elapsed_time(ev1) / reps)
+        return spread(per_call)
+
+    def hbm(stat, nbytes, **more):
+        d = dict(stat, GBps=nbytes / stat["ms"] / 1e6, frac=nbytes / stat["ms"] / 1e6 / hbm_peak, **more)
+        return d
+
+    def tensor(stat, flops, **more):
+        return dict(stat, TFLOPs=flops / stat["ms"] / 1e9, frac=flops / stat["ms"] / 1e9 / tf_peak, **more)
+
+    def row(name, d, bound):
+        table[name] = {"ms": round(d["ms"], 5), "best_ms": round(d["best_ms"], 5), "frac": round(d["frac"], 4), "bound": bound}
 
     # ---- small and odd sizes (launch latency, tails): FP32 encode TA + decode, 20 call pairs per graph replay
     small = {}
@@ -172,8 +245,10 @@ def extra_results(H, torch, hbm_peak, peak_kind):
             for _ in range(20):
                 H.hif8_encode(xs_, H.F32, cq, n, 10, H.RND_TA, stream=cs)
                 H.hif8_decode(cq, bk, H.F32, n, 10, stream=cs)
-        ms = timed(lambda r: gr.replay(), 5) / 20
-        small[str(n)] = {"us_per_encode_decode_pair": ms * 1e3, "GBps": 10 * n / ms / 1e6, "frac": 10 * n / ms / 1e6 / hbm_peak}
+        st = timed(lambda r: gr.replay(), 5)
+        ms = st["ms"] / 20
+        small[str(n)] = {"us_per_encode_decode_pair": ms * 1e3, "best_us": st["best_ms"] / 20 * 1e3, "GBps": 10 * n / ms / 1e6,
+                         "frac": 10 * n / ms / 1e6 / hbm_peak}
         del xs_, cq, bk, gr
     out["small_and_odd_sizes_f32"] = {"bytes_per_element": 10, "sizes": small, "peak": hbm_peak, "peak_kind": f"of {peak_kind}",
                                       "note": "tensors up to 45 M elements fit in L2 between the two calls; a pair is two launches"}
@@ -195,16 +270,19 @@ def extra_results(H, torch, hbm_peak, peak_kind):
     ys = [torch.empty_like(x) for x in xs]
     fq = {}
     for name, mode in (("TA", H.RND_TA), ("HR", H.RND_HR), ("SSR", H.RND_SSR), ("TE", H.RND_TE), ("SR", H.RND_SR)):
-        ms = timed(lambda r: H.hif8_fake_quant(xs[r & 1], ys[r & 1], H.BF16, n, 1, 14, mode, 0, 7, None, None, ws, wsb), 20)
-        fq[name] = {"ms": ms, "GBps": 6 * n / ms / 1e6, "frac": 6 * n / ms / 1e6 / hbm_peak}
-    ms = timed(lambda r: H.hif8_fake_quant(xs[r & 1], ys[r & 1], H.BF16, n, 0, 3, H.RND_TA, 0, 0), 20)
-    fq["TA_given_scale"] = {"ms": ms, "GBps": 4 * n / ms / 1e6, "frac": 4 * n / ms / 1e6 / hbm_peak}
+        st = timed(lambda r: H.hif8_fake_quant(xs[r & 1], ys[r & 1], H.BF16, n, 1, 14, mode, 0, 7, None, None, ws, wsb), 20)
+        fq[name] = hbm(st, 6 * n)
+        row(f"C3_fake_quant_bf16_8192x8192_{name}", fq[name], "hbm")
+    st = timed(lambda r: H.hif8_fake_quant(xs[r & 1], ys[r & 1], H.BF16, n, 0, 3, H.RND_TA, 0, 0), 20)
+    fq["TA_given_scale"] = hbm(st, 4 * n)
+    row("C3_fake_quant_bf16_8192x8192_TA_given_scale", fq["TA_given_scale"], "hbm")
     # the same tensors to HiF8 bytes with a given scale (2 B read + 1 B written): forward (TA) and backward (HR) rounding
     cq = torch.empty(n, dtype=torch.uint8, device="cuda")
     enc = {}
     for name, mode in (("TA", H.RND_TA), ("HR", H.RND_HR)):
-        ms = timed(lambda r: H.hif8_encode(xs[r & 1], H.BF16, cq, n, 3, mode), 20)
-        enc[name] = {"ms": ms, "GBps": 3 * n / ms / 1e6, "frac": 3 * n / ms / 1e6 / hbm_peak}
+        st = timed(lambda r: H.hif8_encode(xs[r & 1], H.BF16, cq, n, 3, mode), 20)
+        enc[name] = hbm(st, 3 * n)
+        row(f"C3_encode_bf16_8192x8192_{name}", enc[name], "hbm")
     out["encode_bf16_8192x8192"] = {"bytes_per_element": 3, "modes": enc, "peak": hbm_peak, "peak_kind": f"of {peak_kind}"}
     del cq
     out["fake_quant_bf16_8192x8192"] = {"bytes_per_element": {"fused_amax": 6, "given_scale": 4}, "modes": fq,
@@ -222,10 +300,12 @@ def extra_results(H, torch, hbm_peak, peak_kind):
     back = torch.empty(n, dtype=torch.float32, device="cuda")
     res = {}
     for name, mode in (("encode_TA", H.RND_TA), ("encode_HR", H.RND_HR)):
-        ms = timed(lambda r: H.hif8_encode(bits, H.F32, codes, n, 0, mode), 10)
-        res[name] = {"ms": ms, "GBps": 5 * n / ms / 1e6, "frac": 5 * n / ms / 1e6 / hbm_peak}
-    ms = timed(lambda r: H.hif8_decode(codes, back, H.F32, n, 0), 10)
-    res["decode"] = {"ms": ms, "GBps": 5 * n / ms / 1e6, "frac": 5 * n / ms / 1e6 / hbm_peak}
+        st = timed(lambda r: H.hif8_encode(bits, H.F32, codes, n, 0, mode), 10)
+        res[name] = hbm(st, 5 * n)
+        row(f"C4a_loguniform_f32_2^28_{name}", res[name], "hbm")
+    st = timed(lambda r: H.hif8_decode(codes, back, H.F32, n, 0), 10)
+    res["decode"] = hbm(st, 5 * n)
+    row("C4a_loguniform_f32_2^28_decode", res["decode"], "hbm")
     out["loguniform_f32_2^28"] = {"bytes_per_element": 5, "calls": res, "peak": hbm_peak, "peak_kind": f"of {peak_kind}"}
     del bits, codes, back
 
@@ -245,32 +325,32 @@ def extra_results(H, torch, hbm_peak, peak_kind):
     ch_amax2 = torch.empty(2 * N, dtype=torch.float32, device="cuda")
     ch_se2 = torch.empty(2 * N, dtype=torch.int32, device="cuda")
     chan = {}
-    ms = timed(lambda r: H.hif8_channel_amax_scale_encode(w, H.BF16, Wq, K, N, 1, 14, H.RND_TA, 0, 0, None, ch_amax, ch_se), 10)
-    chan["columns_[K,N]"] = {"ms": ms, "bytes_per_element": 5, "GBps": 5 * K * N / ms / 1e6, "frac": 5 * K * N / ms / 1e6 / hbm_peak,
-                             "note": "amax kernel (2 B) + encode kernel (2 + 1 B)"}
-    ms = timed(lambda r: H.hif8_channel_amax_scale_encode(w, H.BF16, Wq, N, K, 0, 14, H.RND_TA, 0, 0, None, ch_amax, ch_se), 10)
-    chan["rows_[N,K]"] = {"ms": ms, "bytes_per_element": 3, "GBps": 3 * K * N / ms / 1e6, "frac": 3 * K * N / ms / 1e6 / hbm_peak,
-                          "note": "one kernel, a block per row; the second read of the row hits L1/L2"}
-    ms = timed(lambda r: H.hif8_channel_amax_scale_encode(w, H.BF16, Wq, 2 * N, K // 2, 0, 14, H.RND_TA, 0, 0, None, ch_amax2, ch_se2), 10)
-    chan["rows_[2N,K/2]"] = {"ms": ms, "bytes_per_element": 3, "GBps": 3 * K * N / ms / 1e6, "frac": 3 * K * N / ms / 1e6 / hbm_peak,
-                             "note": "rows of 4096: two rows per block"}
-    ms = timed(lambda r: H.hif8_channel_amax_scale_encode(w, H.BF16, Wq, N // 2, 2 * K, 0, 14, H.RND_TA, 0, 0, None, ch_amax2, ch_se2), 10)
-    chan["rows_[N/2,2K]"] = {"ms": ms, "bytes_per_element": 3, "GBps": 3 * K * N / ms / 1e6, "frac": 3 * K * N / ms / 1e6 / hbm_peak,
-                             "note": "rows of 16384: held in registers, read once"}
-    ms = timed(lambda r: H.hif8_channel_amax_scale_encode(w, H.BF16, Wq, K, N, 1, 14, H.RND_TA, 0, 0, ch_se, None, None), 10)
-    chan["columns_given_exponents"] = {"ms": ms, "bytes_per_element": 3, "GBps": 3 * K * N / ms / 1e6,
-                                       "frac": 3 * K * N / ms / 1e6 / hbm_peak}
+    st = timed(lambda r: H.hif8_channel_amax_scale_encode(w, H.BF16, Wq, K, N, 1, 14, H.RND_TA, 0, 0, None, ch_amax, ch_se), 10)
+    chan["columns_[K,N]"] = hbm(st, 5 * K * N, bytes_per_element=5, note="amax kernel (2 B) + encode kernel (2 + 1 B)")
+    st = timed(lambda r: H.hif8_channel_amax_scale_encode(w, H.BF16, Wq, N, K, 0, 14, H.RND_TA, 0, 0, None, ch_amax, ch_se), 10)
+    chan["rows_[N,K]"] = hbm(st, 3 * K * N, bytes_per_element=3, note="one kernel, a block per row; the second read of the row hits L1/L2")
+    st = timed(lambda r: H.hif8_channel_amax_scale_encode(w, H.BF16, Wq, 2 * N, K // 2, 0, 14, H.RND_TA, 0, 0, None, ch_amax2, ch_se2), 10)
+    chan["rows_[2N,K/2]"] = hbm(st, 3 * K * N, bytes_per_element=3, note="rows of 4096: two rows per block")
+    st = timed(lambda r: H.hif8_channel_amax_scale_encode(w, H.BF16, Wq, N // 2, 2 * K, 0, 14, H.RND_TA, 0, 0, None, ch_amax2, ch_se2), 10)
+    chan["rows_[N/2,2K]"] = hbm(st, 3 * K * N, bytes_per_element=3, note="rows of 16384: held in registers, read once")
+    st = timed(lambda r: H.hif8_channel_amax_scale_encode(w, H.BF16, Wq, K, N, 1, 14, H.RND_TA, 0, 0, ch_se, None, None), 10)
+    chan["columns_given_exponents"] = hbm(st, 3 * K * N, bytes_per_element=3)
+    for k_, v_ in chan.items():
+        row(f"channel_encode_bf16_8192x28672_{k_}", v_, "hbm")
     out["channel_scaled_encode_bf16_8192x28672"] = {"calls": chan, "peak": hbm_peak, "peak_kind": f"of {peak_kind}"}
     state = torch.empty(H.SCALE_STATE_BYTES, dtype=torch.uint8, device="cuda")
     H.hif8_scale_state_init(state, 4)
     dl = {}
     for name, measure in (("measuring_iteration", 1), ("plain_iteration", 0)):
-        ms = timed(lambda r: H.hif8_delayed_scale_encode(a, H.BF16, Aq, M * K, H.RND_TA, 0, 0, state, measure, 14), 20)
-        dl[name] = {"ms": ms, "GBps": 3 * M * K / ms / 1e6, "frac": 3 * M * K / ms / 1e6 / hbm_peak}
-    ms = timed(lambda r: H.hif8_encode_transpose(a, H.BF16, Aq, M, K, 3, None, H.RND_HR), 20)
-    out["encode_transpose_bf16_8192x8192_HR"] = {"ms": ms, "bytes_per_element": 3, "GBps": 3 * M * K / ms / 1e6,
-                                                 "frac": 3 * M * K / ms / 1e6 / hbm_peak, "peak": hbm_peak,
-                                                 "peak_kind": f"of {peak_kind}"}
+        st = timed(lambda r: H.hif8_delayed_scale_encode(a, H.BF16, Aq, M * K, H.RND_TA, 0, 0, state, measure, 14), 20)
+        dl[name] = hbm(st, 3 * M * K)
+        row(f"delayed_scale_encode_bf16_8192x8192_{name}", dl[name], "hbm")
+    tr = {}
+    for name, mode in (("TA", H.RND_TA), ("HR", H.RND_HR)):
+        st = timed(lambda r: H.hif8_encode_transpose(a, H.BF16, Aq, M, K, 3, None, mode), 20)
+        tr[name] = hbm(st, 3 * M * K)
+        row(f"encode_transpose_bf16_8192x8192_{name}", tr[name], "hbm")
+    out["encode_transpose_bf16_8192x8192"] = {"bytes_per_element": 3, "modes": tr, "peak": hbm_peak, "peak_kind": f"of {peak_kind}"}
     out["delayed_scale_encode_bf16_8192x8192"] = {"bytes_per_element": 3, "calls": dl, "peak": hbm_peak,
                                                   "peak_kind": f"of {peak_kind}"}
     H.hif8_amax_scale_encode(a, H.BF16, Aq, M * K, 14, H.RND_TA, 0, 0, None, None, se[0:1], None, ws, wsb)
@@ -279,50 +359,49 @@ def extra_results(H, torch, hbm_peak, peak_kind):
     C = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
     gws_b = H.hif8_workspace_bytes(H.WS_GEMM, M * K + K * N)
     gws = torch.empty(gws_b, dtype=torch.uint8, device="cuda")
-    tf_peak, tf_kind = 1590.0, "fallback"
-    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    if os.path.exists(path):
-        tf_peak, tf_kind = float(json.load(open(path))["bf16_tflops"]), "measured"
     flops = 2.0 * M * N * K
-    ms = timed(lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, C, N, H.BF16, M, N, K, se[0:1], se[1:2], gws, gws_b), 10)
-    st1 = H.hif8_gemm_status(gws)
-    ms_f = timed(lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, C, N, H.BF16, M, N, K, se[0:1], se[1:2], gws, 256), 3)
-    st2 = H.hif8_gemm_status(gws)
+    g_once = tensor(timed(lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, C, N, H.BF16, M, N, K, se[0:1], se[1:2], gws, gws_b), 5),
+                    flops, device_status=H.hif8_last_device_status(),
+                    note="whole call: decode of both operands to BF16 workspace + tcgen05 kernel")
+    g_fused = tensor(timed(lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, C, N, H.BF16, M, N, K, se[0:1], se[1:2], gws, 256), 3),
+                     flops, device_status=H.hif8_last_device_status(),
+                     note="no workspace: byte tiles decoded per CTA pair inside the tensor-core kernel")
     ch_se.fill_(int(se[1]))
-    ms_c = timed(lambda r: H.hif8_gemm_channel_scaled(Aq, K, Wq, N, 0, C, N, H.BF16, M, N, K, se[0:1], ch_se, gws, gws_b), 10)
-    st3 = H.hif8_gemm_status(gws)
+    g_chan = tensor(timed(lambda r: H.hif8_gemm_channel_scaled(Aq, K, Wq, N, 0, C, N, H.BF16, M, N, K, se[0:1], ch_se, gws, gws_b), 5),
+                    flops, device_status=H.hif8_last_device_status(), note="one weight exponent per output column")
+    row("C5_gemm_8192x28672x8192_decode_once", g_once, "tensor")
+    row("C5_gemm_8192x28672x8192_fused", g_fused, "tensor")
+    row("gemm_8192x28672x8192_channel_scaled", g_chan, "tensor")
     # backward-pass forms of the same size: dgrad reads the weight as [N,K], wgrad reads A as [K,M] and accumulates in FP32
     bw = {}
-    ms_d = timed(lambda r: H.hif8_gemm_ex(Aq, K, 0, Wq, K, 1, C, N, H.BF16, M, N, K, se[0:1], se[1:2], None, 0, gws, gws_b), 10)
-    bw["dgrad_form_w_as_[N,K]"] = {"ms": ms_d, "TFLOPs": flops / ms_d / 1e9, "frac": flops / ms_d / 1e9 / tf_peak,
-                                   "device_status": H.hif8_gemm_status(gws)}
+    bw["dgrad_form_w_as_[N,K]"] = tensor(
+        timed(lambda r: H.hif8_gemm_ex(Aq, K, 0, Wq, K, 1, C, N, H.BF16, M, N, K, se[0:1], se[1:2], None, 0, gws, gws_b), 5),
+        flops, device_status=H.hif8_last_device_status())
     C32 = torch.zeros(M, N, dtype=torch.float32, device="cuda")
-    ms_w = timed(lambda r: H.hif8_gemm_ex(Aq, M, 1, Wq, N, 0, C32, N, H.F32, M, N, K, se[0:1], se[1:2], None, 1, gws, gws_b), 10)
-    bw["wgrad_form_a_as_[K,M]_fp32_accumulate"] = {"ms": ms_w, "TFLOPs": flops / ms_w / 1e9, "frac": flops / ms_w / 1e9 / tf_peak,
-                                                   "device_status": H.hif8_gemm_status(gws)}
+    bw["wgrad_form_a_as_[K,M]_fp32_accumulate"] = tensor(
+        timed(lambda r: H.hif8_gemm_ex(Aq, M, 1, Wq, N, 0, C32, N, H.F32, M, N, K, se[0:1], se[1:2], None, 1, gws, gws_b), 5),
+        flops, device_status=H.hif8_last_device_status())
     del C32
+    for k_, v_ in bw.items():
+        row(f"gemm_8192x28672x8192_{k_}", v_, "tensor")
     # inference-decode shapes: a few activation rows against the same weight (bound by reading the weight bytes once)
     narrow = {}
     for Mn in (16, 64):
         Cn = torch.empty(Mn, N, dtype=torch.bfloat16, device="cuda")
         # with the workspace: equal (slab, k-block) ranges per SM; with the 256-byte minimum: one CTA per slab
-        ms_n = timed(lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, Cn, N, H.BF16, Mn, N, K, se[0:1], se[1:2], gws, gws_b), 20)
-        ms_s = timed(lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, Cn, N, H.BF16, Mn, N, K, se[0:1], se[1:2], gws, 256), 20)
         byt = K * N + Mn * K + 2 * Mn * N
-        narrow[f"M={Mn}"] = {"us": ms_n * 1e3, "GBps": byt / ms_n / 1e6, "frac_of_hbm": byt / ms_n / 1e6 / hbm_peak,
-                             "us_one_cta_per_slab": ms_s * 1e3, "device_status": H.hif8_gemm_status(gws)}
+        st = timed(lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, Cn, N, H.BF16, Mn, N, K, se[0:1], se[1:2], gws, gws_b), 20)
+        st_s = timed(lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, Cn, N, H.BF16, Mn, N, K, se[0:1], se[1:2], gws, 256), 20)
+        d = hbm(st, byt, us=st["ms"] * 1e3, us_one_cta_per_slab=st_s["ms"] * 1e3, device_status=H.hif8_last_device_status())
+        d["frac_of_hbm"] = d["frac"]
+        narrow[f"M={Mn}"] = d
+        row(f"gemm_narrow_{Mn}x28672x8192", d, "hbm (weight bytes)")
         del Cn
     out["gemm_narrow_Mx28672x8192"] = {"bound": "hbm", "bytes": "K*N weight bytes + M*K + 2*M*N", "shapes": narrow,
                                        "peak": hbm_peak, "peak_kind": f"of {peak_kind}"}
     out["gemm_8192x28672x8192"] = {
-        "backward_forms": bw,
-        "decode_once_channel_scaled": {"ms": ms_c, "TFLOPs": flops / ms_c / 1e9, "frac": flops / ms_c / 1e9 / tf_peak,
-                                       "device_status": st3, "note": "one weight exponent per output column"},
-        "decode_once": {"ms": ms, "TFLOPs": flops / ms / 1e9, "frac": flops / ms / 1e9 / tf_peak, "device_status": st1,
-                        "note": "whole call: decode of both operands to BF16 workspace + tcgen05 kernel"},
-        "fused": {"ms": ms_f, "TFLOPs": flops / ms_f / 1e9, "frac": flops / ms_f / 1e9 / tf_peak, "device_status": st2,
-                  "note": "no workspace: byte tiles decoded per CTA in shared memory"},
-        "bound": "tensor", "peak": tf_peak, "peak_kind": f"of {tf_kind} (cuBLAS BF16 burst)", "unit": "TFLOP/s",
+        "backward_forms": bw, "decode_once_channel_scaled": g_chan, "decode_once": g_once, "fused": g_fused,
+        "bound": "tensor", "peak": tf_peak, "peak_kind": f"of {peak_kind} (cuBLAS BF16 burst)", "unit": "TFLOP/s",
         "scale_exps": [int(v) for v in se.cpu()], "output": "bf16"}
     del C, gws, Aq, Wq
 
@@ -335,13 +414,124 @@ def extra_results(H, torch, hbm_peak, peak_kind):
     pws = torch.empty(pb, dtype=torch.uint8, device="cuda")
     d_err = torch.zeros(100, dtype=torch.float32, device="cuda")
     d_best = torch.zeros(2, dtype=torch.int32, device="cuda")
-    ms = timed(lambda r: H.hif8_pts_search(a, w, H.BF16, 0, o_ref, N, M, N, K, -4, 5, d_err, d_best, pws, pb), 3)
-    out["pts_search_4096^3"] = {"ms": ms, "TFLOPs_of_100_gemms": 100 * 2.0 * M * N * K / ms / 1e9,
-                                "best_exponents": [int(v) for v in d_best.cpu()], "device_status": H.hif8_pts_status(pws),
-                                "min_mse": float(d_err.min().item())}
-    return out
+    st = timed(lambda r: H.hif8_pts_search(a, w, H.BF16, 0, o_ref, N, M, N, K, -4, 5, d_err, d_best, pws, pb), 2, repeats=3)
+    pts = tensor(st, 100 * 2.0 * M * N * K, best_exponents=[int(v) for v in d_best.cpu()], device_status=H.hif8_pts_status(pws),
+                 min_mse=float(d_err.min().item()))
+    pts["TFLOPs_of_100_gemms"] = pts["TFLOPs"]
+    out["pts_search_4096^3"] = pts
+    row("algorithm1_search_4096^3_10x10", pts, "tensor")
+    return out, table
 
 
+# --------------------------------------------------------------------------------------------------------------
+# Named workloads for a profiler (a few launches each; nothing is timed or printed but a completion line)
+# --------------------------------------------------------------------------------------------------------------
+CASES = ("convert_f32", "fq_bf16", "encode_modes_f32", "encode_modes_bf16", "transpose_bf16", "gemm", "gemm_fused", "gemm_narrow",
+         "gemm_forms", "channel_bf16")
+
+
+def run_case(case, reps):
+    """convert_f32: FP32 4096^2 per-tensor scaled encode + decode over three rotating tensors (the bench step);
+    fq_bf16: BF16 4096x8192 fake-quant, TA / HR / TE, fused amax and given scale; encode_modes_f32 / encode_modes_bf16:
+    2^25 log-uniform values in every rounding mode; transpose_bf16: BF16 8192^2 flat and transposed-store encode, TA and
+    HR; gemm: HiF8 GEMM 4096 x 7168 x 4096 on the decode-once and the fused path (gemm_fused: the fused path only);
+    gemm_forms: the four operand layouts on the decode-once path; gemm_narrow: 16 x 8192 x 8192 with weights as [K,N] and
+    [N,K]; channel_bf16: per-channel scaled encode of a BF16 8192 x 14336 weight by column and by row, plus the overflow
+    check.  Inputs are seeded device-side random tensors."""
+    import torch
+    import paper_2409_16626_b200 as H
+    g = torch.Generator(device="cuda")
+    g.manual_seed(1)
+    ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+    if case == "convert_f32":
+        n = N_EL
+        xs = [torch.randn(n, generator=g, device="cuda") for _ in range(3)]
+        codes = torch.empty(n, dtype=torch.uint8, device="cuda")
+        back = torch.empty(n, dtype=torch.float32, device="cuda")
+        se = torch.zeros(1, dtype=torch.int32, device="cuda")
+        for r in range(reps):
+            H.hif8_amax_scale_encode(xs[r % 3], H.F32, codes, n, 14, H.RND_TA, 0, 0, None, None, se, None, ws, 256)
+            H.hif8_decode(codes, back, H.F32, n, 12)
+    elif case == "fq_bf16":
+        n = 4096 * 8192
+        xs = [torch.randn(n, generator=g, device="cuda").to(torch.bfloat16) for _ in range(3)]
+        y = torch.empty_like(xs[0])
+        for r in range(reps):
+            for mode in (H.RND_TA, H.RND_HR, H.RND_TE):
+                H.hif8_fake_quant(xs[r % 3], y, H.BF16, n, 1, 14, mode, 0, 7, None, None, ws, 256)
+                H.hif8_fake_quant(xs[r % 3], y, H.BF16, n, 0, 12, mode, 0, 7)
+    elif case in ("encode_modes_f32", "encode_modes_bf16"):
+        n = 1 << 25
+        f32 = case == "encode_modes_f32"
+        e = torch.randint(-40, 20, (n,), generator=g, device="cuda", dtype=torch.int32) + 127
+        m = torch.randint(0, 1 << (23 if f32 else 7), (n,), generator=g, device="cuda", dtype=torch.int32)
+        bits = (e << 23) | m if f32 else ((e << 7) | m).to(torch.int16)
+        codes = torch.empty(n, dtype=torch.uint8, device="cuda")
+        for r in range(reps):
+            for mode in (H.RND_TA, H.RND_HR, H.RND_SSR, H.RND_TE, H.RND_SR):
+                H.hif8_encode(bits, H.F32 if f32 else H.BF16, codes, n, 0, mode, 0, 5)
+    elif case == "transpose_bf16":
+        R, Cc = 8192, 8192
+        xs = [torch.randn(R * Cc, generator=g, device="cuda").to(torch.bfloat16) for _ in range(2)]
+        codes = torch.empty(R * Cc, dtype=torch.uint8, device="cuda")
+        for r in range(reps):
+            for mode in (H.RND_TA, H.RND_HR):
+                H.hif8_encode(xs[r & 1], H.BF16, codes, R * Cc, 3, mode, 0, 5)
+                H.hif8_encode_transpose(xs[r & 1], H.BF16, codes, R, Cc, 3, None, mode)
+    elif case in ("gemm", "gemm_fused"):
+        M, N, K = 4096, 7168, 4096
+        A = torch.randint(0, 256, (M, K), dtype=torch.uint8, device="cuda", generator=g)
+        Wt = torch.randint(0, 256, (K, N), dtype=torch.uint8, device="cuda", generator=g)
+        for t in (A, Wt):                                  # keep the operands finite
+            t[(t == 0x80) | ((t & 0x7F) == 0x6F)] = 0x08
+        C = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
+        big = H.hif8_workspace_bytes(H.WS_GEMM, M * K + K * N)
+        gws = torch.empty(big, dtype=torch.uint8, device="cuda")
+        for r in range(reps):
+            if case == "gemm":
+                H.hif8_gemm(A, K, Wt, N, 0, C, N, H.BF16, M, N, K, None, None, gws, big)
+            H.hif8_gemm(A, K, Wt, N, 0, C, N, H.BF16, M, N, K, None, None, gws, 256)
+    elif case == "gemm_narrow":
+        M, N, K = 16, 8192, 8192
+        A = torch.randint(8, 100, (M * K,), dtype=torch.uint8, device="cuda", generator=g)
+        Wt = torch.randint(8, 100, (K * N,), dtype=torch.uint8, device="cuda", generator=g)
+        C = torch.zeros(M, N, dtype=torch.bfloat16, device="cuda")
+        for r in range(reps):
+            H.hif8_gemm(A, K, Wt, N, 0, C, N, H.BF16, M, N, K, None, None, ws, 256)
+            H.hif8_gemm(A, K, Wt, K, 1, C, N, H.BF16, M, N, K, None, None, ws, 256)
+    elif case == "gemm_forms":
+        M, N, K = 4096, 7168, 4096
+        A = torch.randint(8, 100, (M * K,), dtype=torch.uint8, device="cuda", generator=g)
+        Wt = torch.randint(8, 100, (K * N,), dtype=torch.uint8, device="cuda", generator=g)
+        Cb = torch.zeros(M, N, dtype=torch.bfloat16, device="cuda")
+        Cf = torch.zeros(M, N, dtype=torch.float32, device="cuda")
+        big = H.hif8_workspace_bytes(H.WS_GEMM, M * K + K * N)
+        gws = torch.empty(big, dtype=torch.uint8, device="cuda")
+        for r in range(reps):
+            H.hif8_gemm_ex(A, K, 0, Wt, N, 0, Cb, N, H.BF16, M, N, K, None, None, None, 0, gws, big)
+            H.hif8_gemm_ex(A, K, 0, Wt, K, 1, Cb, N, H.BF16, M, N, K, None, None, None, 0, gws, big)
+            H.hif8_gemm_ex(A, M, 1, Wt, N, 0, Cf, N, H.F32, M, N, K, None, None, None, 1, gws, big)
+            H.hif8_gemm_ex(A, M, 1, Wt, K, 1, Cb, N, H.BF16, M, N, K, None, None, None, 0, gws, big)
+    elif case == "channel_bf16":
+        K, N = 8192, 14336
+        w = (torch.randn(K, N, generator=g, device="cuda") * 0.02).to(torch.bfloat16)
+        q = torch.empty(K * N, dtype=torch.uint8, device="cuda")
+        amax = torch.empty(N, dtype=torch.float32, device="cuda")
+        se = torch.empty(N, dtype=torch.int32, device="cuda")
+        flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+        for r in range(reps):
+            H.hif8_channel_amax_scale_encode(w, H.BF16, q, K, N, 1, 14, H.RND_TA, 0, 0, None, amax, se)
+            H.hif8_channel_amax_scale_encode(w, H.BF16, q, N, K, 0, 14, H.RND_TA, 0, 0, None, amax, se)
+            H.hif8_check_finite(w, H.BF16, K * N, flag)
+    else:
+        raise SystemExit(f"unknown case {case}; one of {', '.join(CASES)}")
+    torch.cuda.synchronize()
+    print("done", case, H.hif8_launch_count())
+
+
+# --------------------------------------------------------------------------------------------------------------
+# Reference arm: the CPU oracle
+# --------------------------------------------------------------------------------------------------------------
 def run_reference(args, rank):
     if rank != 0:
         return
@@ -372,6 +562,54 @@ def run_reference(args, rank):
     print(json.dumps(line))
 
 
+# --------------------------------------------------------------------------------------------------------------
+# Multi-GPU figures beside the headline (world > 1): a tensor sharded over the ranks, and the column-sharded GEMM
+# --------------------------------------------------------------------------------------------------------------
+def sharded_results(H, torch, dist, rank, world, stream):
+    from paper_2409_16626_b200 import sharded
+    out = {}
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def timed(fn, reps):
+        for _ in range(3):
+            fn()
+        dist.barrier()
+        torch.cuda.synchronize()
+        ev0.record(stream)
+        for _ in range(reps):
+            fn()
+        ev1.record(stream)
+        torch.cuda.synchronize()
+        dist.barrier()
+        return max_over_ranks([ev0.elapsed_time(ev1) / reps], dist, "cuda")[0]
+
+    # the 4096 x 4096 FP32 tensor split into `world` contiguous slices: hif8_amax -> 4-byte max all-reduce (NCCL) ->
+    # hif8_encode_from_amax; 9 algorithmic bytes per element as for the just-in-time call on one GPU
+    lo, hi = sharded.shard_range(N_EL, world, rank, 16)
+    shard = torch.from_numpy(W.normal_f32((ROWS, COLS), seed=1234).reshape(-1)[lo:hi].copy()).cuda()
+    dst = torch.empty(hi - lo, dtype=torch.uint8, device="cuda")
+    d_amax = torch.zeros(1, dtype=torch.float32, device="cuda")
+    ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+    ms = timed(lambda: sharded.sharded_amax_scale_encode(H, shard, H.F32, dst, hi - lo, 14, H.RND_TA, 0, 0, d_amax, ws, 256), 50)
+    out["sharded_amax_scale_encode_fp32_4096x4096"] = {"ms": ms, "GBps_whole_tensor": 9 * N_EL / ms / 1e6, "scaling": "strong",
+                                                       "collective": "one 4-byte max all-reduce (NCCL)"}
+    # GEMM 8192 x 28672 x 8192 with Wq split along N: every rank multiplies the whole A by its own column block and owns
+    # that block of C; no collective on the data path
+    M, N, K = 8192, 28672, 8192
+    c0, c1 = sharded.shard_range(N, world, rank, 256)
+    g = torch.Generator(device="cuda")
+    g.manual_seed(77)
+    Aq = torch.randint(8, 100, (M, K), dtype=torch.uint8, device="cuda", generator=g)
+    Wq = torch.randint(8, 100, (K, c1 - c0), dtype=torch.uint8, device="cuda", generator=g)
+    C = torch.empty(M, c1 - c0, dtype=torch.bfloat16, device="cuda")
+    gb = H.hif8_workspace_bytes(H.WS_GEMM, M * K + K * (c1 - c0))
+    gws = torch.empty(gb, dtype=torch.uint8, device="cuda")
+    ms = timed(lambda: sharded.column_sharded_gemm(H, Aq, Wq, C, M, c1 - c0, K, None, None, gws, gb), 3)
+    out["gemm_8192x28672x8192_w_sharded_along_n"] = {"ms": ms, "TFLOPs_whole_job": 2.0 * M * N * K / ms / 1e9, "scaling": "strong",
+                                                     "collective": "none", "columns_of_rank0": [c0, c1]}
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -381,10 +619,15 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the secondary workloads (fake-quant, 2^28 stress, GEMM)")
+    ap.add_argument("--case", default=None, help="run one named workload a few times and exit (for a profiler): " + ", ".join(CASES))
+    ap.add_argument("--reps", type=int, default=3, help="repetitions of --case")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     rank, world, local = env_int("RANK", 0), env_int("WORLD_SIZE", 1), env_int("LOCAL_RANK", 0)
 
+    if args.case:
+        run_case(args.case, args.reps)
+        return
     if args.impl == "reference":
         run_reference(args, rank)
         return
@@ -409,20 +652,15 @@ def main():
     stream = torch.cuda.current_stream()
     sp = stream.cuda_stream
 
-    def encode_call(i):
-        H.hif8_amax_scale_encode(srcs[i], H.F32, codes[i], N_EL, 14, H.RND_TA, 0, 0, None, scal[0:1], scal[1:2], scal[2:3],
-                                 ws, wsb, stream=sp)
-
-    def decode_call(i, se):
-        H.hif8_decode(codes[i], backs[i], H.F32, N_EL, se, stream=sp)
-
-    encode_call(0)
+    H.hif8_amax_scale_encode(srcs[0], H.F32, codes[0], N_EL, 14, H.RND_TA, 0, 0, None, scal[0:1], scal[1:2], scal[2:3], ws, wsb, stream=sp)
     torch.cuda.synchronize()
     se = int(scal[1].item())   # same distribution for every tensor of the pool: the descale exponent is fixed up front
+    d_se = scal[1:2].clone()
 
     for w in range(args.warmup):
-        encode_call(w % POOL)
-        decode_call(w % POOL, se)
+        H.hif8_amax_scale_encode(srcs[w % POOL], H.F32, codes[w % POOL], N_EL, 14, H.RND_TA, 0, 0, None, scal[0:1], scal[1:2],
+                                 scal[2:3], ws, wsb, stream=sp)
+        H.hif8_decode(codes[w % POOL], backs[w % POOL], H.F32, N_EL, se, stream=sp)
     torch.cuda.synchronize()
 
     def barrier():
@@ -434,6 +672,8 @@ def main():
     # The launch sequence of POOL consecutive steps (one per buffer set) is captured once in a CUDA graph and
     # replayed, so the host's per-launch cost stays out of the device timeline; K steps = K // POOL replays of that
     # graph plus one replay of a second graph holding the remaining K % POOL steps, so exactly K steps are timed.
+    # The region of K steps is repeated (at least MIN_REPEATS times, more when it is short) and the median region is the
+    # one reported, with the best and the worst beside it.
     K = max(1, args.steps)
     W_REPLAYS = max(1, -(-args.warmup // POOL))   # warm-up in whole replays: at least args.warmup steps
     ws2 = [ws, torch.empty(max(wsb, 256), dtype=torch.uint8, device="cuda")]
@@ -464,67 +704,70 @@ def main():
         if tail is not None:
             tail.replay()
 
-    def time_graph(gr, tail):
+    def time_region(gr, tail, repeats):
+        """per-step times (ms) of `repeats` regions of exactly K steps each; max over ranks per region"""
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        per_step = []
+        for _ in range(repeats):
+            barrier()
+            a.record(stream)
+            replay_steps(gr, tail)
+            b.record(stream)
+            torch.cuda.synchronize()
+            per_step.append(a.elapsed_time(b) / K)
+        barrier()
+        return max_over_ranks(per_step, dist if world > 1 else None, "cuda")
+
+    def warm(gr, tail):
         for _ in range(W_REPLAYS):
             gr.replay()
         if tail is not None:
             tail.replay()
         torch.cuda.synchronize()
+
+    serial, serial_tail = capture(False), (capture(False, K % POOL) if K % POOL else None)
+    graph, graph_tail = capture(True), (capture(True, K % POOL) if K % POOL else None)
+    warm(serial, serial_tail)
+    warm(graph, graph_tail)
+    R = repeats_for(K * 0.035)
+
+    def kernel_stats(call):
+        """one call of the step in a graph of its own (POOL launches over the rotating buffers), replayed between two
+        events: direct launches would time the host's launch rate, not these ~15 us kernels"""
+        gk = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gk):
+            cs = torch.cuda.current_stream().cuda_stream
+            for i in range(POOL):
+                call(i, cs)
+        reps = max(4, min(K, 600) // POOL)
+        for _ in range(3):
+            gk.replay()
+        torch.cuda.synchronize()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream)
-        replay_steps(gr, tail)
-        b.record(stream)
-        torch.cuda.synchronize()
-        return a.elapsed_time(b) / K
-
-    # one stream: every kernel waits for the previous one to drain
-    serial_ms = time_graph(capture(False), capture(False, K % POOL) if K % POOL else None)
-    graph = capture(True)
-    graph_tail = capture(True, K % POOL) if K % POOL else None
-    for _ in range(W_REPLAYS):
-        graph.replay()
-    if graph_tail is not None:
-        graph_tail.replay()
-    torch.cuda.synchronize()
-    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    with ClockSampler(local) as clk:
-        t0.record(stream)
-        replay_steps(graph, graph_tail)
-        t1.record(stream)
-        torch.cuda.synchronize()
-        # per-kernel durations, measured live: each kernel of the step in a graph of its own (POOL launches over the
-        # rotating buffers: hif8_amax -> the two-word clearing kernel + amax_kernel; hif8_encode with the scale known ->
-        # the same convert_kernel the scaled call launches; hif8_decode -> decode_kernel), replayed between two events.
-        # Direct launches would time the host's launch rate, not these ~15 us kernels.
-        amax_out = torch.zeros(1, dtype=torch.float32, device="cuda")
-
-        def kernel_ms(call):
-            gk = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(gk):
-                cs = torch.cuda.current_stream().cuda_stream
-                for i in range(POOL):
-                    call(i, cs)
-            R = max(4, min(K, 600) // POOL)   # own repeat count: these are per-kernel figures, not the timed K steps
-            for _ in range(3):
-                gk.replay()
-            torch.cuda.synchronize()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        per = []
+        for _ in range(MIN_REPEATS):
             a.record(stream)
-            for _ in range(R):
+            for _ in range(reps):
                 gk.replay()
             b.record(stream)
             torch.cuda.synchronize()
-            return a.elapsed_time(b) / (R * POOL)
+            per.append(a.elapsed_time(b) / (reps * POOL))
+        return per
 
-        amax_ms = kernel_ms(lambda i, cs: H.hif8_amax(srcs[i], H.F32, N_EL, amax_out, ws, wsb, stream=cs))
-        conv_ms = kernel_ms(lambda i, cs: H.hif8_encode(srcs[i], H.F32, codes[i], N_EL, se, H.RND_TA, 0, 0, stream=cs))
-        dec_ms = kernel_ms(lambda i, cs: H.hif8_decode(codes[i], backs[i], H.F32, N_EL, se, stream=cs))
-        enc_ms = kernel_ms(lambda i, cs: H.hif8_amax_scale_encode(srcs[i], H.F32, codes[i], N_EL, 14, H.RND_TA, 0, 0, None,
-                                                                  scal[0:1], scal[1:2], scal[2:3], ws, wsb, stream=cs))
-    barrier()
-    launches = 4 * K   # accumulator clear + amax + convert + decode kernels per step (graph replays)
-    total_ms = t0.elapsed_time(t1)
+    amax_out = torch.zeros(1, dtype=torch.float32, device="cuda")
+    with ClockSampler(local) as clk:
+        step_samples = time_region(graph, graph_tail, R)
+        serial_samples = time_region(serial, serial_tail, R)
+        k_amax = kernel_stats(lambda i, cs: H.hif8_amax(srcs[i], H.F32, N_EL, amax_out, ws, wsb, stream=cs))
+        k_conv = kernel_stats(lambda i, cs: H.hif8_encode(srcs[i], H.F32, codes[i], N_EL, se, H.RND_TA, 0, 0, stream=cs))
+        k_dec = kernel_stats(lambda i, cs: H.hif8_decode(codes[i], backs[i], H.F32, N_EL, se, stream=cs))
+        k_enc = kernel_stats(lambda i, cs: H.hif8_amax_scale_encode(srcs[i], H.F32, codes[i], N_EL, 14, H.RND_TA, 0, 0, None,
+                                                                    scal[0:1], scal[1:2], scal[2:3], ws, wsb, stream=cs))
+        # delayed-scaling form of the same conversion: the exponent comes from device memory, amax of this tensor is
+        # reduced in the same pass (one launch, 5 B/element)
+        k_del = kernel_stats(lambda i, cs: H.hif8_amax_scale_encode(srcs[i], H.F32, codes[i], N_EL, 14, H.RND_TA, 0, 0, d_se,
+                                                                    scal[0:1], None, None, ws, wsb, stream=cs))
+    launches = 4 * K   # accumulator clear + amax + convert + decode kernels per step (graph replays), per timed region
 
     # ---- end to end: pinned host input -> device, both calls, results back to pinned host memory.  Consecutive
     # steps alternate between two streams (own host buffers, workspace and scalars each), so the upload of one step
@@ -566,33 +809,61 @@ def main():
     e1.record(stream)
     torch.cuda.synchronize()
     barrier()
-    e2e_ms = e0.elapsed_time(e1) / E
-
-    total_ms, e2e_ms, enc_ms, dec_ms, amax_ms, conv_ms = max_over_ranks(
-        [total_ms, e2e_ms, enc_ms, dec_ms, amax_ms, conv_ms], dist if world > 1 else None, "cuda")
+    e2e_ms = max_over_ranks([e0.elapsed_time(e1) / E], dist if world > 1 else None, "cuda")[0]
+    if world > 1:
+        k_amax, k_conv, k_dec, k_enc, k_del = [max_over_ranks(v, dist, "cuda") for v in (k_amax, k_conv, k_dec, k_enc, k_del)]
+        multi = sharded_results(H, torch, dist, rank, world, stream)
 
     if rank == 0:
-        ms_per_step = total_ms / K
+        step, serial_st = spread(step_samples), spread(serial_samples)
+        ms_per_step = step["ms"]
         value = job_throughput(world, BYTES_STEP, ms_per_step)
-        peak, peak_kind = load_peaks()
+        peak, tf_peak, tf_sustained, peak_kind = load_peaks()
         kernels = {
-            "amax_kernel<f32>": {"ms": amax_ms, "bytes": 4 * N_EL, "note": "hif8_amax call: accumulator-clearing kernel + amax kernel"},
-            "convert_kernel<f32,TA>": {"ms": conv_ms, "bytes": 5 * N_EL},
-            "decode_kernel<f32>": {"ms": dec_ms, "bytes": 5 * N_EL},
+            "amax_kernel<f32>": dict(spread(k_amax), bytes=4 * N_EL, note="hif8_amax call: accumulator-clearing kernel + amax kernel"),
+            "convert_kernel<f32,TA>": dict(spread(k_conv), bytes=5 * N_EL),
+            "decode_kernel<f32>": dict(spread(k_dec), bytes=5 * N_EL),
         }
         for kv in kernels.values():
             kv["GBps"] = kv["bytes"] / (kv["ms"] * 1e-3) / 1e9
             kv["frac"] = kv["GBps"] / peak
+        enc_st, del_st = spread(k_enc), spread(k_del)
         # the dominant kernel: longest live duration among the single-kernel calls
         dom = max(("convert_kernel<f32,TA>", "decode_kernel<f32>"), key=lambda kname: kernels[kname]["ms"])
+
+        def row(st, nbytes):
+            return {"ms": round(st["ms"], 5), "best_ms": round(st["best_ms"], 5), "frac": round(nbytes / st["ms"] / 1e6 / peak, 4),
+                    "bound": "hbm"}
+
+        by_config = {
+            "C2_step_two_streams_14B_per_el_algorithmic": row(step, BYTES_STEP),
+            "C2_step_single_stream_14B_per_el_algorithmic": row(serial_st, BYTES_STEP),
+            "C2_amax_scale_encode_call_9B_per_el": row(enc_st, BYTES_ENCODE),
+            "C2_delayed_scaling_encode_call_5B_per_el": row(del_st, 5 * N_EL),
+            "C2_amax_call_4B_per_el": row(kernels["amax_kernel<f32>"], 4 * N_EL),
+            "C2_convert_kernel_5B_per_el": row(kernels["convert_kernel<f32,TA>"], 5 * N_EL),
+            "C2_decode_kernel_5B_per_el": row(kernels["decode_kernel<f32>"], 5 * N_EL),
+        }
+        in_step = [TRAFFIC_IN_STEP[k] for k in ("amax_kernel<f32>", "convert_kernel<f32,TA>", "decode_kernel<f32>")]
+        dram_step = sum(in_step) if all(v is not None for v in in_step) else None
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "u8", "data": "synthetic",
             "config": {"workload": WORKLOAD, "elements": N_EL, "rounding": "TA", "target_exp": 14,
+                       "value_is": "algorithmic bytes per second (14 B/element: both reads of the source and the read of the "
+                                   "codes are counted although the L2 can serve them), not a DRAM bandwidth",
                        "launch": f"CUDA graph of {POOL} steps replayed (+ one graph of steps % {POOL}); even/odd steps "
                                  "(independent tensors) on two streams",
-                       "ms_per_step_single_stream": serial_ms,
+                       "timed": f"{step['repeats']} regions of exactly {K} steps each; ms_per_step is the median region",
+                       "ms_per_step_best": step["best_ms"], "ms_per_step_worst": step["worst_ms"],
+                       "ms_per_step_single_stream": serial_st["ms"], "ms_per_step_single_stream_best": serial_st["best_ms"],
+                       "GBps_single_stream": job_throughput(world, BYTES_STEP, serial_st["ms"]),
+                       "step_dram": {"bytes_per_step": dram_step,
+                                     "GBps": None if dram_step is None else world * dram_step / (ms_per_step * 1e-3) / 1e9,
+                                     "frac_of_peak": None if dram_step is None else dram_step / (ms_per_step * 1e-3) / 1e9 / peak,
+                                     "source": "dram__bytes_read.sum + dram__bytes_write.sum of the three kernels inside the running "
+                                               "sequence (profiler capture with the caches left alone between launches)"},
                        "l2": f"inputs rotate over {POOL} buffer sets ({POOL * N_EL * 4 >> 20} MiB of sources) > 126 MB L2",
                        "bytes_per_step": BYTES_STEP, "elements_per_s": world * N_EL / (ms_per_step * 1e-3)},
             "clocks": clk.summary(),
@@ -601,15 +872,23 @@ def main():
             "gpu_launches": int(launches),
             "roofline": {"bound": "hbm", "kernel": dom, "achieved": kernels[dom]["GBps"], "peak": peak,
                          "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": kernels[dom]["frac"],
-                         "traffic": TRAFFIC.get(dom), "algorithmic_bytes_per_launch": kernels[dom]["bytes"],
-                         "avg_launch_ms": kernels[dom]["ms"]},
+                         "traffic": TRAFFIC_COLD.get(dom), "traffic_in_step": TRAFFIC_IN_STEP.get(dom),
+                         "algorithmic_bytes_per_launch": kernels[dom]["bytes"],
+                         "avg_launch_ms": kernels[dom]["ms"], "best_launch_ms": kernels[dom]["best_ms"],
+                         "by_config": by_config,
+                         "by_config_peaks": {"hbm": peak, "tensor": tf_peak, "tensor_sustained": tf_sustained, "kind": f"of {peak_kind}",
+                                             "units": "frac = algorithmic GB/s / hbm, or TFLOP/s / tensor (cuBLAS BF16 burst)"}},
             "kernels": kernels,
-            "calls": {"amax_scale_encode_ms": enc_ms, "amax_scale_encode_GBps": BYTES_ENCODE / (enc_ms * 1e-3) / 1e9},
+            "calls": {"amax_scale_encode_ms": enc_st["ms"], "amax_scale_encode_GBps": BYTES_ENCODE / (enc_st["ms"] * 1e-3) / 1e9,
+                      "delayed_scaling_encode_ms": del_st["ms"]},
         }
+        if world > 1:
+            line["sharded"] = multi
         if world == 1 and not args.no_extra:
             del srcs, codes, backs
             torch.cuda.empty_cache()
-            line["extra"] = extra_results(H, torch, peak, peak_kind)
+            line["extra"], table = extra_results(H, torch, peak, tf_peak, peak_kind)
+            by_config.update(table)
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(1 << 23)
         print(json.dumps(line))

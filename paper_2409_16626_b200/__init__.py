@@ -5,7 +5,7 @@ The binding (and with it libhif8.so) is loaded on first attribute access, so tha
 """
 import importlib
 
-_SUBMODULES = ("build", "binding", "profile_cases", "sharded")
+_SUBMODULES = ("build", "binding", "sharded")
 
 
 def __getattr__(name):

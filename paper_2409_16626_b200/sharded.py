@@ -7,6 +7,10 @@ behind that factor is the maximum over all shards.  The data path is three steps
     all_reduce(MAX) over the group        -> the tensor's amax on every rank (NCCL over NVLink; latency only)
     hif8_encode_from_amax(shard, amax)    -> each rank converts its shard with the common exponent
 
+The GEMM shards the same way the paper's layers do: the weight bytes are split along N (`shard_range` gives each rank a
+block of whole 256-column tiles), every rank multiplies the full activation by its block and owns that block of C --
+no collective on the data path (`column_sharded_gemm`).
+
 This module is marshalling around those calls; `ops` is the binding module (injected so that the host logic can be
 exercised without a GPU).  torch.distributed is the plumbing: NCCL for CUDA tensors, gloo in the CPU tests.
 """
@@ -29,3 +33,23 @@ def sharded_amax_scale_encode(ops, shard, src_dtype, dst, n, target_exp, rnd, fl
             dist.all_reduce(d_amax, op=dist.ReduceOp.MAX, group=group)
     ops.hif8_encode_from_amax(shard, src_dtype, dst, n, target_exp, rnd, flags, seed, d_amax, d_scale_exp_out, None, stream)
     return d_amax
+
+
+def shard_range(n, world, rank, align=1):
+    """[lo, hi) of rank `rank` when n units are dealt out in `world` contiguous pieces whose boundaries are multiples of
+    `align` (the last piece takes the ragged end).  Pieces differ by at most `align` units and tile [0, n) exactly."""
+    units = -(-n // align)
+    lo = (units * rank // world) * align
+    hi = (units * (rank + 1) // world) * align
+    return min(lo, n), min(hi, n)
+
+
+def column_sharded_gemm(ops, Aq, Wq_shard, C_shard, M, n_local, K, d_scale_exp_a, d_scale_exp_w, workspace, workspace_bytes,
+                        c_dtype=None, stream=None):
+    """This rank's column block of C = dec(Aq) dec(Wq) * 2^-(sa+sw): Wq_shard is [K, n_local] (contiguous), C_shard
+    [M, n_local].  The per-tensor exponents are those of the whole tensors, so the blocks of all ranks put side by side
+    are the product of the unsharded call."""
+    if n_local == 0:
+        return
+    ops.hif8_gemm(Aq, K, Wq_shard, n_local, 0, C_shard, n_local, ops.BF16 if c_dtype is None else c_dtype, M, n_local, K,
+                  d_scale_exp_a, d_scale_exp_w, workspace, workspace_bytes, stream)

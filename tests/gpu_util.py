@@ -35,3 +35,10 @@ def dev_empty(n, np_dtype, offset_bytes=0):
 def workspace():
     n = H.hif8_workspace_bytes(H.WS_AMAX_SCALE_ENCODE)
     return torch.empty(max(n, 256), dtype=torch.uint8, device="cuda"), n
+
+
+def bf16_half_ulp(x):
+    """Half a unit in the last place of a bfloat16 (8-bit significand) at the binade of |x| (normal range):
+    what one round-to-nearest into BF16 can cost."""
+    e = np.floor(np.log2(np.maximum(np.abs(x), 2.0 ** -126)))
+    return 2.0 ** (e - 8)

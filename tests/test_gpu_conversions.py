@@ -287,8 +287,9 @@ def test_fake_quant_bf16_in_place_scale_edges_and_tails(mode, omode):
 
 
 # ----------------------------------------------------------------------------- full sizes: sampled outputs
-def test_config2_full_size_sampled():
-    # FP32 4096x4096 N(0,1): per-tensor scaled encode + decode, checked on a strided sample and on whole tiles
+def test_config2_full_size():
+    # FP32 4096x4096 N(0,1): per-tensor scaled encode + decode, every element (neighbour-pair oracle), and a strided
+    # sample plus both ends through the oracle's scan of all 256 codes
     x = W.normal_f32((4096, 4096), seed=1234).reshape(-1)
     n = x.size
     ws, wsb = workspace()
@@ -302,11 +303,12 @@ def test_config2_full_size_sampled():
     assert int(outs[1]) == se
     H.hif8_decode(codes, back, H.F32, n, se)
     torch.cuda.synchronize()
-    idx = np.unique(np.concatenate([np.arange(0, n, 53), np.arange(0, 70000), np.arange(n - 70000, n)]))
-    want_codes = O.encode(x[idx], O.F32, se, O.TA, 0, quick=True)
     got_codes = codes.cpu().numpy()
-    assert_same(got_codes[idx], want_codes)
-    assert_same(back.cpu().numpy().view(np.uint32)[idx], O.decode(want_codes, O.F32, se))
+    want_codes = O.encode(x, O.F32, se, O.TA, 0, quick=True)
+    assert_same(got_codes, want_codes)
+    assert_same(back.cpu().numpy().view(np.uint32), O.decode(want_codes, O.F32, se))
+    idx = np.unique(np.concatenate([np.arange(0, n, 53), np.arange(0, 70000), np.arange(n - 70000, n)]))
+    assert_same(got_codes[idx], O.encode(x[idx], O.F32, se, O.TA, 0, quick=False))
 
 
 def test_f32_full_sweep_all_2_32_patterns():
@@ -327,12 +329,12 @@ def test_f32_full_sweep_all_2_32_patterns():
 
 
 @pytest.mark.parametrize("mode", [H.RND_HR, H.RND_SSR, H.RND_TE, H.RND_SR])
-def test_f32_sweep_slices_other_modes(mode):
-    # the slices that hold the HiF8 range (2^-23 .. 2^16), the specials and both signs
+def test_f32_full_sweep_other_modes(mode):
+    # every FP32 encoding of either sign in every other rounding mode, 64 slices of 2^26 patterns
     n = 1 << 26
     out = torch.empty(n, dtype=torch.uint8, device="cuda")
     ar = torch.arange(n, dtype=torch.int64, device="cuda")
-    for chunk in (0, 12, 13, 14, 15, 16, 17, 31, 45, 49, 63):
+    for chunk in range(64):
         first = chunk << 26
         d = (ar + first).to(torch.int32) if first < (1 << 31) else (ar + (first - (1 << 32))).to(torch.int32)
         H.hif8_encode(d, H.F32, out, n, 0, mode, 0, 77)

@@ -9,7 +9,7 @@ import paper_2409_16626_b200 as H
 import workloads as W
 from oracle import hif8_oracle as O
 
-from gpu_util import NP_OF, dev_empty, to_dev
+from gpu_util import NP_OF, bf16_half_ulp, dev_empty, to_dev
 
 pytestmark = pytest.mark.gpu
 MODES = [H.RND_TA, H.RND_HR, H.RND_SSR, H.RND_TE, H.RND_SR]
@@ -140,7 +140,9 @@ def test_gemm_channel_scaled(c_dtype, w_is_nk, staged):
     rows, cols = np.divmod(np.arange(M * N), N)
     Cs, S = O.gemm_entries_channel(Aq, Wq, w_is_nk, sa, sw, rows, cols)
     Cs, S = Cs.reshape(M, N), S.reshape(M, N)
-    tol = 1e-5 * S + (2.0 ** -8 * np.abs(Cs) if c_dtype == H.BF16 else 0.0)
+    tol = 1e-5 * S
+    if c_dtype == H.BF16:
+        tol = tol + bf16_half_ulp(np.abs(Cs) + tol)
     assert np.all(np.abs(out[:, :N] - Cs) <= tol)
 
 

@@ -11,8 +11,12 @@ import torch
 
 import paper_2409_16626_b200 as H
 import workloads as W
+from oracle import hif8_oracle as O
 
 pytestmark = pytest.mark.gpu
+
+
+ORACLE_MODE = {H.RND_TA: O.TA, H.RND_HR: O.HR}
 
 
 def run_both(src, dtype, target, mode, d_se_in=None):
@@ -30,9 +34,20 @@ def run_both(src, dtype, target, mode, d_se_in=None):
         H.hif8_amax_scale_encode_static(src, dtype, codes, n, target, mode, 0, 3, d_se_in, out[0:1], out[1:2], out[2:3])
         results.append((codes, out))
     torch.cuda.synchronize()
+    # what the method defines, from the CPU oracle: amax over the tensor, the scale exponent, the codes
+    host = src.cpu().numpy()
+    host = host.view(np.uint16) if dtype != H.F32 else host
+    amax, se = O.amax_scale(host, dtype, target)
+    if d_se_in is not None:
+        se = int(d_se_in.item())
+    want = O.encode(host, dtype, se, ORACLE_MODE[mode], 0, seed=3, quick=True)
     for codes, out in results:
         assert torch.equal(codes, ref_codes)             # bit-exact, like every conversion test here
         assert torch.equal(out, ref_out)
+        assert np.array_equal(codes.cpu().numpy(), want)
+        o = out.cpu().numpy()
+        assert o[0:1].view(np.float32)[0] == np.float32(amax) and int(o[1]) == se
+        assert o[2:3].view(np.float32)[0] == np.float32(2.0 ** se)
 
 
 def test_static_scratch_matches_workspace_variant():
