@@ -147,9 +147,13 @@ __global__ void __launch_bounds__(kThreads) convert_kernel(const ConvParams p, u
     const uint32_t k0 = (uint32_t)p.seed, k1 = (uint32_t)(p.seed >> 32);
     float amax = 0.f;
 
-    const unsigned long long stride = (unsigned long long)gridDim.x * kThreads * kUnroll;
-    for (unsigned long long base = (unsigned long long)blockIdx.x * kThreads * kUnroll; base < n_vec; base += stride) {
-        if (base + (unsigned long long)kThreads * kUnroll <= n_vec)
+    // group g of the tensor = vectors [g, g + 1) * kThreads * kUnroll; this block takes groups blockIdx.x, + gridDim.x, ...
+    // counted from the front or (p.reverse) from the back of the tensor
+    constexpr unsigned long long kGroupVecs = (unsigned long long)kThreads * kUnroll;
+    const unsigned long long n_groups = (n_vec + kGroupVecs - 1) / kGroupVecs;
+    for (unsigned long long g = blockIdx.x; g < n_groups; g += gridDim.x) {
+        const unsigned long long base = (p.reverse ? n_groups - 1 - g : g) * kGroupVecs;
+        if (base + kGroupVecs <= n_vec)
             convert_group<SRC, MODE, FQ, AMAX, true>(p, sm, base, n_vec, scale, d1, d2, k0, k1, amax);
         else
             convert_group<SRC, MODE, FQ, AMAX, false>(p, sm, base, n_vec, scale, d1, d2, k0, k1, amax);
@@ -316,7 +320,6 @@ __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, uns
     __syncthreads();
 
     const uint4* src = reinterpret_cast<const uint4*>(p.src);
-    const unsigned long long stride = (unsigned long long)gridDim.x * kThreads * kUnroll;
     // one group of kUnroll vectors per thread; a group wholly inside the tensor runs without bounds checks
     auto group = [&](unsigned long long base, auto full_tag) {
         constexpr bool FULL = decltype(full_tag)::value;
@@ -381,9 +384,14 @@ __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, uns
             __stcs(reinterpret_cast<uint4*>(p.dst) + u, make_uint4(o[0], o[1], o[2], o[3]));
         }
     };
-    for (unsigned long long base = (unsigned long long)blockIdx.x * kThreads * kUnroll; base < n_vec; base += stride) {
-        if (base + (unsigned long long)kThreads * kUnroll <= n_vec) group(base, std::true_type{});
-        else group(base, std::false_type{});
+    {
+        constexpr unsigned long long kGroupVecs = (unsigned long long)kThreads * kUnroll;
+        const unsigned long long n_groups = (n_vec + kGroupVecs - 1) / kGroupVecs;
+        for (unsigned long long g = blockIdx.x; g < n_groups; g += gridDim.x) {  // from the back of the tensor with p.reverse
+            const unsigned long long base = (p.reverse ? n_groups - 1 - g : g) * kGroupVecs;
+            if (base + kGroupVecs <= n_vec) group(base, std::true_type{});
+            else group(base, std::false_type{});
+        }
     }
     {   // tail / unaligned elements
         const unsigned long long tid = (unsigned long long)blockIdx.x * kThreads + threadIdx.x;
@@ -723,6 +731,7 @@ static int scaled_convert(bool fq, const void* src, void* dst, int dtype, size_t
         rc = launch_amax(src, dtype, n, ws, nullptr, sms, st);
         if (rc) return rc;
         p.d_amax_bits = ws;
+        p.reverse = 1;  // the amax pass has just read the tensor front to back
         if (inplace_fq) return launch_fq_ta(dtype, rnd, p, vec_ok, sms, st);
         return fq ? dispatch_convert<true, false>(dtype, rnd, p, vec_ok, sms, st)
                   : dispatch_convert<false, false>(dtype, rnd, p, vec_ok, sms, st);
@@ -784,6 +793,7 @@ int hif8_encode_from_amax(const void* src, int src_dtype, uint8_t* dst, size_t n
     ConvParams p{};
     p.src = src; p.dst = dst; p.n = n; p.flags = flags; p.seed = seed; p.target_exp = target_exp;
     p.d_amax_bits = reinterpret_cast<const uint32_t*>(d_amax);  // a non-negative float: its bits order as the value
+    p.reverse = 1;  // the caller has just reduced amax over this tensor (hif8_amax), front to back
     p.d_scale_exp_out = d_scale_exp_out; p.d_scale_out = d_scale_out;
     const bool vec_ok = aligned16(src) && (reinterpret_cast<uintptr_t>(dst) % (src_dtype == HIF8_F32 ? 4 : 8)) == 0;
     return dispatch_convert<false, false>(src_dtype, rnd, p, vec_ok, sms, (cudaStream_t)stream);

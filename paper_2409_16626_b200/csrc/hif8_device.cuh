@@ -196,6 +196,8 @@ struct ConvParams {
     int* d_scale_exp_out;
     float* d_scale_out;
     void* scale_state;            // delayed scaling: ScaleState that the last block of an amax-reducing pass advances
+    int reverse;                  // walk the tensor from its end: set for the second pass of just-in-time scaling, so that
+                                  // the lines the amax pass read last (still in L2) are the ones re-read first
 };
 
 template <int SRC> struct SrcTraits;

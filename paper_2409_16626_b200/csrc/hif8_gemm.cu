@@ -16,7 +16,9 @@
 //   warp  4    TMA producer: HiF8 byte tiles (A: 128 x 64, W: 128 x 64 or 64 x 128) into a 4-stage staging ring
 //   warp  5    MMA issuer: one elected thread of the even CTA issues tcgen05.mma (256 x 256 x 16 over the pair,
 //              BF16 x BF16 -> FP32 in the TMEM of both CTAs)
-//   warps 6-21 decode: staging bytes -> BF16 in the canonical 128-byte-swizzled operand layout (3-stage ring)
+//   warps 6-21 decode: staging bytes -> BF16; W goes into the canonical 128-byte-swizzled shared-memory operand layout,
+//              A ([M,K] form) goes straight into tensor memory (tcgen05.st, one thread per row), from where the MMA
+//              reads it as its A operand: the decoded A tile costs neither a shared-memory store nor an operand read
 // The operand layout follows the shared-memory matrix descriptor of tcgen05: K-major operands are rows of 64 BF16
 // (128 bytes), eight rows form a 1024-byte swizzle atom, 16-byte chunk j of row r is stored at chunk j ^ (r % 8).
 // W given as [K, N] is decoded in place as an MN-major operand (atoms of 8 k-rows x 64 n), so no transpose is needed.
@@ -55,7 +57,10 @@ constexpr int kTmaWarp = 4, kMmaWarp = 5, kFirstDecodeWarp = 6;
 // per CTA of a pair: 128 rows of A and 128 of the 256 columns of W
 constexpr uint32_t kA8Bytes = BM * BK, kB8Bytes = (BN / 2) * BK;            // 8 KiB + 8 KiB
 constexpr uint32_t kABfBytes = BM * BK * 2, kBBfBytes = (BN / 2) * BK * 2;  // 16 KiB + 16 KiB
-constexpr uint32_t kTmemCols = 256;
+// tensor memory of the fused kernel: columns 0-255 the 128 x 256 FP32 accumulator, then one A operand stage (128 rows x
+// 64 BF16 = 32 columns) per operand stage; allocations are powers of two
+constexpr uint32_t kTmemColsAcc = 256, kTmemAStageCols = BK / 2, kTmemCols = 512;
+static_assert(kTmemColsAcc + kStagesBf * kTmemAStageCols <= kTmemCols, "A operand stages must fit beside the accumulator");
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
 
 struct SmemLayout {
@@ -146,6 +151,20 @@ __device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t (&r)
         : "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// 32 consecutive columns of this thread's tensor-memory lane (lane field of taddr = first lane of the warp's quarter)
+__device__ __forceinline__ void tmem_st_32x32b_x32(uint32_t taddr, const uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // ---- CTA pairs (cluster of two CTAs, cta_group::2)
 __device__ __forceinline__ uint32_t cluster_ctarank()
@@ -203,6 +222,16 @@ __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_des
         "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// the same with the A operand in tensor memory (K-major, row i of each CTA's 128 rows in lane i, two BF16 per column)
+__device__ __forceinline__ void tc_mma_bf16_pair_a_tmem(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                                        uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
 
 
 // shared-memory matrix descriptor: start address, leading / stride byte offsets (16-byte units), version 1,
@@ -236,10 +265,12 @@ __device__ __forceinline__ uint32_t hif8_to_bf16_bits(uint32_t c)
 
 // Shared-memory accesses by 32-bit shared-window address: the operand ring lives at a run-time offset inside the dynamic
 // allocation, and spelling the state space out keeps every one of these an LDS / STS (never a generic access).
+// (not volatile: the table is constant once it is built and every address derives from a byte read after the barrier
+// wait, so the compiler is free to issue a whole batch of lookups before the first of them is consumed)
 __device__ __forceinline__ uint32_t lds_u32(uint32_t addr)
 {
     uint32_t v;
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    asm("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
     return v;
 }
 __device__ __forceinline__ uint2 lds_v2(uint32_t addr)
@@ -248,22 +279,36 @@ __device__ __forceinline__ uint2 lds_v2(uint32_t addr)
     asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
     return v;
 }
+__device__ __forceinline__ uint4 lds_v4(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
 __device__ __forceinline__ void sts_v4(uint32_t addr, uint4 v)
 {
     asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
-// eight HiF8 bytes -> eight BF16 (one 16-byte operand chunk).  `lut_lane` points at this lane's column of the
-// lane-replicated table: entry of byte c is the 32-bit word at lut_lane + 128 c, so lane L only ever touches
-// shared-memory bank L and the eight lookups of a warp instruction never conflict.
-__device__ __forceinline__ uint4 decode8(uint2 v, uint32_t lut_lane)  // lut_lane: shared address of this lane's column
+// eight HiF8 bytes -> eight BF16 (one 16-byte operand chunk) through the lane-replicated table: lane L only ever touches
+// shared-memory bank L, so the lookups of a warp instruction never conflict.  `lut_lane` is the shared address of this
+// lane's column.  ROW_SHIFT = 7: rows of 128 bytes, entry of byte c at lut_lane + 128 c (extract, scale, add).
+// ROW_SHIFT = 8: rows of 256 bytes in a table that starts on a 64 KiB boundary of the shared window, so that bits 8-15 of
+// lut_lane are zero and ONE byte permute drops the code into them: address = lut_lane with byte 1 replaced by c.
+template <int ROW_SHIFT>
+__device__ __forceinline__ uint4 decode8(uint2 v, uint32_t lut_lane)
 {
     uint32_t o[4];
 #pragma unroll
     for (int i = 0; i < 4; i++) {
         const uint32_t w = i < 2 ? v.x : v.y;
-        const uint32_t c0 = (w >> (16 * (i & 1))) & 0xFFu, c1 = (w >> (16 * (i & 1) + 8)) & 0xFFu;
-        o[i] = __byte_perm(lds_u32(lut_lane + c0 * 128), lds_u32(lut_lane + c1 * 128), 0x5410);
+        if (ROW_SHIFT == 8) {
+            const uint32_t a0 = __byte_perm(w, lut_lane, (i & 1) ? 0x7624 : 0x7604), a1 = __byte_perm(w, lut_lane, (i & 1) ? 0x7634 : 0x7614);
+            o[i] = __byte_perm(lds_u32(a0), lds_u32(a1), 0x5410);
+        } else {
+            const uint32_t c0 = (w >> (16 * (i & 1))) & 0xFFu, c1 = (w >> (16 * (i & 1) + 8)) & 0xFFu;
+            o[i] = __byte_perm(lds_u32(lut_lane + c0 * 128), lds_u32(lut_lane + c1 * 128), 0x5410);
+        }
     }
     return make_uint4(o[0], o[1], o[2], o[3]);
 }
@@ -365,7 +410,7 @@ __device__ __forceinline__ void load_tile_chunks(uint32_t src8, int dt, uint2 (&
         v[it] = MN_MAJOR ? lds_v2(src8 + (q >> 4) * BM + (q & 15) * 8) : lds_v2(src8 + (q >> 3) * BK + (q & 7) * 8);
     }
 }
-template <bool MN_MAJOR>
+template <bool MN_MAJOR, int ROW_SHIFT = 7>
 __device__ __forceinline__ void decode_tile_chunks(const uint2 (&v)[kChunksPerThread], uint32_t dst, int dt, uint32_t lut)
 {
 #pragma unroll
@@ -373,35 +418,85 @@ __device__ __forceinline__ void decode_tile_chunks(const uint2 (&v)[kChunksPerTh
         const int q = it * kGroupThreads + dt;
         if (MN_MAJOR) {
             const int k = q >> 4, jn = q & 15, atom = (jn >> 3) * 8 + (k >> 3);
-            sts_v4(dst + atom * 1024 + (k & 7) * 128 + (((jn & 7) ^ (k & 7)) << 4), decode8(v[it], lut));
+            sts_v4(dst + atom * 1024 + (k & 7) * 128 + (((jn & 7) ^ (k & 7)) << 4), decode8<ROW_SHIFT>(v[it], lut));
         } else {
             const int r = q >> 3, j = q & 7;
-            sts_v4(dst + (r >> 3) * 1024 + (r & 7) * 128 + ((j ^ (r & 7)) << 4), decode8(v[it], lut));
+            sts_v4(dst + (r >> 3) * 1024 + (r & 7) * 128 + ((j ^ (r & 7)) << 4), decode8<ROW_SHIFT>(v[it], lut));
         }
     }
 }
+
+// Shared memory of the fused kernel.
+// A given as [K,M] (decoded into shared memory): the fixed layout of SmemLayout.
+// A given as [M,K] (decoded into tensor memory): no A operand tiles, and the lookup table has rows of 256 bytes and starts on
+// a 64 KiB boundary of the shared window (see decode8).  Everything else is dealt out in 16 KiB slots around the table: as
+// many as fit in front of it, the rest behind it.  Slots 0-3: W operand stages, slots 4-7: byte stages (A 8 KiB + W 8 KiB).
+constexpr uint32_t kSlotBytes = 16384, kLutBytesWide = 65536, kFusedSlots = kStagesBf + kStages8;
+static_assert(kBBfBytes == kSlotBytes && kA8Bytes + kB8Bytes == kSlotBytes, "one stage per slot");
+constexpr uint32_t kSmemBytesWide = 227 * 1024;  // the whole opt-in maximum; the kernel checks that its plan fits
+
+template <bool A_IS_KM>
+struct FusedSmem {
+    uint32_t base, lut, bars, behind;  // shared-window addresses; base is 1024-byte aligned
+    int n_front;                       // slots in front of the table
+    uint32_t end;                      // first byte behind everything
+
+    __device__ explicit FusedSmem(uint32_t raw)
+    {
+        base = (raw + 1023u) & ~1023u;
+        if (A_IS_KM) {
+            lut = base + SmemLayout::lut; bars = base + SmemLayout::bars; behind = 0; n_front = 0; end = base + SmemLayout::total;
+        } else {
+            lut = (base + kLutBytesWide - 1) & ~(kLutBytesWide - 1);
+            const uint32_t front = lut - base;
+            n_front = (int)min(front / kSlotBytes, kFusedSlots);
+            behind = lut + kLutBytesWide;
+            const uint32_t after_slots = behind + (kFusedSlots - n_front) * kSlotBytes;
+            // barriers, tensor-memory slot and abort flag (256 bytes): in the gap in front of the table if there is one
+            bars = (front - n_front * kSlotBytes >= 256u) ? base + n_front * kSlotBytes : after_slots;
+            end = bars >= after_slots ? bars + 256u : after_slots;
+        }
+    }
+    __device__ uint32_t slot(int i) const { return i < n_front ? base + (uint32_t)i * kSlotBytes : behind + (uint32_t)(i - n_front) * kSlotBytes; }
+    __device__ uint32_t a_bf(int s) const { return base + SmemLayout::bf + s * (kABfBytes + kBBfBytes); }                       // A_IS_KM only
+    __device__ uint32_t w_bf(int s) const { return A_IS_KM ? a_bf(s) + kABfBytes : slot(s); }
+    __device__ uint32_t a_u8(int s) const { return A_IS_KM ? base + SmemLayout::u8 + s * (kA8Bytes + kB8Bytes) : slot(kStagesBf + s); }
+    __device__ uint32_t w_u8(int s) const { return a_u8(s) + kA8Bytes; }
+    __device__ uint32_t tmem_slot() const { return bars + SmemLayout::n_bars * 8; }
+    __device__ uint32_t abort_flag() const { return tmem_slot() + 4; }
+};
 
 template <bool A_IS_KM, bool W_IS_NK>
 __global__ void __launch_bounds__(kThreads, 1)
 hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const GemmParams p)
 {
     extern __shared__ unsigned char smem_raw[];
-    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    unsigned char* sm = smem_raw + (base - smem_u32(smem_raw));
+    constexpr int kLutShift = A_IS_KM ? 7 : 8;
+    const FusedSmem<A_IS_KM> plan(smem_u32(smem_raw));
+    const uint32_t base = plan.base;
+    unsigned char* sm = smem_raw - smem_u32(smem_raw);  // generic pointer of shared-window address 0
+    {
+        uint32_t dyn_bytes;
+        asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn_bytes));
+        if (plan.end > smem_u32(smem_raw) + dyn_bytes) {  // the plan does not fit (same verdict in every thread of the pair)
+            if (threadIdx.x == 0) atomicCAS(p.status, 0, 7);
+            return;
+        }
+    }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();  // 0: leader of the pair (issues the MMAs), 1: peer
     const bool leader = rank == 0;
 
-    const uint32_t bars = base + SmemLayout::bars;
+    const uint32_t bars = plan.bars;
     auto bar_u8_full = [&](int s) { return bars + 8u * s; };                                   // per CTA
     auto bar_u8_empty = [&](int s) { return bars + 8u * (kStages8 + s); };                     // per CTA
     auto bar_bf_full = [&](int s) { return bars + 8u * (2 * kStages8 + s); };                  // leader: both CTAs' decode warps
     auto bar_bf_empty = [&](int s) { return bars + 8u * (2 * kStages8 + kStagesBf + s); };     // per CTA, leader's commits
     const uint32_t bar_acc_full = bars + 8u * (2 * kStages8 + 2 * kStagesBf);                  // per CTA, leader's commit
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + SmemLayout::abort_flag);
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + SmemLayout::tmem_slot);
-    uint32_t* lut_all = reinterpret_cast<uint32_t*>(sm + SmemLayout::lut);
-    const uint32_t lut = base + SmemLayout::lut + 4u * lane;  // this lane's column of the table
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + plan.abort_flag());
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + plan.tmem_slot());
+    uint32_t* lut_all = reinterpret_cast<uint32_t*>(sm + plan.lut);
+    const uint32_t lut = plan.lut + 4u * lane;  // this lane's column of the table
 
     // 256 x 256 tile of this pair (groups of 8 tile-rows share their W tiles in L2); this CTA: 128 rows, 128 columns of W
     int tile_m, tile_n;
@@ -410,7 +505,8 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     const int num_kb = (p.K + BK - 1) / BK;
 
     // ---- set-up
-    for (int i = threadIdx.x; i < 256 * 32; i += kThreads) lut_all[i] = hif8_to_bf16_bits(i >> 5);
+    for (int i = threadIdx.x; i < 256 * 32; i += kThreads)  // entry (code i / 32, lane i % 32): rows of 1 << kLutShift bytes
+        lut_all[((i >> 5) << (kLutShift - 2)) + (i & 31)] = hif8_to_bf16_bits(i >> 5);
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages8; s++) { mbar_init(bar_u8_full(s), 1); mbar_init(bar_u8_empty(s), kGroupWarps); }
         for (int s = 0; s < kStagesBf; s++) { mbar_init(bar_bf_full(s), 2 * kGroupWarps); mbar_init(bar_bf_empty(s), 1); }
@@ -420,7 +516,7 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     }
     if (warp == kMmaWarp) {  // this warp owns the TMEM allocation (both CTAs of the pair take part)
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(base + SmemLayout::tmem_slot), "r"(kTmemCols) : "memory");
+                     ::"r"(plan.tmem_slot()), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -437,7 +533,7 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 const int s = kb % kStages8, round = kb / kStages8;
                 if (round > 0 && !mbar_wait(bar_u8_empty(s), (round - 1) & 1, abort_flag, p.status, 1)) break;
                 if (*abort_flag) break;
-                const uint32_t dst_a = base + SmemLayout::u8 + s * (kA8Bytes + kB8Bytes), dst_b = dst_a + kA8Bytes;
+                const uint32_t dst_a = plan.a_u8(s), dst_b = plan.w_u8(s);
                 mbar_arrive_expect_tx(bar_u8_full(s), kA8Bytes + kB8Bytes);
                 if (A_IS_KM) tma_load_2d(dst_a, &map_a, m0, kb * BK, bar_u8_full(s));
                 else tma_load_2d(dst_a, &map_a, kb * BK, m0, bar_u8_full(s));
@@ -466,15 +562,19 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 ok = mbar_wait(bar_bf_full(s), round & 1, abort_flag, p.status, 2);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t a_addr = base + SmemLayout::bf + s * (kABfBytes + kBBfBytes), b_addr = a_addr + kABfBytes;
+                const uint32_t a_addr = plan.a_bf(s), b_addr = plan.w_bf(s);
 #pragma unroll
                 for (int kk = 0; kk < BK / 16; kk++) {
                     // K-major: 16 k = 32 bytes inside the 128-byte row; MN-major: 16 k = two 1024-byte atoms
-                    const uint64_t da = A_IS_KM ? make_smem_desc(a_addr + kk * 2048, 8192, 1024)
-                                                : make_smem_desc(a_addr + kk * 32, 16, 1024);
                     const uint64_t db = W_IS_NK ? make_smem_desc(b_addr + kk * 32, 16, 1024)
                                                 : make_smem_desc(b_addr + kk * 2048, 8192, 1024);
-                    tc_mma_bf16_pair(tmem_base, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+                    if (A_IS_KM) {
+                        tc_mma_bf16_pair(tmem_base, make_smem_desc(a_addr + kk * 2048, 8192, 1024), db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+                    } else {
+                        // A from tensor memory: stage s, 16 k = 8 columns
+                        tc_mma_bf16_pair_a_tmem(tmem_base, tmem_base + kTmemColsAcc + (uint32_t)(s * kTmemAStageCols + kk * 8), db, idesc,
+                                                (kb > 0 || kk > 0) ? 1u : 0u);
+                    }
                 }
                 tc_commit_pair(bar_bf_empty(s));  // frees this operand stage in both CTAs once the MMAs have read it
             }
@@ -490,16 +590,41 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             ok = mbar_wait(bar_u8_full(s8), r8 & 1, abort_flag, p.status, 3);
             if (ok && rb > 0) ok = mbar_wait(bar_bf_empty(sb), (rb - 1) & 1, abort_flag, p.status, 4);
             if (!ok) break;
-            const uint32_t a8 = base + SmemLayout::u8 + s8 * (kA8Bytes + kB8Bytes), b8 = a8 + kA8Bytes;
-            const uint32_t abf = base + SmemLayout::bf + sb * (kABfBytes + kBBfBytes), bbf = abf + kABfBytes;
-            uint2 va[kChunksPerThread], vw[kChunksPerThread];
-            load_tile_chunks<A_IS_KM>(a8, dt, va);
-            load_tile_chunks<!W_IS_NK>(b8, dt, vw);
-            __syncwarp();  // every lane's reads of the byte stage are done: the producer may refill it during the decode
-            if (lane == 0) mbar_arrive(bar_u8_empty(s8));
-            decode_tile_chunks<A_IS_KM>(va, abf, dt, lut);
-            decode_tile_chunks<!W_IS_NK>(vw, bbf, dt, lut);
+            const uint32_t a8 = plan.a_u8(s8), b8 = plan.w_u8(s8);
+            const uint32_t abf = plan.a_bf(sb), bbf = plan.w_bf(sb);
+            uint2 vw[kChunksPerThread];
+            if (A_IS_KM) {
+                uint2 va[kChunksPerThread];
+                load_tile_chunks<true>(a8, dt, va);
+                load_tile_chunks<!W_IS_NK>(b8, dt, vw);
+                __syncwarp();  // every lane's reads of the byte stage are done: the producer may refill it during the decode
+                if (lane == 0) mbar_arrive(bar_u8_empty(s8));
+                decode_tile_chunks<true, kLutShift>(va, abf, dt, lut);
+            } else {
+                // A [M,K]: this thread owns row (its warp's quarter of the 128 tensor-memory lanes) * 32 + lane.  The byte
+                // tile arrives with the 64-byte TMA swizzle (16-byte chunk j of row r sits at chunk j ^ ((r >> 1) & 3)), so
+                // the lanes of a warp, 64 bytes apart, read their chunk j from different banks.
+                const int quarter = warp & 3, r = quarter * 32 + lane;
+                const uint32_t a_row = a8 + (uint32_t)r * BK, sw = (uint32_t)(r >> 1) & 3u;
+                uint4 va[BK / 16];
+#pragma unroll
+                for (int j = 0; j < BK / 16; j++) va[j] = lds_v4(a_row + (((uint32_t)j ^ sw) << 4));
+                load_tile_chunks<!W_IS_NK>(b8, dt, vw);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_u8_empty(s8));
+                uint32_t o[BK / 2];  // 64 BF16 of this row, two per column
+#pragma unroll
+                for (int j = 0; j < BK / 16; j++) {
+                    const uint4 lo = decode8<kLutShift>(make_uint2(va[j].x, va[j].y), lut), hi = decode8<kLutShift>(make_uint2(va[j].z, va[j].w), lut);
+                    o[8 * j + 0] = lo.x; o[8 * j + 1] = lo.y; o[8 * j + 2] = lo.z; o[8 * j + 3] = lo.w;
+                    o[8 * j + 4] = hi.x; o[8 * j + 5] = hi.y; o[8 * j + 6] = hi.z; o[8 * j + 7] = hi.w;
+                }
+                tmem_st_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + kTmemColsAcc + (uint32_t)(sb * kTmemAStageCols), o);
+            }
+            decode_tile_chunks<!W_IS_NK, kLutShift>(vw, bbf, dt, lut);
+            if (!A_IS_KM) tmem_st_wait();  // the row is in tensor memory
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // make the stores visible to the tensor core
+            tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(bar_bf_full(sb), 0));  // the leader's MMAs read both CTAs' operands
         }
@@ -698,7 +823,7 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
 #pragma unroll
             for (int i = 0; i < kNarrowMaxM * (BK / 8) / kGroupThreads; i++) {
                 const int q = i * kGroupThreads + dt, row = q >> 3, jc = q & 7;
-                if (q < act_chunks) sts_v4(abf + (row >> 3) * 1024 + (row & 7) * 128 + ((jc ^ (row & 7)) << 4), decode8(va[i], lut));
+                if (q < act_chunks) sts_v4(abf + (row >> 3) * 1024 + (row & 7) * 128 + ((jc ^ (row & 7)) << 4), decode8<7>(va[i], lut));
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
@@ -1042,7 +1167,8 @@ struct MapKey {
     const void* ptr;
     uint64_t inner, rows, count, ld;  // ld: row pitch in elements (2-D) or distance between stacked matrices (3-D)
     uint32_t box_inner, box_rows;
-    uint32_t kind;                    // 0: bytes, 2-D; 1: BF16, 2-D, 128-byte swizzle; 2: BF16, 3-D stack, 128-byte swizzle
+    uint32_t kind;                    // 0: bytes, 2-D; 1: BF16, 2-D, 128-byte swizzle; 2: BF16, 3-D stack, 128-byte swizzle;
+                                      // 3: bytes, 2-D, 64-byte swizzle
     uint32_t pad;
 };
 LruCache<MapKey, CUtensorMap, 64> g_map_cache;
@@ -1051,7 +1177,7 @@ bool encode_map(const MapKey& k, CUtensorMap* map)
 {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
-    const bool bf16 = k.kind != 0;
+    const bool bf16 = k.kind == 1 || k.kind == 2;
     if (k.kind == 2) {
         cuuint64_t dims[3] = {k.inner, k.rows, k.count};
         cuuint64_t strides[2] = {k.inner * 2u, (k.count > 1 ? k.ld : k.inner * k.rows) * 2u};
@@ -1066,19 +1192,20 @@ bool encode_map(const MapKey& k, CUtensorMap* map)
     cuuint32_t box[2] = {k.box_inner, k.box_rows};
     cuuint32_t estr[2] = {1, 1};
     return fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(k.ptr), dims,
-              strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, bf16 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+              strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+              bf16 ? CU_TENSOR_MAP_SWIZZLE_128B : (k.kind == 3 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE),
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // 2-D tensor [rows][ld elements] with a box of box_inner x box_rows elements, zero fill out of bounds.
 // bf16 = false: bytes, no swizzle.  bf16 = true: 16-bit elements, 128-byte swizzle (box_inner must be 64).
 bool make_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t rows, uint64_t ld, uint32_t box_inner, uint32_t box_rows,
-              bool bf16 = false)
+              bool bf16 = false, bool bytes_swizzle64 = false)
 {
     MapKey k;
     std::memset(&k, 0, sizeof k);
     k.ptr = ptr; k.inner = inner; k.rows = rows; k.count = 1; k.ld = ld; k.box_inner = box_inner; k.box_rows = box_rows;
-    k.kind = bf16 ? 1u : 0u;
+    k.kind = bf16 ? 1u : (bytes_swizzle64 ? 3u : 0u);
     return g_map_cache.lookup_or_make(k, map, encode_map);
 }
 
@@ -1109,8 +1236,8 @@ bool gemm_kernels_ready(int dev, int* sm_count_out)
         const void* fused[4] = {(const void*)hif8_gemm_kernel<false, false>, (const void*)hif8_gemm_kernel<false, true>,
                                 (const void*)hif8_gemm_kernel<true, false>, (const void*)hif8_gemm_kernel<true, true>};
         const void* pair[2] = {(const void*)bf16_gemm_pair_kernel<false>, (const void*)bf16_gemm_pair_kernel<true>};
-        for (int i = 0; i < 4 && out->rc == cudaSuccess; i++)
-            out->rc = cudaFuncSetAttribute(fused[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        for (int i = 0; i < 4 && out->rc == cudaSuccess; i++)  // [M,K] activations (the first two): the wide-table plan
+            out->rc = cudaFuncSetAttribute(fused[i], cudaFuncAttributeMaxDynamicSharedMemorySize, i < 2 ? kSmemBytesWide : kSmemBytes);
         for (int i = 0; i < 2 && out->rc == cudaSuccess; i++)
             out->rc = cudaFuncSetAttribute(pair[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
         if (out->rc == cudaSuccess)
@@ -1210,8 +1337,9 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t
     if (major != 10) return HIF8_ERR_CUDA;
 
     CUtensorMap map_a, map_w;
+    // ([M,K] activations: 64-byte rows with the 64-byte swizzle, read row-wise by the decode warps of the fused kernel)
     const bool ok_a = a_is_km ? make_map(&map_a, Aq, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BM, BK)
-                              : make_map(&map_a, Aq, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BK, BM);
+                              : make_map(&map_a, Aq, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BK, BM, false, true);
     if (!ok_a) return HIF8_ERR_CUDA;
     // byte tiles of one CTA of a pair: 128 rows of A, 128 of the 256 columns of W
     const bool ok_w = w_is_nk ? make_map(&map_w, Wq, (uint64_t)K, (uint64_t)N, (uint64_t)ldw, BK, BN / 2)
@@ -1291,7 +1419,7 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(2u * (unsigned)tiles2);
     cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.dynamicSmemBytes = a_is_km ? kSmemBytes : kSmemBytesWide;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
