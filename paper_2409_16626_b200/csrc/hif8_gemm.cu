@@ -52,6 +52,20 @@ constexpr int kEpiWarps = 4, kDecodeWarps = 16;
 // more than one phase ahead of the barrier, which a parity wait could not tell apart).
 constexpr int kDecodeGroups = 4, kGroupWarps = kDecodeWarps / kDecodeGroups, kGroupThreads = kGroupWarps * 32;
 static_assert(kStages8 == kDecodeGroups && kStagesBf == kDecodeGroups, "group g owns byte stage g and operand stage g");
+// With A decoded into tensor memory the shared memory freed by the A operand tiles can hold either a deeper byte ring
+// (8 stages, table with 128-byte rows) or the 64 KiB table whose addresses cost one instruction (4 stages).  Measured at
+// 8192 x 28672 x 8192: 4.84 ms against 4.71 ms -- the TMA latency is already covered by four stages, so the wide table is
+// the default.
+#ifndef HIF8_FUSED_BYTE_STAGES
+#define HIF8_FUSED_BYTE_STAGES 4
+#endif
+#ifndef HIF8_FUSED_WIDE_LUT
+#define HIF8_FUSED_WIDE_LUT 1
+#endif
+constexpr int kStages8Deep = HIF8_FUSED_BYTE_STAGES, kMaxStages8 = kStages8Deep > kStages8 ? kStages8Deep : kStages8;
+constexpr bool kWideLut = HIF8_FUSED_WIDE_LUT != 0;
+static_assert(kStages8Deep % kDecodeGroups == 0, "a byte stage is always read by the same group");
+static_assert(!kWideLut || kStages8Deep == 4, "the 64 KiB table leaves room for four byte stages only");
 constexpr int kThreads = (kEpiWarps + 2 + kDecodeWarps) * 32;  // 704
 constexpr int kTmaWarp = 4, kMmaWarp = 5, kFirstDecodeWarp = 6;
 // per CTA of a pair: 128 rows of A and 128 of the 256 columns of W
@@ -68,7 +82,7 @@ struct SmemLayout {
     static constexpr uint32_t u8 = bf + kStagesBf * (kABfBytes + kBBfBytes);           // 96 KiB
     static constexpr uint32_t lut = u8 + kStages8 * (kA8Bytes + kB8Bytes);             // + 64 KiB
     static constexpr uint32_t bars = lut + 256 * 32 * 4;                                // lane-replicated table, 32 KiB
-    static constexpr uint32_t n_bars = 2 * kStages8 + 2 * kStagesBf + 1;
+    static constexpr uint32_t n_bars = 2 * kMaxStages8 + 2 * kStagesBf + 1;
     static constexpr uint32_t tmem_slot = bars + n_bars * 8;
     static constexpr uint32_t abort_flag = tmem_slot + 4;
     static constexpr uint32_t total = abort_flag + 4;
@@ -431,7 +445,7 @@ __device__ __forceinline__ void decode_tile_chunks(const uint2 (&v)[kChunksPerTh
 // A given as [M,K] (decoded into tensor memory): no A operand tiles, and the lookup table has rows of 256 bytes and starts on
 // a 64 KiB boundary of the shared window (see decode8).  Everything else is dealt out in 16 KiB slots around the table: as
 // many as fit in front of it, the rest behind it.  Slots 0-3: W operand stages, slots 4-7: byte stages (A 8 KiB + W 8 KiB).
-constexpr uint32_t kSlotBytes = 16384, kLutBytesWide = 65536, kFusedSlots = kStagesBf + kStages8;
+constexpr uint32_t kSlotBytes = 16384, kLutBytesWide = 65536, kLutBytesNarrow = 256 * 32 * 4, kFusedSlots = kStagesBf + kStages8Deep;
 static_assert(kBBfBytes == kSlotBytes && kA8Bytes + kB8Bytes == kSlotBytes, "one stage per slot");
 constexpr uint32_t kSmemBytesWide = 227 * 1024;  // the whole opt-in maximum; the kernel checks that its plan fits
 
@@ -446,6 +460,10 @@ struct FusedSmem {
         base = (raw + 1023u) & ~1023u;
         if (A_IS_KM) {
             lut = base + SmemLayout::lut; bars = base + SmemLayout::bars; behind = 0; n_front = 0; end = base + SmemLayout::total;
+        } else if (!kWideLut) {
+            // table with rows of 128 bytes: no alignment to honour, everything in a row: slots, table, barriers
+            n_front = (int)kFusedSlots; behind = 0;
+            lut = base + kFusedSlots * kSlotBytes; bars = lut + kLutBytesNarrow; end = bars + 256u;
         } else {
             lut = (base + kLutBytesWide - 1) & ~(kLutBytesWide - 1);
             const uint32_t front = lut - base;
@@ -471,7 +489,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const GemmParams p)
 {
     extern __shared__ unsigned char smem_raw[];
-    constexpr int kLutShift = A_IS_KM ? 7 : 8;
+    constexpr int kLutShift = (A_IS_KM || !kWideLut) ? 7 : 8;
+    constexpr int kS8 = A_IS_KM ? kStages8 : kStages8Deep;  // depth of the byte ring
     const FusedSmem<A_IS_KM> plan(smem_u32(smem_raw));
     const uint32_t base = plan.base;
     unsigned char* sm = smem_raw - smem_u32(smem_raw);  // generic pointer of shared-window address 0
@@ -489,10 +508,10 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 
     const uint32_t bars = plan.bars;
     auto bar_u8_full = [&](int s) { return bars + 8u * s; };                                   // per CTA
-    auto bar_u8_empty = [&](int s) { return bars + 8u * (kStages8 + s); };                     // per CTA
-    auto bar_bf_full = [&](int s) { return bars + 8u * (2 * kStages8 + s); };                  // leader: both CTAs' decode warps
-    auto bar_bf_empty = [&](int s) { return bars + 8u * (2 * kStages8 + kStagesBf + s); };     // per CTA, leader's commits
-    const uint32_t bar_acc_full = bars + 8u * (2 * kStages8 + 2 * kStagesBf);                  // per CTA, leader's commit
+    auto bar_u8_empty = [&](int s) { return bars + 8u * (kMaxStages8 + s); };                     // per CTA
+    auto bar_bf_full = [&](int s) { return bars + 8u * (2 * kMaxStages8 + s); };                  // leader: both CTAs' decode warps
+    auto bar_bf_empty = [&](int s) { return bars + 8u * (2 * kMaxStages8 + kStagesBf + s); };     // per CTA, leader's commits
+    const uint32_t bar_acc_full = bars + 8u * (2 * kMaxStages8 + 2 * kStagesBf);                  // per CTA, leader's commit
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + plan.abort_flag());
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + plan.tmem_slot());
     uint32_t* lut_all = reinterpret_cast<uint32_t*>(sm + plan.lut);
@@ -508,7 +527,7 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     for (int i = threadIdx.x; i < 256 * 32; i += kThreads)  // entry (code i / 32, lane i % 32): rows of 1 << kLutShift bytes
         lut_all[((i >> 5) << (kLutShift - 2)) + (i & 31)] = hif8_to_bf16_bits(i >> 5);
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages8; s++) { mbar_init(bar_u8_full(s), 1); mbar_init(bar_u8_empty(s), kGroupWarps); }
+        for (int s = 0; s < kS8; s++) { mbar_init(bar_u8_full(s), 1); mbar_init(bar_u8_empty(s), kGroupWarps); }
         for (int s = 0; s < kStagesBf; s++) { mbar_init(bar_bf_full(s), 2 * kGroupWarps); mbar_init(bar_bf_empty(s), 1); }
         mbar_init(bar_acc_full, 1);
         *abort_flag = 0;
@@ -530,7 +549,7 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         if (lane == 0) {
             int issued = 0;
             for (int kb = 0; kb < num_kb; kb++) {
-                const int s = kb % kStages8, round = kb / kStages8;
+                const int s = kb % kS8, round = kb / kS8;
                 if (round > 0 && !mbar_wait(bar_u8_empty(s), (round - 1) & 1, abort_flag, p.status, 1)) break;
                 if (*abort_flag) break;
                 const uint32_t dst_a = plan.a_u8(s), dst_b = plan.w_u8(s);
@@ -543,10 +562,10 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             }
             if (*abort_flag) {
                 // let the copies already issued land before this CTA's shared memory goes away
-                for (int kb = max(0, issued - kStages8); kb < issued; kb++) {
-                    const int s = kb % kStages8;
+                for (int kb = max(0, issued - kS8); kb < issued; kb++) {
+                    const int s = kb % kS8;
                     const unsigned long long t0 = global_ns();
-                    while (!mbar_try_wait(bar_u8_full(s), (kb / kStages8) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+                    while (!mbar_try_wait(bar_u8_full(s), (kb / kS8) & 1) && global_ns() - t0 < kWaitLimitNs) {}
                 }
             }
         }
@@ -586,7 +605,7 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         const int dt = threadIdx.x - (kFirstDecodeWarp + group * kGroupWarps) * 32;  // 0..kGroupThreads-1
         bool ok = true;
         for (int kb = group; kb < num_kb && ok; kb += kDecodeGroups) {
-            const int s8 = group, r8 = kb / kStages8, sb = group, rb = kb / kStagesBf;
+            const int s8 = kb % kS8, r8 = kb / kS8, sb = group, rb = kb / kStagesBf;
             ok = mbar_wait(bar_u8_full(s8), r8 & 1, abort_flag, p.status, 3);
             if (ok && rb > 0) ok = mbar_wait(bar_bf_empty(sb), (rb - 1) & 1, abort_flag, p.status, 4);
             if (!ok) break;
