@@ -28,6 +28,7 @@ struct TrParams {
     const int* d_scale_exp;
     unsigned flags;
     unsigned long long seed;
+    int rows_on_x;  // grid x counts row tiles (only for more than 65535 row tiles); else x counts column strips
 };
 
 constexpr int kTileRows = 128;
@@ -53,11 +54,15 @@ __global__ void __launch_bounds__(kThreads, MODE == HIF8_RND_SR ? 4 : 6) encode_
     const long long nvc = p.cols / PV;                        // vectors per source row
     const long long strips = (nvc + kTileVecs - 1) / kTileVecs;
     const int cv = threadIdx.x % kTileVecs, rq = threadIdx.x / kTileVecs;
-    const long long r0 = (long long)blockIdx.x * kTileRows;
+    // x = strip of source columns (fastest), y = tile of source rows: blocks that run together read neighbouring
+    // 128-byte pieces of the same source rows, i.e. whole lines of the row-major source
+    const unsigned bx = p.rows_on_x ? blockIdx.x : blockIdx.y, by = p.rows_on_x ? blockIdx.y : blockIdx.x;
+    const unsigned gy = p.rows_on_x ? gridDim.y : gridDim.x;
+    const long long r0 = (long long)bx * kTileRows;
     const bool rows_full = r0 + kTileRows <= p.rows;
     uint32_t* const my_words = tile + cv * PV * kTileWords + (((rq >> 2) ^ cv) << 2) + (rq & 3);
 
-    for (long long tc = blockIdx.y; tc < strips; tc += gridDim.y) {
+    for (long long tc = by; tc < strips; tc += gy) {
         const long long v0 = tc * kTileVecs, vcol = v0 + cv;
         const bool full = rows_full && v0 + kTileVecs <= nvc;
         const uint4* sp = reinterpret_cast<const uint4*>(p.src) + (r0 + rq * 4) * nvc + vcol;
@@ -133,7 +138,7 @@ __global__ void __launch_bounds__(kThreads, MODE == HIF8_RND_SR ? 4 : 6) encode_
             // rows is a multiple of 16 on this path: a segment is all in or all out
             if (full || (v0 * PV + c < p.cols && r0 + seg * 16 < p.rows)) __stcs(reinterpret_cast<uint4*>(dp + (long long)i * (kThreads / kSegs) * p.rows), q);
         }
-        if (tc + gridDim.y < strips) __syncthreads();  // (block-uniform) the tile is read out before the next one is stored
+        if (tc + gy < strips) __syncthreads();  // (block-uniform) the tile is read out before the next one is stored
     }
 }
 
@@ -217,8 +222,10 @@ int launch(const TrParams& p, bool vec, int sms, cudaStream_t st)
         per_block = per_block < 1 ? 1 : per_block > 4 ? 4 : per_block;
         long long gy = (strips + per_block - 1) / per_block;
         if (gy > 65535) gy = 65535;
-        const dim3 grid((unsigned)row_tiles, (unsigned)gy);
-        encode_transpose_kernel<SRC, MODE><<<grid, kThreads, 0, st>>>(p);
+        TrParams q = p;
+        q.rows_on_x = row_tiles > 65535 ? 1 : 0;
+        const dim3 grid = q.rows_on_x ? dim3((unsigned)row_tiles, (unsigned)gy) : dim3((unsigned)gy, (unsigned)row_tiles);
+        encode_transpose_kernel<SRC, MODE><<<grid, kThreads, 0, st>>>(q);
     } else {
         const unsigned long long n = (unsigned long long)p.rows * (unsigned long long)p.cols;
         const unsigned long long need = (n + kThreads - 1) / kThreads, cap = (unsigned long long)sms * 32;
