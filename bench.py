@@ -307,6 +307,13 @@ def extra_results(H, torch, hbm_peak, tf_peak, peak_kind):
     res["decode"] = hbm(st, 5 * n)
     row("C4a_loguniform_f32_2^28_decode", res["decode"], "hbm")
     out["loguniform_f32_2^28"] = {"bytes_per_element": 5, "calls": res, "peak": hbm_peak, "peak_kind": f"of {peak_kind}"}
+    # the exhaustive FP32 sweep generates its inputs in the kernel: a write-only stream, 1 B/element (one slice of 2^28 patterns)
+    sweep = {}
+    for name, mode in (("TA", H.RND_TA), ("HR", H.RND_HR)):
+        st = timed(lambda r: H.hif8_encode_f32_patterns((r & 15) << 28, codes, n, 0, mode), 10)
+        sweep[name] = hbm(st, n)
+        row(f"C4b_f32_pattern_sweep_2^28_write_only_{name}", sweep[name], "hbm")
+    out["f32_pattern_sweep_2^28"] = {"bytes_per_element": 1, "modes": sweep, "peak": hbm_peak, "peak_kind": f"of {peak_kind}"}
     del bits, codes, back
 
     # ---- GEMM: A BF16 8192x8192 N(0,1), W BF16 8192x28672 N(0,0.02), per-tensor scaled to HiF8, C = dec(A) dec(W)

@@ -83,6 +83,16 @@ int hif8_encode(const void* src, int src_dtype, uint8_t* dst, size_t n, int scal
                 unsigned flags, uint64_t seed, hif8_stream_t stream);
 
 /*
+ * hif8_encode of a source that is generated instead of read: element i is the FP32 value whose encoding is
+ * first_pattern + i (modulo 2^32), i = 0 .. n-1, n <= 2^32.  This is the exhaustive sweep over FP32 inputs (every
+ * exponent including the denormal extension of Eq. 2, underflow to the single zero, overflow, Inf and NaN patterns of
+ * Section 2.1 / Table 4) without a 4-byte-per-element source tensor: the call only writes, one byte per element.
+ * HIF8_RND_SR draws the word of index i.  Arguments and errors otherwise as hif8_encode.
+ */
+int hif8_encode_f32_patterns(uint32_t first_pattern, uint8_t* dst, size_t n, int scale_exp, int rnd, unsigned flags,
+                             uint64_t seed, hif8_stream_t stream);
+
+/*
  * HiF8 bytes -> high-precision tensor (Eq. 1, Eq. 2, Table 4 specials), with the descale of
  * Algorithm 1 ("Restore"):   dst[i] = value(src[i]) * 2^(-scale_exp)
  * rounded to nearest-even into `dst_dtype` when not representable (only possible at the far ends of the

@@ -22,7 +22,7 @@ LIB_PATH = os.path.join(_HERE, "libhif8.so")
 EXPORTS = ["hif8_encode", "hif8_decode", "hif8_amax", "hif8_amax_scale_encode", "hif8_fake_quant", "hif8_gemm", "hif8_gemm_status", "hif8_pts_search", "hif8_pts_workspace_bytes",
            "hif8_pts_status", "hif8_selftest_wait_timeout", "hif8_channel_amax_scale_encode", "hif8_gemm_channel_scaled",
            "hif8_scale_state_init", "hif8_delayed_scale_encode", "hif8_gemm_ex", "hif8_encode_transpose", "hif8_als_state_init", "hif8_als_update", "hif8_check_finite", "hif8_encode_from_amax",
-           "hif8_amax_scale_encode_static", "hif8_last_device_status", "hif8_selftest_host_caches", "hif8_workspace_bytes", "hif8_status_string", "hif8_launch_count"]
+           "hif8_amax_scale_encode_static", "hif8_encode_f32_patterns", "hif8_last_device_status", "hif8_selftest_host_caches", "hif8_workspace_bytes", "hif8_status_string", "hif8_launch_count"]
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2409_16626_b200.build` (needs nvcc)")
@@ -31,6 +31,8 @@ lib = C.CDLL(LIB_PATH)
 _vp, _sz, _i, _u, _u64, _i64 = C.c_void_p, C.c_size_t, C.c_int, C.c_uint, C.c_uint64, C.c_int64
 lib.hif8_encode.argtypes = [_vp, _i, _vp, _sz, _i, _i, _u, _u64, _vp]
 lib.hif8_decode.argtypes = [_vp, _vp, _i, _sz, _i, _vp]
+lib.hif8_encode_f32_patterns.argtypes = [C.c_uint32, _vp, _sz, _i, _i, _u, _u64, _vp]
+lib.hif8_encode_f32_patterns.restype = _i
 lib.hif8_amax_scale_encode.argtypes = [_vp, _i, _vp, _sz, _i, _i, _u, _u64, _vp, _vp, _vp, _vp, _vp, _sz, _vp]
 lib.hif8_amax.argtypes = [_vp, _i, _sz, _vp, _vp, _sz, _vp]
 lib.hif8_amax.restype = _i
@@ -123,6 +125,11 @@ def hif8_launch_count():
 
 def hif8_encode(src, src_dtype, dst, n, scale_exp=0, rnd=RND_TA, flags=0, seed=0, stream=None, check=True):
     return _check(lib.hif8_encode(_ptr(src), src_dtype, _ptr(dst), n, scale_exp, rnd, flags, seed, _stream(stream)), check)
+
+
+def hif8_encode_f32_patterns(first_pattern, dst, n, scale_exp=0, rnd=RND_TA, flags=0, seed=0, stream=None, check=True):
+    return _check(lib.hif8_encode_f32_patterns(int(first_pattern) & 0xFFFFFFFF, _ptr(dst), n, scale_exp, rnd, flags, seed,
+                                               _stream(stream)), check)
 
 
 def hif8_decode(src, dst, dst_dtype, n, scale_exp=0, stream=None, check=True):

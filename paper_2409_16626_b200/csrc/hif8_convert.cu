@@ -39,7 +39,8 @@ namespace {
 
 // One group of kUnroll vectors per thread starting at vector index `base`.  FULL: the whole group lies inside the
 // tensor, so no bounds are checked.
-template <int SRC, int MODE, bool FQ, bool AMAX, bool FULL>
+// PATTERN (FP32 only): the source is not read; element i is the FP32 value with encoding p.pattern_first + i.
+template <int SRC, int MODE, bool FQ, bool AMAX, bool FULL, bool PATTERN = false>
 __device__ __forceinline__ void convert_group(const ConvParams& p, const SmemTables& sm, unsigned long long base, unsigned long long n_vec,
                                               float scale, float d1, float d2, uint32_t k0, uint32_t k1, float& amax)
 {
@@ -49,7 +50,11 @@ __device__ __forceinline__ void convert_group(const ConvParams& p, const SmemTab
 #pragma unroll
     for (int j = 0; j < kUnroll; j++) {
         unsigned long long u = base + (unsigned long long)j * kThreads + threadIdx.x;
-        if (FULL || u < n_vec) v[j] = __ldcs(src + u); else v[j] = make_uint4(0, 0, 0, 0);
+        if (PATTERN) {
+            const uint32_t b = p.pattern_first + (uint32_t)(u * 4u);
+            v[j] = make_uint4(b, b + 1u, b + 2u, b + 3u);
+        } else if (FULL || u < n_vec) v[j] = __ldcs(src + u);
+        else v[j] = make_uint4(0, 0, 0, 0);
     }
 #pragma unroll
     for (int j = 0; j < kUnroll; j++) {
@@ -130,9 +135,10 @@ __device__ __forceinline__ void convert_group(const ConvParams& p, const SmemTab
 // Encode / fake-quant kernel.  FQ = false: bytes out.  FQ = true: dequantized values in the source format.
 // AMAX = true: also reduce amax of the source into p.amax_accum[0]; the last block publishes it.
 // ------------------------------------------------------------------------------------------------
-template <int SRC, int MODE, bool FQ, bool AMAX>
+template <int SRC, int MODE, bool FQ, bool AMAX, bool PATTERN = false>
 __global__ void __launch_bounds__(kThreads) convert_kernel(const ConvParams p, unsigned long long n_vec)
 {
+    static_assert(!PATTERN || (SRC == HIF8_F32 && !FQ && !AMAX), "generated sources are FP32 patterns, encode only");
     __shared__ SmemTables sm;
     pdl_launch_dependents();
     constexpr bool kPair16 = SRC == HIF8_BF16 && (MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR) && !FQ;
@@ -154,9 +160,9 @@ __global__ void __launch_bounds__(kThreads) convert_kernel(const ConvParams p, u
     for (unsigned long long g = blockIdx.x; g < n_groups; g += gridDim.x) {
         const unsigned long long base = (p.reverse ? n_groups - 1 - g : g) * kGroupVecs;
         if (base + kGroupVecs <= n_vec)
-            convert_group<SRC, MODE, FQ, AMAX, true>(p, sm, base, n_vec, scale, d1, d2, k0, k1, amax);
+            convert_group<SRC, MODE, FQ, AMAX, true, PATTERN>(p, sm, base, n_vec, scale, d1, d2, k0, k1, amax);
         else
-            convert_group<SRC, MODE, FQ, AMAX, false>(p, sm, base, n_vec, scale, d1, d2, k0, k1, amax);
+            convert_group<SRC, MODE, FQ, AMAX, false, PATTERN>(p, sm, base, n_vec, scale, d1, d2, k0, k1, amax);
     }
     // elements not covered by whole vectors (tail, or everything when the pointers are not 16-byte aligned)
     {
@@ -164,7 +170,8 @@ __global__ void __launch_bounds__(kThreads) convert_kernel(const ConvParams p, u
         const unsigned long long tid = (unsigned long long)blockIdx.x * kThreads + threadIdx.x;
         for (unsigned long long i = first + tid; i < p.n; i += (unsigned long long)gridDim.x * kThreads) {
             float x; uint32_t raw;
-            load_scalar<SRC>(p.src, i, x, raw);
+            if (PATTERN) { raw = p.pattern_first + (uint32_t)i; x = __uint_as_float(raw); }
+            else load_scalar<SRC>(p.src, i, x, raw);
             if (AMAX) amax = amax_step(amax, x);
             uint32_t word = 0;
             if (MODE == HIF8_RND_SR) {
@@ -676,6 +683,33 @@ int hif8_encode(const void* src, int src_dtype, uint8_t* dst, size_t n, int scal
     size_t out_align = src_dtype == HIF8_F32 ? 4 : 8;
     bool vec_ok = aligned16(src) && (reinterpret_cast<uintptr_t>(dst) % out_align) == 0;
     return dispatch_convert<false, false>(src_dtype, rnd, p, vec_ok, sms, (cudaStream_t)stream);
+}
+
+int hif8_encode_f32_patterns(uint32_t first_pattern, uint8_t* dst, size_t n, int scale_exp, int rnd, unsigned flags,
+                             uint64_t seed, hif8_stream_t stream)
+{
+    int rc = check_common(HIF8_F32, rnd, flags);
+    if (rc) return rc;
+    if (scale_exp < -126 || scale_exp > 126) return HIF8_ERR_SCALE_RANGE;
+    if (n > ((size_t)1 << 32)) return HIF8_ERR_SHAPE;
+    if (n == 0) return HIF8_OK;
+    if (!dst) return HIF8_ERR_NULL;
+    int sms; rc = device_info(&sms);
+    if (rc) return rc;
+    ConvParams p{};
+    p.dst = dst; p.n = n; p.scale_exp = scale_exp; p.flags = flags; p.seed = seed; p.pattern_first = first_pattern;
+    const unsigned long long n_vec = (reinterpret_cast<uintptr_t>(dst) & 3u) ? 0 : n / 4;
+    const unsigned grid = grid_for(n_vec, n, sms, kUnroll, kGroupsConvert);
+    cudaStream_t st = (cudaStream_t)stream;
+    switch (rnd) {
+        case HIF8_RND_TA: launch_pdl(convert_kernel<HIF8_F32, HIF8_RND_TA, false, false, true>, grid, st, p, n_vec); break;
+        case HIF8_RND_HR: launch_pdl(convert_kernel<HIF8_F32, HIF8_RND_HR, false, false, true>, grid, st, p, n_vec); break;
+        case HIF8_RND_SSR: launch_pdl(convert_kernel<HIF8_F32, HIF8_RND_SSR, false, false, true>, grid, st, p, n_vec); break;
+        case HIF8_RND_TE: launch_pdl(convert_kernel<HIF8_F32, HIF8_RND_TE, false, false, true>, grid, st, p, n_vec); break;
+        default: launch_pdl(convert_kernel<HIF8_F32, HIF8_RND_SR, false, false, true>, grid, st, p, n_vec); break;
+    }
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
 }
 
 int hif8_decode(const uint8_t* src, void* dst, int dst_dtype, size_t n, int scale_exp, hif8_stream_t stream)

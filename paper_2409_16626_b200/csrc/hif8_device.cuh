@@ -196,6 +196,7 @@ struct ConvParams {
     int* d_scale_exp_out;
     float* d_scale_out;
     void* scale_state;            // delayed scaling: ScaleState that the last block of an amax-reducing pass advances
+    uint32_t pattern_first;       // PATTERN kernels only: element i is the FP32 value whose encoding is pattern_first + i
     int reverse;                  // walk the tensor from its end: set for the second pass of just-in-time scaling, so that
                                   // the lines the amax pass read last (still in L2) are the ones re-read first
 };

@@ -38,6 +38,10 @@ def test_argument_errors_before_any_launch():
     assert H.hif8_encode(0, H.F32, 0, 16, flags=8, stream=0, check=False) == 4
     assert H.hif8_encode(0, H.F32, 0, 16, scale_exp=127, stream=0, check=False) == 5
     assert H.hif8_encode(0, H.F32, 0, 0, stream=0, check=False) == 0         # empty tensor is fine
+    assert H.hif8_encode_f32_patterns(0, 0, 16, rnd=9, stream=0, check=False) == 3
+    assert H.hif8_encode_f32_patterns(0, 0, (1 << 32) + 1, stream=0, check=False) == 6
+    assert H.hif8_encode_f32_patterns(0, 0, 16, stream=0, check=False) == 1
+    assert H.hif8_encode_f32_patterns(0, 0, 0, stream=0, check=False) == 0
     assert H.hif8_decode(0, 0, 5, 16, stream=0, check=False) == 2
     assert H.hif8_decode(0, 0, H.F16, 16, scale_exp=-127, stream=0, check=False) == 5
     assert H.hif8_decode(0, 0, H.F16, 0, stream=0, check=False) == 0

@@ -344,3 +344,32 @@ def test_f32_full_sweep_other_modes(mode):
         if not np.array_equal(got, want):
             i = int(np.nonzero(got != want)[0][0])
             raise AssertionError(f"pattern {first + i:#010x}: got {got[i]:#x} want {want[i]:#x}")
+
+
+@pytest.mark.parametrize("mode", [H.RND_TA, H.RND_HR, H.RND_SSR, H.RND_TE, H.RND_SR])
+def test_generated_f32_patterns_sweep_with_both_options(mode):
+    # hif8_encode_f32_patterns: the whole FP32 range without a source tensor, here with SATURATE and NaN -> 0 switched on
+    # (Section 3: the two options), against the oracle; plus equality with hif8_encode on a slice, wrap-around of the
+    # pattern counter, an unaligned destination and a ragged length
+    n = 1 << 26
+    out = torch.empty(n, dtype=torch.uint8, device="cuda")
+    omode = {H.RND_TA: O.TA, H.RND_HR: O.HR, H.RND_SSR: O.SSR, H.RND_TE: O.TE, H.RND_SR: O.SR}[mode]
+    for chunk in range(64):
+        first = chunk << 26
+        H.hif8_encode_f32_patterns(first, out, n, 0, mode, 3, 91)
+        torch.cuda.synchronize()
+        want = O.encode_f32_range(first, n, 0, omode, 3, 91, quick=True)
+        got = out.cpu().numpy()
+        if not np.array_equal(got, want):
+            i = int(np.nonzero(got != want)[0][0])
+            raise AssertionError(f"pattern {first + i:#010x}: got {got[i]:#x} want {want[i]:#x}")
+    first, m = 0xFFFFFF00, 1003                              # wraps through 0xFFFFFFFF -> 0, scaled, ragged, misaligned
+    raw, ptr, readback = dev_empty(m, np.uint8, offset_bytes=3)
+    H.hif8_encode_f32_patterns(first, ptr, m, 5, mode, 0, 7)
+    bits = ((np.arange(m, dtype=np.uint64) + first) & 0xFFFFFFFF).astype(np.uint32)
+    src = to_dev(bits)
+    ref = torch.empty(m, dtype=torch.uint8, device="cuda")
+    H.hif8_encode(src, H.F32, ref, m, 5, mode, 0, 7)
+    torch.cuda.synchronize()
+    assert np.array_equal(readback(), ref.cpu().numpy())
+    assert np.array_equal(readback(), O.encode(bits, O.F32, 5, omode, 0, seed=7, quick=True))
