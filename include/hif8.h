@@ -258,7 +258,8 @@ int hif8_fake_quant(const void* src, void* dst, int dtype, size_t n, int use_ama
  * multiple of 16 (HIF8_ERR_SHAPE).  NaN / Inf codes propagate as in IEEE arithmetic.
  * workspace: at least hif8_workspace_bytes(HIF8_WS_GEMM, 0) = 256 bytes, 16-byte aligned; its first int is a device
  * status word that the call clears and the kernel sets if one of its bounded waits ever gives up (see
- * hif8_gemm_status).  With only that, the fused kernel decodes the HiF8 tiles of every CTA in shared memory.
+ * hif8_gemm_status).  With only that, the fused kernel decodes the HiF8 byte tiles of every CTA pair inside the
+ * tensor-core kernel (W into shared memory, an A given as [M,K] straight into tensor memory).
  * With hif8_workspace_bytes(HIF8_WS_GEMM, M*K + K*N) bytes, 256-byte aligned, and contiguous operands (lda = K,
  * ldw = row length of Wq), each operand byte is instead decoded once into the workspace (BF16, exact) and the
  * tensor-core kernel streams BF16 tiles: several times faster for compute-bound shapes, same results.
