@@ -232,8 +232,10 @@ constexpr uint32_t kRareMask = 1u;  // never a legitimate mask: legitimate ones 
 // one element, any input: value-level rounding through the scaled binary32 value.
 // MODE: round half away, round half to even, or (BF16 sources) the 2-bit simplified stochastic rounding SR2 / hybrid
 // rounding of Eq. 3.
+// MODE = standard stochastic rounding (BF16 sources): T16 is the 16-bit threshold of the element (Section 3.2: one is added
+// to the kept bits iff the discarded fraction, taken to 16 bits, is non-zero and at least T).
 template <int SRC, int MODE>
-__device__ __noinline__ uint32_t fq_rare(uint32_t raw, int se, unsigned flags)
+__device__ __noinline__ uint32_t fq_rare(uint32_t raw, int se, unsigned flags, uint32_t T16 = 0u)
 {
     const float x = __uint_as_float(SRC == HIF8_F32 ? raw : raw << 16);
     const float y = x * pow2f(se);
@@ -257,6 +259,18 @@ __device__ __noinline__ uint32_t fq_rare(uint32_t raw, int se, unsigned flags)
         else if (a < 0x34000000u) return 0u;                                               // < 2^-23: the single zero
         else if (E < -22) r = 0x34800000u;                                                 // [2^-23, 2^-22) -> 2^-22
         else { const uint32_t k = 23u - (uint32_t)mant_width(E); r = (a + (1u << (k - 1))) & (0xFFFFFFFFu << k); }
+    } else if (MODE == HIF8_RND_SR) {
+        if (a >= 0x47400000u) r = top;                                                     // >= 1.5 * 2^15
+        else if (E < -22) {                                                                // F = |y| / 2^-22, F16 = floor(2^16 F)
+            const uint32_t f16 = E < -38 ? 0u : (uint32_t)floorf(fabsf(y) * 274877906944.f);  // |y| * 2^38, exact: < 2^16
+            if (f16 == 0u || f16 < T16) return 0u;
+            r = 0x34800000u;
+        } else {
+            const uint32_t k = 23u - (uint32_t)mant_width(E);                              // >= 20: the low 16 bits of a are zero
+            const uint32_t f16 = (a & ((1u << k) - 1u)) >> (k - 16);
+            r = (a & (0xFFFFFFFFu << k)) + (((f16 != 0u && f16 >= T16) ? 1u : 0u) << k);
+            if (r >= 0x47400000u) r = top;
+        }
     } else {
         const uint32_t T2 = 2u * (raw & 1u) + 1u;                                          // {source LSB, fixed 1}
         if (a >= 0x47400000u) r = top;                                                     // >= 1.5 * 2^15
@@ -295,8 +309,10 @@ __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, uns
     {
         const int e = threadIdx.x, E = e - 127 + se;
         uint32_t inc = 0, mask = 0, kfac = 0;
-        if (e == 255 || (e == 0 && se > 100) || (e > 0 && E >= 15)) mask = kRareMask;
+        // (subnormal sources: below 2^(se - 126); standard SR can still round up from 2^-38 on, the other modes from 2^-24)
+        if (e == 255 || (e == 0 && se > (MODE == HIF8_RND_SR ? 88 : 100)) || (e > 0 && E >= 15)) mask = kRareMask;
         else if ((MODE == HIF8_RND_HR || MODE == HIF8_RND_SSR) && e > 0 && (E == -23 || E == -24)) mask = kRareMask;  // result is 0 or 2^-22
+        else if (MODE == HIF8_RND_SR && e > 0 && E <= -23 && E >= -38) mask = kRareMask;    // 0 or 2^-22, by the threshold
         else if (e == 0 || E <= -24) { inc = 0; mask = 0; }                                 // underflow to +0
         else if (E == -23) { inc = 1u << MB; mask = 0xFFFFFFFFu << MB; }                    // up to 2^-22
         else {
@@ -319,7 +335,11 @@ __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, uns
             const bool rare = mask == kRareMask || cb < 1 || cb > 254;
             s_inc[e] = rare ? kRareMask : (uint32_t)cb << 23;  // C in the high half
         } else if (SRC == HIF8_F32) { s_inc[e] = inc; s_mask[e] = mask; }
-        else {
+        else if (MODE == HIF8_RND_SR) {
+            // mask16 | (16 - discarded bits) << 16; exponents that underflow to +0 keep mask 0 and a shift of 16 (no increment)
+            const uint32_t kbits = (mask == kRareMask || mask == 0u) ? 0u : (uint32_t)__popc(~mask & 0xFFFFu);
+            s_inc[e] = (mask & 0xFFFFu) | ((16u - kbits) << 16);
+        } else {
             s_inc[e] = (mask & 0xFFFFu) | (inc << 16);
             if (kThr) s_mask[e] = kfac;
         }
@@ -354,6 +374,34 @@ __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, uns
 #pragma unroll
                     for (int k = 0; k < 4; k++)
                         if (m[k] == kRareMask) o[k] = fq_rare<SRC, MODE>(w[k], se, p.flags);
+                }
+            } else if (MODE == HIF8_RND_SR) {
+                // Standard SR on the source pattern: with k discarded bits and threshold T, one is added to the kept bits iff
+                // the discarded field d is non-zero and d * 2^(16 - k) >= T, i.e. iff d >= max(1, ceil(T / 2^(16 - k))): add
+                // (2^k - 1) - ((max(T, 1) - 1) >> (16 - k)) and let the carry out of the field do it, then clear the field.
+                // Element 8 u + j takes word j mod 4 of the Philox block 2 u + j / 4.
+                const uint32_t k0 = (uint32_t)p.seed, k1 = (uint32_t)(p.seed >> 32);
+                const uint4 q0 = philox4x32_10((uint32_t)(u * 2), (uint32_t)((u * 2) >> 32), k0, k1);
+                const uint4 q1 = philox4x32_10((uint32_t)(u * 2 + 1), (uint32_t)((u * 2 + 1) >> 32), k0, k1);
+                const uint32_t rw[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+                uint32_t tl[4], th[4];
+#pragma unroll
+                for (int k = 0; k < 4; k++) {
+                    tl[k] = s_inc[(w[k] >> 7) & 0xFFu];
+                    th[k] = s_inc[(w[k] >> 23) & 0xFFu];
+                    const uint32_t Tl = rw[2 * k] >> 16, Th = rw[2 * k + 1] >> 16, sl = tl[k] >> 16, sh = th[k] >> 16;  // s = 16 - k
+                    // (2^k - 1) - d per half; flagged and underflowing exponents carry s = 16: no increment at all
+                    const uint32_t il = (0xFFFFu >> sl) - ((Tl - (Tl != 0u)) >> sl), ih = (0xFFFFu >> sh) - ((Th - (Th != 0u)) >> sh);
+                    const uint32_t mask2 = __byte_perm(tl[k], th[k], 0x5410);
+                    o[k] = (w[k] + (il | (ih << 16))) & mask2;  // no carry between the halves: only finite, in-range values add
+                    rare |= tl[k] | th[k];
+                }
+                if (rare & kRareMask) {
+#pragma unroll
+                    for (int k = 0; k < 4; k++) {
+                        if (tl[k] & kRareMask) o[k] = (o[k] & 0xFFFF0000u) | fq_rare<SRC, MODE>(w[k] & 0xFFFFu, se, p.flags, rw[2 * k] >> 16);
+                        if (th[k] & kRareMask) o[k] = (o[k] & 0x0000FFFFu) | (fq_rare<SRC, MODE>(w[k] >> 16, se, p.flags, rw[2 * k + 1] >> 16) << 16);
+                    }
                 }
             } else {
                 uint32_t tl[4], th[4];
@@ -408,7 +456,13 @@ __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, uns
                 reinterpret_cast<uint32_t*>(p.dst)[i] = fq_rare<SRC, MODE>(raw, se, p.flags);
             } else {
                 const uint32_t raw = reinterpret_cast<const unsigned short*>(p.src)[i];
-                reinterpret_cast<unsigned short*>(p.dst)[i] = (unsigned short)fq_rare<SRC, MODE>(raw, se, p.flags);
+                uint32_t T16 = 0u;
+                if (MODE == HIF8_RND_SR) {
+                    const uint4 q = philox4x32_10((uint32_t)(i >> 2), (uint32_t)(i >> 34), (uint32_t)p.seed, (uint32_t)(p.seed >> 32));
+                    const uint32_t qq[4] = {q.x, q.y, q.z, q.w};
+                    T16 = qq[i & 3] >> 16;
+                }
+                reinterpret_cast<unsigned short*>(p.dst)[i] = (unsigned short)fq_rare<SRC, MODE>(raw, se, p.flags, T16);
             }
         }
     }
@@ -627,6 +681,7 @@ int launch_fq_ta(int dtype, int rnd, const ConvParams& p, bool vec_ok, int sms, 
     else if (rnd == HIF8_RND_TA) launch_pdl(fq_ta_kernel<HIF8_BF16, HIF8_RND_TA>, grid, st, p, n_vec);
     else if (rnd == HIF8_RND_HR) launch_pdl(fq_ta_kernel<HIF8_BF16, HIF8_RND_HR>, grid, st, p, n_vec);
     else if (rnd == HIF8_RND_TE) launch_pdl(fq_ta_kernel<HIF8_BF16, HIF8_RND_TE>, grid, st, p, n_vec);
+    else if (rnd == HIF8_RND_SR) launch_pdl(fq_ta_kernel<HIF8_BF16, HIF8_RND_SR>, grid, st, p, n_vec);
     else launch_pdl(fq_ta_kernel<HIF8_BF16, HIF8_RND_SSR>, grid, st, p, n_vec);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
@@ -760,7 +815,7 @@ static int scaled_convert(bool fq, const void* src, void* dst, int dtype, size_t
     }
     p.scale_state = scale_state;
     const bool inplace_fq = fq && !want_amax && ((rnd == HIF8_RND_TA && (dtype == HIF8_F32 || dtype == HIF8_BF16)) ||
-                                                ((rnd == HIF8_RND_HR || rnd == HIF8_RND_SSR || rnd == HIF8_RND_TE) && dtype == HIF8_BF16));
+                                                ((rnd == HIF8_RND_HR || rnd == HIF8_RND_SSR || rnd == HIF8_RND_TE || rnd == HIF8_RND_SR) && dtype == HIF8_BF16));
     if (jit) {
         rc = launch_amax(src, dtype, n, ws, nullptr, sms, st);
         if (rc) return rc;

@@ -262,7 +262,19 @@ def test_fake_quant(dtype, mode):
     assert_same(got, O.fake_quant(src, dtype, se, mode, 0, seed=9, quick=True), src)
 
 
-@pytest.mark.parametrize("mode,omode", [(H.RND_TA, O.TA), (H.RND_TE, O.TE), (H.RND_HR, O.HR), (H.RND_SSR, O.SSR)])
+def test_fake_quant_bf16_standard_sr_many_thresholds_per_pattern():
+    # the in-place kernel's standard SR: every BF16 pattern at 32 positions (32 different Philox words each), several
+    # scales and seeds, both options; the last positions run through the scalar tail
+    src = np.tile(W.all_u16(), 32)[:-3]
+    d_src = to_dev(src)
+    for se, flags, seed in [(0, 0, 1), (5, 3, 2), (-20, 0, 3), (14, 1, 0xDEADBEEF12345678), (30, 2, 5)]:
+        _, dptr, rb = dev_empty(src.size, np.uint16)
+        H.hif8_fake_quant(d_src, dptr, H.BF16, src.size, 0, se, H.RND_SR, flags, seed)
+        torch.cuda.synchronize()
+        assert_same(rb(), O.fake_quant(src, O.BF16, se, O.SR, flags, seed=seed, quick=True), src)
+
+
+@pytest.mark.parametrize("mode,omode", [(H.RND_TA, O.TA), (H.RND_TE, O.TE), (H.RND_HR, O.HR), (H.RND_SSR, O.SSR), (H.RND_SR, O.SR)])
 def test_fake_quant_bf16_in_place_scale_edges_and_tails(mode, omode):
     # the in-place kernel rounds BF16 with per-exponent constants (packed BF16 arithmetic except for round half away):
     # scales at which a constant leaves the BF16 range or subnormal sources come into range, every pattern; then ragged,
