@@ -226,3 +226,30 @@ def test_gemm_narrow_channel_scales_and_accumulate(K):
     P, S = O.gemm_entries_channel(Aq, Wkn, 0, 2, sw, rows, cols)
     want = P.reshape(M, N) + c0
     assert np.all(np.abs(C.cpu().numpy().astype(np.float64) - want) <= 1e-5 * S.reshape(M, N) + 2.0 ** -24 * np.abs(want))
+
+
+def test_tensor_map_cache_survives_eviction_and_pointer_reuse():
+    # more distinct (pointer, shape) pairs than the library's tensor-map cache holds, each product exact in small integers;
+    # then the same device buffers again with other shapes and contents (a cached map must never serve a different tensor)
+    ints = np.array([0x00, 0x08, 0x10, 0x14, 0x88, 0x90], dtype=np.uint8)          # 0, 1, 2, 3, -1, -2
+    tab = np.array([O.value(c) for c in range(256)])
+    rng = np.random.default_rng(11)
+    bufA = torch.empty(512 * 1024, dtype=torch.uint8, device="cuda")
+    bufW = torch.empty(1024 * 512, dtype=torch.uint8, device="cuda")
+    ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+    stream2 = torch.cuda.Stream()
+    for it in range(80):
+        M, N, K = 16 * int(rng.integers(1, 20)), 16 * int(rng.integers(1, 24)), 16 * int(rng.integers(1, 40))
+        Aq = ints[rng.integers(0, len(ints), (M, K))]
+        Wq = ints[rng.integers(0, len(ints), (K, N))]
+        bufA[:M * K].copy_(torch.from_numpy(Aq.reshape(-1)))
+        bufW[:K * N].copy_(torch.from_numpy(Wq.reshape(-1)))
+        C = torch.zeros(M, N, dtype=torch.float32, device="cuda")
+        st = stream2 if it % 3 == 0 else None
+        if st is not None:
+            st.wait_stream(torch.cuda.current_stream())
+        H.hif8_gemm(bufA, K, bufW, N, 0, C, N, H.F32, M, N, K, None, None, ws, 256, stream=st)
+        assert H.hif8_last_device_status(st) == 0            # synchronises that stream
+        want = (tab[Aq].astype(np.int64) @ tab[Wq].astype(np.int64)).astype(np.float64)
+        assert np.array_equal(C.cpu().numpy().astype(np.float64), want), (it, M, N, K)
+    assert H.hif8_last_device_status(torch.cuda.Stream()) == 0   # a stream that never saw a GEMM
