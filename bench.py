@@ -822,7 +822,10 @@ def main():
     e2e_ms = max_over_ranks([e0.elapsed_time(e1) / E], dist if world > 1 else None, "cuda")[0]
     if world > 1:
         k_amax, k_conv, k_dec, k_enc, k_del = [max_over_ranks(v, dist, "cuda") for v in (k_amax, k_conv, k_dec, k_enc, k_del)]
-        multi = sharded_results(H, torch, dist, rank, world, stream)
+        try:   # secondary figures: a failure here must not take the headline line with it
+            multi = sharded_results(H, torch, dist, rank, world, stream)
+        except Exception as exc:  # noqa: BLE001
+            multi = {"error": f"{type(exc).__name__}: {exc}"}
 
     if rank == 0:
         step, serial_st = spread(step_samples), spread(serial_samples)
