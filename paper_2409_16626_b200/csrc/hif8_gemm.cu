@@ -215,13 +215,14 @@ __device__ __forceinline__ void tc_commit_cta(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tc_mma_bf16_cta(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
+// one-CTA form with the A operand (128 rows) in tensor memory
+__device__ __forceinline__ void tc_mma_bf16_cta_a_tmem(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
 {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar)  // arrives on `bar` in both CTAs of the pair
 {
@@ -277,6 +278,19 @@ __device__ __forceinline__ uint32_t hif8_to_bf16_bits(uint32_t c)
     return sign | ((uint32_t)(E + 127) << 7) | (M << (7 - w));
 }
 
+// Fills the decode table: entry (code c, lane l) at word c * ROW_WORDS + l holds the BF16 bits of code c (one copy per
+// lane, so that a warp's lookups never meet in a bank).  A warp takes 32 codes: each lane works out one code's value
+// once and the warp hands the 32 values round.
+template <int ROW_WORDS>
+__device__ __forceinline__ void fill_decode_table(uint32_t* table, int warp, int lane, int n_warps)
+{
+    for (int c0 = warp * 32; c0 < 256; c0 += n_warps * 32) {
+        const uint32_t v = hif8_to_bf16_bits((uint32_t)(c0 + lane));
+#pragma unroll 8
+        for (int k = 0; k < 32; k++) table[(c0 + k) * ROW_WORDS + lane] = __shfl_sync(0xFFFFFFFFu, v, k);
+    }
+}
+
 // Shared-memory accesses by 32-bit shared-window address: the operand ring lives at a run-time offset inside the dynamic
 // allocation, and spelling the state space out keeps every one of these an LDS / STS (never a generic access).
 // (not volatile: the table is constant once it is built and every address derives from a byte read after the barrier
@@ -291,6 +305,12 @@ __device__ __forceinline__ uint2 lds_v2(uint32_t addr)
 {
     uint2 v;
     asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds_u8(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(addr));
     return v;
 }
 __device__ __forceinline__ uint4 lds_v4(uint32_t addr)
@@ -524,8 +544,7 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     const int num_kb = (p.K + BK - 1) / BK;
 
     // ---- set-up
-    for (int i = threadIdx.x; i < 256 * 32; i += kThreads)  // entry (code i / 32, lane i % 32): rows of 1 << kLutShift bytes
-        lut_all[((i >> 5) << (kLutShift - 2)) + (i & 31)] = hif8_to_bf16_bits(i >> 5);
+    fill_decode_table<(1 << (kLutShift - 2))>(lut_all, warp, lane, kThreads / 32);  // rows of 1 << kLutShift bytes
     if (threadIdx.x == 0) {
         for (int s = 0; s < kS8; s++) { mbar_init(bar_u8_full(s), 1); mbar_init(bar_u8_empty(s), kGroupWarps); }
         for (int s = 0; s < kStagesBf; s++) { mbar_init(bar_bf_full(s), 2 * kGroupWarps); mbar_init(bar_bf_empty(s), 1); }
@@ -682,43 +701,65 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 // ---------------------------------------------------------------------------------------------------------
 // Narrow products (M <= 64 rows of activations: the decode phase of inference).  The product is bound by reading the
 // weight bytes once, so the roles are swapped: a CTA streams a slab of 128 weight columns as the 128-row MMA operand and
-// the few activation rows are the narrow operand (MMA N = M rounded up to 16).  Same machinery as the fused kernel
-// (byte tiles by TMA, four decode groups on four k-blocks, operands in the 128-byte-swizzled layout), one CTA per slab,
-// no pairs.  The accumulator holds C transposed (row = weight column n, column = activation row m); the epilogue writes
-// C[m][n] with consecutive lanes on consecutive n.
+// the few activation rows are the narrow operand (MMA N = M rounded up to 16).  One CTA per SM, no pairs:
+//   warp 4        copies: per pair block (two k-blocks) one tile of weight bytes and one of activation bytes
+//   warps 6-21    four decode groups, group g on the k-blocks it = g (mod 4): a thread owns one weight column of the slab,
+//                 decodes its 64 bytes of the k-block and stores them as its lane of a weight stage in tensor memory (the A
+//                 operand of tcgen05.mma may live there); the group also decodes the activation tile into shared memory
+//   warps 5, 22-24  MMA issuers (below)
+//   warps 0-3     epilogue
+// The accumulator holds C transposed (row = weight column n, column = activation row m); the epilogue writes C[m][n] with
+// consecutive lanes on consecutive n.
 // ---------------------------------------------------------------------------------------------------------
 constexpr int kNarrowMaxM = 64;
 constexpr uint32_t kNwW8 = BM * BK, kNwA8 = kNarrowMaxM * BK;          // byte tiles per stage: 8 KiB weights, 4 KiB activations
-constexpr uint32_t kNwWBf = BM * BK * 2, kNwABf = kNarrowMaxM * BK * 2;  // operand tiles per stage: 16 KiB + 8 KiB
-constexpr int kNwByteStages = 8;  // byte ring deeper than the operand ring: 8 x 8 KiB of weights in flight per SM
+constexpr uint32_t kNwABf = kNarrowMaxM * BK * 2;  // activation operand tile per stage: 8 KiB (the weights go to tensor memory)
+// A copy brings two k-blocks (a "pair block": 128 bytes of k) of weights and of activations: issuing a tile copy costs
+// its thread a few hundred cycles whatever the size, and with one copy of each kind per k-block that thread set the pace.
+// Four stages of 16 KiB + 8 KiB: 64 KiB of weights in flight per SM.
+constexpr int kNwByteStages = 4, BK2 = 2 * BK;
+// Operand stages (32 tensor-memory columns of weights + 8 KiB of activations in shared memory each): two per group, so
+// that a group starts its next k-block without waiting for the MMAs of its previous one
+constexpr int kNwTmemStages = 2 * kDecodeGroups;
 struct SmemLayoutN {
     static constexpr uint32_t bf = 0;
-    static constexpr uint32_t u8 = bf + kDecodeGroups * (kNwWBf + kNwABf);
-    static constexpr uint32_t lut = u8 + kNwByteStages * (kNwW8 + kNwA8);
+    static constexpr uint32_t u8 = bf + kNwTmemStages * kNwABf;
+    static constexpr uint32_t lut = u8 + kNwByteStages * 2 * (kNwW8 + kNwA8);
     static constexpr uint32_t bars = lut + 256 * 32 * 4;
-    static constexpr uint32_t n_bars = 2 * kNwByteStages + 2 * kDecodeGroups + 4;
+    static constexpr uint32_t n_bars = 2 * kNwByteStages + 2 * kNwTmemStages + 4;
     static constexpr uint32_t tmem_slot = bars + n_bars * 8;
     static constexpr uint32_t abort_flag = tmem_slot + 4;
     static constexpr uint32_t total = abort_flag + 4;
 };
 constexpr uint32_t kSmemBytesN = SmemLayoutN::total + 1024;
-constexpr uint32_t kTmemColsN = 2 * kNarrowMaxM;  // two accumulators: the epilogue of one segment overlaps the next segment's MMAs
+// Tensor memory: the accumulators (two per issuer: the epilogue of one segment overlaps the next segment's MMAs), then
+// one weight stage (128 rows x 64 BF16 = 32 columns) per operand stage.
+// MMA issuers.  One thread that waits for a stage, issues its four MMAs and commits spends about a thousand cycles per
+// k-block, more than the decode groups or the copies need; so up to four threads (one per warp) share the k-blocks,
+// issuer q taking the k-blocks it = q (mod issuers) into accumulators of its own, which the epilogue adds.  Four issuers
+// for up to 32 activation rows, two above: 2 buffers x issuers x rows stays within 256 columns.
+constexpr int kNwMaxIssuers = 4;
+constexpr int kThreadsN = kThreads + (kNwMaxIssuers - 1) * 32;  // 800: the first issuer is the MMA warp of the other kernels
+constexpr uint32_t kTmemAccN = 2 * 2 * kNarrowMaxM, kTmemColsN = 512;
+static_assert(kTmemAccN + kNwTmemStages * (BK / 2) <= kTmemColsN, "weight stages fit beside the accumulators");
+static_assert(2 * kNwMaxIssuers * 32 <= kTmemAccN, "four issuers x two buffers x 32 rows");
 
-// Work split of the narrow kernel.  The (slab, k-block) pairs are numbered slab-major, total = slabs * k-blocks, and CTA c
-// of G takes the contiguous range [total c / G, total (c + 1) / G): every SM streams the same number of weight bytes
-// whatever the number of slabs.  A range cuts slabs into segments.  A segment that covers its whole slab is finished by
+// Work split of the narrow kernel.  The unit is a pair block (two k-blocks; the second one of a slab's last pair may lie
+// beyond K, where the copies fill zeros).  The (slab, pair block) units are numbered slab-major, total = slabs * pair
+// blocks, and CTA c of G takes the contiguous range [total c / G, total (c + 1) / G): every SM streams the same number of
+// weight bytes whatever the number of slabs.  A range cuts slabs into segments.  A segment that covers its whole slab is finished by
 // its CTA; otherwise the CTA stores its FP32 partial sums as slice (slab, its position among the slab's contributors),
 // and the last contributor to arrive (one ticket per slab and epilogue warp) adds the slices in position order - so the
 // result does not depend on arrival order - and writes C.
 struct NarrowPlan {
-    long long total;     // slabs * k-blocks
+    long long total;     // slabs * pair blocks
     float* part;         // [slab][pmax][mp][128] partial sums, or nullptr when every range is made of whole slabs
     unsigned* tickets;   // [slab][4], zero at launch
     int pmax;            // slices per slab
 };
 
 template <bool W_IS_NK>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreadsN, 1)
 hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_constant__ CUtensorMap map_w, const GemmParams p, int mp,
                         const NarrowPlan plan)
 {
@@ -726,9 +767,10 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     unsigned char* sm = smem_raw + (base - smem_u32(smem_raw));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    constexpr int S = kDecodeGroups;    // operand ring: group g owns stage g
-    constexpr int S8 = kNwByteStages;   // byte ring: the it-th k-block of this CTA lands in stage it % S8
-    static_assert(S8 % kDecodeGroups == 0, "a byte stage is always read by the same group");
+    constexpr int S = kNwTmemStages;  // operand ring: the it-th k-block uses stage it % S
+    static_assert(S % kDecodeGroups == 0, "an operand stage is always written by the same group");
+    constexpr int S8 = kNwByteStages;   // byte ring: the i-th pair block of this CTA lands in stage i % S8
+    constexpr uint32_t kU8Stage = 2 * (kNwW8 + kNwA8), kU8Act = 2 * kNwW8;  // byte stage: 128 weight columns x 128 k, then act rows x 128 k
     const uint32_t bars = base + SmemLayoutN::bars;
     auto bar_u8_full = [&](int s) { return bars + 8u * s; };
     auto bar_u8_empty = [&](int s) { return bars + 8u * (S8 + s); };
@@ -740,17 +782,20 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + SmemLayoutN::tmem_slot);
     uint32_t* lut_all = reinterpret_cast<uint32_t*>(sm + SmemLayoutN::lut);
     const uint32_t lut = base + SmemLayoutN::lut + 4u * lane;
-    const int num_kb = (p.K + BK - 1) / BK;
+    const int num_pb = (p.K + BK2 - 1) / BK2, num_kb = 2 * num_pb;  // per slab
     const long long G = gridDim.x;
-    const long long lin0 = plan.total * blockIdx.x / G, lin1 = plan.total * (blockIdx.x + 1) / G;  // this CTA's (slab, k-block) range
-    const int n_it = (int)(lin1 - lin0);
-    const uint32_t act_bytes = (uint32_t)mp * BK;
+    const long long pair0 = plan.total * blockIdx.x / G, pair1 = plan.total * (blockIdx.x + 1) / G;  // this CTA's (slab, pair block) range
+    const long long lin0 = 2 * pair0, lin1 = 2 * pair1;  // the same in k-blocks
+    const int n_pairs = (int)(pair1 - pair0), n_it = 2 * n_pairs;
+    const uint32_t act_bytes = (uint32_t)mp * BK2;
+    const int issuers = mp <= 32 ? kNwMaxIssuers : 2;
+    auto acc_col = [&](int q, int buf) { return (uint32_t)((q * 2 + buf) * mp); };  // accumulator of issuer q, buffer buf
 
-    for (int i = threadIdx.x; i < 256 * 32; i += kThreads) lut_all[i] = hif8_to_bf16_bits(i >> 5);
+    fill_decode_table<32>(lut_all, warp, lane, kThreadsN / 32);
     if (threadIdx.x == 0) {
-        for (int s = 0; s < S8; s++) { mbar_init(bar_u8_full(s), 1); mbar_init(bar_u8_empty(s), kGroupWarps); }
+        for (int s = 0; s < S8; s++) { mbar_init(bar_u8_full(s), 1); mbar_init(bar_u8_empty(s), 2 * kGroupWarps); }  // both halves' groups
         for (int s = 0; s < S; s++) { mbar_init(bar_bf_full(s), kGroupWarps); mbar_init(bar_bf_empty(s), 1); }
-        for (int b = 0; b < 2; b++) { mbar_init(bar_acc_full(b), 1); mbar_init(bar_acc_empty(b), kEpiWarps); }
+        for (int b = 0; b < 2; b++) { mbar_init(bar_acc_full(b), issuers); mbar_init(bar_acc_empty(b), kEpiWarps); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -767,18 +812,18 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
     if (warp == kTmaWarp) {
         if (lane == 0) {
             int issued = 0;
-            int j = (int)(lin0 / num_kb), kb = (int)(lin0 % num_kb);
-            for (int it = 0; it < n_it; it++) {
+            int j = (int)(pair0 / num_pb), pb = (int)(pair0 % num_pb);
+            for (int it = 0; it < n_pairs; it++) {
                 const int s = it % S8, round = it / S8;
                 if (round > 0 && !mbar_wait(bar_u8_empty(s), (round - 1) & 1, abort_flag, p.status, 31)) break;
                 if (*abort_flag) break;
-                const uint32_t dst_w = base + SmemLayoutN::u8 + s * (kNwW8 + kNwA8), dst_a = dst_w + kNwW8;
-                mbar_arrive_expect_tx(bar_u8_full(s), kNwW8 + act_bytes);
-                if (W_IS_NK) tma_load_2d(dst_w, &map_w, kb * BK, j * BM, bar_u8_full(s));
-                else tma_load_2d(dst_w, &map_w, j * BM, kb * BK, bar_u8_full(s));
-                tma_load_2d(dst_a, &map_act, kb * BK, 0, bar_u8_full(s));
+                const uint32_t dst_w = base + SmemLayoutN::u8 + s * kU8Stage, dst_a = dst_w + kU8Act;
+                mbar_arrive_expect_tx(bar_u8_full(s), 2 * kNwW8 + act_bytes);
+                if (W_IS_NK) tma_load_2d(dst_w, &map_w, pb * BK2, j * BM, bar_u8_full(s));
+                else tma_load_2d(dst_w, &map_w, j * BM, pb * BK2, bar_u8_full(s));
+                tma_load_2d(dst_a, &map_act, pb * BK2, 0, bar_u8_full(s));
                 issued = it + 1;
-                if (++kb == num_kb) { kb = 0; j++; }
+                if (++pb == num_pb) { pb = 0; j++; }
             }
             if (*abort_flag) {  // let the copies already issued land before this CTA's shared memory goes away
                 for (int it = max(0, issued - S8); it < issued; it++) {
@@ -787,32 +832,37 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
                 }
             }
         }
-    } else if (warp == kMmaWarp) {
-        if (lane == 0) {
+    } else if (warp == kMmaWarp || warp >= kFirstDecodeWarp + kDecodeWarps) {
+        const int q = warp == kMmaWarp ? 0 : warp - (kFirstDecodeWarp + kDecodeWarps) + 1;  // issuer number
+        if (lane == 0 && q < issuers) {
             // FP32 accumulator, BF16 operands; A = weight slab (K-major for [N,K] weights, MN-major for [K,N]), B = activations
             // (K-major), N = mp, M = 128
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((W_IS_NK ? 0u : 1u) << 15) | ((uint32_t)(mp >> 3) << 17) |
-                                   ((uint32_t)(BM >> 4) << 24);
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(mp >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+            // descriptor of stage 0; a stage or a 16-k step further on adds to the address field only
+            const uint64_t da0 = make_smem_desc(base + SmemLayoutN::bf, 16, 1024);
             bool ok = true, first = true;
             int kb = (int)(lin0 % num_kb), seg = 0;
             for (int it = 0; it < n_it && ok; it++) {
-                const int s = it % S, round = it / S, buf = seg & 1;
-                // a segment's first MMA overwrites the accumulator: the epilogue must have read its previous contents
-                if (first && seg >= 2) ok = mbar_wait(bar_acc_empty(buf), ((seg >> 1) - 1) & 1, abort_flag, p.status, 36);
-                if (ok) ok = mbar_wait(bar_bf_full(s), round & 1, abort_flag, p.status, 32);
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t w_addr = base + SmemLayoutN::bf + s * (kNwWBf + kNwABf), a_addr = w_addr + kNwWBf;
+                const int buf = seg & 1;
+                if ((it & (issuers - 1)) == q) {
+                    const int s = it % S, round = it / S;
+                    // a segment's first MMA overwrites the accumulator: the epilogue must have read its previous contents
+                    if (first && seg >= 2) ok = mbar_wait(bar_acc_empty(buf), ((seg >> 1) - 1) & 1, abort_flag, p.status, 36);
+                    if (ok) ok = mbar_wait(bar_bf_full(s), round & 1, abort_flag, p.status, 32);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + acc_col(q, buf);
 #pragma unroll
-                for (int kk = 0; kk < BK / 16; kk++) {
-                    const uint64_t dw = W_IS_NK ? make_smem_desc(w_addr + kk * 32, 16, 1024) : make_smem_desc(w_addr + kk * 2048, 8192, 1024);
-                    const uint64_t da = make_smem_desc(a_addr + kk * 32, 16, 1024);
-                    tc_mma_bf16_cta(tmem_base + (uint32_t)(buf * kNarrowMaxM), dw, da, idesc, (!first || kk > 0) ? 1u : 0u);
+                    for (int kk = 0; kk < BK / 16; kk++) {
+                        // weights from tensor memory: operand stage s, 16 k = 8 columns
+                        tc_mma_bf16_cta_a_tmem(d_tmem, tmem_base + kTmemAccN + (uint32_t)(s * (BK / 2) + kk * 8),
+                                               da0 + (uint64_t)((s * kNwABf + kk * 32) >> 4), idesc, (!first || kk > 0) ? 1u : 0u);
+                    }
+                    tc_commit_cta(bar_bf_empty(s));
+                    first = false;
                 }
-                tc_commit_cta(bar_bf_empty(s));
-                first = false;
                 if (++kb == num_kb || it == n_it - 1) {  // the segment ends with its slab or with this CTA's range
-                    tc_commit_cta(bar_acc_full(buf));
+                    tc_commit_cta(bar_acc_full(buf));    // (an issuer without a k-block in the segment arrives at once)
                     kb = 0; seg++; first = true;
                 }
             }
@@ -823,28 +873,60 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
         const int act_chunks = mp * (BK / 8);  // 8-byte chunks of the activation tile
         bool ok = true;
         for (int it = group; it < n_it && ok; it += kDecodeGroups) {
-            const int s = group, r = it / S, s8 = it % S8;
-            ok = mbar_wait(bar_u8_full(s8), (it / S8) & 1, abort_flag, p.status, 33);
+            const int s = it % S, r = it / S, s8 = (it >> 1) % S8, h = it & 1;  // h: which k-block of its pair block
+            ok = mbar_wait(bar_u8_full(s8), ((it >> 1) / S8) & 1, abort_flag, p.status, 33);
             if (ok && r > 0) ok = mbar_wait(bar_bf_empty(s), (r - 1) & 1, abort_flag, p.status, 34);
             if (!ok) break;
-            const uint32_t w8 = base + SmemLayoutN::u8 + s8 * (kNwW8 + kNwA8), a8 = w8 + kNwW8;
-            const uint32_t wbf = base + SmemLayoutN::bf + s * (kNwWBf + kNwABf), abf = wbf + kNwWBf;
-            uint2 vw[kChunksPerThread], va[kNarrowMaxM * (BK / 8) / kGroupThreads];
-            load_tile_chunks<!W_IS_NK>(w8, dt, vw);
+            const uint32_t w8 = base + SmemLayoutN::u8 + s8 * kU8Stage, a8 = w8 + kU8Act + (uint32_t)h * BK;
+            const uint32_t abf = base + SmemLayoutN::bf + s * kNwABf;
+            uint2 va[kNarrowMaxM * (BK / 8) / kGroupThreads];
+            uint4 vr[BK / 16];
+            // this thread owns weight column (operand row, tensor-memory lane) quarter * 32 + lane of the slab
+            const int wr = (warp & 3) * 32 + lane;
+            if (W_IS_NK) {
+                // [N,K] weights: the byte tile (rows of 128 k) arrives with the 128-byte TMA swizzle (chunk j of row r at chunk
+                // j ^ (r & 7)): conflict-free row reads
+                const uint32_t w_row = w8 + (uint32_t)wr * BK2, sw = (uint32_t)wr & 7u;
+#pragma unroll
+                for (int jj = 0; jj < BK / 16; jj++) vr[jj] = lds_v4(w_row + (((uint32_t)(4 * h + jj) ^ sw) << 4));
+            }
 #pragma unroll
             for (int i = 0; i < kNarrowMaxM * (BK / 8) / kGroupThreads; i++) {
                 const int q = i * kGroupThreads + dt;
-                if (q < act_chunks) va[i] = lds_v2(a8 + (q >> 3) * BK + (q & 7) * 8);
+                if (q < act_chunks) va[i] = lds_v2(a8 + (q >> 3) * BK2 + (q & 7) * 8);
             }
-            __syncwarp();  // the byte stage has been read: the producer may refill it during the decode
-            if (lane == 0) mbar_arrive(bar_u8_empty(s8));
-            decode_tile_chunks<!W_IS_NK>(vw, wbf, dt, lut);
+            uint32_t o[BK / 2];  // 64 BF16 of this weight column, two per tensor-memory column
+            if (W_IS_NK) {
+                __syncwarp();  // the byte stage has been read: the producer may refill it during the decode
+                if (lane == 0) mbar_arrive(bar_u8_empty(s8));
+#pragma unroll
+                for (int jj = 0; jj < BK / 16; jj++) {
+                    const uint4 lo = decode8<7>(make_uint2(vr[jj].x, vr[jj].y), lut), hi = decode8<7>(make_uint2(vr[jj].z, vr[jj].w), lut);
+                    o[8 * jj + 0] = lo.x; o[8 * jj + 1] = lo.y; o[8 * jj + 2] = lo.z; o[8 * jj + 3] = lo.w;
+                    o[8 * jj + 4] = hi.x; o[8 * jj + 5] = hi.y; o[8 * jj + 6] = hi.z; o[8 * jj + 7] = hi.w;
+                }
+            } else {
+                // [K,N] weights: row k of the pair's tile holds the 128 columns of the slab (the pair's second k-block is its
+                // rows 64-127), so the column is read a byte per k: the 32 lanes of a warp read 32 consecutive bytes, one
+                // wavefront, and the byte is the table row without any extraction
+                const uint32_t w_col = w8 + (uint32_t)h * kNwW8 + (uint32_t)wr;
+#pragma unroll
+                for (int j = 0; j < BK / 2; j++) {
+                    const uint32_t c0 = lds_u8(w_col + (uint32_t)(2 * j) * BM), c1 = lds_u8(w_col + (uint32_t)(2 * j + 1) * BM);
+                    o[j] = __byte_perm(lds_u32(lut + (c0 << 7)), lds_u32(lut + (c1 << 7)), 0x5410);
+                }
+                __syncwarp();  // the byte stage has been read
+                if (lane == 0) mbar_arrive(bar_u8_empty(s8));
+            }
+            tmem_st_32x32b_x32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + kTmemAccN + (uint32_t)(s * (BK / 2)), o);
 #pragma unroll
             for (int i = 0; i < kNarrowMaxM * (BK / 8) / kGroupThreads; i++) {
                 const int q = i * kGroupThreads + dt, row = q >> 3, jc = q & 7;
                 if (q < act_chunks) sts_v4(abf + (row >> 3) * 1024 + (row & 7) * 128 + ((jc ^ (row & 7)) << 4), decode8<7>(va[i], lut));
             }
+            tmem_st_wait();  // the weight column is in tensor memory
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_bf_full(s));
         }
@@ -874,27 +956,37 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
                     *out = (unsigned short)((v != v) ? 0x7FC0u : ((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16));
                 }
             };
-            // contributors of slab j are the CTAs owner(first k-block) .. owner(last k-block);
+            // contributors of slab j are the CTAs owner(first pair block) .. owner(last pair block);
             // owner(x) = the largest c with total c / G <= x
-            const long long c_first = ((slab_end - num_kb + 1) * G - 1) / plan.total, c_last = (slab_end * G - 1) / plan.total;
+            const long long c_first = (((long long)j * num_pb + 1) * G - 1) / plan.total, c_last = ((long long)(j + 1) * num_pb * G - 1) / plan.total;
             const int pos = (int)(blockIdx.x - c_first), count = (int)(c_last - c_first + 1);
             float* slab_part = whole ? nullptr : plan.part + (size_t)j * plan.pmax * mp * BM + warp * 32 + lane;
             float* mine = whole ? nullptr : slab_part + (size_t)pos * mp * BM;
-            const uint32_t taddr = tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(buf * kNarrowMaxM);
+            const uint32_t tlane = tmem_base + ((uint32_t)(warp * 32) << 16);
+            const int it_a = (int)(lin - lin0), it_n = (int)(seg_end - lin);  // the segment's k-blocks, counted within this CTA's range
             for (int c = 0; c < mp; c += 32) {
-                uint32_t r[32];  // this lane's row of the accumulator, columns c .. c + 31
-                tmem_ld_32x32b_x32(taddr + c, r);
-                tmem_ld_wait();
+                float r[32];  // this lane's row of the segment's sum, columns c .. c + 31: the issuers' accumulators added in order
+#pragma unroll
+                for (int i = 0; i < 32; i++) r[i] = 0.f;
+                for (int q = 0; q < issuers; q++) {
+                    // issuer q took the k-blocks it = q (mod issuers): none of them in a short segment leaves its accumulator stale
+                    if (it_n < issuers && ((q - it_a) & (issuers - 1)) >= it_n) continue;
+                    uint32_t t[32];
+                    tmem_ld_32x32b_x32(tlane + acc_col(q, buf) + c, t);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 32; i++) r[i] += __uint_as_float(t[i]);
+                }
                 if (whole) {
                     if (n < p.N) {
 #pragma unroll
                         for (int i = 0; i < 32; i++)
-                            if (c + i < p.M) finish(c + i, __uint_as_float(r[i]));
+                            if (c + i < p.M) finish(c + i, r[i]);
                     }
                 } else {
 #pragma unroll
                     for (int i = 0; i < 32; i++)
-                        if (c + i < mp) __stcg(mine + (c + i) * BM, __uint_as_float(r[i]));
+                        if (c + i < mp) __stcg(mine + (c + i) * BM, r[i]);
                 }
             }
             tc_fence_before();
@@ -1187,7 +1279,7 @@ struct MapKey {
     uint64_t inner, rows, count, ld;  // ld: row pitch in elements (2-D) or distance between stacked matrices (3-D)
     uint32_t box_inner, box_rows;
     uint32_t kind;                    // 0: bytes, 2-D; 1: BF16, 2-D, 128-byte swizzle; 2: BF16, 3-D stack, 128-byte swizzle;
-                                      // 3: bytes, 2-D, 64-byte swizzle
+                                      // 3: bytes, 2-D, 64-byte swizzle; 4: bytes, 2-D, 128-byte swizzle
     uint32_t pad;
 };
 LruCache<MapKey, CUtensorMap, 64> g_map_cache;
@@ -1212,19 +1304,20 @@ bool encode_map(const MapKey& k, CUtensorMap* map)
     cuuint32_t estr[2] = {1, 1};
     return fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(k.ptr), dims,
               strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-              bf16 ? CU_TENSOR_MAP_SWIZZLE_128B : (k.kind == 3 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE),
+              (bf16 || k.kind == 4) ? CU_TENSOR_MAP_SWIZZLE_128B : (k.kind == 3 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE),
               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 // 2-D tensor [rows][ld elements] with a box of box_inner x box_rows elements, zero fill out of bounds.
-// bf16 = false: bytes, no swizzle.  bf16 = true: 16-bit elements, 128-byte swizzle (box_inner must be 64).
+// bf16 = false: bytes, with no swizzle or the 64- or 128-byte one (box_inner at most that many bytes).  bf16 = true: 16-bit
+// elements, 128-byte swizzle (box_inner must be 64).
 bool make_map(CUtensorMap* map, const void* ptr, uint64_t inner, uint64_t rows, uint64_t ld, uint32_t box_inner, uint32_t box_rows,
-              bool bf16 = false, bool bytes_swizzle64 = false)
+              bool bf16 = false, uint32_t bytes_swizzle = 0)
 {
     MapKey k;
     std::memset(&k, 0, sizeof k);
     k.ptr = ptr; k.inner = inner; k.rows = rows; k.count = 1; k.ld = ld; k.box_inner = box_inner; k.box_rows = box_rows;
-    k.kind = bf16 ? 1u : (bytes_swizzle64 ? 3u : 0u);
+    k.kind = bf16 ? 1u : (bytes_swizzle == 64 ? 3u : (bytes_swizzle == 128 ? 4u : 0u));
     return g_map_cache.lookup_or_make(k, map, encode_map);
 }
 
@@ -1358,7 +1451,7 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t
     CUtensorMap map_a, map_w;
     // ([M,K] activations: 64-byte rows with the 64-byte swizzle, read row-wise by the decode warps of the fused kernel)
     const bool ok_a = a_is_km ? make_map(&map_a, Aq, (uint64_t)M, (uint64_t)K, (uint64_t)lda, BM, BK)
-                              : make_map(&map_a, Aq, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BK, BM, false, true);
+                              : make_map(&map_a, Aq, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BK, BM, false, 64);
     if (!ok_a) return HIF8_ERR_CUDA;
     // byte tiles of one CTA of a pair: 128 rows of A, 128 of the 256 columns of W
     const bool ok_w = w_is_nk ? make_map(&map_w, Wq, (uint64_t)K, (uint64_t)N, (uint64_t)ldw, BK, BN / 2)
@@ -1375,33 +1468,35 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t
     const long long tiles2 = (long long)((M + 2 * BM - 1) / (2 * BM)) * p.tiles_n;
     if (tiles2 > 0x3FFFFFFF) return HIF8_ERR_SHAPE;
     cudaStream_t st = (cudaStream_t)stream;
-    if (cudaMemsetAsync(workspace, 0, 4, st) != cudaSuccess) return HIF8_ERR_CUDA;
     note_status_word(st, reinterpret_cast<const int*>(workspace));
 
     int sm_count = 0;
     if (!gemm_kernels_ready(dev, &sm_count)) return HIF8_ERR_CUDA;
+    // the status word is cleared on the stream before the kernels; the narrow path clears its tickets in the same operation
+    size_t clear_bytes = 4;
 
     // Narrow products: the weight-streaming kernel, whatever the workspace
     if (!a_is_km && M <= kNarrowMaxM) {
         const int mp = (M + 15) & ~15;
         CUtensorMap map_act, map_ws;
-        if (!make_map(&map_act, Aq, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BK, (uint32_t)mp)) return HIF8_ERR_CUDA;
-        const bool okn = w_is_nk ? make_map(&map_ws, Wq, (uint64_t)K, (uint64_t)N, (uint64_t)ldw, BK, BM)
-                                 : make_map(&map_ws, Wq, (uint64_t)N, (uint64_t)K, (uint64_t)ldw, BM, BK);
+        if (!make_map(&map_act, Aq, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BK2, (uint32_t)mp)) return HIF8_ERR_CUDA;
+        // ([N,K] weights: 64-byte rows with the 64-byte swizzle, read row-wise and decoded into tensor memory)
+        const bool okn = w_is_nk ? make_map(&map_ws, Wq, (uint64_t)K, (uint64_t)N, (uint64_t)ldw, BK2, BM, false, 128)
+                                 : make_map(&map_ws, Wq, (uint64_t)N, (uint64_t)K, (uint64_t)ldw, BM, BK2);
         if (!okn) return HIF8_ERR_CUDA;
-        const long long slabs = (N + BM - 1) / BM, num_kb = (K + BK - 1) / BK;
+        const long long slabs = (N + BM - 1) / BM, num_pb = (K + BK2 - 1) / BK2;  // pair blocks: two k-blocks
         NarrowPlan plan{};
-        plan.total = slabs * num_kb;
+        plan.total = slabs * num_pb;
         // One CTA per SM, equal k-block ranges, when the workspace holds the partial sums of the slabs that a range
         // boundary cuts; otherwise one CTA per slab.
         long long grid = slabs;
         {
-            // aim at eight or more k-blocks per CTA, but never fewer CTAs than the per-slab grid would keep busy
-            long long g = plan.total / 8 < sm_count ? plan.total / 8 : sm_count;
+            // aim at four or more pair blocks per CTA, but never fewer CTAs than the per-slab grid would keep busy
+            long long g = plan.total / 4 < sm_count ? plan.total / 4 : sm_count;
             const long long floor_g = slabs < sm_count ? slabs : sm_count;
             if (g < floor_g) g = floor_g;
             const long long per = plan.total / g;
-            const long long pmax = (num_kb + per - 1) / per + 1;
+            const long long pmax = (num_pb + per - 1) / per + 1;
             const size_t ticket_bytes = (((size_t)slabs * kEpiWarps * 4) + 255) & ~(size_t)255;
             const size_t part_bytes = (size_t)slabs * pmax * mp * BM * 4;
             if (g != slabs && workspace_bytes >= kGemmWorkspaceBytes + ticket_bytes + part_bytes && !(reinterpret_cast<uintptr_t>(workspace) & 255)) {
@@ -1410,16 +1505,18 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t
                 plan.part = reinterpret_cast<float*>(wsb + ticket_bytes);
                 plan.pmax = (int)pmax;
                 grid = g;
-                if (cudaMemsetAsync(plan.tickets, 0, ticket_bytes, st) != cudaSuccess) return HIF8_ERR_CUDA;
+                clear_bytes = kGemmWorkspaceBytes + ticket_bytes;  // the tickets follow the status block
             }
         }
         if (grid > 0x7FFFFFFFll) return HIF8_ERR_SHAPE;
-        if (w_is_nk) hif8_gemm_narrow_kernel<true><<<(unsigned)grid, kThreads, kSmemBytesN, st>>>(map_act, map_ws, p, mp, plan);
-        else hif8_gemm_narrow_kernel<false><<<(unsigned)grid, kThreads, kSmemBytesN, st>>>(map_act, map_ws, p, mp, plan);
+        if (cudaMemsetAsync(workspace, 0, clear_bytes, st) != cudaSuccess) return HIF8_ERR_CUDA;
+        if (w_is_nk) hif8_gemm_narrow_kernel<true><<<(unsigned)grid, kThreadsN, kSmemBytesN, st>>>(map_act, map_ws, p, mp, plan);
+        else hif8_gemm_narrow_kernel<false><<<(unsigned)grid, kThreadsN, kSmemBytesN, st>>>(map_act, map_ws, p, mp, plan);
         g_launches.fetch_add(1, std::memory_order_relaxed);
         return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
     }
 
+    if (cudaMemsetAsync(workspace, 0, clear_bytes, st) != cudaSuccess) return HIF8_ERR_CUDA;
     // Decode-once path: with room for both operands as BF16 in the workspace (and contiguous operands), each HiF8
     // byte is decoded exactly once by the conversion kernel and the tensor-core kernel reads BF16 tiles through TMA.
     // Otherwise the fused kernel decodes the byte tiles of every CTA in shared memory.
