@@ -402,7 +402,10 @@ def extra_results(H, torch, hbm_peak, tf_peak, peak_kind):
         byt = K * N + Mn * K + 2 * Mn * N
         st = timed(lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, Cn, N, H.BF16, Mn, N, K, se[0:1], se[1:2], gws, gws_b), 20)
         st_s = timed(lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, Cn, N, H.BF16, Mn, N, K, se[0:1], se[1:2], gws, 256), 20)
-        d = hbm(st, byt, us=st["ms"] * 1e3, us_one_cta_per_slab=st_s["ms"] * 1e3, device_status=H.hif8_last_device_status())
+        # the same bytes read as an [N,K] weight (the layout of a stored checkpoint; values differ, time does not depend on them)
+        st_nk = timed(lambda r: H.hif8_gemm(Aq, K, Wq, K, 1, Cn, N, H.BF16, Mn, N, K, se[0:1], se[1:2], gws, gws_b), 20)
+        d = hbm(st, byt, us=st["ms"] * 1e3, us_one_cta_per_slab=st_s["ms"] * 1e3, us_weights_as_NK=st_nk["ms"] * 1e3,
+                device_status=H.hif8_last_device_status())
         d["frac_of_hbm"] = d["frac"]
         narrow[f"M={Mn}"] = d
         row(f"gemm_narrow_{Mn}x28672x8192", d, "hbm (weight bytes)")
@@ -446,7 +449,7 @@ def run_case(case, reps):
     2^25 log-uniform values in every rounding mode; transpose_bf16: BF16 8192^2 flat and transposed-store encode, TA and
     HR; gemm: HiF8 GEMM 4096 x 7168 x 4096 on the decode-once and the fused path (gemm_fused: the fused path only);
     gemm_forms: the four operand layouts on the decode-once path; gemm_narrow: 16 x 8192 x 8192 with weights as [K,N] and
-    [N,K]; channel_bf16: per-channel scaled encode of a BF16 8192 x 14336 weight by column and by row, plus the overflow
+    [N,K] (equal ranges of the weight per SM); channel_bf16: per-channel scaled encode of a BF16 8192 x 14336 weight by column and by row, plus the overflow
     check.  Inputs are seeded device-side random tensors."""
     import torch
     import paper_2409_16626_b200 as H
@@ -506,9 +509,11 @@ def run_case(case, reps):
         A = torch.randint(8, 100, (M * K,), dtype=torch.uint8, device="cuda", generator=g)
         Wt = torch.randint(8, 100, (K * N,), dtype=torch.uint8, device="cuda", generator=g)
         C = torch.zeros(M, N, dtype=torch.bfloat16, device="cuda")
+        big = H.hif8_workspace_bytes(H.WS_GEMM, M * K + K * N)
+        gws = torch.empty(big, dtype=torch.uint8, device="cuda")
         for r in range(reps):
-            H.hif8_gemm(A, K, Wt, N, 0, C, N, H.BF16, M, N, K, None, None, ws, 256)
-            H.hif8_gemm(A, K, Wt, K, 1, C, N, H.BF16, M, N, K, None, None, ws, 256)
+            H.hif8_gemm(A, K, Wt, N, 0, C, N, H.BF16, M, N, K, None, None, gws, big)
+            H.hif8_gemm(A, K, Wt, K, 1, C, N, H.BF16, M, N, K, None, None, gws, big)
     elif case == "gemm_forms":
         M, N, K = 4096, 7168, 4096
         A = torch.randint(8, 100, (M * K,), dtype=torch.uint8, device="cuda", generator=g)

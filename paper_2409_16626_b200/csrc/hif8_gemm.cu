@@ -716,7 +716,7 @@ constexpr uint32_t kNwW8 = BM * BK, kNwA8 = kNarrowMaxM * BK;          // byte t
 constexpr uint32_t kNwABf = kNarrowMaxM * BK * 2;  // activation operand tile per stage: 8 KiB (the weights go to tensor memory)
 // A copy brings two k-blocks (a "pair block": 128 bytes of k) of weights and of activations: issuing a tile copy costs
 // its thread a few hundred cycles whatever the size, and with one copy of each kind per k-block that thread set the pace.
-// Four stages of 16 KiB + 8 KiB: 64 KiB of weights in flight per SM.
+// Four stages of 16 KiB + 8 KiB: 64 KiB of weights in flight per SM (a fifth stage changed nothing).
 constexpr int kNwByteStages = 4, BK2 = 2 * BK;
 // Operand stages (32 tensor-memory columns of weights + 8 KiB of activations in shared memory each): two per group, so
 // that a group starts its next k-block without waiting for the MMAs of its previous one
