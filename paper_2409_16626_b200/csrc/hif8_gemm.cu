@@ -1037,15 +1037,18 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
 // Decode-once path: operands already decoded to BF16 (by the conversion kernels of this library, into the caller's
 // workspace).  Persistent kernel on CTA pairs (cta_group::2), 64-wide k-blocks.
 //   warps 0-3  epilogue (TMEM -> global), overlapped with the next tile through two TMEM accumulators
-//   warp  4    TMA producer: BF16 tiles land directly in the 128-byte-swizzled operand layout
+//   warp  4    TMA producer of the A tiles: BF16 tiles land directly in the 128-byte-swizzled operand layout
 //   warp  5    MMA issuer
+//   warp  6    TMA producer of the W tiles (issuing a tile copy costs its thread about 200 cycles; one thread issuing the
+//              two or three copies of a k-block, with its waits, took longer than the 512 cycles of the k-block's MMAs)
 // A cluster of two CTAs on two SMs computes one 256 x 256 tile: each CTA stages its own 128 rows of A and its own 128
 // columns of W (so the tensor core reads half as many operand bytes per SM and flop as with one CTA per tile, which is
 // what bounds a one-CTA kernel), both accumulate their 128 rows in their own TMEM.  The even CTA of the pair (the
 // leader) issues every tcgen05.mma; its commits arrive on the barriers of both CTAs.  TMA copies of both CTAs complete
 // on the leader's "full" barrier (no multicast loads).
 // ---------------------------------------------------------------------------------------------------------
-constexpr int kThreadsP = 6 * 32;
+constexpr int kThreadsP = 7 * 32;
+constexpr int kTmaWarpW = 6;
 constexpr int kStages2 = 6;
 constexpr uint32_t kStageBytes2 = kABfBytes + kBBfBytes;            // 32 KiB per CTA and stage
 struct SmemLayout2 {
@@ -1098,34 +1101,37 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    if (warp == kTmaWarp) {
+    if (warp == kTmaWarp || warp == kTmaWarpW) {
         if (lane == 0) {
-            long long it = 0, issued = 0;
-            bool ok = true;
+            const bool loads_a = warp == kTmaWarp;
+            long long issued = 0;
+            int s = 0;            // stage of the next k-block
+            uint32_t ph = 0;      // parity of the round the ring is in
+            bool ok = true, wrapped = false;
             for (int t = pair_id; t < tiles && ok; t += pairs) {
                 int tile_m, tile_n;
                 const int b = t / tiles_one, ia = b / nb, iw = b - ia * nb;
                 tile_coords(t - b * tiles_one, tiles_m2, tiles_n2, tile_m, tile_n);
                 const int m0 = tile_m * 2 * BM + (int)rank * BM, n0 = tile_n * BN + (int)rank * (BN / 2);
-                for (int kb = 0; kb < num_kb; kb++, it++) {
-                    const int s = (int)(it % kStages2);
-                    const long long round = it / kStages2;
-                    if (round > 0) ok = mbar_wait(bar_empty(s), (uint32_t)((round - 1) & 1), abort_flag, p.status, 21);
+                for (int kb = 0; kb < num_kb; kb++) {
+                    if (wrapped) ok = mbar_wait(bar_empty(s), ph ^ 1u, abort_flag, p.status, 21);  // the previous round's use of the stage
                     if (!ok || *abort_flag) { ok = false; break; }
                     const uint32_t dst_a = base + s * kStageBytes2, dst_b = dst_a + kABfBytes;
                     const uint32_t full = map_to_cta(bar_full(s), 0);
-                    if (leader) mbar_arrive_expect_tx(bar_full(s), 2 * kStageBytes2);  // bytes of both CTAs
-                    tma_load_3d_pair(dst_a, &map_a, kb * BK, m0, ia, full);
-                    if (W_IS_NK) tma_load_3d_pair(dst_b, &map_w, kb * BK, n0, iw, full);
+                    if (loads_a) {
+                        if (leader) mbar_arrive_expect_tx(bar_full(s), 2 * kStageBytes2);  // bytes of both CTAs, both operands
+                        tma_load_3d_pair(dst_a, &map_a, kb * BK, m0, ia, full);
+                    } else if (W_IS_NK) tma_load_3d_pair(dst_b, &map_w, kb * BK, n0, iw, full);
                     else {
 #pragma unroll
                         for (int c = 0; c < BN / 2 / 64; c++)
                             tma_load_3d_pair(dst_b + c * 8192, &map_w, n0 + c * 64, kb * BK, iw, full);
                     }
-                    issued = it + 1;
+                    issued++;
+                    if (++s == kStages2) { s = 0; ph ^= 1u; wrapped = true; }
                 }
             }
-            if (*abort_flag && leader) {  // let copies in flight land (their completions are counted on the leader)
+            if (*abort_flag && leader && loads_a) {  // let copies in flight land (their completions are counted on the leader)
                 for (long long j = issued > kStages2 ? issued - kStages2 : 0; j < issued; j++) {
                     const unsigned long long t0 = global_ns();
                     while (!mbar_try_wait(bar_full((int)(j % kStages2)), (uint32_t)((j / kStages2) & 1)) &&
@@ -1138,8 +1144,8 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
             // M = 256 over the pair, N = 256
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((W_IS_NK ? 0u : 1u) << 16) |
                                    ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
-            long long it = 0;
-            int local = 0;
+            int local = 0, s = 0;
+            uint32_t ph = 0;
             bool ok = true;
             for (int t = pair_id; t < tiles && ok; t += pairs, local++) {
                 const int acc = local & 1, use = local >> 1;
@@ -1147,9 +1153,8 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * 256;
-                for (int kb = 0; kb < num_kb; kb++, it++) {
-                    const int s = (int)(it % kStages2);
-                    ok = mbar_wait(bar_full(s), (uint32_t)((it / kStages2) & 1), abort_flag, p.status, 23);
+                for (int kb = 0; kb < num_kb; kb++) {
+                    ok = mbar_wait(bar_full(s), ph, abort_flag, p.status, 23);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t a_addr = base + s * kStageBytes2, b_addr = a_addr + kABfBytes;
@@ -1161,6 +1166,7 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                         tc_mma_bf16_pair(d_tmem, da, db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
                     }
                     tc_commit_pair(bar_empty(s));
+                    if (++s == kStages2) { s = 0; ph ^= 1u; }
                 }
                 if (ok) tc_commit_pair(bar_acc_full(acc));
             }
