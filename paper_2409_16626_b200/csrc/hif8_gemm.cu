@@ -378,7 +378,11 @@ __device__ __forceinline__ void store_chunk(const GemmParams& p, int row, int co
                        make_float4(__uint_as_float(r[4 * i]) * f1 * f2 + c[i].x, __uint_as_float(r[4 * i + 1]) * f1 * f2 + c[i].y,
                                    __uint_as_float(r[4 * i + 2]) * f1 * f2 + c[i].z, __uint_as_float(r[4 * i + 3]) * f1 * f2 + c[i].w));
         } else {
-            for (int i = 0; i < 32 && col + i < p.N; i++) out[i] = __uint_as_float(r[i]) * f1 * f2 + (p.accumulate ? out[i] : 0.f);
+            // (every index a compile-time constant: a loop that stops at the ragged edge would index the chunk by a
+            // variable and put it, for all paths, into local memory -- which has next to no L1 behind it in these kernels)
+#pragma unroll
+            for (int i = 0; i < 32; i++)
+                if (col + i < p.N) out[i] = __uint_as_float(r[i]) * f1 * f2 + (p.accumulate ? out[i] : 0.f);
         }
     } else {
         unsigned short* out = reinterpret_cast<unsigned short*>(p.C) + (long long)row * p.ldc + col;
@@ -410,7 +414,9 @@ __device__ __forceinline__ void store_chunk(const GemmParams& p, int row, int co
                        make_uint4(h[i] | (h[i + 1] << 16), h[i + 2] | (h[i + 3] << 16),
                                   h[i + 4] | (h[i + 5] << 16), h[i + 6] | (h[i + 7] << 16)));
         } else {
-            for (int i = 0; i < 32 && col + i < p.N; i++) out[i] = (unsigned short)h[i];
+#pragma unroll
+            for (int i = 0; i < 32; i++)
+                if (col + i < p.N) out[i] = (unsigned short)h[i];
         }
     }
 }
@@ -666,8 +672,16 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(map_to_cta(bar_bf_full(sb), 0));  // the leader's MMAs read both CTAs' operands
         }
-    } else {
-        // ------------------------------------------------------------------ epilogue warps 0-3 (each CTA drains its rows)
+    }
+    if (warp != kTmaWarp && warp != kMmaWarp) {
+        // ------------------------------------------------------------------ epilogue (each CTA drains its rows)
+        // Warps 0-3 and, once their k-blocks are done, the sixteen decode warps: a warp reaches the quarter (warp % 4) of
+        // the tensor-memory lanes, so every quarter has five warps, which share its eight 32-column chunks (the drain is
+        // not overlapped with anything: with four warps it took a tenth of the tile's time).
+        const int quarter = warp & 3;
+        const int share = warp < kEpiWarps ? 0 : (warp - quarter) / 4 - (quarter < 2 ? 1 : 0);  // 0..4 within the quarter
+        static_assert(kEpiWarps == 4 && kTmaWarp == 4 && kMmaWarp == 5 && kFirstDecodeWarp == 6 && kDecodeWarps == 16,
+                      "five warps per lane quarter: w, and w + 4k without the two single-thread warps");
         const bool ok = mbar_wait(bar_acc_full, 0, abort_flag, p.status, 5);
         if (ok) {
             tc_fence_after();
@@ -675,11 +689,11 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             const int s = p.d_sw_channel ? 0 : -(sa + (p.d_sw ? *p.d_sw : 0));
             const int s1 = s / 2, s2 = s - s1;  // |s1|, |s2| <= 126: two exact power-of-two factors
             const float f1 = __uint_as_float((uint32_t)(s1 + 127) << 23), f2 = __uint_as_float((uint32_t)(s2 + 127) << 23);
-            const int row = m0 + warp * 32 + lane;
+            const int row = m0 + quarter * 32 + lane;
 #pragma unroll 1
-            for (int c = 0; c < BN; c += 32) {
+            for (int c = share * 32; c < BN; c += 5 * 32) {
                 uint32_t r[32];
-                tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(warp * 32) << 16) + c, r);
+                tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + c, r);
                 tmem_ld_wait();
                 if (p.d_sw_channel) apply_channel_scale(p, n0 + c, lane, sa, r);
                 store_chunk(p, row, n0 + c, r, f1, f2);
@@ -1216,9 +1230,12 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
                                 err_acc += d0 * d0 + d1 * d1 + d2 * d2 + d3 * d3;
                             }
                         } else {
-                            for (int i = 0; i < 32 && col + i < p.N; i++) {
-                                const double d = (double)(__uint_as_float(r[i]) * f1 * f2) - (double)__ldg(ref + i);
-                                err_acc += d * d;
+#pragma unroll
+                            for (int i = 0; i < 32; i++) {  // (constant indices: see store_chunk)
+                                if (col + i < p.N) {
+                                    const double d = (double)(__uint_as_float(r[i]) * f1 * f2) - (double)__ldg(ref + i);
+                                    err_acc += d * d;
+                                }
                             }
                         }
                     }
