@@ -400,23 +400,21 @@ __device__ __forceinline__ void store_chunk(const GemmParams& p, int row, int co
                 for (int i = 0; i < 32; i++) h[i] = (col + i < p.N) ? (uint32_t)out[i] << 16 : 0u;
             }
         }
+        uint32_t pk[16];  // two BF16 per word, rounded to nearest even by the conversion instruction (a NaN stays a NaN)
 #pragma unroll
-        for (int i = 0; i < 32; i++) {
-            float v = __uint_as_float(r[i]) * f1 * f2;
-            if (p.accumulate) v += __uint_as_float(h[i]);
-            uint32_t u = __float_as_uint(v);
-            h[i] = (v != v) ? 0x7FC0u : ((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);  // round to nearest even
+        for (int i = 0; i < 32; i += 2) {
+            float v0 = __uint_as_float(r[i]) * f1 * f2, v1 = __uint_as_float(r[i + 1]) * f1 * f2;
+            if (p.accumulate) { v0 += __uint_as_float(h[i]); v1 += __uint_as_float(h[i + 1]); }
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk[i >> 1]) : "f"(v1), "f"(v0));  // first source -> upper half
         }
         if (full) {
 #pragma unroll
-            for (int i = 0; i < 32; i += 8)
-                __stcs(reinterpret_cast<uint4*>(out + i),
-                       make_uint4(h[i] | (h[i + 1] << 16), h[i + 2] | (h[i + 3] << 16),
-                                  h[i + 4] | (h[i + 5] << 16), h[i + 6] | (h[i + 7] << 16)));
+            for (int i = 0; i < 16; i += 4)
+                __stcs(reinterpret_cast<uint4*>(out + 2 * i), make_uint4(pk[i], pk[i + 1], pk[i + 2], pk[i + 3]));
         } else {
 #pragma unroll
             for (int i = 0; i < 32; i++)
-                if (col + i < p.N) out[i] = (unsigned short)h[i];
+                if (col + i < p.N) out[i] = (unsigned short)(pk[i >> 1] >> (16 * (i & 1)));
         }
     }
 }
@@ -966,8 +964,9 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
                 } else {
                     unsigned short* out = reinterpret_cast<unsigned short*>(p.C) + (long long)m * p.ldc + n;
                     if (p.accumulate) v += __uint_as_float((uint32_t)*out << 16);
-                    const uint32_t u = __float_as_uint(v);
-                    *out = (unsigned short)((v != v) ? 0x7FC0u : ((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16));
+                    unsigned short b;
+                    asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(b) : "f"(v));  // round to nearest even; a NaN stays a NaN
+                    *out = b;
                 }
             };
             // contributors of slab j are the CTAs owner(first pair block) .. owner(last pair block);
