@@ -182,11 +182,13 @@ def test_bounded_wait_gives_up_and_reports_without_disturbing_the_device():
 @pytest.mark.parametrize("c_dtype", [H.F32, H.BF16])
 @pytest.mark.parametrize("staged", [False, True])
 @pytest.mark.parametrize("shape", [(1, 256, 64), (16, 1008, 272), (17, 640, 1040), (33, 128, 16), (64, 400, 208), (48, 2064, 4096),
-                                   (8, 304, 8192), (20, 912, 1472), (64, 1296, 2048)])
+                                   (8, 304, 8192), (20, 912, 1472), (64, 1296, 2048), (16, 1168, 2432), (40, 1168, 2368)])
 def test_gemm_narrow_products(shape, c_dtype, w_is_nk, staged):
     # M <= 64: the weight-streaming kernel (weights as the 128-row tensor-core operand, C accumulated transposed).
-    # staged: with a workspace for partial sums the (slab, k-block) pairs are dealt out in equal contiguous ranges, so
-    # slabs are cut (the last three shapes: 16, ~3 and 4 contributors per slab) and summed from per-contributor slices
+    # staged: with a workspace for partial sums the (slab, two-k-block unit) pairs are dealt out in equal contiguous ranges, so
+    # slabs are cut (16, ~3 and 4 contributors per slab) and summed from per-contributor slices.  The last two shapes have 19
+    # units per slab against ranges of 4.04 units: range and slab boundaries never line up, segments come as short as one
+    # unit (fewer k-blocks than MMA-issuing threads: four for M <= 32, two above), and K = 2368 ends in half a unit.
     M, N, K = shape
     N16 = (N + 15) // 16 * 16
     Aq = W.random_codes((M, K), seed=M + K)
