@@ -419,6 +419,32 @@ __device__ __forceinline__ void store_chunk(const GemmParams& p, int row, int co
     }
 }
 
+// The same chunk, descaled and rounded to BF16, into a staging tile in shared memory from which a tile store writes C:
+// boxes of 64 columns x 128 rows in the 128-byte-swizzled layout of the tensor map (16-byte piece j of row r sits at
+// piece j ^ (r % 8) of its 128-byte line; lines of eight rows form 1024-byte atoms).  `piece0` = first 16-byte piece of
+// the chunk within its row of the box (0 or 4).  A thread's four stores hit four different pieces; the eight rows of an
+// atom hit eight different ones: no bank conflicts.
+__device__ __forceinline__ void stage_chunk_bf16(uint32_t box, int row, int piece0, const uint32_t (&r)[32], float f1, float f2)
+{
+    const uint32_t line = box + (uint32_t)(row >> 3) * 1024u + (uint32_t)(row & 7) * 128u;
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+        uint32_t pk[4];
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+            const float v0 = __uint_as_float(r[8 * i + 2 * j]) * f1 * f2, v1 = __uint_as_float(r[8 * i + 2 * j + 1]) * f1 * f2;
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk[j]) : "f"(v1), "f"(v0));
+        }
+        sts_v4(line + ((uint32_t)((piece0 + i) ^ (row & 7)) << 4), make_uint4(pk[0], pk[1], pk[2], pk[3]));
+    }
+}
+// tile store shared -> global (clipped at the edges of the matrix); the caller commits and waits for the group
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+
 // Per-channel weight scales: multiply column col + i of the chunk by 2^-(sa + sw[col + i]).  Lane L fetches the
 // exponent of column col + L once; every lane then walks the 32 columns of its own row.
 __device__ __forceinline__ void apply_channel_scale(const GemmParams& p, int col, int lane, int sa, uint32_t (&r)[32])
@@ -510,7 +536,8 @@ struct FusedSmem {
 
 template <bool A_IS_KM, bool W_IS_NK>
 __global__ void __launch_bounds__(kThreads, 1)
-hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w, const GemmParams p)
+hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
+                 const __grid_constant__ CUtensorMap map_c, const GemmParams p)
 {
     extern __shared__ unsigned char smem_raw[];
     constexpr int kLutShift = (A_IS_KM || !kWideLut) ? 7 : 8;
@@ -694,7 +721,22 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + c, r);
                 tmem_ld_wait();
                 if (p.d_sw_channel) apply_channel_scale(p, n0 + c, lane, sa, r);
-                store_chunk(p, row, n0 + c, r, f1, f2);
+                // (the operand and byte stages are idle once the accumulator is complete: slot c / 64 stages box c / 64)
+                if (!A_IS_KM && p.c_by_tma) stage_chunk_bf16(plan.slot(c >> 6), quarter * 32 + lane, (c & 63) >> 3, r, f1, f2);
+                else store_chunk(p, row, n0 + c, r, f1, f2);
+            }
+        }
+        if (!A_IS_KM && p.c_by_tma) {
+            // Stores of 16 bytes per lane to 32 different rows made the drain as slow as one L2 transaction per clock allows
+            // (4096 of them per CTA); four tile stores write whole lines instead.  All twenty warps meet (named barrier 1),
+            // then one thread issues the stores and waits until shared memory has been read.
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            asm volatile("bar.sync 1, %0;" ::"n"((kEpiWarps + kDecodeWarps) * 32) : "memory");
+            if (threadIdx.x == 0 && ok && !*abort_flag) {
+#pragma unroll
+                for (int j = 0; j < BN / 64; j++) tma_store_2d(&map_c, plan.slot(j), n0 + j * 64, m0);
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
             }
         }
     }
@@ -1564,10 +1606,14 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
     cudaError_t lrc;
-    if (a_is_km) lrc = w_is_nk ? cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<true, true>, map_a, map_w, p)
-                               : cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<true, false>, map_a, map_w, p);
-    else lrc = w_is_nk ? cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<false, true>, map_a, map_w, p)
-                       : cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<false, false>, map_a, map_w, p);
+    // BF16 results that replace C leave the [M,K]-activation kernel through tile stores (boxes of 64 columns x 128 rows)
+    CUtensorMap map_c = map_a;  // (a valid map in any case; only read when c_by_tma is set)
+    p.c_by_tma = (!a_is_km && c_dtype == HIF8_BF16 && !accumulate) ? 1 : 0;
+    if (p.c_by_tma && !make_map(&map_c, C, (uint64_t)N, (uint64_t)M, (uint64_t)ldc, 64, BM, true)) return HIF8_ERR_CUDA;
+    if (a_is_km) lrc = w_is_nk ? cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<true, true>, map_a, map_w, map_c, p)
+                               : cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<true, false>, map_a, map_w, map_c, p);
+    else lrc = w_is_nk ? cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<false, true>, map_a, map_w, map_c, p)
+                       : cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<false, false>, map_a, map_w, map_c, p);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return (lrc == cudaSuccess && cudaGetLastError() == cudaSuccess) ? HIF8_OK : HIF8_ERR_CUDA;
 }

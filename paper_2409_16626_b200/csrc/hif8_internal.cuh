@@ -24,6 +24,7 @@ struct GemmParams {
     // batch_n = n > 0: n x n products in one launch, A variant ia with W variant iw for product ia * n + iw; d_sa / d_sw
     // are then arrays of n exponents and err_sum an array of n * n sums
     int batch_n;
+    int c_by_tma;             // fused kernel: the BF16 result tile is staged in shared memory and written by tile stores
 };
 
 // C (or the squared error) from operands that are already BF16 in device memory: a_bf [M,K], w_bf [K,N] or (w_is_nk) [N,K],
