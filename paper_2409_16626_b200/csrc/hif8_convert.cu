@@ -176,8 +176,7 @@ __global__ void __launch_bounds__(kThreads) convert_kernel(const ConvParams p, u
             uint32_t word = 0;
             if (MODE == HIF8_RND_SR) {
                 uint4 r = philox4x32_10((uint32_t)(i >> 2), (uint32_t)(i >> 34), k0, k1);
-                const uint32_t rr[4] = {r.x, r.y, r.z, r.w};
-                word = rr[i & 3];
+                word = philox_word(r, (unsigned)i & 3u);
             }
             uint32_t c;
             if constexpr (kPair16) {
@@ -459,8 +458,7 @@ __global__ void __launch_bounds__(kThreads) fq_ta_kernel(const ConvParams p, uns
                 uint32_t T16 = 0u;
                 if (MODE == HIF8_RND_SR) {
                     const uint4 q = philox4x32_10((uint32_t)(i >> 2), (uint32_t)(i >> 34), (uint32_t)p.seed, (uint32_t)(p.seed >> 32));
-                    const uint32_t qq[4] = {q.x, q.y, q.z, q.w};
-                    T16 = qq[i & 3] >> 16;
+                    T16 = philox_word(q, (unsigned)i & 3u) >> 16;
                 }
                 reinterpret_cast<unsigned short*>(p.dst)[i] = (unsigned short)fq_rare<SRC, MODE>(raw, se, p.flags, T16);
             }

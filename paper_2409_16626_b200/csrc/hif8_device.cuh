@@ -158,6 +158,13 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
     return make_uint4(x0, x1, x2, x3);
 }
 
+// word `lane` (0..3) of a Philox block, picked with selects (an array indexed by a variable would live in local memory)
+__device__ __forceinline__ uint32_t philox_word(const uint4& r, unsigned lane)
+{
+    const uint32_t lo = (lane & 1u) ? r.y : r.x, hi = (lane & 1u) ? r.w : r.z;
+    return (lane & 2u) ? hi : lo;
+}
+
 // ------------------------------------------------------------------------------------------------
 // Programmatic dependent launch.  Every kernel here is launched so that it may be scheduled while the previous
 // kernel of the stream is still draining: it signals its own dependents at once (they can only start after all of

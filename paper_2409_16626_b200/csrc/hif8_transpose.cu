@@ -158,8 +158,7 @@ __global__ void __launch_bounds__(kThreads) encode_transpose_scalar_kernel(const
         uint32_t word = 0;
         if (MODE == HIF8_RND_SR) {
             const uint4 q = philox4x32_10((uint32_t)(i >> 2), (uint32_t)(i >> 34), k0, k1);
-            const uint32_t qq[4] = {q.x, q.y, q.z, q.w};
-            word = qq[i & 3];
+            word = philox_word(q, (unsigned)i & 3u);
         }
         p.dst[c * (unsigned long long)p.rows + r] = (uint8_t)encode_one<MODE, SRC>(x, raw, scale, sm.ta, sm.thr, word);
     }
