@@ -196,7 +196,7 @@ def cpu_baseline(sample_elems, legs=True):
 # --------------------------------------------------------------------------------------------------------------
 # Secondary workloads
 # --------------------------------------------------------------------------------------------------------------
-def extra_results(H, torch, hbm_peak, tf_peak, peak_kind):
+def extra_results(H, torch, hbm_peak, tf_peak, peak_kind, tf_sustained=None):
     """Secondary workloads (each with its own roofline fraction): BF16 fake-quant of an LLM-activation tensor,
     gradient-range FP32 encode/decode, and the HiF8-operand GEMM.  Inputs are generated on the device from a
     seeded torch generator with the same recipes as workloads/ (shapes and distributions, not the same bytes).
@@ -208,13 +208,16 @@ def extra_results(H, torch, hbm_peak, tf_peak, peak_kind):
     wsb = H.hif8_workspace_bytes(H.WS_FAKE_QUANT, 0)
     ws = torch.empty(max(wsb, 256), dtype=torch.uint8, device="cuda")
 
-    def timed(fn, reps, repeats=MIN_REPEATS):
-        """`repeats` timed regions of `reps` calls each; median / best / worst per call."""
+    def timed(fn, reps, repeats=MIN_REPEATS, rest_s=0.0):
+        """`repeats` timed regions of `reps` calls each; median / best / worst per call.  rest_s: idle time in front of
+        every region (the tensor-bound legs: a region is then a burst, like the cuBLAS burst figure it is divided by)."""
         for _ in range(3):
             fn(0)
         torch.cuda.synchronize()
         per_call = []
         for _ in range(repeats):
+            if rest_s:
+                time.sleep(rest_s)
             ev0.record()
             for r in range(reps):
                 fn(r)
@@ -230,11 +233,34 @@ def extra_results(H, torch, hbm_peak, tf_peak, peak_kind):
     def tensor(stat, flops, **more):
         return dict(stat, TFLOPs=flops / stat["ms"] / 1e9, frac=flops / stat["ms"] / 1e9 / tf_peak, **more)
 
+    REST = 0.3  # seconds of idle in front of every timed region of a tensor-bound leg
+
+    def sustained(fn, flops, seconds=1.0):
+        """The same call back to back for about `seconds` (under the power cap), against the sustained cuBLAS figure."""
+        fn(0)
+        torch.cuda.synchronize()
+        ev0.record(); fn(0); ev1.record(); torch.cuda.synchronize()
+        n = max(8, int(seconds * 1e3 / max(ev0.elapsed_time(ev1), 1e-3)))
+        ev0.record()
+        for r in range(n):
+            fn(r)
+        ev1.record()
+        torch.cuda.synchronize()
+        ms = ev0.elapsed_time(ev1) / n
+        d = {"ms": ms, "calls": n, "TFLOPs": flops / ms / 1e9}
+        if tf_sustained:
+            d["frac_of_sustained_peak"] = flops / ms / 1e9 / tf_sustained
+        return d
+
     def row(name, d, bound):
         # frac: of the measured peak of the bound; frac_nominal: of 8 TB/s (HBM3e) or 2.25 PFLOP/s (dense BF16)
         nominal = d["frac"] * (tf_peak / 2250.0 if bound == "tensor" else hbm_peak / 8000.0)
         table[name] = {"ms": round(d["ms"], 5), "best_ms": round(d["best_ms"], 5), "frac": round(d["frac"], 4),
                        "frac_nominal": round(nominal, 4), "bound": bound}
+        if "back_to_back" in d:  # about a second of calls in a row, against the sustained cuBLAS figure
+            table[name]["back_to_back_ms"] = round(d["back_to_back"]["ms"], 5)
+            if "frac_of_sustained_peak" in d["back_to_back"]:
+                table[name]["frac_of_sustained_peak"] = round(d["back_to_back"]["frac_of_sustained_peak"], 4)
 
     # ---- small and odd sizes (launch latency, tails): FP32 encode TA + decode, 20 call pairs per graph replay
     small = {}
@@ -370,14 +396,17 @@ def extra_results(H, torch, hbm_peak, tf_peak, peak_kind):
     gws_b = H.hif8_workspace_bytes(H.WS_GEMM, M * K + K * N)
     gws = torch.empty(gws_b, dtype=torch.uint8, device="cuda")
     flops = 2.0 * M * N * K
-    g_once = tensor(timed(lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, C, N, H.BF16, M, N, K, se[0:1], se[1:2], gws, gws_b), 5),
-                    flops, device_status=H.hif8_last_device_status(),
-                    note="whole call: decode of both operands to BF16 workspace + tcgen05 kernel")
-    g_fused = tensor(timed(lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, C, N, H.BF16, M, N, K, se[0:1], se[1:2], gws, 256), 3),
-                     flops, device_status=H.hif8_last_device_status(),
-                     note="no workspace: byte tiles decoded per CTA pair inside the tensor-core kernel")
+    f_once = lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, C, N, H.BF16, M, N, K, se[0:1], se[1:2], gws, gws_b)
+    f_fused = lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, C, N, H.BF16, M, N, K, se[0:1], se[1:2], gws, 256)
+    g_once = tensor(timed(f_once, 5, rest_s=REST), flops, device_status=H.hif8_last_device_status(),
+                    note="whole call: decode of both operands to BF16 workspace + tcgen05 kernel",
+                    back_to_back=sustained(f_once, flops))
+    g_fused = tensor(timed(f_fused, 3, rest_s=REST), flops, device_status=H.hif8_last_device_status(),
+                     note="no workspace: byte tiles decoded per CTA pair inside the tensor-core kernel",
+                     back_to_back=sustained(f_fused, flops))
     ch_se.fill_(int(se[1]))
-    g_chan = tensor(timed(lambda r: H.hif8_gemm_channel_scaled(Aq, K, Wq, N, 0, C, N, H.BF16, M, N, K, se[0:1], ch_se, gws, gws_b), 5),
+    g_chan = tensor(timed(lambda r: H.hif8_gemm_channel_scaled(Aq, K, Wq, N, 0, C, N, H.BF16, M, N, K, se[0:1], ch_se, gws, gws_b), 5,
+                          rest_s=REST),
                     flops, device_status=H.hif8_last_device_status(), note="one weight exponent per output column")
     row("C5_gemm_8192x28672x8192_decode_once", g_once, "tensor")
     row("C5_gemm_8192x28672x8192_fused", g_fused, "tensor")
@@ -385,11 +414,11 @@ def extra_results(H, torch, hbm_peak, tf_peak, peak_kind):
     # backward-pass forms of the same size: dgrad reads the weight as [N,K], wgrad reads A as [K,M] and accumulates in FP32
     bw = {}
     bw["dgrad_form_w_as_[N,K]"] = tensor(
-        timed(lambda r: H.hif8_gemm_ex(Aq, K, 0, Wq, K, 1, C, N, H.BF16, M, N, K, se[0:1], se[1:2], None, 0, gws, gws_b), 5),
+        timed(lambda r: H.hif8_gemm_ex(Aq, K, 0, Wq, K, 1, C, N, H.BF16, M, N, K, se[0:1], se[1:2], None, 0, gws, gws_b), 5, rest_s=REST),
         flops, device_status=H.hif8_last_device_status())
     C32 = torch.zeros(M, N, dtype=torch.float32, device="cuda")
     bw["wgrad_form_a_as_[K,M]_fp32_accumulate"] = tensor(
-        timed(lambda r: H.hif8_gemm_ex(Aq, M, 1, Wq, N, 0, C32, N, H.F32, M, N, K, se[0:1], se[1:2], None, 1, gws, gws_b), 5),
+        timed(lambda r: H.hif8_gemm_ex(Aq, M, 1, Wq, N, 0, C32, N, H.F32, M, N, K, se[0:1], se[1:2], None, 1, gws, gws_b), 5, rest_s=REST),
         flops, device_status=H.hif8_last_device_status())
     del C32
     for k_, v_ in bw.items():
@@ -415,6 +444,8 @@ def extra_results(H, torch, hbm_peak, tf_peak, peak_kind):
     out["gemm_8192x28672x8192"] = {
         "backward_forms": bw, "decode_once_channel_scaled": g_chan, "decode_once": g_once, "fused": g_fused,
         "bound": "tensor", "peak": tf_peak, "peak_kind": f"of {peak_kind} (cuBLAS BF16 burst)", "unit": "TFLOP/s",
+        "timing": f"every timed region starts after {REST} s of idle (bursts, like the peak); back_to_back: about one second of calls "
+                  "in a row under the power cap, against the sustained cuBLAS figure",
         "scale_exps": [int(v) for v in se.cpu()], "output": "bf16"}
     del C, gws, Aq, Wq
 
@@ -905,7 +936,7 @@ def main():
         if world == 1 and not args.no_extra:
             del srcs, codes, backs
             torch.cuda.empty_cache()
-            line["extra"], table = extra_results(H, torch, peak, tf_peak, peak_kind)
+            line["extra"], table = extra_results(H, torch, peak, tf_peak, peak_kind, tf_sustained)
             by_config.update(table)
         if world == 1 and not args.no_cpu_baseline:
             line["cpu_baseline"] = cpu_baseline(1 << 23)
