@@ -127,3 +127,41 @@ def test_config5_gemm_8192x28672x8192(staged):
     tol = tol + 2.0 ** (np.floor(np.log2(np.maximum(np.abs(Cs) + tol, 2.0 ** -126))) - 8)   # + half a BF16 ulp of the result
     err = np.abs(got - Cs)
     assert np.all(err <= tol), f"{np.count_nonzero(err > tol)} outside tolerance, worst ratio {np.max(err / tol):.3g}"
+
+
+@pytest.mark.parametrize("w_is_nk", [0, 1])
+@pytest.mark.parametrize("Mn", [16, 64])
+def test_config5_narrow_products_full_weight(Mn, w_is_nk):
+    # the few-row products of the bench (decode phase of inference): Mn activation rows against the 8192 x 28672 weight, with
+    # the workspace that makes the kernel deal equal ranges of the weight to all SMs (slabs cut between CTAs, four or two
+    # MMA-issuing threads); sampled outputs, every row, against the FP64 oracle
+    N, K = 28672, 8192
+    g = _gen(987 + Mn)
+    a = torch.randn(Mn, K, generator=g, device="cuda").to(torch.bfloat16)
+    w = (torch.randn(K, N, generator=g, device="cuda") * 0.02).to(torch.bfloat16)
+    Aq = torch.empty(Mn * K, dtype=torch.uint8, device="cuda")
+    Wq = torch.empty(K * N, dtype=torch.uint8, device="cuda")
+    se = torch.zeros(2, dtype=torch.int32, device="cuda")
+    wsb = H.hif8_workspace_bytes(H.WS_AMAX_SCALE_ENCODE, 0)
+    ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
+    H.hif8_amax_scale_encode(a, H.BF16, Aq, Mn * K, 14, H.RND_TA, 0, 0, None, None, se[0:1], None, ws, wsb)
+    H.hif8_amax_scale_encode(w, H.BF16, Wq, K * N, 14, H.RND_TA, 0, 0, None, None, se[1:2], None, ws, wsb)
+    del a, w
+    Wdev = Wq.view(K, N).t().contiguous().view(-1) if w_is_nk else Wq
+    C = torch.full((Mn, N), float("nan"), dtype=torch.bfloat16, device="cuda")
+    gb = H.hif8_workspace_bytes(H.WS_GEMM, Mn * K + K * N)
+    gws = torch.empty(gb, dtype=torch.uint8, device="cuda")
+    H.hif8_gemm(Aq, K, Wdev, K if w_is_nk else N, w_is_nk, C, N, H.BF16, Mn, N, K, se[0:1], se[1:2], gws, gb)
+    assert H.hif8_last_device_status() == 0
+    sa, sw = [int(v) for v in se.cpu()]
+    rng = np.random.default_rng(5)
+    # random entries, the last slab, and the columns around a slab boundary that a range boundary cuts
+    cols = np.concatenate([rng.integers(0, N, 40000), np.tile(np.arange(N - 128, N), Mn), np.tile(np.arange(96 * 128 - 64, 96 * 128 + 64), Mn)])
+    rows = np.concatenate([rng.integers(0, Mn, 40000), np.repeat(np.arange(Mn), 128), np.repeat(np.arange(Mn), 128)])
+    Cs, S = O.gemm_entries(Aq.cpu().numpy().reshape(Mn, K), Wq.cpu().numpy().reshape(K, N), False, sa, sw, rows, cols)
+    got = C[torch.from_numpy(rows).cuda(), torch.from_numpy(cols).cuda()].float().cpu().numpy().astype(np.float64)
+    tol = 1e-5 * S
+    tol = tol + 2.0 ** (np.floor(np.log2(np.maximum(np.abs(Cs) + tol, 2.0 ** -126))) - 8)   # + half a BF16 ulp of the result
+    err = np.abs(got - Cs)
+    assert np.all(err <= tol), f"{np.count_nonzero(err > tol)} outside tolerance, worst ratio {np.max(err / tol):.3g}"
+    assert not torch.isnan(C.float()).any()                  # every output was written
