@@ -404,12 +404,17 @@ def extra_results(H, torch, hbm_peak, tf_peak, peak_kind, tf_sustained=None):
     g_fused = tensor(timed(f_fused, 3, rest_s=REST), flops, device_status=H.hif8_last_device_status(),
                      note="no workspace: byte tiles decoded per CTA pair inside the tensor-core kernel",
                      back_to_back=sustained(f_fused, flops))
+    gws_a = H.hif8_workspace_bytes(H.WS_GEMM, M * K)
+    g_aexp = tensor(timed(lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, C, N, H.BF16, M, N, K, se[0:1], se[1:2], gws, gws_a), 3, rest_s=REST),
+                    flops, device_status=H.hif8_last_device_status(),
+                    note="workspace for A alone: A expanded once to BF16, W tiles decoded inside the tensor-core kernel")
     ch_se.fill_(int(se[1]))
     g_chan = tensor(timed(lambda r: H.hif8_gemm_channel_scaled(Aq, K, Wq, N, 0, C, N, H.BF16, M, N, K, se[0:1], ch_se, gws, gws_b), 5,
                           rest_s=REST),
                     flops, device_status=H.hif8_last_device_status(), note="one weight exponent per output column")
     row("C5_gemm_8192x28672x8192_decode_once", g_once, "tensor")
     row("C5_gemm_8192x28672x8192_fused", g_fused, "tensor")
+    row("C5_gemm_8192x28672x8192_A_expanded_W_fused", g_aexp, "tensor")
     row("gemm_8192x28672x8192_channel_scaled", g_chan, "tensor")
     # backward-pass forms of the same size: dgrad reads the weight as [N,K], wgrad reads A as [K,M] and accumulates in FP32
     bw = {}
@@ -442,7 +447,7 @@ def extra_results(H, torch, hbm_peak, tf_peak, peak_kind, tf_sustained=None):
     out["gemm_narrow_Mx28672x8192"] = {"bound": "hbm", "bytes": "K*N weight bytes + M*K + 2*M*N", "shapes": narrow,
                                        "peak": hbm_peak, "peak_kind": f"of {peak_kind}"}
     out["gemm_8192x28672x8192"] = {
-        "backward_forms": bw, "decode_once_channel_scaled": g_chan, "decode_once": g_once, "fused": g_fused,
+        "backward_forms": bw, "decode_once_channel_scaled": g_chan, "decode_once": g_once, "fused": g_fused, "a_expanded_w_fused": g_aexp,
         "bound": "tensor", "peak": tf_peak, "peak_kind": f"of {peak_kind} (cuBLAS BF16 burst)", "unit": "TFLOP/s",
         "timing": f"every timed region starts after {REST} s of idle (bursts, like the peak); back_to_back: about one second of calls "
                   "in a row under the power cap, against the sustained cuBLAS figure",

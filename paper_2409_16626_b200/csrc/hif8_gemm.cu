@@ -499,7 +499,7 @@ constexpr uint32_t kSlotBytes = 16384, kLutBytesWide = 65536, kLutBytesNarrow = 
 static_assert(kBBfBytes == kSlotBytes && kA8Bytes + kB8Bytes == kSlotBytes, "one stage per slot");
 constexpr uint32_t kSmemBytesWide = 227 * 1024;  // the whole opt-in maximum; the kernel checks that its plan fits
 
-template <bool A_IS_KM>
+template <bool FIXED>  // FIXED: the layout of SmemLayout (A operand tiles in shared memory)
 struct FusedSmem {
     uint32_t base, lut, bars, behind;  // shared-window addresses; base is 1024-byte aligned
     int n_front;                       // slots in front of the table
@@ -508,7 +508,7 @@ struct FusedSmem {
     __device__ explicit FusedSmem(uint32_t raw)
     {
         base = (raw + 1023u) & ~1023u;
-        if (A_IS_KM) {
+        if (FIXED) {
             lut = base + SmemLayout::lut; bars = base + SmemLayout::bars; behind = 0; n_front = 0; end = base + SmemLayout::total;
         } else if (!kWideLut) {
             // table with rows of 128 bytes: no alignment to honour, everything in a row: slots, table, barriers
@@ -526,23 +526,29 @@ struct FusedSmem {
         }
     }
     __device__ uint32_t slot(int i) const { return i < n_front ? base + (uint32_t)i * kSlotBytes : behind + (uint32_t)(i - n_front) * kSlotBytes; }
-    __device__ uint32_t a_bf(int s) const { return base + SmemLayout::bf + s * (kABfBytes + kBBfBytes); }                       // A_IS_KM only
-    __device__ uint32_t w_bf(int s) const { return A_IS_KM ? a_bf(s) + kABfBytes : slot(s); }
-    __device__ uint32_t a_u8(int s) const { return A_IS_KM ? base + SmemLayout::u8 + s * (kA8Bytes + kB8Bytes) : slot(kStagesBf + s); }
+    __device__ uint32_t a_bf(int s) const { return base + SmemLayout::bf + s * (kABfBytes + kBBfBytes); }                       // FIXED only
+    __device__ uint32_t w_bf(int s) const { return FIXED ? a_bf(s) + kABfBytes : slot(s); }
+    __device__ uint32_t a_u8(int s) const { return FIXED ? base + SmemLayout::u8 + s * (kA8Bytes + kB8Bytes) : slot(kStagesBf + s); }
+    // staging box j (16 KiB) of the result tile: the operand stages, idle once the accumulator is complete
+    __device__ uint32_t box(int j) const { return FIXED ? base + SmemLayout::bf + (uint32_t)j * kSlotBytes : slot(j); }
     __device__ uint32_t w_u8(int s) const { return a_u8(s) + kA8Bytes; }
     __device__ uint32_t tmem_slot() const { return bars + SmemLayout::n_bars * 8; }
     __device__ uint32_t abort_flag() const { return tmem_slot() + 4; }
 };
 
-template <bool A_IS_KM, bool W_IS_NK>
+// A_MODE 0: A given as [M,K] bytes, decoded into tensor memory.  1: A given as [K,M] bytes, decoded into shared memory
+// (MN-major operand).  2: A already expanded to BF16 [M,K] in the caller's workspace (only W is decoded here): its tiles
+// come by TMA straight into the K-major operand stages, completing on the leader's "operands ready" barrier.
+template <int A_MODE, bool W_IS_NK>
 __global__ void __launch_bounds__(kThreads, 1)
 hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
                  const __grid_constant__ CUtensorMap map_c, const GemmParams p)
 {
     extern __shared__ unsigned char smem_raw[];
-    constexpr int kLutShift = (A_IS_KM || !kWideLut) ? 7 : 8;
-    constexpr int kS8 = A_IS_KM ? kStages8 : kStages8Deep;  // depth of the byte ring
-    const FusedSmem<A_IS_KM> plan(smem_u32(smem_raw));
+    constexpr bool A_IS_KM = A_MODE == 1, A_BF16 = A_MODE == 2, kFixed = A_MODE != 0;
+    constexpr int kLutShift = (kFixed || !kWideLut) ? 7 : 8;
+    constexpr int kS8 = kFixed ? kStages8 : kStages8Deep;  // depth of the byte ring
+    const FusedSmem<kFixed> plan(smem_u32(smem_raw));
     const uint32_t base = plan.base;
     unsigned char* sm = smem_raw - smem_u32(smem_raw);  // generic pointer of shared-window address 0
     {
@@ -578,7 +584,8 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     fill_decode_table<(1 << (kLutShift - 2))>(lut_all, warp, lane, kThreads / 32);  // rows of 1 << kLutShift bytes
     if (threadIdx.x == 0) {
         for (int s = 0; s < kS8; s++) { mbar_init(bar_u8_full(s), 1); mbar_init(bar_u8_empty(s), kGroupWarps); }
-        for (int s = 0; s < kStagesBf; s++) { mbar_init(bar_bf_full(s), 2 * kGroupWarps); mbar_init(bar_bf_empty(s), 1); }
+        // operands ready: both CTAs' decode group, plus (A_BF16) the leader's announcement of the A tile bytes
+        for (int s = 0; s < kStagesBf; s++) { mbar_init(bar_bf_full(s), 2 * kGroupWarps + (A_BF16 ? 1 : 0)); mbar_init(bar_bf_empty(s), 1); }
         mbar_init(bar_acc_full, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -603,12 +610,20 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 if (round > 0 && !mbar_wait(bar_u8_empty(s), (round - 1) & 1, abort_flag, p.status, 1)) break;
                 if (*abort_flag) break;
                 const uint32_t dst_a = plan.a_u8(s), dst_b = plan.w_u8(s);
-                mbar_arrive_expect_tx(bar_u8_full(s), kA8Bytes + kB8Bytes);
+                mbar_arrive_expect_tx(bar_u8_full(s), (A_BF16 ? 0u : kA8Bytes) + kB8Bytes);
                 if (A_IS_KM) tma_load_2d(dst_a, &map_a, m0, kb * BK, bar_u8_full(s));
-                else tma_load_2d(dst_a, &map_a, kb * BK, m0, bar_u8_full(s));
+                else if (!A_BF16) tma_load_2d(dst_a, &map_a, kb * BK, m0, bar_u8_full(s));
                 if (W_IS_NK) tma_load_2d(dst_b, &map_w, kb * BK, nh, bar_u8_full(s));
                 else tma_load_2d(dst_b, &map_w, nh, kb * BK, bar_u8_full(s));
                 issued = kb + 1;
+                if (A_BF16) {
+                    // the BF16 A tile goes straight into operand stage sb, once the MMAs of its previous k-block have read
+                    // it; both CTAs' copies complete on the leader's "operands ready" barrier, which the leader arms
+                    const int sb = kb % kStagesBf, rb = kb / kStagesBf;
+                    if (rb > 0 && !mbar_wait(bar_bf_empty(sb), (rb - 1) & 1, abort_flag, p.status, 6)) break;
+                    if (leader) mbar_arrive_expect_tx(bar_bf_full(sb), 2 * kABfBytes);
+                    tma_load_3d_pair(plan.a_bf(sb), &map_a, kb * BK, m0, 0, map_to_cta(bar_bf_full(sb), 0));
+                }
             }
             if (*abort_flag) {
                 // let the copies already issued land before this CTA's shared memory goes away
@@ -616,6 +631,11 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     const int s = kb % kS8;
                     const unsigned long long t0 = global_ns();
                     while (!mbar_try_wait(bar_u8_full(s), (kb / kS8) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+                }
+                if (A_BF16) {  // (the A tiles complete on a barrier that also counts the decode groups, which have given up:
+                               // their copies get a fixed 50 us instead)
+                    const unsigned long long t0 = global_ns();
+                    while (global_ns() - t0 < 50000ull) {}
                 }
             }
         }
@@ -639,6 +659,8 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                                                 : make_smem_desc(b_addr + kk * 2048, 8192, 1024);
                     if (A_IS_KM) {
                         tc_mma_bf16_pair(tmem_base, make_smem_desc(a_addr + kk * 2048, 8192, 1024), db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
+                    } else if (A_BF16) {
+                        tc_mma_bf16_pair(tmem_base, make_smem_desc(a_addr + kk * 32, 16, 1024), db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
                     } else {
                         // A from tensor memory: stage s, 16 k = 8 columns
                         tc_mma_bf16_pair_a_tmem(tmem_base, tmem_base + kTmemColsAcc + (uint32_t)(s * kTmemAStageCols + kk * 8), db, idesc,
@@ -669,6 +691,11 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 __syncwarp();  // every lane's reads of the byte stage are done: the producer may refill it during the decode
                 if (lane == 0) mbar_arrive(bar_u8_empty(s8));
                 decode_tile_chunks<true, kLutShift>(va, abf, dt, lut);
+            } else if (A_BF16) {
+                // A was expanded beforehand and arrives by TMA: only the W tile is decoded here
+                load_tile_chunks<!W_IS_NK>(b8, dt, vw);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_u8_empty(s8));
             } else {
                 // A [M,K]: this thread owns row (its warp's quarter of the 128 tensor-memory lanes) * 32 + lane.  The byte
                 // tile arrives with the 64-byte TMA swizzle (16-byte chunk j of row r sits at chunk j ^ ((r >> 1) & 3)), so
@@ -691,7 +718,7 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 tmem_st_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + kTmemColsAcc + (uint32_t)(sb * kTmemAStageCols), o);
             }
             decode_tile_chunks<!W_IS_NK, kLutShift>(vw, bbf, dt, lut);
-            if (!A_IS_KM) tmem_st_wait();  // the row is in tensor memory
+            if (A_MODE == 0) tmem_st_wait();  // the row is in tensor memory
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // make the stores visible to the tensor core
             tc_fence_before();
             __syncwarp();
@@ -715,15 +742,26 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             const int s1 = s / 2, s2 = s - s1;  // |s1|, |s2| <= 126: two exact power-of-two factors
             const float f1 = __uint_as_float((uint32_t)(s1 + 127) << 23), f2 = __uint_as_float((uint32_t)(s2 + 127) << 23);
             const int row = m0 + quarter * 32 + lane;
+            // (two loops rather than a branch inside one: the register allocation of each stays that of its own path)
+            if (!A_IS_KM && p.c_by_tma) {
 #pragma unroll 1
-            for (int c = share * 32; c < BN; c += 5 * 32) {
-                uint32_t r[32];
-                tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + c, r);
-                tmem_ld_wait();
-                if (p.d_sw_channel) apply_channel_scale(p, n0 + c, lane, sa, r);
-                // (the operand and byte stages are idle once the accumulator is complete: slot c / 64 stages box c / 64)
-                if (!A_IS_KM && p.c_by_tma) stage_chunk_bf16(plan.slot(c >> 6), quarter * 32 + lane, (c & 63) >> 3, r, f1, f2);
-                else store_chunk(p, row, n0 + c, r, f1, f2);
+                for (int c = share * 32; c < BN; c += 5 * 32) {
+                    uint32_t r[32];
+                    tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + c, r);
+                    tmem_ld_wait();
+                    if (p.d_sw_channel) apply_channel_scale(p, n0 + c, lane, sa, r);
+                    // the operand stages are idle once the accumulator is complete: box c / 64 of the result tile goes there
+                    stage_chunk_bf16(plan.box(c >> 6), quarter * 32 + lane, (c & 63) >> 3, r, f1, f2);
+                }
+            } else {
+#pragma unroll 1
+                for (int c = share * 32; c < BN; c += 5 * 32) {
+                    uint32_t r[32];
+                    tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + c, r);
+                    tmem_ld_wait();
+                    if (p.d_sw_channel) apply_channel_scale(p, n0 + c, lane, sa, r);
+                    store_chunk(p, row, n0 + c, r, f1, f2);
+                }
             }
         }
         if (!A_IS_KM && p.c_by_tma) {
@@ -734,7 +772,7 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             asm volatile("bar.sync 1, %0;" ::"n"((kEpiWarps + kDecodeWarps) * 32) : "memory");
             if (threadIdx.x == 0 && ok && !*abort_flag) {
 #pragma unroll
-                for (int j = 0; j < BN / 64; j++) tma_store_2d(&map_c, plan.slot(j), n0 + j * 64, m0);
+                for (int j = 0; j < BN / 64; j++) tma_store_2d(&map_c, plan.box(j), n0 + j * 64, m0);
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
             }
@@ -1409,10 +1447,11 @@ bool gemm_kernels_ready(int dev, int* sm_count_out)
     const GemmDeviceSetup* s = g_gemm_setup.get(dev, [](int d, GemmDeviceSetup* out) {
         out->rc = cudaSuccess;
         out->sm_count = 0;
-        const void* fused[4] = {(const void*)hif8_gemm_kernel<false, false>, (const void*)hif8_gemm_kernel<false, true>,
-                                (const void*)hif8_gemm_kernel<true, false>, (const void*)hif8_gemm_kernel<true, true>};
+        const void* fused[6] = {(const void*)hif8_gemm_kernel<0, false>, (const void*)hif8_gemm_kernel<0, true>,
+                                (const void*)hif8_gemm_kernel<1, false>, (const void*)hif8_gemm_kernel<1, true>,
+                                (const void*)hif8_gemm_kernel<2, false>, (const void*)hif8_gemm_kernel<2, true>};
         const void* pair[2] = {(const void*)bf16_gemm_pair_kernel<false>, (const void*)bf16_gemm_pair_kernel<true>};
-        for (int i = 0; i < 4 && out->rc == cudaSuccess; i++)  // [M,K] activations (the first two): the wide-table plan
+        for (int i = 0; i < 6 && out->rc == cudaSuccess; i++)  // [M,K] byte activations (the first two): the wide-table plan
             out->rc = cudaFuncSetAttribute(fused[i], cudaFuncAttributeMaxDynamicSharedMemorySize, i < 2 ? kSmemBytesWide : kSmemBytes);
         for (int i = 0; i < 2 && out->rc == cudaSuccess; i++)
             out->rc = cudaFuncSetAttribute(pair[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
@@ -1595,11 +1634,22 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t
         if (rc != HIF8_OK) return rc;
         return launch_bf16_pair_gemm(a_bf, w_bf, w_is_nk, p, st);
     }
+    // In between: room for A alone as BF16 (2 M K bytes; W, usually the larger operand, stays bytes).  A is expanded once
+    // (as [M,K] whichever way it was given) and the fused kernel decodes only its W tiles; W may have any leading dimension.
+    int a_mode = a_is_km ? 1 : 0;
+    if (lda == (a_is_km ? M : K) && workspace_bytes >= kGemmWorkspaceBytes + bytes_a && !(reinterpret_cast<uintptr_t>(workspace) & 255)) {
+        unsigned char* a_bf = reinterpret_cast<unsigned char*>(workspace) + kGemmWorkspaceBytes;
+        const int rc = a_is_km ? decode_transpose_bf16(Aq, a_bf, K, M, st) : hif8_decode(Aq, a_bf, HIF8_BF16, (size_t)M * K, 0, stream);
+        if (rc != HIF8_OK) return rc;
+        // boxes of 64 k x 128 rows in the 128-byte-swizzled operand layout (a stack of one matrix: the pair form of the copy)
+        if (!make_map3(&map_a, a_bf, (uint64_t)K, (uint64_t)M, 1, 0, BK, BM)) return HIF8_ERR_CUDA;
+        a_mode = 2;
+    }
 
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3(2u * (unsigned)tiles2);
     cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = a_is_km ? kSmemBytes : kSmemBytesWide;
+    cfg.dynamicSmemBytes = a_mode == 0 ? kSmemBytesWide : kSmemBytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -1608,12 +1658,14 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t
     cudaError_t lrc;
     // BF16 results that replace C leave the [M,K]-activation kernel through tile stores (boxes of 64 columns x 128 rows)
     CUtensorMap map_c = map_a;  // (a valid map in any case; only read when c_by_tma is set)
-    p.c_by_tma = (!a_is_km && c_dtype == HIF8_BF16 && !accumulate) ? 1 : 0;
+    p.c_by_tma = (a_mode != 1 && c_dtype == HIF8_BF16 && !accumulate) ? 1 : 0;
     if (p.c_by_tma && !make_map(&map_c, C, (uint64_t)N, (uint64_t)M, (uint64_t)ldc, 64, BM, true)) return HIF8_ERR_CUDA;
-    if (a_is_km) lrc = w_is_nk ? cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<true, true>, map_a, map_w, map_c, p)
-                               : cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<true, false>, map_a, map_w, map_c, p);
-    else lrc = w_is_nk ? cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<false, true>, map_a, map_w, map_c, p)
-                       : cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<false, false>, map_a, map_w, map_c, p);
+    if (a_mode == 1) lrc = w_is_nk ? cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<1, true>, map_a, map_w, map_c, p)
+                                   : cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<1, false>, map_a, map_w, map_c, p);
+    else if (a_mode == 2) lrc = w_is_nk ? cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<2, true>, map_a, map_w, map_c, p)
+                                        : cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<2, false>, map_a, map_w, map_c, p);
+    else lrc = w_is_nk ? cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<0, true>, map_a, map_w, map_c, p)
+                       : cudaLaunchKernelEx(&cfg, hif8_gemm_kernel<0, false>, map_a, map_w, map_c, p);
     g_launches.fetch_add(1, std::memory_order_relaxed);
     return (lrc == cudaSuccess && cudaGetLastError() == cudaSuccess) ? HIF8_OK : HIF8_ERR_CUDA;
 }

@@ -24,8 +24,9 @@ def run_gemm(Aq, Wq, w_is_nk, c_dtype, sa=None, sw=None, M=None, N=None, K=None,
     dA, dW = to_dev(Aq), to_dev(Wq)
     ldc = (N + 7) // 8 * 8
     C = torch.full((M, ldc), float("nan"), dtype=torch.float32 if c_dtype == H.F32 else torch.bfloat16, device="cuda")
-    # staged: workspace with room for both operands in BF16 -> decode-once path; else the fused kernel
-    wsb = H.hif8_workspace_bytes(H.WS_GEMM, M * K + K * N) if staged else H.hif8_workspace_bytes(H.WS_GEMM, 0)
+    # staged = True: workspace with room for both operands in BF16 -> decode-once path; "a": room for A alone -> A expanded
+    # once, W decoded inside the tensor-core kernel; False: the fused kernel decodes both
+    wsb = H.hif8_workspace_bytes(H.WS_GEMM, M * K if staged == "a" else M * K + K * N) if staged else H.hif8_workspace_bytes(H.WS_GEMM, 0)
     ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
     dsa = torch.tensor([sa], dtype=torch.int32, device="cuda") if sa is not None else None
     dsw = torch.tensor([sw], dtype=torch.int32, device="cuda") if sw is not None else None
@@ -46,7 +47,7 @@ def check(C, Cstar, S, c_dtype):
     assert not bad.any(), f"{bad.sum()} of {bad.size} outside tolerance; worst ratio {np.max(err / np.maximum(tol, 1e-300)):.3g}"
 
 
-@pytest.mark.parametrize("staged", [False, True])
+@pytest.mark.parametrize("staged", [False, True, "a"])
 @pytest.mark.parametrize("w_is_nk", [0, 1])
 @pytest.mark.parametrize("c_dtype", [H.F32, H.BF16])
 @pytest.mark.parametrize("shape", [(128, 256, 64), (128, 256, 256), (256, 512, 192), (130, 264, 208), (77, 40, 16),
@@ -64,7 +65,7 @@ def test_gemm_small_full_compare(shape, c_dtype, w_is_nk, staged):
     check(C, Cs, S, c_dtype)
 
 
-@pytest.mark.parametrize("staged", [False, True])
+@pytest.mark.parametrize("staged", [False, True, "a"])
 @pytest.mark.parametrize("w_is_nk", [0, 1])
 def test_gemm_one_hot_rows_pin_tile_and_k_indexing(w_is_nk, staged):
     # A picks one k per row (value 1.0): C[m, :] must equal row perm[m] of W exactly
@@ -107,7 +108,7 @@ def test_gemm_specials_propagate():
     Wq = np.full((K, N), 0x08, dtype=np.uint8)
     Aq[3, 5] = 0x80                                           # NaN
     Aq[7, 9] = 0x6F                                           # +Inf
-    for staged in (False, True):
+    for staged in (False, True, "a"):
         C = run_gemm(Aq, Wq, 0, H.F32, staged=staged)
         assert np.all(np.isnan(C[3])) and np.all(np.isposinf(C[7]))
         ok = np.ones(M, bool); ok[[3, 7]] = False
@@ -128,7 +129,7 @@ def test_gemm_medium_scaled_operands_sampled(w_is_nk):
     cols = np.concatenate([rng.integers(0, N, 20000), np.tile(np.arange(256), 128), np.tile(np.arange(N - 256, N), 128)])
     Cs, S = O.gemm_entries(Aq, Wkn, False, sa, sw, rows, cols)
     for c_dtype in (H.F32, H.BF16):
-        for staged in (False, True):
+        for staged in (False, True, "a"):
             C = run_gemm(Aq, np.ascontiguousarray(Wkn.T) if w_is_nk else Wkn, w_is_nk, c_dtype, sa=sa, sw=sw, staged=staged)
             check(C[rows, cols], Cs, S, c_dtype)
 
@@ -147,7 +148,7 @@ def _same_sign_operands(M, N, K, relu_only):
 
 
 @pytest.mark.parametrize("relu_only", [False, True])
-@pytest.mark.parametrize("path", ["fused", "staged", "narrow"])
+@pytest.mark.parametrize("path", ["fused", "staged", "a_expanded", "narrow"])
 def test_gemm_same_sign_operands_k8192(path, relu_only):
     # Section 4.1: activations are GEMM inputs, and activations behind a ReLU are non-negative.  With operands of one
     # sign nothing cancels, S equals |C*|, and 512 sequential FP32 accumulator updates per output must stay inside
@@ -157,7 +158,7 @@ def test_gemm_same_sign_operands_k8192(path, relu_only):
     Cs, S = O.gemm_full(Aq, Wkn, False, sa, sw)
     if not relu_only:
         assert np.allclose(Cs, S, rtol=1e-12)
-    C = run_gemm(Aq, Wkn, 0, H.F32, sa=sa, sw=sw, staged=(path == "staged"))
+    C = run_gemm(Aq, Wkn, 0, H.F32, sa=sa, sw=sw, staged={"staged": True, "a_expanded": "a"}.get(path, False))
     ratio = np.max(np.abs(C - Cs) / (1e-5 * S))
     print(f"same-sign K=8192 {path} relu_only={relu_only}: worst |err| / (1e-5 S) = {ratio:.3f}")
     assert ratio <= 1.0, ratio
