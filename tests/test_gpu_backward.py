@@ -83,7 +83,7 @@ def codes(shape, seed):
     return q
 
 
-@pytest.mark.parametrize("staged", [False, True])
+@pytest.mark.parametrize("staged", [False, True, "a"])  # "a": workspace for A alone (A expanded once, W decoded in the kernel)
 @pytest.mark.parametrize("a_is_km,w_is_nk", [(1, 0), (1, 1), (0, 1)])
 @pytest.mark.parametrize("c_dtype,accumulate", [(H.F32, 0), (H.F32, 1), (H.BF16, 1)])
 def test_gemm_ex_layouts_and_accumulate(c_dtype, accumulate, a_is_km, w_is_nk, staged):
@@ -97,7 +97,7 @@ def test_gemm_ex_layouts_and_accumulate(c_dtype, accumulate, a_is_km, w_is_nk, s
     c0 = (rng.standard_normal((M, ldc)) * 50).astype(np.float32)
     C = torch.from_numpy(c0).cuda().to(torch.float32 if c_dtype == H.F32 else torch.bfloat16)
     c0 = C.float().cpu().numpy().astype(np.float64)
-    wsb = H.hif8_workspace_bytes(H.WS_GEMM, M * K + K * N if staged else 0)
+    wsb = H.hif8_workspace_bytes(H.WS_GEMM, (M * K if staged == "a" else M * K + K * N) if staged else 0)
     ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
     H.hif8_gemm_ex(to_dev(Aq), Aq.shape[1], a_is_km, to_dev(Wq), Wq.shape[1], w_is_nk, C, ldc, c_dtype, M, N, K,
                    torch.tensor([sa], dtype=torch.int32, device="cuda"), torch.tensor([sw], dtype=torch.int32, device="cuda"),
