@@ -45,6 +45,7 @@ namespace {
 constexpr int BM = 128, BN = 256, BK = 64;
 constexpr int kStages8 = 4;    // staging ring of HiF8 byte tiles
 constexpr int kStagesBf = 4;   // ring of decoded BF16 operand tiles
+constexpr int kStagesBfSwapped = 8, kMaxStagesBf = 8;  // the swapped form (see hif8_gemm_kernel) has room for two stages per group
 constexpr int kEpiWarps = 4, kDecodeWarps = 16;
 // The decode warps work in groups, group g on the k-blocks kb = g (mod kDecodeGroups): several k-blocks are in the
 // decode stage at once, which covers the latency of each one's lookups, proxy fence and barrier hand-over.  Group g
@@ -74,7 +75,7 @@ constexpr uint32_t kABfBytes = BM * BK * 2, kBBfBytes = (BN / 2) * BK * 2;  // 1
 // tensor memory of the fused kernel: columns 0-255 the 128 x 256 FP32 accumulator, then one A operand stage (128 rows x
 // 64 BF16 = 32 columns) per operand stage; allocations are powers of two
 constexpr uint32_t kTmemColsAcc = 256, kTmemAStageCols = BK / 2, kTmemCols = 512;
-static_assert(kTmemColsAcc + kStagesBf * kTmemAStageCols <= kTmemCols, "A operand stages must fit beside the accumulator");
+static_assert(kTmemColsAcc + kMaxStagesBf * kTmemAStageCols <= kTmemCols, "A operand stages must fit beside the accumulator");
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s per wait
 
 struct SmemLayout {
@@ -82,7 +83,7 @@ struct SmemLayout {
     static constexpr uint32_t u8 = bf + kStagesBf * (kABfBytes + kBBfBytes);           // 96 KiB
     static constexpr uint32_t lut = u8 + kStages8 * (kA8Bytes + kB8Bytes);             // + 64 KiB
     static constexpr uint32_t bars = lut + 256 * 32 * 4;                                // lane-replicated table, 32 KiB
-    static constexpr uint32_t n_bars = 2 * kMaxStages8 + 2 * kStagesBf + 1;
+    static constexpr uint32_t n_bars = 2 * kMaxStages8 + 2 * kMaxStagesBf + 1;
     static constexpr uint32_t tmem_slot = bars + n_bars * 8;
     static constexpr uint32_t abort_flag = tmem_slot + 4;
     static constexpr uint32_t total = abort_flag + 4;
@@ -499,8 +500,12 @@ constexpr uint32_t kSlotBytes = 16384, kLutBytesWide = 65536, kLutBytesNarrow = 
 static_assert(kBBfBytes == kSlotBytes && kA8Bytes + kB8Bytes == kSlotBytes, "one stage per slot");
 constexpr uint32_t kSmemBytesWide = 227 * 1024;  // the whole opt-in maximum; the kernel checks that its plan fits
 
-template <bool FIXED>  // FIXED: the layout of SmemLayout (A operand tiles in shared memory)
+// PLAN 0: slots around the 64 KiB table.  1: the layout of SmemLayout (A operand tiles in shared memory).  2: the swapped
+// form -- eight operand stages of 16 KiB, four byte stages of 8 KiB, the 32 KiB table, barriers, one after the other.
+constexpr uint32_t kSmemBytesSwapped = kStagesBfSwapped * kBBfBytes + kStages8 * kA8Bytes + 256 * 32 * 4 + 256 + 1024;
+template <int PLAN>
 struct FusedSmem {
+    static constexpr bool FIXED = PLAN == 1;
     uint32_t base, lut, bars, behind;  // shared-window addresses; base is 1024-byte aligned
     int n_front;                       // slots in front of the table
     uint32_t end;                      // first byte behind everything
@@ -510,6 +515,9 @@ struct FusedSmem {
         base = (raw + 1023u) & ~1023u;
         if (FIXED) {
             lut = base + SmemLayout::lut; bars = base + SmemLayout::bars; behind = 0; n_front = 0; end = base + SmemLayout::total;
+        } else if (PLAN == 2) {
+            behind = 0; n_front = kStagesBfSwapped;
+            lut = base + kStagesBfSwapped * kBBfBytes + kStages8 * kA8Bytes; bars = lut + kLutBytesNarrow; end = bars + 256u;
         } else if (!kWideLut) {
             // table with rows of 128 bytes: no alignment to honour, everything in a row: slots, table, barriers
             n_front = (int)kFusedSlots; behind = 0;
@@ -528,7 +536,11 @@ struct FusedSmem {
     __device__ uint32_t slot(int i) const { return i < n_front ? base + (uint32_t)i * kSlotBytes : behind + (uint32_t)(i - n_front) * kSlotBytes; }
     __device__ uint32_t a_bf(int s) const { return base + SmemLayout::bf + s * (kABfBytes + kBBfBytes); }                       // FIXED only
     __device__ uint32_t w_bf(int s) const { return FIXED ? a_bf(s) + kABfBytes : slot(s); }
-    __device__ uint32_t a_u8(int s) const { return FIXED ? base + SmemLayout::u8 + s * (kA8Bytes + kB8Bytes) : slot(kStagesBf + s); }
+    __device__ uint32_t a_u8(int s) const
+    {
+        if (PLAN == 2) return base + kStagesBfSwapped * kBBfBytes + (uint32_t)s * kA8Bytes;
+        return FIXED ? base + SmemLayout::u8 + s * (kA8Bytes + kB8Bytes) : slot(kStagesBf + s);
+    }
     // staging box j (16 KiB) of the result tile: the operand stages, idle once the accumulator is complete
     __device__ uint32_t box(int j) const { return FIXED ? base + SmemLayout::bf + (uint32_t)j * kSlotBytes : slot(j); }
     __device__ uint32_t w_u8(int s) const { return a_u8(s) + kA8Bytes; }
@@ -539,16 +551,24 @@ struct FusedSmem {
 // A_MODE 0: A given as [M,K] bytes, decoded into tensor memory.  1: A given as [K,M] bytes, decoded into shared memory
 // (MN-major operand).  2: A already expanded to BF16 [M,K] in the caller's workspace (only W is decoded here): its tiles
 // come by TMA straight into the K-major operand stages, completing on the leader's "operands ready" barrier.
-template <int A_MODE, bool W_IS_NK>
+// SWAPPED (with A_MODE 0 and W_IS_NK): the kernel computes C^T = W^T A^T.  Its byte operand -- rows decoded into tensor
+// memory -- is the caller's [N,K] weight, its shared-memory operand the caller's activations, already expanded to BF16
+// [M,K] and brought by TMA; nothing decoded here is stored to shared memory or read back from it by the tensor core.  The
+// kernel's "M" is the caller's N and vice versa, and the epilogue writes the accumulator transposed.
+template <int A_MODE, bool W_IS_NK, bool SWAPPED = false>
 __global__ void __launch_bounds__(kThreads, 1)
 hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
                  const __grid_constant__ CUtensorMap map_c, const GemmParams p)
 {
     extern __shared__ unsigned char smem_raw[];
     constexpr bool A_IS_KM = A_MODE == 1, A_BF16 = A_MODE == 2, kFixed = A_MODE != 0;
-    constexpr int kLutShift = (kFixed || !kWideLut) ? 7 : 8;
-    constexpr int kS8 = kFixed ? kStages8 : kStages8Deep;  // depth of the byte ring
-    const FusedSmem<kFixed> plan(smem_u32(smem_raw));
+    static_assert(!SWAPPED || (A_MODE == 0 && W_IS_NK), "the swapped form reads both operands K-major");
+    constexpr int kLutShift = (kFixed || SWAPPED || !kWideLut) ? 7 : 8;
+    constexpr int kS8 = (kFixed || SWAPPED) ? kStages8 : kStages8Deep;  // depth of the byte ring
+    // operand stages: one per decode group, or (SWAPPED: nothing decoded goes to shared memory, which leaves the room) two, so
+    // that a group starts its next k-block while the MMAs of its last one are still queued behind the other groups'
+    constexpr int kSB = SWAPPED ? kStagesBfSwapped : kStagesBf;
+    const FusedSmem<SWAPPED ? 2 : (kFixed ? 1 : 0)> plan(smem_u32(smem_raw));
     const uint32_t base = plan.base;
     unsigned char* sm = smem_raw - smem_u32(smem_raw);  // generic pointer of shared-window address 0
     {
@@ -567,8 +587,8 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     auto bar_u8_full = [&](int s) { return bars + 8u * s; };                                   // per CTA
     auto bar_u8_empty = [&](int s) { return bars + 8u * (kMaxStages8 + s); };                     // per CTA
     auto bar_bf_full = [&](int s) { return bars + 8u * (2 * kMaxStages8 + s); };                  // leader: both CTAs' decode warps
-    auto bar_bf_empty = [&](int s) { return bars + 8u * (2 * kMaxStages8 + kStagesBf + s); };     // per CTA, leader's commits
-    const uint32_t bar_acc_full = bars + 8u * (2 * kMaxStages8 + 2 * kStagesBf);                  // per CTA, leader's commit
+    auto bar_bf_empty = [&](int s) { return bars + 8u * (2 * kMaxStages8 + kMaxStagesBf + s); };  // per CTA, leader's commits
+    const uint32_t bar_acc_full = bars + 8u * (2 * kMaxStages8 + 2 * kMaxStagesBf);                  // per CTA, leader's commit
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + plan.abort_flag());
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + plan.tmem_slot());
     uint32_t* lut_all = reinterpret_cast<uint32_t*>(sm + plan.lut);
@@ -585,7 +605,7 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     if (threadIdx.x == 0) {
         for (int s = 0; s < kS8; s++) { mbar_init(bar_u8_full(s), 1); mbar_init(bar_u8_empty(s), kGroupWarps); }
         // operands ready: both CTAs' decode group, plus (A_BF16) the leader's announcement of the A tile bytes
-        for (int s = 0; s < kStagesBf; s++) { mbar_init(bar_bf_full(s), 2 * kGroupWarps + (A_BF16 ? 1 : 0)); mbar_init(bar_bf_empty(s), 1); }
+        for (int s = 0; s < kSB; s++) { mbar_init(bar_bf_full(s), 2 * kGroupWarps + ((A_BF16 || SWAPPED) ? 1 : 0)); mbar_init(bar_bf_empty(s), 1); }
         mbar_init(bar_acc_full, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -605,24 +625,34 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         // ------------------------------------------------------------------ TMA producer (each CTA feeds itself)
         if (lane == 0) {
             int issued = 0;
-            for (int kb = 0; kb < num_kb; kb++) {
-                const int s = kb % kS8, round = kb / kS8;
-                if (round > 0 && !mbar_wait(bar_u8_empty(s), (round - 1) & 1, abort_flag, p.status, 1)) break;
-                if (*abort_flag) break;
-                const uint32_t dst_a = plan.a_u8(s), dst_b = plan.w_u8(s);
-                mbar_arrive_expect_tx(bar_u8_full(s), (A_BF16 ? 0u : kA8Bytes) + kB8Bytes);
-                if (A_IS_KM) tma_load_2d(dst_a, &map_a, m0, kb * BK, bar_u8_full(s));
-                else if (!A_BF16) tma_load_2d(dst_a, &map_a, kb * BK, m0, bar_u8_full(s));
-                if (W_IS_NK) tma_load_2d(dst_b, &map_w, kb * BK, nh, bar_u8_full(s));
-                else tma_load_2d(dst_b, &map_w, nh, kb * BK, bar_u8_full(s));
-                issued = kb + 1;
-                if (A_BF16) {
-                    // the BF16 A tile goes straight into operand stage sb, once the MMAs of its previous k-block have read
-                    // it; both CTAs' copies complete on the leader's "operands ready" barrier, which the leader arms
-                    const int sb = kb % kStagesBf, rb = kb / kStagesBf;
+            // With a BF16 operand by TMA (A_BF16, SWAPPED) its tile for k-block kb can only be asked for when the MMAs of kb - 4
+            // have read the stage, a late event; so that waiting for it never holds up the byte tiles, the bytes run kLag
+            // k-blocks ahead of the BF16 tiles in this loop.
+            constexpr bool kBf16Tiles = A_BF16 || SWAPPED;
+            constexpr int kLag = kBf16Tiles ? kS8 - 1 : 0;
+            for (int t = 0; t < num_kb + kLag; t++) {
+                if (t < num_kb) {
+                    const int kb = t, s = kb % kS8, round = kb / kS8;
+                    if (round > 0 && !mbar_wait(bar_u8_empty(s), (round - 1) & 1, abort_flag, p.status, 1)) break;
+                    if (*abort_flag) break;
+                    const uint32_t dst_a = plan.a_u8(s), dst_b = plan.w_u8(s);
+                    mbar_arrive_expect_tx(bar_u8_full(s), (A_BF16 ? 0u : kA8Bytes) + (SWAPPED ? 0u : kB8Bytes));
+                    if (A_IS_KM) tma_load_2d(dst_a, &map_a, m0, kb * BK, bar_u8_full(s));
+                    else if (!A_BF16) tma_load_2d(dst_a, &map_a, kb * BK, m0, bar_u8_full(s));
+                    if (SWAPPED) {}
+                    else if (W_IS_NK) tma_load_2d(dst_b, &map_w, kb * BK, nh, bar_u8_full(s));
+                    else tma_load_2d(dst_b, &map_w, nh, kb * BK, bar_u8_full(s));
+                    issued = kb + 1;
+                }
+                if (kBf16Tiles && t >= kLag) {
+                    // the BF16 tile goes straight into operand stage sb (this CTA's 128 rows); both CTAs' copies complete on
+                    // the leader's "operands ready" barrier, which the leader arms with the bytes of both
+                    const int kb = t - kLag, sb = kb % kSB, rb = kb / kSB;
                     if (rb > 0 && !mbar_wait(bar_bf_empty(sb), (rb - 1) & 1, abort_flag, p.status, 6)) break;
-                    if (leader) mbar_arrive_expect_tx(bar_bf_full(sb), 2 * kABfBytes);
-                    tma_load_3d_pair(plan.a_bf(sb), &map_a, kb * BK, m0, 0, map_to_cta(bar_bf_full(sb), 0));
+                    if (*abort_flag) break;
+                    if (leader) mbar_arrive_expect_tx(bar_bf_full(sb), 2 * (SWAPPED ? kBBfBytes : kABfBytes));
+                    if (SWAPPED) tma_load_3d_pair(plan.w_bf(sb), &map_w, kb * BK, nh, 0, map_to_cta(bar_bf_full(sb), 0));
+                    else tma_load_3d_pair(plan.a_bf(sb), &map_a, kb * BK, m0, 0, map_to_cta(bar_bf_full(sb), 0));
                 }
             }
             if (*abort_flag) {
@@ -632,7 +662,7 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                     const unsigned long long t0 = global_ns();
                     while (!mbar_try_wait(bar_u8_full(s), (kb / kS8) & 1) && global_ns() - t0 < kWaitLimitNs) {}
                 }
-                if (A_BF16) {  // (the A tiles complete on a barrier that also counts the decode groups, which have given up:
+                if (A_BF16 || SWAPPED) {  // (the BF16 tiles complete on a barrier that also counts the decode groups, which have given up:
                                // their copies get a fixed 50 us instead)
                     const unsigned long long t0 = global_ns();
                     while (global_ns() - t0 < 50000ull) {}
@@ -647,7 +677,7 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                                    ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
             bool ok = true;
             for (int kb = 0; kb < num_kb && ok; kb++) {
-                const int s = kb % kStagesBf, round = kb / kStagesBf;
+                const int s = kb % kSB, round = kb / kSB;
                 ok = mbar_wait(bar_bf_full(s), round & 1, abort_flag, p.status, 2);
                 if (!ok) break;
                 tc_fence_after();
@@ -677,7 +707,7 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
         const int dt = threadIdx.x - (kFirstDecodeWarp + group * kGroupWarps) * 32;  // 0..kGroupThreads-1
         bool ok = true;
         for (int kb = group; kb < num_kb && ok; kb += kDecodeGroups) {
-            const int s8 = kb % kS8, r8 = kb / kS8, sb = group, rb = kb / kStagesBf;
+            const int s8 = kb % kS8, r8 = kb / kS8, sb = kb % kSB, rb = kb / kSB;
             ok = mbar_wait(bar_u8_full(s8), r8 & 1, abort_flag, p.status, 3);
             if (ok && rb > 0) ok = mbar_wait(bar_bf_empty(sb), (rb - 1) & 1, abort_flag, p.status, 4);
             if (!ok) break;
@@ -705,7 +735,7 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 uint4 va[BK / 16];
 #pragma unroll
                 for (int j = 0; j < BK / 16; j++) va[j] = lds_v4(a_row + (((uint32_t)j ^ sw) << 4));
-                load_tile_chunks<!W_IS_NK>(b8, dt, vw);
+                if (!SWAPPED) load_tile_chunks<!W_IS_NK>(b8, dt, vw);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_u8_empty(s8));
                 uint32_t o[BK / 2];  // 64 BF16 of this row, two per column
@@ -717,7 +747,7 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 }
                 tmem_st_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + kTmemColsAcc + (uint32_t)(sb * kTmemAStageCols), o);
             }
-            decode_tile_chunks<!W_IS_NK, kLutShift>(vw, bbf, dt, lut);
+            if (!SWAPPED) decode_tile_chunks<!W_IS_NK, kLutShift>(vw, bbf, dt, lut);
             if (A_MODE == 0) tmem_st_wait();  // the row is in tensor memory
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // make the stores visible to the tensor core
             tc_fence_before();
@@ -742,8 +772,39 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             const int s1 = s / 2, s2 = s - s1;  // |s1|, |s2| <= 126: two exact power-of-two factors
             const float f1 = __uint_as_float((uint32_t)(s1 + 127) << 23), f2 = __uint_as_float((uint32_t)(s2 + 127) << 23);
             const int row = m0 + quarter * 32 + lane;
-            // (two loops rather than a branch inside one: the register allocation of each stays that of its own path)
-            if (!A_IS_KM && p.c_by_tma) {
+            // (separate loops rather than branches inside one: the register allocation of each stays that of its own path)
+            if (SWAPPED) {
+                // accumulator row = the caller's column n (one weight exponent per thread), accumulator column = the caller's
+                // row m: for every m the warp writes 32 consecutive n
+                const int sw = p.d_sw_channel ? (row < p.M ? __ldg(p.d_sw_channel + row) : 0) : (p.d_sw ? *p.d_sw : 0);
+                const int sc = -(sa + sw), t1 = sc / 2, t2 = sc - t1;
+                const float g1 = __uint_as_float((uint32_t)(t1 + 127) << 23), g2 = __uint_as_float((uint32_t)(t2 + 127) << 23);
+#pragma unroll 1
+                for (int c = share * 32; c < BN; c += 5 * 32) {
+                    uint32_t r[32];
+                    tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + c, r);
+                    tmem_ld_wait();
+                    if (row < p.M) {
+#pragma unroll
+                        for (int i = 0; i < 32; i++) {
+                            const int m = n0 + c + i;
+                            if (m < p.N) {
+                                float v = __uint_as_float(r[i]) * g1 * g2;
+                                if (p.c_is_f32) {
+                                    float* out = reinterpret_cast<float*>(p.C) + (long long)m * p.ldc + row;
+                                    *out = p.accumulate ? v + *out : v;
+                                } else {
+                                    unsigned short* out = reinterpret_cast<unsigned short*>(p.C) + (long long)m * p.ldc + row;
+                                    if (p.accumulate) v += __uint_as_float((uint32_t)*out << 16);
+                                    unsigned short b;
+                                    asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(b) : "f"(v));
+                                    *out = b;
+                                }
+                            }
+                        }
+                    }
+                }
+            } else if (!A_IS_KM && p.c_by_tma) {
 #pragma unroll 1
                 for (int c = share * 32; c < BN; c += 5 * 32) {
                     uint32_t r[32];
@@ -1447,6 +1508,8 @@ bool gemm_kernels_ready(int dev, int* sm_count_out)
     const GemmDeviceSetup* s = g_gemm_setup.get(dev, [](int d, GemmDeviceSetup* out) {
         out->rc = cudaSuccess;
         out->sm_count = 0;
+        if (out->rc == cudaSuccess)
+            out->rc = cudaFuncSetAttribute(hif8_gemm_kernel<0, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytesSwapped);
         const void* fused[6] = {(const void*)hif8_gemm_kernel<0, false>, (const void*)hif8_gemm_kernel<0, true>,
                                 (const void*)hif8_gemm_kernel<1, false>, (const void*)hif8_gemm_kernel<1, true>,
                                 (const void*)hif8_gemm_kernel<2, false>, (const void*)hif8_gemm_kernel<2, true>};
@@ -1644,6 +1707,30 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t
         // boxes of 64 k x 128 rows in the 128-byte-swizzled operand layout (a stack of one matrix: the pair form of the copy)
         if (!make_map3(&map_a, a_bf, (uint64_t)K, (uint64_t)M, 1, 0, BK, BM)) return HIF8_ERR_CUDA;
         a_mode = 2;
+        if (w_is_nk) {
+            // [N,K] weights: the swapped form, C^T = W^T A^T.  The weight rows are the operand that is decoded into tensor
+            // memory, the expanded activations the one in shared memory; the kernel's M is N and its N is M.
+            GemmParams q = p;
+            q.M = N; q.N = M; q.c_by_tma = 0;
+            q.tiles_m = (N + BM - 1) / BM; q.tiles_n = (M + BN - 1) / BN;
+            const long long tiles2s = (long long)((N + 2 * BM - 1) / (2 * BM)) * q.tiles_n;
+            if (tiles2s > 0x3FFFFFFF) return HIF8_ERR_SHAPE;
+            CUtensorMap map_wb, map_ab;
+            if (!make_map(&map_wb, Wq, (uint64_t)K, (uint64_t)N, (uint64_t)ldw, BK, BM, false, 64)) return HIF8_ERR_CUDA;
+            if (!make_map3(&map_ab, a_bf, (uint64_t)K, (uint64_t)M, 1, 0, BK, BN / 2)) return HIF8_ERR_CUDA;
+            cudaLaunchConfig_t cs{};
+            cs.gridDim = dim3(2u * (unsigned)tiles2s);
+            cs.blockDim = dim3(kThreads);
+            cs.dynamicSmemBytes = kSmemBytesSwapped;
+            cs.stream = st;
+            cudaLaunchAttribute at[1];
+            at[0].id = cudaLaunchAttributeClusterDimension;
+            at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
+            cs.attrs = at; cs.numAttrs = 1;
+            const cudaError_t src = cudaLaunchKernelEx(&cs, hif8_gemm_kernel<0, true, true>, map_wb, map_ab, map_ab, q);
+            g_launches.fetch_add(1, std::memory_order_relaxed);
+            return (src == cudaSuccess && cudaGetLastError() == cudaSuccess) ? HIF8_OK : HIF8_ERR_CUDA;
+        }
     }
 
     cudaLaunchConfig_t cfg{};
