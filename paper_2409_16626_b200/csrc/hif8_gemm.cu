@@ -63,7 +63,8 @@ static_assert(kStages8 == kDecodeGroups && kStagesBf == kDecodeGroups, "group g 
 #ifndef HIF8_FUSED_WIDE_LUT
 #define HIF8_FUSED_WIDE_LUT 1
 #endif
-constexpr int kStages8Deep = HIF8_FUSED_BYTE_STAGES, kMaxStages8 = kStages8Deep > kStages8 ? kStages8Deep : kStages8;
+constexpr int kStages8Deep = HIF8_FUSED_BYTE_STAGES, kMaxStages8 = 8;  // (barrier slots for up to eight byte stages)
+static_assert(kStages8Deep <= kMaxStages8 && kStages8 <= kMaxStages8, "barrier slots");
 constexpr bool kWideLut = HIF8_FUSED_WIDE_LUT != 0;
 static_assert(kStages8Deep % kDecodeGroups == 0, "a byte stage is always read by the same group");
 static_assert(!kWideLut || kStages8Deep == 4, "the 64 KiB table leaves room for four byte stages only");
@@ -89,6 +90,8 @@ struct SmemLayout {
     static constexpr uint32_t total = abort_flag + 4;
 };
 constexpr uint32_t kSmemBytes = SmemLayout::total + 1024;  // slack for manual 1024-byte alignment
+constexpr uint32_t kBarsBytes = 320;                       // barriers, tensor-memory slot, abort flag
+static_assert(SmemLayout::n_bars * 8 + 8 <= kBarsBytes, "barrier block");
 
 // ---------------------------------------------------------------------------------------------------------
 // PTX wrappers
@@ -194,6 +197,15 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank)
     uint32_t r;
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
     return r;
+}
+// Arrival on a barrier of a CTA of the cluster with the default semantics (release at CTA scope).  For the decode warps of
+// the fused kernel: what they hand over is read by the tensor core -- tensor memory, ordered by tcgen05.wait::st and
+// tcgen05.fence::before_thread_sync, and shared memory, made visible to the async proxy by fence.proxy.async -- not by
+// threads of the other CTA.  A release at cluster scope here cost about 2200 cycles per arrival (a per-k-block timeline of
+// the groups showed it): it waits for every memory operation the SM has in flight.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
 {
@@ -502,7 +514,8 @@ constexpr uint32_t kSmemBytesWide = 227 * 1024;  // the whole opt-in maximum; th
 
 // PLAN 0: slots around the 64 KiB table.  1: the layout of SmemLayout (A operand tiles in shared memory).  2: the swapped
 // form -- eight operand stages of 16 KiB, four byte stages of 8 KiB, the 32 KiB table, barriers, one after the other.
-constexpr uint32_t kSmemBytesSwapped = kStagesBfSwapped * kBBfBytes + kStages8 * kA8Bytes + 256 * 32 * 4 + 256 + 1024;
+constexpr int kStages8Swapped = 8;  // byte stages of the swapped form (A bytes only: 8 KiB each)
+constexpr uint32_t kSmemBytesSwapped = kStagesBfSwapped * kBBfBytes + kStages8Swapped * kA8Bytes + 256 * 32 * 4 + kBarsBytes + 1024;
 template <int PLAN>
 struct FusedSmem {
     static constexpr bool FIXED = PLAN == 1;
@@ -517,11 +530,11 @@ struct FusedSmem {
             lut = base + SmemLayout::lut; bars = base + SmemLayout::bars; behind = 0; n_front = 0; end = base + SmemLayout::total;
         } else if (PLAN == 2) {
             behind = 0; n_front = kStagesBfSwapped;
-            lut = base + kStagesBfSwapped * kBBfBytes + kStages8 * kA8Bytes; bars = lut + kLutBytesNarrow; end = bars + 256u;
+            lut = base + kStagesBfSwapped * kBBfBytes + kStages8Swapped * kA8Bytes; bars = lut + kLutBytesNarrow; end = bars + kBarsBytes;
         } else if (!kWideLut) {
             // table with rows of 128 bytes: no alignment to honour, everything in a row: slots, table, barriers
             n_front = (int)kFusedSlots; behind = 0;
-            lut = base + kFusedSlots * kSlotBytes; bars = lut + kLutBytesNarrow; end = bars + 256u;
+            lut = base + kFusedSlots * kSlotBytes; bars = lut + kLutBytesNarrow; end = bars + kBarsBytes;
         } else {
             lut = (base + kLutBytesWide - 1) & ~(kLutBytesWide - 1);
             const uint32_t front = lut - base;
@@ -529,8 +542,8 @@ struct FusedSmem {
             behind = lut + kLutBytesWide;
             const uint32_t after_slots = behind + (kFusedSlots - n_front) * kSlotBytes;
             // barriers, tensor-memory slot and abort flag (256 bytes): in the gap in front of the table if there is one
-            bars = (front - n_front * kSlotBytes >= 256u) ? base + n_front * kSlotBytes : after_slots;
-            end = bars >= after_slots ? bars + 256u : after_slots;
+            bars = (front - n_front * kSlotBytes >= kBarsBytes) ? base + n_front * kSlotBytes : after_slots;
+            end = bars >= after_slots ? bars + kBarsBytes : after_slots;
         }
     }
     __device__ uint32_t slot(int i) const { return i < n_front ? base + (uint32_t)i * kSlotBytes : behind + (uint32_t)(i - n_front) * kSlotBytes; }
@@ -564,7 +577,7 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     constexpr bool A_IS_KM = A_MODE == 1, A_BF16 = A_MODE == 2, kFixed = A_MODE != 0;
     static_assert(!SWAPPED || (A_MODE == 0 && W_IS_NK), "the swapped form reads both operands K-major");
     constexpr int kLutShift = (kFixed || SWAPPED || !kWideLut) ? 7 : 8;
-    constexpr int kS8 = (kFixed || SWAPPED) ? kStages8 : kStages8Deep;  // depth of the byte ring
+    constexpr int kS8 = SWAPPED ? kStages8Swapped : (kFixed ? kStages8 : kStages8Deep);  // depth of the byte ring
     // operand stages: one per decode group, or (SWAPPED: nothing decoded goes to shared memory, which leaves the room) two, so
     // that a group starts its next k-block while the MMAs of its last one are still queued behind the other groups'
     constexpr int kSB = SWAPPED ? kStagesBfSwapped : kStagesBf;
@@ -621,39 +634,40 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
+    if ((A_BF16 || SWAPPED) && warp == 0) {
+        // ------------------------------------------------------------------ second producer (an epilogue warp, idle until the
+        // accumulator is complete): the BF16 tiles of the operand that was expanded beforehand.  Issuing a tile copy costs its
+        // thread a few hundred cycles, and with both kinds of copy on one thread that thread set the pace.  The tile of k-block
+        // kb goes straight into operand stage sb (this CTA's 128 rows) once the MMAs of its previous use have read it; both
+        // CTAs' copies complete on the leader's "operands ready" barrier, which the leader arms with the bytes of both.
+        if (lane == 0) {
+            for (int kb = 0; kb < num_kb; kb++) {
+                const int sb = kb % kSB, rb = kb / kSB;
+                if (rb > 0 && !mbar_wait(bar_bf_empty(sb), (rb - 1) & 1, abort_flag, p.status, 6)) break;
+                if (*abort_flag) break;
+                if (leader) mbar_arrive_expect_tx(bar_bf_full(sb), 2 * (SWAPPED ? kBBfBytes : kABfBytes));
+                if (SWAPPED) tma_load_3d_pair(plan.w_bf(sb), &map_w, kb * BK, nh, 0, map_to_cta(bar_bf_full(sb), 0));
+                else tma_load_3d_pair(plan.a_bf(sb), &map_a, kb * BK, m0, 0, map_to_cta(bar_bf_full(sb), 0));
+            }
+        }
+        __syncwarp();
+    }
     if (warp == kTmaWarp) {
         // ------------------------------------------------------------------ TMA producer (each CTA feeds itself)
         if (lane == 0) {
             int issued = 0;
-            // With a BF16 operand by TMA (A_BF16, SWAPPED) its tile for k-block kb can only be asked for when the MMAs of kb - 4
-            // have read the stage, a late event; so that waiting for it never holds up the byte tiles, the bytes run kLag
-            // k-blocks ahead of the BF16 tiles in this loop.
-            constexpr bool kBf16Tiles = A_BF16 || SWAPPED;
-            constexpr int kLag = kBf16Tiles ? kS8 - 1 : 0;
-            for (int t = 0; t < num_kb + kLag; t++) {
-                if (t < num_kb) {
-                    const int kb = t, s = kb % kS8, round = kb / kS8;
-                    if (round > 0 && !mbar_wait(bar_u8_empty(s), (round - 1) & 1, abort_flag, p.status, 1)) break;
-                    if (*abort_flag) break;
-                    const uint32_t dst_a = plan.a_u8(s), dst_b = plan.w_u8(s);
-                    mbar_arrive_expect_tx(bar_u8_full(s), (A_BF16 ? 0u : kA8Bytes) + (SWAPPED ? 0u : kB8Bytes));
-                    if (A_IS_KM) tma_load_2d(dst_a, &map_a, m0, kb * BK, bar_u8_full(s));
-                    else if (!A_BF16) tma_load_2d(dst_a, &map_a, kb * BK, m0, bar_u8_full(s));
-                    if (SWAPPED) {}
-                    else if (W_IS_NK) tma_load_2d(dst_b, &map_w, kb * BK, nh, bar_u8_full(s));
-                    else tma_load_2d(dst_b, &map_w, nh, kb * BK, bar_u8_full(s));
-                    issued = kb + 1;
-                }
-                if (kBf16Tiles && t >= kLag) {
-                    // the BF16 tile goes straight into operand stage sb (this CTA's 128 rows); both CTAs' copies complete on
-                    // the leader's "operands ready" barrier, which the leader arms with the bytes of both
-                    const int kb = t - kLag, sb = kb % kSB, rb = kb / kSB;
-                    if (rb > 0 && !mbar_wait(bar_bf_empty(sb), (rb - 1) & 1, abort_flag, p.status, 6)) break;
-                    if (*abort_flag) break;
-                    if (leader) mbar_arrive_expect_tx(bar_bf_full(sb), 2 * (SWAPPED ? kBBfBytes : kABfBytes));
-                    if (SWAPPED) tma_load_3d_pair(plan.w_bf(sb), &map_w, kb * BK, nh, 0, map_to_cta(bar_bf_full(sb), 0));
-                    else tma_load_3d_pair(plan.a_bf(sb), &map_a, kb * BK, m0, 0, map_to_cta(bar_bf_full(sb), 0));
-                }
+            for (int kb = 0; kb < num_kb; kb++) {
+                const int s = kb % kS8, round = kb / kS8;
+                if (round > 0 && !mbar_wait(bar_u8_empty(s), (round - 1) & 1, abort_flag, p.status, 1)) break;
+                if (*abort_flag) break;
+                const uint32_t dst_a = plan.a_u8(s), dst_b = plan.w_u8(s);
+                mbar_arrive_expect_tx(bar_u8_full(s), (A_BF16 ? 0u : kA8Bytes) + (SWAPPED ? 0u : kB8Bytes));
+                if (A_IS_KM) tma_load_2d(dst_a, &map_a, m0, kb * BK, bar_u8_full(s));
+                else if (!A_BF16) tma_load_2d(dst_a, &map_a, kb * BK, m0, bar_u8_full(s));
+                if (SWAPPED) {}
+                else if (W_IS_NK) tma_load_2d(dst_b, &map_w, kb * BK, nh, bar_u8_full(s));
+                else tma_load_2d(dst_b, &map_w, nh, kb * BK, bar_u8_full(s));
+                issued = kb + 1;
             }
             if (*abort_flag) {
                 // let the copies already issued land before this CTA's shared memory goes away
@@ -752,7 +766,7 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // make the stores visible to the tensor core
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(map_to_cta(bar_bf_full(sb), 0));  // the leader's MMAs read both CTAs' operands
+            if (lane == 0) mbar_arrive_remote(map_to_cta(bar_bf_full(sb), 0));  // the leader's MMAs read both CTAs' operands
         }
     }
     if (warp != kTmaWarp && warp != kMmaWarp) {
