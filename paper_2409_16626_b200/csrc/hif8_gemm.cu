@@ -332,6 +332,10 @@ __device__ __forceinline__ uint4 lds_v4(uint32_t addr)
     asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;
 }
+__device__ __forceinline__ void sts_u16(uint32_t addr, unsigned short v)
+{
+    asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(v) : "memory");
+}
 __device__ __forceinline__ void sts_v4(uint32_t addr, uint4 v)
 {
     asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
@@ -793,6 +797,27 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 const int sw = p.d_sw_channel ? (row < p.M ? __ldg(p.d_sw_channel + row) : 0) : (p.d_sw ? *p.d_sw : 0);
                 const int sc = -(sa + sw), t1 = sc / 2, t2 = sc - t1;
                 const float g1 = __uint_as_float((uint32_t)(t1 + 127) << 23), g2 = __uint_as_float((uint32_t)(t2 + 127) << 23);
+                if (p.c_by_tma) {
+                    // BF16 result that replaces C: into the staging boxes of the tile stores (64 of the caller's columns x 128
+                    // of its rows each, 128-byte-swizzled; box = column half + 2 * row half of this CTA's 256 x 128 piece).  For
+                    // one row m the 32 lanes write 32 consecutive columns: 64 contiguous bytes of one line.
+                    const int nl = quarter * 32 + lane;
+                    const uint32_t piece = (uint32_t)((nl & 63) >> 3), within = (uint32_t)(nl & 7) * 2u;
+#pragma unroll 1
+                    for (int c = share * 32; c < BN; c += 5 * 32) {
+                        uint32_t r[32];
+                        tmem_ld_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + c, r);
+                        tmem_ld_wait();
+                        const uint32_t box = plan.box((nl >> 6) + 2 * (c >> 7));
+#pragma unroll
+                        for (int i = 0; i < 32; i++) {
+                            const uint32_t rr = (uint32_t)((c + i) & 127);
+                            unsigned short b;
+                            asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(b) : "f"(__uint_as_float(r[i]) * g1 * g2));
+                            sts_u16(box + (rr >> 3) * 1024u + (rr & 7u) * 128u + ((piece ^ (rr & 7u)) << 4) + within, b);
+                        }
+                    }
+                } else
 #pragma unroll 1
                 for (int c = share * 32; c < BN; c += 5 * 32) {
                     uint32_t r[32];
@@ -846,8 +871,13 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             asm volatile("bar.sync 1, %0;" ::"n"((kEpiWarps + kDecodeWarps) * 32) : "memory");
             if (threadIdx.x == 0 && ok && !*abort_flag) {
+                if (SWAPPED) {  // x = the caller's column (this CTA's 128, two boxes), y = its row (256, two boxes)
 #pragma unroll
-                for (int j = 0; j < BN / 64; j++) tma_store_2d(&map_c, plan.box(j), n0 + j * 64, m0);
+                    for (int j = 0; j < 4; j++) tma_store_2d(&map_c, plan.box(j), m0 + (j & 1) * 64, n0 + (j >> 1) * 128);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < BN / 64; j++) tma_store_2d(&map_c, plan.box(j), n0 + j * 64, m0);
+                }
                 asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
             }
@@ -1725,7 +1755,10 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t
             // [N,K] weights: the swapped form, C^T = W^T A^T.  The weight rows are the operand that is decoded into tensor
             // memory, the expanded activations the one in shared memory; the kernel's M is N and its N is M.
             GemmParams q = p;
-            q.M = N; q.N = M; q.c_by_tma = 0;
+            q.M = N; q.N = M;
+            q.c_by_tma = (c_dtype == HIF8_BF16 && !accumulate) ? 1 : 0;
+            CUtensorMap map_cs;
+            if (q.c_by_tma && !make_map(&map_cs, C, (uint64_t)N, (uint64_t)M, (uint64_t)ldc, 64, BM, true)) return HIF8_ERR_CUDA;
             q.tiles_m = (N + BM - 1) / BM; q.tiles_n = (M + BN - 1) / BN;
             const long long tiles2s = (long long)((N + 2 * BM - 1) / (2 * BM)) * q.tiles_n;
             if (tiles2s > 0x3FFFFFFF) return HIF8_ERR_SHAPE;
@@ -1741,7 +1774,7 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t
             at[0].id = cudaLaunchAttributeClusterDimension;
             at[0].val.clusterDim.x = 2; at[0].val.clusterDim.y = 1; at[0].val.clusterDim.z = 1;
             cs.attrs = at; cs.numAttrs = 1;
-            const cudaError_t src = cudaLaunchKernelEx(&cs, hif8_gemm_kernel<0, true, true>, map_wb, map_ab, map_ab, q);
+            const cudaError_t src = cudaLaunchKernelEx(&cs, hif8_gemm_kernel<0, true, true>, map_wb, map_ab, q.c_by_tma ? map_cs : map_ab, q);
             g_launches.fetch_add(1, std::memory_order_relaxed);
             return (src == cudaSuccess && cudaGetLastError() == cudaSuccess) ? HIF8_OK : HIF8_ERR_CUDA;
         }
