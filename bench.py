@@ -408,6 +408,11 @@ def extra_results(H, torch, hbm_peak, tf_peak, peak_kind, tf_sustained=None):
     g_aexp = tensor(timed(lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, C, N, H.BF16, M, N, K, se[0:1], se[1:2], gws, gws_a), 3, rest_s=REST),
                     flops, device_status=H.hif8_last_device_status(),
                     note="workspace for A alone: A expanded once to BF16, W tiles decoded inside the tensor-core kernel")
+    # the same with the weight bytes read as [N,K] (the layout of a stored checkpoint; values differ, time does not depend on
+    # them): the swapped form, weight rows decoded into tensor memory
+    g_aexp_nk = tensor(timed(lambda r: H.hif8_gemm(Aq, K, Wq, K, 1, C, N, H.BF16, M, N, K, se[0:1], se[1:2], gws, gws_a), 3, rest_s=REST),
+                       flops, device_status=H.hif8_last_device_status(),
+                       note="workspace for A alone, [N,K] weights: C^T = W^T A^T, weight rows decoded into tensor memory")
     ch_se.fill_(int(se[1]))
     g_chan = tensor(timed(lambda r: H.hif8_gemm_channel_scaled(Aq, K, Wq, N, 0, C, N, H.BF16, M, N, K, se[0:1], ch_se, gws, gws_b), 5,
                           rest_s=REST),
@@ -415,6 +420,7 @@ def extra_results(H, torch, hbm_peak, tf_peak, peak_kind, tf_sustained=None):
     row("C5_gemm_8192x28672x8192_decode_once", g_once, "tensor")
     row("C5_gemm_8192x28672x8192_fused", g_fused, "tensor")
     row("C5_gemm_8192x28672x8192_A_expanded_W_fused", g_aexp, "tensor")
+    row("C5_gemm_8192x28672x8192_A_expanded_W_[N,K]_fused", g_aexp_nk, "tensor")
     row("gemm_8192x28672x8192_channel_scaled", g_chan, "tensor")
     # backward-pass forms of the same size: dgrad reads the weight as [N,K], wgrad reads A as [K,M] and accumulates in FP32
     bw = {}
@@ -447,7 +453,7 @@ def extra_results(H, torch, hbm_peak, tf_peak, peak_kind, tf_sustained=None):
     out["gemm_narrow_Mx28672x8192"] = {"bound": "hbm", "bytes": "K*N weight bytes + M*K + 2*M*N", "shapes": narrow,
                                        "peak": hbm_peak, "peak_kind": f"of {peak_kind}"}
     out["gemm_8192x28672x8192"] = {
-        "backward_forms": bw, "decode_once_channel_scaled": g_chan, "decode_once": g_once, "fused": g_fused, "a_expanded_w_fused": g_aexp,
+        "backward_forms": bw, "decode_once_channel_scaled": g_chan, "decode_once": g_once, "fused": g_fused, "a_expanded_w_fused": g_aexp, "a_expanded_w_nk_fused": g_aexp_nk,
         "bound": "tensor", "peak": tf_peak, "peak_kind": f"of {peak_kind} (cuBLAS BF16 burst)", "unit": "TFLOP/s",
         "timing": f"every timed region starts after {REST} s of idle (bursts, like the peak); back_to_back: about one second of calls "
                   "in a row under the power cap, against the sustained cuBLAS figure",
