@@ -693,15 +693,24 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
             // instruction descriptor: FP32 accumulator, BF16 A and B, A K-major, B K- or MN-major, N = 256, M = 256 (pair)
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((A_IS_KM ? 1u : 0u) << 15) | ((W_IS_NK ? 0u : 1u) << 16) |
                                    ((uint32_t)(BN >> 3) << 17) | ((uint32_t)((2 * BM) >> 4) << 24);
-            bool ok = true;
+            // An MMA is accepted only when the tensor pipe has room, so whatever this thread does between two of them leaves
+            // the pipe idle: the barrier of the next k-block is probed, and its addresses are formed, between the third and
+            // the fourth MMA of the current one (while the third runs), not after the commit.
+            bool ok = mbar_wait(bar_bf_full(0), 0, abort_flag, p.status, 2);
+            uint32_t a_addr = plan.a_bf(0), b_addr = plan.w_bf(0), a_tmem = tmem_base + kTmemColsAcc;
             for (int kb = 0; kb < num_kb && ok; kb++) {
-                const int s = kb % kSB, round = kb / kSB;
-                ok = mbar_wait(bar_bf_full(s), round & 1, abort_flag, p.status, 2);
-                if (!ok) break;
+                const int s = kb % kSB;
                 tc_fence_after();
-                const uint32_t a_addr = plan.a_bf(s), b_addr = plan.w_bf(s);
+                bool next_ready = true;
+                uint32_t a_next = 0, b_next = 0, t_next = 0;
 #pragma unroll
                 for (int kk = 0; kk < BK / 16; kk++) {
+                    if (kk == BK / 16 - 1 && kb + 1 < num_kb) {
+                        const int sn = (kb + 1) % kSB;
+                        next_ready = mbar_try_wait(bar_bf_full(sn), (uint32_t)(((kb + 1) / kSB) & 1));
+                        a_next = plan.a_bf(sn); b_next = plan.w_bf(sn);
+                        t_next = tmem_base + kTmemColsAcc + (uint32_t)(sn * kTmemAStageCols);
+                    }
                     // K-major: 16 k = 32 bytes inside the 128-byte row; MN-major: 16 k = two 1024-byte atoms
                     const uint64_t db = W_IS_NK ? make_smem_desc(b_addr + kk * 32, 16, 1024)
                                                 : make_smem_desc(b_addr + kk * 2048, 8192, 1024);
@@ -711,11 +720,14 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                         tc_mma_bf16_pair(tmem_base, make_smem_desc(a_addr + kk * 32, 16, 1024), db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
                     } else {
                         // A from tensor memory: stage s, 16 k = 8 columns
-                        tc_mma_bf16_pair_a_tmem(tmem_base, tmem_base + kTmemColsAcc + (uint32_t)(s * kTmemAStageCols + kk * 8), db, idesc,
-                                                (kb > 0 || kk > 0) ? 1u : 0u);
+                        tc_mma_bf16_pair_a_tmem(tmem_base, a_tmem + (uint32_t)(kk * 8), db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
                     }
                 }
                 tc_commit_pair(bar_bf_empty(s));  // frees this operand stage in both CTAs once the MMAs have read it
+                if (kb + 1 < num_kb) {
+                    if (!next_ready) ok = mbar_wait(bar_bf_full((kb + 1) % kSB), (uint32_t)(((kb + 1) / kSB) & 1), abort_flag, p.status, 2);
+                    a_addr = a_next; b_addr = b_next; a_tmem = t_next;
+                }
             }
             if (ok) tc_commit_pair(bar_acc_full);
         }
