@@ -207,10 +207,6 @@ __device__ __forceinline__ void mbar_arrive_remote(uint32_t cluster_addr)
 {
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
-{
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
 __device__ __forceinline__ void cluster_sync_all()
 {
     asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -1439,7 +1435,9 @@ bf16_gemm_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(map_to_cta(bar_acc_empty(acc), 0));  // tell the leader: accumulator drained
+            // (default semantics: what the leader's MMAs must not overtake are this warp's tensor-memory loads, ordered by
+            // tcgen05.wait::ld and the fence above -- not its stores to C, which a release at cluster scope would wait for)
+            if (lane == 0) mbar_arrive_remote(map_to_cta(bar_acc_empty(acc), 0));  // tell the leader: accumulator drained
         }
         if (p.err_sum) flush_error();
     }
