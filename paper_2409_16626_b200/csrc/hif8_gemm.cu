@@ -587,7 +587,7 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     {
         uint32_t dyn_bytes;
         asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn_bytes));
-        if (plan.end > smem_u32(smem_raw) + dyn_bytes) {  // the plan does not fit (same verdict in every thread of the pair)
+        if (plan.end > smem_u32(smem_raw) + dyn_bytes) {  // the plan does not fit (the same answer in every thread of the pair)
             if (threadIdx.x == 0) atomicCAS(p.status, 0, 7);
             return;
         }
