@@ -322,6 +322,16 @@ int hif8_encode_transpose(const void* src, int src_dtype, uint8_t* dst, int64_t 
 int hif8_gemm_status(const void* workspace, hif8_stream_t stream);
 
 /*
+ * Which general kernel a large workspace selects.  HIF8_GEMM_PATH_AUTO (the default): with room for both operands W is
+ * expanded too only when the product is large enough to win that pass back (about 1600 rows of A and more); below that A
+ * alone is expanded.  HIF8_GEMM_PATH_EXPAND_BOTH: both operands are expanded whenever the workspace has room (for
+ * measurements and tests of that kernel on small products).  Process-wide; returns the previous setting (0 or 1), or
+ * HIF8_ERR_FLAGS for an unknown one.  Results do not depend on it.
+ */
+enum { HIF8_GEMM_PATH_AUTO = 0, HIF8_GEMM_PATH_EXPAND_BOTH = 1 };
+int hif8_gemm_path_policy(int policy);
+
+/*
  * Status of the most recent GEMM-class call (hif8_gemm, hif8_gemm_ex, hif8_gemm_channel_scaled, hif8_pts_search,
  * hif8_selftest_wait_timeout) enqueued on `stream` of the current device, without the caller naming the workspace:
  * the library remembers, per stream, where that call's status word lives.  SYNCHRONISES `stream`, then returns HIF8_OK,

@@ -22,7 +22,7 @@ LIB_PATH = os.path.join(_HERE, "libhif8.so")
 EXPORTS = ["hif8_encode", "hif8_decode", "hif8_amax", "hif8_amax_scale_encode", "hif8_fake_quant", "hif8_gemm", "hif8_gemm_status", "hif8_pts_search", "hif8_pts_workspace_bytes",
            "hif8_pts_status", "hif8_selftest_wait_timeout", "hif8_channel_amax_scale_encode", "hif8_gemm_channel_scaled",
            "hif8_scale_state_init", "hif8_delayed_scale_encode", "hif8_gemm_ex", "hif8_encode_transpose", "hif8_als_state_init", "hif8_als_update", "hif8_check_finite", "hif8_encode_from_amax",
-           "hif8_amax_scale_encode_static", "hif8_encode_f32_patterns", "hif8_last_device_status", "hif8_selftest_host_caches", "hif8_workspace_bytes", "hif8_status_string", "hif8_launch_count"]
+           "hif8_amax_scale_encode_static", "hif8_encode_f32_patterns", "hif8_last_device_status", "hif8_selftest_host_caches", "hif8_gemm_path_policy", "hif8_workspace_bytes", "hif8_status_string", "hif8_launch_count"]
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2409_16626_b200.build` (needs nvcc)")
@@ -42,6 +42,8 @@ lib.hif8_fake_quant.argtypes = [_vp, _vp, _i, _sz, _i, _i, _i, _u, _u64, _vp, _v
 lib.hif8_gemm.argtypes = [_vp, _i64, _vp, _i64, _i, _vp, _i64, _i, _i, _i, _i, _vp, _vp, _vp, _sz, _vp]
 lib.hif8_gemm_status.argtypes = [_vp, _vp]
 lib.hif8_gemm_status.restype = _i
+lib.hif8_gemm_path_policy.argtypes = [_i]
+lib.hif8_gemm_path_policy.restype = _i
 lib.hif8_pts_search.argtypes = [_vp, _vp, _i, _i, _vp, _i64, _i, _i, _i, _i, _i, _vp, _vp, _vp, _sz, _vp]
 lib.hif8_pts_search.restype = _i
 lib.hif8_pts_workspace_bytes.argtypes = [_i, _i, _i, _i]
@@ -173,6 +175,14 @@ def hif8_gemm(Aq, lda, Wq, ldw, w_is_nk, Cmat, ldc, c_dtype, M, N, K, d_scale_ex
 
 def hif8_gemm_status(workspace, stream=None):
     return int(lib.hif8_gemm_status(_ptr(workspace), _stream(stream)))
+
+
+GEMM_PATH_AUTO, GEMM_PATH_EXPAND_BOTH = 0, 1
+
+
+def hif8_gemm_path_policy(policy):
+    """Sets which general kernel a large workspace selects; returns the previous setting, or 4 (HIF8_ERR_FLAGS) for an unknown one."""
+    return int(lib.hif8_gemm_path_policy(int(policy)))
 
 
 def hif8_pts_workspace_bytes(M, N, K, n_exp):

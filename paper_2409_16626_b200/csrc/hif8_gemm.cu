@@ -1646,6 +1646,14 @@ int launch_bf16_pair_gemm(const void* a_bf, const void* w_bf, int w_is_nk, GemmP
 
 using namespace hif8;
 
+static std::atomic<int> g_path_policy{HIF8_GEMM_PATH_AUTO};
+
+extern "C" int hif8_gemm_path_policy(int policy)
+{
+    if (policy != HIF8_GEMM_PATH_AUTO && policy != HIF8_GEMM_PATH_EXPAND_BOTH) return HIF8_ERR_FLAGS;
+    return g_path_policy.exchange(policy, std::memory_order_relaxed);
+}
+
 static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t* Wq, int64_t ldw, int w_is_nk, void* C,
                       int64_t ldc, int c_dtype, int M, int N, int K, const int* d_scale_exp_a, const int* d_scale_exp_w,
                       const int* d_scale_exp_w_channel, int accumulate, void* workspace, size_t workspace_bytes,
@@ -1742,7 +1750,14 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t
     // Otherwise the fused kernel decodes the byte tiles of every CTA in shared memory.
     const size_t bytes_a = (((size_t)M * K * 2) + 255) & ~(size_t)255, bytes_w = (((size_t)K * N * 2) + 255) & ~(size_t)255;
     const bool contiguous = lda == (a_is_km ? M : K) && ldw == (w_is_nk ? K : N);
-    if (contiguous && workspace_bytes >= kGemmWorkspaceBytes + bytes_a + bytes_w && !(reinterpret_cast<uintptr_t>(workspace) & 255)) {
+    // Expanding W as well only pays when the product is large enough to win back the pass over W (3 bytes per element
+    // moved) at the higher rate of the decode-once kernel: with about 267 flops per byte of copy bandwidth for that kernel and
+    // 217 for the A-expanded forms (their measured rates against the copy rate) the two meet near M = 1600 whatever N and K.
+    const double mk = (double)M * K, kn = (double)K * N, flops = 2.0 * mk * N;
+    const bool w_expansion_pays = g_path_policy.load(std::memory_order_relaxed) == HIF8_GEMM_PATH_EXPAND_BOTH ||
+                                  3.0 * kn + flops / 267.0 < flops / 217.0;
+    if (contiguous && w_expansion_pays && workspace_bytes >= kGemmWorkspaceBytes + bytes_a + bytes_w &&
+        !(reinterpret_cast<uintptr_t>(workspace) & 255)) {
         unsigned char* a_bf = reinterpret_cast<unsigned char*>(workspace) + kGemmWorkspaceBytes;
         unsigned char* w_bf = a_bf + bytes_a;
         // an A given as [K,M] is written as [M,K] while it is expanded: the tensor-core kernel streams a K-major A fastest

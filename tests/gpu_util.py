@@ -42,3 +42,18 @@ def bf16_half_ulp(x):
     what one round-to-nearest into BF16 can cost."""
     e = np.floor(np.log2(np.maximum(np.abs(x), 2.0 ** -126)))
     return 2.0 ** (e - 8)
+
+
+import contextlib
+
+
+@contextlib.contextmanager
+def both_operands_expanded(on):
+    """Within the block a workspace with room for both operands selects the kernel that expands both, whatever the size of
+    the product (hif8_gemm_path_policy); the previous setting is restored afterwards."""
+    import paper_2409_16626_b200 as H
+    before = H.hif8_gemm_path_policy(H.GEMM_PATH_EXPAND_BOTH if on else H.GEMM_PATH_AUTO)
+    try:
+        yield
+    finally:
+        H.hif8_gemm_path_policy(before)

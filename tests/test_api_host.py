@@ -91,3 +91,12 @@ def test_gemm_argument_errors_before_any_launch():
     assert g(M=0) == 0
     assert H.hif8_workspace_bytes(H.WS_GEMM) == 256
     assert H.hif8_launch_count() == before
+
+
+def test_gemm_path_policy_setting_round_trips():
+    # host-only: the setting is a process-wide integer; unknown values are refused and leave it alone
+    before = H.hif8_gemm_path_policy(H.GEMM_PATH_EXPAND_BOTH)
+    assert before in (H.GEMM_PATH_AUTO, H.GEMM_PATH_EXPAND_BOTH)
+    assert H.hif8_gemm_path_policy(7) == 4                   # HIF8_ERR_FLAGS
+    assert H.hif8_gemm_path_policy(H.GEMM_PATH_AUTO) == H.GEMM_PATH_EXPAND_BOTH
+    assert H.hif8_gemm_path_policy(before) == H.GEMM_PATH_AUTO

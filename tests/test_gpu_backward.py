@@ -9,7 +9,7 @@ import paper_2409_16626_b200 as H
 import workloads as W
 from oracle import hif8_oracle as O
 
-from gpu_util import bf16_half_ulp, dev_empty, to_dev
+from gpu_util import bf16_half_ulp, both_operands_expanded, dev_empty, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -99,9 +99,10 @@ def test_gemm_ex_layouts_and_accumulate(c_dtype, accumulate, a_is_km, w_is_nk, s
     c0 = C.float().cpu().numpy().astype(np.float64)
     wsb = H.hif8_workspace_bytes(H.WS_GEMM, (M * K if staged == "a" else M * K + K * N) if staged else 0)
     ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
-    H.hif8_gemm_ex(to_dev(Aq), Aq.shape[1], a_is_km, to_dev(Wq), Wq.shape[1], w_is_nk, C, ldc, c_dtype, M, N, K,
-                   torch.tensor([sa], dtype=torch.int32, device="cuda"), torch.tensor([sw], dtype=torch.int32, device="cuda"),
-                   None, accumulate, ws, wsb)
+    with both_operands_expanded(staged is True):
+        H.hif8_gemm_ex(to_dev(Aq), Aq.shape[1], a_is_km, to_dev(Wq), Wq.shape[1], w_is_nk, C, ldc, c_dtype, M, N, K,
+                       torch.tensor([sa], dtype=torch.int32, device="cuda"), torch.tensor([sw], dtype=torch.int32, device="cuda"),
+                       None, accumulate, ws, wsb)
     assert H.hif8_gemm_status(ws) == 0
     out = C.float().cpu().numpy().astype(np.float64)
     assert np.array_equal(out[:, N:], c0[:, N:])             # padding columns untouched

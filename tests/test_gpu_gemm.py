@@ -30,8 +30,13 @@ def run_gemm(Aq, Wq, w_is_nk, c_dtype, sa=None, sw=None, M=None, N=None, K=None,
     ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
     dsa = torch.tensor([sa], dtype=torch.int32, device="cuda") if sa is not None else None
     dsw = torch.tensor([sw], dtype=torch.int32, device="cuda") if sw is not None else None
-    H.hif8_gemm(dA, Aq.shape[1] if lda is None else lda, dW, Wq.shape[1] if ldw is None else ldw, int(w_is_nk), C, ldc,
-                c_dtype, M, N, K, dsa, dsw, ws, wsb)
+    # (staged = True means the kernel that takes both operands expanded, whatever the size of the product)
+    before = H.hif8_gemm_path_policy(H.GEMM_PATH_EXPAND_BOTH if staged is True else H.GEMM_PATH_AUTO)
+    try:
+        H.hif8_gemm(dA, Aq.shape[1] if lda is None else lda, dW, Wq.shape[1] if ldw is None else ldw, int(w_is_nk), C, ldc,
+                    c_dtype, M, N, K, dsa, dsw, ws, wsb)
+    finally:
+        H.hif8_gemm_path_policy(before)
     assert H.hif8_gemm_status(ws) == 0
     out = C.float().cpu().numpy().astype(np.float64)
     assert np.all(np.isnan(out[:, N:]))                      # padding columns untouched

@@ -9,7 +9,7 @@ import paper_2409_16626_b200 as H
 import workloads as W
 from oracle import hif8_oracle as O
 
-from gpu_util import NP_OF, bf16_half_ulp, dev_empty, to_dev
+from gpu_util import NP_OF, bf16_half_ulp, both_operands_expanded, dev_empty, to_dev
 
 pytestmark = pytest.mark.gpu
 MODES = [H.RND_TA, H.RND_HR, H.RND_SSR, H.RND_TE, H.RND_SR]
@@ -132,8 +132,9 @@ def test_gemm_channel_scaled(c_dtype, w_is_nk, staged):
     C = torch.full((M, ldc), float("nan"), dtype=torch.float32 if c_dtype == H.F32 else torch.bfloat16, device="cuda")
     wsb = H.hif8_workspace_bytes(H.WS_GEMM, M * K + K * N if staged else 0)
     ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
-    H.hif8_gemm_channel_scaled(to_dev(Aq), K, to_dev(Wq), Wq.shape[1], w_is_nk, C, ldc, c_dtype, M, N, K,
-                               torch.tensor([sa], dtype=torch.int32, device="cuda"), to_dev(sw.view(np.uint32)), ws, wsb)
+    with both_operands_expanded(bool(staged)):
+        H.hif8_gemm_channel_scaled(to_dev(Aq), K, to_dev(Wq), Wq.shape[1], w_is_nk, C, ldc, c_dtype, M, N, K,
+                                   torch.tensor([sa], dtype=torch.int32, device="cuda"), to_dev(sw.view(np.uint32)), ws, wsb)
     assert H.hif8_gemm_status(ws) == 0
     out = C.float().cpu().numpy().astype(np.float64)
     assert np.all(np.isnan(out[:, N:]))
