@@ -116,7 +116,8 @@ def test_channel_encode_degenerate_shapes():
     assert H.hif8_channel_amax_scale_encode(x, 7, out, 4, 4, 1, d_amax=d_amax, check=False) == 2
 
 
-@pytest.mark.parametrize("staged", [False, True])
+@pytest.mark.parametrize("staged", [False, True, "a"])  # "a": workspace for A alone (with [N,K] weights: the swapped form,
+                                                        # one weight exponent per accumulator row)
 @pytest.mark.parametrize("w_is_nk", [0, 1])
 @pytest.mark.parametrize("c_dtype", [H.F32, H.BF16])
 def test_gemm_channel_scaled(c_dtype, w_is_nk, staged):
@@ -130,9 +131,9 @@ def test_gemm_channel_scaled(c_dtype, w_is_nk, staged):
     sa = -7
     ldc = (N + 7) // 8 * 8
     C = torch.full((M, ldc), float("nan"), dtype=torch.float32 if c_dtype == H.F32 else torch.bfloat16, device="cuda")
-    wsb = H.hif8_workspace_bytes(H.WS_GEMM, M * K + K * N if staged else 0)
+    wsb = H.hif8_workspace_bytes(H.WS_GEMM, (M * K if staged == "a" else M * K + K * N) if staged else 0)
     ws = torch.empty(wsb, dtype=torch.uint8, device="cuda")
-    with both_operands_expanded(bool(staged)):
+    with both_operands_expanded(staged is True):
         H.hif8_gemm_channel_scaled(to_dev(Aq), K, to_dev(Wq), Wq.shape[1], w_is_nk, C, ldc, c_dtype, M, N, K,
                                    torch.tensor([sa], dtype=torch.int32, device="cuda"), to_dev(sw.view(np.uint32)), ws, wsb)
     assert H.hif8_gemm_status(ws) == 0
