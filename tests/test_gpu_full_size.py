@@ -97,7 +97,7 @@ def test_config4a_gradient_range_fp32_2_28():
     assert np.array_equal(got, want), f"SR: {np.count_nonzero(got != want)} mismatches"
 
 
-@pytest.mark.parametrize("staged", [True, False])
+@pytest.mark.parametrize("staged", [True, False, "a", "a_nk"])  # "a": workspace for A alone; "a_nk": the same with [N,K] weights
 def test_config5_gemm_8192x28672x8192(staged):
     # A BF16 8192 x 8192 N(0,1), W BF16 8192 x 28672 N(0,0.02): per-tensor scaled, encoded, multiplied; BF16 out
     M, N, K = 8192, 28672, 8192
@@ -113,9 +113,14 @@ def test_config5_gemm_8192x28672x8192(staged):
     H.hif8_amax_scale_encode(w, H.BF16, Wq, K * N, 14, H.RND_TA, 0, 0, None, None, se[1:2], None, ws, wsb)
     del a, w
     C = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
-    gb = H.hif8_workspace_bytes(H.WS_GEMM, M * K + K * N) if staged else H.hif8_workspace_bytes(H.WS_GEMM, 0)
+    gb = H.hif8_workspace_bytes(H.WS_GEMM, (M * K + K * N) if staged is True else (M * K if staged else 0))
     gws = torch.empty(gb, dtype=torch.uint8, device="cuda")
-    H.hif8_gemm(Aq, K, Wq, N, 0, C, N, H.BF16, M, N, K, se[0:1], se[1:2], gws, gb)
+    if staged == "a_nk":
+        Wt = Wq.view(K, N).t().contiguous().view(-1)
+        H.hif8_gemm(Aq, K, Wt, K, 1, C, N, H.BF16, M, N, K, se[0:1], se[1:2], gws, gb)
+        del Wt
+    else:
+        H.hif8_gemm(Aq, K, Wq, N, 0, C, N, H.BF16, M, N, K, se[0:1], se[1:2], gws, gb)
     assert H.hif8_gemm_status(gws) == 0
     sa, sw = [int(v) for v in se.cpu()]
     rng = np.random.default_rng(3)
