@@ -265,7 +265,8 @@ int hif8_fake_quant(const void* src, void* dst, int dtype, size_t n, int use_ama
  * tensor-core kernel streams BF16 tiles: several times faster for compute-bound shapes, same results.
  * In between -- hif8_workspace_bytes(HIF8_WS_GEMM, M*K) bytes or more, 256-byte aligned, A contiguous -- A alone is
  * expanded into the workspace and the kernel decodes only the W tiles (any ldw): for when the weight's BF16 copy does
- * not fit but the activation's does; same results.
+ * not fit but the activation's does; same results.  A workspace with room for both operands takes this form too while
+ * the product is too small to win the pass over W back (see hif8_gemm_path_policy).
  * Products with at most 64 rows of A (and A given as [M,K]) take a weight-streaming kernel whatever the workspace;
  * with the workspace size above it spreads the weight bytes evenly over all SMs (partial sums of a column slab that
  * two SMs share go through the workspace and are added in a fixed order: results are reproducible run to run).
