@@ -482,7 +482,7 @@ def extra_results(H, torch, hbm_peak, tf_peak, peak_kind, tf_sustained=None):
 # Named workloads for a profiler (a few launches each; nothing is timed or printed but a completion line)
 # --------------------------------------------------------------------------------------------------------------
 CASES = ("convert_f32", "fq_bf16", "encode_modes_f32", "encode_modes_bf16", "transpose_bf16", "gemm", "gemm_fused", "gemm_narrow",
-         "gemm_forms", "channel_bf16")
+         "gemm_forms", "gemm_a_expanded", "channel_bf16")
 
 
 def run_case(case, reps):
@@ -490,7 +490,8 @@ def run_case(case, reps):
     fq_bf16: BF16 4096x8192 fake-quant, TA / HR / TE, fused amax and given scale; encode_modes_f32 / encode_modes_bf16:
     2^25 log-uniform values in every rounding mode; transpose_bf16: BF16 8192^2 flat and transposed-store encode, TA and
     HR; gemm: HiF8 GEMM 4096 x 7168 x 4096 on the decode-once and the fused path (gemm_fused: the fused path only);
-    gemm_forms: the four operand layouts on the decode-once path; gemm_narrow: 16 x 8192 x 8192 with weights as [K,N] and
+    gemm_forms: the four operand layouts on the decode-once path; gemm_a_expanded: the same size with a workspace for A alone, [K,N] and [N,K] weights;
+    gemm_narrow: 16 x 8192 x 8192 with weights as [K,N] and
     [N,K] (equal ranges of the weight per SM); channel_bf16: per-channel scaled encode of a BF16 8192 x 14336 weight by column and by row, plus the overflow
     check.  Inputs are seeded device-side random tensors."""
     import torch
@@ -556,6 +557,16 @@ def run_case(case, reps):
         for r in range(reps):
             H.hif8_gemm(A, K, Wt, N, 0, C, N, H.BF16, M, N, K, None, None, gws, big)
             H.hif8_gemm(A, K, Wt, K, 1, C, N, H.BF16, M, N, K, None, None, gws, big)
+    elif case == "gemm_a_expanded":
+        M, N, K = 4096, 7168, 4096
+        A = torch.randint(8, 100, (M * K,), dtype=torch.uint8, device="cuda", generator=g)
+        Wt = torch.randint(8, 100, (K * N,), dtype=torch.uint8, device="cuda", generator=g)
+        C = torch.zeros(M, N, dtype=torch.bfloat16, device="cuda")
+        a_only = H.hif8_workspace_bytes(H.WS_GEMM, M * K)
+        gws = torch.empty(a_only, dtype=torch.uint8, device="cuda")
+        for r in range(reps):
+            H.hif8_gemm(A, K, Wt, N, 0, C, N, H.BF16, M, N, K, None, None, gws, a_only)   # [K,N] weights
+            H.hif8_gemm(A, K, Wt, K, 1, C, N, H.BF16, M, N, K, None, None, gws, a_only)   # [N,K] weights: the swapped form
     elif case == "gemm_forms":
         M, N, K = 4096, 7168, 4096
         A = torch.randint(8, 100, (M * K,), dtype=torch.uint8, device="cuda", generator=g)
