@@ -450,6 +450,16 @@ def extra_results(H, torch, hbm_peak, tf_peak, peak_kind, tf_sustained=None):
         narrow[f"M={Mn}"] = d
         row(f"gemm_narrow_{Mn}x28672x8192", d, "hbm (weight bytes)")
         del Cn
+    # prefill-sized products against the same weight, with the full workspace: below about 1600 rows the call expands A alone
+    mid = {}
+    for Mm in (256, 1024):
+        Cm = torch.empty(Mm, N, dtype=torch.bfloat16, device="cuda")
+        stm = timed(lambda r: H.hif8_gemm(Aq, K, Wq, N, 0, Cm, N, H.BF16, Mm, N, K, se[0:1], se[1:2], gws, gws_b), 10, rest_s=REST)
+        mid[f"M={Mm}"] = tensor(stm, 2.0 * Mm * N * K, us=stm["ms"] * 1e3, device_status=H.hif8_last_device_status())
+        row(f"gemm_{Mm}x28672x8192_full_workspace", mid[f"M={Mm}"], "tensor")
+        del Cm
+    out["gemm_midM_x28672x8192"] = {"bound": "tensor", "shapes": mid, "peak": tf_peak, "peak_kind": f"of {peak_kind} (cuBLAS BF16 burst)",
+                                    "note": "the weight bytes alone take 36 us at the copy rate; 256 rows run as one tile row of 256"}
     out["gemm_narrow_Mx28672x8192"] = {"bound": "hbm", "bytes": "K*N weight bytes + M*K + 2*M*N", "shapes": narrow,
                                        "peak": hbm_peak, "peak_kind": f"of {peak_kind}"}
     out["gemm_8192x28672x8192"] = {
