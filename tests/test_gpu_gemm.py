@@ -261,3 +261,27 @@ def test_tensor_map_cache_survives_eviction_and_pointer_reuse():
         want = (tab[Aq].astype(np.int64) @ tab[Wq].astype(np.int64)).astype(np.float64)
         assert np.array_equal(C.cpu().numpy().astype(np.float64), want), (it, M, N, K)
     assert H.hif8_last_device_status(torch.cuda.Stream()) == 0   # a stream that never saw a GEMM
+
+
+@pytest.mark.parametrize("mode", ["fused", "a", "a_nk", "staged"])
+def test_gemm_repeated_runs_are_bit_identical(mode):
+    # The order of the sums is fixed (k-blocks in order, one accumulator per output), so repeated runs of one product must
+    # agree bit for bit; an operand tile handed to the tensor core before its last byte was in place -- the hand-over between
+    # the decode warps of both CTAs of a pair and the MMA thread -- would show as a difference in some run.  Full tiles, many
+    # k-blocks, every general kernel; the first run is checked against the oracle on sampled outputs.
+    M, N, K = 1024, 2048, 8192
+    Aq = W.random_codes((M, K), seed=77)
+    Wkn = W.random_codes((K, N), seed=78)
+    for t in (Aq, Wkn):
+        t[(t == 0x80) | ((t & 0x7F) == 0x6F)] = 0x21
+    w_is_nk = mode == "a_nk"
+    Wq = np.ascontiguousarray(Wkn.T) if w_is_nk else Wkn
+    staged = {"fused": False, "a": "a", "a_nk": "a", "staged": True}[mode]
+    first = run_gemm(Aq, Wq, w_is_nk, H.F32, sa=2, sw=-3, staged=staged)
+    rng = np.random.default_rng(9)
+    rows, cols = rng.integers(0, M, 4000), rng.integers(0, N, 4000)
+    Cs, S = O.gemm_entries(Aq, Wkn, False, 2, -3, rows, cols)
+    assert np.all(np.abs(first[rows, cols] - Cs) <= 1e-5 * S)
+    for _ in range(8):
+        again = run_gemm(Aq, Wq, w_is_nk, H.F32, sa=2, sw=-3, staged=staged)
+        assert np.array_equal(first, again)
