@@ -45,7 +45,7 @@ namespace {
 constexpr int BM = 128, BN = 256, BK = 64;
 constexpr int kStages8 = 4;    // staging ring of HiF8 byte tiles
 constexpr int kStagesBf = 4;   // ring of decoded BF16 operand tiles
-constexpr int kStagesBfSwapped = 8, kMaxStagesBf = 8;  // the swapped form (see hif8_gemm_kernel) has room for two stages per group
+constexpr int kStagesBfSwapped = 4, kMaxStagesBf = 8;  // the swapped form (see hif8_gemm_kernel): stages of 128 k, twice the size
 constexpr int kEpiWarps = 4, kDecodeWarps = 16;
 // The decode warps work in groups, group g on the k-blocks kb = g (mod kDecodeGroups): several k-blocks are in the
 // decode stage at once, which covers the latency of each one's lookups, proxy fence and barrier hand-over.  Group g
@@ -514,8 +514,8 @@ constexpr uint32_t kSmemBytesWide = 227 * 1024;  // the whole opt-in maximum; th
 
 // PLAN 0: slots around the 64 KiB table.  1: the layout of SmemLayout (A operand tiles in shared memory).  2: the swapped
 // form -- eight operand stages of 16 KiB, four byte stages of 8 KiB, the 32 KiB table, barriers, one after the other.
-constexpr int kStages8Swapped = 8;  // byte stages of the swapped form (A bytes only: 8 KiB each)
-constexpr uint32_t kSmemBytesSwapped = kStagesBfSwapped * kBBfBytes + kStages8Swapped * kA8Bytes + 256 * 32 * 4 + kBarsBytes + 1024;
+constexpr int kStages8Swapped = 4;  // byte stages of the swapped form (A bytes only, 128 k: 16 KiB each)
+constexpr uint32_t kSmemBytesSwapped = kStagesBfSwapped * 2 * kBBfBytes + kStages8Swapped * 2 * kA8Bytes + 256 * 32 * 4 + kBarsBytes + 1024;
 template <int PLAN>
 struct FusedSmem {
     static constexpr bool FIXED = PLAN == 1;
@@ -529,8 +529,8 @@ struct FusedSmem {
         if (FIXED) {
             lut = base + SmemLayout::lut; bars = base + SmemLayout::bars; behind = 0; n_front = 0; end = base + SmemLayout::total;
         } else if (PLAN == 2) {
-            behind = 0; n_front = kStagesBfSwapped;
-            lut = base + kStagesBfSwapped * kBBfBytes + kStages8Swapped * kA8Bytes; bars = lut + kLutBytesNarrow; end = bars + kBarsBytes;
+            behind = 0; n_front = 2 * kStagesBfSwapped;
+            lut = base + kStagesBfSwapped * 2 * kBBfBytes + kStages8Swapped * 2 * kA8Bytes; bars = lut + kLutBytesNarrow; end = bars + kBarsBytes;
         } else if (!kWideLut) {
             // table with rows of 128 bytes: no alignment to honour, everything in a row: slots, table, barriers
             n_front = (int)kFusedSlots; behind = 0;
@@ -548,10 +548,10 @@ struct FusedSmem {
     }
     __device__ uint32_t slot(int i) const { return i < n_front ? base + (uint32_t)i * kSlotBytes : behind + (uint32_t)(i - n_front) * kSlotBytes; }
     __device__ uint32_t a_bf(int s) const { return base + SmemLayout::bf + s * (kABfBytes + kBBfBytes); }                       // FIXED only
-    __device__ uint32_t w_bf(int s) const { return FIXED ? a_bf(s) + kABfBytes : slot(s); }
+    __device__ uint32_t w_bf(int s) const { return PLAN == 2 ? base + (uint32_t)s * 2 * kBBfBytes : (FIXED ? a_bf(s) + kABfBytes : slot(s)); }
     __device__ uint32_t a_u8(int s) const
     {
-        if (PLAN == 2) return base + kStagesBfSwapped * kBBfBytes + (uint32_t)s * kA8Bytes;
+        if (PLAN == 2) return base + kStagesBfSwapped * 2 * kBBfBytes + (uint32_t)s * 2 * kA8Bytes;
         return FIXED ? base + SmemLayout::u8 + s * (kA8Bytes + kB8Bytes) : slot(kStagesBf + s);
     }
     // staging box j (16 KiB) of the result tile: the operand stages, idle once the accumulator is complete
@@ -611,7 +611,9 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
     int tile_m, tile_n;
     tile_coords((int)(blockIdx.x >> 1), (p.M + 2 * BM - 1) / (2 * BM), p.tiles_n, tile_m, tile_n);
     const int m0 = tile_m * 2 * BM + (int)rank * BM, n0 = tile_n * BN, nh = n0 + (int)rank * (BN / 2);
-    const int num_kb = (p.K + BK - 1) / BK;
+    // k per operand stage: 64, or (SWAPPED) 128 -- one hand-over, one commit and one probe by the MMA thread per 128 k
+    constexpr int KB = SWAPPED ? 2 * BK : BK;
+    const int num_kb = (p.K + KB - 1) / KB;
 
     // ---- set-up
     fill_decode_table<(1 << (kLutShift - 2))>(lut_all, warp, lane, kThreads / 32);  // rows of 1 << kLutShift bytes
@@ -645,9 +647,11 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 const int sb = kb % kSB, rb = kb / kSB;
                 if (rb > 0 && !mbar_wait(bar_bf_empty(sb), (rb - 1) & 1, abort_flag, p.status, 6)) break;
                 if (*abort_flag) break;
-                if (leader) mbar_arrive_expect_tx(bar_bf_full(sb), 2 * (SWAPPED ? kBBfBytes : kABfBytes));
-                if (SWAPPED) tma_load_3d_pair(plan.w_bf(sb), &map_w, kb * BK, nh, 0, map_to_cta(bar_bf_full(sb), 0));
-                else tma_load_3d_pair(plan.a_bf(sb), &map_a, kb * BK, m0, 0, map_to_cta(bar_bf_full(sb), 0));
+                if (leader) mbar_arrive_expect_tx(bar_bf_full(sb), SWAPPED ? 4 * kBBfBytes : 2 * kABfBytes);
+                if (SWAPPED) {  // 128 k of BF16 are two boxes of 64 (the swizzle span), into the two halves of the stage
+                    tma_load_3d_pair(plan.w_bf(sb), &map_w, kb * KB, nh, 0, map_to_cta(bar_bf_full(sb), 0));
+                    tma_load_3d_pair(plan.w_bf(sb) + kBBfBytes, &map_w, kb * KB + BK, nh, 0, map_to_cta(bar_bf_full(sb), 0));
+                } else tma_load_3d_pair(plan.a_bf(sb), &map_a, kb * BK, m0, 0, map_to_cta(bar_bf_full(sb), 0));
             }
         }
         __syncwarp();
@@ -661,9 +665,9 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 if (round > 0 && !mbar_wait(bar_u8_empty(s), (round - 1) & 1, abort_flag, p.status, 1)) break;
                 if (*abort_flag) break;
                 const uint32_t dst_a = plan.a_u8(s), dst_b = plan.w_u8(s);
-                mbar_arrive_expect_tx(bar_u8_full(s), (A_BF16 ? 0u : kA8Bytes) + (SWAPPED ? 0u : kB8Bytes));
+                mbar_arrive_expect_tx(bar_u8_full(s), (A_BF16 ? 0u : (SWAPPED ? 2 * kA8Bytes : kA8Bytes)) + (SWAPPED ? 0u : kB8Bytes));
                 if (A_IS_KM) tma_load_2d(dst_a, &map_a, m0, kb * BK, bar_u8_full(s));
-                else if (!A_BF16) tma_load_2d(dst_a, &map_a, kb * BK, m0, bar_u8_full(s));
+                else if (!A_BF16) tma_load_2d(dst_a, &map_a, kb * KB, m0, bar_u8_full(s));  // (SWAPPED: one box of 128 k)
                 if (SWAPPED) {}
                 else if (W_IS_NK) tma_load_2d(dst_b, &map_w, kb * BK, nh, bar_u8_full(s));
                 else tma_load_2d(dst_b, &map_w, nh, kb * BK, bar_u8_full(s));
@@ -700,15 +704,16 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 bool next_ready = true;
                 uint32_t a_next = 0, b_next = 0, t_next = 0;
 #pragma unroll
-                for (int kk = 0; kk < BK / 16; kk++) {
-                    if (kk == BK / 16 - 1 && kb + 1 < num_kb) {
+                for (int kk = 0; kk < KB / 16; kk++) {
+                    if (kk == KB / 16 - 1 && kb + 1 < num_kb) {
                         const int sn = (kb + 1) % kSB;
                         next_ready = mbar_try_wait(bar_bf_full(sn), (uint32_t)(((kb + 1) / kSB) & 1));
                         a_next = plan.a_bf(sn); b_next = plan.w_bf(sn);
-                        t_next = tmem_base + kTmemColsAcc + (uint32_t)(sn * kTmemAStageCols);
+                        t_next = tmem_base + kTmemColsAcc + (uint32_t)(sn * (KB / 2));
                     }
-                    // K-major: 16 k = 32 bytes inside the 128-byte row; MN-major: 16 k = two 1024-byte atoms
-                    const uint64_t db = W_IS_NK ? make_smem_desc(b_addr + kk * 32, 16, 1024)
+                    // K-major: 16 k = 32 bytes inside the 128-byte row (SWAPPED: the second 64 k are the stage's second half);
+                    // MN-major: 16 k = two 1024-byte atoms
+                    const uint64_t db = W_IS_NK ? make_smem_desc(b_addr + (kk >> 2) * kBBfBytes + (kk & 3) * 32, 16, 1024)
                                                 : make_smem_desc(b_addr + kk * 2048, 8192, 1024);
                     if (A_IS_KM) {
                         tc_mma_bf16_pair(tmem_base, make_smem_desc(a_addr + kk * 2048, 8192, 1024), db, idesc, (kb > 0 || kk > 0) ? 1u : 0u);
@@ -752,6 +757,28 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 load_tile_chunks<!W_IS_NK>(b8, dt, vw);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_u8_empty(s8));
+            } else if (SWAPPED) {
+                // As below, with rows of 128 k: the byte tile arrives with the 128-byte TMA swizzle (chunk j of row r at chunk
+                // j ^ (r & 7)), the row is decoded in two halves of 64 into the two halves of the 64-column stage.
+                const int quarter = warp & 3, r = quarter * 32 + lane;
+                const uint32_t a_row = a8 + (uint32_t)r * KB, sw = (uint32_t)r & 7u;
+                uint4 va[KB / 16];
+#pragma unroll
+                for (int j = 0; j < KB / 16; j++) va[j] = lds_v4(a_row + (((uint32_t)j ^ sw) << 4));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_u8_empty(s8));
+#pragma unroll
+                for (int half = 0; half < 2; half++) {
+                    uint32_t o[BK / 2];
+#pragma unroll
+                    for (int j = 0; j < BK / 16; j++) {
+                        const uint4 v = va[half * (BK / 16) + j];
+                        const uint4 lo = decode8<kLutShift>(make_uint2(v.x, v.y), lut), hi = decode8<kLutShift>(make_uint2(v.z, v.w), lut);
+                        o[8 * j + 0] = lo.x; o[8 * j + 1] = lo.y; o[8 * j + 2] = lo.z; o[8 * j + 3] = lo.w;
+                        o[8 * j + 4] = hi.x; o[8 * j + 5] = hi.y; o[8 * j + 6] = hi.z; o[8 * j + 7] = hi.w;
+                    }
+                    tmem_st_32x32b_x32(tmem_base + ((uint32_t)(quarter * 32) << 16) + kTmemColsAcc + (uint32_t)(sb * (KB / 2) + half * (BK / 2)), o);
+                }
             } else {
                 // A [M,K]: this thread owns row (its warp's quarter of the 128 tensor-memory lanes) * 32 + lane.  The byte
                 // tile arrives with the 64-byte TMA swizzle (16-byte chunk j of row r sits at chunk j ^ ((r >> 1) & 3)), so
@@ -761,7 +788,7 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
                 uint4 va[BK / 16];
 #pragma unroll
                 for (int j = 0; j < BK / 16; j++) va[j] = lds_v4(a_row + (((uint32_t)j ^ sw) << 4));
-                if (!SWAPPED) load_tile_chunks<!W_IS_NK>(b8, dt, vw);
+                load_tile_chunks<!W_IS_NK>(b8, dt, vw);
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_u8_empty(s8));
                 uint32_t o[BK / 2];  // 64 BF16 of this row, two per column
@@ -1788,7 +1815,7 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t
             const long long tiles2s = (long long)((N + 2 * BM - 1) / (2 * BM)) * q.tiles_n;
             if (tiles2s > 0x3FFFFFFF) return HIF8_ERR_SHAPE;
             CUtensorMap map_wb, map_ab;
-            if (!make_map(&map_wb, Wq, (uint64_t)K, (uint64_t)N, (uint64_t)ldw, BK, BM, false, 64)) return HIF8_ERR_CUDA;
+            if (!make_map(&map_wb, Wq, (uint64_t)K, (uint64_t)N, (uint64_t)ldw, 2 * BK, BM, false, 128)) return HIF8_ERR_CUDA;  // rows of 128 k
             if (!make_map3(&map_ab, a_bf, (uint64_t)K, (uint64_t)M, 1, 0, BK, BN / 2)) return HIF8_ERR_CUDA;
             cudaLaunchConfig_t cs{};
             cs.gridDim = dim3(2u * (unsigned)tiles2s);
