@@ -509,6 +509,8 @@ def run_case(case, reps):
     g = torch.Generator(device="cuda")
     g.manual_seed(1)
     ws = torch.empty(256, dtype=torch.uint8, device="cuda")
+    if case in ("gemm", "gemm_forms"):  # these cases exist to capture the decode-once kernel: ask for it whatever the size
+        H.hif8_gemm_path_policy(H.GEMM_PATH_EXPAND_BOTH)
     if case == "convert_f32":
         n = N_EL
         xs = [torch.randn(n, generator=g, device="cuda") for _ in range(3)]

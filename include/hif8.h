@@ -324,8 +324,8 @@ int hif8_gemm_status(const void* workspace, hif8_stream_t stream);
 
 /*
  * Which general kernel a large workspace selects.  HIF8_GEMM_PATH_AUTO (the default): with room for both operands W is
- * expanded too only when the product is large enough to win that pass back (about 1600 rows of A and more); below that A
- * alone is expanded.  HIF8_GEMM_PATH_EXPAND_BOTH: both operands are expanded whenever the workspace has room (for
+ * expanded too only when the product is large enough to win that pass back (from about 1500 rows of A with [K,N] weights,
+ * about 4800 with [N,K] weights); below that A alone is expanded.  HIF8_GEMM_PATH_EXPAND_BOTH: both operands are expanded whenever the workspace has room (for
  * measurements and tests of that kernel on small products).  Process-wide; returns the previous setting (0 or 1), or
  * HIF8_ERR_FLAGS for an unknown one.  Results do not depend on it.
  */

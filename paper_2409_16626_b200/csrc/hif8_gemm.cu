@@ -1778,11 +1778,12 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t
     const size_t bytes_a = (((size_t)M * K * 2) + 255) & ~(size_t)255, bytes_w = (((size_t)K * N * 2) + 255) & ~(size_t)255;
     const bool contiguous = lda == (a_is_km ? M : K) && ldw == (w_is_nk ? K : N);
     // Expanding W as well only pays when the product is large enough to win back the pass over W (3 bytes per element
-    // moved) at the higher rate of the decode-once kernel: with about 267 flops per byte of copy bandwidth for that kernel and
-    // 217 for the A-expanded forms (their measured rates against the copy rate) the two meet near M = 1600 whatever N and K.
+    // moved) at the higher rate of the decode-once kernel: with about 268 flops per byte of copy bandwidth for that kernel,
+    // 233 for the swapped A-expanded form ([N,K] weights) and 210 for the other (their measured rates against the copy rate)
+    // they meet near M = 4800 and M = 1450, whatever N and K.
     const double mk = (double)M * K, kn = (double)K * N, flops = 2.0 * mk * N;
     const bool w_expansion_pays = g_path_policy.load(std::memory_order_relaxed) == HIF8_GEMM_PATH_EXPAND_BOTH ||
-                                  3.0 * kn + flops / 267.0 < flops / 217.0;
+                                  3.0 * kn + flops / 268.0 < flops / (w_is_nk ? 233.0 : 210.0);
     if (contiguous && w_expansion_pays && workspace_bytes >= kGemmWorkspaceBytes + bytes_a + bytes_w &&
         !(reinterpret_cast<uintptr_t>(workspace) & 255)) {
         unsigned char* a_bf = reinterpret_cast<unsigned char*>(workspace) + kGemmWorkspaceBytes;
