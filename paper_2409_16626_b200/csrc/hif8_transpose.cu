@@ -112,6 +112,28 @@ __global__ void __launch_bounds__(kThreads, MODE == HIF8_RND_SR ? 4 : 6) encode_
                 my_words[(2 * m) * kTileWords] = __byte_perm(c01, c23, 0x5410) & (~__byte_perm(s01, s23, 0x5410) | 0x7F7F7F7Fu);
                 my_words[(2 * m + 1) * kTileWords] = __byte_perm(c01, c23, 0x7632) & (~__byte_perm(s01, s23, 0x7632) | 0x7F7F7F7Fu);
             }
+        } else if constexpr (MODE == HIF8_RND_TA) {
+            // The table is read with the sign folded away (its non-negative half): the lanes of a warp then meet in
+            // about half as many distinct words, and the byte lookups, which share the load/store pipe with the tile,
+            // cost about half the wavefronts on zero-centred data.  The signs of the four rows of a column go back
+            // onto the packed word: bit 7 of every code that is not the single zero (code + 0x7F carries into bit 7
+            // for 0x01 .. 0x80; NaN, 0x80, keeps its encoding either way).
+#pragma unroll
+            for (int k = 0; k < PV; k++) {
+                uint32_t c[4], w[4];
+#pragma unroll
+                for (int j = 0; j < 4; j++) {
+                    float x; uint32_t raw;
+                    unpack<SRC>(v[j], k, x, raw);
+                    c[j] = sm.ta[__float_as_uint(fabsf(x) * scale) >> 19];
+                    constexpr int kDiv = SRC == HIF8_F32 ? 1 : 2;
+                    w[j] = (k / kDiv) == 0 ? v[j].x : ((k / kDiv) == 1 ? v[j].y : ((k / kDiv) == 2 ? v[j].z : v[j].w));
+                }
+                const bool top = SRC == HIF8_F32 || (k & 1);  // the element's sign is bit 7 of byte 3 (else of byte 1) of its word
+                const uint32_t s01 = __byte_perm(w[0], w[1], top ? 0x0073u : 0x0051u), s23 = __byte_perm(w[2], w[3], top ? 0x0073u : 0x0051u);
+                const uint32_t word = c[0] | (c[1] << 8) | (c[2] << 16) | (c[3] << 24);
+                my_words[k * kTileWords] = word | ((word + 0x7F7F7F7Fu) & __byte_perm(s01, s23, 0x5410u) & 0x80808080u);
+            }
         } else {
             // columns outermost: the four codes of a column are packed and stored at once
 #pragma unroll

@@ -66,6 +66,17 @@ def test_encode_transpose_modes_flags_device_exponent_and_misalignment(dtype, mo
     assert np.array_equal(flat.cpu().numpy().reshape(x.shape).T, q)
 
 
+@pytest.mark.parametrize("flags", [0, H.FLAG_SATURATE | H.FLAG_NAN_TO_ZERO])
+@pytest.mark.parametrize("dtype", [H.BF16, H.F16])
+def test_encode_transpose_every_16_bit_pattern(dtype, flags):
+    # every sign, zero, subnormal, Inf and NaN pattern through the tiled kernel (Section 3: special values and options)
+    x = np.arange(65536, dtype=np.uint16).reshape(256, 256)
+    for mode, omode in ((H.RND_TA, O.TA), (H.RND_HR, O.HR), (H.RND_TE, O.TE)):
+        for se in (0, -9):
+            q = run_transpose(x, dtype, scale_exp=se, rnd=mode, flags=flags)
+            assert np.array_equal(q, O.encode_transpose(x, dtype, se, omode, flags, 0, quick=True)), (mode, se)
+
+
 def test_encode_transpose_argument_checks():
     x = torch.ones(64, device="cuda")
     out = torch.empty(64, dtype=torch.uint8, device="cuda")
