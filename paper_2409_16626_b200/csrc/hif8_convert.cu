@@ -99,28 +99,20 @@ __device__ __forceinline__ void convert_group(const ConvParams& p, const SmemTab
             continue;
         }
         if constexpr (MODE == HIF8_RND_TA && !FQ && !PATTERN) {  // (a pattern sweep has neighbouring lanes in one table word anyway)
-            // The code table is read with the sign folded away (its non-negative half; the negative half lies a multiple of
-            // the bank period above it, so +x and -x of one binade would meet in one bank).  The signs go back onto the
-            // packed words: bit 7 of every code that is not the single zero (code + 0x7F carries into bit 7 for 0x01 .. 0x80;
-            // NaN, 0x80, keeps its encoding either way).
-            uint32_t c[PV];
+            // the code table is read sign-free, the signs go back onto the packed words (see ta_magnitude_code)
+            uint32_t c[8];
 #pragma unroll
             for (int k = 0; k < PV; k++) {
                 float x; uint32_t raw;
                 unpack<SRC>(v[j], k, x, raw);
                 if (AMAX) amax = amax_step(amax, x);
-                c[k] = sm.ta[__float_as_uint(fabsf(x) * scale) >> 19];
+                c[k] = ta_magnitude_code(x, scale, sm.ta);
             }
-            const uint32_t w0 = c[0] | (c[1] << 8) | (c[2] << 16) | (c[3] << 24);
-            if (PV == 4) {
-                const uint32_t sg = __byte_perm(__byte_perm(v[j].x, v[j].y, 0x0073u), __byte_perm(v[j].z, v[j].w, 0x0073u), 0x5410u);
-                __stcs(reinterpret_cast<uint32_t*>(p.dst) + u, w0 | ((w0 + 0x7F7F7F7Fu) & sg & 0x80808080u));
-            } else {
-                const uint32_t w1 = c[PV - 4] | (c[PV - 3] << 8) | (c[PV - 2] << 16) | (c[PV - 1] << 24);
-                const uint32_t s0 = __byte_perm(v[j].x, v[j].y, 0x7531u), s1 = __byte_perm(v[j].z, v[j].w, 0x7531u);  // bytes 1 and 3 of each word
-                __stcs(reinterpret_cast<uint2*>(p.dst) + u, make_uint2(w0 | ((w0 + 0x7F7F7F7Fu) & s0 & 0x80808080u),
-                                                                       w1 | ((w1 + 0x7F7F7F7Fu) & s1 & 0x80808080u)));
-            }
+            uint32_t w0 = c[0] | (c[1] << 8) | (c[2] << 16) | (c[3] << 24), w1 = 0;
+            if (PV == 8) w1 = c[4] | (c[5] << 8) | (c[6] << 16) | (c[7] << 24);
+            put_signs<SRC>(v[j], w0, w1);
+            if (PV == 4) __stcs(reinterpret_cast<uint32_t*>(p.dst) + u, w0);
+            else __stcs(reinterpret_cast<uint2*>(p.dst) + u, make_uint2(w0, w1));
             continue;
         }
         uint32_t codes[PV];

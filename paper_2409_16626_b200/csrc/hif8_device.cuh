@@ -289,6 +289,30 @@ __device__ __forceinline__ bool pair32_lookup(float y, uint32_t raw, const uint3
     return u >= thr;
 }
 
+// Round half away with the code table read sign-free.  The table's negative half lies 4096 bytes (a multiple of the
+// 128-byte bank period) above the positive one, so +x and -x of one binade would always meet in one bank; reading the
+// non-negative half only costs a warp about half the shared-memory wavefronts on zero-centred data.
+__device__ __forceinline__ uint32_t ta_magnitude_code(float x, float scale, const uint8_t* s_ta)
+{
+    return s_ta[__float_as_uint(fabsf(x) * scale) >> 19];
+}
+
+// ... and the signs of a source vector's elements put back onto their packed magnitude codes (w0: elements 0-3, w1:
+// elements 4-7 of a 16-bit source): bit 7 of every code that is not the single zero (code + 0x7F carries into bit 7 for
+// 0x01 .. 0x80; NaN, 0x80, keeps its encoding either way).
+template <int SRC>
+__device__ __forceinline__ void put_signs(const uint4& v, uint32_t& w0, uint32_t& w1)
+{
+    if (SRC == HIF8_F32) {
+        const uint32_t s = __byte_perm(__byte_perm(v.x, v.y, 0x0073u), __byte_perm(v.z, v.w, 0x0073u), 0x5410u);  // byte 3 of each word
+        w0 |= (w0 + 0x7F7F7F7Fu) & s & 0x80808080u;
+    } else {
+        const uint32_t s0 = __byte_perm(v.x, v.y, 0x7531u), s1 = __byte_perm(v.z, v.w, 0x7531u);  // bytes 1 and 3 of each word
+        w0 |= (w0 + 0x7F7F7F7Fu) & s0 & 0x80808080u;
+        w1 |= (w1 + 0x7F7F7F7Fu) & s1 & 0x80808080u;
+    }
+}
+
 template <int MODE, int SRC>
 __device__ __forceinline__ uint32_t encode_one(float x, uint32_t raw, float scale, const uint8_t* s_ta,
                                                const uint32_t* s_thr, uint32_t word)

@@ -113,11 +113,9 @@ __global__ void __launch_bounds__(kThreads, MODE == HIF8_RND_SR ? 4 : 6) encode_
                 my_words[(2 * m + 1) * kTileWords] = __byte_perm(c01, c23, 0x7632) & (~__byte_perm(s01, s23, 0x7632) | 0x7F7F7F7Fu);
             }
         } else if constexpr (MODE == HIF8_RND_TA) {
-            // The table is read with the sign folded away (its non-negative half): the lanes of a warp then meet in
-            // about half as many distinct words, and the byte lookups, which share the load/store pipe with the tile,
-            // cost about half the wavefronts on zero-centred data.  The signs of the four rows of a column go back
-            // onto the packed word: bit 7 of every code that is not the single zero (code + 0x7F carries into bit 7
-            // for 0x01 .. 0x80; NaN, 0x80, keeps its encoding either way).
+            // The table is read sign-free (see ta_magnitude_code: the byte lookups share the load/store pipe with the
+            // tile) and the signs of the four rows of a column go back onto the packed word: bit 7 of every code that
+            // is not the single zero (code + 0x7F carries into bit 7 for 0x01 .. 0x80; NaN, 0x80, keeps its encoding).
 #pragma unroll
             for (int k = 0; k < PV; k++) {
                 uint32_t c[4], w[4];
@@ -125,7 +123,7 @@ __global__ void __launch_bounds__(kThreads, MODE == HIF8_RND_SR ? 4 : 6) encode_
                 for (int j = 0; j < 4; j++) {
                     float x; uint32_t raw;
                     unpack<SRC>(v[j], k, x, raw);
-                    c[j] = sm.ta[__float_as_uint(fabsf(x) * scale) >> 19];
+                    c[j] = ta_magnitude_code(x, scale, sm.ta);
                     constexpr int kDiv = SRC == HIF8_F32 ? 1 : 2;
                     w[j] = (k / kDiv) == 0 ? v[j].x : ((k / kDiv) == 1 ? v[j].y : ((k / kDiv) == 2 ? v[j].z : v[j].w));
                 }
