@@ -935,6 +935,8 @@ hif8_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constan
 // weight bytes once, so the roles are swapped: a CTA streams a slab of 128 weight columns as the 128-row MMA operand and
 // the few activation rows are the narrow operand (MMA N = M rounded up to 16).  One CTA per SM, no pairs:
 //   warp 4        copies: per pair block (two k-blocks) one tile of weight bytes and one of activation bytes
+//                 (activations expanded to BF16 beforehand, when the workspace has room: their tiles instead, one per
+//                 k-block, straight into the operand stages; the groups then decode weights only)
 //   warps 6-21    four decode groups, group g on the k-blocks it = g (mod 4): a thread owns one weight column of the slab,
 //                 decodes its 64 bytes of the k-block and stores them as its lane of a weight stage in tensor memory (the A
 //                 operand of tcgen05.mma may live there); the group also decodes the activation tile into shared memory
@@ -990,7 +992,7 @@ struct NarrowPlan {
     int pmax;            // slices per slab
 };
 
-template <bool W_IS_NK>
+template <bool W_IS_NK, bool ACT_BF16>
 __global__ void __launch_bounds__(kThreadsN, 1)
 hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_constant__ CUtensorMap map_w, const GemmParams p, int mp,
                         const NarrowPlan plan)
@@ -1026,7 +1028,8 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
     fill_decode_table<32>(lut_all, warp, lane, kThreadsN / 32);
     if (threadIdx.x == 0) {
         for (int s = 0; s < S8; s++) { mbar_init(bar_u8_full(s), 1); mbar_init(bar_u8_empty(s), 2 * kGroupWarps); }  // both halves' groups
-        for (int s = 0; s < S; s++) { mbar_init(bar_bf_full(s), kGroupWarps); mbar_init(bar_bf_empty(s), 1); }
+        // operands ready: the group's warps, plus (ACT_BF16) the announcement of the activation tile's bytes
+        for (int s = 0; s < S; s++) { mbar_init(bar_bf_full(s), kGroupWarps + (ACT_BF16 ? 1 : 0)); mbar_init(bar_bf_empty(s), 1); }
         for (int b = 0; b < 2; b++) { mbar_init(bar_acc_full(b), issuers); mbar_init(bar_acc_empty(b), kEpiWarps); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -1043,24 +1046,44 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
 
     if (warp == kTmaWarp) {
         if (lane == 0) {
-            int issued = 0;
+            int issued = 0, issued_act = 0;
+            bool aborted = false;
             int j = (int)(pair0 / num_pb), pb = (int)(pair0 % num_pb);
             for (int it = 0; it < n_pairs; it++) {
                 const int s = it % S8, round = it / S8;
                 if (round > 0 && !mbar_wait(bar_u8_empty(s), (round - 1) & 1, abort_flag, p.status, 31)) break;
                 if (*abort_flag) break;
                 const uint32_t dst_w = base + SmemLayoutN::u8 + s * kU8Stage, dst_a = dst_w + kU8Act;
-                mbar_arrive_expect_tx(bar_u8_full(s), 2 * kNwW8 + act_bytes);
+                mbar_arrive_expect_tx(bar_u8_full(s), 2 * kNwW8 + (ACT_BF16 ? 0u : act_bytes));
                 if (W_IS_NK) tma_load_2d(dst_w, &map_w, pb * BK2, j * BM, bar_u8_full(s));
                 else tma_load_2d(dst_w, &map_w, j * BM, pb * BK2, bar_u8_full(s));
-                tma_load_2d(dst_a, &map_act, pb * BK2, 0, bar_u8_full(s));
+                if (!ACT_BF16) tma_load_2d(dst_a, &map_act, pb * BK2, 0, bar_u8_full(s));
                 issued = it + 1;
+                if (ACT_BF16) {
+                    // Activations expanded to BF16 beforehand (map_act is then the map of that copy): the tiles of the pair's
+                    // two k-blocks go straight into their operand stages, in the 128-byte-swizzled layout the MMA reads, once
+                    // the MMAs of each stage's previous use have read it.  (The byte copy above is needed eight k-blocks later;
+                    // these are needed by the end of their k-block's decode, and their waits end about when the next byte
+                    // stage falls free, so one thread keeps both streams going.)
+                    for (int h = 0; h < 2 && !aborted; h++) {
+                        const int ik = 2 * it + h, sb = ik % S, rb = ik / S;
+                        if (rb > 0 && !mbar_wait(bar_bf_empty(sb), (rb - 1) & 1, abort_flag, p.status, 37)) { aborted = true; break; }
+                        mbar_arrive_expect_tx(bar_bf_full(sb), (uint32_t)mp * BK * 2u);
+                        tma_load_2d(base + SmemLayoutN::bf + sb * kNwABf, &map_act, (2 * pb + h) * BK, 0, bar_bf_full(sb));
+                        issued_act = ik + 1;
+                    }
+                    if (aborted) break;
+                }
                 if (++pb == num_pb) { pb = 0; j++; }
             }
             if (*abort_flag) {  // let the copies already issued land before this CTA's shared memory goes away
                 for (int it = max(0, issued - S8); it < issued; it++) {
                     const unsigned long long t0 = global_ns();
                     while (!mbar_try_wait(bar_u8_full(it % S8), (it / S8) & 1) && global_ns() - t0 < kWaitLimitNs) {}
+                }
+                for (int ik = max(0, issued_act - S); ik < issued_act; ik++) {
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(bar_bf_full(ik % S), (ik / S) & 1) && global_ns() - t0 < kWaitLimitNs) {}
                 }
             }
         }
@@ -1122,10 +1145,12 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
 #pragma unroll
                 for (int jj = 0; jj < BK / 16; jj++) vr[jj] = lds_v4(w_row + (((uint32_t)(4 * h + jj) ^ sw) << 4));
             }
+            if (!ACT_BF16) {
 #pragma unroll
-            for (int i = 0; i < kNarrowMaxM * (BK / 8) / kGroupThreads; i++) {
-                const int q = i * kGroupThreads + dt;
-                if (q < act_chunks) va[i] = lds_v2(a8 + (q >> 3) * BK2 + (q & 7) * 8);
+                for (int i = 0; i < kNarrowMaxM * (BK / 8) / kGroupThreads; i++) {
+                    const int q = i * kGroupThreads + dt;
+                    if (q < act_chunks) va[i] = lds_v2(a8 + (q >> 3) * BK2 + (q & 7) * 8);
+                }
             }
             uint32_t o[BK / 2];  // 64 BF16 of this weight column, two per tensor-memory column
             if (W_IS_NK) {
@@ -1151,13 +1176,15 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
                 if (lane == 0) mbar_arrive(bar_u8_empty(s8));
             }
             tmem_st_32x32b_x32(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + kTmemAccN + (uint32_t)(s * (BK / 2)), o);
+            if (!ACT_BF16) {
 #pragma unroll
-            for (int i = 0; i < kNarrowMaxM * (BK / 8) / kGroupThreads; i++) {
-                const int q = i * kGroupThreads + dt, row = q >> 3, jc = q & 7;
-                if (q < act_chunks) sts_v4(abf + (row >> 3) * 1024 + (row & 7) * 128 + ((jc ^ (row & 7)) << 4), decode8<7>(va[i], lut));
+                for (int i = 0; i < kNarrowMaxM * (BK / 8) / kGroupThreads; i++) {
+                    const int q = i * kGroupThreads + dt, row = q >> 3, jc = q & 7;
+                    if (q < act_chunks) sts_v4(abf + (row >> 3) * 1024 + (row & 7) * 128 + ((jc ^ (row & 7)) << 4), decode8<7>(va[i], lut));
+                }
             }
             tmem_st_wait();  // the weight column is in tensor memory
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            if (!ACT_BF16) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_bf_full(s));
@@ -1599,10 +1626,10 @@ bool gemm_kernels_ready(int dev, int* sm_count_out)
             out->rc = cudaFuncSetAttribute(fused[i], cudaFuncAttributeMaxDynamicSharedMemorySize, i < 2 ? kSmemBytesWide : kSmemBytes);
         for (int i = 0; i < 2 && out->rc == cudaSuccess; i++)
             out->rc = cudaFuncSetAttribute(pair[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
-        if (out->rc == cudaSuccess)
-            out->rc = cudaFuncSetAttribute(hif8_gemm_narrow_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytesN);
-        if (out->rc == cudaSuccess)
-            out->rc = cudaFuncSetAttribute(hif8_gemm_narrow_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytesN);
+        const void* narrow[4] = {(const void*)hif8_gemm_narrow_kernel<false, false>, (const void*)hif8_gemm_narrow_kernel<false, true>,
+                                 (const void*)hif8_gemm_narrow_kernel<true, false>, (const void*)hif8_gemm_narrow_kernel<true, true>};
+        for (int i = 0; i < 4 && out->rc == cudaSuccess; i++)
+            out->rc = cudaFuncSetAttribute(narrow[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytesN);
         if (out->rc == cudaSuccess) out->rc = cudaDeviceGetAttribute(&out->sm_count, cudaDevAttrMultiProcessorCount, d);
     });
     if (!s) return false;
@@ -1764,9 +1791,29 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t
             }
         }
         if (grid > 0x7FFFFFFFll) return HIF8_ERR_SHAPE;
+        // With room left for the activations as BF16 (2 M K bytes behind the partial sums) they are expanded once, here,
+        // and their tiles are copied straight into the operand stages: otherwise every CTA decodes the activation tile of
+        // every k-block again for each of its slabs, a seventh (16 rows) to a third (64 rows) of the kernel's table lookups.
+        bool act_bf16 = false;
+        {
+            const size_t used = clear_bytes > 4 ? clear_bytes + (size_t)slabs * plan.pmax * mp * BM * 4 : kGemmWorkspaceBytes;
+            const size_t off = (used + 255) & ~(size_t)255, bytes_act = (size_t)M * K * 2;
+            if (lda == K && workspace_bytes >= off + bytes_act && !(reinterpret_cast<uintptr_t>(workspace) & 255)) {
+                unsigned char* a_bf = reinterpret_cast<unsigned char*>(workspace) + off;
+                const int rc = hif8_decode(Aq, a_bf, HIF8_BF16, (size_t)M * K, 0, stream);
+                if (rc != HIF8_OK) return rc;
+                if (!make_map(&map_act, a_bf, (uint64_t)K, (uint64_t)M, (uint64_t)K, BK, (uint32_t)mp, true)) return HIF8_ERR_CUDA;
+                act_bf16 = true;
+            }
+        }
         if (cudaMemsetAsync(workspace, 0, clear_bytes, st) != cudaSuccess) return HIF8_ERR_CUDA;
-        if (w_is_nk) hif8_gemm_narrow_kernel<true><<<(unsigned)grid, kThreadsN, kSmemBytesN, st>>>(map_act, map_ws, p, mp, plan);
-        else hif8_gemm_narrow_kernel<false><<<(unsigned)grid, kThreadsN, kSmemBytesN, st>>>(map_act, map_ws, p, mp, plan);
+        if (w_is_nk) {
+            if (act_bf16) hif8_gemm_narrow_kernel<true, true><<<(unsigned)grid, kThreadsN, kSmemBytesN, st>>>(map_act, map_ws, p, mp, plan);
+            else hif8_gemm_narrow_kernel<true, false><<<(unsigned)grid, kThreadsN, kSmemBytesN, st>>>(map_act, map_ws, p, mp, plan);
+        } else {
+            if (act_bf16) hif8_gemm_narrow_kernel<false, true><<<(unsigned)grid, kThreadsN, kSmemBytesN, st>>>(map_act, map_ws, p, mp, plan);
+            else hif8_gemm_narrow_kernel<false, false><<<(unsigned)grid, kThreadsN, kSmemBytesN, st>>>(map_act, map_ws, p, mp, plan);
+        }
         g_launches.fetch_add(1, std::memory_order_relaxed);
         return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
     }
