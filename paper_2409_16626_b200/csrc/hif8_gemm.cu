@@ -966,6 +966,35 @@ struct SmemLayoutN {
     static constexpr uint32_t total = abort_flag + 4;
 };
 constexpr uint32_t kSmemBytesN = SmemLayoutN::total + 1024;
+// Where the narrow kernel keeps what.  WIDE = false: the fixed layout above.  WIDE = true ([N,K] weights with the activations
+// expanded beforehand: the byte stages hold weights only, 16 KiB each): the decode table has rows of 256 bytes and starts on a 64 KiB boundary
+// of the shared window, so that one byte permute makes a lookup's address (see decode8); as many operand stages (8 KiB) as
+// fit lie in front of it, the other operand stages, the byte stages and the barriers behind it.
+template <bool WIDE>
+struct NarrowSmem {
+    uint32_t base, lut, bars, end;  // shared-window addresses; base is 1024-byte aligned
+    uint32_t behind, u8_0;
+    int n_front;
+    __device__ explicit NarrowSmem(uint32_t raw)
+    {
+        base = (raw + 1023u) & ~1023u;
+        if (!WIDE) {
+            lut = base + SmemLayoutN::lut; bars = base + SmemLayoutN::bars; end = base + SmemLayoutN::total;
+            behind = 0; u8_0 = base + SmemLayoutN::u8; n_front = kNwTmemStages;
+        } else {
+            lut = (base + kLutBytesWide - 1) & ~(kLutBytesWide - 1);
+            n_front = (int)min((lut - base) / kNwABf, (uint32_t)kNwTmemStages);
+            behind = lut + kLutBytesWide;
+            u8_0 = behind + (uint32_t)(kNwTmemStages - n_front) * kNwABf;
+            bars = u8_0 + kNwByteStages * 2 * kNwW8;
+            end = bars + SmemLayoutN::n_bars * 8 + 8;
+        }
+    }
+    __device__ uint32_t bf(int s) const { return s < n_front ? base + (uint32_t)s * kNwABf : behind + (uint32_t)(s - n_front) * kNwABf; }
+    __device__ uint32_t u8(int s) const { return u8_0 + (uint32_t)s * (WIDE ? 2 * kNwW8 : 2 * (kNwW8 + kNwA8)); }
+    __device__ uint32_t tmem_slot() const { return bars + SmemLayoutN::n_bars * 8; }
+    __device__ uint32_t abort_flag() const { return tmem_slot() + 4; }
+};
 // Tensor memory: the accumulators (two per issuer: the epilogue of one segment overlaps the next segment's MMAs), then
 // one weight stage (128 rows x 64 BF16 = 32 columns) per operand stage.
 // MMA issuers.  One thread that waits for a stage, issues its four MMAs and commits spends about a thousand cycles per
@@ -998,24 +1027,36 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
                         const NarrowPlan plan)
 {
     extern __shared__ unsigned char smem_raw[];
-    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    unsigned char* sm = smem_raw + (base - smem_u32(smem_raw));
+    // the 64 KiB table pays for [N,K] weights, whose bytes are extracted from registers (76 against 85 us at 16 x 28672 x 8192);
+    // [K,N] weights arrive a byte per load and ran slower with it (84 against 81 us)
+    constexpr bool kWideN = ACT_BF16 && W_IS_NK;
+    constexpr int kLutShiftN = kWideN ? 8 : 7;
+    const NarrowSmem<kWideN> lay(smem_u32(smem_raw));
+    unsigned char* sm = smem_raw - smem_u32(smem_raw);  // generic pointer of shared-window address 0
+    {
+        uint32_t dyn_bytes;
+        asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn_bytes));
+        if (lay.end > smem_u32(smem_raw) + dyn_bytes) {  // the layout does not fit (the same answer in every thread)
+            if (threadIdx.x == 0) atomicCAS(p.status, 0, 7);
+            return;
+        }
+    }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr int S = kNwTmemStages;  // operand ring: the it-th k-block uses stage it % S
     static_assert(S % kDecodeGroups == 0, "an operand stage is always written by the same group");
     constexpr int S8 = kNwByteStages;   // byte ring: the i-th pair block of this CTA lands in stage i % S8
-    constexpr uint32_t kU8Stage = 2 * (kNwW8 + kNwA8), kU8Act = 2 * kNwW8;  // byte stage: 128 weight columns x 128 k, then act rows x 128 k
-    const uint32_t bars = base + SmemLayoutN::bars;
+    constexpr uint32_t kU8Act = 2 * kNwW8;  // byte stage: 128 weight columns x 128 k, then (activations as bytes) act rows x 128 k
+    const uint32_t bars = lay.bars;
     auto bar_u8_full = [&](int s) { return bars + 8u * s; };
     auto bar_u8_empty = [&](int s) { return bars + 8u * (S8 + s); };
     auto bar_bf_full = [&](int s) { return bars + 8u * (2 * S8 + s); };
     auto bar_bf_empty = [&](int s) { return bars + 8u * (2 * S8 + S + s); };
     auto bar_acc_full = [&](int b) { return bars + 8u * (2 * S8 + 2 * S + b); };
     auto bar_acc_empty = [&](int b) { return bars + 8u * (2 * S8 + 2 * S + 2 + b); };
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + SmemLayoutN::abort_flag);
-    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + SmemLayoutN::tmem_slot);
-    uint32_t* lut_all = reinterpret_cast<uint32_t*>(sm + SmemLayoutN::lut);
-    const uint32_t lut = base + SmemLayoutN::lut + 4u * lane;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + lay.abort_flag());
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + lay.tmem_slot());
+    uint32_t* lut_all = reinterpret_cast<uint32_t*>(sm + lay.lut);
+    const uint32_t lut = lay.lut + 4u * lane;
     const int num_pb = (p.K + BK2 - 1) / BK2, num_kb = 2 * num_pb;  // per slab
     const long long G = gridDim.x;
     const long long pair0 = plan.total * blockIdx.x / G, pair1 = plan.total * (blockIdx.x + 1) / G;  // this CTA's (slab, pair block) range
@@ -1025,7 +1066,7 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
     const int issuers = mp <= 32 ? kNwMaxIssuers : 2;
     auto acc_col = [&](int q, int buf) { return (uint32_t)((q * 2 + buf) * mp); };  // accumulator of issuer q, buffer buf
 
-    fill_decode_table<32>(lut_all, warp, lane, kThreadsN / 32);
+    fill_decode_table<(1 << (kLutShiftN - 2))>(lut_all, warp, lane, kThreadsN / 32);  // rows of 1 << kLutShiftN bytes
     if (threadIdx.x == 0) {
         for (int s = 0; s < S8; s++) { mbar_init(bar_u8_full(s), 1); mbar_init(bar_u8_empty(s), 2 * kGroupWarps); }  // both halves' groups
         // operands ready: the group's warps, plus (ACT_BF16) the announcement of the activation tile's bytes
@@ -1036,7 +1077,7 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
     }
     if (warp == kMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(base + SmemLayoutN::tmem_slot), "r"(kTmemColsN) : "memory");
+                     ::"r"(lay.tmem_slot()), "r"(kTmemColsN) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -1053,7 +1094,7 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
                 const int s = it % S8, round = it / S8;
                 if (round > 0 && !mbar_wait(bar_u8_empty(s), (round - 1) & 1, abort_flag, p.status, 31)) break;
                 if (*abort_flag) break;
-                const uint32_t dst_w = base + SmemLayoutN::u8 + s * kU8Stage, dst_a = dst_w + kU8Act;
+                const uint32_t dst_w = lay.u8(s), dst_a = dst_w + kU8Act;
                 mbar_arrive_expect_tx(bar_u8_full(s), 2 * kNwW8 + (ACT_BF16 ? 0u : act_bytes));
                 if (W_IS_NK) tma_load_2d(dst_w, &map_w, pb * BK2, j * BM, bar_u8_full(s));
                 else tma_load_2d(dst_w, &map_w, j * BM, pb * BK2, bar_u8_full(s));
@@ -1069,7 +1110,7 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
                         const int ik = 2 * it + h, sb = ik % S, rb = ik / S;
                         if (rb > 0 && !mbar_wait(bar_bf_empty(sb), (rb - 1) & 1, abort_flag, p.status, 37)) { aborted = true; break; }
                         mbar_arrive_expect_tx(bar_bf_full(sb), (uint32_t)mp * BK * 2u);
-                        tma_load_2d(base + SmemLayoutN::bf + sb * kNwABf, &map_act, (2 * pb + h) * BK, 0, bar_bf_full(sb));
+                        tma_load_2d(lay.bf(sb), &map_act, (2 * pb + h) * BK, 0, bar_bf_full(sb));
                         issued_act = ik + 1;
                     }
                     if (aborted) break;
@@ -1094,7 +1135,7 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
             // (K-major), N = mp, M = 128
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(mp >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
             // descriptor of stage 0; a stage or a 16-k step further on adds to the address field only
-            const uint64_t da0 = make_smem_desc(base + SmemLayoutN::bf, 16, 1024);
+            const uint64_t da0 = make_smem_desc(lay.bf(0), 16, 1024);
             bool ok = true, first = true;
             int kb = (int)(lin0 % num_kb), seg = 0;
             for (int it = 0; it < n_it && ok; it++) {
@@ -1111,7 +1152,7 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
                     for (int kk = 0; kk < BK / 16; kk++) {
                         // weights from tensor memory: operand stage s, 16 k = 8 columns
                         tc_mma_bf16_cta_a_tmem(d_tmem, tmem_base + kTmemAccN + (uint32_t)(s * (BK / 2) + kk * 8),
-                                               da0 + (uint64_t)((s * kNwABf + kk * 32) >> 4), idesc, (!first || kk > 0) ? 1u : 0u);
+                                               da0 + (uint64_t)((lay.bf(s) - lay.bf(0) + kk * 32) >> 4), idesc, (!first || kk > 0) ? 1u : 0u);
                     }
                     tc_commit_cta(bar_bf_empty(s));
                     first = false;
@@ -1132,8 +1173,8 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
             ok = mbar_wait(bar_u8_full(s8), ((it >> 1) / S8) & 1, abort_flag, p.status, 33);
             if (ok && r > 0) ok = mbar_wait(bar_bf_empty(s), (r - 1) & 1, abort_flag, p.status, 34);
             if (!ok) break;
-            const uint32_t w8 = base + SmemLayoutN::u8 + s8 * kU8Stage, a8 = w8 + kU8Act + (uint32_t)h * BK;
-            const uint32_t abf = base + SmemLayoutN::bf + s * kNwABf;
+            const uint32_t w8 = lay.u8(s8), a8 = w8 + kU8Act + (uint32_t)h * BK;
+            const uint32_t abf = lay.bf(s);
             uint2 va[kNarrowMaxM * (BK / 8) / kGroupThreads];
             uint4 vr[BK / 16];
             // this thread owns weight column (operand row, tensor-memory lane) quarter * 32 + lane of the slab
@@ -1158,7 +1199,7 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
                 if (lane == 0) mbar_arrive(bar_u8_empty(s8));
 #pragma unroll
                 for (int jj = 0; jj < BK / 16; jj++) {
-                    const uint4 lo = decode8<7>(make_uint2(vr[jj].x, vr[jj].y), lut), hi = decode8<7>(make_uint2(vr[jj].z, vr[jj].w), lut);
+                    const uint4 lo = decode8<kLutShiftN>(make_uint2(vr[jj].x, vr[jj].y), lut), hi = decode8<kLutShiftN>(make_uint2(vr[jj].z, vr[jj].w), lut);
                     o[8 * jj + 0] = lo.x; o[8 * jj + 1] = lo.y; o[8 * jj + 2] = lo.z; o[8 * jj + 3] = lo.w;
                     o[8 * jj + 4] = hi.x; o[8 * jj + 5] = hi.y; o[8 * jj + 6] = hi.z; o[8 * jj + 7] = hi.w;
                 }
@@ -1170,7 +1211,9 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
 #pragma unroll
                 for (int j = 0; j < BK / 2; j++) {
                     const uint32_t c0 = lds_u8(w_col + (uint32_t)(2 * j) * BM), c1 = lds_u8(w_col + (uint32_t)(2 * j + 1) * BM);
-                    o[j] = __byte_perm(lds_u32(lut + (c0 << 7)), lds_u32(lut + (c1 << 7)), 0x5410);
+                    // (rows of 256 bytes: the byte replaces byte 1 of the lane's table address, one permute)
+                    if (kLutShiftN == 8) o[j] = __byte_perm(lds_u32(__byte_perm(c0, lut, 0x7604)), lds_u32(__byte_perm(c1, lut, 0x7604)), 0x5410);
+                    else o[j] = __byte_perm(lds_u32(lut + (c0 << 7)), lds_u32(lut + (c1 << 7)), 0x5410);
                 }
                 __syncwarp();  // the byte stage has been read
                 if (lane == 0) mbar_arrive(bar_u8_empty(s8));
@@ -1629,7 +1672,7 @@ bool gemm_kernels_ready(int dev, int* sm_count_out)
         const void* narrow[4] = {(const void*)hif8_gemm_narrow_kernel<false, false>, (const void*)hif8_gemm_narrow_kernel<false, true>,
                                  (const void*)hif8_gemm_narrow_kernel<true, false>, (const void*)hif8_gemm_narrow_kernel<true, true>};
         for (int i = 0; i < 4 && out->rc == cudaSuccess; i++)
-            out->rc = cudaFuncSetAttribute(narrow[i], cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytesN);
+            out->rc = cudaFuncSetAttribute(narrow[i], cudaFuncAttributeMaxDynamicSharedMemorySize, i == 3 ? kSmemBytesWide : kSmemBytesN);  // (the last one: wide table)
         if (out->rc == cudaSuccess) out->rc = cudaDeviceGetAttribute(&out->sm_count, cudaDevAttrMultiProcessorCount, d);
     });
     if (!s) return false;
@@ -1808,7 +1851,7 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t
         }
         if (cudaMemsetAsync(workspace, 0, clear_bytes, st) != cudaSuccess) return HIF8_ERR_CUDA;
         if (w_is_nk) {
-            if (act_bf16) hif8_gemm_narrow_kernel<true, true><<<(unsigned)grid, kThreadsN, kSmemBytesN, st>>>(map_act, map_ws, p, mp, plan);
+            if (act_bf16) hif8_gemm_narrow_kernel<true, true><<<(unsigned)grid, kThreadsN, kSmemBytesWide, st>>>(map_act, map_ws, p, mp, plan);
             else hif8_gemm_narrow_kernel<true, false><<<(unsigned)grid, kThreadsN, kSmemBytesN, st>>>(map_act, map_ws, p, mp, plan);
         } else {
             if (act_bf16) hif8_gemm_narrow_kernel<false, true><<<(unsigned)grid, kThreadsN, kSmemBytesN, st>>>(map_act, map_ws, p, mp, plan);
