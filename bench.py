@@ -461,7 +461,9 @@ def extra_results(H, torch, hbm_peak, tf_peak, peak_kind, tf_sustained=None):
     out["gemm_midM_x28672x8192"] = {"bound": "tensor", "shapes": mid, "peak": tf_peak, "peak_kind": f"of {peak_kind} (cuBLAS BF16 burst)",
                                     "note": "the weight bytes alone take 36 us at the copy rate; 256 rows run as one tile row of 256"}
     out["gemm_narrow_Mx28672x8192"] = {"bound": "hbm", "bytes": "K*N weight bytes + M*K + 2*M*N", "shapes": narrow,
-                                       "peak": hbm_peak, "peak_kind": f"of {peak_kind}"}
+                                       "peak": hbm_peak, "peak_kind": f"of {peak_kind}",
+                                       "note": "whole call; with the workspace it first expands the activations to BF16 (one more launch, "
+                                               "2*M*K bytes) and splits the weight evenly over the SMs"}
     out["gemm_8192x28672x8192"] = {
         "backward_forms": bw, "decode_once_channel_scaled": g_chan, "decode_once": g_once, "fused": g_fused, "a_expanded_w_fused": g_aexp, "a_expanded_w_nk_fused": g_aexp_nk,
         "bound": "tensor", "peak": tf_peak, "peak_kind": f"of {peak_kind} (cuBLAS BF16 burst)", "unit": "TFLOP/s",

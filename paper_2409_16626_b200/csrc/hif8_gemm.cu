@@ -1106,6 +1106,9 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
                     // the MMAs of each stage's previous use have read it.  (The byte copy above is needed eight k-blocks later;
                     // these are needed by the end of their k-block's decode, and their waits end about when the next byte
                     // stage falls free, so one thread keeps both streams going.)
+                    // (the expansion runs right in front of this kernel, which is launched so that its set-up and its first
+                    // weight copy overlap it: the expanded activations are complete once this wait returns)
+                    if (it == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
                     for (int h = 0; h < 2 && !aborted; h++) {
                         const int ik = 2 * it + h, sb = ik % S, rb = ik / S;
                         if (rb > 0 && !mbar_wait(bar_bf_empty(sb), (rb - 1) & 1, abort_flag, p.status, 37)) { aborted = true; break; }
@@ -1838,6 +1841,7 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t
         // and their tiles are copied straight into the operand stages: otherwise every CTA decodes the activation tile of
         // every k-block again for each of its slabs, a seventh (16 rows) to a third (64 rows) of the kernel's table lookups.
         bool act_bf16 = false;
+        if (cudaMemsetAsync(workspace, 0, clear_bytes, st) != cudaSuccess) return HIF8_ERR_CUDA;
         {
             const size_t used = clear_bytes > 4 ? clear_bytes + (size_t)slabs * plan.pmax * mp * BM * 4 : kGemmWorkspaceBytes;
             const size_t off = (used + 255) & ~(size_t)255, bytes_act = (size_t)M * K * 2;
@@ -1849,14 +1853,23 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t
                 act_bf16 = true;
             }
         }
-        if (cudaMemsetAsync(workspace, 0, clear_bytes, st) != cudaSuccess) return HIF8_ERR_CUDA;
-        if (w_is_nk) {
-            if (act_bf16) hif8_gemm_narrow_kernel<true, true><<<(unsigned)grid, kThreadsN, kSmemBytesWide, st>>>(map_act, map_ws, p, mp, plan);
-            else hif8_gemm_narrow_kernel<true, false><<<(unsigned)grid, kThreadsN, kSmemBytesN, st>>>(map_act, map_ws, p, mp, plan);
-        } else {
-            if (act_bf16) hif8_gemm_narrow_kernel<false, true><<<(unsigned)grid, kThreadsN, kSmemBytesN, st>>>(map_act, map_ws, p, mp, plan);
-            else hif8_gemm_narrow_kernel<false, false><<<(unsigned)grid, kThreadsN, kSmemBytesN, st>>>(map_act, map_ws, p, mp, plan);
-        }
+        cudaLaunchConfig_t cn{};
+        cn.gridDim = dim3((unsigned)grid);
+        cn.blockDim = dim3(kThreadsN);
+        cn.dynamicSmemBytes = (act_bf16 && w_is_nk) ? kSmemBytesWide : kSmemBytesN;
+        cn.stream = st;
+        // with the expansion kernel right in front: programmatic stream serialization (that kernel lets its dependents start
+        // at once; this one waits for its completion before the first read of the expanded activations)
+        cudaLaunchAttribute an[1];
+        an[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        an[0].val.programmaticStreamSerializationAllowed = 1;
+        cn.attrs = an; cn.numAttrs = act_bf16 ? 1 : 0;
+        cudaError_t nrc;
+        if (w_is_nk) nrc = act_bf16 ? cudaLaunchKernelEx(&cn, hif8_gemm_narrow_kernel<true, true>, map_act, map_ws, p, mp, plan)
+                                    : cudaLaunchKernelEx(&cn, hif8_gemm_narrow_kernel<true, false>, map_act, map_ws, p, mp, plan);
+        else nrc = act_bf16 ? cudaLaunchKernelEx(&cn, hif8_gemm_narrow_kernel<false, true>, map_act, map_ws, p, mp, plan)
+                            : cudaLaunchKernelEx(&cn, hif8_gemm_narrow_kernel<false, false>, map_act, map_ws, p, mp, plan);
+        if (nrc != cudaSuccess) return HIF8_ERR_CUDA;
         g_launches.fetch_add(1, std::memory_order_relaxed);
         return cudaGetLastError() == cudaSuccess ? HIF8_OK : HIF8_ERR_CUDA;
     }
