@@ -1021,6 +1021,32 @@ struct NarrowPlan {
     int pmax;            // slices per slab
 };
 
+// In front of the narrow kernel when the workspace has room: the activations [M,K] (contiguous bytes) expanded to BF16, and
+// the status word and the tickets cleared, in one launch.  Its dependents may start at once (the narrow kernel builds its
+// table meanwhile and waits for this grid's completion before it reads any of this).
+__global__ void __launch_bounds__(256) narrow_prepare_kernel(const uint4* __restrict__ a, uint4* __restrict__ a_bf, unsigned long long n_vec,
+                                                             uint32_t* __restrict__ clear, unsigned clear_words)
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    __shared__ uint32_t lut[256];
+    lut[threadIdx.x] = hif8_to_bf16_bits(threadIdx.x);
+    __syncthreads();
+    if (blockIdx.x == 0)
+        for (unsigned i = threadIdx.x; i < clear_words; i += 256) clear[i] = 0u;
+    for (unsigned long long u = (unsigned long long)blockIdx.x * 256 + threadIdx.x; u < n_vec; u += (unsigned long long)gridDim.x * 256) {
+        const uint4 v = a[u];
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        uint32_t o[8];
+#pragma unroll
+        for (int i = 0; i < 4; i++) {
+            o[2 * i] = lut[w[i] & 0xFFu] | (lut[(w[i] >> 8) & 0xFFu] << 16);
+            o[2 * i + 1] = lut[(w[i] >> 16) & 0xFFu] | (lut[w[i] >> 24] << 16);
+        }
+        a_bf[2 * u] = make_uint4(o[0], o[1], o[2], o[3]);
+        a_bf[2 * u + 1] = make_uint4(o[4], o[5], o[6], o[7]);
+    }
+}
+
 template <bool W_IS_NK, bool ACT_BF16>
 __global__ void __launch_bounds__(kThreadsN, 1)
 hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __grid_constant__ CUtensorMap map_w, const GemmParams p, int mp,
@@ -1037,6 +1063,7 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
         uint32_t dyn_bytes;
         asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn_bytes));
         if (lay.end > smem_u32(smem_raw) + dyn_bytes) {  // the layout does not fit (the same answer in every thread)
+            if (ACT_BF16) asm volatile("griddepcontrol.wait;" ::: "memory");  // (the launch in front clears the status word)
             if (threadIdx.x == 0) atomicCAS(p.status, 0, 7);
             return;
         }
@@ -1084,6 +1111,9 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // The launch in front of this kernel expands the activations and clears the status word and the tickets; this kernel was
+    // started while that one ran, so that the set-up above overlaps it.  From here on its results are complete.
+    if (ACT_BF16) asm volatile("griddepcontrol.wait;" ::: "memory");
 
     if (warp == kTmaWarp) {
         if (lane == 0) {
@@ -1106,9 +1136,6 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
                     // the MMAs of each stage's previous use have read it.  (The byte copy above is needed eight k-blocks later;
                     // these are needed by the end of their k-block's decode, and their waits end about when the next byte
                     // stage falls free, so one thread keeps both streams going.)
-                    // (the expansion runs right in front of this kernel, which is launched so that its set-up and its first
-                    // weight copy overlap it: the expanded activations are complete once this wait returns)
-                    if (it == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
                     for (int h = 0; h < 2 && !aborted; h++) {
                         const int ik = 2 * it + h, sb = ik % S, rb = ik / S;
                         if (rb > 0 && !mbar_wait(bar_bf_empty(sb), (rb - 1) & 1, abort_flag, p.status, 37)) { aborted = true; break; }
@@ -1841,25 +1868,30 @@ static int gemm_entry(const uint8_t* Aq, int64_t lda, int a_is_km, const uint8_t
         // and their tiles are copied straight into the operand stages: otherwise every CTA decodes the activation tile of
         // every k-block again for each of its slabs, a seventh (16 rows) to a third (64 rows) of the kernel's table lookups.
         bool act_bf16 = false;
-        if (cudaMemsetAsync(workspace, 0, clear_bytes, st) != cudaSuccess) return HIF8_ERR_CUDA;
         {
             const size_t used = clear_bytes > 4 ? clear_bytes + (size_t)slabs * plan.pmax * mp * BM * 4 : kGemmWorkspaceBytes;
             const size_t off = (used + 255) & ~(size_t)255, bytes_act = (size_t)M * K * 2;
             if (lda == K && workspace_bytes >= off + bytes_act && !(reinterpret_cast<uintptr_t>(workspace) & 255)) {
                 unsigned char* a_bf = reinterpret_cast<unsigned char*>(workspace) + off;
-                const int rc = hif8_decode(Aq, a_bf, HIF8_BF16, (size_t)M * K, 0, stream);
-                if (rc != HIF8_OK) return rc;
                 if (!make_map(&map_act, a_bf, (uint64_t)K, (uint64_t)M, (uint64_t)K, BK, (uint32_t)mp, true)) return HIF8_ERR_CUDA;
+                const unsigned long long n_vec = (unsigned long long)M * K / 16;  // K is a multiple of 16
+                const unsigned long long want = (n_vec + 255) / 256, cap = (unsigned long long)sm_count * 4;
+                narrow_prepare_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(
+                    reinterpret_cast<const uint4*>(Aq), reinterpret_cast<uint4*>(a_bf), n_vec, reinterpret_cast<uint32_t*>(workspace),
+                    (unsigned)(clear_bytes / 4));
+                if (cudaGetLastError() != cudaSuccess) return HIF8_ERR_CUDA;
+                g_launches.fetch_add(1, std::memory_order_relaxed);
                 act_bf16 = true;
             }
         }
+        if (!act_bf16 && cudaMemsetAsync(workspace, 0, clear_bytes, st) != cudaSuccess) return HIF8_ERR_CUDA;
         cudaLaunchConfig_t cn{};
         cn.gridDim = dim3((unsigned)grid);
         cn.blockDim = dim3(kThreadsN);
         cn.dynamicSmemBytes = (act_bf16 && w_is_nk) ? kSmemBytesWide : kSmemBytesN;
         cn.stream = st;
-        // with the expansion kernel right in front: programmatic stream serialization (that kernel lets its dependents start
-        // at once; this one waits for its completion before the first read of the expanded activations)
+        // with the preparing kernel right in front: programmatic stream serialization (that kernel lets its dependents start
+        // at once; this one waits for its completion once its own set-up is done)
         cudaLaunchAttribute an[1];
         an[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         an[0].val.programmaticStreamSerializationAllowed = 1;
