@@ -269,7 +269,8 @@ int hif8_fake_quant(const void* src, void* dst, int dtype, size_t n, int use_ama
  * the product is too small to win the pass over W back (see hif8_gemm_path_policy).
  * Products with at most 64 rows of A (and A given as [M,K]) take a weight-streaming kernel whatever the workspace;
  * with the workspace size above it spreads the weight bytes evenly over all SMs (partial sums of a column slab that
- * two SMs share go through the workspace and are added in a fixed order: results are reproducible run to run).
+ * two SMs share go through the workspace and are added in a fixed order: results are reproducible run to run) and,
+ * with A contiguous, first expands the few rows of A to BF16 there (one small launch more, same results).
  */
 int hif8_gemm(const uint8_t* Aq, int64_t lda, const uint8_t* Wq, int64_t ldw, int w_is_nk, void* C,
               int64_t ldc, int c_dtype, int M, int N, int K, const int* d_scale_exp_a,
