@@ -214,6 +214,28 @@ def test_gemm_narrow_products(shape, c_dtype, w_is_nk, staged):
         assert np.array_equal(out, again)
 
 
+@pytest.mark.parametrize("w_is_nk", [0, 1])
+@pytest.mark.parametrize("form", ["padded_lda", "room_for_a_only"])
+def test_gemm_narrow_activation_forms(form, w_is_nk):
+    # With a workspace the narrow kernel takes its activations expanded to BF16 by a launch in front of it -- unless A has a
+    # padded leading dimension (then the kernel decodes the activation bytes itself, with the slabs still cut between CTAs).
+    # A workspace with room for A alone has no room for partial sums: expanded activations with one CTA per slab.
+    M, N, K = 24, 1168, 2432
+    Aq = W.random_codes((M, K), seed=5)
+    Wkn = W.random_codes((K, N), seed=6)
+    for t in (Aq, Wkn):
+        t[(t == 0x80) | ((t & 0x7F) == 0x6F)] = 0x33
+    Cs, S = O.gemm_full(Aq, Wkn, False, 1, 2)
+    Wq = np.ascontiguousarray(Wkn.T) if w_is_nk else Wkn
+    if form == "padded_lda":
+        Ap = np.full((M, K + 32), 0x7B, dtype=np.uint8)
+        Ap[:, :K] = Aq
+        out = run_gemm(Ap, Wq, w_is_nk, H.F32, sa=1, sw=2, M=M, N=N, K=K, lda=K + 32, staged=True)
+    else:
+        out = run_gemm(Aq, Wq, w_is_nk, H.F32, sa=1, sw=2, M=M, N=N, K=K, staged="a")
+    check(out, Cs, S, H.F32)
+
+
 @pytest.mark.parametrize("K", [272, 2112])
 def test_gemm_narrow_channel_scales_and_accumulate(K):
     # K = 2112 with the large workspace: slabs cut between CTAs, finished by whichever contributor arrives last
