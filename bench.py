@@ -40,8 +40,8 @@ WORKLOAD = "fp32_4096x4096_normal_amax_scale_encode_then_decode"
 # workload.  "cold": every launch alone with the caches flushed in front of it.  "in_step": the same launches inside the
 # running amax -> convert -> decode sequence with the caches left as the previous kernel left them.  None: the kernel
 # has changed since its capture.
-TRAFFIC_COLD = {"amax_kernel<f32>": 67.43e6, "convert_kernel<f32,TA>": 69.83e6, "decode_kernel<f32>": 26.10e6}
-TRAFFIC_IN_STEP = {"amax_kernel<f32>": 88.4e6, "convert_kernel<f32,TA>": 19.0e6, "decode_kernel<f32>": 53.2e6}
+TRAFFIC_COLD = {"amax_kernel<f32>": 67.14e6, "convert_kernel<f32,TA>": 67.38e6, "decode_kernel<f32>": 22.59e6}
+TRAFFIC_IN_STEP = {"amax_kernel<f32>": 88.7e6, "convert_kernel<f32,TA>": 18.4e6, "decode_kernel<f32>": 52.5e6}
 METRIC = "hif8_encode_decode_throughput"
 UNIT = "GB/s"
 MIN_REPEATS = 7
