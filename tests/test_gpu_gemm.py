@@ -258,6 +258,45 @@ def test_gemm_narrow_channel_scales_and_accumulate(K):
     assert np.all(np.abs(C.cpu().numpy().astype(np.float64) - want) <= 1e-5 * S.reshape(M, N) + 2.0 ** -24 * np.abs(want))
 
 
+def test_gemm_calls_replay_from_a_cuda_graph():
+    # the narrow call is two launches chained by programmatic stream serialization, the general one a memset node and a
+    # cluster launch: both are captured into one graph and replayed on new operand contents
+    M, N, K = 16, 1168, 2432
+    M2 = 256
+    dA, dW = torch.empty(M2 * K, dtype=torch.uint8, device="cuda"), torch.empty(K * N, dtype=torch.uint8, device="cuda")
+    Cn = torch.zeros(M, N, dtype=torch.float32, device="cuda")
+    Cg = torch.zeros(M2, N, dtype=torch.float32, device="cuda")
+    wsb = H.hif8_workspace_bytes(H.WS_GEMM, M2 * K + K * N)
+    ws_n, ws_g = torch.empty(wsb, dtype=torch.uint8, device="cuda"), torch.empty(wsb, dtype=torch.uint8, device="cuda")
+
+    def calls():
+        H.hif8_gemm(dA, K, dW, N, 0, Cn, N, H.F32, M, N, K, None, None, ws_n, wsb)
+        H.hif8_gemm(dA, K, dW, N, 0, Cg, N, H.F32, M2, N, K, None, None, ws_g, 256)
+
+    def load(seed):
+        Aq, Wq = W.random_codes((M2, K), seed=seed), W.random_codes((K, N), seed=seed + 1)
+        for t in (Aq, Wq):
+            t[(t == 0x80) | ((t & 0x7F) == 0x6F)] = 0x33
+        dA.copy_(torch.from_numpy(Aq.reshape(-1)))
+        dW.copy_(torch.from_numpy(Wq.reshape(-1)))
+        return Aq, Wq
+
+    load(1)
+    calls()                                                   # eager first: one-time set-up happens outside the capture
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        calls()
+    for seed in (7, 9):
+        Aq, Wq = load(seed)
+        g.replay()
+        torch.cuda.synchronize()
+        assert H.hif8_gemm_status(ws_n) == 0 and H.hif8_gemm_status(ws_g) == 0
+        Cs, S = O.gemm_full(Aq, Wq, False, 0, 0)
+        check(Cg.cpu().numpy().astype(np.float64), Cs, S, H.F32)
+        check(Cn.cpu().numpy().astype(np.float64), Cs[:M], S[:M], H.F32)
+
+
 def test_tensor_map_cache_survives_eviction_and_pointer_reuse():
     # more distinct (pointer, shape) pairs than the library's tensor-map cache holds, each product exact in small integers;
     # then the same device buffers again with other shapes and contents (a cached map must never serve a different tensor)
