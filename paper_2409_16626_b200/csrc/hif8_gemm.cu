@@ -999,8 +999,9 @@ struct NarrowSmem {
 // one weight stage (128 rows x 64 BF16 = 32 columns) per operand stage.
 // MMA issuers.  One thread that waits for a stage, issues its four MMAs and commits spends about a thousand cycles per
 // k-block, more than the decode groups or the copies need; so up to four threads (one per warp) share the k-blocks,
-// issuer q taking the k-blocks it = q (mod issuers) into accumulators of its own, which the epilogue adds.  Four issuers
-// for up to 32 activation rows, two above: 2 buffers x issuers x rows stays within 256 columns.
+// issuer q taking the k-blocks it = q (mod issuers) into accumulators of its own, which the epilogue adds.  Up to 32
+// activation rows every issuer has two accumulators; above that either four issuers with one accumulator each or two with
+// two (the kernel says which): issuers x buffers x rows stays within 256 columns.
 constexpr int kNwMaxIssuers = 4;
 constexpr int kThreadsN = kThreads + (kNwMaxIssuers - 1) * 32;  // 800: the first issuer is the MMA warp of the other kernels
 constexpr uint32_t kTmemAccN = 2 * 2 * kNarrowMaxM, kTmemColsN = 512;
@@ -1090,8 +1091,12 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
     const long long lin0 = 2 * pair0, lin1 = 2 * pair1;  // the same in k-blocks
     const int n_pairs = (int)(pair1 - pair0), n_it = 2 * n_pairs;
     const uint32_t act_bytes = (uint32_t)mp * BK2;
-    const int issuers = mp <= 32 ? kNwMaxIssuers : 2;
-    auto acc_col = [&](int q, int buf) { return (uint32_t)((q * 2 + buf) * mp); };  // accumulator of issuer q, buffer buf
+    // Up to 32 activation rows: four issuers with two accumulators each (the epilogue of one segment overlaps the next
+    // segment's MMAs).  Above that issuers x buffers x rows must stay within 256 columns: four issuers with one accumulator
+    // for [N,K] weights (91 against 94 us at 64 x 28672 x 8192), two with two for [K,N] weights (92 against 95 us).
+    const int issuers = (mp <= 32 || W_IS_NK) ? kNwMaxIssuers : 2;
+    const int bufs = (mp <= 32 || issuers == 2) ? 2 : 1;
+    auto acc_col = [&](int q, int buf) { return (uint32_t)((q * bufs + buf) * mp); };  // accumulator of issuer q, buffer buf
 
     fill_decode_table<(1 << (kLutShiftN - 2))>(lut_all, warp, lane, kThreadsN / 32);  // rows of 1 << kLutShiftN bytes
     if (threadIdx.x == 0) {
@@ -1169,11 +1174,11 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
             bool ok = true, first = true;
             int kb = (int)(lin0 % num_kb), seg = 0;
             for (int it = 0; it < n_it && ok; it++) {
-                const int buf = seg & 1;
+                const int buf = bufs == 2 ? seg & 1 : 0, use = bufs == 2 ? seg >> 1 : seg;  // use: how often the buffer was filled before
                 if ((it & (issuers - 1)) == q) {
                     const int s = it % S, round = it / S;
                     // a segment's first MMA overwrites the accumulator: the epilogue must have read its previous contents
-                    if (first && seg >= 2) ok = mbar_wait(bar_acc_empty(buf), ((seg >> 1) - 1) & 1, abort_flag, p.status, 36);
+                    if (first && use >= 1) ok = mbar_wait(bar_acc_empty(buf), (use - 1) & 1, abort_flag, p.status, 36);
                     if (ok) ok = mbar_wait(bar_bf_full(s), round & 1, abort_flag, p.status, 32);
                     if (!ok) break;
                     tc_fence_after();
@@ -1188,7 +1193,12 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
                     first = false;
                 }
                 if (++kb == num_kb || it == n_it - 1) {  // the segment ends with its slab or with this CTA's range
-                    tc_commit_cta(bar_acc_full(buf));    // (an issuer without a k-block in the segment arrives at once)
+                    // An issuer without a k-block in the segment only arrives.  With one buffer that arrival must not fall
+                    // into the barrier's previous phase (the other issuers' commits of the last segment may still be on
+                    // their way): it waits until the epilogue has read the last segment, as a first MMA would have.
+                    if (first && bufs == 1 && use >= 1) ok = mbar_wait(bar_acc_empty(buf), (use - 1) & 1, abort_flag, p.status, 36);
+                    if (!ok) break;
+                    tc_commit_cta(bar_acc_full(buf));
                     kb = 0; seg++; first = true;
                 }
             }
@@ -1267,10 +1277,10 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
         const int sa = p.d_sa ? *p.d_sa : 0;
         long long lin = lin0;
         for (int seg = 0; lin < lin1; seg++) {
-            const int j = (int)(lin / num_kb), kb_a = (int)(lin % num_kb), buf = seg & 1;
+            const int j = (int)(lin / num_kb), kb_a = (int)(lin % num_kb), buf = bufs == 2 ? seg & 1 : 0, use = bufs == 2 ? seg >> 1 : seg;
             const long long slab_end = (long long)(j + 1) * num_kb, seg_end = slab_end < lin1 ? slab_end : lin1;
             const bool whole = kb_a == 0 && seg_end == slab_end;
-            if (!mbar_wait(bar_acc_full(buf), (seg >> 1) & 1, abort_flag, p.status, 35)) break;
+            if (!mbar_wait(bar_acc_full(buf), use & 1, abort_flag, p.status, 35)) break;
             tc_fence_after();
             const int n = j * BM + warp * 32 + lane;
             const int sw = p.d_sw_channel ? (n < p.N ? p.d_sw_channel[n] : 0) : (p.d_sw ? *p.d_sw : 0);
