@@ -194,7 +194,7 @@ def test_gemm_narrow_products(shape, c_dtype, w_is_nk, staged):
     # staged: with a workspace for partial sums the (slab, two-k-block unit) pairs are dealt out in equal contiguous ranges, so
     # slabs are cut (16, ~3 and 4 contributors per slab) and summed from per-contributor slices.  The last two shapes have 19
     # units per slab against ranges of 4.04 units: range and slab boundaries never line up, segments come as short as one
-    # unit (fewer k-blocks than MMA-issuing threads: four for M <= 32, two above), and K = 2368 ends in half a unit.
+    # unit (fewer k-blocks than MMA-issuing threads: four, or two for more than 32 rows against [K,N] weights), and K = 2368 ends in half a unit.
     M, N, K = shape
     N16 = (N + 15) // 16 * 16
     Aq = W.random_codes((M, K), seed=M + K)
