@@ -153,6 +153,20 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
 
+// the same with an L2 eviction policy for the lines the copy brings in
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar, uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "l"(policy) : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -1124,6 +1138,7 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
         if (lane == 0) {
             int issued = 0, issued_act = 0;
             bool aborted = false;
+            const uint64_t w_policy = l2_policy_evict_first();
             int j = (int)(pair0 / num_pb), pb = (int)(pair0 % num_pb);
             for (int it = 0; it < n_pairs; it++) {
                 const int s = it % S8, round = it / S8;
@@ -1131,8 +1146,10 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
                 if (*abort_flag) break;
                 const uint32_t dst_w = lay.u8(s), dst_a = dst_w + kU8Act;
                 mbar_arrive_expect_tx(bar_u8_full(s), 2 * kNwW8 + (ACT_BF16 ? 0u : act_bytes));
-                if (W_IS_NK) tma_load_2d(dst_w, &map_w, pb * BK2, j * BM, bar_u8_full(s));
-                else tma_load_2d(dst_w, &map_w, j * BM, pb * BK2, bar_u8_full(s));
+                // (the weight is read once: its lines are the first to leave L2 again, so that the expanded activations, which
+                // every CTA reads, and the slices of the slabs that two CTAs share stay there)
+                if (W_IS_NK) tma_load_2d_hint(dst_w, &map_w, pb * BK2, j * BM, bar_u8_full(s), w_policy);
+                else tma_load_2d_hint(dst_w, &map_w, j * BM, pb * BK2, bar_u8_full(s), w_policy);
                 if (!ACT_BF16) tma_load_2d(dst_a, &map_act, pb * BK2, 0, bar_u8_full(s));
                 issued = it + 1;
                 if (ACT_BF16) {
