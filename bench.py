@@ -449,6 +449,7 @@ def extra_results(H, torch, hbm_peak, tf_peak, peak_kind, tf_sustained=None):
         d["frac_of_hbm"] = d["frac"]
         narrow[f"M={Mn}"] = d
         row(f"gemm_narrow_{Mn}x28672x8192", d, "hbm (weight bytes)")
+        row(f"gemm_narrow_{Mn}x28672x8192_weights_as_[N,K]", hbm(st_nk, byt), "hbm (weight bytes)")
         del Cn
     # prefill-sized products against the same weight, with the full workspace: below about 1600 rows the call expands A alone
     mid = {}
