@@ -1364,6 +1364,18 @@ hif8_gemm_narrow_kernel(const __grid_constant__ CUtensorMap map_act, const __gri
                         // sixteen rows at a time: their loads are independent, so the L2 latency is paid once per slice
                         for (int m0 = 0; m0 < p.M; m0 += 16) {
                             float acc[16];
+                            if (count == 2) {
+                                // two contributors (the usual case): both slices' loads in flight together, same order of addition
+                                float v0[16], v1[16];
+#pragma unroll
+                                for (int u = 0; u < 16; u++) v0[u] = __ldcg(slab_part + (size_t)m0 * BM + u * BM);
+#pragma unroll
+                                for (int u = 0; u < 16; u++) v1[u] = __ldcg(slab_part + ((size_t)mp + m0) * BM + u * BM);
+#pragma unroll
+                                for (int u = 0; u < 16; u++)
+                                    if (m0 + u < p.M) finish(m0 + u, (0.f + v0[u]) + v1[u]);
+                                continue;
+                            }
 #pragma unroll
                             for (int u = 0; u < 16; u++) acc[u] = 0.f;
                             for (int i = 0; i < count; i++) {
